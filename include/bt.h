@@ -1,0 +1,278 @@
+/*
+ * bt -- FP32 GPT-2 training step for NVIDIA B200 (sm_100a), C ABI.
+ *
+ * The library runs the forward pass, the backward pass and the AdamW update of a
+ * decoder-only pre-LayerNorm transformer with tied embeddings (the paper's evaluation
+ * model: architecture-figure caption and hyper-parameter table of Section 5; step
+ * structure of Algorithm 1: forward, cross-entropy against the target, backward,
+ * optimizer step).  Every step of the path runs in hand-written CUDA kernels; there is
+ * no CPU fallback.
+ *
+ * Conventions that hold for every entry point
+ * -------------------------------------------
+ * Memory    All array arguments are DEVICE pointers unless the name starts with `h_`
+ *           (host).  The caller owns every buffer, including the model workspace and
+ *           any `scratch` argument; the library allocates no device memory.  Device
+ *           pointers must be 16-byte aligned.  Arrays are row-major FP32 unless
+ *           declared int32.
+ * Streams   `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *           stream).  Calls enqueue work and return; only calls with a non-NULL host
+ *           output pointer (h_loss, h_grad_norm) synchronise the stream.
+ * Errors    Every call returns a bt_status.  Arguments are validated on the host
+ *           before any launch; nothing is thrown or aborted.  bt_last_error() returns
+ *           a thread-local description of the last failure.  Kernels that wait on
+ *           hardware barriers bound every wait; a wait that runs out sets a device
+ *           error word that the next synchronising call reports as
+ *           BT_ERR_DEVICE_TIMEOUT.
+ * Split     The tensor-core GEMMs compute FP32 products as three TF32 products
+ *           (a_hi*b_hi + a_hi*b_lo + a_lo*b_hi, FP32 accumulate).  Operands are therefore
+ *           stored as two FP32 planes, `hi` = the value with its low 13 mantissa bits
+ *           cleared and `lo` = value - hi (exact).  A "split" array of R x C values is
+ *           [2][R][C]: plane 0 = hi, plane 1 = lo.  Kernels that produce GEMM operands
+ *           can write the split form directly.
+ * Tokens    Token and target ids must lie in [0, vocab_size); this is not checked on
+ *           the device.
+ */
+#ifndef BT_H_
+#define BT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#if defined(__GNUC__)
+#define BT_API __attribute__((visibility("default")))
+#else
+#define BT_API
+#endif
+
+typedef struct bt_model bt_model; /* opaque host object */
+
+typedef enum {
+    BT_OK = 0,
+    BT_ERR_INVALID_ARG = 1,    /* null / misaligned pointer, bad size, bad configuration */
+    BT_ERR_UNSUPPORTED = 2,    /* valid request the compiled kernels do not cover */
+    BT_ERR_OOM = 3,            /* workspace or scratch too small */
+    BT_ERR_CUDA = 4,           /* a CUDA runtime / driver call failed */
+    BT_ERR_DEVICE_TIMEOUT = 5, /* a bounded device-side wait ran out */
+    BT_ERR_NOT_FOUND = 6       /* unknown tensor / activation name */
+} bt_status;
+
+/* Model configuration ("layers / d_model / heads / seq_len / vocab").  The MLP width is
+ * 4 * d_model.  padded_vocab_size >= vocab_size is the number of rows of the tied
+ * embedding / LM-head matrix; the softmax and the loss run over all padded columns. */
+typedef struct {
+    int32_t n_layers, d_model, n_heads, seq_len, vocab_size, padded_vocab_size, max_batch;
+    uint32_t flags;
+} bt_config;
+
+enum {
+    BT_FLAG_GELU_TANH = 1u,  /* tanh-form GELU instead of the exact erf form */
+    BT_FLAG_GEMM_SIMT = 2u,  /* plain FP32 FMA GEMM (bring-up reference) instead of tcgen05 */
+    BT_FLAG_ATTN_SIMT = 4u   /* plain FP32 FMA attention (bring-up reference) */
+};
+
+/* AdamW hyper-parameters (hyper-parameter table, "Optimization" column).  grad_clip <= 0
+ * disables global-norm clipping. */
+typedef struct {
+    float lr, beta1, beta2, eps, weight_decay, grad_clip;
+} bt_adamw_config;
+
+/* ----------------------------------------------------------------------------------
+ * Model lifetime
+ * -------------------------------------------------------------------------------- */
+
+/* Bytes of device workspace a model of this configuration needs (parameters, gradients,
+ * both moments, split weight copies, activations for max_batch sequences, scratch).
+ * Returns 0 for an invalid configuration. */
+BT_API size_t bt_workspace_bytes(const bt_config* cfg);
+
+/* Builds the host-side model over a caller-allocated device workspace of at least
+ * bt_workspace_bytes(cfg) bytes, 256-byte aligned.  Moments and the step counter start
+ * at zero; parameters are NOT initialised (load them through bt_tensor_ptr, or call
+ * bt_model_init).  All later calls on the model enqueue on `stream`.
+ * Errors: BT_ERR_INVALID_ARG (bad cfg: d_model % n_heads, d_model % 32, head_dim not in
+ * {16,32,64,128}, padded_vocab % 32, seq_len or max_batch < 1, ...), BT_ERR_OOM. */
+BT_API bt_status bt_model_create(const bt_config* cfg, void* d_workspace, size_t workspace_bytes,
+                                 void* stream, bt_model** out);
+
+/* Frees the host object only; the workspace stays with the caller. */
+BT_API void bt_model_destroy(bt_model* m);
+
+/* Fills the parameters on the device with the paper's initialisation (hyper-parameter
+ * table: weight std 0.02, residual projections 0.02/sqrt(2*n_layers); biases 0, LayerNorm
+ * gain 1 / shift 0) from a counter-based generator, and zeroes moments and step counter.
+ * Meant for benchmarks; parity tests load explicit arrays instead. */
+BT_API bt_status bt_model_init(bt_model* m, uint64_t seed);
+
+/* Parameter registry.  Order: wte [Vp,C], wpe [T,C], then per block l: h{l}.ln1.g, h{l}.ln1.b,
+ * h{l}.attn.qkv.w [3C,C], h{l}.attn.qkv.b, h{l}.attn.proj.w [C,C], h{l}.attn.proj.b, h{l}.ln2.g,
+ * h{l}.ln2.b, h{l}.mlp.fc.w [4C,C], h{l}.mlp.fc.b, h{l}.mlp.proj.w [C,4C], h{l}.mlp.proj.b, then
+ * lnf.g, lnf.b.  Weights are [out,in] row-major.  `decay` is 1 for the two-dimensional
+ * tensors (weight decay applies), 0 otherwise.  The LM head is wte (tied). */
+BT_API int32_t bt_num_tensors(const bt_model* m);
+BT_API bt_status bt_tensor_info(const bt_model* m, int32_t index, const char** name, int64_t* numel,
+                                int32_t* decay);
+/* kind: 0 parameter, 1 gradient, 2 first moment, 3 second moment.  The pointer addresses
+ * `numel` floats inside the workspace and stays valid for the model's lifetime. */
+BT_API bt_status bt_tensor_ptr(bt_model* m, const char* name, int32_t kind, float** d_ptr);
+
+/* Activations of the last forward/backward, for tests: per-layer "x", "qkv", "x1", "h",
+ * "ln1.mean", "ln1.rstd", "ln2.mean", "ln2.rstd", "lse"; split per-layer "a", "o", "m", "g"
+ * (pointer to the hi plane; lo plane follows at +numel); global "xL", "logits", "losses",
+ * split "xf", "dlogits".  `numel` (nullable) receives the element count of one plane for
+ * the current batch. */
+BT_API bt_status bt_activation_ptr(bt_model* m, const char* name, int32_t layer, float** d_ptr,
+                                   int64_t* numel);
+
+/* Optimizer step counter t (number of AdamW updates applied so far). */
+BT_API int64_t bt_get_step(const bt_model* m);
+BT_API bt_status bt_set_step(bt_model* m, int64_t t);
+
+/* ----------------------------------------------------------------------------------
+ * The training step (Algorithm 1, loop body: forward + loss, backward, optimizer step)
+ * -------------------------------------------------------------------------------- */
+
+/* Forward pass and mean cross-entropy of B sequences: d_tokens, d_targets are int32
+ * [B, seq_len].  If h_loss is non-NULL the stream is synchronised and the loss written. */
+BT_API bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int32_t* d_targets, int32_t B,
+                            float* h_loss);
+
+/* Gradient of the last bt_forward's loss with respect to every parameter (overwrites the
+ * gradient tensors). */
+BT_API bt_status bt_backward(bt_model* m);
+
+/* Global-norm clip (scale = min(1, clip / (norm + 1e-6))) followed by one AdamW update of
+ * every tensor in a single launch: p <- p (1 - lr wd [decay]); m, v moment updates on the
+ * clipped gradient; p <- p - lr mhat / (sqrt(vhat) + eps), t incremented first (t = 1 on
+ * the first call).  h_grad_norm (nullable) receives the unclipped norm (synchronises). */
+BT_API bt_status bt_adamw_step(bt_model* m, const bt_adamw_config* opt, float* h_grad_norm);
+
+/* bt_forward + bt_backward + bt_adamw_step. */
+BT_API bt_status bt_train_step(bt_model* m, const int32_t* d_tokens, const int32_t* d_targets, int32_t B,
+                               const bt_adamw_config* opt, float* h_loss);
+
+/* Same step with HOST token / target buffers (int32 [B, seq_len], pinned for a truly
+ * asynchronous copy): the ids are copied into the workspace on the model's stream first. */
+BT_API bt_status bt_train_step_host(bt_model* m, const int32_t* h_tokens, const int32_t* h_targets,
+                                    int32_t B, const bt_adamw_config* opt, float* h_loss);
+
+/* Synchronises and reads the loss of the last forward. */
+BT_API bt_status bt_get_loss(bt_model* m, float* h_loss);
+
+/* Number of kernels the library has launched on behalf of this model since creation. */
+BT_API int64_t bt_launch_count(const bt_model* m);
+
+BT_API const char* bt_last_error(void);
+
+/* Optional per-kernel timing of the step (the paper's profiler module reports exact
+ * kernel-level timings).  While enabled, every launch group of bt_forward / bt_backward /
+ * bt_adamw_step is bracketed by two CUDA events on the model's stream and tagged with a
+ * category and its algorithmic FLOPs and bytes.  bt_profile_enable synchronises and clears the
+ * records; bt_profile_read synchronises and returns, for one category, the summed event time
+ * in milliseconds, the number of launch groups, and their summed algorithmic FLOPs and bytes
+ * (any output may be NULL).  Events are host objects; no device memory is allocated. */
+BT_API bt_status bt_profile_enable(bt_model* m, int32_t on);
+BT_API int32_t bt_profile_num_categories(void);
+BT_API const char* bt_profile_category_name(int32_t category);
+BT_API bt_status bt_profile_read(bt_model* m, int32_t category, double* ms_total, int64_t* launches, double* flops,
+                                 double* bytes);
+
+/* ----------------------------------------------------------------------------------
+ * Per-operation entry points (the kernels of the step, one at a time, for tests and
+ * micro-benchmarks).  Optional outputs may be NULL.  `*_split` outputs are [2][rows][cols].
+ * -------------------------------------------------------------------------------- */
+
+/* x[n,:] = wte[tok[n],:] + wpe[n mod T,:], one IEEE single-precision add per element
+ * (architecture caption: token + learned position embedding). */
+BT_API bt_status bt_op_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N,
+                                     int32_t T, int32_t C, float* x, void* stream);
+
+/* dwte[tok[n],:] += dx[n,:] summed in ascending n (deterministic); dwpe[t,:] = sum_b dx[b*T+t,:].
+ * dwte is accumulated into (the tied LM-head gradient is already there), dwpe overwritten. */
+BT_API bt_status bt_op_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int32_t T, int32_t C,
+                                     float* dwte, float* dwpe, void* stream);
+
+/* y = gamma * (x - mean) * rstd + beta over the C features of each of N rows; biased
+ * variance, eps = 1e-5.  C % 4 == 0. */
+BT_API bt_status bt_op_layernorm_fwd(const float* x, const float* gamma, const float* beta, int64_t N,
+                                     int32_t C, float* y, float* y_split, float* mean, float* rstd,
+                                     void* stream);
+
+/* dx = rstd * (dxhat - mean_c dxhat - xhat * mean_c(dxhat * xhat)) [+ dres], dxhat = dy * gamma;
+ * dgamma = sum_n dy * xhat, dbeta = sum_n dy (overwritten, fixed summation order). */
+BT_API size_t bt_op_layernorm_bwd_scratch_bytes(int64_t N, int32_t C);
+BT_API bt_status bt_op_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
+                                     const float* rstd, const float* dres, int64_t N, int32_t C, float* dx,
+                                     float* dx_split, float* dgamma, float* dbeta, void* scratch,
+                                     size_t scratch_bytes, void* stream);
+
+/* Dense FP32 GEMM with 3xTF32 split accumulation on the tensor cores (the paper's GEMM
+ * library serves QKV, attention-output and MLP projections in all forward and backward
+ * layouts):  D[M,N] = op(A) op(B) (+ bias[N]) (+ residual[M,N]).
+ *   BT_GEMM_NT: A [M,K], B [N,K]   (forward:  Y  = X W^T)
+ *   BT_GEMM_NN: A [M,K], B [K,N]   (backward: dX = dY W)
+ *   BT_GEMM_TN: A [K,M], B [K,N]   (backward: dW = dY^T X)
+ * M, N, K multiples of 4 (NN/TN: the contiguous extents multiples of 32).  A and B are
+ * raw FP32; they are split into hi/lo planes in `scratch` first.  flags: BT_FLAG_GEMM_SIMT
+ * selects the FP32 FMA reference kernel. */
+enum { BT_GEMM_NT = 0, BT_GEMM_NN = 1, BT_GEMM_TN = 2 };
+BT_API size_t bt_op_gemm_scratch_bytes(int32_t layout, int64_t M, int64_t N, int64_t K);
+BT_API bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A, const float* B,
+                            float* D, const float* bias, const float* residual, void* scratch,
+                            size_t scratch_bytes, uint32_t flags, void* stream);
+
+/* Causal multi-head self-attention over fused qkv [B*T, 3C] (columns q | k | v, head h at
+ * columns h*d..(h+1)*d-1 of each part): o = softmax(q k^T / sqrt(d) + causal mask) v,
+ * lse [B,H,T] = log of the softmax normaliser.  d = C/H in {16, 32, 64, 128}. */
+BT_API bt_status bt_op_attention_fwd(const float* qkv, int32_t B, int32_t T, int32_t C, int32_t H, float* o,
+                                     float* o_split, float* lse, uint32_t flags, void* stream);
+
+/* Backward of the above with recomputed probabilities: dV = P^T do, dP = do V^T,
+ * dS = P o (dP - rowsum(do o o)), dq = dS k / sqrt(d), dk = dS^T q / sqrt(d).
+ * scratch: B*H*T floats. */
+BT_API bt_status bt_op_attention_bwd(const float* qkv, const float* o, const float* lse, const float* d_o,
+                                     int32_t B, int32_t T, int32_t C, int32_t H, float* dqkv,
+                                     float* dqkv_split, void* scratch, size_t scratch_bytes, uint32_t flags,
+                                     void* stream);
+
+/* y = GELU(x) (exact erf form, or tanh form), n % 4 == 0. */
+BT_API bt_status bt_op_gelu_fwd(const float* x, int64_t n, int32_t tanh_form, float* y, float* y_split,
+                                void* stream);
+/* dx = dy * GELU'(x). */
+BT_API bt_status bt_op_gelu_bwd(const float* x, const float* dy, int64_t n, int32_t tanh_form, float* dx,
+                                float* dx_split, void* stream);
+
+/* Fused softmax cross-entropy over all Vp columns: losses[n] = logsumexp(logits[n,:]) -
+ * logits[n, y_n]; dlogits = (softmax - onehot) * inv_count; loss_mean (1 float) =
+ * inv_count * sum_n losses[n] in fixed order.  Vp % 4 == 0. */
+BT_API bt_status bt_op_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int32_t Vp,
+                                    float inv_count, float* losses, float* loss_mean, float* dlogits,
+                                    float* dlogits_split, void* stream);
+
+/* out[c] = sum_n x[n,c] (bias gradients), fixed summation order. */
+BT_API size_t bt_op_colsum_scratch_bytes(int64_t N, int32_t C);
+BT_API bt_status bt_op_colsum(const float* x, int64_t N, int32_t C, float* out, void* scratch,
+                              size_t scratch_bytes, void* stream);
+
+/* out[0] = sqrt(sum g^2), out[1] = clip > 0 ? min(1, clip / (out[0] + 1e-6)) : 1. */
+BT_API size_t bt_op_grad_norm_scratch_bytes(int64_t n);
+BT_API bt_status bt_op_grad_norm(const float* g, int64_t n, float clip, float* out2, void* scratch,
+                                 size_t scratch_bytes, void* stream);
+
+/* One AdamW update at step t >= 1 of n_tensors tensors in one launch (the paper's
+ * horizontally fused multi-tensor optimizer).  h_p/h_g/h_m/h_v are HOST arrays of device
+ * pointers, h_numel/h_decay host arrays; d_scale (nullable) is a device float multiplying
+ * every gradient (the clip factor).  n_tensors <= 64 per call. */
+BT_API bt_status bt_op_adamw_multi(int32_t n_tensors, float* const* h_p, const float* const* h_g,
+                                   float* const* h_m, float* const* h_v, const int64_t* h_numel,
+                                   const int32_t* h_decay, const bt_adamw_config* opt, int64_t t,
+                                   const float* d_scale, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BT_H_ */

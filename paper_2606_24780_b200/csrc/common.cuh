@@ -1,0 +1,145 @@
+// Shared device helpers and the internal launcher interface of the bt library.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+
+namespace bt {
+
+// Every launcher bumps this counter once per kernel launch (read by bt_launch_count).
+extern std::atomic<long long> g_launches;
+#define BT_COUNT_LAUNCH() (::bt::g_launches.fetch_add(1, std::memory_order_relaxed))
+
+constexpr float kLnEps = 1e-5f;
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+__device__ __forceinline__ float warp_max(float v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ double warp_sum_d(double v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// TF32 split: hi keeps sign, exponent and the top 10 mantissa bits, lo = x - hi is exact
+// in FP32.  x = hi + lo always holds bit for bit.
+__device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
+    hi = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+    lo = x - hi;
+}
+__device__ __forceinline__ void split_tf32(const float4& x, float4& hi, float4& lo) {
+    split_tf32(x.x, hi.x, lo.x);
+    split_tf32(x.y, hi.y, lo.y);
+    split_tf32(x.z, hi.z, lo.z);
+    split_tf32(x.w, hi.w, lo.w);
+}
+
+// Writes v to the raw array and/or to the hi/lo planes at float4 index i.
+__device__ __forceinline__ void store_raw_split(float4 v, float* raw, float* hi, float* lo, int64_t i4) {
+    if (raw) reinterpret_cast<float4*>(raw)[i4] = v;
+    if (hi) {
+        float4 h, l;
+        split_tf32(v, h, l);
+        reinterpret_cast<float4*>(hi)[i4] = h;
+        reinterpret_cast<float4*>(lo)[i4] = l;
+    }
+}
+
+__device__ __forceinline__ float4 ld4(const float* p, int64_t i4) {
+    return reinterpret_cast<const float4*>(p)[i4];
+}
+__device__ __forceinline__ float4 add4(float4 a, float4 b) {
+    return make_float4(a.x + b.x, a.y + b.y, a.z + b.z, a.w + b.w);
+}
+
+// A GEMM operand stored as two FP32 planes (hi at `hi`, lo at `hi + plane`), row-major
+// with `ld` floats between rows.
+struct SplitMat {
+    const float* hi;
+    int64_t plane;
+    int64_t rows, cols, ld;
+};
+
+enum GemmLayout { kNT = 0, kNN = 1, kTN = 2 };
+
+struct AdamParams {
+    float lr, beta1, beta2, eps, weight_decay;
+    float inv_c1, inv_c2;  // 1 / (1 - beta^t), computed on the host in double
+};
+
+// ---------------------------------------------------------------- launchers (host)
+// All return cudaGetLastError() of their launches.
+
+cudaError_t launch_split(const float* x, float* hi, float* lo, int64_t n, cudaStream_t s);
+cudaError_t launch_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int T,
+                                 int C, float* x, cudaStream_t s);
+cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, float* dwte,
+                                 float* dwpe, cudaStream_t s);
+cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float* beta, int64_t N, int C,
+                                 float* y, float* y_hi, float* y_lo, float* mean, float* rstd, cudaStream_t s);
+size_t layernorm_bwd_scratch_floats(int64_t N, int C);
+cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
+                                 const float* rstd, const float* dres, int64_t N, int C, float* dx, float* dx_hi,
+                                 float* dx_lo, float* dgamma, float* dbeta, float* scratch, cudaStream_t s);
+cudaError_t launch_gelu_fwd(const float* x, int64_t n, int tanh_form, float* y, float* y_hi, float* y_lo,
+                            cudaStream_t s);
+cudaError_t launch_gelu_bwd(const float* x, const float* dy, int64_t n, int tanh_form, float* dx, float* dx_hi,
+                            float* dx_lo, cudaStream_t s);
+cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int Vp, float inv_count,
+                                float* losses, float* loss_mean, float* dl, float* dl_hi, float* dl_lo,
+                                cudaStream_t s);
+size_t colsum_scratch_floats(int64_t N, int C);
+// x_lo (nullable): second plane added to the first (sums a split array).
+cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, float* out, float* scratch,
+                          cudaStream_t s);
+size_t grad_norm_scratch_bytes(int64_t n);
+cudaError_t launch_grad_norm(const float* g, int64_t n, float clip, float* out2, void* scratch, cudaStream_t s);
+// Flat-arena AdamW: n floats (multiple of 1024), decay_flags[n / 1024].
+cudaError_t launch_adamw_flat(float* p, const float* g, float* m, float* v, int64_t n, const uint8_t* decay_flags,
+                              AdamParams hp, const float* d_scale, cudaStream_t s);
+struct AdamTensorList {
+    enum { kMax = 64 };
+    float* p[kMax];
+    const float* g[kMax];
+    float* m[kMax];
+    float* v[kMax];
+    long long numel[kMax];
+    int decay[kMax];
+    int chunk_begin[kMax + 1];
+    int n;
+};
+cudaError_t launch_adamw_multi(const AdamTensorList& tl, AdamParams hp, const float* d_scale, cudaStream_t s);
+cudaError_t launch_splitk_reduce(const float* partials, int splits, int64_t n, float* out, cudaStream_t s);
+cudaError_t launch_init_normal(float* p, int64_t n, float std, uint64_t seed, uint64_t offset, cudaStream_t s);
+cudaError_t launch_fill(float* p, int64_t n, float v, cudaStream_t s);
+
+// SIMT reference GEMM: D = op(A) op(B) (+bias) (+residual), operands given as split planes
+// (lo may be absent: plane == 0 means "hi only").
+cudaError_t launch_gemm_simt(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
+                             int64_t ldd, const float* bias, const float* residual, cudaStream_t s);
+
+// tcgen05 GEMM.  `partials` (nullable) receives split-K partial sums; max_partial_floats its size.
+// err_word: device int set non-zero when a bounded wait ran out.
+cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
+                           int64_t ldd, const float* bias, const float* residual, float* partials,
+                           size_t max_partial_floats, int* err_word, cudaStream_t s);
+size_t gemm_tc_partial_floats_bound();
+bool gemm_tc_init(char* err, size_t errlen);  // resolves the tensor-map encoder
+
+// Attention.  lo planes are written when the hi pointer is non-null.
+cudaError_t launch_attention_fwd(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi, float* o_lo,
+                                 float* lse, bool simt, cudaStream_t s);
+// o given raw (o_lo == nullptr) or as hi/lo planes.  dvec: B*H*T floats of scratch.
+cudaError_t launch_attention_bwd(const float* qkv, const float* o, const float* o_lo, const float* lse,
+                                 const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
+                                 float* dqkv_lo, float* dvec, bool simt, cudaStream_t s);
+
+}  // namespace bt

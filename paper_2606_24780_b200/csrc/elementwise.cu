@@ -1,0 +1,450 @@
+// Memory-bound kernels of the training step: TF32 split, embedding gather and its
+// deterministic scatter-add backward, GELU, column sums (bias gradients), gradient norm,
+// multi-tensor AdamW, split-K reduction, parameter initialisation.
+//
+// All of them stream their operands once with 128-bit accesses; reductions use warp
+// shuffles and fixed summation orders (no floating-point atomics anywhere).
+#include "common.cuh"
+
+namespace bt {
+
+std::atomic<long long> g_launches{0};
+
+static inline int grid_for(int64_t work, int block, int cap) {
+    int64_t g = (work + block - 1) / block;
+    if (g < 1) g = 1;
+    if (g > cap) g = cap;
+    return (int)g;
+}
+// Grid-stride kernels: enough CTAs to fill 148 SMs several times over.
+constexpr int kStreamGridCap = 148 * 16;
+
+// ------------------------------------------------------------------ split
+
+__global__ void __launch_bounds__(256) split_kernel(const float* __restrict__ x, float* __restrict__ hi,
+                                                    float* __restrict__ lo, int64_t n4) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        float4 v = ld4(x, i), h, l;
+        split_tf32(v, h, l);
+        reinterpret_cast<float4*>(hi)[i] = h;
+        reinterpret_cast<float4*>(lo)[i] = l;
+    }
+}
+
+cudaError_t launch_split(const float* x, float* hi, float* lo, int64_t n, cudaStream_t s) {
+    int64_t n4 = n / 4;
+    split_kernel<<<grid_for(n4, 256, kStreamGridCap), 256, 0, s>>>(x, hi, lo, n4);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ embedding forward
+
+// One thread per float4 of the output: x[n,:] = wte[tok[n],:] + wpe[n mod T,:].
+__global__ void __launch_bounds__(256) embedding_fwd_kernel(const int32_t* __restrict__ tok,
+                                                            const float* __restrict__ wte,
+                                                            const float* __restrict__ wpe, int64_t N, int T, int C4,
+                                                            float* __restrict__ x) {
+    int64_t total = N * C4;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        int64_t n = i / C4;
+        int c = (int)(i - n * C4);
+        float4 e = ld4(wte, (int64_t)tok[n] * C4 + c);
+        float4 p = ld4(wpe, (n % T) * C4 + c);
+        float4 r;
+        r.x = __fadd_rn(e.x, p.x);
+        r.y = __fadd_rn(e.y, p.y);
+        r.z = __fadd_rn(e.z, p.z);
+        r.w = __fadd_rn(e.w, p.w);
+        reinterpret_cast<float4*>(x)[i] = r;
+    }
+}
+
+cudaError_t launch_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int T, int C,
+                                 float* x, cudaStream_t s) {
+    embedding_fwd_kernel<<<grid_for(N * (C / 4), 256, kStreamGridCap), 256, 0, s>>>(tok, wte, wpe, N, T, C / 4, x);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ embedding backward
+
+// One CTA per position n.  The CTA owning the FIRST occurrence of a token id gathers all
+// later positions with that id, in ascending order, and adds the row sum to dwte[id,:]; all
+// other CTAs exit.  One writer per row and a fixed order: deterministic, no atomics, and the
+// heavy-tailed (Zipf) token distribution costs one long row sum instead of contended atomics.
+__global__ void __launch_bounds__(256) embedding_bwd_wte_kernel(const int32_t* __restrict__ tok,
+                                                                const float* __restrict__ dx, int N, int C4,
+                                                                float* __restrict__ dwte) {
+    const int n = blockIdx.x;
+    const int t = tok[n];
+    int found = 0;
+    for (int j = threadIdx.x; j < n; j += blockDim.x) found |= (tok[j] == t);
+    if (__syncthreads_or(found)) return;
+
+    __shared__ int list[256];
+    __shared__ int wcount[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (int c0 = 0; c0 < C4; c0 += 256) {
+        const int c = c0 + threadIdx.x;
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int base = n; base < N; base += 256) {
+            int j = base + threadIdx.x;
+            bool flag = (j < N) && (tok[j] == t);
+            unsigned b = __ballot_sync(0xffffffffu, flag);
+            if (lane == 0) wcount[warp] = __popc(b);
+            __syncthreads();
+            int off = 0, total = 0;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) {
+                if (k < warp) off += wcount[k];
+                total += wcount[k];
+            }
+            if (flag) list[off + __popc(b & ((1u << lane) - 1u))] = j;
+            __syncthreads();
+            if (c < C4) {
+                for (int k = 0; k < total; ++k) acc = add4(acc, ld4(dx, (int64_t)list[k] * C4 + c));
+            }
+            __syncthreads();
+        }
+        if (c < C4) {
+            float4* dst = reinterpret_cast<float4*>(dwte) + (int64_t)t * C4 + c;
+            *dst = add4(*dst, acc);
+        }
+    }
+}
+
+// dwpe[t,:] = sum over sequences b (ascending) of dx[b*T + t,:].
+__global__ void __launch_bounds__(256) embedding_bwd_wpe_kernel(const float* __restrict__ dx, int B, int T, int C4,
+                                                                float* __restrict__ dwpe) {
+    int64_t total = (int64_t)T * C4;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
+         i += (int64_t)gridDim.x * blockDim.x) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int b = 0; b < B; ++b) acc = add4(acc, ld4(dx, (int64_t)b * total + i));
+        reinterpret_cast<float4*>(dwpe)[i] = acc;
+    }
+}
+
+cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, float* dwte,
+                                 float* dwpe, cudaStream_t s) {
+    embedding_bwd_wte_kernel<<<(int)N, 256, 0, s>>>(tok, dx, (int)N, C / 4, dwte);
+    BT_COUNT_LAUNCH();
+    embedding_bwd_wpe_kernel<<<grid_for((int64_t)T * (C / 4), 256, kStreamGridCap), 256, 0, s>>>(
+        dx, (int)(N / T), T, C / 4, dwpe);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ GELU
+
+__device__ __forceinline__ float gelu_f(float x, bool tanh_form) {
+    if (tanh_form) {
+        float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+        return 0.5f * x * (1.0f + tanhf(u));
+    }
+    return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f));
+}
+__device__ __forceinline__ float gelu_grad_f(float x, bool tanh_form) {
+    if (tanh_form) {
+        float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+        float t = tanhf(u);
+        float du = 0.7978845608028654f * (1.0f + 3.0f * 0.044715f * x * x);
+        return 0.5f * (1.0f + t) + 0.5f * x * (1.0f - t * t) * du;
+    }
+    // Phi(x) + x phi(x)
+    return 0.5f * (1.0f + erff(x * 0.7071067811865476f)) + x * 0.3989422804014327f * expf(-0.5f * x * x);
+}
+
+__global__ void __launch_bounds__(256) gelu_fwd_kernel(const float* __restrict__ x, int64_t n4, int tanh_form,
+                                                       float* y, float* y_hi, float* y_lo) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        float4 v = ld4(x, i), r;
+        r.x = gelu_f(v.x, tanh_form);
+        r.y = gelu_f(v.y, tanh_form);
+        r.z = gelu_f(v.z, tanh_form);
+        r.w = gelu_f(v.w, tanh_form);
+        store_raw_split(r, y, y_hi, y_lo, i);
+    }
+}
+
+__global__ void __launch_bounds__(256) gelu_bwd_kernel(const float* __restrict__ x, const float* __restrict__ dy,
+                                                       int64_t n4, int tanh_form, float* dx, float* dx_hi,
+                                                       float* dx_lo) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        float4 v = ld4(x, i), d = ld4(dy, i), r;
+        r.x = d.x * gelu_grad_f(v.x, tanh_form);
+        r.y = d.y * gelu_grad_f(v.y, tanh_form);
+        r.z = d.z * gelu_grad_f(v.z, tanh_form);
+        r.w = d.w * gelu_grad_f(v.w, tanh_form);
+        store_raw_split(r, dx, dx_hi, dx_lo, i);
+    }
+}
+
+cudaError_t launch_gelu_fwd(const float* x, int64_t n, int tanh_form, float* y, float* y_hi, float* y_lo,
+                            cudaStream_t s) {
+    gelu_fwd_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(x, n / 4, tanh_form, y, y_hi, y_lo);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+cudaError_t launch_gelu_bwd(const float* x, const float* dy, int64_t n, int tanh_form, float* dx, float* dx_hi,
+                            float* dx_lo, cudaStream_t s) {
+    gelu_bwd_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(x, dy, n / 4, tanh_form, dx, dx_hi, dx_lo);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ column sums
+
+// Stage 1: CTA (cb, st) sums rows of strip st for the 128 columns of block cb; warp w takes
+// rows w, w+8, ... of the strip, lanes hold one float4 column group; warps are combined in
+// warp order.  Stage 2 adds the strips in strip order.
+static inline int colsum_strips(int64_t N, int C) {
+    int cblocks = (C + 127) / 128;
+    int64_t strips = (2 * 148 + cblocks - 1) / cblocks;
+    int64_t max_strips = (N + 63) / 64;
+    if (strips > max_strips) strips = max_strips;
+    if (strips < 1) strips = 1;
+    return (int)strips;
+}
+size_t colsum_scratch_floats(int64_t N, int C) { return (size_t)colsum_strips(N, C) * C; }
+
+__global__ void __launch_bounds__(256) colsum_stage1_kernel(const float* __restrict__ x,
+                                                            const float* __restrict__ x_lo, int64_t N, int C4,
+                                                            int strips, float* __restrict__ partial) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + lane;
+    const int st = blockIdx.y;
+    const int64_t rows_per = (N + strips - 1) / strips;
+    const int64_t r0 = st * rows_per, r1 = (r0 + rows_per < N) ? r0 + rows_per : N;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < C4) {
+        for (int64_t r = r0 + warp; r < r1; r += 8) {
+            float4 v = ld4(x, r * C4 + c);
+            if (x_lo) v = add4(v, ld4(x_lo, r * C4 + c));
+            acc = add4(acc, v);
+        }
+    }
+    __shared__ float4 sm[8][32];
+    sm[warp][lane] = acc;
+    __syncthreads();
+    if (warp == 0 && c < C4) {
+        float4 t = sm[0][lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) t = add4(t, sm[w][lane]);
+        reinterpret_cast<float4*>(partial)[(int64_t)st * C4 + c] = t;
+    }
+}
+
+__global__ void __launch_bounds__(128) colsum_stage2_kernel(const float* __restrict__ partial, int strips, int C4,
+                                                            float* __restrict__ out) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c >= C4) return;
+    float4 t = ld4(partial, c);
+    for (int s = 1; s < strips; ++s) t = add4(t, ld4(partial, (int64_t)s * C4 + c));
+    reinterpret_cast<float4*>(out)[c] = t;
+}
+
+cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, float* out, float* scratch,
+                          cudaStream_t s) {
+    int C4 = C / 4, strips = colsum_strips(N, C);
+    dim3 grid((C4 + 31) / 32, strips);
+    colsum_stage1_kernel<<<grid, 256, 0, s>>>(x, x_lo, N, C4, strips, scratch);
+    BT_COUNT_LAUNCH();
+    colsum_stage2_kernel<<<(C4 + 127) / 128, 128, 0, s>>>(scratch, strips, C4, out);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ gradient norm
+
+constexpr int kNormBlocks = 148 * 8;
+size_t grad_norm_scratch_bytes(int64_t) { return kNormBlocks * sizeof(double); }
+
+__global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ g, int64_t n4, int64_t n,
+                                                    double* __restrict__ partial) {
+    float acc = 0.f;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        float4 v = ld4(g, i);
+        acc += v.x * v.x + v.y * v.y + v.z * v.z + v.w * v.w;
+    }
+    // scalar tail (n not a multiple of 4)
+    if (blockIdx.x == 0 && threadIdx.x < (n - n4 * 4)) {
+        float v = g[n4 * 4 + threadIdx.x];
+        acc += v * v;
+    }
+    double d = warp_sum_d((double)acc);
+    __shared__ double sm[8];
+    if ((threadIdx.x & 31) == 0) sm[threadIdx.x >> 5] = d;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int w = 0; w < 8; ++w) t += sm[w];
+        partial[blockIdx.x] = t;
+    }
+}
+
+__global__ void __launch_bounds__(256) norm_finalize_kernel(const double* __restrict__ partial, int nb, float clip,
+                                                            float* __restrict__ out2) {
+    __shared__ double sm[256];
+    double t = 0.0;
+    for (int i = threadIdx.x; i < nb; i += 256) t += partial[i];
+    sm[threadIdx.x] = t;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) sm[threadIdx.x] += sm[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        double norm = sqrt(sm[0]);
+        double sc = 1.0;
+        if (clip > 0.f) {
+            sc = (double)clip / (norm + 1e-6);
+            if (sc > 1.0) sc = 1.0;
+        }
+        out2[0] = (float)norm;
+        out2[1] = (float)sc;
+    }
+}
+
+cudaError_t launch_grad_norm(const float* g, int64_t n, float clip, float* out2, void* scratch, cudaStream_t s) {
+    int nb = grid_for(n / 4, 256, kNormBlocks);
+    sumsq_kernel<<<nb, 256, 0, s>>>(g, n / 4, n, (double*)scratch);
+    BT_COUNT_LAUNCH();
+    norm_finalize_kernel<<<1, 256, 0, s>>>((const double*)scratch, nb, clip, out2);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ AdamW
+
+__device__ __forceinline__ void adamw_elem(float& p, float g, float& m, float& v, bool decay, const AdamParams& hp,
+                                           float scale) {
+    g *= scale;
+    float pp = decay ? p * (1.0f - hp.lr * hp.weight_decay) : p;
+    m = hp.beta1 * m + (1.0f - hp.beta1) * g;
+    v = hp.beta2 * v + (1.0f - hp.beta2) * g * g;
+    float mh = m * hp.inv_c1;
+    float vh = v * hp.inv_c2;
+    p = pp - hp.lr * mh / (sqrtf(vh) + hp.eps);
+}
+__device__ __forceinline__ void adamw_vec(float4& p, float4 g, float4& m, float4& v, bool decay,
+                                          const AdamParams& hp, float scale) {
+    adamw_elem(p.x, g.x, m.x, v.x, decay, hp, scale);
+    adamw_elem(p.y, g.y, m.y, v.y, decay, hp, scale);
+    adamw_elem(p.z, g.z, m.z, v.z, decay, hp, scale);
+    adamw_elem(p.w, g.w, m.w, v.w, decay, hp, scale);
+}
+
+// Flat arena: all tensors live back to back (each padded to 1024 floats), so the whole
+// optimizer step is ONE grid-stride pass; decay_flags has one byte per 1024-float chunk.
+__global__ void __launch_bounds__(256) adamw_flat_kernel(float* __restrict__ p, const float* __restrict__ g,
+                                                         float* __restrict__ m, float* __restrict__ v, int64_t n4,
+                                                         const uint8_t* __restrict__ decay_flags, AdamParams hp,
+                                                         const float* __restrict__ d_scale) {
+    const float scale = d_scale ? *d_scale : 1.0f;
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        float4 pv = ld4(p, i), gv = ld4(g, i), mv = ld4(m, i), vv = ld4(v, i);
+        adamw_vec(pv, gv, mv, vv, decay_flags[i >> 8] != 0, hp, scale);
+        reinterpret_cast<float4*>(p)[i] = pv;
+        reinterpret_cast<float4*>(m)[i] = mv;
+        reinterpret_cast<float4*>(v)[i] = vv;
+    }
+}
+
+cudaError_t launch_adamw_flat(float* p, const float* g, float* m, float* v, int64_t n, const uint8_t* decay_flags,
+                              AdamParams hp, const float* d_scale, cudaStream_t s) {
+    adamw_flat_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(p, g, m, v, n / 4, decay_flags, hp,
+                                                                            d_scale);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// Explicit tensor list: CTA b works on one 4096-element chunk of one tensor; the chunk table
+// balances the load across tensors of very different sizes.
+constexpr int kAdamChunk = 4096;
+__global__ void __launch_bounds__(256) adamw_multi_kernel(const __grid_constant__ AdamTensorList tl, AdamParams hp,
+                                                          const float* __restrict__ d_scale) {
+    const float scale = d_scale ? *d_scale : 1.0f;
+    int t = 0;
+    while (t + 1 < tl.n && (int)blockIdx.x >= tl.chunk_begin[t + 1]) ++t;
+    const int64_t start = (int64_t)(blockIdx.x - tl.chunk_begin[t]) * kAdamChunk;
+    const int64_t numel = tl.numel[t];
+    const int64_t end = (start + kAdamChunk < numel) ? start + kAdamChunk : numel;
+    float* p = tl.p[t];
+    const float* g = tl.g[t];
+    float* m = tl.m[t];
+    float* v = tl.v[t];
+    const bool decay = tl.decay[t] != 0;
+    const int64_t vec_end = start + ((end - start) / 4) * 4;
+    for (int64_t i = start + threadIdx.x * 4; i < vec_end; i += 256 * 4) {
+        float4 pv = ld4(p, i / 4), gv = ld4(g, i / 4), mv = ld4(m, i / 4), vv = ld4(v, i / 4);
+        adamw_vec(pv, gv, mv, vv, decay, hp, scale);
+        reinterpret_cast<float4*>(p)[i / 4] = pv;
+        reinterpret_cast<float4*>(m)[i / 4] = mv;
+        reinterpret_cast<float4*>(v)[i / 4] = vv;
+    }
+    for (int64_t i = vec_end + threadIdx.x; i < end; i += 256) adamw_elem(p[i], g[i], m[i], v[i], decay, hp, scale);
+}
+
+cudaError_t launch_adamw_multi(const AdamTensorList& tl, AdamParams hp, const float* d_scale, cudaStream_t s) {
+    int chunks = tl.chunk_begin[tl.n];
+    if (chunks <= 0) return cudaSuccess;
+    adamw_multi_kernel<<<chunks, 256, 0, s>>>(tl, hp, d_scale);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+int adamw_chunk_elems() { return kAdamChunk; }
+
+// ------------------------------------------------------------------ split-K reduction
+
+__global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partials, int splits,
+                                                            int64_t n4, float* __restrict__ out) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        float4 t = ld4(partials, i);
+        for (int s = 1; s < splits; ++s) t = add4(t, ld4(partials, (int64_t)s * n4 + i));
+        reinterpret_cast<float4*>(out)[i] = t;
+    }
+}
+cudaError_t launch_splitk_reduce(const float* partials, int splits, int64_t n, float* out, cudaStream_t s) {
+    splitk_reduce_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(partials, splits, n / 4, out);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ initialisation
+
+// Counter-based normal generator: SplitMix64 of (seed, element index) -> two uniforms ->
+// Box-Muller.  Only the distribution matters (the paper fixes std, not bit values).
+__device__ __forceinline__ uint64_t splitmix64(uint64_t z) {
+    z += 0x9E3779B97F4A7C15ull;
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+__global__ void __launch_bounds__(256) init_normal_kernel(float* __restrict__ p, int64_t n, float std, uint64_t seed,
+                                                          uint64_t offset) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
+        uint64_t r = splitmix64(splitmix64(seed) ^ (offset + (uint64_t)i));
+        float u1 = ((float)(uint32_t)(r >> 40) + 0.5f) * (1.0f / 16777216.0f);
+        float u2 = ((float)(uint32_t)((r >> 8) & 0xFFFFFFu) + 0.5f) * (1.0f / 16777216.0f);
+        p[i] = std * sqrtf(-2.0f * logf(u1)) * cospif(2.0f * u2);
+    }
+}
+__global__ void __launch_bounds__(256) fill_kernel(float* __restrict__ p, int64_t n, float v) {
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
+        p[i] = v;
+}
+cudaError_t launch_init_normal(float* p, int64_t n, float std, uint64_t seed, uint64_t offset, cudaStream_t s) {
+    init_normal_kernel<<<grid_for(n, 256, kStreamGridCap), 256, 0, s>>>(p, n, std, seed, offset);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+cudaError_t launch_fill(float* p, int64_t n, float v, cudaStream_t s) {
+    fill_kernel<<<grid_for(n, 256, kStreamGridCap), 256, 0, s>>>(p, n, v);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+}  // namespace bt

@@ -1,0 +1,478 @@
+// FP32 GEMM on the 5th-generation tensor cores with 3xTF32 split accumulation.
+//
+//   D[M,N] = op(A) op(B) (+ bias) (+ residual),   x*y ~= x_hi*y_hi + x_hi*y_lo + x_lo*y_hi
+//
+// Operands live in HBM as two FP32 planes (hi = top 19 bits, lo = exact remainder); their
+// producers write them that way, so this kernel is a pure TMA -> shared memory -> tcgen05.mma
+// -> TMEM pipeline with no conversion work on the SM:
+//
+//   warp 0 (one lane)  TMA producer: 3-D tiled loads (k, row, plane) of the hi and lo tiles of A
+//                      and B into a ring of shared-memory stages, completion on mbarriers.
+//   warp 1 (one lane)  MMA issuer: per 8-deep k-step three tcgen05.mma.kind::tf32 (lo*hi, hi*lo,
+//                      hi*hi; small terms first) into a 128 x BN FP32 accumulator in TMEM;
+//                      tcgen05.commit releases the stage / publishes the accumulator.
+//   warps 2-5          epilogue: tcgen05.ld the accumulator (one row per thread), add bias and
+//                      residual, store.  Two accumulators alternate so the epilogue of tile i
+//                      overlaps the main loop of tile i+1.
+//
+// The kernel is persistent (one CTA per SM, work units = output tiles x K-splits, tile-row index
+// fastest so concurrently running CTAs share the B tile and keep A resident in L2).
+//
+// Operand layouts.  "K-major" operands (rows of K contiguous: A of NT/NN, B of NT) use the
+// 128-byte swizzle; "MN-major" operands (K rows of M or N contiguous: A of TN, B of NN/TN) use
+// the 128-byte swizzle with 32-byte atoms, the only shared-memory layout the tensor core accepts
+// for transposed 32-bit operands.  No cluster multicast is used anywhere.
+//
+// Every mbarrier wait is bounded: a wait that runs out raises a device error word and the CTA
+// drains and exits, still releasing its TMEM.
+#include <cuda.h>
+
+#include <cstdio>
+#include <mutex>
+
+#include "common.cuh"
+
+namespace bt {
+
+namespace {
+
+constexpr int BM = 128;
+constexpr int BK = 32;            // floats per k-block = one 128-byte swizzle row
+constexpr int kThreads = 192;
+constexpr int kEpiWarps = 4;
+constexpr uint32_t kATileBytes = 2u * BM * BK * 4u;  // hi + lo
+
+template <int BN>
+struct Cfg {
+    static constexpr uint32_t kBTileBytes = 2u * BN * BK * 4u;
+    static constexpr uint32_t kStageBytes = kATileBytes + kBTileBytes;
+    static constexpr int kStages = (BN == 256) ? 2 : 3;
+    static constexpr uint32_t kTmemCols = 2u * BN;  // two accumulators; 256 or 512 (power of two)
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+};
+
+struct GemmArgs {
+    int M, N, K;
+    float* D;
+    long long ldd;
+    const float* bias;
+    const float* residual;
+    int tiles_m, tiles_n, splits, kb_per_split, kb_total;
+    float* partials;
+    int* err;
+};
+
+// ------------------------------------------------------------------ PTX wrappers
+
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok;
+}
+__device__ __forceinline__ unsigned long long globaltimer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait (about one second).  Returns false after raising the error word.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, int code) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = globaltimer_ns();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (globaltimer_ns() - t0 > 1000000000ull) {
+            atomicExch(err, code);
+            return false;
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
+                                            int c2) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
+        ::"r"(dst), "l"((unsigned long long)tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
+        : "memory");
+}
+
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
+                                          uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
+          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
+          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr));
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets
+// (all >> 4), descriptor version 1, swizzle mode in bits 61-63.
+//   K-major, 128B swizzle          : mode 2, SBO = 1024 (8 rows x 128 B), LBO unused.
+//   MN-major, 128B swizzle/32B atom: mode 1, SBO = 512 (4 k-rows x 128 B), LBO = distance between
+//                                    32-element column groups.
+__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t mode) {
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
+    d |= (uint64_t)1 << 46;
+    d |= (uint64_t)mode << 61;
+    return d;
+}
+
+// Bytes between consecutive 32-wide column groups of an MN-major tile: hi rows then lo rows.
+constexpr uint32_t kMnAtomBytes = 2u * BK * 128u;
+
+template <bool MN>
+__device__ __forceinline__ uint64_t operand_desc(uint32_t tile_base, int rows, bool lo_plane, int kstep) {
+    if (MN) {
+        uint32_t addr = tile_base + (lo_plane ? BK * 128u : 0u) + (uint32_t)kstep * 8u * 128u;
+        return make_desc(addr, kMnAtomBytes, 512u, 1u);
+    } else {
+        uint32_t addr = tile_base + (lo_plane ? (uint32_t)rows * 128u : 0u) + (uint32_t)kstep * 32u;
+        return make_desc(addr, 16u, 1024u, 2u);
+    }
+}
+
+template <bool A_MN, bool B_MN, int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
+    using C = Cfg<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t bars = smem_base + C::kStages * C::kStageBytes;  // 8-byte barriers
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (C::kStages + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * C::kStages + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * C::kStages + 2 + a); };
+    const uint32_t tmem_slot = bars + 8u * (2 * C::kStages + 4);
+    volatile uint32_t* tmem_slot_ptr =
+        reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; ++s) {
+            mbar_init(full_bar(s), 1);
+            mbar_init(empty_bar(s), 1);
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), kEpiWarps);
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot),
+                     "r"(C::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+
+    const int units = g.tiles_m * g.tiles_n * g.splits;
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
+                const int tm = u % g.tiles_m, r = u / g.tiles_m, tn = r % g.tiles_n, sp = r / g.tiles_n;
+                const int kb0 = sp * g.kb_per_split;
+                const int kb1 = min(g.kb_total, kb0 + g.kb_per_split);
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = it % C::kStages;
+                    const uint32_t ph = (it / C::kStages) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, g.err, 1)) { ok = false; break; }
+                    const uint32_t a_dst = smem_base + s * C::kStageBytes;
+                    const uint32_t b_dst = a_dst + kATileBytes;
+                    mbar_expect_tx(full_bar(s), C::kStageBytes);
+                    if (A_MN) {
+#pragma unroll
+                        for (int a = 0; a < BM / 32; ++a)
+                            tma_load_3d(a_dst + a * kMnAtomBytes, &tmA, full_bar(s), tm * BM + 32 * a, kb * BK, 0);
+                    } else {
+                        tma_load_3d(a_dst, &tmA, full_bar(s), kb * BK, tm * BM, 0);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int a = 0; a < BN / 32; ++a)
+                            tma_load_3d(b_dst + a * kMnAtomBytes, &tmB, full_bar(s), tn * BN + 32 * a, kb * BK, 0);
+                    } else {
+                        tma_load_3d(b_dst, &tmB, full_bar(s), kb * BK, tn * BN, 0);
+                    }
+                }
+            }
+            if (!ok) {
+                // let loads already in flight land before the CTA's shared memory is released
+                for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((A_MN ? 1u : 0u) << 15) |
+                                   ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) |
+                                   ((uint32_t)(BM >> 4) << 24);
+            uint32_t it = 0, ut = 0;
+            bool ok = true;
+            for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++ut) {
+                const int r = u / g.tiles_m, sp = r / g.tiles_n;
+                const int kb0 = sp * g.kb_per_split;
+                const int kb1 = min(g.kb_total, kb0 + g.kb_per_split);
+                const int acc = ut & 1;
+                const uint32_t aph = (ut >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(acc), aph ^ 1u, g.err, 2)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = it % C::kStages;
+                    const uint32_t ph = (it / C::kStages) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, g.err, 3)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_base = smem_base + s * C::kStageBytes;
+                    const uint32_t b_base = a_base + kATileBytes;
+#pragma unroll
+                    for (int j = 0; j < BK / 8; ++j) {
+                        const uint64_t a_hi = operand_desc<A_MN>(a_base, BM, false, j);
+                        const uint64_t a_lo = operand_desc<A_MN>(a_base, BM, true, j);
+                        const uint64_t b_hi = operand_desc<B_MN>(b_base, BN, false, j);
+                        const uint64_t b_lo = operand_desc<B_MN>(b_base, BN, true, j);
+                        umma_tf32(d_tmem, a_lo, b_hi, idesc, (kb > kb0 || j > 0) ? 1u : 0u);
+                        umma_tf32(d_tmem, a_hi, b_lo, idesc, 1u);
+                        umma_tf32(d_tmem, a_hi, b_hi, idesc, 1u);
+                    }
+                    umma_commit(empty_bar(s));  // stage free once these MMAs have read it
+                }
+                if (ok) umma_commit(tfull_bar(acc));  // accumulator complete
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps
+        const int lane_group = warp & 3;  // TMEM lanes 32*lane_group .. +31 belong to this warp
+        uint32_t ut = 0;
+        bool ok = true;
+        for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++ut) {
+            const int tm = u % g.tiles_m, r = u / g.tiles_m, tn = r % g.tiles_n, sp = r / g.tiles_n;
+            const int acc = ut & 1;
+            const uint32_t aph = (ut >> 1) & 1u;
+            if (!mbar_wait(tfull_bar(acc), aph, g.err, 4)) { ok = false; break; }
+            tc_fence_after();
+            const int row = tm * BM + lane_group * 32 + lane;
+            float* Dp = g.D;
+            long long ldd = g.ldd;
+            if (g.splits > 1) {
+                Dp = g.partials + (long long)sp * g.M * g.N;
+                ldd = g.N;
+            }
+            const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)acc * BN;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int col0 = tn * BN + c * 32;
+                if (col0 >= g.N) break;  // warp-uniform
+                uint32_t rr[32];
+                tmem_ld32(t_row + c * 32, rr);
+                tmem_ld_wait();
+                if (row < g.M) {
+                    float* drow = Dp + (long long)row * ldd + col0;
+                    const float* rrow = g.residual ? g.residual + (long long)row * g.ldd + col0 : nullptr;
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) {
+                        if (col0 + q * 4 < g.N) {
+                            float4 v = make_float4(__uint_as_float(rr[4 * q]), __uint_as_float(rr[4 * q + 1]),
+                                                   __uint_as_float(rr[4 * q + 2]), __uint_as_float(rr[4 * q + 3]));
+                            if (g.bias) v = add4(v, *reinterpret_cast<const float4*>(g.bias + col0 + q * 4));
+                            if (rrow) v = add4(v, *reinterpret_cast<const float4*>(rrow + q * 4));
+                            *reinterpret_cast<float4*>(drow + q * 4) = v;
+                        }
+                    }
+                }
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(acc));
+        }
+    }
+
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols)
+                     : "memory");
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+int g_num_sms = 0;
+std::once_flag g_once;
+char g_init_err[256] = {0};
+
+template <bool A_MN, bool B_MN, int BN>
+cudaError_t set_attr() {
+    return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)Cfg<BN>::kSmemBytes);
+}
+
+void init_once() {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess || q != cudaDriverEntryPointSuccess || !fn) {
+        snprintf(g_init_err, sizeof(g_init_err), "cuTensorMapEncodeTiled not available: %s", cudaGetErrorString(e));
+        return;
+    }
+    g_encode = (EncodeTiledFn)fn;
+    int dev = 0;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
+    cudaError_t a = cudaSuccess;
+#define BT_ATTR(AM, BMN)                                                        \
+    if (a == cudaSuccess) a = set_attr<AM, BMN, 256>();                         \
+    if (a == cudaSuccess) a = set_attr<AM, BMN, 128>()
+    BT_ATTR(false, false);
+    BT_ATTR(false, true);
+    BT_ATTR(true, true);
+#undef BT_ATTR
+    if (a != cudaSuccess) {
+        snprintf(g_init_err, sizeof(g_init_err), "cudaFuncSetAttribute(smem) failed: %s", cudaGetErrorString(a));
+        g_encode = nullptr;
+    }
+}
+
+// 3-D map over a split matrix: (contiguous cols, rows, plane).
+bool encode_map(CUtensorMap* tm, const SplitMat& m, uint32_t box_cols, uint32_t box_rows, bool mn_major) {
+    cuuint64_t dims[3] = {(cuuint64_t)m.cols, (cuuint64_t)m.rows, 2};
+    cuuint64_t strides[2] = {(cuuint64_t)m.ld * 4, (cuuint64_t)m.plane * 4};
+    cuuint32_t box[3] = {box_cols, box_rows, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)m.hi, dims, strides, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE,
+                          mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    return r == CUDA_SUCCESS;
+}
+
+constexpr int kMaxUnitsForSplit = 4 * 148;
+
+}  // namespace
+
+bool gemm_tc_init(char* err, size_t errlen) {
+    std::call_once(g_once, init_once);
+    if (!g_encode && err) snprintf(err, errlen, "%s", g_init_err);
+    return g_encode != nullptr;
+}
+
+size_t gemm_tc_partial_floats_bound() { return (size_t)kMaxUnitsForSplit * BM * 256; }
+
+cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D, int64_t ldd,
+                           const float* bias, const float* residual, float* partials, size_t max_partial_floats,
+                           int* err_word, cudaStream_t s) {
+    if (!gemm_tc_init(nullptr, 0)) return cudaErrorNotSupported;
+    const bool a_mn = (layout == kTN), b_mn = (layout != kNT);
+    const int sms = g_num_sms > 0 ? g_num_sms : 148;
+
+    // Tile width: 256 unless the 128-wide tiling wastes clearly fewer SM-rounds.
+    const int tiles_m = (int)((M + BM - 1) / BM);
+    auto rounds_cost = [&](int bn) {
+        long long tiles = (long long)tiles_m * ((N + bn - 1) / bn);
+        long long rounds = (tiles + sms - 1) / sms;
+        return (double)rounds * bn;  // time ~ rounds x tile width
+    };
+    int bn = 256;
+    if (N <= 128 || rounds_cost(128) < 0.9 * rounds_cost(256)) bn = 128;
+    const int tiles_n = (int)((N + bn - 1) / bn);
+    const int kb_total = (int)((K + BK - 1) / BK);
+
+    // Split K when the tile grid alone cannot fill the machine (the weight-gradient GEMMs:
+    // small outputs, K = number of tokens).
+    int splits = 1;
+    const long long tiles = (long long)tiles_m * tiles_n;
+    if (!bias && !residual && partials && ldd == N && tiles * 2 <= sms && kb_total >= 8) {
+        splits = (int)((2LL * sms + tiles - 1) / tiles);
+        if (splits > kb_total / 4) splits = kb_total / 4;
+        while (splits > 1 && (size_t)splits * M * N > max_partial_floats) --splits;
+        if (splits < 1) splits = 1;
+    }
+    int kb_per_split = (kb_total + splits - 1) / splits;
+    splits = (kb_total + kb_per_split - 1) / kb_per_split;  // no empty split
+
+    CUtensorMap tmA, tmB;
+    bool ok = a_mn ? encode_map(&tmA, A, 32, BK, true) : encode_map(&tmA, A, BK, BM, false);
+    ok = ok && (b_mn ? encode_map(&tmB, B, 32, BK, true) : encode_map(&tmB, B, BK, (uint32_t)bn, false));
+    if (!ok) return cudaErrorInvalidValue;
+
+    GemmArgs g;
+    g.M = (int)M; g.N = (int)N; g.K = (int)K;
+    g.D = D; g.ldd = ldd; g.bias = bias; g.residual = residual;
+    g.tiles_m = tiles_m; g.tiles_n = tiles_n; g.splits = splits;
+    g.kb_per_split = kb_per_split; g.kb_total = kb_total;
+    g.partials = partials; g.err = err_word;
+    const long long units = tiles * splits;
+    const int grid = (int)(units < sms ? units : sms);
+
+#define BT_LAUNCH(AM, BMN, BNV)                                                                              \
+    gemm_tc_kernel<AM, BMN, BNV><<<grid, kThreads, Cfg<BNV>::kSmemBytes, s>>>(tmA, tmB, g)
+    if (bn == 256) {
+        if (layout == kNT) BT_LAUNCH(false, false, 256);
+        else if (layout == kNN) BT_LAUNCH(false, true, 256);
+        else BT_LAUNCH(true, true, 256);
+    } else {
+        if (layout == kNT) BT_LAUNCH(false, false, 128);
+        else if (layout == kNN) BT_LAUNCH(false, true, 128);
+        else BT_LAUNCH(true, true, 128);
+    }
+#undef BT_LAUNCH
+    BT_COUNT_LAUNCH();
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    if (splits > 1) return launch_splitk_reduce(partials, splits, M * N, D, s);
+    return cudaSuccess;
+}
+
+}  // namespace bt

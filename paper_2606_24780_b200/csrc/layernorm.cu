@@ -1,0 +1,198 @@
+// LayerNorm forward and backward.  One warp owns one row: the row is read once into
+// registers with 128-bit loads, both row reductions are warp shuffles (no shared memory on
+// the row path), and the output is written once -- raw and/or as TF32 hi/lo planes for the
+// GEMM that consumes it.  The backward's parameter gradients are accumulated per lane over a
+// strip of rows, combined across the CTA's warps in warp order, written as per-CTA partials
+// and summed by a second kernel in CTA order (deterministic).
+#include "common.cuh"
+
+namespace bt {
+
+constexpr int kLnWarps = 8;
+
+// VPL = float4 values per lane (C <= 128 * VPL).
+template <int VPL>
+__global__ void __launch_bounds__(kLnWarps * 32) ln_fwd_kernel(const float* __restrict__ x,
+                                                               const float* __restrict__ gamma,
+                                                               const float* __restrict__ beta, int64_t N, int C4,
+                                                               float* y, float* y_hi, float* y_lo,
+                                                               float* __restrict__ mean, float* __restrict__ rstd) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t row = (int64_t)blockIdx.x * kLnWarps + warp;
+    if (row >= N) return;
+    const float inv_c = 1.0f / (float)(C4 * 4);
+    float4 v[VPL];
+    float s = 0.f;
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        int idx = lane + 32 * k;
+        if (idx < C4) {
+            v[k] = ld4(x, row * C4 + idx);
+            s += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+        }
+    }
+    const float mu = warp_sum(s) * inv_c;
+    float q = 0.f;
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        int idx = lane + 32 * k;
+        if (idx < C4) {
+            float a = v[k].x - mu, b = v[k].y - mu, c = v[k].z - mu, d = v[k].w - mu;
+            q += (a * a + b * b) + (c * c + d * d);
+        }
+    }
+    const float var = warp_sum(q) * inv_c;
+    const float rs = 1.0f / sqrtf(var + kLnEps);
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        int idx = lane + 32 * k;
+        if (idx < C4) {
+            float4 g = ld4(gamma, idx), b = ld4(beta, idx), r;
+            r.x = g.x * ((v[k].x - mu) * rs) + b.x;
+            r.y = g.y * ((v[k].y - mu) * rs) + b.y;
+            r.z = g.z * ((v[k].z - mu) * rs) + b.z;
+            r.w = g.w * ((v[k].w - mu) * rs) + b.w;
+            store_raw_split(r, y, y_hi, y_lo, row * C4 + idx);
+        }
+    }
+    if (lane == 0) {
+        if (mean) mean[row] = mu;
+        if (rstd) rstd[row] = rs;
+    }
+}
+
+cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float* beta, int64_t N, int C, float* y,
+                                 float* y_hi, float* y_lo, float* mean, float* rstd, cudaStream_t s) {
+    const int C4 = C / 4;
+    const int vpl = (C4 + 31) / 32;
+    const int grid = (int)((N + kLnWarps - 1) / kLnWarps);
+#define BT_LN_FWD(V)                                                                                     \
+    ln_fwd_kernel<V><<<grid, kLnWarps * 32, 0, s>>>(x, gamma, beta, N, C4, y, y_hi, y_lo, mean, rstd)
+    if (vpl <= 1) BT_LN_FWD(1);
+    else if (vpl <= 2) BT_LN_FWD(2);
+    else if (vpl <= 4) BT_LN_FWD(4);
+    else if (vpl <= 6) BT_LN_FWD(6);
+    else if (vpl <= 8) BT_LN_FWD(8);
+    else if (vpl <= 16) BT_LN_FWD(16);
+    else if (vpl <= 32) BT_LN_FWD(32);
+    else return cudaErrorInvalidValue;
+#undef BT_LN_FWD
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// ------------------------------------------------------------------ backward
+
+static inline int ln_bwd_ctas(int64_t N) {
+    int64_t g = (N + kLnWarps - 1) / kLnWarps;
+    if (g > 148 * 4) g = 148 * 4;
+    return (int)g;
+}
+size_t layernorm_bwd_scratch_floats(int64_t N, int C) { return (size_t)ln_bwd_ctas(N) * 2 * C; }
+
+template <int VPL>
+__global__ void __launch_bounds__(kLnWarps * 32) ln_bwd_kernel(
+    const float* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ gamma,
+    const float* __restrict__ mean, const float* __restrict__ rstd, const float* dres, int64_t N, int C4,
+    float* dx, float* dx_hi, float* dx_lo, float* __restrict__ partial) {
+    extern __shared__ float4 sm[];  // [2][C4]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const float inv_c = 1.0f / (float)(C4 * 4);
+    float4 ag[VPL], ab[VPL], gm[VPL];
+#pragma unroll
+    for (int k = 0; k < VPL; ++k) {
+        ag[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        ab[k] = make_float4(0.f, 0.f, 0.f, 0.f);
+        int idx = lane + 32 * k;
+        gm[k] = (idx < C4) ? ld4(gamma, idx) : make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    for (int64_t row = (int64_t)blockIdx.x * kLnWarps + warp; row < N; row += (int64_t)gridDim.x * kLnWarps) {
+        const float mu = mean[row], rs = rstd[row];
+        float4 xh[VPL], dh[VPL];
+        float s1 = 0.f, s2 = 0.f;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            int idx = lane + 32 * k;
+            if (idx < C4) {
+                float4 xv = ld4(x, row * C4 + idx), d = ld4(dy, row * C4 + idx);
+                xh[k] = make_float4((xv.x - mu) * rs, (xv.y - mu) * rs, (xv.z - mu) * rs, (xv.w - mu) * rs);
+                dh[k] = make_float4(d.x * gm[k].x, d.y * gm[k].y, d.z * gm[k].z, d.w * gm[k].w);
+                s1 += (dh[k].x + dh[k].y) + (dh[k].z + dh[k].w);
+                s2 += (dh[k].x * xh[k].x + dh[k].y * xh[k].y) + (dh[k].z * xh[k].z + dh[k].w * xh[k].w);
+                ag[k].x += d.x * xh[k].x; ag[k].y += d.y * xh[k].y; ag[k].z += d.z * xh[k].z; ag[k].w += d.w * xh[k].w;
+                ab[k] = add4(ab[k], d);
+            }
+        }
+        s1 = warp_sum(s1) * inv_c;
+        s2 = warp_sum(s2) * inv_c;
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            int idx = lane + 32 * k;
+            if (idx < C4) {
+                float4 r;
+                r.x = rs * (dh[k].x - s1 - xh[k].x * s2);
+                r.y = rs * (dh[k].y - s1 - xh[k].y * s2);
+                r.z = rs * (dh[k].z - s1 - xh[k].z * s2);
+                r.w = rs * (dh[k].w - s1 - xh[k].w * s2);
+                if (dres) r = add4(r, ld4(dres, row * C4 + idx));
+                store_raw_split(r, dx, dx_hi, dx_lo, row * C4 + idx);
+            }
+        }
+    }
+    // combine the CTA's warps in warp order, then publish the CTA partial
+    for (int w = 0; w < kLnWarps; ++w) {
+        if (warp == w) {
+#pragma unroll
+            for (int k = 0; k < VPL; ++k) {
+                int idx = lane + 32 * k;
+                if (idx < C4) {
+                    if (w == 0) {
+                        sm[idx] = ag[k];
+                        sm[C4 + idx] = ab[k];
+                    } else {
+                        sm[idx] = add4(sm[idx], ag[k]);
+                        sm[C4 + idx] = add4(sm[C4 + idx], ab[k]);
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+    float4* dst = reinterpret_cast<float4*>(partial) + (int64_t)blockIdx.x * 2 * C4;
+    for (int i = threadIdx.x; i < 2 * C4; i += blockDim.x) dst[i] = sm[i];
+}
+
+__global__ void __launch_bounds__(128) ln_bwd_reduce_kernel(const float* __restrict__ partial, int nparts, int C4,
+                                                            float* __restrict__ dgamma, float* __restrict__ dbeta) {
+    int c = blockIdx.x * blockDim.x + threadIdx.x;  // float4 column over [2*C4): first dgamma, then dbeta
+    if (c >= 2 * C4) return;
+    float4 t = ld4(partial, c);
+    for (int p = 1; p < nparts; ++p) t = add4(t, ld4(partial, (int64_t)p * 2 * C4 + c));
+    if (c < C4) reinterpret_cast<float4*>(dgamma)[c] = t;
+    else reinterpret_cast<float4*>(dbeta)[c - C4] = t;
+}
+
+cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
+                                 const float* rstd, const float* dres, int64_t N, int C, float* dx, float* dx_hi,
+                                 float* dx_lo, float* dgamma, float* dbeta, float* scratch, cudaStream_t s) {
+    const int C4 = C / 4;
+    const int vpl = (C4 + 31) / 32;
+    const int grid = ln_bwd_ctas(N);
+    const size_t smem = (size_t)2 * C4 * sizeof(float4);
+#define BT_LN_BWD(V)                                                                                         \
+    ln_bwd_kernel<V><<<grid, kLnWarps * 32, smem, s>>>(dy, x, gamma, mean, rstd, dres, N, C4, dx, dx_hi, dx_lo, \
+                                                        scratch)
+    if (vpl <= 1) BT_LN_BWD(1);
+    else if (vpl <= 2) BT_LN_BWD(2);
+    else if (vpl <= 4) BT_LN_BWD(4);
+    else if (vpl <= 6) BT_LN_BWD(6);
+    else if (vpl <= 8) BT_LN_BWD(8);
+    else return cudaErrorInvalidValue;
+#undef BT_LN_BWD
+    BT_COUNT_LAUNCH();
+    ln_bwd_reduce_kernel<<<(2 * C4 + 127) / 128, 128, 0, s>>>(scratch, grid, C4, dgamma, dbeta);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+}  // namespace bt

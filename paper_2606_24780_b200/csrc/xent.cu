@@ -1,0 +1,156 @@
+// Fused softmax cross-entropy forward + backward over the padded vocabulary.
+//
+// One CTA of 512 threads owns one row of logits.  The row (201 KB at Vp = 50304) is read
+// from HBM exactly once into registers with 128-bit loads, reduced (max, then sum of
+// exponentials) with warp shuffles plus one shared-memory hop, and the gradient
+// (softmax - onehot) * inv_count is written once, raw and/or as TF32 hi/lo planes for the two
+// LM-head backward GEMMs.  Per-row losses go to an array that a second one-CTA kernel sums in
+// index order, so the mean loss is deterministic.
+#include "common.cuh"
+
+namespace bt {
+
+constexpr int kXentThreads = 512;
+
+__device__ __forceinline__ float block_reduce(float v, bool is_max, float* sm) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    v = is_max ? warp_max(v) : warp_sum(v);
+    __syncthreads();  // protect sm reuse between consecutive reductions
+    if (lane == 0) sm[warp] = v;
+    __syncthreads();
+    float r = sm[0];
+    for (int w = 1; w < kXentThreads / 32; ++w) r = is_max ? fmaxf(r, sm[w]) : r + sm[w];
+    return r;
+}
+
+template <int ITEMS>
+__global__ void __launch_bounds__(kXentThreads) xent_kernel(const float* __restrict__ logits,
+                                                            const int32_t* __restrict__ targets, int V4,
+                                                            float inv_count, float* __restrict__ losses, float* dl,
+                                                            float* dl_hi, float* dl_lo) {
+    __shared__ float sm[kXentThreads / 32];
+    const int64_t row = blockIdx.x;
+    const int64_t base = row * V4;
+    float4 v[ITEMS];
+    float mx = -INFINITY;
+#pragma unroll
+    for (int k = 0; k < ITEMS; ++k) {
+        int idx = threadIdx.x + kXentThreads * k;
+        if (idx < V4) {
+            v[k] = __ldcs(reinterpret_cast<const float4*>(logits) + base + idx);
+            mx = fmaxf(mx, fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w)));
+        }
+    }
+    mx = block_reduce(mx, true, sm);
+    float sum = 0.f;
+#pragma unroll
+    for (int k = 0; k < ITEMS; ++k) {
+        int idx = threadIdx.x + kXentThreads * k;
+        if (idx < V4) {
+            v[k].x = expf(v[k].x - mx);
+            v[k].y = expf(v[k].y - mx);
+            v[k].z = expf(v[k].z - mx);
+            v[k].w = expf(v[k].w - mx);
+            sum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+        }
+    }
+    sum = block_reduce(sum, false, sm);
+    const int t = targets[row];
+    if (threadIdx.x == 0) losses[row] = (mx + logf(sum)) - logits[row * V4 * 4 + t];
+    if (dl == nullptr && dl_hi == nullptr) return;
+    const float sc = inv_count / sum;
+#pragma unroll
+    for (int k = 0; k < ITEMS; ++k) {
+        int idx = threadIdx.x + kXentThreads * k;
+        if (idx < V4) {
+            float4 r = make_float4(v[k].x * sc, v[k].y * sc, v[k].z * sc, v[k].w * sc);
+            if ((t >> 2) == idx) {
+                int j = t & 3;
+                if (j == 0) r.x -= inv_count;
+                else if (j == 1) r.y -= inv_count;
+                else if (j == 2) r.z -= inv_count;
+                else r.w -= inv_count;
+            }
+            store_raw_split(r, dl, dl_hi, dl_lo, base + idx);
+        }
+    }
+}
+
+// Rows longer than the register path covers: three passes over global memory (the second and
+// third are served by L2 for rows of a few hundred KB).
+__global__ void __launch_bounds__(kXentThreads) xent_generic_kernel(const float* __restrict__ logits,
+                                                                    const int32_t* __restrict__ targets, int V4,
+                                                                    float inv_count, float* __restrict__ losses,
+                                                                    float* dl, float* dl_hi, float* dl_lo) {
+    __shared__ float sm[kXentThreads / 32];
+    const int64_t row = blockIdx.x;
+    const int64_t base = row * V4;
+    float mx = -INFINITY;
+    for (int idx = threadIdx.x; idx < V4; idx += kXentThreads) {
+        float4 a = ld4(logits, base + idx);
+        mx = fmaxf(mx, fmaxf(fmaxf(a.x, a.y), fmaxf(a.z, a.w)));
+    }
+    mx = block_reduce(mx, true, sm);
+    float sum = 0.f;
+    for (int idx = threadIdx.x; idx < V4; idx += kXentThreads) {
+        float4 a = ld4(logits, base + idx);
+        sum += (expf(a.x - mx) + expf(a.y - mx)) + (expf(a.z - mx) + expf(a.w - mx));
+    }
+    sum = block_reduce(sum, false, sm);
+    const int t = targets[row];
+    if (threadIdx.x == 0) losses[row] = (mx + logf(sum)) - logits[row * V4 * 4 + t];
+    if (dl == nullptr && dl_hi == nullptr) return;
+    const float sc = inv_count / sum;
+    for (int idx = threadIdx.x; idx < V4; idx += kXentThreads) {
+        float4 a = ld4(logits, base + idx);
+        float4 r = make_float4(expf(a.x - mx) * sc, expf(a.y - mx) * sc, expf(a.z - mx) * sc, expf(a.w - mx) * sc);
+        if ((t >> 2) == idx) {
+            int j = t & 3;
+            if (j == 0) r.x -= inv_count;
+            else if (j == 1) r.y -= inv_count;
+            else if (j == 2) r.z -= inv_count;
+            else r.w -= inv_count;
+        }
+        store_raw_split(r, dl, dl_hi, dl_lo, base + idx);
+    }
+}
+
+// loss_mean = inv_count * sum_n losses[n], summed in a fixed tree order by one CTA.
+__global__ void __launch_bounds__(1024) loss_mean_kernel(const float* __restrict__ losses, int64_t N, float inv_count,
+                                                         float* __restrict__ loss_mean) {
+    __shared__ double sm[1024];
+    double t = 0.0;
+    for (int64_t i = threadIdx.x; i < N; i += 1024) t += (double)losses[i];
+    sm[threadIdx.x] = t;
+    __syncthreads();
+    for (int o = 512; o > 0; o >>= 1) {
+        if (threadIdx.x < o) sm[threadIdx.x] += sm[threadIdx.x + o];
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *loss_mean = (float)(sm[0] * (double)inv_count);
+}
+
+cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int Vp, float inv_count,
+                                float* losses, float* loss_mean, float* dl, float* dl_hi, float* dl_lo,
+                                cudaStream_t s) {
+    const int V4 = Vp / 4;
+    const int items = (V4 + kXentThreads - 1) / kXentThreads;
+#define BT_XENT(I)                                                                                              \
+    xent_kernel<I><<<(int)N, kXentThreads, 0, s>>>(logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo)
+    if (items <= 1) BT_XENT(1);
+    else if (items <= 2) BT_XENT(2);
+    else if (items <= 4) BT_XENT(4);
+    else if (items <= 8) BT_XENT(8);
+    else if (items <= 16) BT_XENT(16);
+    else if (items <= 25) BT_XENT(25);
+    else xent_generic_kernel<<<(int)N, kXentThreads, 0, s>>>(logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo);
+#undef BT_XENT
+    BT_COUNT_LAUNCH();
+    if (loss_mean) {
+        loss_mean_kernel<<<1, 1024, 0, s>>>(losses, N, inv_count, loss_mean);
+        BT_COUNT_LAUNCH();
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace bt

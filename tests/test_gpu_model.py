@@ -1,0 +1,166 @@
+"""Whole-step GPU parity: forward, backward and AdamW of the CUDA library against the CPU
+float64 oracle on the same seeded parameters and tokens.
+
+Tolerances (the target the build is held to): logits and loss 1e-4 relative; every gradient
+tensor 1e-3 relative L2; post-AdamW parameters 1e-5 absolute.  "Relative" for a tensor means
+max|diff| / max|reference| and ||diff||_2 / ||reference||_2.  A gradient that is
+mathematically zero (the key bias: softmax is shift invariant) is held to an absolute bound
+scaled by the neighbouring query-bias gradient instead.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import seeded_inputs as si
+from paper_2606_24780_b200 import binding as b
+
+from gpu_util import dev, host, rel_l2, rel_max
+
+pytestmark = pytest.mark.gpu
+
+TOL_LOGITS, TOL_LOSS, TOL_GRAD, TOL_PARAM = 1e-4, 1e-4, 1e-3, 1e-5
+
+
+def make_pair(cfg, seed, flags, max_batch, jitter=0.02):
+    params = si.init_params(cfg, seed, jitter=jitter)
+    gm = b.Model(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["seq_len"], cfg["vocab_size"],
+                 cfg["padded_vocab_size"], max_batch, flags)
+    gm.load_params(params)
+    om = oracle.Model(cfg)
+    om.set_params(params)
+    return gm, om
+
+
+def compare_gradients(gm, om, cfg):
+    C = cfg["d_model"]
+    worst = 0.0
+    for name in om.names():
+        ref = om.get(name, 1)
+        got = host(gm.tensor(name, 1))
+        if name.endswith("attn.qkv.b"):
+            # q and v parts relative; the k part is exactly zero in exact arithmetic
+            for lo, hi in ((0, C), (2 * C, 3 * C)):
+                e = rel_l2(got[lo:hi], ref[lo:hi])
+                assert e < TOL_GRAD, (name, lo, e)
+                worst = max(worst, e)
+            assert np.abs(ref[C:2 * C]).max() < 1e-12
+            assert np.abs(got[C:2 * C]).max() < 1e-3 * np.abs(ref[:C]).max(), name
+            continue
+        e = rel_l2(got, ref)
+        assert e < TOL_GRAD, (name, e)
+        worst = max(worst, e)
+    return worst
+
+
+def run_steps(cfg, seed, flags, B, steps, chunk=0):
+    gm, om = make_pair(cfg, seed, flags, B)
+    hp = si.ADAMW
+    opt = b.make_adamw(**hp)
+    Vp = cfg["padded_vocab_size"]
+    for step in range(steps):
+        tok, tgt = si.tokens_for(cfg, 1000 * seed + step, B)
+        dtok, dtgt = dev(tok), dev(tgt)
+        loss = gm.forward(dtok, dtgt)
+        ref_loss = om.loss_and_grad(tok, tgt, chunk)
+        assert abs(loss - ref_loss) < TOL_LOSS * abs(ref_loss), (step, loss, ref_loss)
+        if chunk == 0:
+            ref_logits = om.activation("logits")
+            got_logits = host(gm.activation("logits")).reshape(-1, Vp)
+            assert rel_max(got_logits, ref_logits) < TOL_LOGITS and rel_l2(got_logits, ref_logits) < TOL_LOGITS
+        gm.backward()
+        compare_gradients(gm, om, cfg)
+        gn = gm.adamw_step(opt)
+        ref_gn = om.adamw_step(hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], hp["grad_clip"])
+        assert abs(gn - ref_gn) < 1e-4 * ref_gn
+        for name in om.names():
+            d = np.abs(host(gm.tensor(name)) - om.get(name)).max()
+            assert d < TOL_PARAM, (step, name, d)
+            # feed the oracle's FP32-rounded parameters forward so steps stay comparable
+        assert b.bt_get_step(gm.h) == step + 1
+    launches = b.bt_launch_count(gm.h)
+    gm.close()
+    return launches
+
+
+@pytest.mark.parametrize("flags", [b.BT_FLAG_GEMM_SIMT | b.BT_FLAG_ATTN_SIMT, b.BT_FLAG_ATTN_SIMT, 0])
+def test_tiny_config_three_steps(flags):
+    """BASELINE config 0, three consecutive optimizer steps (the first alone barely exercises
+    the moments, the bias correction or the clip)."""
+    cfg = si.config(0)
+    launches = run_steps(cfg, seed=0, flags=flags, B=cfg["batch"], steps=3)
+    assert launches > 3 * 50
+
+
+def test_initial_loss_near_log_vocab():
+    cfg = si.config(0)
+    gm, _ = make_pair(cfg, 0, 0, cfg["batch"], jitter=0.0)
+    tok, tgt = si.tokens_for(cfg, 0)
+    loss = gm.forward(dev(tok), dev(tgt))
+    assert abs(loss - (math.log(cfg["padded_vocab_size"]) + 0.5 * cfg["d_model"] * 0.02 ** 2)) < 0.05
+    gm.close()
+
+
+def test_medium_config_spans_tiles_and_ragged_tails():
+    """GPT-2-small width with a short context and a small vocabulary: several GEMM tiles in every
+    dimension, ragged M (B*T = 3*200 = 600 rows), Zipf tokens, head_dim 64."""
+    cfg = si.make_config(n_layers=2, d_model=768, n_heads=12, seq_len=200, vocab_size=4000,
+                         padded_vocab_size=4032, batch=3, tokens="zipf")
+    run_steps(cfg, seed=3, flags=0, B=3, steps=2)
+
+
+def test_partial_batch_and_host_tokens():
+    """A batch smaller than max_batch, and the host-buffer entry point, give the same step."""
+    cfg = si.config(0)
+    params = si.init_params(cfg, 5, jitter=0.02)
+    opt = b.make_adamw(**si.ADAMW)
+    tok, tgt = si.tokens_for(cfg, 5, 3)
+    results = []
+    for host_path in (False, True):
+        gm = b.Model(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["seq_len"], cfg["vocab_size"],
+                     cfg["padded_vocab_size"], 8)
+        gm.load_params(params)
+        if host_path:
+            loss = gm.train_step_host(torch.as_tensor(tok).pin_memory(), torch.as_tensor(tgt).pin_memory(), opt)
+        else:
+            loss = gm.train_step(dev(tok), dev(tgt), opt)
+        results.append((loss, host(gm.tensor("h1.mlp.fc.w")), host(gm.tensor("wte"))))
+        gm.close()
+    assert results[0][0] == results[1][0]
+    assert np.array_equal(results[0][1], results[1][1]) and np.array_equal(results[0][2], results[1][2])
+    om = oracle.Model(cfg)
+    om.set_params(params)
+    ref = om.loss_and_grad(tok, tgt)
+    assert abs(results[0][0] - ref) < TOL_LOSS * ref
+
+
+def test_step_is_deterministic():
+    cfg = si.config(0)
+    params = si.init_params(cfg, 6, jitter=0.02)
+    opt = b.make_adamw(**si.ADAMW)
+    tok, tgt = si.tokens_for(cfg, 6)
+    outs = []
+    for _ in range(2):
+        gm = b.Model(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["seq_len"], cfg["vocab_size"],
+                     cfg["padded_vocab_size"], cfg["batch"])
+        gm.load_params(params)
+        gm.train_step(dev(tok), dev(tgt), opt)
+        outs.append(torch.cat([gm.tensor(n).clone() for n, _, _ in gm.names]))
+        gm.close()
+    assert torch.equal(outs[0], outs[1])
+
+
+def test_model_init_distribution():
+    cfg = si.config(0)
+    gm = b.Model(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["seq_len"], cfg["vocab_size"],
+                 cfg["padded_vocab_size"], 1)
+    gm.init(1234)
+    wte = host(gm.tensor("wte"))
+    assert abs(wte.mean()) < 1e-3 and abs(wte.std() - 0.02) < 5e-4
+    pr = host(gm.tensor("h1.mlp.proj.w"))
+    assert abs(pr.std() - 0.02 / math.sqrt(2 * cfg["n_layers"])) < 5e-4
+    assert np.all(host(gm.tensor("h0.ln1.g")) == 1.0) and not host(gm.tensor("h0.attn.qkv.b")).any()
+    assert not host(gm.tensor("wte", 2)).any()
+    gm.close()

@@ -1,0 +1,256 @@
+"""GPU parity tests, one kernel at a time: every per-op C-ABI entry point against the CPU
+float64 oracle on the same seeded FP32 inputs.
+
+Tolerances: embedding gather bit-exact; plain-FP32 kernels (LayerNorm, GELU, softmax
+cross-entropy, column sums, norm, AdamW) 1e-5 relative L2; 3xTF32 tensor-core GEMM and
+attention outputs 1e-4 relative (max and L2).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import seeded_inputs as si
+from paper_2606_24780_b200 import binding as b
+
+from gpu_util import check_split, dev, empty, host, rel_l2, rel_max, scratch, zeros
+
+pytestmark = pytest.mark.gpu
+
+
+# ------------------------------------------------------------------ embedding
+
+@pytest.mark.parametrize("B,T,C,V,zipf", [(4, 64, 64, 512, False), (3, 100, 768, 50257, True), (1, 1, 64, 8, False)])
+def test_embedding_fwd_bit_exact(B, T, C, V, zipf):
+    wte, wpe = si.normal_f32(1, (V, C), 0.02), si.normal_f32(2, (T, C), 0.02)
+    tok = (si.zipf_tokens(3, B, T, V) if zipf else si.uniform_tokens(3, B, T, V))[0]
+    x = empty(B * T, C)
+    b.bt_op_embedding_fwd(dev(tok), dev(wte), dev(wpe), B * T, T, C, x)
+    ref = oracle.embedding_fwd(tok, wte, wpe, T, round_fp32=True).astype(np.float32)
+    got = x.cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+
+
+@pytest.mark.parametrize("B,T,C,V,zipf", [(4, 64, 64, 512, False), (8, 300, 768, 50257, True), (2, 513, 128, 7, False)])
+def test_embedding_bwd(B, T, C, V, zipf):
+    tok = (si.zipf_tokens(5, B, T, V) if zipf else si.uniform_tokens(5, B, T, V))[0]
+    dx = si.normal_f32(6, (B * T, C), 1e-2)
+    base = si.normal_f32(7, (V, C), 1e-2)          # the LM-head gradient already in dwte
+    dwte, dwpe = dev(base), empty(T, C)
+    b.bt_op_embedding_bwd(dev(tok), dev(dx), B * T, T, C, dwte, dwpe)
+    rw, rp = oracle.embedding_bwd(tok, dx, T, V)
+    assert rel_l2(host(dwte), rw + base) < 1e-5
+    assert rel_l2(host(dwpe), rp) < 1e-5
+    untouched = np.setdiff1d(np.arange(V), np.unique(tok))
+    if untouched.size:
+        assert np.array_equal(dwte.cpu().numpy()[untouched], base[untouched])
+    # deterministic: a second run gives identical bits
+    dwte2, dwpe2 = dev(base), empty(T, C)
+    b.bt_op_embedding_bwd(dev(tok), dev(dx), B * T, T, C, dwte2, dwpe2)
+    assert torch.equal(dwte, dwte2) and torch.equal(dwpe, dwpe2)
+
+
+# ------------------------------------------------------------------ LayerNorm
+
+@pytest.mark.parametrize("N,C", [(256, 64), (1000, 768), (37, 1024), (5, 128), (300, 2048)])
+def test_layernorm_fwd(N, C):
+    x = si.normal_f32(10, (N, C), 2.0) + 0.5
+    g, be = si.normal_f32(11, (C,), 0.3) + 1.0, si.normal_f32(12, (C,), 0.3)
+    y, ys, mean, rstd = empty(N, C), empty(2, N, C), empty(N), empty(N)
+    b.bt_op_layernorm_fwd(dev(x), dev(g), dev(be), N, C, y, ys, mean, rstd)
+    ry, rm, rr = oracle.layernorm_fwd(x, g, be)
+    assert rel_l2(host(y), ry) < 1e-5 and rel_max(host(y), ry) < 1e-5
+    assert rel_l2(host(mean), rm) < 1e-5 and rel_l2(host(rstd), rr) < 1e-5
+    check_split(ys, host(y))
+
+
+@pytest.mark.parametrize("N,C,res", [(256, 64, True), (1000, 768, True), (4100, 768, False), (37, 1024, True)])
+def test_layernorm_bwd(N, C, res):
+    x = si.normal_f32(13, (N, C), 1.5) - 0.2
+    g = si.normal_f32(14, (C,), 0.3) + 1.0
+    dy = si.normal_f32(15, (N, C), 1e-2)
+    dres = si.normal_f32(16, (N, C), 1e-2) if res else None
+    _, rm, rr = oracle.layernorm_fwd(x, g, np.zeros(C))
+    mean, rstd = dev(rm, torch.float32), dev(rr, torch.float32)
+    dx, dxs, dg, db = empty(N, C), empty(2, N, C), empty(C), empty(C)
+    nb = b.bt_op_layernorm_bwd_scratch_bytes(N, C)
+    b.bt_op_layernorm_bwd(dev(dy), dev(x), dev(g), mean, rstd, dev(dres) if res else None, N, C, dx, dxs, dg, db,
+                          scratch(nb), nb)
+    rdx, rdg, rdb = oracle.layernorm_bwd(dy, x, g, host(mean), host(rstd))
+    if res:
+        rdx = rdx + dres
+    assert rel_l2(host(dx), rdx) < 1e-5
+    assert rel_l2(host(dg), rdg) < 1e-5 and rel_l2(host(db), rdb) < 1e-5
+    check_split(dxs, host(dx))
+
+
+def test_layernorm_bwd_in_place_residual():
+    """The step updates the residual-stream gradient in place (dx aliases dres)."""
+    N, C = 600, 768
+    x, g = si.normal_f32(17, (N, C)), si.normal_f32(18, (C,), 0.2) + 1.0
+    dy, dres = si.normal_f32(19, (N, C), 1e-2), si.normal_f32(20, (N, C), 1e-2)
+    _, rm, rr = oracle.layernorm_fwd(x, g, np.zeros(C))
+    buf = dev(dres)
+    nb = b.bt_op_layernorm_bwd_scratch_bytes(N, C)
+    b.bt_op_layernorm_bwd(dev(dy), dev(x), dev(g), dev(rm, torch.float32), dev(rr, torch.float32), buf, N, C, buf,
+                          None, empty(C), empty(C), scratch(nb), nb)
+    rdx, _, _ = oracle.layernorm_bwd(dy, x, g, rm.astype(np.float32), rr.astype(np.float32))
+    assert rel_l2(host(buf), rdx + dres) < 1e-5
+
+
+# ------------------------------------------------------------------ GELU
+
+@pytest.mark.parametrize("tanh_form", [0, 1])
+def test_gelu_fwd_bwd(tanh_form):
+    n = 4 * 12345
+    x = np.concatenate([si.normal_f32(21, (n - 8,), 2.0), np.array([0, -0.0, 10, -10, 30, -30, 1e-20, -5], np.float32)])
+    dy = si.normal_f32(22, (n,), 1e-2)
+    y, ys, dx, dxs = empty(n), empty(2, n), empty(n), empty(2, n)
+    b.bt_op_gelu_fwd(dev(x), n, tanh_form, y, ys)
+    b.bt_op_gelu_bwd(dev(x), dev(dy), n, tanh_form, dx, dxs)
+    ry, rdx = oracle.gelu_fwd(x, tanh_form), oracle.gelu_bwd(x, dy, tanh_form)
+    assert rel_l2(host(y), ry) < 1e-5 and np.abs(host(y) - ry).max() < 2e-6
+    assert rel_l2(host(dx), rdx) < 1e-5
+    check_split(ys, host(y))
+    check_split(dxs, host(dx))
+
+
+# ------------------------------------------------------------------ softmax cross-entropy
+
+@pytest.mark.parametrize("N,Vp", [(256, 512), (64, 50304), (7, 1000), (3, 131072), (5, 4)])
+def test_softmax_xent(N, Vp):
+    z = si.normal_f32(23, (N, Vp), 3.0)
+    z[0, :] = 0.0
+    if N > 1:
+        z[1, 3 % Vp] = 80.0
+    y = si.uniform_tokens(24, 1, N, Vp)[0].ravel()
+    inv = 1.0 / (4 * N)                      # as if this were one chunk of a larger batch
+    losses, lm, dl, dls = empty(N), empty(1), empty(N, Vp), empty(2, N, Vp)
+    b.bt_op_softmax_xent(dev(z), dev(y), N, Vp, inv, losses, lm, dl, dls)
+    rl, rdl = oracle.softmax_xent(z, y, inv)
+    assert rel_l2(host(losses), rl) < 1e-5 and np.abs(host(losses) - rl).max() < 1e-4
+    assert abs(float(host(lm)[0]) - rl.sum() * inv) < 1e-5 * abs(rl.sum() * inv)
+    assert rel_l2(host(dl), rdl) < 1e-5
+    assert np.abs(host(dl).sum(1)).max() < 1e-6 * inv * Vp ** 0.5 + 1e-9
+    check_split(dls, host(dl))
+
+
+# ------------------------------------------------------------------ reductions
+
+@pytest.mark.parametrize("N,C", [(256, 64), (8192, 768), (1000, 3072), (33, 2304)])
+def test_colsum(N, C):
+    x = si.normal_f32(25, (N, C), 1e-2)
+    out = empty(C)
+    nb = b.bt_op_colsum_scratch_bytes(N, C)
+    b.bt_op_colsum(dev(x), N, C, out, scratch(nb), nb)
+    assert rel_l2(host(out), x.astype(np.float64).sum(0)) < 1e-5
+
+
+@pytest.mark.parametrize("n,mag", [(136960, 1e-3), (5_000_003, 1.0), (4, 100.0)])
+def test_grad_norm_and_clip(n, mag):
+    g = si.normal_f32(26, (n,), mag)
+    out = empty(2)
+    nb = b.bt_op_grad_norm_scratch_bytes(n)
+    b.bt_op_grad_norm(dev(g), n, 1.0, out, scratch(nb), nb)
+    gn = oracle.grad_norm([g])
+    got = host(out)
+    assert abs(got[0] - gn) < 1e-6 * gn
+    assert abs(got[1] - oracle.clip_scale(gn, 1.0)) < 1e-6
+    b.bt_op_grad_norm(dev(g), n, 0.0, out, scratch(nb), nb)
+    assert host(out)[1] == 1.0
+
+
+# ------------------------------------------------------------------ AdamW
+
+def test_adamw_multi_matches_oracle_at_step_seven():
+    shapes = [(50304 * 8,), (768,), (4097,), (3,), (2304 * 64,)]
+    decay = [1, 0, 1, 0, 1]
+    hp = si.ADAMW
+    opt = b.make_adamw(**hp)
+    t, scale = 7, 0.37
+    ps, gs, ms, vs = [], [], [], []
+    for i, s in enumerate(shapes):
+        ps.append(si.normal_f32(30 + i, s, 0.02))
+        gs.append(si.normal_f32(40 + i, s, 10.0 ** -(i + 1)))
+        ms.append(si.normal_f32(50 + i, s, 1e-3))
+        vs.append(np.abs(si.normal_f32(60 + i, s, 1e-5)))
+    dp, dg, dm, dv = [dev(a) for a in ps], [dev(a) for a in gs], [dev(a) for a in ms], [dev(a) for a in vs]
+    b.bt_op_adamw_multi(dp, dg, dm, dv, decay, opt, t, d_scale=dev(np.array([scale], np.float32)))
+    for i in range(len(shapes)):
+        rp, rm, rv = oracle.adamw(ps[i], gs[i], ms[i], vs[i], hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                  hp["weight_decay"], decay[i], t, np.float32(scale))
+        assert np.abs(host(dp[i]) - rp).max() < 1e-6, i
+        assert rel_l2(host(dm[i]), rm) < 1e-6 and rel_l2(host(dv[i]), rv) < 1e-6
+
+
+# ------------------------------------------------------------------ GEMM
+
+GEMM_SHAPES = [
+    (0, 256, 192, 64), (1, 256, 64, 192), (2, 192, 64, 256),          # tiny model
+    (0, 1000, 2304, 768), (0, 520, 768, 3072),                        # ragged M, both tile widths
+    (1, 1000, 768, 2304), (1, 384, 3072, 768),
+    (2, 768, 768, 4096), (2, 2304, 768, 2000), (2, 1056, 160, 520),   # split-K, ragged everything
+    (0, 128, 1056, 128), (0, 4, 4, 4),
+]
+
+
+@pytest.mark.parametrize("flags", [0, b.BT_FLAG_GEMM_SIMT])
+@pytest.mark.parametrize("layout,M,N,K", GEMM_SHAPES)
+def test_gemm(layout, M, N, K, flags):
+    if flags == 0 and ((layout == 2 and M % 32) or (layout != 0 and N % 32)):
+        pytest.skip("transposed extents must be multiples of 32 on the tensor-core path")
+    a_shape = (K, M) if layout == 2 else (M, K)
+    b_shape = (N, K) if layout == 0 else (K, N)
+    A, Bm = si.normal_f32(70, a_shape), si.normal_f32(71, b_shape, 0.05)
+    bias, res = si.normal_f32(72, (N,)), si.normal_f32(73, (M, N))
+    A64 = A.astype(np.float64).T if layout == 2 else A.astype(np.float64)
+    B64 = Bm.astype(np.float64).T if layout == 0 else Bm.astype(np.float64)
+    nb = b.bt_op_gemm_scratch_bytes(layout, M, N, K)
+    sc = scratch(nb)
+    for use_epi in (False, True):
+        D = zeros(M, N)
+        b.bt_op_gemm(layout, M, N, K, dev(A), dev(Bm), D, dev(bias) if use_epi else None,
+                     dev(res) if use_epi else None, sc, nb, flags)
+        ref = A64 @ B64
+        if use_epi:
+            ref = ref + bias + res
+        assert rel_l2(host(D), ref) < 1e-5 if flags else rel_l2(host(D), ref) < 1e-4, (layout, M, N, K, use_epi)
+        assert rel_max(host(D), ref) < 1e-4
+
+
+def test_gemm_matches_oracle_linear_layer():
+    """The three layouts are the forward, input-gradient and weight-gradient of a linear layer."""
+    N, cin, cout = 640, 768, 1024
+    x, w, bias = si.normal_f32(74, (N, cin)), si.normal_f32(75, (cout, cin), 0.02), si.normal_f32(76, (cout,), 0.1)
+    dy = si.normal_f32(77, (N, cout), 1e-2)
+    y, dx, dw = empty(N, cout), empty(N, cin), empty(cout, cin)
+    for lay, M, Nn, K, A, Bm, D, bi in [(0, N, cout, cin, x, w, y, bias), (1, N, cin, cout, dy, w, dx, None),
+                                       (2, cout, cin, N, dy, x, dw, None)]:
+        nb = b.bt_op_gemm_scratch_bytes(lay, M, Nn, K)
+        b.bt_op_gemm(lay, M, Nn, K, dev(A), dev(Bm), D, dev(bi) if bi is not None else None, None, scratch(nb), nb)
+    ry = oracle.linear_fwd(x, w, bias)
+    rdx, rdw, _ = oracle.linear_bwd(dy, x, w)
+    assert rel_l2(host(y), ry) < 1e-4 and rel_l2(host(dx), rdx) < 1e-4 and rel_l2(host(dw), rdw) < 1e-4
+
+
+# ------------------------------------------------------------------ attention
+
+@pytest.mark.parametrize("flags", [0, b.BT_FLAG_ATTN_SIMT])
+@pytest.mark.parametrize("B,T,H,d", [(4, 64, 4, 16), (2, 200, 3, 64), (1, 1, 2, 64), (1, 129, 2, 32), (1, 96, 1, 128)])
+def test_attention_fwd_bwd(B, T, H, d, flags):
+    C = H * d
+    qkv = si.normal_f32(80, (B * T, 3 * C))
+    d_o = si.normal_f32(81, (B * T, C), 1e-2)
+    o, os_, lse = empty(B * T, C), empty(2, B * T, C), empty(B, H, T)
+    b.bt_op_attention_fwd(dev(qkv), B, T, C, H, o, os_, lse, flags)
+    ro, rlse = oracle.attention_fwd(qkv, B, T, H)
+    assert rel_l2(host(o), ro) < 1e-4 and rel_max(host(o), ro) < 1e-4
+    assert np.abs(host(lse) - rlse).max() < 1e-4
+    check_split(os_, host(o))
+    dqkv, dqs = empty(B * T, 3 * C), empty(2, B * T, 3 * C)
+    nb = B * H * T * 4
+    b.bt_op_attention_bwd(dev(qkv), o, lse, dev(d_o), B, T, C, H, dqkv, dqs, scratch(nb), nb, flags)
+    rd = oracle.attention_bwd(qkv, d_o, B, T, H)
+    for part in range(3):
+        assert rel_l2(host(dqkv)[:, part * C:(part + 1) * C], rd[:, part * C:(part + 1) * C]) < 1e-4, part
+    check_split(dqs, host(dqkv))

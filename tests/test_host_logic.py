@@ -1,0 +1,77 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every declared symbol, and
+validates arguments on the host before any launch (no compute call is made here)."""
+import ctypes
+import os
+import re
+
+import pytest
+
+from paper_2606_24780_b200 import binding as b
+from paper_2606_24780_b200 import build as bt_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    bt_build.build()
+    return b.lib()
+
+
+def test_exports_every_declared_symbol(lib):
+    with open(os.path.join(ROOT, "include", "bt.h")) as f:
+        text = f.read()
+    declared = set(re.findall(r"\b(bt_[a-z0-9_]+)\s*\(", text))
+    declared -= {"bt_model", "bt_status", "bt_config", "bt_adamw_config"}
+    assert declared, "no declarations found"
+    raw = ctypes.CDLL(b.LIB_PATH)
+    for name in sorted(declared):
+        assert hasattr(raw, name), f"{name} declared in bt.h but not exported"
+    assert declared == set(b.exported_symbols()), declared ^ set(b.exported_symbols())
+
+
+def test_workspace_bytes_and_config_validation(lib):
+    good = b.make_config(2, 64, 4, 64, 512, 512, 4)
+    n = b.bt_workspace_bytes(good)
+    assert n > 0 and n % 256 == 0
+    bigger = b.make_config(2, 64, 4, 64, 512, 512, 8)
+    assert b.bt_workspace_bytes(bigger) > n
+    for bad in [b.make_config(0, 64, 4, 64, 512, 512, 4), b.make_config(2, 66, 4, 64, 512, 512, 4),
+                b.make_config(2, 64, 4, 64, 512, 500, 4), b.make_config(2, 64, 4, 64, 512, 520, 4),
+                b.make_config(2, 96, 4, 64, 512, 512, 4), b.make_config(2, 64, 4, 64, 512, 512, 0),
+                b.make_config(2, 2048, 16, 64, 512, 512, 1)]:
+        assert b.bt_workspace_bytes(bad) == 0
+        assert lib.bt_last_error()
+
+
+def test_null_and_misaligned_arguments_are_rejected(lib):
+    cfg = b.make_config(2, 64, 4, 64, 512, 512, 4)
+    with pytest.raises(b.BtError) as e:
+        b.bt_model_create(cfg, None, 1 << 30, stream=0)
+    assert e.value.status == 1
+    with pytest.raises(b.BtError) as e:
+        b.bt_model_create(cfg, 0x1001, 1 << 30, stream=0)
+    assert e.value.status == 1
+    with pytest.raises(b.BtError) as e:
+        b.bt_model_create(cfg, 0x10000, 1024, stream=0)          # workspace too small
+    assert e.value.status == 3
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_gelu_fwd(0x1000, 6, 0, 0x2000, None, stream=0)   # n not a multiple of 4
+    assert e.value.status == 1
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_gelu_fwd(0x1004, 8, 0, 0x2000, None, stream=0)   # misaligned
+    assert e.value.status == 1
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_gemm(7, 128, 128, 128, 0x1000, 0x2000, 0x3000, None, None, 0x4000, 1 << 40, 0, stream=0)
+    assert e.value.status == 1
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_gemm(0, 128, 128, 128, 0x1000, 0x2000, 0x3000, None, None, 0x4000, 16, 0, stream=0)
+    assert e.value.status == 3
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_attention_fwd(0x1000, 1, 8, 48, 2, 0x2000, None, 0x3000, 0, stream=0)   # head_dim 24
+    assert e.value.status == 2
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_softmax_xent(0x1000, 0x2000, 4, 10, 0.25, 0x3000, None, None, None, stream=0)
+    assert e.value.status == 1
+    assert b.bt_op_gemm_scratch_bytes(0, 128, 128, 128) > 0
+    assert b.bt_op_layernorm_bwd_scratch_bytes(1000, 768) > 0
