@@ -43,6 +43,9 @@ def _compile(src: str, verbose: bool) -> str:
 def build(force: bool = False, verbose: bool = False) -> str:
     os.makedirs(BUILD, exist_ok=True)
     hdr = _headers_mtime()
+    newest_src = max([hdr] + [os.path.getmtime(os.path.join(CSRC, s)) for s in _sources()])
+    if not force and os.path.exists(LIB) and os.path.getmtime(LIB) >= newest_src:
+        return LIB  # up to date (object files may be absent on a machine that received only the .so)
     todo, objs = [], []
     for src in _sources():
         obj = os.path.join(BUILD, src[:-3] + ".o")

@@ -55,10 +55,52 @@ def compare_gradients(gm, om, cfg):
     return worst
 
 
-def run_steps(cfg, seed, flags, B, steps, chunk=0):
-    gm, om = make_pair(cfg, seed, flags, B)
+def adamw_step_and_compare(gm, om, step):
+    """One optimizer step on both sides from IDENTICAL state (p, m, v, t), two comparisons.
+
+    (A) optimizer exactness: the oracle's AdamW applied to the GPU's own gradient must give the
+        GPU's new parameters within 1e-5 absolute on EVERY element (and the moments within 1e-5
+        relative L2).  This is the post-AdamW tolerance for the update itself.
+    (B) end to end against the oracle's own gradient: the update lr * mhat / (sqrt(vhat) + eps)
+        is ill-conditioned where an element's gradient history is ~0 (at t = 1 it is
+        lr * g / (|g| + eps): slope lr / eps = 6e4 at g = 0, so an FP32-rounding-sized gradient
+        error flips the whole +-lr step).  Elements outside 1e-5 must therefore be rare and
+        bounded by 2.2 lr; their count is reported.
+    """
     hp = si.ADAMW
     opt = b.make_adamw(**hp)
+    names = om.names()
+    g_gpu = {n: host(gm.tensor(n, 1)) for n in names}
+    state = {n: (om.get(n, 0), om.get(n, 2), om.get(n, 3)) for n in names}
+    gn_gpu_ref = oracle.grad_norm(list(g_gpu.values()))
+    scale = oracle.clip_scale(gn_gpu_ref, hp["grad_clip"])
+    gn = gm.adamw_step(opt)
+    ref_gn = om.adamw_step(hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], hp["grad_clip"])
+    assert abs(gn - ref_gn) < 1e-4 * ref_gn and abs(gn - gn_gpu_ref) < 1e-5 * gn_gpu_ref
+    total, outside, worst_a = 0, 0, 0.0
+    for n in names:
+        p0, m0, v0 = state[n]
+        pb, mb, vb = oracle.adamw(p0, g_gpu[n], m0, v0, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+                                  hp["weight_decay"], om.decay(n), step + 1, scale)
+        got = host(gm.tensor(n))
+        da = np.abs(got - pb).max()
+        worst_a = max(worst_a, da)
+        assert da < TOL_PARAM, (step, n, da)                                   # (A)
+        assert rel_l2(host(gm.tensor(n, 2)), mb) < 1e-5 and rel_l2(host(gm.tensor(n, 3)), vb) < 1e-5, n
+        db = np.abs(got - om.get(n))                                           # (B)
+        total += db.size
+        outside += int((db >= TOL_PARAM).sum())
+        assert db.max() <= 2.2 * hp["lr"], (step, n, db.max())
+    assert outside <= 0.02 * total, (step, outside, total)
+    # continue from identical state: the oracle adopts the GPU's FP32 parameters and moments
+    for n in names:
+        for kind in (0, 2, 3):
+            om.set_tensor(n, host(gm.tensor(n, kind)), kind)
+    return outside / total, worst_a
+
+
+def run_steps(cfg, seed, flags, B, steps, chunk=0):
+    gm, om = make_pair(cfg, seed, flags, B)
     Vp = cfg["padded_vocab_size"]
     for step in range(steps):
         tok, tgt = si.tokens_for(cfg, 1000 * seed + step, B)
@@ -72,13 +114,9 @@ def run_steps(cfg, seed, flags, B, steps, chunk=0):
             assert rel_max(got_logits, ref_logits) < TOL_LOGITS and rel_l2(got_logits, ref_logits) < TOL_LOGITS
         gm.backward()
         compare_gradients(gm, om, cfg)
-        gn = gm.adamw_step(opt)
-        ref_gn = om.adamw_step(hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], hp["grad_clip"])
-        assert abs(gn - ref_gn) < 1e-4 * ref_gn
-        for name in om.names():
-            d = np.abs(host(gm.tensor(name)) - om.get(name)).max()
-            assert d < TOL_PARAM, (step, name, d)
-            # feed the oracle's FP32-rounded parameters forward so steps stay comparable
+        frac, worst = adamw_step_and_compare(gm, om, step)
+        print(f"step {step}: loss {loss:.6f} (oracle {ref_loss:.6f}); AdamW exactness {worst:.2e}; "
+              f"{100 * frac:.3f}% of parameters ill-conditioned")
         assert b.bt_get_step(gm.h) == step + 1
     launches = b.bt_launch_count(gm.h)
     gm.close()
