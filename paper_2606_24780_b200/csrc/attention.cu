@@ -1,4 +1,5 @@
-// Attention dispatch: tensor-core kernels by default, the FP32 FMA reference on request.
+// Attention dispatch: tensor-core kernels by default, the FP32 FMA reference on request (and
+// for head_dim 128, which the tensor-core kernels are not instantiated for).
 #include "common.cuh"
 
 namespace bt {
@@ -8,18 +9,29 @@ cudaError_t launch_attention_fwd_simt(const float* qkv, int B, int T, int C, int
 cudaError_t launch_attention_bwd_simt(const float* qkv, const float* o, const float* o_lo, const float* lse,
                                       const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
                                       float* dqkv_lo, float* dvec, cudaStream_t s);
+cudaError_t launch_attention_dvec(const float* o, const float* o_lo, const float* d_o, int B, int T, int C, int H,
+                                  float* dvec, cudaStream_t s);
+bool attention_mma_supports(int head_dim);
+cudaError_t launch_attention_fwd_mma(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi,
+                                     float* o_lo, float* lse, cudaStream_t s);
+cudaError_t launch_attention_bwd_mma(const float* qkv, const float* lse, const float* d_o, const float* dvec, int B,
+                                     int T, int C, int H, float* dqkv, float* dqkv_hi, float* dqkv_lo,
+                                     cudaStream_t s);
 
 cudaError_t launch_attention_fwd(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi, float* o_lo,
                                  float* lse, bool simt, cudaStream_t s) {
-    (void)simt;
-    return launch_attention_fwd_simt(qkv, B, T, C, H, o, o_hi, o_lo, lse, s);
+    if (simt || !attention_mma_supports(C / H)) return launch_attention_fwd_simt(qkv, B, T, C, H, o, o_hi, o_lo, lse, s);
+    return launch_attention_fwd_mma(qkv, B, T, C, H, o, o_hi, o_lo, lse, s);
 }
 
 cudaError_t launch_attention_bwd(const float* qkv, const float* o, const float* o_lo, const float* lse,
                                  const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
                                  float* dqkv_lo, float* dvec, bool simt, cudaStream_t s) {
-    (void)simt;
-    return launch_attention_bwd_simt(qkv, o, o_lo, lse, d_o, B, T, C, H, dqkv, dqkv_hi, dqkv_lo, dvec, s);
+    if (simt || !attention_mma_supports(C / H))
+        return launch_attention_bwd_simt(qkv, o, o_lo, lse, d_o, B, T, C, H, dqkv, dqkv_hi, dqkv_lo, dvec, s);
+    cudaError_t e = launch_attention_dvec(o, o_lo, d_o, B, T, C, H, dvec, s);
+    if (e != cudaSuccess) return e;
+    return launch_attention_bwd_mma(qkv, lse, d_o, dvec, B, T, C, H, dqkv, dqkv_hi, dqkv_lo, s);
 }
 
 }  // namespace bt

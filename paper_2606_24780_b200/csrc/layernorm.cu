@@ -91,36 +91,46 @@ static inline int ln_bwd_ctas(int64_t N) {
 size_t layernorm_bwd_scratch_floats(int64_t N, int C) { return (size_t)ln_bwd_ctas(N) * 2 * C; }
 
 template <int VPL>
-__global__ void __launch_bounds__(kLnWarps * 32) ln_bwd_kernel(
+__global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     const float* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ gamma,
     const float* __restrict__ mean, const float* __restrict__ rstd, const float* dres, int64_t N, int C4,
     float* dx, float* dx_hi, float* dx_lo, float* __restrict__ partial) {
     extern __shared__ float4 sm[];  // [2][C4]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const float inv_c = 1.0f / (float)(C4 * 4);
-    float4 ag[VPL], ab[VPL], gm[VPL];
+    // Per-lane running sums of dy*xhat and dy for the columns this lane owns.  Only x, dy and
+    // these sums stay in registers (gamma is re-read through L1 each row), which keeps the kernel
+    // at two CTAs per SM.
+    float4 ag[VPL], ab[VPL];
 #pragma unroll
     for (int k = 0; k < VPL; ++k) {
         ag[k] = make_float4(0.f, 0.f, 0.f, 0.f);
         ab[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        int idx = lane + 32 * k;
-        gm[k] = (idx < C4) ? ld4(gamma, idx) : make_float4(0.f, 0.f, 0.f, 0.f);
     }
     for (int64_t row = (int64_t)blockIdx.x * kLnWarps + warp; row < N; row += (int64_t)gridDim.x * kLnWarps) {
         const float mu = mean[row], rs = rstd[row];
-        float4 xh[VPL], dh[VPL];
+        float4 xv[VPL], dv[VPL];
         float s1 = 0.f, s2 = 0.f;
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
             int idx = lane + 32 * k;
             if (idx < C4) {
-                float4 xv = ld4(x, row * C4 + idx), d = ld4(dy, row * C4 + idx);
-                xh[k] = make_float4((xv.x - mu) * rs, (xv.y - mu) * rs, (xv.z - mu) * rs, (xv.w - mu) * rs);
-                dh[k] = make_float4(d.x * gm[k].x, d.y * gm[k].y, d.z * gm[k].z, d.w * gm[k].w);
-                s1 += (dh[k].x + dh[k].y) + (dh[k].z + dh[k].w);
-                s2 += (dh[k].x * xh[k].x + dh[k].y * xh[k].y) + (dh[k].z * xh[k].z + dh[k].w * xh[k].w);
-                ag[k].x += d.x * xh[k].x; ag[k].y += d.y * xh[k].y; ag[k].z += d.z * xh[k].z; ag[k].w += d.w * xh[k].w;
-                ab[k] = add4(ab[k], d);
+                xv[k] = ld4(x, row * C4 + idx);
+                dv[k] = ld4(dy, row * C4 + idx);
+            }
+        }
+#pragma unroll
+        for (int k = 0; k < VPL; ++k) {
+            int idx = lane + 32 * k;
+            if (idx < C4) {
+                const float4 gm = ld4(gamma, idx);
+                xv[k] = make_float4((xv[k].x - mu) * rs, (xv[k].y - mu) * rs, (xv[k].z - mu) * rs, (xv[k].w - mu) * rs);
+                ag[k].x += dv[k].x * xv[k].x; ag[k].y += dv[k].y * xv[k].y;
+                ag[k].z += dv[k].z * xv[k].z; ag[k].w += dv[k].w * xv[k].w;
+                ab[k] = add4(ab[k], dv[k]);
+                dv[k] = make_float4(dv[k].x * gm.x, dv[k].y * gm.y, dv[k].z * gm.z, dv[k].w * gm.w);
+                s1 += (dv[k].x + dv[k].y) + (dv[k].z + dv[k].w);
+                s2 += (dv[k].x * xv[k].x + dv[k].y * xv[k].y) + (dv[k].z * xv[k].z + dv[k].w * xv[k].w);
             }
         }
         s1 = warp_sum(s1) * inv_c;
@@ -130,10 +140,10 @@ __global__ void __launch_bounds__(kLnWarps * 32) ln_bwd_kernel(
             int idx = lane + 32 * k;
             if (idx < C4) {
                 float4 r;
-                r.x = rs * (dh[k].x - s1 - xh[k].x * s2);
-                r.y = rs * (dh[k].y - s1 - xh[k].y * s2);
-                r.z = rs * (dh[k].z - s1 - xh[k].z * s2);
-                r.w = rs * (dh[k].w - s1 - xh[k].w * s2);
+                r.x = rs * (dv[k].x - s1 - xv[k].x * s2);
+                r.y = rs * (dv[k].y - s1 - xv[k].y * s2);
+                r.z = rs * (dv[k].z - s1 - xv[k].z * s2);
+                r.w = rs * (dv[k].w - s1 - xv[k].w * s2);
                 if (dres) r = add4(r, ld4(dres, row * C4 + idx));
                 store_raw_split(r, dx, dx_hi, dx_lo, row * C4 + idx);
             }
