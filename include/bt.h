@@ -216,10 +216,26 @@ BT_API bt_status bt_op_layernorm_bwd(const float* dy, const float* x, const floa
  *   BT_GEMM_NT: A [M,K], B [N,K]   (forward:  Y  = X W^T)
  *   BT_GEMM_NN: A [M,K], B [K,N]   (backward: dX = dY W)
  *   BT_GEMM_TN: A [K,M], B [K,N]   (backward: dW = dY^T X)
- * M, N, K multiples of 4 (NN/TN: the contiguous extents multiples of 32).  A and B are
- * raw FP32; they are split into hi/lo planes in `scratch` first.  flags: BT_FLAG_GEMM_SIMT
- * selects the FP32 FMA reference kernel. */
+ * M, N, K multiples of 4 (NN/TN: the contiguous extents multiples of 32).
+ * flags: BT_FLAG_GEMM_SIMT selects the FP32 FMA reference kernel. */
 enum { BT_GEMM_NT = 0, BT_GEMM_NN = 1, BT_GEMM_TN = 2 };
+
+/* x_split[0][i] = hi(x[i]), x_split[1][i] = lo(x[i]) for n values (n % 4 == 0). */
+BT_API bt_status bt_op_split(const float* x, int64_t n, float* x_split, void* stream);
+
+/* The GEMM as the training step calls it: operands already stored as hi/lo planes
+ * (A_split is [2][rows_A][cols_A], B_split likewise).  Asynchronous; `scratch` (256-byte
+ * aligned, bt_op_gemm_split_scratch_bytes() bytes) holds split-K partial sums and the device
+ * error word that bt_op_gemm_check reads (it synchronises the stream and returns
+ * BT_ERR_DEVICE_TIMEOUT if a bounded wait inside the kernel ran out). */
+BT_API size_t bt_op_gemm_split_scratch_bytes(void);
+BT_API bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
+                                  const float* B_split, float* D, const float* bias, const float* residual,
+                                  void* scratch, size_t scratch_bytes, uint32_t flags, void* stream);
+BT_API bt_status bt_op_gemm_check(const void* scratch, void* stream);
+
+/* Convenience form on raw FP32 operands: bt_op_split of A and B into `scratch`, then
+ * bt_op_gemm_split, then bt_op_gemm_check (synchronises). */
 BT_API size_t bt_op_gemm_scratch_bytes(int32_t layout, int64_t M, int64_t N, int64_t K);
 BT_API bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A, const float* B,
                             float* D, const float* bias, const float* residual, void* scratch,

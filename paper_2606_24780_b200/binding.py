@@ -67,6 +67,10 @@ _SIGNATURES = {
     "bt_op_layernorm_bwd_scratch_bytes": (_sz, [_i64, _i32]),
     "bt_op_layernorm_bwd": (_i32, [_vp] * 6 + [_i64, _i32] + [_vp] * 5 + [_sz, _vp]),
     "bt_op_gemm_scratch_bytes": (_sz, [_i32, _i64, _i64, _i64]),
+    "bt_op_split": (_i32, [_vp, _i64, _vp, _vp]),
+    "bt_op_gemm_split_scratch_bytes": (_sz, []),
+    "bt_op_gemm_split": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
+    "bt_op_gemm_check": (_i32, [_vp, _vp]),
     "bt_op_gemm": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
     "bt_op_attention_fwd": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _u32, _vp]),
     "bt_op_attention_bwd": (_i32, [_vp] * 4 + [_i32] * 4 + [_vp] * 3 + [_sz, _u32, _vp]),
@@ -279,6 +283,24 @@ def bt_op_gemm_scratch_bytes(layout, M, N, K):
 def bt_op_gemm(layout, M, N, K, A, B, D, bias, residual, scratch, scratch_bytes, flags=0, stream=None):
     _check(lib().bt_op_gemm(layout, M, N, K, _ptr(A), _ptr(B), _ptr(D), _ptr(bias), _ptr(residual), _ptr(scratch),
                             scratch_bytes, flags, _stream(stream)))
+
+
+def bt_op_split(x, n, x_split, stream=None):
+    _check(lib().bt_op_split(_ptr(x), n, _ptr(x_split), _stream(stream)))
+
+
+def bt_op_gemm_split_scratch_bytes():
+    return int(lib().bt_op_gemm_split_scratch_bytes())
+
+
+def bt_op_gemm_split(layout, M, N, K, A_split, B_split, D, bias, residual, scratch, scratch_bytes, flags=0,
+                     stream=None):
+    _check(lib().bt_op_gemm_split(layout, M, N, K, _ptr(A_split), _ptr(B_split), _ptr(D), _ptr(bias), _ptr(residual),
+                                  _ptr(scratch), scratch_bytes, flags, _stream(stream)))
+
+
+def bt_op_gemm_check(scratch, stream=None):
+    _check(lib().bt_op_gemm_check(_ptr(scratch), _stream(stream)))
 
 
 def bt_op_attention_fwd(qkv, B, T, C, H, o, o_split, lse, flags=0, stream=None):

@@ -688,32 +688,38 @@ GemmShapes gemm_shapes(int layout, int64_t M, int64_t N, int64_t K) {
 inline size_t pad256(size_t n) { return (n + 63) / 64 * 64; }  // floats
 }  // namespace
 
+extern "C" size_t bt_op_gemm_split_scratch_bytes(void) {
+    return (gemm_tc_partial_floats_bound() + 64) * sizeof(float);
+}
+
 extern "C" size_t bt_op_gemm_scratch_bytes(int32_t layout, int64_t M, int64_t N, int64_t K) {
     if (layout < 0 || layout > 2 || M < 1 || N < 1 || K < 1) return 0;
     GemmShapes s = gemm_shapes(layout, M, N, K);
-    return (pad256(2 * s.a_rows * s.a_cols) + pad256(2 * s.b_rows * s.b_cols) + gemm_tc_partial_floats_bound() + 64) *
-           sizeof(float);
+    return (pad256(2 * s.a_rows * s.a_cols) + pad256(2 * s.b_rows * s.b_cols)) * sizeof(float) +
+           bt_op_gemm_split_scratch_bytes();
 }
 
-extern "C" bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A, const float* B,
-                                float* D, const float* bias, const float* residual, void* scratch,
-                                size_t scratch_bytes, uint32_t flags, void* stream) {
-    BT_PTR(A); BT_PTR(B); BT_PTR(D); BT_OPT_PTR(bias); BT_OPT_PTR(residual); BT_PTR(scratch);
+extern "C" bt_status bt_op_split(const float* x, int64_t n, float* x_split, void* stream) {
+    BT_PTR(x); BT_PTR(x_split);
+    if (n < 0 || n % 4) return fail(BT_ERR_INVALID_ARG, "split: n must be a non-negative multiple of 4");
+    if (n == 0) return BT_OK;
+    BT_CUDA(launch_split(x, x_split, x_split + n, n, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
+                                      const float* B_split, float* D, const float* bias, const float* residual,
+                                      void* scratch, size_t scratch_bytes, uint32_t flags, void* stream) {
+    BT_PTR(A_split); BT_PTR(B_split); BT_PTR(D); BT_OPT_PTR(bias); BT_OPT_PTR(residual); BT_PTR(scratch);
     if (layout < 0 || layout > 2) return fail(BT_ERR_INVALID_ARG, "gemm: layout %d", layout);
     if (M < 1 || N < 1 || K < 1 || M % 4 || N % 4 || K % 4) return fail(BT_ERR_INVALID_ARG, "gemm: M, N, K must be positive multiples of 4");
     if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return fail(BT_ERR_INVALID_ARG, "gemm: size too large");
-    if (scratch_bytes < bt_op_gemm_scratch_bytes(layout, M, N, K)) return fail(BT_ERR_OOM, "gemm: scratch too small");
+    if (scratch_bytes < bt_op_gemm_split_scratch_bytes()) return fail(BT_ERR_OOM, "gemm: scratch too small");
     if (reinterpret_cast<uintptr_t>(scratch) & 255u) return fail(BT_ERR_INVALID_ARG, "gemm: scratch not 256-byte aligned");
     cudaStream_t s = (cudaStream_t)stream;
     GemmShapes sh = gemm_shapes(layout, M, N, K);
-    float* a_s = (float*)scratch;
-    float* b_s = a_s + pad256(2 * sh.a_rows * sh.a_cols);
-    float* partials = b_s + pad256(2 * sh.b_rows * sh.b_cols);
-    int* err = (int*)(partials + gemm_tc_partial_floats_bound());
     const int64_t na = sh.a_rows * sh.a_cols, nb = sh.b_rows * sh.b_cols;
-    BT_CUDA(launch_split(A, a_s, a_s + na, na, s));
-    BT_CUDA(launch_split(B, b_s, b_s + nb, nb, s));
-    SplitMat Am{a_s, na, sh.a_rows, sh.a_cols, sh.a_cols}, Bm{b_s, nb, sh.b_rows, sh.b_cols, sh.b_cols};
+    SplitMat Am{A_split, na, sh.a_rows, sh.a_cols, sh.a_cols}, Bm{B_split, nb, sh.b_rows, sh.b_cols, sh.b_cols};
     if (flags & BT_FLAG_GEMM_SIMT) {
         BT_CUDA(launch_gemm_simt(layout, M, N, K, Am, Bm, D, N, bias, residual, s));
         return BT_OK;
@@ -722,13 +728,44 @@ extern "C" bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K,
         return fail(BT_ERR_UNSUPPORTED, "gemm: transposed operands need their contiguous extent to be a multiple of 32");
     char msg[256];
     if (!gemm_tc_init(msg, sizeof(msg))) return fail(BT_ERR_CUDA, "tensor-core GEMM unavailable: %s", msg);
+    float* partials = (float*)scratch;
+    int* err = (int*)(partials + gemm_tc_partial_floats_bound());
     BT_CUDA(cudaMemsetAsync(err, 0, sizeof(int), s));
     BT_CUDA(launch_gemm_tc(layout, M, N, K, Am, Bm, D, N, bias, residual, partials, gemm_tc_partial_floats_bound(), err, s));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_gemm_check(const void* scratch, void* stream) {
+    BT_PTR(scratch);
+    const int* err = (const int*)((const float*)scratch + gemm_tc_partial_floats_bound());
     int herr = 0;
-    BT_CUDA(cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, s));
-    BT_CUDA(cudaStreamSynchronize(s));
+    BT_CUDA(cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+    BT_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
     if (herr) return fail(BT_ERR_DEVICE_TIMEOUT, "gemm: a bounded device-side wait ran out (code %d)", herr);
     return BT_OK;
+}
+
+extern "C" bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A, const float* B,
+                                float* D, const float* bias, const float* residual, void* scratch,
+                                size_t scratch_bytes, uint32_t flags, void* stream) {
+    BT_PTR(A); BT_PTR(B); BT_PTR(scratch);
+    if (layout < 0 || layout > 2) return fail(BT_ERR_INVALID_ARG, "gemm: layout %d", layout);
+    if (M < 1 || N < 1 || K < 1 || M % 4 || N % 4 || K % 4) return fail(BT_ERR_INVALID_ARG, "gemm: M, N, K must be positive multiples of 4");
+    if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return fail(BT_ERR_INVALID_ARG, "gemm: size too large");
+    if (scratch_bytes < bt_op_gemm_scratch_bytes(layout, M, N, K)) return fail(BT_ERR_OOM, "gemm: scratch too small");
+    if (reinterpret_cast<uintptr_t>(scratch) & 255u) return fail(BT_ERR_INVALID_ARG, "gemm: scratch not 256-byte aligned");
+    GemmShapes sh = gemm_shapes(layout, M, N, K);
+    float* a_s = (float*)scratch;
+    float* b_s = a_s + pad256(2 * sh.a_rows * sh.a_cols);
+    float* rest = b_s + pad256(2 * sh.b_rows * sh.b_cols);
+    bt_status st = bt_op_split(A, sh.a_rows * sh.a_cols, a_s, stream);
+    if (st == BT_OK) st = bt_op_split(B, sh.b_rows * sh.b_cols, b_s, stream);
+    if (st == BT_OK)
+        st = bt_op_gemm_split(layout, M, N, K, a_s, b_s, D, bias, residual, rest, bt_op_gemm_split_scratch_bytes(), flags,
+                              stream);
+    if (st != BT_OK) return st;
+    if (flags & BT_FLAG_GEMM_SIMT) return BT_OK;
+    return bt_op_gemm_check(rest, stream);
 }
 
 extern "C" bt_status bt_op_attention_fwd(const float* qkv, int32_t B, int32_t T, int32_t C, int32_t H, float* o,

@@ -2,9 +2,10 @@
 //
 // Every product (Q K^T, P V, dO V^T, dS K, dS^T Q, P^T dO) is a warp-level m16n8k8 TF32
 // tensor-core MMA evaluated three times on hi/lo splits (a_lo*b_hi + a_hi*b_lo + a_hi*b_hi,
-// FP32 accumulate).  K/V (or Q/dO) tiles are split once while being staged into shared memory
-// (row stride head_dim + 4 floats: both fragment access patterns are bank-conflict free);
-// per-warp operands are split in registers.  The softmax is the online (running max / running
+// FP32 accumulate).  The streamed tiles (K/V in the forward and dq kernels, Q/dO in the dkv kernel)
+// are copied raw into double-buffered shared memory with cp.async while the previous tile is
+// being consumed (row stride head_dim + 4 floats: both fragment access patterns are bank-conflict
+// free); their fragments are split into hi/lo in registers, as are the per-warp operands.  The softmax is the online (running max / running
 // sum) form in base 2 with the 1/sqrt(d) log2(e) factor folded into Q; row reductions are
 // warp shuffles inside the 4-lane quad that owns a row.
 //
@@ -59,6 +60,25 @@ __device__ __forceinline__ void stage_split(const float* __restrict__ src, int64
     }
 }
 
+// Asynchronously copies ROWS rows x HD floats (global row stride `gstride`; rows past the end are
+// clamped to the last valid row, their results are masked or never stored) into a raw FP32
+// shared tile with row stride HD + 4.  One cp.async group per call.
+template <int HD, int ROWS, int NT>
+__device__ __forceinline__ void stage_raw_async(const float* __restrict__ src, int64_t gstride, int row0, int nvalid,
+                                                float* __restrict__ dst) {
+    constexpr int LDS = HD + 4, V4 = HD / 4;
+    for (int idx = threadIdx.x; idx < ROWS * V4; idx += NT) {
+        const int r = idx / V4, c4 = idx - r * V4;
+        const int gr = min(row0 + r, nvalid - 1);
+        const uint32_t d = (uint32_t)__cvta_generic_to_shared(dst + r * LDS + c4 * 4);
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d), "l"(src + (int64_t)gr * gstride + c4 * 4)
+                     : "memory");
+    }
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
+
 // A fragment (16 rows x 8 k) of a shared hi/lo tile: rows row16 + g (+8), columns k0 + t4 (+4).
 template <int LDS>
 __device__ __forceinline__ void load_a_frag(const float* s_hi, const float* s_lo, int row16, int k0, int g, int t4,
@@ -70,38 +90,53 @@ __device__ __forceinline__ void load_a_frag(const float* s_hi, const float* s_lo
     a_hi[3] = __float_as_uint(s_hi[o1 + 4]); a_lo[3] = __float_as_uint(s_lo[o1 + 4]);
 }
 
-// acc[nt] (16 x 8 tiles over the 64 tile rows) += A(16 x HD) . X^T, X a shared tile [64][HD]:
-// B fragment element (k, n) = X[n0 + n][k0 + k].
+// acc[nt] (16 x 8 tiles over the 64 tile rows) += A(16 x 8 k-slice ks) . X^T, X a RAW shared tile
+// [64][HD]: B fragment element (k, n) = X[n0 + n][k0 + k], split into hi/lo in registers.  The
+// three TF32 terms are issued term-major so that consecutive MMAs hit different accumulators.
 template <int HD>
 __device__ __forceinline__ void mma_a_xT(float (&acc)[8][4], const uint32_t (&a_hi)[4], const uint32_t (&a_lo)[4],
-                                         const float* x_hi, const float* x_lo, int ks, int g, int t4) {
+                                         const float* x, int ks, int g, int t4) {
     constexpr int LDS = HD + 4;
+    uint32_t bh0[8], bh1[8], bl0[8], bl1[8];
 #pragma unroll
     for (int nt = 0; nt < 8; ++nt) {
         const int o = (nt * 8 + g) * LDS + ks * 8 + t4;
-        mma3(acc[nt], a_hi, a_lo, __float_as_uint(x_hi[o]), __float_as_uint(x_hi[o + 4]), __float_as_uint(x_lo[o]),
-             __float_as_uint(x_lo[o + 4]));
+        split_u(x[o], bh0[nt], bl0[nt]);
+        split_u(x[o + 4], bh1[nt], bl1[nt]);
     }
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) mma_tf32(acc[nt], a_lo, bh0[nt], bh1[nt]);
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) mma_tf32(acc[nt], a_hi, bl0[nt], bl1[nt]);
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) mma_tf32(acc[nt], a_hi, bh0[nt], bh1[nt]);
 }
 
-// acc[dt] (16 x 8 tiles over HD) += P(16 x 8 slice nt of a 16 x 64 C-layout tile) . X, X a shared
-// tile [64][HD].  The C-fragment columns 2*t4, 2*t4+1 serve as the A-fragment k indices t4, t4+4,
-// so B fragment element (k = t4 | t4+4, n) = X[nt*8 + 2*t4 | 2*t4+1][n0 + n].
+// acc[dt] (16 x 8 tiles over HD) += P(16 x 8 slice nt of a 16 x 64 C-layout tile) . X, X a RAW
+// shared tile [64][HD].  The C-fragment columns 2*t4, 2*t4+1 serve as the A-fragment k indices
+// t4, t4+4, so B fragment element (k = t4 | t4+4, n) = X[nt*8 + 2*t4 | 2*t4+1][n0 + n].
 template <int HD>
-__device__ __forceinline__ void mma_p_x(float (&acc)[HD / 8][4], const float (&p)[4], const float* x_hi,
-                                        const float* x_lo, int nt, int g, int t4) {
-    constexpr int LDS = HD + 4;
+__device__ __forceinline__ void mma_p_x(float (&acc)[HD / 8][4], const float (&p)[4], const float* x, int nt, int g,
+                                        int t4) {
+    constexpr int LDS = HD + 4, KS = HD / 8;
     uint32_t a_hi[4], a_lo[4];
     split_u(p[0], a_hi[0], a_lo[0]);
     split_u(p[2], a_hi[1], a_lo[1]);
     split_u(p[1], a_hi[2], a_lo[2]);
     split_u(p[3], a_hi[3], a_lo[3]);
+    uint32_t bh0[KS], bh1[KS], bl0[KS], bl1[KS];
 #pragma unroll
-    for (int dt = 0; dt < HD / 8; ++dt) {
+    for (int dt = 0; dt < KS; ++dt) {
         const int o = (nt * 8 + 2 * t4) * LDS + dt * 8 + g;
-        mma3(acc[dt], a_hi, a_lo, __float_as_uint(x_hi[o]), __float_as_uint(x_hi[o + LDS]),
-             __float_as_uint(x_lo[o]), __float_as_uint(x_lo[o + LDS]));
+        split_u(x[o], bh0[dt], bl0[dt]);
+        split_u(x[o + LDS], bh1[dt], bl1[dt]);
     }
+#pragma unroll
+    for (int dt = 0; dt < KS; ++dt) mma_tf32(acc[dt], a_lo, bh0[dt], bh1[dt]);
+#pragma unroll
+    for (int dt = 0; dt < KS; ++dt) mma_tf32(acc[dt], a_hi, bl0[dt], bl1[dt]);
+#pragma unroll
+    for (int dt = 0; dt < KS; ++dt) mma_tf32(acc[dt], a_hi, bh0[dt], bh1[dt]);
 }
 
 __device__ __forceinline__ float quad_max(float v) {
@@ -132,12 +167,11 @@ __device__ __forceinline__ void load_q_frags(const float* __restrict__ base, int
 // ------------------------------------------------------------------ forward
 
 template <int HD>
-__global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const float* __restrict__ qkv, int T, int C, int H,
-                                                           float* o, float* o_hi, float* o_lo,
-                                                           float* __restrict__ lse) {
+__global__ void __launch_bounds__(128, 2) attn_fwd_mma_kernel(const float* __restrict__ qkv, int T, int C, int H,
+                                                              float* o, float* o_hi, float* o_lo,
+                                                              float* __restrict__ lse) {
     constexpr int LDS = HD + 4, KS = HD / 8, TILE = 64 * LDS;
-    extern __shared__ float sm[];
-    float *k_hi = sm, *k_lo = sm + TILE, *v_hi = sm + 2 * TILE, *v_lo = sm + 3 * TILE;
+    extern __shared__ float sm[];  // K[2], V[2] raw tiles (double buffered)
     const int qt = gridDim.x - 1 - blockIdx.x;
     const int b = blockIdx.y / H, h = blockIdx.y % H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
@@ -145,6 +179,10 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const float* __restri
     const float* base = qkv + (int64_t)b * T * gs + h * HD;
     const int r0 = qt * 64 + warp * 16 + g, r1 = r0 + 8;
     const float qmul = kLog2e / sqrtf((float)HD);
+
+    stage_raw_async<HD, 64, 128>(base + C, gs, 0, T, sm);
+    stage_raw_async<HD, 64, 128>(base + 2 * C, gs, 0, T, sm + 2 * TILE);
+    cp_async_commit();
 
     uint32_t q_hi[KS][4], q_lo[KS][4];
     load_q_frags<HD>(base, gs, r0, r1, T, qmul, t4, q_hi, q_lo);
@@ -155,15 +193,23 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const float* __restri
     float m0 = -INFINITY, m1 = -INFINITY, l0 = 0.f, l1 = 0.f;
 
     for (int kt = 0; kt <= qt; ++kt) {
+        const int buf = kt & 1;
+        if (kt < qt) {  // prefetch the next tile into the other buffer
+            stage_raw_async<HD, 64, 128>(base + C, gs, (kt + 1) * 64, T, sm + (buf ^ 1) * TILE);
+            stage_raw_async<HD, 64, 128>(base + 2 * C, gs, (kt + 1) * 64, T, sm + (2 + (buf ^ 1)) * TILE);
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
         __syncthreads();
-        stage_split<HD, 64, 128>(base + C, gs, kt * 64, T, 1.0f, k_hi, k_lo);
-        stage_split<HD, 64, 128>(base + 2 * C, gs, kt * 64, T, 1.0f, v_hi, v_lo);
-        __syncthreads();
+        const float* k_s = sm + buf * TILE;
+        const float* v_s = sm + (2 + buf) * TILE;
         float s[8][4];
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
 #pragma unroll
-        for (int ks = 0; ks < KS; ++ks) mma_a_xT<HD>(s, q_hi[ks], q_lo[ks], k_hi, k_lo, ks, g, t4);
+        for (int ks = 0; ks < KS; ++ks) mma_a_xT<HD>(s, q_hi[ks], q_lo[ks], k_s, ks, g, t4);
         if (kt == qt) {
 #pragma unroll
             for (int nt = 0; nt < 8; ++nt) {
@@ -195,8 +241,9 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const float* __restri
             p[2] = exp2f(s[nt][2] - mn1); p[3] = exp2f(s[nt][3] - mn1);
             l0 += p[0] + p[1];
             l1 += p[2] + p[3];
-            mma_p_x<HD>(acc, p, v_hi, v_lo, nt, g, t4);
+            mma_p_x<HD>(acc, p, v_s, nt, g, t4);
         }
+        __syncthreads();  // everyone is done with this buffer before it is refilled
     }
     l0 = quad_sum(l0);
     l1 = quad_sum(l1);
@@ -205,21 +252,13 @@ __global__ void __launch_bounds__(128) attn_fwd_mma_kernel(const float* __restri
 #pragma unroll
     for (int dt = 0; dt < KS; ++dt) {
         const int col = dt * 8 + 2 * t4;
-        if (r0 < T) {
-            float2 v = make_float2(acc[dt][0] * i0, acc[dt][1] * i0);
-            const int64_t off = ob + (int64_t)r0 * C + col;
-            if (o) *reinterpret_cast<float2*>(o + off) = v;
-            if (o_hi) {
-                float2 hh, ll;
-                split_tf32(v.x, hh.x, ll.x);
-                split_tf32(v.y, hh.y, ll.y);
-                *reinterpret_cast<float2*>(o_hi + off) = hh;
-                *reinterpret_cast<float2*>(o_lo + off) = ll;
-            }
-        }
-        if (r1 < T) {
-            float2 v = make_float2(acc[dt][2] * i1, acc[dt][3] * i1);
-            const int64_t off = ob + (int64_t)r1 * C + col;
+#pragma unroll
+        for (int half = 0; half < 2; ++half) {
+            const int r = half ? r1 : r0;
+            if (r >= T) continue;
+            const float inv = half ? i1 : i0;
+            float2 v = make_float2(acc[dt][2 * half] * inv, acc[dt][2 * half + 1] * inv);
+            const int64_t off = ob + (int64_t)r * C + col;
             if (o) *reinterpret_cast<float2*>(o + off) = v;
             if (o_hi) {
                 float2 hh, ll;
@@ -246,9 +285,8 @@ __global__ void __launch_bounds__(128, 2) attn_bwd_dq_mma_kernel(const float* __
                                                                  const float* __restrict__ dvec, int T, int C, int H,
                                                                  float* dqkv, float* dqkv_hi, float* dqkv_lo) {
     constexpr int LDS = HD + 4, KS = HD / 8, TILE = 64 * LDS;
-    extern __shared__ float sm[];
-    float *k_hi = sm, *k_lo = sm + TILE, *v_hi = sm + 2 * TILE, *v_lo = sm + 3 * TILE, *do_hi = sm + 4 * TILE,
-          *do_lo = sm + 5 * TILE;
+    extern __shared__ float sm[];  // K[2], V[2] raw (double buffered), dO hi, dO lo
+    float *do_hi = sm + 4 * TILE, *do_lo = sm + 5 * TILE;
     const int qt = gridDim.x - 1 - blockIdx.x;
     const int b = blockIdx.y / H, h = blockIdx.y % H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
@@ -256,6 +294,10 @@ __global__ void __launch_bounds__(128, 2) attn_bwd_dq_mma_kernel(const float* __
     const float* base = qkv + (int64_t)b * T * gs + h * HD;
     const int r0 = qt * 64 + warp * 16 + g, r1 = r0 + 8;
     const float scale = 1.0f / sqrtf((float)HD);
+
+    stage_raw_async<HD, 64, 128>(base + C, gs, 0, T, sm);
+    stage_raw_async<HD, 64, 128>(base + 2 * C, gs, 0, T, sm + 2 * TILE);
+    cp_async_commit();
 
     uint32_t q_hi[KS][4], q_lo[KS][4];
     load_q_frags<HD>(base, gs, r0, r1, T, scale * kLog2e, t4, q_hi, q_lo);
@@ -269,10 +311,18 @@ __global__ void __launch_bounds__(128, 2) attn_bwd_dq_mma_kernel(const float* __
     for (int dt = 0; dt < KS; ++dt) dq[dt][0] = dq[dt][1] = dq[dt][2] = dq[dt][3] = 0.f;
 
     for (int kt = 0; kt <= qt; ++kt) {
+        const int buf = kt & 1;
+        if (kt < qt) {
+            stage_raw_async<HD, 64, 128>(base + C, gs, (kt + 1) * 64, T, sm + (buf ^ 1) * TILE);
+            stage_raw_async<HD, 64, 128>(base + 2 * C, gs, (kt + 1) * 64, T, sm + (2 + (buf ^ 1)) * TILE);
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
+        }
         __syncthreads();
-        stage_split<HD, 64, 128>(base + C, gs, kt * 64, T, 1.0f, k_hi, k_lo);
-        stage_split<HD, 64, 128>(base + 2 * C, gs, kt * 64, T, 1.0f, v_hi, v_lo);
-        __syncthreads();
+        const float* k_s = sm + buf * TILE;
+        const float* v_s = sm + (2 + buf) * TILE;
         float s[8][4], dp[8][4];
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
@@ -281,10 +331,10 @@ __global__ void __launch_bounds__(128, 2) attn_bwd_dq_mma_kernel(const float* __
         }
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
-            mma_a_xT<HD>(s, q_hi[ks], q_lo[ks], k_hi, k_lo, ks, g, t4);
+            mma_a_xT<HD>(s, q_hi[ks], q_lo[ks], k_s, ks, g, t4);
             uint32_t a_hi[4], a_lo[4];
             load_a_frag<LDS>(do_hi, do_lo, warp * 16, ks * 8, g, t4, a_hi, a_lo);
-            mma_a_xT<HD>(dp, a_hi, a_lo, v_hi, v_lo, ks, g, t4);
+            mma_a_xT<HD>(dp, a_hi, a_lo, v_s, ks, g, t4);
         }
 #pragma unroll
         for (int nt = 0; nt < 8; ++nt) {
@@ -299,8 +349,9 @@ __global__ void __launch_bounds__(128, 2) attn_bwd_dq_mma_kernel(const float* __
             ds[1] = p[1] * (dp[nt][1] - D0);
             ds[2] = p[2] * (dp[nt][2] - D1);
             ds[3] = p[3] * (dp[nt][3] - D1);
-            mma_p_x<HD>(dq, ds, k_hi, k_lo, nt, g, t4);
+            mma_p_x<HD>(dq, ds, k_s, nt, g, t4);
         }
+        __syncthreads();
     }
     const int64_t ob = ((int64_t)b * T) * gs + h * HD;
 #pragma unroll
@@ -334,9 +385,11 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_mma_kernel(const float* __re
                                                                float* dqkv, float* dqkv_hi, float* dqkv_lo) {
     constexpr int LDS = HD + 4, KS = HD / 8, KT = 128 * LDS, QT = 64 * LDS;
     extern __shared__ float sm[];
+    // K', V of this CTA's 128 keys as hi/lo (A operands); Q[2], dO[2] raw query tiles (double
+    // buffered B operands); lse[2][64], D[2][64].
     float *k_hi = sm, *k_lo = sm + KT, *v_hi = sm + 2 * KT, *v_lo = sm + 3 * KT;
-    float *q_hi = sm + 4 * KT, *q_lo = q_hi + QT, *do_hi = q_hi + 2 * QT, *do_lo = q_hi + 3 * QT;
-    float *lse_s = q_hi + 4 * QT, *d_s = lse_s + 64;
+    float *q_raw = sm + 4 * KT, *do_raw = q_raw + 2 * QT;
+    float *lse_s = q_raw + 4 * QT, *d_s = lse_s + 128;
     const int j0 = blockIdx.x * 128;
     const int b = blockIdx.y / H, h = blockIdx.y % H;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, g = lane >> 2, t4 = lane & 3;
@@ -347,7 +400,11 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_mma_kernel(const float* __re
     const float scale = 1.0f / sqrtf((float)HD);
     const int jw = j0 + warp * 16;             // first key of this warp
     const int jr0 = jw + g, jr1 = jr0 + 8;     // the two key rows of this thread
+    const int n_qt = (T + 63) / 64, qt0 = j0 / 64;
 
+    stage_raw_async<HD, 64, 256>(base, gs, qt0 * 64, T, q_raw);
+    stage_raw_async<HD, 64, 256>(dob, C, qt0 * 64, T, do_raw);
+    cp_async_commit();
     // K is staged pre-multiplied by scale*log2(e) (it only feeds the score recomputation)
     stage_split<HD, 128, 256>(base + C, gs, j0, T, scale * kLog2e, k_hi, k_lo);
     stage_split<HD, 128, 256>(base + 2 * C, gs, j0, T, 1.0f, v_hi, v_lo);
@@ -358,51 +415,60 @@ __global__ void __launch_bounds__(256) attn_bwd_dkv_mma_kernel(const float* __re
         dk[dt][0] = dk[dt][1] = dk[dt][2] = dk[dt][3] = 0.f;
         dv[dt][0] = dv[dt][1] = dv[dt][2] = dv[dt][3] = 0.f;
     }
-    const int n_qt = (T + 63) / 64;
-    for (int qt = j0 / 64; qt < n_qt; ++qt) {
-        const int q0 = qt * 64;
-        __syncthreads();
-        stage_split<HD, 64, 256>(base, gs, q0, T, 1.0f, q_hi, q_lo);
-        stage_split<HD, 64, 256>(dob, C, q0, T, 1.0f, do_hi, do_lo);
+    for (int qt = qt0; qt < n_qt; ++qt) {
+        const int q0 = qt * 64, buf = (qt - qt0) & 1;
         if (threadIdx.x < 64) {
             const int r = q0 + threadIdx.x;
-            lse_s[threadIdx.x] = (r < T) ? lse[lb + r] * kLog2e : INFINITY;
-            d_s[threadIdx.x] = (r < T) ? dvec[lb + r] : 0.f;
+            lse_s[buf * 64 + threadIdx.x] = (r < T) ? lse[lb + r] * kLog2e : INFINITY;
+            d_s[buf * 64 + threadIdx.x] = (r < T) ? dvec[lb + r] : 0.f;
+        }
+        if (qt + 1 < n_qt) {
+            stage_raw_async<HD, 64, 256>(base, gs, q0 + 64, T, q_raw + (buf ^ 1) * QT);
+            stage_raw_async<HD, 64, 256>(dob, C, q0 + 64, T, do_raw + (buf ^ 1) * QT);
+            cp_async_commit();
+            cp_async_wait<1>();
+        } else {
+            cp_async_wait<0>();
         }
         __syncthreads();
-        if (q0 + 63 < jw) continue;  // every query row of this tile precedes this warp's keys
-        float s[8][4], dp[8][4];
+        if (q0 + 63 >= jw) {  // otherwise every query row of this tile precedes this warp's keys
+            const float* q_s = q_raw + buf * QT;
+            const float* do_s = do_raw + buf * QT;
+            float s[8][4], dp[8][4];
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
-            dp[nt][0] = dp[nt][1] = dp[nt][2] = dp[nt][3] = 0.f;
-        }
+            for (int nt = 0; nt < 8; ++nt) {
+                s[nt][0] = s[nt][1] = s[nt][2] = s[nt][3] = 0.f;
+                dp[nt][0] = dp[nt][1] = dp[nt][2] = dp[nt][3] = 0.f;
+            }
 #pragma unroll
-        for (int ks = 0; ks < KS; ++ks) {
-            uint32_t a_hi[4], a_lo[4];
-            load_a_frag<LDS>(k_hi, k_lo, warp * 16, ks * 8, g, t4, a_hi, a_lo);
-            mma_a_xT<HD>(s, a_hi, a_lo, q_hi, q_lo, ks, g, t4);       // S^T = K Q^T
-            load_a_frag<LDS>(v_hi, v_lo, warp * 16, ks * 8, g, t4, a_hi, a_lo);
-            mma_a_xT<HD>(dp, a_hi, a_lo, do_hi, do_lo, ks, g, t4);    // dP^T = V dO^T
-        }
+            for (int ks = 0; ks < KS; ++ks) {
+                uint32_t a_hi[4], a_lo[4];
+                load_a_frag<LDS>(k_hi, k_lo, warp * 16, ks * 8, g, t4, a_hi, a_lo);
+                mma_a_xT<HD>(s, a_hi, a_lo, q_s, ks, g, t4);       // S^T = K Q^T
+                load_a_frag<LDS>(v_hi, v_lo, warp * 16, ks * 8, g, t4, a_hi, a_lo);
+                mma_a_xT<HD>(dp, a_hi, a_lo, do_s, ks, g, t4);     // dP^T = V dO^T
+            }
 #pragma unroll
-        for (int nt = 0; nt < 8; ++nt) {
-            const int ci = nt * 8 + 2 * t4;      // query row (column of S^T) inside the tile
-            const int i = q0 + ci;
-            const float La = lse_s[ci], Lb = lse_s[ci + 1], Da = d_s[ci], Db = d_s[ci + 1];
-            float p[4];
-            p[0] = (i < jr0) ? 0.f : exp2f(s[nt][0] - La);
-            p[1] = (i + 1 < jr0) ? 0.f : exp2f(s[nt][1] - Lb);
-            p[2] = (i < jr1) ? 0.f : exp2f(s[nt][2] - La);
-            p[3] = (i + 1 < jr1) ? 0.f : exp2f(s[nt][3] - Lb);
-            mma_p_x<HD>(dv, p, do_hi, do_lo, nt, g, t4);              // dV += P^T dO
-            float ds[4];
-            ds[0] = p[0] * (dp[nt][0] - Da);
-            ds[1] = p[1] * (dp[nt][1] - Db);
-            ds[2] = p[2] * (dp[nt][2] - Da);
-            ds[3] = p[3] * (dp[nt][3] - Db);
-            mma_p_x<HD>(dk, ds, q_hi, q_lo, nt, g, t4);               // dK += dS^T Q
+            for (int nt = 0; nt < 8; ++nt) {
+                const int ci = nt * 8 + 2 * t4;      // query row (column of S^T) inside the tile
+                const int i = q0 + ci;
+                const float La = lse_s[buf * 64 + ci], Lb = lse_s[buf * 64 + ci + 1];
+                const float Da = d_s[buf * 64 + ci], Db = d_s[buf * 64 + ci + 1];
+                float p[4];
+                p[0] = (i < jr0) ? 0.f : exp2f(s[nt][0] - La);
+                p[1] = (i + 1 < jr0) ? 0.f : exp2f(s[nt][1] - Lb);
+                p[2] = (i < jr1) ? 0.f : exp2f(s[nt][2] - La);
+                p[3] = (i + 1 < jr1) ? 0.f : exp2f(s[nt][3] - Lb);
+                mma_p_x<HD>(dv, p, do_s, nt, g, t4);               // dV += P^T dO
+                float ds[4];
+                ds[0] = p[0] * (dp[nt][0] - Da);
+                ds[1] = p[1] * (dp[nt][1] - Db);
+                ds[2] = p[2] * (dp[nt][2] - Da);
+                ds[3] = p[3] * (dp[nt][3] - Db);
+                mma_p_x<HD>(dk, ds, q_s, nt, g, t4);               // dK += dS^T Q
+            }
         }
+        __syncthreads();
     }
     const int64_t ob = ((int64_t)b * T) * gs + h * HD;
 #pragma unroll
@@ -439,7 +505,7 @@ constexpr size_t fwd_smem() { return (size_t)4 * 64 * (HD + 4) * sizeof(float); 
 template <int HD>
 constexpr size_t dq_smem() { return (size_t)6 * 64 * (HD + 4) * sizeof(float); }
 template <int HD>
-constexpr size_t dkv_smem() { return ((size_t)4 * 128 * (HD + 4) + 4 * 64 * (HD + 4) + 128) * sizeof(float); }
+constexpr size_t dkv_smem() { return ((size_t)4 * 128 * (HD + 4) + 4 * 64 * (HD + 4) + 256) * sizeof(float); }
 
 template <int HD>
 cudaError_t set_attrs() {

@@ -202,7 +202,7 @@ cudaError_t launch_gelu_bwd(const float* x, const float* dy, int64_t n, int tanh
 // warp order.  Stage 2 adds the strips in strip order.
 static inline int colsum_strips(int64_t N, int C) {
     int cblocks = (C + 127) / 128;
-    int64_t strips = (2 * 148 + cblocks - 1) / cblocks;
+    int64_t strips = (4 * 148 + cblocks - 1) / cblocks;
     int64_t max_strips = (N + 63) / 64;
     if (strips > max_strips) strips = max_strips;
     if (strips < 1) strips = 1;
@@ -220,7 +220,19 @@ __global__ void __launch_bounds__(256) colsum_stage1_kernel(const float* __restr
     const int64_t r0 = st * rows_per, r1 = (r0 + rows_per < N) ? r0 + rows_per : N;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
     if (c < C4) {
-        for (int64_t r = r0 + warp; r < r1; r += 8) {
+        int64_t r = r0 + warp;
+        for (; r + 24 < r1; r += 32) {  // four rows in flight per lane
+            float4 v0 = ld4(x, r * C4 + c), v1 = ld4(x, (r + 8) * C4 + c), v2 = ld4(x, (r + 16) * C4 + c),
+                   v3 = ld4(x, (r + 24) * C4 + c);
+            if (x_lo) {
+                v0 = add4(v0, ld4(x_lo, r * C4 + c));
+                v1 = add4(v1, ld4(x_lo, (r + 8) * C4 + c));
+                v2 = add4(v2, ld4(x_lo, (r + 16) * C4 + c));
+                v3 = add4(v3, ld4(x_lo, (r + 24) * C4 + c));
+            }
+            acc = add4(add4(add4(add4(acc, v0), v1), v2), v3);
+        }
+        for (; r < r1; r += 8) {
             float4 v = ld4(x, r * C4 + c);
             if (x_lo) v = add4(v, ld4(x_lo, r * C4 + c));
             acc = add4(acc, v);

@@ -28,6 +28,7 @@
 #include <cuda.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <mutex>
 
 #include "common.cuh"
@@ -37,17 +38,21 @@ namespace bt {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BK = 32;            // floats per k-block = one 128-byte swizzle row
 constexpr int kThreads = 192;
 constexpr int kEpiWarps = 4;
-constexpr uint32_t kATileBytes = 2u * BM * BK * 4u;  // hi + lo
+constexpr uint32_t kSmemBudget = 227u * 1024u;
 
-template <int BN>
+// BN: tile width (128, 192 or 256).  BK: floats per k-block; 32 = one 128-byte swizzle row,
+// 16 = one 64-byte swizzle row (smaller stages, deeper ring).
+template <int BN, int BK>
 struct Cfg {
+    static constexpr uint32_t kATileBytes = 2u * BM * BK * 4u;  // hi + lo
     static constexpr uint32_t kBTileBytes = 2u * BN * BK * 4u;
     static constexpr uint32_t kStageBytes = kATileBytes + kBTileBytes;
-    static constexpr int kStages = (BN == 256) ? 2 : 3;
-    static constexpr uint32_t kTmemCols = 2u * BN;  // two accumulators; 256 or 512 (power of two)
+    static constexpr int kStagesFit = (int)((kSmemBudget - 2048u) / kStageBytes);
+    static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
+    static constexpr uint32_t kAccStride = (BN <= 128) ? 128u : 256u;  // TMEM columns per accumulator
+    static constexpr uint32_t kTmemCols = 2u * kAccStride;             // 256 or 512 (power of two)
     static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
 };
 
@@ -157,24 +162,29 @@ __device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes,
     return d;
 }
 
-// Bytes between consecutive 32-wide column groups of an MN-major tile: hi rows then lo rows.
-constexpr uint32_t kMnAtomBytes = 2u * BK * 128u;
-
-template <bool MN>
+// Descriptor of one 8-deep k-step of an operand tile.
+//   K-major (rows of BK floats): [plane][rows][BK]; BK = 32 -> 128B swizzle (mode 2, SBO 1024),
+//                                BK = 16 -> 64B swizzle (mode 4, SBO 512); a k-step advances 32 B.
+//   MN-major: per 32-wide column group [plane][BK k-rows][128 B], 128B swizzle with 32B atoms
+//             (mode 1, SBO = 512: four k-rows; LBO = distance between column groups); a k-step
+//             advances 8 k-rows = 1024 B.
+template <bool MN, int BK>
 __device__ __forceinline__ uint64_t operand_desc(uint32_t tile_base, int rows, bool lo_plane, int kstep) {
     if (MN) {
+        constexpr uint32_t kAtom = 2u * BK * 128u;
         uint32_t addr = tile_base + (lo_plane ? BK * 128u : 0u) + (uint32_t)kstep * 8u * 128u;
-        return make_desc(addr, kMnAtomBytes, 512u, 1u);
+        return make_desc(addr, kAtom, 512u, 1u);
     } else {
-        uint32_t addr = tile_base + (lo_plane ? (uint32_t)rows * 128u : 0u) + (uint32_t)kstep * 32u;
-        return make_desc(addr, 16u, 1024u, 2u);
+        uint32_t addr = tile_base + (lo_plane ? (uint32_t)rows * BK * 4u : 0u) + (uint32_t)kstep * 32u;
+        return (BK == 32) ? make_desc(addr, 16u, 1024u, 2u) : make_desc(addr, 16u, 512u, 4u);
     }
 }
 
-template <bool A_MN, bool B_MN, int BN>
+template <bool A_MN, bool B_MN, int BN, int BK>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
-    using C = Cfg<BN>;
+    using C = Cfg<BN, BK>;
+    constexpr uint32_t kMnAtomBytes = 2u * BK * 128u;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t bars = smem_base + C::kStages * C::kStageBytes;  // 8-byte barriers
@@ -226,7 +236,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                     const uint32_t ph = (it / C::kStages) & 1u;
                     if (!mbar_wait(empty_bar(s), ph ^ 1u, g.err, 1)) { ok = false; break; }
                     const uint32_t a_dst = smem_base + s * C::kStageBytes;
-                    const uint32_t b_dst = a_dst + kATileBytes;
+                    const uint32_t b_dst = a_dst + C::kATileBytes;
                     mbar_expect_tx(full_bar(s), C::kStageBytes);
                     if (A_MN) {
 #pragma unroll
@@ -265,20 +275,20 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 const uint32_t aph = (ut >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(acc), aph ^ 1u, g.err, 2)) { ok = false; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)acc * BN;
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * C::kAccStride;
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int s = it % C::kStages;
                     const uint32_t ph = (it / C::kStages) & 1u;
                     if (!mbar_wait(full_bar(s), ph, g.err, 3)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t a_base = smem_base + s * C::kStageBytes;
-                    const uint32_t b_base = a_base + kATileBytes;
+                    const uint32_t b_base = a_base + C::kATileBytes;
 #pragma unroll
                     for (int j = 0; j < BK / 8; ++j) {
-                        const uint64_t a_hi = operand_desc<A_MN>(a_base, BM, false, j);
-                        const uint64_t a_lo = operand_desc<A_MN>(a_base, BM, true, j);
-                        const uint64_t b_hi = operand_desc<B_MN>(b_base, BN, false, j);
-                        const uint64_t b_lo = operand_desc<B_MN>(b_base, BN, true, j);
+                        const uint64_t a_hi = operand_desc<A_MN, BK>(a_base, BM, false, j);
+                        const uint64_t a_lo = operand_desc<A_MN, BK>(a_base, BM, true, j);
+                        const uint64_t b_hi = operand_desc<B_MN, BK>(b_base, BN, false, j);
+                        const uint64_t b_lo = operand_desc<B_MN, BK>(b_base, BN, true, j);
                         umma_tf32(d_tmem, a_lo, b_hi, idesc, (kb > kb0 || j > 0) ? 1u : 0u);
                         umma_tf32(d_tmem, a_hi, b_lo, idesc, 1u);
                         umma_tf32(d_tmem, a_hi, b_hi, idesc, 1u);
@@ -306,7 +316,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 Dp = g.partials + (long long)sp * g.M * g.N;
                 ldd = g.N;
             }
-            const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)acc * BN;
+            const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)acc * C::kAccStride;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 const int col0 = tn * BN + c * 32;
@@ -350,13 +360,25 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 int g_num_sms = 0;
+int g_bk = 16;       // k-block depth in use (BT_GEMM_BK=32 selects the 128-byte-row variant)
+int g_force_bn = 0;  // BT_GEMM_BN=128|192|256 pins the tile width (tuning aid)
 std::once_flag g_once;
 char g_init_err[256] = {0};
 
-template <bool A_MN, bool B_MN, int BN>
+template <bool A_MN, bool B_MN, int BN, int BK>
 cudaError_t set_attr() {
-    return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                (int)Cfg<BN>::kSmemBytes);
+    return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, BN, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)Cfg<BN, BK>::kSmemBytes);
+}
+template <bool A_MN, bool B_MN>
+cudaError_t set_attr_layout() {
+    cudaError_t a = set_attr<A_MN, B_MN, 256, 16>();
+    if (a == cudaSuccess) a = set_attr<A_MN, B_MN, 192, 16>();
+    if (a == cudaSuccess) a = set_attr<A_MN, B_MN, 128, 16>();
+    if (a == cudaSuccess) a = set_attr<A_MN, B_MN, 256, 32>();
+    if (a == cudaSuccess) a = set_attr<A_MN, B_MN, 192, 32>();
+    if (a == cudaSuccess) a = set_attr<A_MN, B_MN, 128, 32>();
+    return a;
 }
 
 void init_once() {
@@ -367,38 +389,72 @@ void init_once() {
         snprintf(g_init_err, sizeof(g_init_err), "cuTensorMapEncodeTiled not available: %s", cudaGetErrorString(e));
         return;
     }
-    g_encode = (EncodeTiledFn)fn;
     int dev = 0;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
-    cudaError_t a = cudaSuccess;
-#define BT_ATTR(AM, BMN)                                                        \
-    if (a == cudaSuccess) a = set_attr<AM, BMN, 256>();                         \
-    if (a == cudaSuccess) a = set_attr<AM, BMN, 128>()
-    BT_ATTR(false, false);
-    BT_ATTR(false, true);
-    BT_ATTR(true, true);
-#undef BT_ATTR
+    if (const char* v = getenv("BT_GEMM_BK")) g_bk = (atoi(v) == 32) ? 32 : 16;
+    if (const char* v = getenv("BT_GEMM_BN")) {
+        int bn = atoi(v);
+        if (bn == 128 || bn == 192 || bn == 256) g_force_bn = bn;
+    }
+    cudaError_t a = set_attr_layout<false, false>();
+    if (a == cudaSuccess) a = set_attr_layout<false, true>();
+    if (a == cudaSuccess) a = set_attr_layout<true, true>();
     if (a != cudaSuccess) {
         snprintf(g_init_err, sizeof(g_init_err), "cudaFuncSetAttribute(smem) failed: %s", cudaGetErrorString(a));
-        g_encode = nullptr;
+        return;
     }
+    g_encode = (EncodeTiledFn)fn;
 }
 
 // 3-D map over a split matrix: (contiguous cols, rows, plane).
-bool encode_map(CUtensorMap* tm, const SplitMat& m, uint32_t box_cols, uint32_t box_rows, bool mn_major) {
+bool encode_map(CUtensorMap* tm, const SplitMat& m, uint32_t box_cols, uint32_t box_rows, CUtensorMapSwizzle sw) {
     cuuint64_t dims[3] = {(cuuint64_t)m.cols, (cuuint64_t)m.rows, 2};
     cuuint64_t strides[2] = {(cuuint64_t)m.ld * 4, (cuuint64_t)m.plane * 4};
     cuuint32_t box[3] = {box_cols, box_rows, 2};
     cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = g_encode(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)m.hi, dims, strides, box, estr,
-                          CU_TENSOR_MAP_INTERLEAVE_NONE,
-                          mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
-                          CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, sw, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     return r == CUDA_SUCCESS;
 }
 
 constexpr int kMaxUnitsForSplit = 4 * 148;
+
+struct Plan {
+    int bn, splits, kb_per_split;
+    double cost;
+};
+
+// Picks tile width and K-split by a simple wave model.  Every work unit of one launch costs the
+// same, so the launch takes ceil(units / SMs) unit times; a unit is (k-blocks + fixed overhead)
+// x tile width, narrower tiles pay a small efficiency penalty, and a K-split pays for writing
+// and re-reading its partial sums.
+Plan make_plan(int64_t M, int64_t N, int kb_total, int bk, int sms, bool can_split, size_t max_partial_floats) {
+    const int tiles_m = (int)((M + BM - 1) / BM);
+    const double kOverheadKb = 96.0 / bk;                     // pipeline fill + exposed epilogue, in k-blocks
+    const double kb_seconds = 768.0 * (bk / 16.0) / 1.9e9;    // one 128x256 k-block of 3 MMAs at peak
+    static const int kSplits[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 20, 24, 32};
+    Plan best{256, 1, kb_total, 1e300};
+    for (int bn : {256, 192, 128}) {
+        if (g_force_bn && bn != g_force_bn) continue;
+        if (bn > 128 && N <= bn - 64) continue;               // mostly padding
+        const double pen = bn == 256 ? 1.0 : bn == 192 ? 1.04 : 1.12;
+        const long long tiles = (long long)tiles_m * ((N + bn - 1) / bn);
+        for (int sp : kSplits) {
+            if (sp > 1 && (!can_split || kb_total / sp < 8 || (size_t)sp * M * N > max_partial_floats)) continue;
+            const int kbps = (kb_total + sp - 1) / sp;
+            const int real_sp = (kb_total + kbps - 1) / kbps;
+            if (real_sp != sp) continue;
+            const long long units = tiles * sp;
+            const long long rounds = (units + sms - 1) / sms;
+            double cost = (double)rounds * (kbps + kOverheadKb) * (bn / 256.0) * pen;
+            if (sp > 1) cost += (double)(sp + 1) * M * N * 4.0 / 6.0e12 / kb_seconds;
+            if (cost < best.cost) best = Plan{bn, sp, kbps, cost};
+        }
+    }
+    return best;
+}
 
 }  // namespace
 
@@ -410,69 +466,62 @@ bool gemm_tc_init(char* err, size_t errlen) {
 
 size_t gemm_tc_partial_floats_bound() { return (size_t)kMaxUnitsForSplit * BM * 256; }
 
-cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D, int64_t ldd,
-                           const float* bias, const float* residual, float* partials, size_t max_partial_floats,
-                           int* err_word, cudaStream_t s) {
-    if (!gemm_tc_init(nullptr, 0)) return cudaErrorNotSupported;
+template <int BK>
+static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const SplitMat& A, const SplitMat& B,
+                             float* D, int64_t ldd, const float* bias, const float* residual, float* partials,
+                             size_t max_partial_floats, int* err_word, cudaStream_t s) {
     const bool a_mn = (layout == kTN), b_mn = (layout != kNT);
     const int sms = g_num_sms > 0 ? g_num_sms : 148;
-
-    // Tile width: 256 unless the 128-wide tiling wastes clearly fewer SM-rounds.
-    const int tiles_m = (int)((M + BM - 1) / BM);
-    auto rounds_cost = [&](int bn) {
-        long long tiles = (long long)tiles_m * ((N + bn - 1) / bn);
-        long long rounds = (tiles + sms - 1) / sms;
-        return (double)rounds * bn;  // time ~ rounds x tile width
-    };
-    int bn = 256;
-    if (N <= 128 || rounds_cost(128) < 0.9 * rounds_cost(256)) bn = 128;
-    const int tiles_n = (int)((N + bn - 1) / bn);
     const int kb_total = (int)((K + BK - 1) / BK);
+    const bool can_split = !bias && !residual && partials && ldd == N;
+    const Plan plan = make_plan(M, N, kb_total, BK, sms, can_split, max_partial_floats);
+    const int bn = plan.bn;
 
-    // Split K when the tile grid alone cannot fill the machine (the weight-gradient GEMMs:
-    // small outputs, K = number of tokens).
-    int splits = 1;
-    const long long tiles = (long long)tiles_m * tiles_n;
-    if (!bias && !residual && partials && ldd == N && tiles * 2 <= sms && kb_total >= 8) {
-        splits = (int)((2LL * sms + tiles - 1) / tiles);
-        if (splits > kb_total / 4) splits = kb_total / 4;
-        while (splits > 1 && (size_t)splits * M * N > max_partial_floats) --splits;
-        if (splits < 1) splits = 1;
-    }
-    int kb_per_split = (kb_total + splits - 1) / splits;
-    splits = (kb_total + kb_per_split - 1) / kb_per_split;  // no empty split
-
+    const CUtensorMapSwizzle sw_k = (BK == 32) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
+    const CUtensorMapSwizzle sw_mn = CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B;
     CUtensorMap tmA, tmB;
-    bool ok = a_mn ? encode_map(&tmA, A, 32, BK, true) : encode_map(&tmA, A, BK, BM, false);
-    ok = ok && (b_mn ? encode_map(&tmB, B, 32, BK, true) : encode_map(&tmB, B, BK, (uint32_t)bn, false));
+    bool ok = a_mn ? encode_map(&tmA, A, 32, BK, sw_mn) : encode_map(&tmA, A, BK, BM, sw_k);
+    ok = ok && (b_mn ? encode_map(&tmB, B, 32, BK, sw_mn) : encode_map(&tmB, B, BK, (uint32_t)bn, sw_k));
     if (!ok) return cudaErrorInvalidValue;
 
     GemmArgs g;
     g.M = (int)M; g.N = (int)N; g.K = (int)K;
     g.D = D; g.ldd = ldd; g.bias = bias; g.residual = residual;
-    g.tiles_m = tiles_m; g.tiles_n = tiles_n; g.splits = splits;
-    g.kb_per_split = kb_per_split; g.kb_total = kb_total;
+    g.tiles_m = (int)((M + BM - 1) / BM);
+    g.tiles_n = (int)((N + bn - 1) / bn);
+    g.splits = plan.splits;
+    g.kb_per_split = plan.kb_per_split; g.kb_total = kb_total;
     g.partials = partials; g.err = err_word;
-    const long long units = tiles * splits;
+    const long long units = (long long)g.tiles_m * g.tiles_n * g.splits;
     const int grid = (int)(units < sms ? units : sms);
 
 #define BT_LAUNCH(AM, BMN, BNV)                                                                              \
-    gemm_tc_kernel<AM, BMN, BNV><<<grid, kThreads, Cfg<BNV>::kSmemBytes, s>>>(tmA, tmB, g)
-    if (bn == 256) {
-        if (layout == kNT) BT_LAUNCH(false, false, 256);
-        else if (layout == kNN) BT_LAUNCH(false, true, 256);
-        else BT_LAUNCH(true, true, 256);
-    } else {
-        if (layout == kNT) BT_LAUNCH(false, false, 128);
-        else if (layout == kNN) BT_LAUNCH(false, true, 128);
-        else BT_LAUNCH(true, true, 128);
-    }
+    gemm_tc_kernel<AM, BMN, BNV, BK><<<grid, kThreads, Cfg<BNV, BK>::kSmemBytes, s>>>(tmA, tmB, g)
+#define BT_LAUNCH_BN(BNV)                                                                                    \
+    do {                                                                                                     \
+        if (layout == kNT) BT_LAUNCH(false, false, BNV);                                                     \
+        else if (layout == kNN) BT_LAUNCH(false, true, BNV);                                                 \
+        else BT_LAUNCH(true, true, BNV);                                                                     \
+    } while (0)
+    if (bn == 256) BT_LAUNCH_BN(256);
+    else if (bn == 192) BT_LAUNCH_BN(192);
+    else BT_LAUNCH_BN(128);
+#undef BT_LAUNCH_BN
 #undef BT_LAUNCH
     BT_COUNT_LAUNCH();
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    if (splits > 1) return launch_splitk_reduce(partials, splits, M * N, D, s);
+    if (g.splits > 1) return launch_splitk_reduce(partials, g.splits, M * N, D, s);
     return cudaSuccess;
+}
+
+cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D, int64_t ldd,
+                           const float* bias, const float* residual, float* partials, size_t max_partial_floats,
+                           int* err_word, cudaStream_t s) {
+    if (!gemm_tc_init(nullptr, 0)) return cudaErrorNotSupported;
+    if (g_bk == 32)
+        return launch_bk<32>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word, s);
+    return launch_bk<16>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word, s);
 }
 
 }  // namespace bt

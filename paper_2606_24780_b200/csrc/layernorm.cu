@@ -85,7 +85,7 @@ cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float
 
 static inline int ln_bwd_ctas(int64_t N) {
     int64_t g = (N + kLnWarps - 1) / kLnWarps;
-    if (g > 148 * 4) g = 148 * 4;
+    if (g > 148 * 2) g = 148 * 2;  // two CTAs per SM, one wave
     return (int)g;
 }
 size_t layernorm_bwd_scratch_floats(int64_t N, int C) { return (size_t)ln_bwd_ctas(N) * 2 * C; }
@@ -172,14 +172,32 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     for (int i = threadIdx.x; i < 2 * C4; i += blockDim.x) dst[i] = sm[i];
 }
 
-__global__ void __launch_bounds__(128) ln_bwd_reduce_kernel(const float* __restrict__ partial, int nparts, int C4,
+// Sums the per-CTA partials in a fixed order: lane = float4 column, warp w takes partials
+// w, w+8, ... (four loads in flight), the eight warp sums are combined in warp order.
+__global__ void __launch_bounds__(256) ln_bwd_reduce_kernel(const float* __restrict__ partial, int nparts, int C4,
                                                             float* __restrict__ dgamma, float* __restrict__ dbeta) {
-    int c = blockIdx.x * blockDim.x + threadIdx.x;  // float4 column over [2*C4): first dgamma, then dbeta
-    if (c >= 2 * C4) return;
-    float4 t = ld4(partial, c);
-    for (int p = 1; p < nparts; ++p) t = add4(t, ld4(partial, (int64_t)p * 2 * C4 + c));
-    if (c < C4) reinterpret_cast<float4*>(dgamma)[c] = t;
-    else reinterpret_cast<float4*>(dbeta)[c - C4] = t;
+    __shared__ float4 sm[8][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + lane;  // float4 column over [2*C4): first dgamma, then dbeta
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < 2 * C4) {
+        int p = warp;
+        for (; p + 24 < nparts; p += 32) {
+            float4 a0 = ld4(partial, (int64_t)p * 2 * C4 + c), a1 = ld4(partial, (int64_t)(p + 8) * 2 * C4 + c);
+            float4 a2 = ld4(partial, (int64_t)(p + 16) * 2 * C4 + c), a3 = ld4(partial, (int64_t)(p + 24) * 2 * C4 + c);
+            t = add4(add4(add4(add4(t, a0), a1), a2), a3);
+        }
+        for (; p < nparts; p += 8) t = add4(t, ld4(partial, (int64_t)p * 2 * C4 + c));
+    }
+    sm[warp][lane] = t;
+    __syncthreads();
+    if (warp == 0 && c < 2 * C4) {
+        float4 r = sm[0][lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) r = add4(r, sm[w][lane]);
+        if (c < C4) reinterpret_cast<float4*>(dgamma)[c] = r;
+        else reinterpret_cast<float4*>(dbeta)[c - C4] = r;
+    }
 }
 
 cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
@@ -200,7 +218,7 @@ cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* g
     else return cudaErrorInvalidValue;
 #undef BT_LN_BWD
     BT_COUNT_LAUNCH();
-    ln_bwd_reduce_kernel<<<(2 * C4 + 127) / 128, 128, 0, s>>>(scratch, grid, C4, dgamma, dbeta);
+    ln_bwd_reduce_kernel<<<(2 * C4 + 31) / 32, 256, 0, s>>>(scratch, grid, C4, dgamma, dbeta);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }

@@ -1,0 +1,204 @@
+"""Per-kernel micro-benchmarks through the per-op C-ABI entry points.
+
+Default workload: one GPT-2-small decoder block in isolation (d_model 768, 12 heads, MLP
+3072, batch 8 x 1024 tokens), forward and backward, plus the LM-head GEMMs, the fused
+softmax cross-entropy and AdamW at GPT-2 124M sizes.  Methodology (the paper's appendix on
+benchmarking): warm-up iterations, then timed runs with the L2 flushed (a buffer larger than
+L2 is overwritten) between iterations, CUDA events on the launching stream, median reported.
+
+    python -m paper_2606_24780_b200.opbench [--only NAME[,NAME]] [--iters 100] [--warmup 25]
+                                            [--batch 8] [--seq 1024] [--no-flush] [--json out.json]
+
+Each line: kernel, median microseconds, achieved TFLOP/s (model FLOPs) for the contractions or
+GB/s (algorithmic bytes) for the memory-bound kernels.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import sys
+
+import torch
+
+from . import binding as b
+
+
+def _rand(*shape, std=1.0):
+    return torch.randn(*shape, device="cuda", dtype=torch.float32) * std
+
+
+def _split(x):
+    s = torch.empty((2,) + tuple(x.shape), device="cuda", dtype=torch.float32)
+    b.bt_op_split(x, x.numel(), s)
+    return s
+
+
+def build_cases(B, T, C, H, Vp, n_params):
+    N, F = B * T, 4 * C
+    cases = {}
+    gsb = b.bt_op_gemm_split_scratch_bytes()
+    gscratch = torch.empty(gsb + 512, dtype=torch.uint8, device="cuda")
+    gscratch = gscratch[(-gscratch.data_ptr()) % 256:]
+
+    def gemm_case(name, layout, M, Nn, K, bias=False, residual=False):
+        a_shape = (K, M) if layout == 2 else (M, K)
+        b_shape = (Nn, K) if layout == 0 else (K, Nn)
+        A, Bm = _split(_rand(*a_shape)), _split(_rand(*b_shape, std=0.02))
+        D = torch.empty(M, Nn, device="cuda")
+        bi = _rand(Nn) if bias else None
+        res = _rand(M, Nn) if residual else None
+
+        def run():
+            b.bt_op_gemm_split(layout, M, Nn, K, A, Bm, D, bi, res, gscratch, gsb)
+        cases[name] = dict(run=run, flops=2.0 * M * Nn * K, bytes=8.0 * (M * K + Nn * K) + 4.0 * M * Nn,
+                           bound="tensor", keep=(A, Bm, D, bi, res), check=lambda: b.bt_op_gemm_check(gscratch))
+
+    # forward GEMMs of the block, the two backward layouts of each, and the LM head
+    gemm_case("gemm_nt_qkv", 0, N, 3 * C, C, bias=True)
+    gemm_case("gemm_nt_attnproj", 0, N, C, C, bias=True, residual=True)
+    gemm_case("gemm_nt_fc", 0, N, F, C, bias=True)
+    gemm_case("gemm_nt_mlpproj", 0, N, C, F, bias=True, residual=True)
+    gemm_case("gemm_nn_dqkv", 1, N, C, 3 * C)
+    gemm_case("gemm_nn_dattnproj", 1, N, C, C)
+    gemm_case("gemm_nn_dfc", 1, N, C, F)
+    gemm_case("gemm_nn_dmlpproj", 1, N, F, C)
+    gemm_case("gemm_tn_wqkv", 2, 3 * C, C, N)
+    gemm_case("gemm_tn_wattnproj", 2, C, C, N)
+    gemm_case("gemm_tn_wfc", 2, F, C, N)
+    gemm_case("gemm_tn_wmlpproj", 2, C, F, N)
+    if Vp:
+        gemm_case("gemm_nt_lmhead", 0, N, Vp, C)
+        gemm_case("gemm_nn_dlmhead", 1, N, C, Vp)
+        gemm_case("gemm_tn_wlmhead", 2, Vp, C, N)
+
+    # LayerNorm
+    x, g, be = _rand(N, C), _rand(C) * 0.1 + 1.0, _rand(C) * 0.1
+    ys, mean, rstd = torch.empty(2, N, C, device="cuda"), torch.empty(N, device="cuda"), torch.empty(N, device="cuda")
+    cases["layernorm_fwd"] = dict(run=lambda: b.bt_op_layernorm_fwd(x, g, be, N, C, None, ys, mean, rstd),
+                                  bytes=12.0 * N * C, bound="hbm", keep=(x, g, be, ys, mean, rstd))
+    b.bt_op_layernorm_fwd(x, g, be, N, C, None, ys, mean, rstd)
+    dy, dres = _rand(N, C, std=1e-2), _rand(N, C, std=1e-2)
+    dxs, dg, db = torch.empty(2, N, C, device="cuda"), torch.empty(C, device="cuda"), torch.empty(C, device="cuda")
+    lnb = b.bt_op_layernorm_bwd_scratch_bytes(N, C)
+    lscr = torch.empty(lnb + 256, dtype=torch.uint8, device="cuda")
+    lscr = lscr[(-lscr.data_ptr()) % 256:]
+    cases["layernorm_bwd"] = dict(
+        run=lambda: b.bt_op_layernorm_bwd(dy, x, g, mean, rstd, dres, N, C, dres, dxs, dg, db, lscr, lnb),
+        bytes=24.0 * N * C, bound="hbm", keep=(dy, dres, dxs, dg, db, lscr))
+
+    # GELU
+    h, dgl = _rand(N, F), _rand(N, F, std=1e-2)
+    gs, dhs = torch.empty(2, N, F, device="cuda"), torch.empty(2, N, F, device="cuda")
+    cases["gelu_fwd"] = dict(run=lambda: b.bt_op_gelu_fwd(h, N * F, 0, None, gs), bytes=12.0 * N * F, bound="hbm",
+                             keep=(h, gs))
+    cases["gelu_bwd"] = dict(run=lambda: b.bt_op_gelu_bwd(h, dgl, N * F, 0, None, dhs), bytes=16.0 * N * F,
+                             bound="hbm", keep=(dgl, dhs))
+
+    # attention
+    qkv, d_o = _rand(N, 3 * C), _rand(N, C, std=1e-2)
+    o, os_, lse = torch.empty(N, C, device="cuda"), torch.empty(2, N, C, device="cuda"), torch.empty(B, H, T, device="cuda")
+    dqs = torch.empty(2, N, 3 * C, device="cuda")
+    dv = torch.empty(B * H * T, device="cuda")
+    afl = 4.0 * B * H * (C // H) * (T * (T + 1) / 2.0)
+    cases["attention_fwd"] = dict(run=lambda: b.bt_op_attention_fwd(qkv, B, T, C, H, o, os_, lse), flops=afl,
+                                  bytes=24.0 * N * C, bound="tensor", keep=(qkv, o, os_, lse))
+    b.bt_op_attention_fwd(qkv, B, T, C, H, o, os_, lse)
+    cases["attention_bwd"] = dict(
+        run=lambda: b.bt_op_attention_bwd(qkv, o, lse, d_o, B, T, C, H, None, dqs, dv, dv.numel() * 4),
+        flops=2.5 * afl, bytes=48.0 * N * C, bound="tensor", keep=(d_o, dqs, dv))
+
+    # column sums (bias gradients)
+    csb = b.bt_op_colsum_scratch_bytes(N, F)
+    cscr = torch.empty(csb + 256, dtype=torch.uint8, device="cuda")
+    cscr = cscr[(-cscr.data_ptr()) % 256:]
+    cout = torch.empty(F, device="cuda")
+    cases["colsum_fc"] = dict(run=lambda: b.bt_op_colsum(h, N, F, cout, cscr, csb), bytes=4.0 * N * F, bound="hbm",
+                              keep=(cout, cscr))
+
+    if Vp:
+        rows = min(N, 2048)      # 2048 x 50304 logits = 412 MB: several times L2, still a small case
+        z = _rand(rows, Vp, std=2.0)
+        tg = torch.randint(0, Vp, (rows,), device="cuda", dtype=torch.int32)
+        losses, lm = torch.empty(rows, device="cuda"), torch.empty(1, device="cuda")
+        dls = torch.empty(2, rows, Vp, device="cuda")
+        cases["softmax_xent"] = dict(
+            run=lambda: b.bt_op_softmax_xent(z, tg, rows, Vp, 1.0 / rows, losses, lm, None, dls),
+            bytes=12.0 * rows * Vp, bound="hbm", keep=(z, tg, losses, lm, dls))
+    if n_params:
+        shapes = [n_params // 8] * 8
+        ps = [_rand(s, std=0.02) for s in shapes]
+        gr = [_rand(s, std=1e-3) for s in shapes]
+        ms = [torch.zeros(s, device="cuda") for s in shapes]
+        vs = [torch.zeros(s, device="cuda") for s in shapes]
+        opt = b.make_adamw()
+        cases["adamw"] = dict(run=lambda: b.bt_op_adamw_multi(ps, gr, ms, vs, [1] * 8, opt, 3),
+                              bytes=28.0 * sum(shapes), bound="hbm", keep=(ps, gr, ms, vs))
+        gnb = b.bt_op_grad_norm_scratch_bytes(shapes[0])
+        nscr = torch.empty(gnb + 256, dtype=torch.uint8, device="cuda")
+        nscr = nscr[(-nscr.data_ptr()) % 256:]
+        out2 = torch.empty(2, device="cuda")
+        cases["grad_norm"] = dict(run=lambda: b.bt_op_grad_norm(gr[0], shapes[0], 1.0, out2, nscr, gnb),
+                                  bytes=4.0 * shapes[0], bound="hbm", keep=(nscr, out2))
+    return cases
+
+
+def time_case(case, iters, warmup, flush_buf):
+    for _ in range(warmup):
+        case["run"]()
+    times = []
+    for _ in range(iters):
+        if flush_buf is not None:
+            flush_buf.add_(1.0)          # rewrite a buffer larger than L2
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        case["run"]()
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    if "check" in case:
+        case["check"]()
+    times.sort()
+    return times[len(times) // 2] * 1e3  # microseconds
+
+
+def main(argv=None):
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--only", default="")
+    ap.add_argument("--iters", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=25)
+    ap.add_argument("--batch", type=int, default=8)
+    ap.add_argument("--seq", type=int, default=1024)
+    ap.add_argument("--d-model", type=int, default=768)
+    ap.add_argument("--heads", type=int, default=12)
+    ap.add_argument("--vocab", type=int, default=50304)
+    ap.add_argument("--params", type=int, default=124_475_904)
+    ap.add_argument("--no-flush", action="store_true")
+    ap.add_argument("--json", default="")
+    args = ap.parse_args(argv)
+    torch.cuda.set_device(0)
+    only = [s for s in args.only.split(",") if s]
+    need_big = not only or any(s.startswith(("gemm_nt_lm", "gemm_nn_dlm", "gemm_tn_wlm", "softmax", "adamw", "grad"))
+                               for s in only)
+    cases = build_cases(args.batch, args.seq, args.d_model, args.heads, args.vocab if need_big else 0,
+                        args.params if need_big else 0)
+    flush = None if args.no_flush else torch.zeros(64 * 1024 * 1024, device="cuda")  # 256 MB > 126 MB L2
+    results = {}
+    for name, case in cases.items():
+        if only and name not in only:
+            continue
+        us = time_case(case, args.iters, args.warmup, flush)
+        r = {"us": us, "bound": case["bound"]}
+        if "flops" in case:
+            r["tflops"] = case["flops"] / us / 1e6
+        r["gbs"] = case["bytes"] / us / 1e3
+        results[name] = r
+        print(f"{name:22s} {us:10.1f} us  " + (f"{r['tflops']:8.1f} TFLOP/s  " if "tflops" in r else " " * 19) +
+              f"{r['gbs']:8.0f} GB/s", flush=True)
+    if args.json:
+        with open(args.json, "w") as f:
+            json.dump({"config": vars(args), "results": results}, f, indent=1)
+    return 0
+
+
+if __name__ == "__main__":
+    sys.exit(main())
