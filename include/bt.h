@@ -26,8 +26,8 @@
  *           BT_ERR_DEVICE_TIMEOUT.
  * Split     The tensor-core GEMMs compute FP32 products as three TF32 products
  *           (a_hi*b_hi + a_hi*b_lo + a_lo*b_hi, FP32 accumulate).  Operands are therefore
- *           stored as two FP32 planes, `hi` = the value with its low 13 mantissa bits
- *           cleared and `lo` = value - hi (exact).  A "split" array of R x C values is
+ *           stored as two FP32 planes, `hi` = the value rounded to the nearest TF32 number
+ *           (low 13 mantissa bits zero) and `lo` = value - hi (exact).  A "split" array of R x C values is
  *           [2][R][C]: plane 0 = hi, plane 1 = lo.  Kernels that produce GEMM operands
  *           can write the split form directly.
  * Tokens    Token and target ids must lie in [0, vocab_size); this is not checked on
@@ -273,6 +273,23 @@ BT_API bt_status bt_op_softmax_xent(const float* logits, const int32_t* targets,
 BT_API size_t bt_op_colsum_scratch_bytes(int64_t N, int32_t C);
 BT_API bt_status bt_op_colsum(const float* x, int64_t N, int32_t C, float* out, void* scratch,
                               size_t scratch_bytes, void* stream);
+
+/* Column sums for callers that cannot provide scratch memory.  (The paper has no counterpart;
+ * this entry point exists for integration.)  Some hosts of this library may not allocate device
+ * memory at the point of the call: a serving process whose device memory was handed out in full
+ * at start-up, a real-time control loop where cudaMalloc's implicit device synchronisation is
+ * forbidden, a plug-in that is only given its input and output buffers.  For them the partial
+ * sums live in a fixed array inside the library image: 98,304 floats (384 KB) that every GPU
+ * loading the library holds until the process exits.  The call allocates nothing (no cudaMalloc,
+ * cudaFree or allocating library routine) and returns BT_ERR_UNSUPPORTED when
+ * bt_op_colsum_scratch_bytes(N, C) exceeds that size (roughly C > 22,000).
+ * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
+ * that device current) and caches it; make that first call before starting any stream capture.
+ * Every call on a device shares the one array and overwrites the part it uses, so calls that
+ * may overlap on the GPU (different streams, no ordering between them) race; keep them on one
+ * stream or order them with events.  Same result as bt_op_colsum, bit for bit. */
+BT_API size_t bt_op_colsum_static_max_floats(void);
+BT_API bt_status bt_op_colsum_static(const float* x, int64_t N, int32_t C, float* out, void* stream);
 
 /* out[0] = sqrt(sum g^2), out[1] = clip > 0 ? min(1, clip / (out[0] + 1e-6)) : 1. */
 BT_API size_t bt_op_grad_norm_scratch_bytes(int64_t n);

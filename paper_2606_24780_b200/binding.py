@@ -79,6 +79,8 @@ _SIGNATURES = {
     "bt_op_softmax_xent": (_i32, [_vp, _vp, _i64, _i32, _f, _vp, _vp, _vp, _vp, _vp]),
     "bt_op_colsum_scratch_bytes": (_sz, [_i64, _i32]),
     "bt_op_colsum": (_i32, [_vp, _i64, _i32, _vp, _vp, _sz, _vp]),
+    "bt_op_colsum_static_max_floats": (_sz, []),
+    "bt_op_colsum_static": (_i32, [_vp, _i64, _i32, _vp, _vp]),
     "bt_op_grad_norm_scratch_bytes": (_sz, [_i64]),
     "bt_op_grad_norm": (_i32, [_vp, _i64, _f, _vp, _vp, _sz, _vp]),
     "bt_op_adamw_multi": (_i32, [_i32] + [ctypes.POINTER(_vp)] * 4 + [ctypes.POINTER(_i64), ctypes.POINTER(_i32),
@@ -332,6 +334,15 @@ def bt_op_colsum_scratch_bytes(N, C):
 
 def bt_op_colsum(x, N, C, out, scratch, scratch_bytes, stream=None):
     _check(lib().bt_op_colsum(_ptr(x), N, C, _ptr(out), _ptr(scratch), scratch_bytes, _stream(stream)))
+
+
+def bt_op_colsum_static_max_floats():
+    return int(lib().bt_op_colsum_static_max_floats())
+
+
+def bt_op_colsum_static(x, N, C, out, stream=None):
+    """Column sums with the library's built-in scratch: for callers that cannot allocate device memory."""
+    _check(lib().bt_op_colsum_static(_ptr(x), N, C, _ptr(out), _stream(stream)))
 
 
 def bt_op_grad_norm_scratch_bytes(n):

@@ -30,6 +30,15 @@ bt_status fail(bt_status st, const char* fmt, ...) {
     return st;
 }
 
+}  // namespace
+
+extern "C" __attribute__((visibility("hidden"))) int bt_internal_fail_int(int status, const char* message) {
+    g_last_error = message ? message : "";
+    return status;
+}
+
+namespace {
+
 #define BT_CUDA(call)                                                                           \
     do {                                                                                        \
         cudaError_t e__ = (call);                                                               \

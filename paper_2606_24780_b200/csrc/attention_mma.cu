@@ -38,7 +38,7 @@ __device__ __forceinline__ void mma3(float (&d)[4], const uint32_t (&a_hi)[4], c
     mma_tf32(d, a_hi, bh0, bh1);
 }
 __device__ __forceinline__ void split_u(float x, uint32_t& hi, uint32_t& lo) {
-    hi = __float_as_uint(x) & 0xFFFFE000u;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(hi) : "f"(x));  // nearest TF32 value (see split_tf32)
     lo = __float_as_uint(x - __uint_as_float(hi));
 }
 

@@ -5,6 +5,10 @@
 
 #include <atomic>
 
+// Records the thread-local error string returned by bt_last_error() and passes `status` through
+// (defined with the C ABI; status is a bt_status).
+extern "C" int bt_internal_fail_int(int status, const char* message);
+
 namespace bt {
 
 // Every launcher bumps this counter once per kernel launch (read by bt_launch_count).
@@ -29,10 +33,15 @@ __device__ __forceinline__ double warp_sum_d(double v) {
     return v;
 }
 
-// TF32 split: hi keeps sign, exponent and the top 10 mantissa bits, lo = x - hi is exact
-// in FP32.  x = hi + lo always holds bit for bit.
+// TF32 split: hi = x rounded to the nearest TF32 value (10 mantissa bits, low 13 bits zero),
+// lo = x - hi, which is exact in FP32; x = hi + lo holds bit for bit.  Rounding to nearest
+// (instead of clearing the low bits) keeps |lo| <= 2^-11 |x| and, more importantly, gives lo a
+// random sign, so the terms the three-product scheme drops (lo*lo, and the low bits of lo the
+// tensor core ignores) do not add up to a systematic shrink over a chain of GEMMs.
 __device__ __forceinline__ void split_tf32(float x, float& hi, float& lo) {
-    hi = __uint_as_float(__float_as_uint(x) & 0xFFFFE000u);
+    uint32_t h;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h) : "f"(x));
+    hi = __uint_as_float(h);
     lo = x - hi;
 }
 __device__ __forceinline__ void split_tf32(const float4& x, float4& hi, float4& lo) {

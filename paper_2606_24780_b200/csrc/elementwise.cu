@@ -4,7 +4,14 @@
 //
 // All of them stream their operands once with 128-bit accesses; reductions use warp
 // shuffles and fixed summation orders (no floating-point atomics anywhere).
+#include <mutex>
+
+#include "../../include/bt.h"
 #include "common.cuh"
+
+static inline bt_status bt_internal_fail(bt_status st, const char* msg) {
+    return (bt_status)bt_internal_fail_int((int)st, msg);
+}
 
 namespace bt {
 
@@ -268,6 +275,56 @@ cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, f
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
+
+// ------------------------------------------------------------------ column sums without allocation
+
+// Scratch for bt_op_colsum_static: lives in the library image, so every GPU that loads the
+// library holds these 384 KB until the process exits.  All calls share it.
+constexpr size_t kStaticColsumFloats = 96 * 1024;
+static __device__ __align__(256) float g_colsum_static_scratch[kStaticColsumFloats];
+
+static std::mutex g_static_mutex;
+static float* g_static_scratch_ptr[64] = {nullptr};  // device address of the array, per device ordinal
+
+// In host code the array's name is only a handle; the device address must be asked for, once
+// per device, with that device current.
+static cudaError_t static_scratch_address(float** out) {
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    if (g_static_scratch_ptr[dev] == nullptr) {
+        float* p = nullptr;
+        e = cudaGetSymbolAddress((void**)&p, g_colsum_static_scratch);
+        if (e != cudaSuccess) return e;
+        g_static_scratch_ptr[dev] = p;
+    }
+    *out = g_static_scratch_ptr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace bt
+
+extern "C" size_t bt_op_colsum_static_max_floats(void) { return bt::kStaticColsumFloats; }
+
+extern "C" bt_status bt_op_colsum_static(const float* x, int64_t N, int32_t C, float* out, void* stream) {
+    using namespace bt;
+    if (!x || !out) return bt_internal_fail(BT_ERR_INVALID_ARG, "colsum_static: NULL argument");
+    if ((reinterpret_cast<uintptr_t>(x) | reinterpret_cast<uintptr_t>(out)) & 15u)
+        return bt_internal_fail(BT_ERR_INVALID_ARG, "colsum_static: pointers must be 16-byte aligned");
+    if (N < 1 || C < 4 || C % 4) return bt_internal_fail(BT_ERR_INVALID_ARG, "colsum_static: bad sizes");
+    if (colsum_scratch_floats(N, C) > kStaticColsumFloats)
+        return bt_internal_fail(BT_ERR_UNSUPPORTED, "colsum_static: N x C needs more than the built-in scratch "
+                                                    "(98304 floats); use bt_op_colsum with caller scratch");
+    float* scratch = nullptr;
+    cudaError_t e = static_scratch_address(&scratch);
+    if (e == cudaSuccess) e = launch_colsum(x, nullptr, N, C, out, scratch, (cudaStream_t)stream);
+    if (e != cudaSuccess) return bt_internal_fail(BT_ERR_CUDA, cudaGetErrorString(e));
+    return BT_OK;
+}
+
+namespace bt {
 
 // ------------------------------------------------------------------ gradient norm
 

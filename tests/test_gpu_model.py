@@ -55,7 +55,7 @@ def compare_gradients(gm, om, cfg):
     return worst
 
 
-def adamw_step_and_compare(gm, om, step):
+def adamw_step_and_compare(gm, om, step, max_outside=0.02):
     """One optimizer step on both sides from IDENTICAL state (p, m, v, t), two comparisons.
 
     (A) optimizer exactness: the oracle's AdamW applied to the GPU's own gradient must give the
@@ -76,7 +76,10 @@ def adamw_step_and_compare(gm, om, step):
     scale = oracle.clip_scale(gn_gpu_ref, hp["grad_clip"])
     gn = gm.adamw_step(opt)
     ref_gn = om.adamw_step(hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], hp["grad_clip"])
-    assert abs(gn - ref_gn) < 1e-4 * ref_gn and abs(gn - gn_gpu_ref) < 1e-5 * gn_gpu_ref
+    # the norm is a gradient quantity: held to the gradient tolerance against the oracle's own
+    # gradient, and to FP32 accuracy against the norm of the GPU's gradient
+    assert abs(gn - ref_gn) < TOL_GRAD * ref_gn and abs(gn - gn_gpu_ref) < 1e-5 * gn_gpu_ref
+    print(f"grad norm {gn:.6f} (oracle {ref_gn:.6f}, rel diff {(gn - ref_gn) / ref_gn:+.2e})")
     total, outside, worst_a = 0, 0, 0.0
     for n in names:
         p0, m0, v0 = state[n]
@@ -91,7 +94,7 @@ def adamw_step_and_compare(gm, om, step):
         total += db.size
         outside += int((db >= TOL_PARAM).sum())
         assert db.max() <= 2.2 * hp["lr"], (step, n, db.max())
-    assert outside <= 0.02 * total, (step, outside, total)
+    assert outside <= max_outside * total, (step, outside, total)
     # continue from identical state: the oracle adopts the GPU's FP32 parameters and moments
     for n in names:
         for kind in (0, 2, 3):
@@ -147,6 +150,38 @@ def test_medium_config_spans_tiles_and_ragged_tails():
     cfg = si.make_config(n_layers=2, d_model=768, n_heads=12, seq_len=200, vocab_size=4000,
                          padded_vocab_size=4032, batch=3, tokens="zipf")
     run_steps(cfg, seed=3, flags=0, B=3, steps=2)
+
+
+def test_gpt2_124m_full_size_step():
+    """BASELINE config 2 at full size, in the launch configuration the benchmark times: 12 layers,
+    d_model 768, vocabulary 50257 (padded 50304), batch 8 x 1024 Zipf tokens.  The oracle runs
+    the eight sequences one at a time (about two minutes on 16 host cores) and supplies the loss,
+    the logits of the last sequence, every gradient tensor and the AdamW update."""
+    import time
+    cfg = si.config(2)
+    B = cfg["batch"]
+    t0 = time.time()
+    gm, om = make_pair(cfg, seed=2, flags=0, max_batch=B, jitter=0.0)
+    tok, tgt = si.tokens_for(cfg, 2, B)
+    loss = gm.forward(dev(tok), dev(tgt))
+    gm.backward()
+    ref_loss = om.loss_and_grad(tok, tgt, chunk=1)
+    print(f"oracle forward+backward of {B} x {cfg['seq_len']} tokens: {time.time() - t0:.0f} s; "
+          f"loss {loss:.6f} vs {ref_loss:.6f}")
+    assert abs(loss - ref_loss) < TOL_LOSS * abs(ref_loss)
+    # "initial loss ~ ln(vocab)": with tied embeddings and Zipf text a position whose target repeats
+    # its input token sees a large target logit, which pulls the mean a little below
+    # ln(Vp) + (logit variance) / 2 = 10.98
+    assert abs(ref_loss - math.log(cfg["padded_vocab_size"])) < 0.2
+    T, Vp = cfg["seq_len"], cfg["padded_vocab_size"]
+    ref_logits = om.activation("logits")                      # last chunk = last sequence
+    got_logits = host(gm.activation("logits")).reshape(-1, Vp)[(B - 1) * T:]
+    assert rel_max(got_logits, ref_logits) < TOL_LOGITS and rel_l2(got_logits, ref_logits) < TOL_LOGITS
+    worst = compare_gradients(gm, om, cfg)
+    frac, exact = adamw_step_and_compare(gm, om, 0, max_outside=0.05)
+    print(f"worst gradient rel-L2 {worst:.2e}; AdamW exactness {exact:.2e}; {100 * frac:.2f}% of parameters "
+          f"ill-conditioned at t = 1")
+    gm.close()
 
 
 def test_partial_batch_and_host_tokens():
