@@ -243,9 +243,13 @@ BT_API bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K, con
 
 /* Causal multi-head self-attention over fused qkv [B*T, 3C] (columns q | k | v, head h at
  * columns h*d..(h+1)*d-1 of each part): o = softmax(q k^T / sqrt(d) + causal mask) v,
- * lse [B,H,T] = log of the softmax normaliser.  d = C/H in {16, 32, 64, 128}. */
-BT_API bt_status bt_op_attention_fwd(const float* qkv, int32_t B, int32_t T, int32_t C, int32_t H, float* o,
-                                     float* o_split, float* lse, uint32_t flags, void* stream);
+ * lse [B,H,T] = log of the softmax normaliser.  d = C/H in {16, 32, 64, 128}.
+ * qkv_split (nullable) is the same array as hi/lo planes [2][B*T][3C]; when it is given and d = 64
+ * the tcgen05 kernel runs (TMA-fed, scores and probabilities in tensor memory; synchronises to
+ * report a device timeout), otherwise the warp-MMA kernel runs on the raw array.  One of qkv,
+ * qkv_split may be NULL. */
+BT_API bt_status bt_op_attention_fwd(const float* qkv, const float* qkv_split, int32_t B, int32_t T, int32_t C,
+                                     int32_t H, float* o, float* o_split, float* lse, uint32_t flags, void* stream);
 
 /* Backward of the above with recomputed probabilities: dV = P^T do, dP = do V^T,
  * dS = P o (dP - rowsum(do o o)), dq = dS k / sqrt(d), dk = dS^T q / sqrt(d).

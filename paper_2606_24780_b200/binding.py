@@ -72,7 +72,7 @@ _SIGNATURES = {
     "bt_op_gemm_split": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
     "bt_op_gemm_check": (_i32, [_vp, _vp]),
     "bt_op_gemm": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
-    "bt_op_attention_fwd": (_i32, [_vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _u32, _vp]),
+    "bt_op_attention_fwd": (_i32, [_vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _u32, _vp]),
     "bt_op_attention_bwd": (_i32, [_vp] * 4 + [_i32] * 4 + [_vp] * 3 + [_sz, _u32, _vp]),
     "bt_op_gelu_fwd": (_i32, [_vp, _i64, _i32, _vp, _vp, _vp]),
     "bt_op_gelu_bwd": (_i32, [_vp, _vp, _i64, _i32, _vp, _vp, _vp]),
@@ -305,8 +305,8 @@ def bt_op_gemm_check(scratch, stream=None):
     _check(lib().bt_op_gemm_check(_ptr(scratch), _stream(stream)))
 
 
-def bt_op_attention_fwd(qkv, B, T, C, H, o, o_split, lse, flags=0, stream=None):
-    _check(lib().bt_op_attention_fwd(_ptr(qkv), B, T, C, H, _ptr(o), _ptr(o_split), _ptr(lse), flags,
+def bt_op_attention_fwd(qkv, B, T, C, H, o, o_split, lse, flags=0, stream=None, qkv_split=None):
+    _check(lib().bt_op_attention_fwd(_ptr(qkv), _ptr(qkv_split), B, T, C, H, _ptr(o), _ptr(o_split), _ptr(lse), flags,
                                      _stream(stream)))
 
 

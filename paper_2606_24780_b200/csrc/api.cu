@@ -81,7 +81,7 @@ const char* const kCatNames[kNumCats] = {
     "adamw"};
 
 struct LayerAct {
-    float *x, *mean1, *rstd1, *a_s, *qkv, *o_s, *lse, *x1, *mean2, *rstd2, *m_s, *h, *g_s;
+    float *x, *mean1, *rstd1, *a_s, *qkv, *qkv_s, *o_s, *lse, *x1, *mean2, *rstd2, *m_s, *h, *g_s;
 };
 
 // Bump allocator over the workspace; with base == nullptr it only measures.
@@ -194,6 +194,7 @@ size_t layout(bt_model* m, uint8_t* base) {
         a.rstd1 = b.take<float>(N);
         a.a_s = b.take<float>(2 * N * C);
         a.qkv = b.take<float>(N * 3 * C);
+        a.qkv_s = b.take<float>(2 * N * 3 * C);
         a.o_s = b.take<float>(2 * N * C);
         a.lse = b.take<float>((int64_t)m->maxB * m->H * m->T);
         a.x1 = b.take<float>(N * C);
@@ -293,15 +294,24 @@ inline double attn_fwd_flops(int64_t B, int64_t H, int64_t T, int64_t d) {
 
 // D = op(A) op(B) (+bias)(+residual) through the tensor-core kernel or the FMA reference.
 cudaError_t gemm_raw(bt_model* m, int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
-                 const float* bias, const float* residual) {
-    if (m->cfg.flags & BT_FLAG_GEMM_SIMT) return launch_gemm_simt(layout, M, N, K, A, B, D, N, bias, residual, m->stream);
+                 const float* bias, const float* residual, float* d_split = nullptr) {
+    if (m->cfg.flags & BT_FLAG_GEMM_SIMT) {
+        // the FMA reference writes the raw output; the planes are made by a separate pass
+        cudaError_t e = launch_gemm_simt(layout, M, N, K, A, B, D, N, bias, residual, m->stream);
+        if (e == cudaSuccess && d_split) e = launch_split(D, d_split, d_split + M * N, M * N, m->stream);
+        return e;
+    }
     return launch_gemm_tc(layout, M, N, K, A, B, D, N, bias, residual, m->partials, m->partial_floats, m->err_word,
-                          m->stream);
+                          m->stream, d_split, M * N);
 }
 
 #define BT_GEMM(layout, M, N, K, A, B, D, bias, res)                                                        \
     BT_STEP((layout) == kNT ? kCatGemmNT : (layout) == kNN ? kCatGemmNN : kCatGemmTN, gemm_flops(M, N, K),     \
             gemm_bytes(M, N, K), gemm_raw(m, layout, M, N, K, A, B, D, bias, res))
+// same, the output also written as TF32 hi/lo planes at DS
+#define BT_GEMM_SPLIT_OUT(layout, M, N, K, A, B, D, DS, bias, res)                                           \
+    BT_STEP((layout) == kNT ? kCatGemmNT : (layout) == kNN ? kCatGemmNN : kCatGemmTN, gemm_flops(M, N, K),     \
+            gemm_bytes(M, N, K) + 8.0 * (M) * (N), gemm_raw(m, layout, M, N, K, A, B, D, bias, res, DS))
 
 bt_status check_device_error(bt_model* m) {
     int err = 0;
@@ -508,9 +518,10 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
         float* xout = (l + 1 < m->L) ? m->act[l + 1].x : m->xL;
         auto P = [&](int k) { return m->params + layer_tensor(m, l, k).off; };
         BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x, P(LN1G), P(LN1B), N, C, nullptr, a.a_s, a.a_s + N * C, a.mean1, a.rstd1, s));
-        BT_GEMM(kNT, N, 3 * C, C, act_mat(a.a_s, N, C, N), weight_mat(m, layer_tensor(m, l, QKVW), 3 * C, C),
-                     a.qkv, P(QKVB), nullptr);
-        BT_STEP(kCatAttnFwd, attn_fwd_flops(B, H, T, C / H), 20.0 * N * C, launch_attention_fwd(a.qkv, B, T, C, H, nullptr, a.o_s, a.o_s + N * C, a.lse, simt_attn, s));
+        BT_GEMM_SPLIT_OUT(kNT, N, 3 * C, C, act_mat(a.a_s, N, C, N), weight_mat(m, layer_tensor(m, l, QKVW), 3 * C, C),
+                          a.qkv, a.qkv_s, P(QKVB), nullptr);
+        BT_STEP(kCatAttnFwd, attn_fwd_flops(B, H, T, C / H), 20.0 * N * C, launch_attention_fwd(a.qkv, a.qkv_s, N * 3 * C, B, T, C, H, nullptr, a.o_s, a.o_s + N * C, a.lse, simt_attn,
+                                     m->err_word, s));
         BT_GEMM(kNT, N, C, C, act_mat(a.o_s, N, C, N), weight_mat(m, layer_tensor(m, l, PROJW), C, C), a.x1,
                      P(PROJB), a.x);
         BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x1, P(LN2G), P(LN2B), N, C, nullptr, a.m_s, a.m_s + N * C, a.mean2, a.rstd2, s));
@@ -777,14 +788,33 @@ extern "C" bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K,
     return bt_op_gemm_check(rest, stream);
 }
 
-extern "C" bt_status bt_op_attention_fwd(const float* qkv, int32_t B, int32_t T, int32_t C, int32_t H, float* o,
-                                         float* o_split, float* lse, uint32_t flags, void* stream) {
-    BT_PTR(qkv); BT_OPT_PTR(o); BT_OPT_PTR(o_split); BT_PTR(lse);
+extern "C" bt_status bt_op_attention_fwd(const float* qkv, const float* qkv_split, int32_t B, int32_t T, int32_t C,
+                                         int32_t H, float* o, float* o_split, float* lse, uint32_t flags,
+                                         void* stream) {
+    BT_OPT_PTR(qkv); BT_OPT_PTR(qkv_split); BT_OPT_PTR(o); BT_OPT_PTR(o_split); BT_PTR(lse);
+    if (!qkv && !qkv_split) return fail(BT_ERR_INVALID_ARG, "attention_fwd: qkv and qkv_split both NULL");
     if (B < 1 || T < 1 || C < 1 || H < 1 || C % H) return fail(BT_ERR_INVALID_ARG, "attention_fwd: bad sizes");
     int d = C / H;
     if (d != 16 && d != 32 && d != 64 && d != 128) return fail(BT_ERR_UNSUPPORTED, "attention: head_dim %d", d);
-    BT_CUDA(launch_attention_fwd(qkv, B, T, C, H, o, o_split, o_split ? o_split + (int64_t)B * T * C : nullptr, lse,
-                                 (flags & BT_FLAG_ATTN_SIMT) != 0, (cudaStream_t)stream));
+    const bool simt = (flags & BT_FLAG_ATTN_SIMT) != 0;
+    if (!qkv && (simt || d != 64))
+        return fail(BT_ERR_INVALID_ARG, "attention_fwd: this kernel needs the raw qkv array");
+    int* err = nullptr;
+    if (qkv_split && d == 64 && !simt) {
+        char msg[256];
+        if (!gemm_tc_init(msg, sizeof(msg))) return fail(BT_ERR_CUDA, "tensor-core attention unavailable: %s", msg);
+        BT_CUDA(attention_tc_default_err(&err));
+        BT_CUDA(cudaMemsetAsync(err, 0, sizeof(int), (cudaStream_t)stream));
+    }
+    BT_CUDA(launch_attention_fwd(qkv, qkv_split, (int64_t)B * T * 3 * C, B, T, C, H, o, o_split,
+                                 o_split ? o_split + (int64_t)B * T * C : nullptr, lse, simt, err,
+                                 (cudaStream_t)stream));
+    if (err) {
+        int herr = 0;
+        BT_CUDA(cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, (cudaStream_t)stream));
+        BT_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+        if (herr) return fail(BT_ERR_DEVICE_TIMEOUT, "attention_fwd: a bounded device-side wait ran out (code %d)", herr);
+    }
     return BT_OK;
 }
 

@@ -18,8 +18,18 @@ cudaError_t launch_attention_bwd_mma(const float* qkv, const float* lse, const f
                                      int T, int C, int H, float* dqkv, float* dqkv_hi, float* dqkv_lo,
                                      cudaStream_t s);
 
-cudaError_t launch_attention_fwd(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi, float* o_lo,
-                                 float* lse, bool simt, cudaStream_t s) {
+bool attention_tc_supports(int head_dim, int C);
+cudaError_t launch_attention_fwd_tc(const float* qkv_hi, int64_t qkv_plane, int B, int T, int C, int H, float* o,
+                                    float* o_hi, float* o_lo, float* lse, int* err_word, cudaStream_t s);
+
+// qkv_hi (nullable): the same qkv as TF32 hi/lo planes (lo at qkv_hi + qkv_plane); with it and
+// head_dim 64 the tcgen05 kernel runs, otherwise the warp-MMA kernel on the raw array.
+cudaError_t launch_attention_fwd(const float* qkv, const float* qkv_hi, int64_t qkv_plane, int B, int T, int C, int H,
+                                 float* o, float* o_hi, float* o_lo, float* lse, bool simt, int* err_word,
+                                 cudaStream_t s) {
+    if (!simt && qkv_hi && attention_tc_supports(C / H, C))
+        return launch_attention_fwd_tc(qkv_hi, qkv_plane, B, T, C, H, o, o_hi, o_lo, lse, err_word, s);
+    if (!qkv) return cudaErrorInvalidValue;
     if (simt || !attention_mma_supports(C / H)) return launch_attention_fwd_simt(qkv, B, T, C, H, o, o_hi, o_lo, lse, s);
     return launch_attention_fwd_mma(qkv, B, T, C, H, o, o_hi, o_lo, lse, s);
 }

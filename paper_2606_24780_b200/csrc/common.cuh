@@ -136,16 +136,21 @@ cudaError_t launch_gemm_simt(int layout, int64_t M, int64_t N, int64_t K, SplitM
                              int64_t ldd, const float* bias, const float* residual, cudaStream_t s);
 
 // tcgen05 GEMM.  `partials` (nullable) receives split-K partial sums; max_partial_floats its size.
+// D may be null when d_hi is given: the output is then written only as TF32 hi/lo planes
+// (d_hi[row*ldd + col], lo plane at d_hi + d_plane).
 // err_word: device int set non-zero when a bounded wait ran out.
 cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
                            int64_t ldd, const float* bias, const float* residual, float* partials,
-                           size_t max_partial_floats, int* err_word, cudaStream_t s);
+                           size_t max_partial_floats, int* err_word, cudaStream_t s, float* d_hi = nullptr,
+                           int64_t d_plane = 0);
 size_t gemm_tc_partial_floats_bound();
 bool gemm_tc_init(char* err, size_t errlen);  // resolves the tensor-map encoder
 
 // Attention.  lo planes are written when the hi pointer is non-null.
-cudaError_t launch_attention_fwd(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi, float* o_lo,
-                                 float* lse, bool simt, cudaStream_t s);
+cudaError_t launch_attention_fwd(const float* qkv, const float* qkv_hi, int64_t qkv_plane, int B, int T, int C, int H,
+                                 float* o, float* o_hi, float* o_lo, float* lse, bool simt, int* err_word,
+                                 cudaStream_t s);
+cudaError_t attention_tc_default_err(int** out);
 // o given raw (o_lo == nullptr) or as hi/lo planes.  dvec: B*H*T floats of scratch.
 cudaError_t launch_attention_bwd(const float* qkv, const float* o, const float* o_lo, const float* lse,
                                  const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,

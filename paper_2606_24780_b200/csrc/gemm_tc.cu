@@ -32,8 +32,11 @@
 #include <mutex>
 
 #include "common.cuh"
+#include "tc_common.cuh"
 
 namespace bt {
+
+using namespace tc;
 
 namespace {
 
@@ -65,102 +68,9 @@ struct GemmArgs {
     int tiles_m, tiles_n, splits, kb_per_split, kb_total;
     float* partials;
     int* err;
+    float* d_hi;        // optional TF32 hi/lo planes of the output (lo = d_hi + d_plane)
+    long long d_plane;
 };
-
-// ------------------------------------------------------------------ PTX wrappers
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ uint32_t mbar_try_wait(uint32_t bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok)
-        : "r"(bar), "r"(parity)
-        : "memory");
-    return ok;
-}
-__device__ __forceinline__ unsigned long long globaltimer_ns() {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-    return t;
-}
-// Bounded wait (about one second).  Returns false after raising the error word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, int code) {
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = globaltimer_ns();
-    for (;;) {
-        for (int i = 0; i < 256; ++i)
-            if (mbar_try_wait(bar, parity)) return true;
-        if (globaltimer_ns() - t0 > 1000000000ull) {
-            atomicExch(err, code);
-            return false;
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,
-                                            int c2) {
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];"
-        ::"r"(dst), "l"((unsigned long long)tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2)
-        : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc,
-                                          uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
-        : "memory");
-}
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
-          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]),
-          "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]),
-          "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr));
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor (sm_100 format): start address, leading / stride byte offsets
-// (all >> 4), descriptor version 1, swizzle mode in bits 61-63.
-//   K-major, 128B swizzle          : mode 2, SBO = 1024 (8 rows x 128 B), LBO unused.
-//   MN-major, 128B swizzle/32B atom: mode 1, SBO = 512 (4 k-rows x 128 B), LBO = distance between
-//                                    32-element column groups.
-__device__ __forceinline__ uint64_t make_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t mode) {
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFFu);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)mode << 61;
-    return d;
-}
 
 // Descriptor of one 8-deep k-step of an operand tile.
 //   K-major (rows of BK floats): [plane][rows][BK]; BK = 32 -> 128B swizzle (mode 2, SBO 1024),
@@ -262,9 +172,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     } else if (warp == 1) {
         // ---------------------------------------------------------------- MMA issuer
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((A_MN ? 1u : 0u) << 15) |
-                                   ((B_MN ? 1u : 0u) << 16) | ((uint32_t)(BN >> 3) << 17) |
-                                   ((uint32_t)(BM >> 4) << 24);
+            constexpr uint32_t idesc = make_idesc_tf32(BM, BN, A_MN, B_MN);
             uint32_t it = 0, ut = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++ut) {
@@ -334,7 +242,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                                    __uint_as_float(rr[4 * q + 2]), __uint_as_float(rr[4 * q + 3]));
                             if (g.bias) v = add4(v, *reinterpret_cast<const float4*>(g.bias + col0 + q * 4));
                             if (rrow) v = add4(v, *reinterpret_cast<const float4*>(rrow + q * 4));
-                            *reinterpret_cast<float4*>(drow + q * 4) = v;
+                            if (Dp) *reinterpret_cast<float4*>(drow + q * 4) = v;
+                            if (g.d_hi) {
+                                float4 hh, ll;
+                                split_tf32(v, hh, ll);
+                                float* hrow = g.d_hi + (long long)row * g.ldd + col0 + q * 4;
+                                *reinterpret_cast<float4*>(hrow) = hh;
+                                *reinterpret_cast<float4*>(hrow + g.d_plane) = ll;
+                            }
                         }
                     }
                 }
@@ -355,9 +270,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 
 // ------------------------------------------------------------------ host side
 
-typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
-                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
-                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 EncodeTiledFn g_encode = nullptr;
 int g_num_sms = 0;
 int g_bk = 16;       // k-block depth in use (BT_GEMM_BK=32 selects the 128-byte-row variant)
@@ -458,6 +370,17 @@ Plan make_plan(int64_t M, int64_t N, int kb_total, int bk, int sms, bool can_spl
 
 }  // namespace
 
+namespace tc {
+EncodeTiledFn tensor_map_encoder() {
+    gemm_tc_init(nullptr, 0);
+    return g_encode;
+}
+int sm_count() {
+    gemm_tc_init(nullptr, 0);
+    return g_num_sms > 0 ? g_num_sms : 148;
+}
+}  // namespace tc
+
 bool gemm_tc_init(char* err, size_t errlen) {
     std::call_once(g_once, init_once);
     if (!g_encode && err) snprintf(err, errlen, "%s", g_init_err);
@@ -469,11 +392,12 @@ size_t gemm_tc_partial_floats_bound() { return (size_t)kMaxUnitsForSplit * BM * 
 template <int BK>
 static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const SplitMat& A, const SplitMat& B,
                              float* D, int64_t ldd, const float* bias, const float* residual, float* partials,
-                             size_t max_partial_floats, int* err_word, cudaStream_t s) {
+                             size_t max_partial_floats, int* err_word, float* d_hi, int64_t d_plane,
+                             cudaStream_t s) {
     const bool a_mn = (layout == kTN), b_mn = (layout != kNT);
     const int sms = g_num_sms > 0 ? g_num_sms : 148;
     const int kb_total = (int)((K + BK - 1) / BK);
-    const bool can_split = !bias && !residual && partials && ldd == N;
+    const bool can_split = !bias && !residual && partials && ldd == N && D && !d_hi;
     const Plan plan = make_plan(M, N, kb_total, BK, sms, can_split, max_partial_floats);
     const int bn = plan.bn;
 
@@ -492,6 +416,7 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     g.splits = plan.splits;
     g.kb_per_split = plan.kb_per_split; g.kb_total = kb_total;
     g.partials = partials; g.err = err_word;
+    g.d_hi = d_hi; g.d_plane = d_plane;
     const long long units = (long long)g.tiles_m * g.tiles_n * g.splits;
     const int grid = (int)(units < sms ? units : sms);
 
@@ -517,11 +442,14 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
 
 cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D, int64_t ldd,
                            const float* bias, const float* residual, float* partials, size_t max_partial_floats,
-                           int* err_word, cudaStream_t s) {
+                           int* err_word, cudaStream_t s, float* d_hi, int64_t d_plane) {
     if (!gemm_tc_init(nullptr, 0)) return cudaErrorNotSupported;
+    if (!D && !d_hi) return cudaErrorInvalidValue;
     if (g_bk == 32)
-        return launch_bk<32>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word, s);
-    return launch_bk<16>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word, s);
+        return launch_bk<32>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word,
+                             d_hi, d_plane, s);
+    return launch_bk<16>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word, d_hi,
+                         d_plane, s);
 }
 
 }  // namespace bt

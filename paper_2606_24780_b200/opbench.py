@@ -103,6 +103,11 @@ def build_cases(B, T, C, H, Vp, n_params):
     cases["attention_fwd"] = dict(run=lambda: b.bt_op_attention_fwd(qkv, B, T, C, H, o, os_, lse), flops=afl,
                                   bytes=24.0 * N * C, bound="tensor", keep=(qkv, o, os_, lse))
     b.bt_op_attention_fwd(qkv, B, T, C, H, o, os_, lse)
+    if C // H == 64:
+        qkv_s = _split(qkv)
+        cases["attention_fwd_tcgen05"] = dict(
+            run=lambda: b.bt_op_attention_fwd(None, B, T, C, H, None, os_, lse, qkv_split=qkv_s), flops=afl,
+            bytes=32.0 * N * C, bound="tensor", keep=(qkv_s,))
     cases["attention_bwd"] = dict(
         run=lambda: b.bt_op_attention_bwd(qkv, o, lse, d_o, B, T, C, H, None, dqs, dv, dv.numel() * 4),
         flops=2.5 * afl, bytes=48.0 * N * C, bound="tensor", keep=(d_o, dqs, dv))

@@ -254,3 +254,24 @@ def test_attention_fwd_bwd(B, T, H, d, flags):
     for part in range(3):
         assert rel_l2(host(dqkv)[:, part * C:(part + 1) * C], rd[:, part * C:(part + 1) * C]) < 1e-4, part
     check_split(dqs, host(dqkv))
+
+
+@pytest.mark.parametrize("B,T,H", [(2, 200, 3), (1, 1024, 2), (1, 1, 2), (3, 129, 1), (1, 130, 12), (2, 64, 1), (1, 65, 1)])
+def test_attention_fwd_tcgen05_kernel(B, T, H):
+    """head_dim 64 with the qkv array given as hi/lo planes: the TMA + tcgen05 + TMEM kernel."""
+    d = 64
+    C = H * d
+    qkv = si.normal_f32(82, (B * T, 3 * C))
+    dq = dev(qkv)
+    qs = empty(2, B * T, 3 * C)
+    b.bt_op_split(dq, dq.numel(), qs)
+    o, os_, lse = empty(B * T, C), empty(2, B * T, C), empty(B, H, T)
+    b.bt_op_attention_fwd(None, B, T, C, H, o, os_, lse, 0, qkv_split=qs)
+    ro, rlse = oracle.attention_fwd(qkv, B, T, H)
+    assert rel_l2(host(o), ro) < 1e-4 and rel_max(host(o), ro) < 1e-4
+    assert np.abs(host(lse) - rlse).max() < 1e-4
+    check_split(os_, host(o))
+    # and it agrees with the warp-MMA kernel on the raw array
+    o2, lse2 = empty(B * T, C), empty(B, H, T)
+    b.bt_op_attention_fwd(dq, B, T, C, H, o2, None, lse2, 0)
+    assert rel_max(host(o), host(o2)) < 1e-5
