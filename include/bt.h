@@ -253,11 +253,14 @@ BT_API bt_status bt_op_attention_fwd(const float* qkv, const float* qkv_split, i
 
 /* Backward of the above with recomputed probabilities: dV = P^T do, dP = do V^T,
  * dS = P o (dP - rowsum(do o o)), dq = dS k / sqrt(d), dk = dS^T q / sqrt(d).
- * scratch: B*H*T floats. */
-BT_API bt_status bt_op_attention_bwd(const float* qkv, const float* o, const float* lse, const float* d_o,
-                                     int32_t B, int32_t T, int32_t C, int32_t H, float* dqkv,
-                                     float* dqkv_split, void* scratch, size_t scratch_bytes, uint32_t flags,
-                                     void* stream);
+ * scratch: B*H*T floats.  qkv and d_o may be given raw and/or as hi/lo planes (qkv_split
+ * [2][B*T][3C], d_o_split [2][B*T][C]); with both split inputs, d = 64 and only dqkv_split
+ * requested (dqkv NULL) the tcgen05 kernels run (they synchronise to report a device timeout),
+ * otherwise the warp-MMA kernels run on the raw arrays, which must then be given. */
+BT_API bt_status bt_op_attention_bwd(const float* qkv, const float* qkv_split, const float* o, const float* lse,
+                                     const float* d_o, const float* d_o_split, int32_t B, int32_t T, int32_t C,
+                                     int32_t H, float* dqkv, float* dqkv_split, void* scratch, size_t scratch_bytes,
+                                     uint32_t flags, void* stream);
 
 /* y = GELU(x) (exact erf form, or tanh form), n % 4 == 0. */
 BT_API bt_status bt_op_gelu_fwd(const float* x, int64_t n, int32_t tanh_form, float* y, float* y_split,

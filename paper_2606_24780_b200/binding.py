@@ -73,7 +73,7 @@ _SIGNATURES = {
     "bt_op_gemm_check": (_i32, [_vp, _vp]),
     "bt_op_gemm": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
     "bt_op_attention_fwd": (_i32, [_vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _u32, _vp]),
-    "bt_op_attention_bwd": (_i32, [_vp] * 4 + [_i32] * 4 + [_vp] * 3 + [_sz, _u32, _vp]),
+    "bt_op_attention_bwd": (_i32, [_vp] * 6 + [_i32] * 4 + [_vp] * 3 + [_sz, _u32, _vp]),
     "bt_op_gelu_fwd": (_i32, [_vp, _i64, _i32, _vp, _vp, _vp]),
     "bt_op_gelu_bwd": (_i32, [_vp, _vp, _i64, _i32, _vp, _vp, _vp]),
     "bt_op_softmax_xent": (_i32, [_vp, _vp, _i64, _i32, _f, _vp, _vp, _vp, _vp, _vp]),
@@ -310,9 +310,11 @@ def bt_op_attention_fwd(qkv, B, T, C, H, o, o_split, lse, flags=0, stream=None, 
                                      _stream(stream)))
 
 
-def bt_op_attention_bwd(qkv, o, lse, d_o, B, T, C, H, dqkv, dqkv_split, scratch, scratch_bytes, flags=0, stream=None):
-    _check(lib().bt_op_attention_bwd(_ptr(qkv), _ptr(o), _ptr(lse), _ptr(d_o), B, T, C, H, _ptr(dqkv),
-                                     _ptr(dqkv_split), _ptr(scratch), scratch_bytes, flags, _stream(stream)))
+def bt_op_attention_bwd(qkv, o, lse, d_o, B, T, C, H, dqkv, dqkv_split, scratch, scratch_bytes, flags=0, stream=None,
+                        qkv_split=None, d_o_split=None):
+    _check(lib().bt_op_attention_bwd(_ptr(qkv), _ptr(qkv_split), _ptr(o), _ptr(lse), _ptr(d_o), _ptr(d_o_split), B, T,
+                                     C, H, _ptr(dqkv), _ptr(dqkv_split), _ptr(scratch), scratch_bytes, flags,
+                                     _stream(stream)))
 
 
 def bt_op_gelu_fwd(x, n, tanh_form, y, y_split, stream=None):

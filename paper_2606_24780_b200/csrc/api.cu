@@ -109,7 +109,7 @@ struct bt_model {
     uint8_t* decay_flags;
     std::vector<LayerAct> act;
     float *xL, *meanf, *rstdf, *xf_s, *logits, *dlogits_s, *losses, *loss, *norm_out;
-    float *dres, *dres_s, *dtmp, *dqkv_s, *dh_s, *dg, *dvec;
+    float *dres, *dres_s, *dtmp, *do_s, *dqkv_s, *dh_s, *dg, *dvec;
     float *partials, *ln_scratch, *colsum_scratch;
     void* norm_scratch;
     size_t partial_floats;
@@ -216,6 +216,7 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->dres = b.take<float>(N * C);
     m->dres_s = b.take<float>(2 * N * C);
     m->dtmp = b.take<float>(N * C);
+    m->do_s = b.take<float>(2 * N * C);
     m->dqkv_s = b.take<float>(2 * N * 3 * C);
     m->dh_s = b.take<float>(2 * N * F);
     m->dg = b.take<float>(N * F);
@@ -588,11 +589,12 @@ extern "C" bt_status bt_backward(bt_model* m) {
         BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, a.x1, m->params + LT(LN2G).off, a.mean2, a.rstd2, m->dres, N, C, m->dres,
                                      m->dres_s, m->dres_s + N * C, G(LT(LN2G)), G(LT(LN2B)), m->ln_scratch, s));
         // attention output projection: x1 = x + o . Wo^T + bo
-        BT_GEMM(kNN, N, C, C, dres, weight_mat(m, LT(PROJW), C, C), m->dtmp, nullptr, nullptr);
+        // d o, raw for the FMA / warp-MMA attention kernels, as hi/lo planes for the tcgen05 ones
+        BT_GEMM_SPLIT_OUT(kNN, N, C, C, dres, weight_mat(m, LT(PROJW), C, C), m->dtmp, m->do_s, nullptr, nullptr);
         BT_GEMM(kTN, C, C, N, dres, act_mat(a.o_s, N, C, N), G(LT(PROJW)), nullptr, nullptr);
         BT_STEP(kCatColsum, 0, 4.0 * N * C, launch_colsum(m->dres, nullptr, N, C, G(LT(PROJB)), m->colsum_scratch, s));
-        BT_STEP(kCatAttnBwd, 2.5 * attn_fwd_flops(B, H, T, C / H), 48.0 * N * C, launch_attention_bwd(a.qkv, a.o_s, a.o_s + N * C, a.lse, m->dtmp, B, T, C, H, nullptr, m->dqkv_s,
-                                     m->dqkv_s + N * 3 * C, m->dvec, simt_attn, s));
+        BT_STEP(kCatAttnBwd, 2.5 * attn_fwd_flops(B, H, T, C / H), 48.0 * N * C, launch_attention_bwd(a.qkv, a.qkv_s, N * 3 * C, a.o_s, a.o_s + N * C, a.lse, m->dtmp, m->do_s, N * C, B, T,
+                                     C, H, nullptr, m->dqkv_s, m->dqkv_s + N * 3 * C, m->dvec, simt_attn, m->err_word, s));
         // QKV projection: qkv = a . Wqkv^T + bqkv
         SplitMat dqkv = act_mat(m->dqkv_s, N, 3 * C, N);
         BT_GEMM(kNN, N, C, 3 * C, dqkv, weight_mat(m, LT(QKVW), 3 * C, C), m->dtmp, nullptr, nullptr);
@@ -818,17 +820,37 @@ extern "C" bt_status bt_op_attention_fwd(const float* qkv, const float* qkv_spli
     return BT_OK;
 }
 
-extern "C" bt_status bt_op_attention_bwd(const float* qkv, const float* o, const float* lse, const float* d_o,
-                                         int32_t B, int32_t T, int32_t C, int32_t H, float* dqkv, float* dqkv_split,
-                                         void* scratch, size_t scratch_bytes, uint32_t flags, void* stream) {
-    BT_PTR(qkv); BT_PTR(o); BT_PTR(lse); BT_PTR(d_o); BT_OPT_PTR(dqkv); BT_OPT_PTR(dqkv_split); BT_PTR(scratch);
+extern "C" bt_status bt_op_attention_bwd(const float* qkv, const float* qkv_split, const float* o, const float* lse,
+                                         const float* d_o, const float* d_o_split, int32_t B, int32_t T, int32_t C,
+                                         int32_t H, float* dqkv, float* dqkv_split, void* scratch,
+                                         size_t scratch_bytes, uint32_t flags, void* stream) {
+    BT_OPT_PTR(qkv); BT_OPT_PTR(qkv_split); BT_PTR(o); BT_PTR(lse); BT_OPT_PTR(d_o); BT_OPT_PTR(d_o_split);
+    BT_OPT_PTR(dqkv); BT_OPT_PTR(dqkv_split); BT_PTR(scratch);
     if (B < 1 || T < 1 || C < 1 || H < 1 || C % H) return fail(BT_ERR_INVALID_ARG, "attention_bwd: bad sizes");
     int d = C / H;
     if (d != 16 && d != 32 && d != 64 && d != 128) return fail(BT_ERR_UNSUPPORTED, "attention: head_dim %d", d);
     if (scratch_bytes < (size_t)B * H * T * sizeof(float)) return fail(BT_ERR_OOM, "attention_bwd: scratch too small");
-    BT_CUDA(launch_attention_bwd(qkv, o, nullptr, lse, d_o, B, T, C, H, dqkv, dqkv_split,
-                                 dqkv_split ? dqkv_split + (int64_t)B * T * 3 * C : nullptr, (float*)scratch,
-                                 (flags & BT_FLAG_ATTN_SIMT) != 0, (cudaStream_t)stream));
+    if (!dqkv && !dqkv_split) return fail(BT_ERR_INVALID_ARG, "attention_bwd: no output requested");
+    const bool simt = (flags & BT_FLAG_ATTN_SIMT) != 0;
+    const bool tc = !simt && qkv_split && d_o_split && dqkv_split && !dqkv && d == 64;
+    if (!tc && (!qkv || !d_o)) return fail(BT_ERR_INVALID_ARG, "attention_bwd: this kernel needs the raw qkv and d_o arrays");
+    int* err = nullptr;
+    cudaStream_t s = (cudaStream_t)stream;
+    if (tc) {
+        char msg[256];
+        if (!gemm_tc_init(msg, sizeof(msg))) return fail(BT_ERR_CUDA, "tensor-core attention unavailable: %s", msg);
+        BT_CUDA(attention_tc_default_err(&err));
+        BT_CUDA(cudaMemsetAsync(err, 0, sizeof(int), s));
+    }
+    const int64_t n = (int64_t)B * T;
+    BT_CUDA(launch_attention_bwd(qkv, qkv_split, n * 3 * C, o, nullptr, lse, d_o, d_o_split, n * C, B, T, C, H, dqkv,
+                                 dqkv_split, dqkv_split ? dqkv_split + n * 3 * C : nullptr, (float*)scratch, simt, err, s));
+    if (err) {
+        int herr = 0;
+        BT_CUDA(cudaMemcpyAsync(&herr, err, sizeof(int), cudaMemcpyDeviceToHost, s));
+        BT_CUDA(cudaStreamSynchronize(s));
+        if (herr) return fail(BT_ERR_DEVICE_TIMEOUT, "attention_bwd: a bounded device-side wait ran out (code %d)", herr);
+    }
     return BT_OK;
 }
 

@@ -9,8 +9,11 @@ cudaError_t launch_attention_fwd_simt(const float* qkv, int B, int T, int C, int
 cudaError_t launch_attention_bwd_simt(const float* qkv, const float* o, const float* o_lo, const float* lse,
                                       const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
                                       float* dqkv_lo, float* dvec, cudaStream_t s);
-cudaError_t launch_attention_dvec(const float* o, const float* o_lo, const float* d_o, int B, int T, int C, int H,
-                                  float* dvec, cudaStream_t s);
+cudaError_t launch_attention_dvec(const float* o, const float* o_lo, const float* d_o, const float* d_o_lo, int B,
+                                  int T, int C, int H, float* dvec, cudaStream_t s);
+cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, const float* do_hi, int64_t do_plane,
+                                    const float* lse, const float* dvec, int B, int T, int C, int H, float* dqkv_hi,
+                                    int64_t dqkv_plane, int* err_word, cudaStream_t s);
 bool attention_mma_supports(int head_dim);
 cudaError_t launch_attention_fwd_mma(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi,
                                      float* o_lo, float* lse, cudaStream_t s);
@@ -34,12 +37,26 @@ cudaError_t launch_attention_fwd(const float* qkv, const float* qkv_hi, int64_t 
     return launch_attention_fwd_mma(qkv, B, T, C, H, o, o_hi, o_lo, lse, s);
 }
 
-cudaError_t launch_attention_bwd(const float* qkv, const float* o, const float* o_lo, const float* lse,
-                                 const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
-                                 float* dqkv_lo, float* dvec, bool simt, cudaStream_t s) {
+// Inputs may be given raw and/or as hi/lo planes (qkv_hi, do_hi; lo at +plane).  With head_dim 64,
+// both split inputs and only the split output requested, the tcgen05 kernels run; otherwise the
+// warp-MMA kernels run on the raw arrays.
+cudaError_t launch_attention_bwd(const float* qkv, const float* qkv_hi, int64_t qkv_plane, const float* o,
+                                 const float* o_lo, const float* lse, const float* d_o, const float* do_hi,
+                                 int64_t do_plane, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
+                                 float* dqkv_lo, float* dvec, bool simt, int* err_word, cudaStream_t s) {
+    const bool tc = !simt && qkv_hi && do_hi && dqkv_hi && !dqkv && attention_tc_supports(C / H, C) &&
+                    dqkv_lo == dqkv_hi + (int64_t)B * T * 3 * C;
+    if (tc) {
+        cudaError_t e = d_o ? launch_attention_dvec(o, o_lo, d_o, nullptr, B, T, C, H, dvec, s)
+                            : launch_attention_dvec(o, o_lo, do_hi, do_hi + do_plane, B, T, C, H, dvec, s);
+        if (e != cudaSuccess) return e;
+        return launch_attention_bwd_tc(qkv_hi, qkv_plane, do_hi, do_plane, lse, dvec, B, T, C, H, dqkv_hi,
+                                       (int64_t)B * T * 3 * C, err_word, s);
+    }
+    if (!qkv || !d_o) return cudaErrorInvalidValue;
     if (simt || !attention_mma_supports(C / H))
         return launch_attention_bwd_simt(qkv, o, o_lo, lse, d_o, B, T, C, H, dqkv, dqkv_hi, dqkv_lo, dvec, s);
-    cudaError_t e = launch_attention_dvec(o, o_lo, d_o, B, T, C, H, dvec, s);
+    cudaError_t e = launch_attention_dvec(o, o_lo, d_o, nullptr, B, T, C, H, dvec, s);
     if (e != cudaSuccess) return e;
     return launch_attention_bwd_mma(qkv, lse, d_o, dvec, B, T, C, H, dqkv, dqkv_hi, dqkv_lo, s);
 }

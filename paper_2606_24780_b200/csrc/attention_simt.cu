@@ -76,8 +76,9 @@ __global__ void __launch_bounds__(kAsWarps * 32) attn_fwd_simt_kernel(const floa
 template <int DPL>
 __global__ void __launch_bounds__(kAsWarps * 32) attn_dvec_kernel(const float* __restrict__ o,
                                                                    const float* __restrict__ o_lo,
-                                                                   const float* __restrict__ d_o, int B, int T, int C,
-                                                                   int H, float* __restrict__ dvec) {
+                                                                   const float* __restrict__ d_o,
+                                                                   const float* __restrict__ d_o_lo, int B, int T,
+                                                                   int C, int H, float* __restrict__ dvec) {
     const int lane = threadIdx.x & 31;
     const int64_t gw = (int64_t)blockIdx.x * kAsWarps + (threadIdx.x >> 5);
     if (gw >= (int64_t)B * H * T) return;
@@ -93,6 +94,12 @@ __global__ void __launch_bounds__(kAsWarps * 32) attn_dvec_kernel(const float* _
         for (int k = 0; k < DPL; ++k) a[k] += t[k];
     }
     load_vec<DPL>(d_o + row, d, lane, g);
+    if (d_o_lo) {
+        float t[DPL];
+        load_vec<DPL>(d_o_lo + row, d, lane, t);
+#pragma unroll
+        for (int k = 0; k < DPL; ++k) g[k] += t[k];
+    }
     float s = dot_vec<DPL>(a, g);
     if (lane == 0) dvec[gw] = s;
 }
@@ -190,14 +197,14 @@ cudaError_t launch_attention_fwd_simt(const float* qkv, int B, int T, int C, int
     return cudaGetLastError();
 }
 
-cudaError_t launch_attention_dvec(const float* o, const float* o_lo, const float* d_o, int B, int T, int C, int H,
-                                  float* dvec, cudaStream_t s) {
+cudaError_t launch_attention_dvec(const float* o, const float* o_lo, const float* d_o, const float* d_o_lo, int B,
+                                  int T, int C, int H, float* dvec, cudaStream_t s) {
     const int d = C / H;
     const int64_t warps = (int64_t)B * H * T;
     const int grid = (int)((warps + kAsWarps - 1) / kAsWarps);
-    if (d <= 32) attn_dvec_kernel<1><<<grid, kAsWarps * 32, 0, s>>>(o, o_lo, d_o, B, T, C, H, dvec);
-    else if (d <= 64) attn_dvec_kernel<2><<<grid, kAsWarps * 32, 0, s>>>(o, o_lo, d_o, B, T, C, H, dvec);
-    else attn_dvec_kernel<4><<<grid, kAsWarps * 32, 0, s>>>(o, o_lo, d_o, B, T, C, H, dvec);
+    if (d <= 32) attn_dvec_kernel<1><<<grid, kAsWarps * 32, 0, s>>>(o, o_lo, d_o, d_o_lo, B, T, C, H, dvec);
+    else if (d <= 64) attn_dvec_kernel<2><<<grid, kAsWarps * 32, 0, s>>>(o, o_lo, d_o, d_o_lo, B, T, C, H, dvec);
+    else attn_dvec_kernel<4><<<grid, kAsWarps * 32, 0, s>>>(o, o_lo, d_o, d_o_lo, B, T, C, H, dvec);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -205,7 +212,7 @@ cudaError_t launch_attention_dvec(const float* o, const float* o_lo, const float
 cudaError_t launch_attention_bwd_simt(const float* qkv, const float* o, const float* o_lo, const float* lse,
                                       const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
                                       float* dqkv_lo, float* dvec, cudaStream_t s) {
-    cudaError_t e = launch_attention_dvec(o, o_lo, d_o, B, T, C, H, dvec, s);
+    cudaError_t e = launch_attention_dvec(o, o_lo, d_o, nullptr, B, T, C, H, dvec, s);
     if (e != cudaSuccess) return e;
     const int d = C / H;
     const int64_t warps = (int64_t)B * H * T;

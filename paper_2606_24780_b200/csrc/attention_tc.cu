@@ -192,7 +192,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
         auto add_output = [&](int kt, float corr) -> bool {
             const int buf = kt & 1;
-            if (!mbar_wait(o_full(buf), (kt >> 1) & 1u, g.err, 17)) return false;
+            if (!mbar_wait_warp(o_full(buf), (kt >> 1) & 1u, g.err, 17)) return false;
             tc_fence_after();
             uint32_t r0[32], r1[32];
             tmem_ld32(t_lane + buf * 256u + 192u, r0);
@@ -208,7 +208,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
         for (int kt = 0; kt < n_kt && ok; ++kt) {
             const int buf = kt & 1;
-            if (!mbar_wait(s_full(buf), (kt >> 1) & 1u, g.err, 18)) { ok = false; break; }
+            if (!mbar_wait_warp(s_full(buf), (kt >> 1) & 1u, g.err, 18)) { ok = false; break; }
             tc_fence_after();
             uint32_t s0[32], s1[32];
             tmem_ld32(t_lane + buf * 256u, s0);

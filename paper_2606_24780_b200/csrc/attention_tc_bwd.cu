@@ -1,0 +1,560 @@
+// Causal flash attention backward on the 5th-generation tensor cores (head_dim 64), 3xTF32.
+//
+// Two deterministic kernels (no atomics) that recompute the probabilities from (q, k, lse):
+//
+//   dkv kernel  one CTA owns 128 keys (one per TMEM lane) of one (sequence, head) and walks the
+//               32-row query tiles at or below the diagonal:
+//                 S^T  = K' Q^T      A = K' (pre-scaled, hi/lo) held in TENSOR MEMORY, B = Q tile (smem)
+//                 dP^T = V  dO^T     A = V (smem, resident),                           B = dO tile
+//                 P^T  = exp2(S^T - lse),  dS^T = P^T o (dP^T - D)       (thread = key row)
+//                 dV  += P^T  dO     A = P^T  (hi/lo written back to tensor memory),   B = dO tile
+//                 dK  += dS^T Q      A = dS^T (tensor memory),                          B = Q tile
+//               dK and dV accumulate in tensor memory over the whole walk (the backward needs no
+//               running-max rescaling).
+//   dq kernel   one CTA owns 128 query rows and walks the 32-key tiles up to the diagonal:
+//                 S  = Q' K^T (A = Q' in tensor memory),  dP = dO V^T (A = dO resident in smem),
+//                 dS = P o (dP - D),  dQ += dS K (A = dS in tensor memory).
+//
+// Streamed tiles arrive by TMA as hi/lo planes in the two shared-memory layouts the tensor core
+// needs: K-major (128-byte swizzle) where the tile is the B operand of a "row . row" product, and
+// MN-major (128-byte swizzle, 32-byte atoms) where its rows are the contraction index.  The two
+// layouts have their own full/empty barriers, so a tile's K-major half is refilled as soon as the
+// first pair of products has consumed it.  Score/gradient buffers in tensor memory are double
+// buffered: the products of tile t+1 are issued before the accumulating products of tile t, so
+// the tensor pipe runs while the 128 element-wise threads work.
+// Every mbarrier wait is bounded and reports through the device error word.
+#include "common.cuh"
+#include "tc_common.cuh"
+
+namespace bt {
+
+using namespace tc;
+
+namespace {
+
+constexpr int HD = 64, BR = 128, BT_ = 32;  // head dim, rows owned by the CTA, streamed tile rows
+constexpr int kThreads = 192;
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr uint32_t kResBytes = 2u * 2u * BR * 128u;   // resident 128-row operand: 2 k-blocks x (hi,lo)
+constexpr uint32_t kTileBytes = 2u * 2u * BT_ * 128u; // one streamed 32-row tile in one layout (16 KB)
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Thread-owned row (64 floats given as hi/lo planes) -> x * mul -> hi/lo columns of tensor memory.
+__device__ __forceinline__ void row_to_tmem(const float* hi_row, const float* lo_row, float mul, uint32_t t_hi,
+                                            uint32_t t_lo) {
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        uint32_t h[32], l[32];
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            const float4 a = *reinterpret_cast<const float4*>(hi_row + half * 32 + i);
+            const float4 b = *reinterpret_cast<const float4*>(lo_row + half * 32 + i);
+            const float x[4] = {(a.x + b.x) * mul, (a.y + b.y) * mul, (a.z + b.z) * mul, (a.w + b.w) * mul};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float fh, fl;
+                split_tf32(x[e], fh, fl);
+                h[i + e] = __float_as_uint(fh);
+                l[i + e] = __float_as_uint(fl);
+            }
+        }
+        tmem_st32(t_hi + half * 32, h);
+        tmem_st32(t_lo + half * 32, l);
+    }
+    tmem_st_wait();
+}
+
+// Thread-owned accumulator row (64 tensor-memory columns) * mul -> hi/lo planes in global memory.
+// The tensor-memory loads are .sync.aligned: EVERY lane of the warp must call this; `store` says
+// whether this lane's row exists (rows past the end of the sequence are read and dropped).
+__device__ __forceinline__ void tmem_row_to_split(uint32_t t_row, float mul, float* hi_row, float* lo_row,
+                                                  bool store) {
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        uint32_t r[32];
+        tmem_ld32(t_row + half * 32, r);
+        tmem_ld_wait();
+        if (!store) continue;
+#pragma unroll
+        for (int i = 0; i < 32; i += 4) {
+            float4 v = make_float4(__uint_as_float(r[i]) * mul, __uint_as_float(r[i + 1]) * mul,
+                                   __uint_as_float(r[i + 2]) * mul, __uint_as_float(r[i + 3]) * mul);
+            float4 h, l;
+            split_tf32(v, h, l);
+            *reinterpret_cast<float4*>(hi_row + half * 32 + i) = h;
+            *reinterpret_cast<float4*>(lo_row + half * 32 + i) = l;
+        }
+    }
+}
+
+// Descriptors of one 8-deep k-step.
+//  K-major tile (rows x 64 floats as 2 k-blocks of [hi|lo][rows][128 B]), contraction over d.
+__device__ __forceinline__ uint64_t kmaj_desc(uint32_t tile, int rows, int ks, bool lo) {
+    const uint32_t kb_bytes = 2u * (uint32_t)rows * 128u;
+    const uint32_t addr = tile + (uint32_t)(ks >> 2) * kb_bytes + (lo ? (uint32_t)rows * 128u : 0u) + (uint32_t)(ks & 3) * 32u;
+    return make_desc(addr, 16u, 1024u, 2u);
+}
+//  MN-major 32-row tile (2 column groups of [hi|lo][32 rows][128 B]), contraction over the rows.
+__device__ __forceinline__ uint64_t mnmaj_desc(uint32_t tile, int ks, bool lo) {
+    const uint32_t addr = tile + (lo ? BT_ * 128u : 0u) + (uint32_t)ks * 1024u;
+    return make_desc(addr, 2u * BT_ * 128u, 512u, 1u);
+}
+
+struct BwdArgs {
+    int T, C, H;
+    const float* qkv_hi;      // split qkv [2][B*T][3C]
+    long long qkv_plane;
+    const float* lse;
+    const float* dvec;
+    float* dqkv_hi;           // split output [2][B*T][3C]
+    long long dqkv_plane;
+    int* err;
+};
+
+// Shared prologue: barriers + TMEM allocation.  Returns the TMEM base address.
+__device__ __forceinline__ uint32_t setup(uint32_t bars, int n_bars_count1, uint32_t p_bar0, int n_p_bars,
+                                          uint32_t tmem_slot, uint8_t* smem_raw, int warp) {
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < n_bars_count1; ++i) mbar_init(bars + 8u * i, 1);
+        for (int i = 0; i < n_p_bars; ++i) mbar_init(p_bar0 + 8u * i, 4);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    return *reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+}
+
+// ------------------------------------------------------------------------------------------ dkv
+
+constexpr uint32_t kDkvSmem = 1024u + kResBytes + 2u * 4u * kTileBytes + 1024u;
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_constant__ CUtensorMap tmQm,
+                       const __grid_constant__ CUtensorMap tmDOk, const __grid_constant__ CUtensorMap tmDOm,
+                       const __grid_constant__ CUtensorMap tmVres, const BwdArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t v_s = base;                                  // resident V (A operand of dP^T)
+    auto qk_s = [&](int st) { return base + kResBytes + (uint32_t)st * 4u * kTileBytes; };
+    auto dok_s = [&](int st) { return qk_s(st) + kTileBytes; };
+    auto qm_s = [&](int st) { return qk_s(st) + 2u * kTileBytes; };
+    auto dom_s = [&](int st) { return qk_s(st) + 3u * kTileBytes; };
+    const uint32_t bars = base + kResBytes + 8u * kTileBytes;
+    // count-1 barriers: 0 v_full, 1-2 kfull, 3-4 kempty, 5-6 mfull, 7-8 mempty, 9-10 sdp_full, 11 acc_full
+    const uint32_t v_full = bars;
+    auto kfull = [&](int s) { return bars + 8u * (1 + s); };
+    auto kempty = [&](int s) { return bars + 8u * (3 + s); };
+    auto mfull = [&](int s) { return bars + 8u * (5 + s); };
+    auto mempty = [&](int s) { return bars + 8u * (7 + s); };
+    auto sdp_full = [&](int b) { return bars + 8u * (9 + b); };
+    const uint32_t acc_full = bars + 8u * 11;
+    // count-4 barriers: 12-13 pds_full, 14 k_ready
+    auto pds_full = [&](int b) { return bars + 8u * (12 + b); };
+    const uint32_t k_ready = bars + 8u * 14;
+    const uint32_t tmem_slot = bars + 8u * 15;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int b = blockIdx.y / g.H, h = blockIdx.y % g.H;
+    const int j0 = blockIdx.x * BR;
+    const int row_base = b * g.T;
+    const int n_qt = (g.T + BT_ - 1) / BT_, qt0 = j0 / BT_;
+    const int n_t = n_qt - qt0;
+
+    const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp);
+    // TMEM columns
+    const uint32_t tK_hi = tmem, tK_lo = tmem + 64, tdK = tmem + 128, tdV = tmem + 192;
+    auto tbuf = [&](int bb) { return tmem + 256u + 128u * (uint32_t)bb; };  // +0 S^T|P^T_hi, +32 P^T_lo, +64 dP^T|dS^T_hi, +96 dS^T_lo
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_expect_tx(v_full, kResBytes);
+            for (int kb = 0; kb < 2; ++kb)
+                tma_load_3d(v_s + kb * (kResBytes / 2), &tmVres, v_full, 2 * g.C + h * HD + kb * 32, row_base + j0, 0);
+            bool ok = true;
+            for (int t = 0; t < n_t && ok; ++t) {
+                const int st = t & 1, q0 = (qt0 + t) * BT_;
+                const uint32_t ph = (t >> 1) & 1u;
+                if (!mbar_wait(kempty(st), ph ^ 1u, g.err, 21)) { ok = false; break; }
+                mbar_expect_tx(kfull(st), 2u * kTileBytes);
+                for (int kb = 0; kb < 2; ++kb) {
+                    tma_load_3d(qk_s(st) + kb * (kTileBytes / 2), &tmQk, kfull(st), h * HD + kb * 32, row_base + q0, 0);
+                    tma_load_3d(dok_s(st) + kb * (kTileBytes / 2), &tmDOk, kfull(st), h * HD + kb * 32, row_base + q0, 0);
+                }
+                if (!mbar_wait(mempty(st), ph ^ 1u, g.err, 22)) { ok = false; break; }
+                mbar_expect_tx(mfull(st), 2u * kTileBytes);
+                for (int grp = 0; grp < 2; ++grp) {
+                    tma_load_3d(qm_s(st) + grp * (kTileBytes / 2), &tmQm, mfull(st), h * HD + grp * 32, row_base + q0, 0);
+                    tma_load_3d(dom_s(st) + grp * (kTileBytes / 2), &tmDOm, mfull(st), h * HD + grp * 32, row_base + q0, 0);
+                }
+            }
+            if (!ok)
+                for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT_, false, false);   // 128 x 32, B K-major
+            constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
+            bool ok = mbar_wait(v_full, 0, g.err, 23) && mbar_wait(k_ready, 0, g.err, 24);
+            auto issue_a = [&](int t) -> bool {
+                const int st = t & 1, bb = t & 1;
+                if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 25)) return false;
+                tc_fence_after();
+                const uint32_t dS = tbuf(bb), dP = tbuf(bb) + 64u;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t q_hi = kmaj_desc(qk_s(st), BT_, ks, false), q_lo = kmaj_desc(qk_s(st), BT_, ks, true);
+                    umma_tf32_ts(dS, tK_lo + ks * 8, q_hi, idesc_a, ks > 0 ? 1u : 0u);
+                    umma_tf32_ts(dS, tK_hi + ks * 8, q_lo, idesc_a, 1u);
+                    umma_tf32_ts(dS, tK_hi + ks * 8, q_hi, idesc_a, 1u);
+                }
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t v_hi = kmaj_desc(v_s, BR, ks, false), v_lo = kmaj_desc(v_s, BR, ks, true);
+                    const uint64_t o_hi = kmaj_desc(dok_s(st), BT_, ks, false), o_lo = kmaj_desc(dok_s(st), BT_, ks, true);
+                    umma_tf32(dP, v_lo, o_hi, idesc_a, ks > 0 ? 1u : 0u);
+                    umma_tf32(dP, v_hi, o_lo, idesc_a, 1u);
+                    umma_tf32(dP, v_hi, o_hi, idesc_a, 1u);
+                }
+                umma_commit(kempty(st));
+                umma_commit(sdp_full(bb));
+                return true;
+            };
+            auto issue_b = [&](int t) -> bool {
+                const int st = t & 1, bb = t & 1;
+                if (!mbar_wait(pds_full(bb), (t >> 1) & 1u, g.err, 26)) return false;
+                if (!mbar_wait(mfull(st), (t >> 1) & 1u, g.err, 27)) return false;
+                tc_fence_after();
+                const uint32_t p_hi = tbuf(bb), p_lo = tbuf(bb) + 32u, s_hi = tbuf(bb) + 64u, s_lo = tbuf(bb) + 96u;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t o_hi = mnmaj_desc(dom_s(st), ks, false), o_lo = mnmaj_desc(dom_s(st), ks, true);
+                    const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
+                    umma_tf32_ts(tdV, p_lo + ks * 8, o_hi, idesc_b, acc);
+                    umma_tf32_ts(tdV, p_hi + ks * 8, o_lo, idesc_b, 1u);
+                    umma_tf32_ts(tdV, p_hi + ks * 8, o_hi, idesc_b, 1u);
+                }
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t q_hi = mnmaj_desc(qm_s(st), ks, false), q_lo = mnmaj_desc(qm_s(st), ks, true);
+                    const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
+                    umma_tf32_ts(tdK, s_lo + ks * 8, q_hi, idesc_b, acc);
+                    umma_tf32_ts(tdK, s_hi + ks * 8, q_lo, idesc_b, 1u);
+                    umma_tf32_ts(tdK, s_hi + ks * 8, q_hi, idesc_b, 1u);
+                }
+                umma_commit(mempty(st));
+                return true;
+            };
+            if (ok && n_t > 0) ok = issue_a(0);
+            for (int t = 0; t < n_t && ok; ++t) {
+                if (t + 1 < n_t) ok = issue_a(t + 1);
+                if (ok) ok = issue_b(t);
+            }
+            if (ok) umma_commit(acc_full);
+        }
+    } else {
+        const int lane_group = warp & 3;
+        const int etid = lane_group * 32 + lane;          // 0..127: row owned inside the CTA
+        const int key = j0 + etid;
+        const uint32_t t_lane = ((uint32_t)(lane_group * 32) << 16);
+        const float scale = 1.0f / sqrtf((float)HD);
+        const int64_t gs = 3 * (int64_t)g.C;
+        const int64_t lb = ((int64_t)b * g.H + h) * g.T;
+        {   // K' = K * scale * log2(e) into tensor memory
+            const int64_t off = (int64_t)(row_base + min(key, g.T - 1)) * gs + g.C + h * HD;
+            row_to_tmem(g.qkv_hi + off, g.qkv_hi + g.qkv_plane + off, scale * kLog2e, tK_hi + t_lane, tK_lo + t_lane);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(k_ready);
+        }
+        bool ok = true;
+        for (int t = 0; t < n_t && ok; ++t) {
+            const int bb = t & 1, q0 = (qt0 + t) * BT_;
+            // per-column softmax statistics of this query tile (same addresses in every thread:
+            // broadcast loads); rows past the sequence end get lse = +inf, i.e. probability 0
+            const int nvalid = min(BT_, g.T - q0);
+            const float* lse_t = g.lse + lb + q0;
+            const float* d_t = g.dvec + lb + q0;
+            if (!mbar_wait_warp(sdp_full(bb), (t >> 1) & 1u, g.err, 28)) { ok = false; break; }
+            tc_fence_after();
+            uint32_t s[32], dp[32];
+            tmem_ld32(tbuf(bb) + t_lane, s);
+            tmem_ld32(tbuf(bb) + 64u + t_lane, dp);
+            tmem_ld_wait();
+            uint32_t p_hi[32], p_lo[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const bool live = (i < nvalid) && (q0 + i >= key);   // in the sequence and not before this key
+                const float Li = live ? __ldg(lse_t + i) * kLog2e : 0.f;
+                const float Di = live ? __ldg(d_t + i) : 0.f;
+                const float p = live ? ex2_approx(__uint_as_float(s[i]) - Li) : 0.f;
+                const float ds = p * (__uint_as_float(dp[i]) - Di);
+                float fh, fl;
+                split_tf32(p, fh, fl);
+                p_hi[i] = __float_as_uint(fh);
+                p_lo[i] = __float_as_uint(fl);
+                split_tf32(ds, fh, fl);
+                s[i] = __float_as_uint(fh);                      // reuse: dS^T hi
+                dp[i] = __float_as_uint(fl);                     //        dS^T lo
+            }
+            tmem_st32(tbuf(bb) + t_lane, p_hi);
+            tmem_st32(tbuf(bb) + 32u + t_lane, p_lo);
+            tmem_st32(tbuf(bb) + 64u + t_lane, s);
+            tmem_st32(tbuf(bb) + 96u + t_lane, dp);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pds_full(bb));
+        }
+        if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 29);
+        if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
+            tc_fence_after();
+            const bool valid = key < g.T;
+            const int64_t off = (int64_t)(row_base + (valid ? key : 0)) * gs + h * HD;
+            float* hi = g.dqkv_hi + off;
+            float* lo = hi + g.dqkv_plane;
+            tmem_row_to_split(tdK + t_lane, scale, hi + g.C, lo + g.C, valid);
+            tmem_row_to_split(tdV + t_lane, 1.0f, hi + 2 * g.C, lo + 2 * g.C, valid);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
+// ------------------------------------------------------------------------------------------- dq
+
+constexpr uint32_t kDqSmem = 1024u + kResBytes + 2u * 3u * kTileBytes + 256u;
+
+__global__ void __launch_bounds__(kThreads, 1)
+attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_constant__ CUtensorMap tmKm,
+                      const __grid_constant__ CUtensorMap tmVk, const __grid_constant__ CUtensorMap tmDOres,
+                      const BwdArgs g) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t do_s = base;                                 // resident dO (A operand of dP)
+    auto kk_s = [&](int st) { return base + kResBytes + (uint32_t)st * 3u * kTileBytes; };
+    auto vk_s = [&](int st) { return kk_s(st) + kTileBytes; };
+    auto km_s = [&](int st) { return kk_s(st) + 2u * kTileBytes; };
+    const uint32_t bars = base + kResBytes + 6u * kTileBytes;
+    // count-1: 0 do_full, 1-2 kfull, 3-4 kempty, 5-6 mfull, 7-8 mempty, 9-10 sdp_full, 11 acc_full
+    const uint32_t do_full = bars;
+    auto kfull = [&](int s) { return bars + 8u * (1 + s); };
+    auto kempty = [&](int s) { return bars + 8u * (3 + s); };
+    auto mfull = [&](int s) { return bars + 8u * (5 + s); };
+    auto mempty = [&](int s) { return bars + 8u * (7 + s); };
+    auto sdp_full = [&](int b) { return bars + 8u * (9 + b); };
+    const uint32_t acc_full = bars + 8u * 11;
+    // count-4: 12-13 ds_full, 14 q_ready
+    auto ds_full = [&](int b) { return bars + 8u * (12 + b); };
+    const uint32_t q_ready = bars + 8u * 14;
+    const uint32_t tmem_slot = bars + 8u * 15;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int qt = gridDim.x - 1 - blockIdx.x;                  // heaviest query tiles first
+    const int b = blockIdx.y / g.H, h = blockIdx.y % g.H;
+    const int q0 = qt * BR;
+    const int row_base = b * g.T;
+    const int n_t = min(q0 + BR - 1, g.T - 1) / BT_ + 1;         // key tiles up to the diagonal
+
+    const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp);
+    const uint32_t tQ_hi = tmem, tQ_lo = tmem + 64, tdQ = tmem + 128;
+    auto tbuf = [&](int bb) { return tmem + 192u + 96u * (uint32_t)bb; };   // +0 S|dS_hi, +32 dS_lo, +64 dP
+
+    if (warp == 0) {
+        if (lane == 0) {
+            mbar_expect_tx(do_full, kResBytes);
+            for (int kb = 0; kb < 2; ++kb)
+                tma_load_3d(do_s + kb * (kResBytes / 2), &tmDOres, do_full, h * HD + kb * 32, row_base + q0, 0);
+            bool ok = true;
+            for (int t = 0; t < n_t && ok; ++t) {
+                const int st = t & 1, k0 = t * BT_;
+                const uint32_t ph = (t >> 1) & 1u;
+                if (!mbar_wait(kempty(st), ph ^ 1u, g.err, 31)) { ok = false; break; }
+                mbar_expect_tx(kfull(st), 2u * kTileBytes);
+                for (int kb = 0; kb < 2; ++kb) {
+                    tma_load_3d(kk_s(st) + kb * (kTileBytes / 2), &tmKk, kfull(st), g.C + h * HD + kb * 32, row_base + k0, 0);
+                    tma_load_3d(vk_s(st) + kb * (kTileBytes / 2), &tmVk, kfull(st), 2 * g.C + h * HD + kb * 32, row_base + k0, 0);
+                }
+                if (!mbar_wait(mempty(st), ph ^ 1u, g.err, 32)) { ok = false; break; }
+                mbar_expect_tx(mfull(st), kTileBytes);
+                for (int grp = 0; grp < 2; ++grp)
+                    tma_load_3d(km_s(st) + grp * (kTileBytes / 2), &tmKm, mfull(st), g.C + h * HD + grp * 32, row_base + k0, 0);
+            }
+            if (!ok)
+                for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT_, false, false);
+            constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);
+            bool ok = mbar_wait(do_full, 0, g.err, 33) && mbar_wait(q_ready, 0, g.err, 34);
+            auto issue_a = [&](int t) -> bool {
+                const int st = t & 1, bb = t & 1;
+                if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 35)) return false;
+                tc_fence_after();
+                const uint32_t dS = tbuf(bb), dP = tbuf(bb) + 64u;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t k_hi = kmaj_desc(kk_s(st), BT_, ks, false), k_lo = kmaj_desc(kk_s(st), BT_, ks, true);
+                    umma_tf32_ts(dS, tQ_lo + ks * 8, k_hi, idesc_a, ks > 0 ? 1u : 0u);
+                    umma_tf32_ts(dS, tQ_hi + ks * 8, k_lo, idesc_a, 1u);
+                    umma_tf32_ts(dS, tQ_hi + ks * 8, k_hi, idesc_a, 1u);
+                }
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t o_hi = kmaj_desc(do_s, BR, ks, false), o_lo = kmaj_desc(do_s, BR, ks, true);
+                    const uint64_t v_hi = kmaj_desc(vk_s(st), BT_, ks, false), v_lo = kmaj_desc(vk_s(st), BT_, ks, true);
+                    umma_tf32(dP, o_lo, v_hi, idesc_a, ks > 0 ? 1u : 0u);
+                    umma_tf32(dP, o_hi, v_lo, idesc_a, 1u);
+                    umma_tf32(dP, o_hi, v_hi, idesc_a, 1u);
+                }
+                umma_commit(kempty(st));
+                umma_commit(sdp_full(bb));
+                return true;
+            };
+            auto issue_b = [&](int t) -> bool {
+                const int st = t & 1, bb = t & 1;
+                if (!mbar_wait(ds_full(bb), (t >> 1) & 1u, g.err, 36)) return false;
+                if (!mbar_wait(mfull(st), (t >> 1) & 1u, g.err, 37)) return false;
+                tc_fence_after();
+                const uint32_t s_hi = tbuf(bb), s_lo = tbuf(bb) + 32u;
+#pragma unroll
+                for (int ks = 0; ks < 4; ++ks) {
+                    const uint64_t k_hi = mnmaj_desc(km_s(st), ks, false), k_lo = mnmaj_desc(km_s(st), ks, true);
+                    const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
+                    umma_tf32_ts(tdQ, s_lo + ks * 8, k_hi, idesc_b, acc);
+                    umma_tf32_ts(tdQ, s_hi + ks * 8, k_lo, idesc_b, 1u);
+                    umma_tf32_ts(tdQ, s_hi + ks * 8, k_hi, idesc_b, 1u);
+                }
+                umma_commit(mempty(st));
+                return true;
+            };
+            if (ok) ok = issue_a(0);
+            for (int t = 0; t < n_t && ok; ++t) {
+                if (t + 1 < n_t) ok = issue_a(t + 1);
+                if (ok) ok = issue_b(t);
+            }
+            if (ok) umma_commit(acc_full);
+        }
+    } else {
+        const int lane_group = warp & 3;
+        const int row = q0 + lane_group * 32 + lane;
+        const uint32_t t_lane = ((uint32_t)(lane_group * 32) << 16);
+        const float scale = 1.0f / sqrtf((float)HD);
+        const int64_t gs = 3 * (int64_t)g.C;
+        const int64_t lb = ((int64_t)b * g.H + h) * g.T;
+        const int rc = min(row, g.T - 1);
+        {
+            const int64_t off = (int64_t)(row_base + rc) * gs + h * HD;
+            row_to_tmem(g.qkv_hi + off, g.qkv_hi + g.qkv_plane + off, scale * kLog2e, tQ_hi + t_lane, tQ_lo + t_lane);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(q_ready);
+        }
+        const float L = g.lse[lb + rc] * kLog2e, D = g.dvec[lb + rc];
+        bool ok = true;
+        for (int t = 0; t < n_t && ok; ++t) {
+            const int bb = t & 1, k0 = t * BT_;
+            if (!mbar_wait_warp(sdp_full(bb), (t >> 1) & 1u, g.err, 38)) { ok = false; break; }
+            tc_fence_after();
+            uint32_t s[32], dp[32];
+            tmem_ld32(tbuf(bb) + t_lane, s);
+            tmem_ld32(tbuf(bb) + 64u + t_lane, dp);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                float p = ex2_approx(__uint_as_float(s[i]) - L);
+                if (k0 + i > row) p = 0.f;                      // key follows this query: masked
+                const float ds = p * (__uint_as_float(dp[i]) - D);
+                float fh, fl;
+                split_tf32(ds, fh, fl);
+                s[i] = __float_as_uint(fh);
+                dp[i] = __float_as_uint(fl);
+            }
+            tmem_st32(tbuf(bb) + t_lane, s);
+            tmem_st32(tbuf(bb) + 32u + t_lane, dp);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(ds_full(bb));
+        }
+        if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 39);
+        if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
+            tc_fence_after();
+            const int64_t off = (int64_t)(row_base + rc) * gs + h * HD;
+            tmem_row_to_split(tdQ + t_lane, scale, g.dqkv_hi + off, g.dqkv_hi + g.dqkv_plane + off, row < g.T);
+        }
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
+    }
+}
+
+bool enc3(CUtensorMap* tm, const float* base, int64_t cols, int64_t rows, int64_t plane, uint32_t box_rows,
+          bool mn_major) {
+    EncodeTiledFn enc = tensor_map_encoder();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)cols, (cuuint64_t)rows, 2};
+    cuuint64_t strides[2] = {(cuuint64_t)cols * 4, (cuuint64_t)plane * 4};
+    cuuint32_t box[3] = {32, box_rows, 2};
+    cuuint32_t estr[3] = {1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, (void*)base, dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE,
+               mn_major ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+cudaError_t attention_tc_default_err(int** out);
+
+// dqkv (hi/lo planes) from qkv (hi/lo planes), dO (hi/lo planes), lse and dvec = rowsum(dO o O).
+cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, const float* do_hi, int64_t do_plane,
+                                    const float* lse, const float* dvec, int B, int T, int C, int H, float* dqkv_hi,
+                                    int64_t dqkv_plane, int* err_word, cudaStream_t s) {
+    static cudaError_t attr = []() {
+        cudaError_t e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)kDkvSmem);
+        if (e == cudaSuccess)
+            e = cudaFuncSetAttribute(attn_bwd_dq_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kDqSmem);
+        return e;
+    }();
+    if (attr != cudaSuccess) return attr;
+    if (!err_word) {
+        cudaError_t e = attention_tc_default_err(&err_word);
+        if (e != cudaSuccess) return e;
+    }
+    const int64_t rows = (int64_t)B * T;
+    CUtensorMap qk32, qm32, dok32, dom32, vres, kres_unused, dores;
+    (void)kres_unused;
+    bool ok = enc3(&qk32, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BT_, false) &&   // 32-row K-major tiles of qkv
+              enc3(&qm32, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BT_, true) &&    // 32-row MN-major tiles of qkv
+              enc3(&dok32, do_hi, C, rows, do_plane, BT_, false) && enc3(&dom32, do_hi, C, rows, do_plane, BT_, true) &&
+              enc3(&vres, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BR, false) &&    // 128-row resident tiles
+              enc3(&dores, do_hi, C, rows, do_plane, BR, false);
+    if (!ok) return cudaErrorInvalidValue;
+    BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dqkv_hi, dqkv_plane, err_word};
+    dim3 gk((T + BR - 1) / BR, B * H);
+    attn_bwd_dkv_tc_kernel<<<gk, kThreads, kDkvSmem, s>>>(qk32, qm32, dok32, dom32, vres, g);
+    BT_COUNT_LAUNCH();
+    attn_bwd_dq_tc_kernel<<<gk, kThreads, kDqSmem, s>>>(qk32, qm32, qk32, dores, g);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+}  // namespace bt

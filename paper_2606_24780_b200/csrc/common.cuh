@@ -151,9 +151,11 @@ cudaError_t launch_attention_fwd(const float* qkv, const float* qkv_hi, int64_t 
                                  float* o, float* o_hi, float* o_lo, float* lse, bool simt, int* err_word,
                                  cudaStream_t s);
 cudaError_t attention_tc_default_err(int** out);
-// o given raw (o_lo == nullptr) or as hi/lo planes.  dvec: B*H*T floats of scratch.
-cudaError_t launch_attention_bwd(const float* qkv, const float* o, const float* o_lo, const float* lse,
-                                 const float* d_o, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
-                                 float* dqkv_lo, float* dvec, bool simt, cudaStream_t s);
+// o given raw (o_lo == nullptr) or as hi/lo planes.  dvec: B*H*T floats of scratch.  qkv and d_o may
+// be given raw and/or as hi/lo planes (see attention.cu for which kernel then runs).
+cudaError_t launch_attention_bwd(const float* qkv, const float* qkv_hi, int64_t qkv_plane, const float* o,
+                                 const float* o_lo, const float* lse, const float* d_o, const float* do_hi,
+                                 int64_t do_plane, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
+                                 float* dqkv_lo, float* dvec, bool simt, int* err_word, cudaStream_t s);
 
 }  // namespace bt

@@ -215,7 +215,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const int tm = u % g.tiles_m, r = u / g.tiles_m, tn = r % g.tiles_n, sp = r / g.tiles_n;
             const int acc = ut & 1;
             const uint32_t aph = (ut >> 1) & 1u;
-            if (!mbar_wait(tfull_bar(acc), aph, g.err, 4)) { ok = false; break; }
+            if (!mbar_wait_warp(tfull_bar(acc), aph, g.err, 4)) { ok = false; break; }
             tc_fence_after();
             const int row = tm * BM + lane_group * 32 + lane;
             float* Dp = g.D;

@@ -44,10 +44,17 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
         if (globaltimer_ns() - t0 > 1000000000ull) {
-            atomicExch(err, code);
+            atomicCAS(err, 0, code);  // the first wait that ran out is the one reported
             return false;
         }
     }
+}
+
+// The same wait made by a whole warp, with a warp-uniform result: the callers go on to issue
+// .sync.aligned tensor-memory instructions, which every lane of the warp must reach together.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* err, int code) {
+    const bool ok = mbar_wait(bar, parity, err, code);
+    return __all_sync(0xffffffffu, ok);
 }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* tm, uint32_t bar, int c0, int c1,

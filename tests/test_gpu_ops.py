@@ -275,3 +275,27 @@ def test_attention_fwd_tcgen05_kernel(B, T, H):
     o2, lse2 = empty(B * T, C), empty(B, H, T)
     b.bt_op_attention_fwd(dq, B, T, C, H, o2, None, lse2, 0)
     assert rel_max(host(o), host(o2)) < 1e-5
+
+
+@pytest.mark.parametrize("B,T,H", [(2, 200, 3), (1, 1024, 2), (1, 1, 2), (3, 129, 1), (1, 130, 12), (2, 64, 1), (1, 33, 1)])
+def test_attention_bwd_tcgen05_kernels(B, T, H):
+    """head_dim 64, qkv and d_o given as hi/lo planes, only the split gradient requested."""
+    d = 64
+    C = H * d
+    qkv = si.normal_f32(83, (B * T, 3 * C))
+    d_o = si.normal_f32(84, (B * T, C), 1e-2)
+    dq, ddo = dev(qkv), dev(d_o)
+    qs, dos = empty(2, B * T, 3 * C), empty(2, B * T, C)
+    b.bt_op_split(dq, dq.numel(), qs)
+    b.bt_op_split(ddo, ddo.numel(), dos)
+    o, lse = empty(B * T, C), empty(B, H, T)
+    b.bt_op_attention_fwd(None, B, T, C, H, o, None, lse, 0, qkv_split=qs)
+    dqs = zeros(2, B * T, 3 * C)
+    nb = B * H * T * 4
+    b.bt_op_attention_bwd(None, o, lse, None, B, T, C, H, None, dqs, scratch(nb), nb, 0, qkv_split=qs, d_o_split=dos)
+    got = host(dqs)
+    got = got[0] + got[1]
+    rd = oracle.attention_bwd(qkv, d_o, B, T, H)
+    for part in range(3):
+        assert rel_l2(got[:, part * C:(part + 1) * C], rd[:, part * C:(part + 1) * C]) < 1e-4, part
+    assert not (dqs[0].cpu().numpy().view(np.uint32) & 0x1FFF).any()
