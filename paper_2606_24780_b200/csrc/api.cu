@@ -936,3 +936,10 @@ extern "C" bt_status bt_op_adamw_multi(int32_t n_tensors, float* const* h_p, con
     BT_CUDA(launch_adamw_multi(tl, hp, d_scale, (cudaStream_t)stream));
     return BT_OK;
 }
+
+// Debug aid (not part of the public header): device buffer of 2 + 2*2000 uint64 that block (0,0)
+// of the tcgen05 attention forward kernel fills with (tag, SM clock) records; NULL switches it off.
+namespace bt { void attention_tc_set_trace(unsigned long long* p); }
+extern "C" __attribute__((visibility("default"))) void bt_debug_set_attention_trace(void* d_buffer) {
+    bt::attention_tc_set_trace(static_cast<unsigned long long*>(d_buffer));
+}

@@ -12,7 +12,8 @@
 //                      O_tile = P V: 24 MMAs with A = P (hi/lo) read from TENSOR MEMORY and B = V
 //                      from shared memory, accumulator O[buf] in TMEM.  S of tile t+1 is issued
 //                      before P V of tile t, so the tensor pipe works while the softmax runs.
-//   warps 2-5          softmax / correction: thread i owns query row i.  It reads its 64 scores
+//   warps 2-5, 6-9     two softmax / correction warpgroups taking alternate key tiles (buffer b
+//                      belongs to warpgroup b), merged at the end; in each, thread i owns query row i.  It reads its 64 scores
 //                      with tcgen05.ld (the row maximum and sum need no shuffles), forms
 //                      p = exp2((s - m) * scale*log2e), splits p into hi/lo and writes both back to
 //                      TMEM with tcgen05.st as the A operand of P V.  The running output is kept in
@@ -33,12 +34,18 @@ using namespace tc;
 namespace {
 
 constexpr int HD = 64, BQ = 128, BKV = 64;
-constexpr int kThreads = 192;
+constexpr int kThreads = 384;   // TMA warp, two MMA-issuing warps, a spare, two softmax warpgroups
 constexpr uint32_t kQBytes = 2u * 2u * BQ * 128u;      // 2 k-blocks x (hi, lo) x 128 rows x 128 B
 constexpr uint32_t kKVBytes = 2u * 2u * BKV * 128u;    // per buffer
 constexpr uint32_t kSmemBytes = 1024u + kQBytes + 4u * kKVBytes + 256u;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
 
 struct AttnArgs {
     int T, C, H;
@@ -47,7 +54,18 @@ struct AttnArgs {
     float* o_lo;
     float* lse;
     int* err;
+    unsigned long long* trace;   // optional timing trace of CTA (0,0) (debug aid, normally null)
 };
+
+// trace record: (tag, SM clock); only block (0,0) records
+__device__ __forceinline__ void trace_mark(unsigned long long* tr, unsigned long long tag) {
+    if (tr == nullptr || blockIdx.x != 0 || blockIdx.y != 0) return;
+    const unsigned long long i = atomicAdd(tr, 1ull);
+    if (i < 2000) {
+        tr[2 + 2 * i] = tag;
+        tr[3 + 2 * i] = clock64();
+    }
+}
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
@@ -67,7 +85,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     auto s_full = [&](int b) { return bars + 8u * (9 + b); };
     auto p_full = [&](int b) { return bars + 8u * (11 + b); };
     auto o_full = [&](int b) { return bars + 8u * (13 + b); };
-    const uint32_t tmem_slot = bars + 8u * 15;
+    const uint32_t merge_full = bars + 8u * 15;
+    const uint32_t all_done = bars + 8u * 16;
+    const uint32_t tmem_slot = bars + 8u * 17;
     volatile uint32_t* tmem_slot_ptr =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
@@ -90,6 +110,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             mbar_init(p_full(i), 4);
             mbar_init(o_full(i), 1);
         }
+        mbar_init(merge_full, 4);
+        mbar_init(all_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -127,62 +149,77 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let loads in flight land
         }
     } else if (warp == 1) {
-        // ------------------------------------------------------------ MMA issuer
+        // ------------------------------------------------------------ MMA issuer 1: S = Q K^T
         if (lane == 0) {
             constexpr uint32_t idesc_s = make_idesc_tf32(BQ, BKV, false, false);
-            constexpr uint32_t idesc_o = make_idesc_tf32(BQ, HD, false, true);
             bool ok = mbar_wait(q_full, 0, g.err, 13);
-            auto issue_s = [&](int kt) -> bool {
+            const DescBase qd = make_desc_base(q_s, 16u, 1024u, 2u);
+            for (int kt = 0; kt < n_kt && ok; ++kt) {
                 const int buf = kt & 1;
-                if (!mbar_wait(k_full(buf), (kt >> 1) & 1u, g.err, 14)) return false;
+                if (!mbar_wait(k_full(buf), (kt >> 1) & 1u, g.err, 14)) { ok = false; break; }
+                // S[buf] is free once the softmax of tile kt-2 has read it (it then publishes P)
+                if (kt >= 2 && !mbar_wait(p_full(buf), ((kt - 2) >> 1) & 1u, g.err, 20)) { ok = false; break; }
                 tc_fence_after();
+                trace_mark(g.trace, 100 + kt);
                 const uint32_t d = tmem_base + (uint32_t)buf * 256u;
+                const DescBase kd = make_desc_base(k_s + buf * kKVBytes, 16u, 1024u, 2u);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const int kb = ks >> 2, j = ks & 3;
-                    const uint32_t qa = q_s + kb * (kQBytes / 2) + j * 32u;
-                    const uint32_t ka = k_s + buf * kKVBytes + kb * (kKVBytes / 2) + j * 32u;
-                    const uint64_t a_hi = make_desc(qa, 16u, 1024u, 2u), a_lo = make_desc(qa + BQ * 128u, 16u, 1024u, 2u);
-                    const uint64_t b_hi = make_desc(ka, 16u, 1024u, 2u), b_lo = make_desc(ka + BKV * 128u, 16u, 1024u, 2u);
+                    const uint32_t qo = (uint32_t)(ks >> 2) * (kQBytes / 2) + (uint32_t)(ks & 3) * 32u;
+                    const uint32_t ko = (uint32_t)(ks >> 2) * (kKVBytes / 2) + (uint32_t)(ks & 3) * 32u;
+                    const uint64_t a_hi = qd.at(qo), a_lo = qd.at(qo + BQ * 128u);
+                    const uint64_t b_hi = kd.at(ko), b_lo = kd.at(ko + BKV * 128u);
                     umma_tf32(d, a_lo, b_hi, idesc_s, ks > 0 ? 1u : 0u);
                     umma_tf32(d, a_hi, b_lo, idesc_s, 1u);
                     umma_tf32(d, a_hi, b_hi, idesc_s, 1u);
                 }
                 umma_commit(k_empty(buf));
                 umma_commit(s_full(buf));
-                return true;
-            };
-            auto issue_pv = [&](int kt) -> bool {
+                trace_mark(g.trace, 200 + kt);
+            }
+        }
+    } else if (warp == 2) {
+        // ------------------------------------------------------------ MMA issuer 2: O_tile = P V
+        // A second issuing thread: the two products of a tile go to different accumulators and are
+        // ordered only through the barriers, so their instruction streams can be issued in parallel.
+        if (lane == 0) {
+            constexpr uint32_t idesc_o = make_idesc_tf32(BQ, HD, false, true);
+            bool ok = true;
+            for (int kt = 0; kt < n_kt && ok; ++kt) {
                 const int buf = kt & 1;
-                if (!mbar_wait(p_full(buf), (kt >> 1) & 1u, g.err, 15)) return false;
-                if (!mbar_wait(v_full(buf), (kt >> 1) & 1u, g.err, 16)) return false;
+                // P(kt) published; the softmax warps read O[buf] of tile kt-2 before publishing it
+                if (!mbar_wait(p_full(buf), (kt >> 1) & 1u, g.err, 15)) { ok = false; break; }
+                if (!mbar_wait(v_full(buf), (kt >> 1) & 1u, g.err, 16)) { ok = false; break; }
                 tc_fence_after();
+                trace_mark(g.trace, 300 + kt);
                 const uint32_t t0 = tmem_base + (uint32_t)buf * 256u;
                 const uint32_t d = t0 + 192u;
-                const uint32_t va = v_s + buf * kKVBytes;
+                const DescBase vd = make_desc_base(v_s + buf * kKVBytes, kKVBytes / 2, 512u, 1u);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
-                    const uint64_t b_hi = make_desc(va + j * 1024u, kKVBytes / 2, 512u, 1u);
-                    const uint64_t b_lo = make_desc(va + BKV * 128u + j * 1024u, kKVBytes / 2, 512u, 1u);
+                    const uint64_t b_hi = vd.at(j * 1024u), b_lo = vd.at(BKV * 128u + j * 1024u);
                     umma_tf32_ts(d, t0 + 128u + j * 8u, b_hi, idesc_o, j > 0 ? 1u : 0u);  // P_lo V_hi
                     umma_tf32_ts(d, t0 + 64u + j * 8u, b_lo, idesc_o, 1u);                // P_hi V_lo
                     umma_tf32_ts(d, t0 + 64u + j * 8u, b_hi, idesc_o, 1u);                // P_hi V_hi
                 }
                 umma_commit(v_empty(buf));
                 umma_commit(o_full(buf));
-                return true;
-            };
-            if (ok) ok = issue_s(0);
-            for (int kt = 0; kt < n_kt && ok; ++kt) {
-                if (kt + 1 < n_kt) ok = issue_s(kt + 1);
-                if (ok) ok = issue_pv(kt);
+                trace_mark(g.trace, 400 + kt);
             }
+            if (ok) umma_commit(all_done);
         }
+    } else if (warp == 3) {
+        // idle (keeps the softmax warps' TMEM lane quadrants aligned with warp index mod 4)
     } else {
         // ------------------------------------------------------------ softmax / correction warps
+        // Two warpgroups (warps 4-7 and 8-11) take alternate key tiles, each with its own running
+        // maximum, sum and output; they are merged at the end.  Two warps per scheduler hide each
+        // other's instruction latencies.
+        const int wg = (warp - 4) >> 2;                              // 0 or 1; owns TMEM buffer wg
         const int lane_group = warp & 3;
-        const int row = q0 + lane_group * 32 + lane;               // query row of this thread
-        const uint32_t t_lane = tmem_base + ((uint32_t)(lane_group * 32) << 16);
+        const int rloc = lane_group * 32 + lane;                    // row inside the CTA
+        const int row = q0 + rloc;                                   // query row of this thread
+        const uint32_t t_lane = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)wg * 256u;
         const float c = kLog2e / sqrtf((float)HD);
         float m = -INFINITY, l = 0.f, corr_prev = 0.f;
         float o_reg[HD];
@@ -191,12 +228,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         bool ok = true;
 
         auto add_output = [&](int kt, float corr) -> bool {
-            const int buf = kt & 1;
-            if (!mbar_wait_warp(o_full(buf), (kt >> 1) & 1u, g.err, 17)) return false;
+            if (!mbar_wait_warp(o_full(wg), (kt >> 1) & 1u, g.err, 17)) return false;
             tc_fence_after();
             uint32_t r0[32], r1[32];
-            tmem_ld32(t_lane + buf * 256u + 192u, r0);
-            tmem_ld32(t_lane + buf * 256u + 224u, r1);
+            tmem_ld32(t_lane + 192u, r0);
+            tmem_ld32(t_lane + 224u, r1);
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
@@ -206,13 +242,18 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             return true;
         };
 
-        for (int kt = 0; kt < n_kt && ok; ++kt) {
-            const int buf = kt & 1;
-            if (!mbar_wait_warp(s_full(buf), (kt >> 1) & 1u, g.err, 18)) { ok = false; break; }
+        int last = -1;
+        for (int kt = wg; kt < n_kt && ok; kt += 2) {
+            // fold in this warpgroup's previous tile first: O[wg] must have been read before P of
+            // this tile is published (the P V product of this tile overwrites O[wg])
+            if (last >= 0 && !add_output(last, corr_prev)) { ok = false; break; }
+            if (rloc == 0) trace_mark(g.trace, 500 + kt);
+            if (!mbar_wait_warp(s_full(wg), (kt >> 1) & 1u, g.err, 18)) { ok = false; break; }
             tc_fence_after();
+            if (rloc == 0) trace_mark(g.trace, 600 + kt);
             uint32_t s0[32], s1[32];
-            tmem_ld32(t_lane + buf * 256u, s0);
-            tmem_ld32(t_lane + buf * 256u + 32u, s1);
+            tmem_ld32(t_lane, s0);
+            tmem_ld32(t_lane + 32u, s1);
             tmem_ld_wait();
             const int key0 = kt * BKV;
             float mx = -INFINITY;
@@ -225,56 +266,77 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             }
 #pragma unroll
             for (int i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(s0[i]), __uint_as_float(s1[i])));
+            // a tile that lies wholly above a row leaves its maximum at -inf; keep the arithmetic finite
             const float m_new = fmaxf(m, mx);
-            // rows of the second half of the tile see no key of a tile that lies wholly above them:
-            // m_new may still be -inf only before the first valid key, which tile 0 always holds
-            const float corr = exp2f((m - m_new) * c);
-            const float mc = m_new * c;
+            const float m_use = (m_new == -INFINITY) ? 0.f : m_new;
+            const float corr = ex2_approx((m - m_use) * c);           // m = -inf -> 0
+            const float mc = m_use * c;
             float sum = 0.f;
             uint32_t hi[32], lo[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-                const float p = exp2f(fmaf(__uint_as_float(s0[i]), c, -mc));
+                const float p = ex2_approx(fmaf(__uint_as_float(s0[i]), c, -mc));
                 sum += p;
-                float fh, fl;
-                split_tf32(p, fh, fl);
-                hi[i] = __float_as_uint(fh);
-                lo[i] = __float_as_uint(fl);
+                split_tf32_int(p, hi[i], lo[i]);
             }
-            tmem_st32(t_lane + buf * 256u + 64u, hi);
-            tmem_st32(t_lane + buf * 256u + 128u, lo);
+            tmem_st32(t_lane + 64u, hi);
+            tmem_st32(t_lane + 128u, lo);
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-                const float p = exp2f(fmaf(__uint_as_float(s1[i]), c, -mc));
+                const float p = ex2_approx(fmaf(__uint_as_float(s1[i]), c, -mc));
                 sum += p;
-                float fh, fl;
-                split_tf32(p, fh, fl);
-                hi[i] = __float_as_uint(fh);
-                lo[i] = __float_as_uint(fl);
+                split_tf32_int(p, hi[i], lo[i]);
             }
-            tmem_st32(t_lane + buf * 256u + 96u, hi);
-            tmem_st32(t_lane + buf * 256u + 160u, lo);
+            tmem_st32(t_lane + 96u, hi);
+            tmem_st32(t_lane + 160u, lo);
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(p_full(buf));
+            if (lane == 0) mbar_arrive(p_full(wg));
+            if (rloc == 0) trace_mark(g.trace, 700 + kt);
             l = fmaf(l, corr, sum);
             m = m_new;
-            // fold in the previous tile's P V while the tensor core works on this one
-            if (kt > 0) ok = add_output(kt - 1, corr_prev);
             corr_prev = corr;
+            last = kt;
         }
-        if (ok) ok = add_output(n_kt - 1, corr_prev);
-        if (ok && row < g.T) {
-            const float inv = 1.0f / l;
-            const int64_t off = ((int64_t)(row_base + row)) * g.C + h * HD;
+        if (ok && last >= 0) ok = add_output(last, corr_prev);
+
+        // merge: warpgroup 1 hands (m, l, O) of its rows to warpgroup 0 through the K buffers, which
+        // are idle once every tile's products have completed
+        float* xch = reinterpret_cast<float*>(smem_raw + (k_s - smem_u32(smem_raw)));   // [128][66]
+        if (wg == 1) {
+            if (ok) ok = mbar_wait_warp(all_done, 0, g.err, 21);   // no product still reads the K buffers
+            float* dst = xch + rloc * 66;
+            dst[64] = m;
+            dst[65] = l;
 #pragma unroll
-            for (int i = 0; i < HD; i += 4) {
-                float4 v = make_float4(o_reg[i] * inv, o_reg[i + 1] * inv, o_reg[i + 2] * inv, o_reg[i + 3] * inv);
-                store_raw_split(v, g.o ? g.o + off : nullptr, g.o_hi ? g.o_hi + off : nullptr,
-                                g.o_lo ? g.o_lo + off : nullptr, i / 4);
+            for (int i = 0; i < HD; ++i) dst[i] = o_reg[i];
+            __threadfence_block();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(merge_full);
+        } else {
+            if (ok) ok = mbar_wait_warp(merge_full, 0, g.err, 19);
+            if (ok) {
+                const float* src = xch + rloc * 66;
+                const float m1 = src[64], l1 = src[65];
+                const float mm = fmaxf(m, m1);                      // finite: tile 0 belongs to warpgroup 0
+                const float f0 = ex2_approx((m - mm) * c), f1 = ex2_approx((m1 - mm) * c);
+                l = l * f0 + l1 * f1;
+                m = mm;
+#pragma unroll
+                for (int i = 0; i < HD; ++i) o_reg[i] = o_reg[i] * f0 + src[i] * f1;
+                if (row < g.T) {
+                    const float inv = 1.0f / l;
+                    const int64_t off = ((int64_t)(row_base + row)) * g.C + h * HD;
+#pragma unroll
+                    for (int i = 0; i < HD; i += 4) {
+                        float4 v = make_float4(o_reg[i] * inv, o_reg[i + 1] * inv, o_reg[i + 2] * inv, o_reg[i + 3] * inv);
+                        store_raw_split(v, g.o ? g.o + off : nullptr, g.o_hi ? g.o_hi + off : nullptr,
+                                        g.o_lo ? g.o_lo + off : nullptr, i / 4);
+                    }
+                    if (g.lse) g.lse[((int64_t)b * g.H + h) * g.T + row] = (m * c + log2f(l)) * kLn2;
+                }
             }
-            if (g.lse) g.lse[((int64_t)b * g.H + h) * g.T + row] = (m * c + log2f(l)) * kLn2;
         }
     }
 
@@ -285,6 +347,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     }
 }
 
+unsigned long long* g_trace_ptr = nullptr;   // set through bt_debug_set_attention_trace
 __device__ int g_attn_err_word = 0;  // error word for the per-op entry points (no caller buffer)
 
 bool encode3(CUtensorMap* tm, const float* base, int64_t cols, int64_t rows, int64_t ld, int64_t plane,
@@ -301,6 +364,8 @@ bool encode3(CUtensorMap* tm, const float* base, int64_t cols, int64_t rows, int
 }
 
 }  // namespace
+
+void attention_tc_set_trace(unsigned long long* p) { g_trace_ptr = p; }
 
 bool attention_tc_supports(int head_dim, int C) { return head_dim == 64 && (C % 4) == 0; }
 
@@ -324,7 +389,7 @@ cudaError_t launch_attention_fwd_tc(const float* qkv_hi, int64_t qkv_plane, int 
               encode3(&tmK, qkv_hi, cols, rows, cols, qkv_plane, 32, BKV, CU_TENSOR_MAP_SWIZZLE_128B) &&
               encode3(&tmV, qkv_hi, cols, rows, cols, qkv_plane, 32, BKV, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
     if (!ok) return cudaErrorInvalidValue;
-    AttnArgs g{T, C, H, o, o_hi, o_lo, lse, err_word};
+    AttnArgs g{T, C, H, o, o_hi, o_lo, lse, err_word, g_trace_ptr};
     dim3 grid((T + BQ - 1) / BQ, B * H);
     attn_fwd_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(tmQ, tmK, tmV, g);
     BT_COUNT_LAUNCH();

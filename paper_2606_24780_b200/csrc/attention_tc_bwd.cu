@@ -33,7 +33,7 @@ using namespace tc;
 namespace {
 
 constexpr int HD = 64, BR = 128, BT_ = 32;  // head dim, rows owned by the CTA, streamed tile rows
-constexpr int kThreads = 192;
+constexpr int kThreads = 320;   // TMA warp, MMA warp, two element-wise warpgroups (alternate tiles)
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr uint32_t kResBytes = 2u * 2u * BR * 128u;   // resident 128-row operand: 2 k-blocks x (hi,lo)
 constexpr uint32_t kTileBytes = 2u * 2u * BT_ * 128u; // one streamed 32-row tile in one layout (16 KB)
@@ -92,18 +92,17 @@ __device__ __forceinline__ void tmem_row_to_split(uint32_t t_row, float mul, flo
     }
 }
 
-// Descriptors of one 8-deep k-step.
+// Byte offsets of one 8-deep k-step inside an operand tile (compile-time after unrolling).
 //  K-major tile (rows x 64 floats as 2 k-blocks of [hi|lo][rows][128 B]), contraction over d.
-__device__ __forceinline__ uint64_t kmaj_desc(uint32_t tile, int rows, int ks, bool lo) {
-    const uint32_t kb_bytes = 2u * (uint32_t)rows * 128u;
-    const uint32_t addr = tile + (uint32_t)(ks >> 2) * kb_bytes + (lo ? (uint32_t)rows * 128u : 0u) + (uint32_t)(ks & 3) * 32u;
-    return make_desc(addr, 16u, 1024u, 2u);
+__device__ __forceinline__ constexpr uint32_t kmaj_off(int rows, int ks, bool lo) {
+    return (uint32_t)(ks >> 2) * 2u * (uint32_t)rows * 128u + (lo ? (uint32_t)rows * 128u : 0u) + (uint32_t)(ks & 3) * 32u;
 }
+__device__ __forceinline__ DescBase kmaj_base(uint32_t tile) { return make_desc_base(tile, 16u, 1024u, 2u); }
 //  MN-major 32-row tile (2 column groups of [hi|lo][32 rows][128 B]), contraction over the rows.
-__device__ __forceinline__ uint64_t mnmaj_desc(uint32_t tile, int ks, bool lo) {
-    const uint32_t addr = tile + (lo ? BT_ * 128u : 0u) + (uint32_t)ks * 1024u;
-    return make_desc(addr, 2u * BT_ * 128u, 512u, 1u);
+__device__ __forceinline__ constexpr uint32_t mnmaj_off(int ks, bool lo) {
+    return (lo ? BT_ * 128u : 0u) + (uint32_t)ks * 1024u;
 }
+__device__ __forceinline__ DescBase mnmaj_base(uint32_t tile) { return make_desc_base(tile, 2u * BT_ * 128u, 512u, 1u); }
 
 struct BwdArgs {
     int T, C, H;
@@ -206,22 +205,24 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT_, false, false);   // 128 x 32, B K-major
             constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
             bool ok = mbar_wait(v_full, 0, g.err, 23) && mbar_wait(k_ready, 0, g.err, 24);
+            const DescBase vd = kmaj_base(v_s);
             auto issue_a = [&](int t) -> bool {
                 const int st = t & 1, bb = t & 1;
                 if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 25)) return false;
                 tc_fence_after();
                 const uint32_t dS = tbuf(bb), dP = tbuf(bb) + 64u;
+                const DescBase qd = kmaj_base(qk_s(st)), od = kmaj_base(dok_s(st));
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t q_hi = kmaj_desc(qk_s(st), BT_, ks, false), q_lo = kmaj_desc(qk_s(st), BT_, ks, true);
+                    const uint64_t q_hi = qd.at(kmaj_off(BT_, ks, false)), q_lo = qd.at(kmaj_off(BT_, ks, true));
                     umma_tf32_ts(dS, tK_lo + ks * 8, q_hi, idesc_a, ks > 0 ? 1u : 0u);
                     umma_tf32_ts(dS, tK_hi + ks * 8, q_lo, idesc_a, 1u);
                     umma_tf32_ts(dS, tK_hi + ks * 8, q_hi, idesc_a, 1u);
                 }
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t v_hi = kmaj_desc(v_s, BR, ks, false), v_lo = kmaj_desc(v_s, BR, ks, true);
-                    const uint64_t o_hi = kmaj_desc(dok_s(st), BT_, ks, false), o_lo = kmaj_desc(dok_s(st), BT_, ks, true);
+                    const uint64_t v_hi = vd.at(kmaj_off(BR, ks, false)), v_lo = vd.at(kmaj_off(BR, ks, true));
+                    const uint64_t o_hi = od.at(kmaj_off(BT_, ks, false)), o_lo = od.at(kmaj_off(BT_, ks, true));
                     umma_tf32(dP, v_lo, o_hi, idesc_a, ks > 0 ? 1u : 0u);
                     umma_tf32(dP, v_hi, o_lo, idesc_a, 1u);
                     umma_tf32(dP, v_hi, o_hi, idesc_a, 1u);
@@ -236,9 +237,10 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 if (!mbar_wait(mfull(st), (t >> 1) & 1u, g.err, 27)) return false;
                 tc_fence_after();
                 const uint32_t p_hi = tbuf(bb), p_lo = tbuf(bb) + 32u, s_hi = tbuf(bb) + 64u, s_lo = tbuf(bb) + 96u;
+                const DescBase omd = mnmaj_base(dom_s(st)), qmd = mnmaj_base(qm_s(st));
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t o_hi = mnmaj_desc(dom_s(st), ks, false), o_lo = mnmaj_desc(dom_s(st), ks, true);
+                    const uint64_t o_hi = omd.at(mnmaj_off(ks, false)), o_lo = omd.at(mnmaj_off(ks, true));
                     const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
                     umma_tf32_ts(tdV, p_lo + ks * 8, o_hi, idesc_b, acc);
                     umma_tf32_ts(tdV, p_hi + ks * 8, o_lo, idesc_b, 1u);
@@ -246,7 +248,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 }
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t q_hi = mnmaj_desc(qm_s(st), ks, false), q_lo = mnmaj_desc(qm_s(st), ks, true);
+                    const uint64_t q_hi = qmd.at(mnmaj_off(ks, false)), q_lo = qmd.at(mnmaj_off(ks, true));
                     const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
                     umma_tf32_ts(tdK, s_lo + ks * 8, q_hi, idesc_b, acc);
                     umma_tf32_ts(tdK, s_hi + ks * 8, q_lo, idesc_b, 1u);
@@ -263,6 +265,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             if (ok) umma_commit(acc_full);
         }
     } else {
+        const int wg = (warp - 2) >> 2;                   // 0 or 1: takes tiles t with (t & 1) == wg, buffer wg
         const int lane_group = warp & 3;
         const int etid = lane_group * 32 + lane;          // 0..127: row owned inside the CTA
         const int key = j0 + etid;
@@ -270,7 +273,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
         const float scale = 1.0f / sqrtf((float)HD);
         const int64_t gs = 3 * (int64_t)g.C;
         const int64_t lb = ((int64_t)b * g.H + h) * g.T;
-        {   // K' = K * scale * log2(e) into tensor memory
+        if (wg == 0) {   // K' = K * scale * log2(e) into tensor memory
             const int64_t off = (int64_t)(row_base + min(key, g.T - 1)) * gs + g.C + h * HD;
             row_to_tmem(g.qkv_hi + off, g.qkv_hi + g.qkv_plane + off, scale * kLog2e, tK_hi + t_lane, tK_lo + t_lane);
             tc_fence_before();
@@ -278,43 +281,45 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             if (lane == 0) mbar_arrive(k_ready);
         }
         bool ok = true;
-        for (int t = 0; t < n_t && ok; ++t) {
-            const int bb = t & 1, q0 = (qt0 + t) * BT_;
+        const uint32_t tb = tbuf(wg) + t_lane;
+        for (int t = wg; t < n_t && ok; t += 2) {
+            const int q0 = (qt0 + t) * BT_;
             // per-column softmax statistics of this query tile (same addresses in every thread:
-            // broadcast loads); rows past the sequence end get lse = +inf, i.e. probability 0
+            // broadcast loads, issued before the wait so their latency is hidden); rows past the
+            // sequence end are clamped here and masked below
             const int nvalid = min(BT_, g.T - q0);
             const float* lse_t = g.lse + lb + q0;
             const float* d_t = g.dvec + lb + q0;
-            if (!mbar_wait_warp(sdp_full(bb), (t >> 1) & 1u, g.err, 28)) { ok = false; break; }
+            float Lc[32], Dc[32];
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const int ic = min(i, nvalid - 1);
+                Lc[i] = __ldg(lse_t + ic) * kLog2e;
+                Dc[i] = __ldg(d_t + ic);
+            }
+            if (!mbar_wait_warp(sdp_full(wg), (t >> 1) & 1u, g.err, 28)) { ok = false; break; }
             tc_fence_after();
             uint32_t s[32], dp[32];
-            tmem_ld32(tbuf(bb) + t_lane, s);
-            tmem_ld32(tbuf(bb) + 64u + t_lane, dp);
+            tmem_ld32(tb, s);
+            tmem_ld32(tb + 64u, dp);
             tmem_ld_wait();
             uint32_t p_hi[32], p_lo[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const bool live = (i < nvalid) && (q0 + i >= key);   // in the sequence and not before this key
-                const float Li = live ? __ldg(lse_t + i) * kLog2e : 0.f;
-                const float Di = live ? __ldg(d_t + i) : 0.f;
-                const float p = live ? ex2_approx(__uint_as_float(s[i]) - Li) : 0.f;
-                const float ds = p * (__uint_as_float(dp[i]) - Di);
-                float fh, fl;
-                split_tf32(p, fh, fl);
-                p_hi[i] = __float_as_uint(fh);
-                p_lo[i] = __float_as_uint(fl);
-                split_tf32(ds, fh, fl);
-                s[i] = __float_as_uint(fh);                      // reuse: dS^T hi
-                dp[i] = __float_as_uint(fl);                     //        dS^T lo
+                const float p = live ? ex2_approx(__uint_as_float(s[i]) - Lc[i]) : 0.f;
+                const float ds = p * (__uint_as_float(dp[i]) - Dc[i]);
+                split_tf32_int(p, p_hi[i], p_lo[i]);
+                split_tf32_int(ds, s[i], dp[i]);                     // reuse: dS^T hi, lo
             }
-            tmem_st32(tbuf(bb) + t_lane, p_hi);
-            tmem_st32(tbuf(bb) + 32u + t_lane, p_lo);
-            tmem_st32(tbuf(bb) + 64u + t_lane, s);
-            tmem_st32(tbuf(bb) + 96u + t_lane, dp);
+            tmem_st32(tb, p_hi);
+            tmem_st32(tb + 32u, p_lo);
+            tmem_st32(tb + 64u, s);
+            tmem_st32(tb + 96u, dp);
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(pds_full(bb));
+            if (lane == 0) mbar_arrive(pds_full(wg));
         }
         if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 29);
         if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
@@ -323,8 +328,8 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             const int64_t off = (int64_t)(row_base + (valid ? key : 0)) * gs + h * HD;
             float* hi = g.dqkv_hi + off;
             float* lo = hi + g.dqkv_plane;
-            tmem_row_to_split(tdK + t_lane, scale, hi + g.C, lo + g.C, valid);
-            tmem_row_to_split(tdV + t_lane, 1.0f, hi + 2 * g.C, lo + 2 * g.C, valid);
+            if (wg == 0) tmem_row_to_split(tdK + t_lane, scale, hi + g.C, lo + g.C, valid);
+            else tmem_row_to_split(tdV + t_lane, 1.0f, hi + 2 * g.C, lo + 2 * g.C, valid);
         }
     }
     tc_fence_before();
@@ -401,22 +406,24 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT_, false, false);
             constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);
             bool ok = mbar_wait(do_full, 0, g.err, 33) && mbar_wait(q_ready, 0, g.err, 34);
+            const DescBase dod = kmaj_base(do_s);
             auto issue_a = [&](int t) -> bool {
                 const int st = t & 1, bb = t & 1;
                 if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 35)) return false;
                 tc_fence_after();
                 const uint32_t dS = tbuf(bb), dP = tbuf(bb) + 64u;
+                const DescBase kd = kmaj_base(kk_s(st)), vkd = kmaj_base(vk_s(st));
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t k_hi = kmaj_desc(kk_s(st), BT_, ks, false), k_lo = kmaj_desc(kk_s(st), BT_, ks, true);
+                    const uint64_t k_hi = kd.at(kmaj_off(BT_, ks, false)), k_lo = kd.at(kmaj_off(BT_, ks, true));
                     umma_tf32_ts(dS, tQ_lo + ks * 8, k_hi, idesc_a, ks > 0 ? 1u : 0u);
                     umma_tf32_ts(dS, tQ_hi + ks * 8, k_lo, idesc_a, 1u);
                     umma_tf32_ts(dS, tQ_hi + ks * 8, k_hi, idesc_a, 1u);
                 }
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t o_hi = kmaj_desc(do_s, BR, ks, false), o_lo = kmaj_desc(do_s, BR, ks, true);
-                    const uint64_t v_hi = kmaj_desc(vk_s(st), BT_, ks, false), v_lo = kmaj_desc(vk_s(st), BT_, ks, true);
+                    const uint64_t o_hi = dod.at(kmaj_off(BR, ks, false)), o_lo = dod.at(kmaj_off(BR, ks, true));
+                    const uint64_t v_hi = vkd.at(kmaj_off(BT_, ks, false)), v_lo = vkd.at(kmaj_off(BT_, ks, true));
                     umma_tf32(dP, o_lo, v_hi, idesc_a, ks > 0 ? 1u : 0u);
                     umma_tf32(dP, o_hi, v_lo, idesc_a, 1u);
                     umma_tf32(dP, o_hi, v_hi, idesc_a, 1u);
@@ -431,9 +438,10 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
                 if (!mbar_wait(mfull(st), (t >> 1) & 1u, g.err, 37)) return false;
                 tc_fence_after();
                 const uint32_t s_hi = tbuf(bb), s_lo = tbuf(bb) + 32u;
+                const DescBase kmd = mnmaj_base(km_s(st));
 #pragma unroll
                 for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t k_hi = mnmaj_desc(km_s(st), ks, false), k_lo = mnmaj_desc(km_s(st), ks, true);
+                    const uint64_t k_hi = kmd.at(mnmaj_off(ks, false)), k_lo = kmd.at(mnmaj_off(ks, true));
                     const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
                     umma_tf32_ts(tdQ, s_lo + ks * 8, k_hi, idesc_b, acc);
                     umma_tf32_ts(tdQ, s_hi + ks * 8, k_lo, idesc_b, 1u);
@@ -450,6 +458,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             if (ok) umma_commit(acc_full);
         }
     } else {
+        const int wg = (warp - 2) >> 2;
         const int lane_group = warp & 3;
         const int row = q0 + lane_group * 32 + lane;
         const uint32_t t_lane = ((uint32_t)(lane_group * 32) << 16);
@@ -457,7 +466,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
         const int64_t gs = 3 * (int64_t)g.C;
         const int64_t lb = ((int64_t)b * g.H + h) * g.T;
         const int rc = min(row, g.T - 1);
-        {
+        if (wg == 0) {
             const int64_t off = (int64_t)(row_base + rc) * gs + h * HD;
             row_to_tmem(g.qkv_hi + off, g.qkv_hi + g.qkv_plane + off, scale * kLog2e, tQ_hi + t_lane, tQ_lo + t_lane);
             tc_fence_before();
@@ -466,36 +475,36 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
         }
         const float L = g.lse[lb + rc] * kLog2e, D = g.dvec[lb + rc];
         bool ok = true;
-        for (int t = 0; t < n_t && ok; ++t) {
-            const int bb = t & 1, k0 = t * BT_;
-            if (!mbar_wait_warp(sdp_full(bb), (t >> 1) & 1u, g.err, 38)) { ok = false; break; }
+        const uint32_t tb = tbuf(wg) + t_lane;
+        for (int t = wg; t < n_t && ok; t += 2) {
+            const int k0 = t * BT_;
+            if (!mbar_wait_warp(sdp_full(wg), (t >> 1) & 1u, g.err, 38)) { ok = false; break; }
             tc_fence_after();
             uint32_t s[32], dp[32];
-            tmem_ld32(tbuf(bb) + t_lane, s);
-            tmem_ld32(tbuf(bb) + 64u + t_lane, dp);
+            tmem_ld32(tb, s);
+            tmem_ld32(tb + 64u, dp);
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 float p = ex2_approx(__uint_as_float(s[i]) - L);
                 if (k0 + i > row) p = 0.f;                      // key follows this query: masked
                 const float ds = p * (__uint_as_float(dp[i]) - D);
-                float fh, fl;
-                split_tf32(ds, fh, fl);
-                s[i] = __float_as_uint(fh);
-                dp[i] = __float_as_uint(fl);
+                split_tf32_int(ds, s[i], dp[i]);
             }
-            tmem_st32(tbuf(bb) + t_lane, s);
-            tmem_st32(tbuf(bb) + 32u + t_lane, dp);
+            tmem_st32(tb, s);
+            tmem_st32(tb + 32u, dp);
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(ds_full(bb));
+            if (lane == 0) mbar_arrive(ds_full(wg));
         }
-        if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 39);
-        if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
-            tc_fence_after();
-            const int64_t off = (int64_t)(row_base + rc) * gs + h * HD;
-            tmem_row_to_split(tdQ + t_lane, scale, g.dqkv_hi + off, g.dqkv_hi + g.dqkv_plane + off, row < g.T);
+        if (wg == 0) {
+            if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 39);
+            if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
+                tc_fence_after();
+                const int64_t off = (int64_t)(row_base + rc) * gs + h * HD;
+                tmem_row_to_split(tdQ + t_lane, scale, g.dqkv_hi + off, g.dqkv_hi + g.dqkv_plane + off, row < g.T);
+            }
         }
     }
     tc_fence_before();

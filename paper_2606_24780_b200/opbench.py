@@ -108,6 +108,12 @@ def build_cases(B, T, C, H, Vp, n_params):
         cases["attention_fwd_tcgen05"] = dict(
             run=lambda: b.bt_op_attention_fwd(None, B, T, C, H, None, os_, lse, qkv_split=qkv_s), flops=afl,
             bytes=32.0 * N * C, bound="tensor", keep=(qkv_s,))
+    if C // H == 64:
+        do_s, dqs2 = _split(d_o), torch.empty(2, N, 3 * C, device="cuda")
+        cases["attention_bwd_tcgen05"] = dict(
+            run=lambda: b.bt_op_attention_bwd(None, o, lse, None, B, T, C, H, None, dqs2, dv, dv.numel() * 4,
+                                              qkv_split=qkv_s, d_o_split=do_s),
+            flops=2.5 * afl, bytes=64.0 * N * C, bound="tensor", keep=(do_s, dqs2))
     cases["attention_bwd"] = dict(
         run=lambda: b.bt_op_attention_bwd(qkv, o, lse, d_o, B, T, C, H, None, dqs, dv, dv.numel() * 4),
         flops=2.5 * afl, bytes=48.0 * N * C, bound="tensor", keep=(d_o, dqs, dv))
