@@ -120,8 +120,9 @@ BT_API bt_status bt_tensor_info(const bt_model* m, int32_t index, const char** n
  * `numel` floats inside the workspace and stays valid for the model's lifetime. */
 BT_API bt_status bt_tensor_ptr(bt_model* m, const char* name, int32_t kind, float** d_ptr);
 
-/* Activations of the last forward/backward, for tests: per-layer "x", "qkv", "x1", "h",
- * "ln1.mean", "ln1.rstd", "ln2.mean", "ln2.rstd", "lse"; split per-layer "a", "o", "m", "g"
+/* Activations of the last forward/backward, for tests: per-layer "x", "qkv" (raw; written only
+ * when head_dim != 64 or a reference-kernel flag is set), "x1", "h",
+ * "ln1.mean", "ln1.rstd", "ln2.mean", "ln2.rstd", "lse"; split per-layer "qkv_split", "a", "o", "m", "g"
  * (pointer to the hi plane; lo plane follows at +numel); global "xL", "logits", "losses",
  * split "xf", "dlogits".  `numel` (nullable) receives the element count of one plane for
  * the current batch. */
@@ -268,6 +269,14 @@ BT_API bt_status bt_op_gelu_fwd(const float* x, int64_t n, int32_t tanh_form, fl
 /* dx = dy * GELU'(x). */
 BT_API bt_status bt_op_gelu_bwd(const float* x, const float* dy, int64_t n, int32_t tanh_form, float* dx,
                                 float* dx_split, void* stream);
+
+/* The same dx for x, dy of shape [N, C] (device), plus colsum[C] (device) = the column sums of
+ * dx: the bias gradient of the linear layer that produced x (Section 2, backward of the MLP's
+ * up-projection), taken in the pass that writes dx.  scratch: device,
+ * bt_op_colsum_scratch_bytes(N, C) bytes, caller-owned.  C % 4 == 0; summation order fixed. */
+BT_API bt_status bt_op_gelu_bwd_colsum(const float* x, const float* dy, int64_t N, int32_t C, int32_t tanh_form,
+                                       float* dx, float* dx_split, float* colsum, void* scratch,
+                                       size_t scratch_bytes, void* stream);
 
 /* Fused softmax cross-entropy over all Vp columns: losses[n] = logsumexp(logits[n,:]) -
  * logits[n, y_n]; dlogits = (softmax - onehot) * inv_count; loss_mean (1 float) =

@@ -76,6 +76,7 @@ _SIGNATURES = {
     "bt_op_attention_bwd": (_i32, [_vp] * 6 + [_i32] * 4 + [_vp] * 3 + [_sz, _u32, _vp]),
     "bt_op_gelu_fwd": (_i32, [_vp, _i64, _i32, _vp, _vp, _vp]),
     "bt_op_gelu_bwd": (_i32, [_vp, _vp, _i64, _i32, _vp, _vp, _vp]),
+    "bt_op_gelu_bwd_colsum": (_i32, [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp]),
     "bt_op_softmax_xent": (_i32, [_vp, _vp, _i64, _i32, _f, _vp, _vp, _vp, _vp, _vp]),
     "bt_op_colsum_scratch_bytes": (_sz, [_i64, _i32]),
     "bt_op_colsum": (_i32, [_vp, _i64, _i32, _vp, _vp, _sz, _vp]),
@@ -323,6 +324,11 @@ def bt_op_gelu_fwd(x, n, tanh_form, y, y_split, stream=None):
 
 def bt_op_gelu_bwd(x, dy, n, tanh_form, dx, dx_split, stream=None):
     _check(lib().bt_op_gelu_bwd(_ptr(x), _ptr(dy), n, tanh_form, _ptr(dx), _ptr(dx_split), _stream(stream)))
+
+
+def bt_op_gelu_bwd_colsum(x, dy, N, C, tanh_form, dx, dx_split, colsum, scratch, scratch_bytes, stream=None):
+    _check(lib().bt_op_gelu_bwd_colsum(_ptr(x), _ptr(dy), N, C, tanh_form, _ptr(dx), _ptr(dx_split), _ptr(colsum),
+                                       _ptr(scratch), scratch_bytes, _stream(stream)))
 
 
 def bt_op_softmax_xent(logits, targets, N, Vp, inv_count, losses, loss_mean, dlogits, dlogits_split, stream=None):

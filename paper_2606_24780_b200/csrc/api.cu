@@ -435,6 +435,7 @@ extern "C" bt_status bt_activation_ptr(bt_model* m, const char* name, int32_t la
         if (layer < 0 || layer >= m->L) return fail(BT_ERR_NOT_FOUND, "layer %d out of range", layer);
         LayerAct& a = m->act[layer];
         if (n == "x") { p = a.x; ne = N * C; }
+        else if (n == "qkv_split") { p = a.qkv_s; ne = N * 3 * C; }
         else if (n == "a") { p = a.a_s; ne = N * C; }
         else if (n == "qkv") { p = a.qkv; ne = N * 3 * C; }
         else if (n == "o") { p = a.o_s; ne = N * C; }
@@ -509,6 +510,9 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
     (void)Nmax;
     const bool simt_attn = (m->cfg.flags & BT_FLAG_ATTN_SIMT) != 0;
     const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
+    // the tcgen05 attention kernels read qkv only as hi/lo planes; the raw copy is written only
+    // for the kernels that need it
+    const bool raw_qkv = simt_attn || (C / H) != 64 || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
 
     // hi/lo planes of every parameter (weights are GEMM operands; one streaming pass)
     BT_STEP(kCatSplit, 0, 12.0 * m->P, launch_split(m->params, m->wsplit, m->wsplit + m->P, m->P, s));
@@ -520,8 +524,8 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
         auto P = [&](int k) { return m->params + layer_tensor(m, l, k).off; };
         BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x, P(LN1G), P(LN1B), N, C, nullptr, a.a_s, a.a_s + N * C, a.mean1, a.rstd1, s));
         BT_GEMM_SPLIT_OUT(kNT, N, 3 * C, C, act_mat(a.a_s, N, C, N), weight_mat(m, layer_tensor(m, l, QKVW), 3 * C, C),
-                          a.qkv, a.qkv_s, P(QKVB), nullptr);
-        BT_STEP(kCatAttnFwd, attn_fwd_flops(B, H, T, C / H), 20.0 * N * C, launch_attention_fwd(a.qkv, a.qkv_s, N * 3 * C, B, T, C, H, nullptr, a.o_s, a.o_s + N * C, a.lse, simt_attn,
+                          raw_qkv ? a.qkv : nullptr, a.qkv_s, P(QKVB), nullptr);
+        BT_STEP(kCatAttnFwd, attn_fwd_flops(B, H, T, C / H), 20.0 * N * C, launch_attention_fwd(raw_qkv ? a.qkv : nullptr, a.qkv_s, N * 3 * C, B, T, C, H, nullptr, a.o_s, a.o_s + N * C, a.lse, simt_attn,
                                      m->err_word, s));
         BT_GEMM(kNT, N, C, C, act_mat(a.o_s, N, C, N), weight_mat(m, layer_tensor(m, l, PROJW), C, C), a.x1,
                      P(PROJB), a.x);
@@ -561,6 +565,7 @@ extern "C" bt_status bt_backward(bt_model* m) {
     const int64_t N = (int64_t)B * T;
     const bool simt_attn = (m->cfg.flags & BT_FLAG_ATTN_SIMT) != 0;
     const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
+    const bool raw_qkv = simt_attn || (C / H) != 64 || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
     auto G = [&](const Tensor& t) { return m->grads + t.off; };
 
     // LM head: dxf = dlogits . wte ; dwte = dlogits^T . xf
@@ -579,21 +584,24 @@ extern "C" bt_status bt_backward(bt_model* m) {
         BT_GEMM(kNN, N, F, C, dres, weight_mat(m, LT(PRW), C, F), m->dg, nullptr, nullptr);
         BT_GEMM(kTN, C, F, N, dres, act_mat(a.g_s, N, F, N), G(LT(PRW)), nullptr, nullptr);
         BT_STEP(kCatColsum, 0, 4.0 * N * C, launch_colsum(m->dres, nullptr, N, C, G(LT(PRB)), m->colsum_scratch, s));
-        BT_STEP(kCatGeluBwd, 0, 16.0 * N * F, launch_gelu_bwd(a.h, m->dg, N * F, tanh_form, nullptr, m->dh_s, m->dh_s + N * F, s));
+        // d h, with its column sums (the gradient of bfc) taken in the same pass
+        BT_STEP(kCatGeluBwd, 0, 16.0 * N * F, launch_gelu_bwd_colsum(a.h, m->dg, N, F, tanh_form, nullptr, m->dh_s, m->dh_s + N * F,
+                                       G(LT(FCB)), m->colsum_scratch, s));
         // MLP up-projection: h = m . Wfc^T + bfc
         SplitMat dh = act_mat(m->dh_s, N, F, N);
         BT_GEMM(kNN, N, C, F, dh, weight_mat(m, LT(FCW), F, C), m->dtmp, nullptr, nullptr);
         BT_GEMM(kTN, F, C, N, dh, act_mat(a.m_s, N, C, N), G(LT(FCW)), nullptr, nullptr);
-        BT_STEP(kCatColsum, 0, 8.0 * N * F, launch_colsum(m->dh_s, m->dh_s + N * F, N, F, G(LT(FCB)), m->colsum_scratch, s));
         // LN2 and the residual: d x1 = d x_out + LN2'(dm)
         BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, a.x1, m->params + LT(LN2G).off, a.mean2, a.rstd2, m->dres, N, C, m->dres,
                                      m->dres_s, m->dres_s + N * C, G(LT(LN2G)), G(LT(LN2B)), m->ln_scratch, s));
         // attention output projection: x1 = x + o . Wo^T + bo
         // d o, raw for the FMA / warp-MMA attention kernels, as hi/lo planes for the tcgen05 ones
-        BT_GEMM_SPLIT_OUT(kNN, N, C, C, dres, weight_mat(m, LT(PROJW), C, C), m->dtmp, m->do_s, nullptr, nullptr);
+        BT_GEMM_SPLIT_OUT(kNN, N, C, C, dres, weight_mat(m, LT(PROJW), C, C), raw_qkv ? m->dtmp : nullptr, m->do_s, nullptr,
+                          nullptr);
         BT_GEMM(kTN, C, C, N, dres, act_mat(a.o_s, N, C, N), G(LT(PROJW)), nullptr, nullptr);
         BT_STEP(kCatColsum, 0, 4.0 * N * C, launch_colsum(m->dres, nullptr, N, C, G(LT(PROJB)), m->colsum_scratch, s));
-        BT_STEP(kCatAttnBwd, 2.5 * attn_fwd_flops(B, H, T, C / H), 48.0 * N * C, launch_attention_bwd(a.qkv, a.qkv_s, N * 3 * C, a.o_s, a.o_s + N * C, a.lse, m->dtmp, m->do_s, N * C, B, T,
+        BT_STEP(kCatAttnBwd, 2.5 * attn_fwd_flops(B, H, T, C / H), 48.0 * N * C, launch_attention_bwd(raw_qkv ? a.qkv : nullptr, a.qkv_s, N * 3 * C, a.o_s, a.o_s + N * C, a.lse,
+                                     raw_qkv ? m->dtmp : nullptr, m->do_s, N * C, B, T,
                                      C, H, nullptr, m->dqkv_s, m->dqkv_s + N * 3 * C, m->dvec, simt_attn, m->err_word, s));
         // QKV projection: qkv = a . Wqkv^T + bqkv
         SplitMat dqkv = act_mat(m->dqkv_s, N, 3 * C, N);
@@ -869,6 +877,17 @@ extern "C" bt_status bt_op_gelu_bwd(const float* x, const float* dy, int64_t n, 
     if (n < 0 || n % 4) return fail(BT_ERR_INVALID_ARG, "gelu_bwd: n must be a non-negative multiple of 4");
     if (n == 0) return BT_OK;
     BT_CUDA(launch_gelu_bwd(x, dy, n, tanh_form, dx, dx_split, dx_split ? dx_split + n : nullptr, (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" bt_status bt_op_gelu_bwd_colsum(const float* x, const float* dy, int64_t N, int32_t C, int32_t tanh_form,
+                                           float* dx, float* dx_split, float* colsum, void* scratch,
+                                           size_t scratch_bytes, void* stream) {
+    BT_PTR(x); BT_PTR(dy); BT_OPT_PTR(dx); BT_OPT_PTR(dx_split); BT_PTR(colsum); BT_PTR(scratch);
+    if (N < 1 || C < 4 || C % 4) return fail(BT_ERR_INVALID_ARG, "gelu_bwd_colsum: bad sizes");
+    if (scratch_bytes < bt_op_colsum_scratch_bytes(N, C)) return fail(BT_ERR_OOM, "gelu_bwd_colsum: scratch too small");
+    BT_CUDA(launch_gelu_bwd_colsum(x, dy, N, C, tanh_form, dx, dx_split, dx_split ? dx_split + N * C : nullptr, colsum,
+                                   (float*)scratch, (cudaStream_t)stream));
     return BT_OK;
 }
 

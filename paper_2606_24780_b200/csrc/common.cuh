@@ -102,6 +102,10 @@ cudaError_t launch_gelu_fwd(const float* x, int64_t n, int tanh_form, float* y, 
                             cudaStream_t s);
 cudaError_t launch_gelu_bwd(const float* x, const float* dy, int64_t n, int tanh_form, float* dx, float* dx_hi,
                             float* dx_lo, cudaStream_t s);
+// GELU backward that also writes the column sums of dx (an N x C matrix) into colsum[C];
+// scratch as for launch_colsum(N, C).
+cudaError_t launch_gelu_bwd_colsum(const float* x, const float* dy, int64_t N, int C, int tanh_form, float* dx,
+                                   float* dx_hi, float* dx_lo, float* colsum, float* scratch, cudaStream_t s);
 cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int Vp, float inv_count,
                                 float* losses, float* loss_mean, float* dl, float* dl_hi, float* dl_lo,
                                 cudaStream_t s);

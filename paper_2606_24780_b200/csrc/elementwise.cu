@@ -256,13 +256,88 @@ __global__ void __launch_bounds__(256) colsum_stage1_kernel(const float* __restr
     }
 }
 
-__global__ void __launch_bounds__(128) colsum_stage2_kernel(const float* __restrict__ partial, int strips, int C4,
+// Stage 2: lane = float4 column, warp w adds strips w, w+8, ... (four loads in flight), the eight
+// warp sums are combined in warp order: a fixed summation order.
+__global__ void __launch_bounds__(256) colsum_stage2_kernel(const float* __restrict__ partial, int strips, int C4,
                                                             float* __restrict__ out) {
-    int c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c >= C4) return;
-    float4 t = ld4(partial, c);
-    for (int s = 1; s < strips; ++s) t = add4(t, ld4(partial, (int64_t)s * C4 + c));
-    reinterpret_cast<float4*>(out)[c] = t;
+    __shared__ float4 sm[8][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + lane;
+    float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (c < C4) {
+        int s = warp;
+        for (; s + 24 < strips; s += 32) {
+            float4 a0 = ld4(partial, (int64_t)s * C4 + c), a1 = ld4(partial, (int64_t)(s + 8) * C4 + c);
+            float4 a2 = ld4(partial, (int64_t)(s + 16) * C4 + c), a3 = ld4(partial, (int64_t)(s + 24) * C4 + c);
+            t = add4(add4(add4(add4(t, a0), a1), a2), a3);
+        }
+        for (; s < strips; s += 8) t = add4(t, ld4(partial, (int64_t)s * C4 + c));
+    }
+    sm[warp][lane] = t;
+    __syncthreads();
+    if (warp == 0 && c < C4) {
+        float4 r = sm[0][lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) r = add4(r, sm[w][lane]);
+        reinterpret_cast<float4*>(out)[c] = r;
+    }
+}
+
+// GELU backward with the column sums of its own output (the bias gradient of the layer that
+// produced x): the strip layout of stage 1 above, so each lane keeps one float4 column and the
+// sums cost no extra pass over dx.
+__global__ void __launch_bounds__(256) gelu_bwd_colsum_kernel(const float* __restrict__ x,
+                                                              const float* __restrict__ dy, int64_t N, int C4,
+                                                              int strips, int tanh_form, float* dx, float* dx_hi,
+                                                              float* dx_lo, float* __restrict__ partial) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int c = blockIdx.x * 32 + lane;
+    const int st = blockIdx.y;
+    const int64_t rows_per = (N + strips - 1) / strips;
+    const int64_t r0 = st * rows_per, r1 = (r0 + rows_per < N) ? r0 + rows_per : N;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    auto one = [&](float4 v, float4 d, int64_t i) {
+        float4 r;
+        r.x = d.x * gelu_grad_f(v.x, tanh_form);
+        r.y = d.y * gelu_grad_f(v.y, tanh_form);
+        r.z = d.z * gelu_grad_f(v.z, tanh_form);
+        r.w = d.w * gelu_grad_f(v.w, tanh_form);
+        store_raw_split(r, dx, dx_hi, dx_lo, i);
+        acc = add4(acc, r);
+    };
+    if (c < C4) {
+        int64_t r = r0 + warp;
+        for (; r + 24 < r1; r += 32) {  // four rows in flight per lane
+            const int64_t i0 = r * C4 + c, i1 = (r + 8) * C4 + c, i2 = (r + 16) * C4 + c, i3 = (r + 24) * C4 + c;
+            float4 v0 = ld4(x, i0), v1 = ld4(x, i1), v2 = ld4(x, i2), v3 = ld4(x, i3);
+            float4 d0 = ld4(dy, i0), d1 = ld4(dy, i1), d2 = ld4(dy, i2), d3 = ld4(dy, i3);
+            one(v0, d0, i0);
+            one(v1, d1, i1);
+            one(v2, d2, i2);
+            one(v3, d3, i3);
+        }
+        for (; r < r1; r += 8) one(ld4(x, r * C4 + c), ld4(dy, r * C4 + c), r * C4 + c);
+    }
+    __shared__ float4 sm[8][32];
+    sm[warp][lane] = acc;
+    __syncthreads();
+    if (warp == 0 && c < C4) {
+        float4 t = sm[0][lane];
+#pragma unroll
+        for (int w = 1; w < 8; ++w) t = add4(t, sm[w][lane]);
+        reinterpret_cast<float4*>(partial)[(int64_t)st * C4 + c] = t;
+    }
+}
+
+cudaError_t launch_gelu_bwd_colsum(const float* x, const float* dy, int64_t N, int C, int tanh_form, float* dx,
+                                   float* dx_hi, float* dx_lo, float* colsum, float* scratch, cudaStream_t s) {
+    int C4 = C / 4, strips = colsum_strips(N, C);
+    dim3 grid((C4 + 31) / 32, strips);
+    gelu_bwd_colsum_kernel<<<grid, 256, 0, s>>>(x, dy, N, C4, strips, tanh_form, dx, dx_hi, dx_lo, scratch);
+    BT_COUNT_LAUNCH();
+    colsum_stage2_kernel<<<(C4 + 31) / 32, 256, 0, s>>>(scratch, strips, C4, colsum);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
 }
 
 cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, float* out, float* scratch,
@@ -271,7 +346,7 @@ cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, f
     dim3 grid((C4 + 31) / 32, strips);
     colsum_stage1_kernel<<<grid, 256, 0, s>>>(x, x_lo, N, C4, strips, scratch);
     BT_COUNT_LAUNCH();
-    colsum_stage2_kernel<<<(C4 + 127) / 128, 128, 0, s>>>(scratch, strips, C4, out);
+    colsum_stage2_kernel<<<(C4 + 31) / 32, 256, 0, s>>>(scratch, strips, C4, out);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }

@@ -94,6 +94,12 @@ def build_cases(B, T, C, H, Vp, n_params):
     cases["gelu_bwd"] = dict(run=lambda: b.bt_op_gelu_bwd(h, dgl, N * F, 0, None, dhs), bytes=16.0 * N * F,
                              bound="hbm", keep=(dgl, dhs))
 
+    gcb = b.bt_op_colsum_scratch_bytes(N, F)
+    gscr, gcs = torch.empty(gcb // 4, device="cuda"), torch.empty(F, device="cuda")
+    cases["gelu_bwd_colsum"] = dict(
+        run=lambda: b.bt_op_gelu_bwd_colsum(h, dgl, N, F, 0, None, dhs, gcs, gscr, gcb), bytes=16.0 * N * F,
+        bound="hbm", keep=(gscr, gcs))
+
     # attention
     qkv, d_o = _rand(N, 3 * C), _rand(N, C, std=1e-2)
     o, os_, lse = torch.empty(N, C, device="cuda"), torch.empty(2, N, C, device="cuda"), torch.empty(B, H, T, device="cuda")

@@ -115,6 +115,24 @@ def test_gelu_fwd_bwd(tanh_form):
     check_split(dxs, host(dx))
 
 
+@pytest.mark.parametrize("N,C", [(1000, 3072), (37, 132), (1, 4), (8192, 768)])
+def test_gelu_bwd_colsum(N, C):
+    """The fused kernel gives the dx of the plain one and its column sums (the bias gradient)."""
+    x, dy = si.normal_f32(25, (N, C), 2.0), si.normal_f32(26, (N, C), 1e-2) + np.float32(3e-3)
+    dx, dxs, cs = empty(N, C), empty(2, N, C), empty(C)
+    nb = b.bt_op_colsum_scratch_bytes(N, C)
+    b.bt_op_gelu_bwd_colsum(dev(x), dev(dy), N, C, 0, dx, dxs, cs, scratch(nb), nb)
+    rdx = oracle.gelu_bwd(x.ravel(), dy.ravel(), 0).reshape(N, C)
+    assert rel_l2(host(dx), rdx) < 1e-5
+    check_split(dxs, host(dx))
+    ref = rdx.astype(np.float64).sum(0)
+    assert np.abs(host(cs) - ref).max() < 1e-5 * np.abs(rdx).sum(0).max() + 1e-12
+    # split-only output (the form the training step uses)
+    cs2 = empty(C)
+    b.bt_op_gelu_bwd_colsum(dev(x), dev(dy), N, C, 0, None, dxs, cs2, scratch(nb), nb)
+    assert np.array_equal(host(cs2), host(cs))
+
+
 # ------------------------------------------------------------------ softmax cross-entropy
 
 @pytest.mark.parametrize("N,Vp", [(256, 512), (64, 50304), (7, 1000), (3, 131072), (5, 4)])
