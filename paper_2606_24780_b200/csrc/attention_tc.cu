@@ -92,8 +92,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int qt = gridDim.x - 1 - blockIdx.x;           // heaviest query tiles first
-    const int b = blockIdx.y / g.H, h = blockIdx.y % g.H;
+    const int qt = gridDim.y - 1 - blockIdx.y;           // heaviest query tiles first, over all heads
+    const int b = blockIdx.x / g.H, h = blockIdx.x % g.H;
     const int q0 = qt * BQ;
     const int last_row = min(q0 + BQ - 1, g.T - 1);
     const int n_kt = last_row / BKV + 1;
@@ -366,6 +366,7 @@ bool encode3(CUtensorMap* tm, const float* base, int64_t cols, int64_t rows, int
 }  // namespace
 
 void attention_tc_set_trace(unsigned long long* p) { g_trace_ptr = p; }
+unsigned long long* attention_tc_get_trace() { return g_trace_ptr; }
 
 bool attention_tc_supports(int head_dim, int C) { return head_dim == 64 && (C % 4) == 0; }
 
@@ -390,7 +391,7 @@ cudaError_t launch_attention_fwd_tc(const float* qkv_hi, int64_t qkv_plane, int 
               encode3(&tmV, qkv_hi, cols, rows, cols, qkv_plane, 32, BKV, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
     if (!ok) return cudaErrorInvalidValue;
     AttnArgs g{T, C, H, o, o_hi, o_lo, lse, err_word, g_trace_ptr};
-    dim3 grid((T + BQ - 1) / BQ, B * H);
+    dim3 grid(B * H, (T + BQ - 1) / BQ);
     attn_fwd_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(tmQ, tmK, tmV, g);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();

@@ -30,6 +30,8 @@ namespace bt {
 
 using namespace tc;
 
+unsigned long long* attention_tc_get_trace();
+
 namespace {
 
 constexpr int HD = 64, BR = 128, BT_ = 32;  // head dim, rows owned by the CTA, streamed tile rows
@@ -113,7 +115,21 @@ struct BwdArgs {
     float* dqkv_hi;           // split output [2][B*T][3C]
     long long dqkv_plane;
     int* err;
+    unsigned long long* trace;   // optional timing trace of CTA (0,0) (debug aid, normally null)
 };
+
+// trace record: (tag, SM clock) in the recording role's own region (no atomics, so a mark costs
+// a few instructions); only block (0,0) records
+constexpr int kTraceRegion = 500;
+__device__ __forceinline__ void trace_mark(unsigned long long* tr, int role, int& n, unsigned long long tag) {
+    if (tr == nullptr || blockIdx.x != 0 || blockIdx.y != 0) return;
+    if (n < kTraceRegion) {
+        unsigned long long* p = tr + 2 + 2 * (role * kTraceRegion + n);
+        p[0] = tag;
+        p[1] = clock64();
+        ++n;
+    }
+}
 
 // Shared prologue: barriers + TMEM allocation.  Returns the TMEM base address.
 __device__ __forceinline__ uint32_t setup(uint32_t bars, int n_bars_count1, uint32_t p_bar0, int n_p_bars,
@@ -164,8 +180,10 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     const uint32_t tmem_slot = bars + 8u * 15;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int b = blockIdx.y / g.H, h = blockIdx.y % g.H;
-    const int j0 = blockIdx.x * BR;
+    // grid = (sequence x head, key block): blocks are dispatched x-fastest, so all the key blocks
+    // with the longest walks (low j0) start first and the short ones fill the tail
+    const int b = blockIdx.x / g.H, h = blockIdx.x % g.H;
+    const int j0 = blockIdx.y * BR;
     const int row_base = b * g.T;
     const int n_qt = (g.T + BT_ - 1) / BT_, qt0 = j0 / BT_;
     const int n_t = n_qt - qt0;
@@ -205,10 +223,13 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT_, false, false);   // 128 x 32, B K-major
             constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
             bool ok = mbar_wait(v_full, 0, g.err, 23) && mbar_wait(k_ready, 0, g.err, 24);
+            int tn = 0;
             const DescBase vd = kmaj_base(v_s);
             auto issue_a = [&](int t) -> bool {
                 const int st = t & 1, bb = t & 1;
+                trace_mark(g.trace, 0, tn, 100 + t);
                 if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 25)) return false;
+                trace_mark(g.trace, 0, tn, 200 + t);
                 tc_fence_after();
                 const uint32_t dS = tbuf(bb), dP = tbuf(bb) + 64u;
                 const DescBase qd = kmaj_base(qk_s(st)), od = kmaj_base(dok_s(st));
@@ -229,12 +250,15 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 }
                 umma_commit(kempty(st));
                 umma_commit(sdp_full(bb));
+                trace_mark(g.trace, 0, tn, 300 + t);
                 return true;
             };
             auto issue_b = [&](int t) -> bool {
                 const int st = t & 1, bb = t & 1;
                 if (!mbar_wait(pds_full(bb), (t >> 1) & 1u, g.err, 26)) return false;
+                trace_mark(g.trace, 0, tn, 400 + t);
                 if (!mbar_wait(mfull(st), (t >> 1) & 1u, g.err, 27)) return false;
+                trace_mark(g.trace, 0, tn, 500 + t);
                 tc_fence_after();
                 const uint32_t p_hi = tbuf(bb), p_lo = tbuf(bb) + 32u, s_hi = tbuf(bb) + 64u, s_lo = tbuf(bb) + 96u;
                 const DescBase omd = mnmaj_base(dom_s(st)), qmd = mnmaj_base(qm_s(st));
@@ -255,6 +279,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                     umma_tf32_ts(tdK, s_hi + ks * 8, q_hi, idesc_b, 1u);
                 }
                 umma_commit(mempty(st));
+                trace_mark(g.trace, 0, tn, 600 + t);
                 return true;
             };
             if (ok && n_t > 0) ok = issue_a(0);
@@ -281,6 +306,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             if (lane == 0) mbar_arrive(k_ready);
         }
         bool ok = true;
+        int tn = 0;
         const uint32_t tb = tbuf(wg) + t_lane;
         for (int t = wg; t < n_t && ok; t += 2) {
             const int q0 = (qt0 + t) * BT_;
@@ -297,12 +323,15 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 Lc[i] = __ldg(lse_t + ic) * kLog2e;
                 Dc[i] = __ldg(d_t + ic);
             }
+            if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 700 + t);
             if (!mbar_wait_warp(sdp_full(wg), (t >> 1) & 1u, g.err, 28)) { ok = false; break; }
+            if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 800 + t);
             tc_fence_after();
             uint32_t s[32], dp[32];
             tmem_ld32(tb, s);
             tmem_ld32(tb + 64u, dp);
             tmem_ld_wait();
+            if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 900 + t);
             uint32_t p_hi[32], p_lo[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
@@ -320,6 +349,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(pds_full(wg));
+            if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 1000 + t);
         }
         if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 29);
         if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
@@ -368,8 +398,8 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
     const uint32_t tmem_slot = bars + 8u * 15;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int qt = gridDim.x - 1 - blockIdx.x;                  // heaviest query tiles first
-    const int b = blockIdx.y / g.H, h = blockIdx.y % g.H;
+    const int qt = gridDim.y - 1 - blockIdx.y;                  // heaviest query tiles first, over all heads
+    const int b = blockIdx.x / g.H, h = blockIdx.x % g.H;
     const int q0 = qt * BR;
     const int row_base = b * g.T;
     const int n_t = min(q0 + BR - 1, g.T - 1) / BT_ + 1;         // key tiles up to the diagonal
@@ -557,8 +587,8 @@ cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, cons
               enc3(&vres, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BR, false) &&    // 128-row resident tiles
               enc3(&dores, do_hi, C, rows, do_plane, BR, false);
     if (!ok) return cudaErrorInvalidValue;
-    BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dqkv_hi, dqkv_plane, err_word};
-    dim3 gk((T + BR - 1) / BR, B * H);
+    BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dqkv_hi, dqkv_plane, err_word, attention_tc_get_trace()};
+    dim3 gk(B * H, (T + BR - 1) / BR);
     attn_bwd_dkv_tc_kernel<<<gk, kThreads, kDkvSmem, s>>>(qk32, qm32, dok32, dom32, vres, g);
     BT_COUNT_LAUNCH();
     attn_bwd_dq_tc_kernel<<<gk, kThreads, kDqSmem, s>>>(qk32, qm32, qk32, dores, g);
