@@ -46,6 +46,19 @@ __device__ __forceinline__ float ex2_approx(float x) {
     return y;
 }
 
+// Per-CTA (start, end, SM, tiles) record behind the mark regions of the trace buffer (debug aid).
+__device__ __forceinline__ void trace_cta(unsigned long long* tr, int kernel_index, int slot, unsigned long long v) {
+    if (tr == nullptr) return;
+    const unsigned long long n = (unsigned long long)gridDim.x * gridDim.y;
+    const unsigned long long id = (unsigned long long)blockIdx.y * gridDim.x + blockIdx.x;
+    tr[4002 + 4 * (kernel_index * n + id) + slot] = v;
+}
+__device__ __forceinline__ unsigned smid() {
+    unsigned r;
+    asm volatile("mov.u32 %0, %%smid;" : "=r"(r));
+    return r;
+}
+
 // Thread-owned row (64 floats given as hi/lo planes) -> x * mul -> hi/lo columns of tensor memory.
 __device__ __forceinline__ void row_to_tmem(const float* hi_row, const float* lo_row, float mul, uint32_t t_hi,
                                             uint32_t t_lo) {
@@ -187,6 +200,11 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     const int row_base = b * g.T;
     const int n_qt = (g.T + BT_ - 1) / BT_, qt0 = j0 / BT_;
     const int n_t = n_qt - qt0;
+    if (threadIdx.x == 0) {
+        trace_cta(g.trace, 0, 0, globaltimer_ns());
+        trace_cta(g.trace, 0, 2, smid());
+        trace_cta(g.trace, 0, 3, n_t);
+    }
 
     const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp);
     // TMEM columns
@@ -367,11 +385,23 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
     }
+    if (threadIdx.x == 0) trace_cta(g.trace, 0, 1, globaltimer_ns());
 }
 
 // ------------------------------------------------------------------------------------------- dq
 
-constexpr uint32_t kDqSmem = 1024u + kResBytes + 2u * 3u * kTileBytes + 256u;
+// The dq kernel streams 64-key tiles: its score products then run with N = 64 (an MMA costs the
+// same ~50 clocks for N = 32 and N = 64), and dS hi/lo overwrite S and dP in place, so two
+// 128-column buffers fit beside Q' and dQ.  Shared memory holds dO (64 KB), two stages of the
+// K-major K and V tiles (4 x 32 KB) and ONE stage of the MN-major K tile (32 KB): 224 KB.
+constexpr int BKT = 64;
+constexpr uint32_t kTileQ = 2u * 2u * BKT * 128u;   // one streamed 64-row tile in one layout (32 KB)
+constexpr uint32_t kDqSmem = 1024u + kResBytes + 5u * kTileQ + 256u;
+//  MN-major 64-row tile (2 column groups of [hi|lo][64 rows][128 B]), contraction over the rows.
+__device__ __forceinline__ constexpr uint32_t mnmaj64_off(int ks, bool lo) {
+    return (lo ? BKT * 128u : 0u) + (uint32_t)ks * 1024u;
+}
+__device__ __forceinline__ DescBase mnmaj64_base(uint32_t tile) { return make_desc_base(tile, 2u * BKT * 128u, 512u, 1u); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_constant__ CUtensorMap tmKm,
@@ -380,16 +410,16 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t do_s = base;                                 // resident dO (A operand of dP)
-    auto kk_s = [&](int st) { return base + kResBytes + (uint32_t)st * 3u * kTileBytes; };
-    auto vk_s = [&](int st) { return kk_s(st) + kTileBytes; };
-    auto km_s = [&](int st) { return kk_s(st) + 2u * kTileBytes; };
-    const uint32_t bars = base + kResBytes + 6u * kTileBytes;
-    // count-1: 0 do_full, 1-2 kfull, 3-4 kempty, 5-6 mfull, 7-8 mempty, 9-10 sdp_full, 11 acc_full
+    auto kk_s = [&](int st) { return base + kResBytes + (uint32_t)st * 2u * kTileQ; };
+    auto vk_s = [&](int st) { return kk_s(st) + kTileQ; };
+    const uint32_t km_s = base + kResBytes + 4u * kTileQ;       // single stage
+    const uint32_t bars = base + kResBytes + 5u * kTileQ;
+    // count-1: 0 do_full, 1-2 kfull, 3-4 kempty, 5 mfull, 7 mempty, 9-10 sdp_full, 11 acc_full
     const uint32_t do_full = bars;
     auto kfull = [&](int s) { return bars + 8u * (1 + s); };
     auto kempty = [&](int s) { return bars + 8u * (3 + s); };
-    auto mfull = [&](int s) { return bars + 8u * (5 + s); };
-    auto mempty = [&](int s) { return bars + 8u * (7 + s); };
+    const uint32_t mfull = bars + 8u * 5;
+    const uint32_t mempty = bars + 8u * 7;
     auto sdp_full = [&](int b) { return bars + 8u * (9 + b); };
     const uint32_t acc_full = bars + 8u * 11;
     // count-4: 12-13 ds_full, 14 q_ready
@@ -402,11 +432,16 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
     const int b = blockIdx.x / g.H, h = blockIdx.x % g.H;
     const int q0 = qt * BR;
     const int row_base = b * g.T;
-    const int n_t = min(q0 + BR - 1, g.T - 1) / BT_ + 1;         // key tiles up to the diagonal
+    const int n_t = min(q0 + BR - 1, g.T - 1) / BKT + 1;         // key tiles up to the diagonal
+    if (threadIdx.x == 0) {
+        trace_cta(g.trace, 1, 0, globaltimer_ns());
+        trace_cta(g.trace, 1, 2, smid());
+        trace_cta(g.trace, 1, 3, n_t);
+    }
 
     const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp);
     const uint32_t tQ_hi = tmem, tQ_lo = tmem + 64, tdQ = tmem + 128;
-    auto tbuf = [&](int bb) { return tmem + 192u + 96u * (uint32_t)bb; };   // +0 S|dS_hi, +32 dS_lo, +64 dP
+    auto tbuf = [&](int bb) { return tmem + 192u + 128u * (uint32_t)bb; };   // +0 S -> dS_hi, +64 dP -> dS_lo
 
     if (warp == 0) {
         if (lane == 0) {
@@ -414,38 +449,48 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             for (int kb = 0; kb < 2; ++kb)
                 tma_load_3d(do_s + kb * (kResBytes / 2), &tmDOres, do_full, h * HD + kb * 32, row_base + q0, 0);
             bool ok = true;
-            for (int t = 0; t < n_t && ok; ++t) {
-                const int st = t & 1, k0 = t * BT_;
-                const uint32_t ph = (t >> 1) & 1u;
-                if (!mbar_wait(kempty(st), ph ^ 1u, g.err, 31)) { ok = false; break; }
-                mbar_expect_tx(kfull(st), 2u * kTileBytes);
+            auto load_kmajor = [&](int t) -> bool {
+                const int st = t & 1, k0 = t * BKT;
+                if (!mbar_wait(kempty(st), ((t >> 1) & 1u) ^ 1u, g.err, 31)) return false;
+                mbar_expect_tx(kfull(st), 2u * kTileQ);
                 for (int kb = 0; kb < 2; ++kb) {
-                    tma_load_3d(kk_s(st) + kb * (kTileBytes / 2), &tmKk, kfull(st), g.C + h * HD + kb * 32, row_base + k0, 0);
-                    tma_load_3d(vk_s(st) + kb * (kTileBytes / 2), &tmVk, kfull(st), 2 * g.C + h * HD + kb * 32, row_base + k0, 0);
+                    tma_load_3d(kk_s(st) + kb * (kTileQ / 2), &tmKk, kfull(st), g.C + h * HD + kb * 32, row_base + k0, 0);
+                    tma_load_3d(vk_s(st) + kb * (kTileQ / 2), &tmVk, kfull(st), 2 * g.C + h * HD + kb * 32, row_base + k0, 0);
                 }
-                if (!mbar_wait(mempty(st), ph ^ 1u, g.err, 32)) { ok = false; break; }
-                mbar_expect_tx(mfull(st), kTileBytes);
+                return true;
+            };
+            // The K-major tiles of tile t+1 go out before the wait for the single MN-major buffer:
+            // the score products of t+1 are issued ahead of the dQ product of t.
+            ok = load_kmajor(0);
+            for (int t = 0; t < n_t && ok; ++t) {
+                if (t + 1 < n_t) ok = load_kmajor(t + 1);
+                if (!ok) break;
+                if (!mbar_wait(mempty, (t & 1u) ^ 1u, g.err, 32)) { ok = false; break; }
+                mbar_expect_tx(mfull, kTileQ);
                 for (int grp = 0; grp < 2; ++grp)
-                    tma_load_3d(km_s(st) + grp * (kTileBytes / 2), &tmKm, mfull(st), g.C + h * HD + grp * 32, row_base + k0, 0);
+                    tma_load_3d(km_s + grp * (kTileQ / 2), &tmKm, mfull, g.C + h * HD + grp * 32, row_base + t * BKT, 0);
             }
             if (!ok)
                 for (int i = 0; i < 2000; ++i) __nanosleep(1000);
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT_, false, false);
-            constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);
+            constexpr uint32_t idesc_a = make_idesc_tf32(BR, BKT, false, false);   // 128 x 64, B K-major
+            constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
             bool ok = mbar_wait(do_full, 0, g.err, 33) && mbar_wait(q_ready, 0, g.err, 34);
+            int tn = 0;
             const DescBase dod = kmaj_base(do_s);
             auto issue_a = [&](int t) -> bool {
                 const int st = t & 1, bb = t & 1;
+                trace_mark(g.trace, 0, tn, 100 + t);
                 if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 35)) return false;
+                trace_mark(g.trace, 0, tn, 200 + t);
                 tc_fence_after();
                 const uint32_t dS = tbuf(bb), dP = tbuf(bb) + 64u;
                 const DescBase kd = kmaj_base(kk_s(st)), vkd = kmaj_base(vk_s(st));
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t k_hi = kd.at(kmaj_off(BT_, ks, false)), k_lo = kd.at(kmaj_off(BT_, ks, true));
+                    const uint64_t k_hi = kd.at(kmaj_off(BKT, ks, false)), k_lo = kd.at(kmaj_off(BKT, ks, true));
                     umma_tf32_ts(dS, tQ_lo + ks * 8, k_hi, idesc_a, ks > 0 ? 1u : 0u);
                     umma_tf32_ts(dS, tQ_hi + ks * 8, k_lo, idesc_a, 1u);
                     umma_tf32_ts(dS, tQ_hi + ks * 8, k_hi, idesc_a, 1u);
@@ -453,31 +498,35 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t o_hi = dod.at(kmaj_off(BR, ks, false)), o_lo = dod.at(kmaj_off(BR, ks, true));
-                    const uint64_t v_hi = vkd.at(kmaj_off(BT_, ks, false)), v_lo = vkd.at(kmaj_off(BT_, ks, true));
+                    const uint64_t v_hi = vkd.at(kmaj_off(BKT, ks, false)), v_lo = vkd.at(kmaj_off(BKT, ks, true));
                     umma_tf32(dP, o_lo, v_hi, idesc_a, ks > 0 ? 1u : 0u);
                     umma_tf32(dP, o_hi, v_lo, idesc_a, 1u);
                     umma_tf32(dP, o_hi, v_hi, idesc_a, 1u);
                 }
                 umma_commit(kempty(st));
                 umma_commit(sdp_full(bb));
+                trace_mark(g.trace, 0, tn, 300 + t);
                 return true;
             };
             auto issue_b = [&](int t) -> bool {
-                const int st = t & 1, bb = t & 1;
+                const int bb = t & 1;
                 if (!mbar_wait(ds_full(bb), (t >> 1) & 1u, g.err, 36)) return false;
-                if (!mbar_wait(mfull(st), (t >> 1) & 1u, g.err, 37)) return false;
+                trace_mark(g.trace, 0, tn, 400 + t);
+                if (!mbar_wait(mfull, t & 1u, g.err, 37)) return false;
+                trace_mark(g.trace, 0, tn, 500 + t);
                 tc_fence_after();
-                const uint32_t s_hi = tbuf(bb), s_lo = tbuf(bb) + 32u;
-                const DescBase kmd = mnmaj_base(km_s(st));
+                const uint32_t s_hi = tbuf(bb), s_lo = tbuf(bb) + 64u;
+                const DescBase kmd = mnmaj64_base(km_s);
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t k_hi = kmd.at(mnmaj_off(ks, false)), k_lo = kmd.at(mnmaj_off(ks, true));
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t k_hi = kmd.at(mnmaj64_off(ks, false)), k_lo = kmd.at(mnmaj64_off(ks, true));
                     const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
                     umma_tf32_ts(tdQ, s_lo + ks * 8, k_hi, idesc_b, acc);
                     umma_tf32_ts(tdQ, s_hi + ks * 8, k_lo, idesc_b, 1u);
                     umma_tf32_ts(tdQ, s_hi + ks * 8, k_hi, idesc_b, 1u);
                 }
-                umma_commit(mempty(st));
+                umma_commit(mempty);
+                trace_mark(g.trace, 0, tn, 600 + t);
                 return true;
             };
             if (ok) ok = issue_a(0);
@@ -505,28 +554,35 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
         }
         const float L = g.lse[lb + rc] * kLog2e, D = g.dvec[lb + rc];
         bool ok = true;
+        int tn = 0;
         const uint32_t tb = tbuf(wg) + t_lane;
         for (int t = wg; t < n_t && ok; t += 2) {
-            const int k0 = t * BT_;
+            const int k0 = t * BKT;
+            if (lane_group == 0 && lane == 0) trace_mark(g.trace, 1 + wg, tn, 700 + t);
             if (!mbar_wait_warp(sdp_full(wg), (t >> 1) & 1u, g.err, 38)) { ok = false; break; }
+            if (lane_group == 0 && lane == 0) trace_mark(g.trace, 1 + wg, tn, 800 + t);
             tc_fence_after();
-            uint32_t s[32], dp[32];
-            tmem_ld32(tb, s);
-            tmem_ld32(tb + 64u, dp);
-            tmem_ld_wait();
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                float p = ex2_approx(__uint_as_float(s[i]) - L);
-                if (k0 + i > row) p = 0.f;                      // key follows this query: masked
-                const float ds = p * (__uint_as_float(dp[i]) - D);
-                split_tf32_int(ds, s[i], dp[i]);
+            for (int half = 0; half < 2; ++half) {
+                uint32_t s[32], dp[32];
+                tmem_ld32(tb + half * 32u, s);
+                tmem_ld32(tb + 64u + half * 32u, dp);
+                tmem_ld_wait();
+#pragma unroll
+                for (int i = 0; i < 32; ++i) {
+                    float p = ex2_approx(__uint_as_float(s[i]) - L);
+                    if (k0 + half * 32 + i > row) p = 0.f;          // key follows this query: masked
+                    const float ds = p * (__uint_as_float(dp[i]) - D);
+                    split_tf32_int(ds, s[i], dp[i]);
+                }
+                tmem_st32(tb + half * 32u, s);                      // dS hi over S
+                tmem_st32(tb + 64u + half * 32u, dp);               // dS lo over dP
             }
-            tmem_st32(tb, s);
-            tmem_st32(tb + 32u, dp);
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(ds_full(wg));
+            if (lane_group == 0 && lane == 0) trace_mark(g.trace, 1 + wg, tn, 1000 + t);
         }
         if (wg == 0) {
             if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 39);
@@ -542,6 +598,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
     if (warp == 1) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(512u) : "memory");
     }
+    if (threadIdx.x == 0) trace_cta(g.trace, 1, 1, globaltimer_ns());
 }
 
 bool enc3(CUtensorMap* tm, const float* base, int64_t cols, int64_t rows, int64_t plane, uint32_t box_rows,
@@ -586,12 +643,15 @@ cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, cons
               enc3(&dok32, do_hi, C, rows, do_plane, BT_, false) && enc3(&dom32, do_hi, C, rows, do_plane, BT_, true) &&
               enc3(&vres, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BR, false) &&    // 128-row resident tiles
               enc3(&dores, do_hi, C, rows, do_plane, BR, false);
+    CUtensorMap qk64, qm64;
+    ok = ok && enc3(&qk64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, false) &&  // 64-row tiles for the dq kernel
+         enc3(&qm64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, true);
     if (!ok) return cudaErrorInvalidValue;
     BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dqkv_hi, dqkv_plane, err_word, attention_tc_get_trace()};
     dim3 gk(B * H, (T + BR - 1) / BR);
     attn_bwd_dkv_tc_kernel<<<gk, kThreads, kDkvSmem, s>>>(qk32, qm32, dok32, dom32, vres, g);
     BT_COUNT_LAUNCH();
-    attn_bwd_dq_tc_kernel<<<gk, kThreads, kDqSmem, s>>>(qk32, qm32, qk32, dores, g);
+    attn_bwd_dq_tc_kernel<<<gk, kThreads, kDqSmem, s>>>(qk64, qm64, qk64, dores, g);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
