@@ -210,6 +210,13 @@ BT_API bt_status bt_op_layernorm_bwd(const float* dy, const float* x, const floa
                                      const float* rstd, const float* dres, int64_t N, int32_t C, float* dx,
                                      float* dx_split, float* dgamma, float* dbeta, void* scratch,
                                      size_t scratch_bytes, void* stream);
+/* The same, plus dx_colsum[C] (device) = the column sums of the dx written (residual included):
+ * in the pre-LN block (Section 2) that dx is the gradient at a residual-stream position, so its
+ * column sums are the bias gradient of the projection that wrote to that position.  Same scratch. */
+BT_API bt_status bt_op_layernorm_bwd_colsum(const float* dy, const float* x, const float* gamma, const float* mean,
+                                            const float* rstd, const float* dres, int64_t N, int32_t C, float* dx,
+                                            float* dx_split, float* dgamma, float* dbeta, float* dx_colsum,
+                                            void* scratch, size_t scratch_bytes, void* stream);
 
 /* Dense FP32 GEMM with 3xTF32 split accumulation on the tensor cores (the paper's GEMM
  * library serves QKV, attention-output and MLP projections in all forward and backward

@@ -66,6 +66,7 @@ _SIGNATURES = {
     "bt_op_layernorm_fwd": (_i32, [_vp, _vp, _vp, _i64, _i32, _vp, _vp, _vp, _vp, _vp]),
     "bt_op_layernorm_bwd_scratch_bytes": (_sz, [_i64, _i32]),
     "bt_op_layernorm_bwd": (_i32, [_vp] * 6 + [_i64, _i32] + [_vp] * 5 + [_sz, _vp]),
+    "bt_op_layernorm_bwd_colsum": (_i32, [_vp] * 6 + [_i64, _i32] + [_vp] * 6 + [_sz, _vp]),
     "bt_op_gemm_scratch_bytes": (_sz, [_i32, _i64, _i64, _i64]),
     "bt_op_split": (_i32, [_vp, _i64, _vp, _vp]),
     "bt_op_gemm_split_scratch_bytes": (_sz, []),
@@ -277,6 +278,13 @@ def bt_op_layernorm_bwd(dy, x, gamma, mean, rstd, dres, N, C, dx, dx_split, dgam
     _check(lib().bt_op_layernorm_bwd(_ptr(dy), _ptr(x), _ptr(gamma), _ptr(mean), _ptr(rstd), _ptr(dres), N, C,
                                      _ptr(dx), _ptr(dx_split), _ptr(dgamma), _ptr(dbeta), _ptr(scratch),
                                      scratch_bytes, _stream(stream)))
+
+
+def bt_op_layernorm_bwd_colsum(dy, x, gamma, mean, rstd, dres, N, C, dx, dx_split, dgamma, dbeta, dx_colsum, scratch,
+                               scratch_bytes, stream=None):
+    _check(lib().bt_op_layernorm_bwd_colsum(_ptr(dy), _ptr(x), _ptr(gamma), _ptr(mean), _ptr(rstd), _ptr(dres), N, C,
+                                            _ptr(dx), _ptr(dx_split), _ptr(dgamma), _ptr(dbeta), _ptr(dx_colsum),
+                                            _ptr(scratch), scratch_bytes, _stream(stream)))
 
 
 def bt_op_gemm_scratch_bytes(layout, M, N, K):

@@ -109,7 +109,7 @@ struct bt_model {
     uint8_t* decay_flags;
     std::vector<LayerAct> act;
     float *xL, *meanf, *rstdf, *xf_s, *logits, *dlogits_s, *losses, *loss, *norm_out;
-    float *dres, *dres_s, *dtmp, *do_s, *dqkv_s, *dh_s, *dg, *dvec;
+    float *dres, *dres_s, *dtmp, *do_s, *dqkv_s, *dh_s, *dg, *dvec, *attn_rg;
     float *partials, *ln_scratch, *colsum_scratch;
     void* norm_scratch;
     size_t partial_floats;
@@ -221,12 +221,15 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->dh_s = b.take<float>(2 * N * F);
     m->dg = b.take<float>(N * F);
     m->dvec = b.take<float>((int64_t)m->maxB * m->H * m->T);
+    m->attn_rg = b.take<float>(attention_bwd_rowgroups(m->maxB, m->T) * 3 * m->C);
     m->partial_floats = gemm_tc_partial_floats_bound();
     m->partials = b.take<float>(m->partial_floats);
     m->ln_scratch = b.take<float>(layernorm_bwd_scratch_floats(N, (int)C));
     size_t cs = colsum_scratch_floats(N, (int)F);
     if (colsum_scratch_floats(N, (int)C) > cs) cs = colsum_scratch_floats(N, (int)C);
     if (colsum_scratch_floats(N, 3 * (int)C) > cs) cs = colsum_scratch_floats(N, 3 * (int)C);
+    const size_t cs_rg = colsum_scratch_floats(attention_bwd_rowgroups(m->maxB, m->T), 3 * (int)C);
+    if (cs_rg > cs) cs = cs_rg;
     m->colsum_scratch = b.take<float>(cs);
     m->norm_scratch = b.take<uint8_t>(grad_norm_scratch_bytes(P));
     m->err_word = b.take<int>(4);
@@ -574,8 +577,10 @@ extern "C" bt_status bt_backward(bt_model* m) {
     BT_GEMM(kTN, Vp, C, N, dlog, act_mat(m->xf_s, N, C, N), G(m->tensors[0]), nullptr, nullptr);
     const Tensor& lnfg = m->tensors[m->tensors.size() - 2];
     const Tensor& lnfb = m->tensors[m->tensors.size() - 1];
+    // Every LayerNorm backward also sums the columns of the residual gradient it writes: that is
+    // the bias gradient of the projection whose output this residual stream position is.
     BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, m->xL, m->params + lnfg.off, m->meanf, m->rstdf, nullptr, N, C, m->dres,
-                                 m->dres_s, m->dres_s + N * C, G(lnfg), G(lnfb), m->ln_scratch, s));
+                                 m->dres_s, m->dres_s + N * C, G(lnfg), G(lnfb), G(layer_tensor(m, m->L - 1, PRB)), m->ln_scratch, s));
     SplitMat dres = act_mat(m->dres_s, N, C, N);
     for (int l = m->L - 1; l >= 0; --l) {
         LayerAct& a = m->act[l];
@@ -583,7 +588,6 @@ extern "C" bt_status bt_backward(bt_model* m) {
         // MLP down-projection: x_out = x1 + g . Wpr^T + bpr
         BT_GEMM(kNN, N, F, C, dres, weight_mat(m, LT(PRW), C, F), m->dg, nullptr, nullptr);
         BT_GEMM(kTN, C, F, N, dres, act_mat(a.g_s, N, F, N), G(LT(PRW)), nullptr, nullptr);
-        BT_STEP(kCatColsum, 0, 4.0 * N * C, launch_colsum(m->dres, nullptr, N, C, G(LT(PRB)), m->colsum_scratch, s));
         // d h, with its column sums (the gradient of bfc) taken in the same pass
         BT_STEP(kCatGeluBwd, 0, 16.0 * N * F, launch_gelu_bwd_colsum(a.h, m->dg, N, F, tanh_form, nullptr, m->dh_s, m->dh_s + N * F,
                                        G(LT(FCB)), m->colsum_scratch, s));
@@ -593,24 +597,31 @@ extern "C" bt_status bt_backward(bt_model* m) {
         BT_GEMM(kTN, F, C, N, dh, act_mat(a.m_s, N, C, N), G(LT(FCW)), nullptr, nullptr);
         // LN2 and the residual: d x1 = d x_out + LN2'(dm)
         BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, a.x1, m->params + LT(LN2G).off, a.mean2, a.rstd2, m->dres, N, C, m->dres,
-                                     m->dres_s, m->dres_s + N * C, G(LT(LN2G)), G(LT(LN2B)), m->ln_scratch, s));
+                                     m->dres_s, m->dres_s + N * C, G(LT(LN2G)), G(LT(LN2B)), G(LT(PROJB)), m->ln_scratch, s));
         // attention output projection: x1 = x + o . Wo^T + bo
         // d o, raw for the FMA / warp-MMA attention kernels, as hi/lo planes for the tcgen05 ones
         BT_GEMM_SPLIT_OUT(kNN, N, C, C, dres, weight_mat(m, LT(PROJW), C, C), raw_qkv ? m->dtmp : nullptr, m->do_s, nullptr,
                           nullptr);
         BT_GEMM(kTN, C, C, N, dres, act_mat(a.o_s, N, C, N), G(LT(PROJW)), nullptr, nullptr);
-        BT_STEP(kCatColsum, 0, 4.0 * N * C, launch_colsum(m->dres, nullptr, N, C, G(LT(PROJB)), m->colsum_scratch, s));
+        bool rg_written = false;
         BT_STEP(kCatAttnBwd, 2.5 * attn_fwd_flops(B, H, T, C / H), 48.0 * N * C, launch_attention_bwd(raw_qkv ? a.qkv : nullptr, a.qkv_s, N * 3 * C, a.o_s, a.o_s + N * C, a.lse,
                                      raw_qkv ? m->dtmp : nullptr, m->do_s, N * C, B, T,
-                                     C, H, nullptr, m->dqkv_s, m->dqkv_s + N * 3 * C, m->dvec, simt_attn, m->err_word, s));
+                                     C, H, nullptr, m->dqkv_s, m->dqkv_s + N * 3 * C, m->dvec, simt_attn, m->err_word, s,
+                                     m->attn_rg, &rg_written));
         // QKV projection: qkv = a . Wqkv^T + bqkv
         SplitMat dqkv = act_mat(m->dqkv_s, N, 3 * C, N);
         BT_GEMM(kNN, N, C, 3 * C, dqkv, weight_mat(m, LT(QKVW), 3 * C, C), m->dtmp, nullptr, nullptr);
         BT_GEMM(kTN, 3 * C, C, N, dqkv, act_mat(a.a_s, N, C, N), G(LT(QKVW)), nullptr, nullptr);
-        BT_STEP(kCatColsum, 0, 24.0 * N * C, launch_colsum(m->dqkv_s, m->dqkv_s + N * 3 * C, N, 3 * C, G(LT(QKVB)), m->colsum_scratch, s));
+        // d bqkv: from the attention kernels' per-row-group sums when they wrote them, else a pass over dqkv
+        if (rg_written)
+            BT_STEP(kCatColsum, 0, 12.0 * attention_bwd_rowgroups(B, T) * C,
+                    launch_colsum(m->attn_rg, nullptr, attention_bwd_rowgroups(B, T), 3 * C, G(LT(QKVB)), m->colsum_scratch, s));
+        else
+            BT_STEP(kCatColsum, 0, 24.0 * N * C, launch_colsum(m->dqkv_s, m->dqkv_s + N * 3 * C, N, 3 * C, G(LT(QKVB)), m->colsum_scratch, s));
         // LN1 and the residual: d x = d x1 + LN1'(da)
         BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, a.x, m->params + LT(LN1G).off, a.mean1, a.rstd1, m->dres, N, C, m->dres,
-                                     m->dres_s, m->dres_s + N * C, G(LT(LN1G)), G(LT(LN1B)), m->ln_scratch, s));
+                                     m->dres_s, m->dres_s + N * C, G(LT(LN1G)), G(LT(LN1B)),
+                                     l > 0 ? G(layer_tensor(m, l - 1, PRB)) : nullptr, m->ln_scratch, s));
     }
     // embeddings: dwte (already holding the LM-head part) += gather-transpose, dwpe = sum over sequences
     BT_STEP(kCatEmbedBwd, 0, 8.0 * N * C, launch_embedding_bwd(m->cur_tok, m->dres, N, T, C, G(m->tensors[0]), G(m->tensors[1]), s));
@@ -692,19 +703,36 @@ extern "C" size_t bt_op_layernorm_bwd_scratch_bytes(int64_t N, int32_t C) {
     return layernorm_bwd_scratch_floats(N, C) * sizeof(float);
 }
 
-extern "C" bt_status bt_op_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
-                                         const float* rstd, const float* dres, int64_t N, int32_t C, float* dx,
-                                         float* dx_split, float* dgamma, float* dbeta, void* scratch,
-                                         size_t scratch_bytes, void* stream) {
+static bt_status layernorm_bwd_impl(const float* dy, const float* x, const float* gamma, const float* mean,
+                                    const float* rstd, const float* dres, int64_t N, int32_t C, float* dx,
+                                    float* dx_split, float* dgamma, float* dbeta, float* dx_colsum, void* scratch,
+                                    size_t scratch_bytes, void* stream) {
     BT_PTR(dy); BT_PTR(x); BT_PTR(gamma); BT_PTR(mean); BT_PTR(rstd); BT_OPT_PTR(dres); BT_OPT_PTR(dx);
-    BT_OPT_PTR(dx_split); BT_PTR(dgamma); BT_PTR(dbeta); BT_PTR(scratch);
+    BT_OPT_PTR(dx_split); BT_PTR(dgamma); BT_PTR(dbeta); BT_OPT_PTR(dx_colsum); BT_PTR(scratch);
     if (N < 1 || C < 4 || C % 4) return fail(BT_ERR_INVALID_ARG, "layernorm_bwd: bad sizes");
     if (C > 1024) return fail(BT_ERR_UNSUPPORTED, "layernorm_bwd: C > 1024");
     if (scratch_bytes < bt_op_layernorm_bwd_scratch_bytes(N, C)) return fail(BT_ERR_OOM, "layernorm_bwd: scratch too small");
     BT_CUDA(launch_layernorm_bwd(dy, x, gamma, mean, rstd, dres, N, C, dx, dx_split,
-                                 dx_split ? dx_split + N * C : nullptr, dgamma, dbeta, (float*)scratch,
+                                 dx_split ? dx_split + N * C : nullptr, dgamma, dbeta, dx_colsum, (float*)scratch,
                                  (cudaStream_t)stream));
     return BT_OK;
+}
+
+extern "C" bt_status bt_op_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
+                                         const float* rstd, const float* dres, int64_t N, int32_t C, float* dx,
+                                         float* dx_split, float* dgamma, float* dbeta, void* scratch,
+                                         size_t scratch_bytes, void* stream) {
+    return layernorm_bwd_impl(dy, x, gamma, mean, rstd, dres, N, C, dx, dx_split, dgamma, dbeta, nullptr, scratch,
+                              scratch_bytes, stream);
+}
+
+extern "C" bt_status bt_op_layernorm_bwd_colsum(const float* dy, const float* x, const float* gamma, const float* mean,
+                                                const float* rstd, const float* dres, int64_t N, int32_t C, float* dx,
+                                                float* dx_split, float* dgamma, float* dbeta, float* dx_colsum,
+                                                void* scratch, size_t scratch_bytes, void* stream) {
+    if (!dx_colsum) return fail(BT_ERR_INVALID_ARG, "layernorm_bwd_colsum: dx_colsum is NULL");
+    return layernorm_bwd_impl(dy, x, gamma, mean, rstd, dres, N, C, dx, dx_split, dgamma, dbeta, dx_colsum, scratch,
+                              scratch_bytes, stream);
 }
 
 namespace {

@@ -13,7 +13,7 @@ cudaError_t launch_attention_dvec(const float* o, const float* o_lo, const float
                                   int T, int C, int H, float* dvec, cudaStream_t s);
 cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, const float* do_hi, int64_t do_plane,
                                     const float* lse, const float* dvec, int B, int T, int C, int H, float* dqkv_hi,
-                                    int64_t dqkv_plane, int* err_word, cudaStream_t s);
+                                    int64_t dqkv_plane, float* rg_sums, int* err_word, cudaStream_t s);
 bool attention_mma_supports(int head_dim);
 cudaError_t launch_attention_fwd_mma(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi,
                                      float* o_lo, float* lse, cudaStream_t s);
@@ -43,15 +43,18 @@ cudaError_t launch_attention_fwd(const float* qkv, const float* qkv_hi, int64_t 
 cudaError_t launch_attention_bwd(const float* qkv, const float* qkv_hi, int64_t qkv_plane, const float* o,
                                  const float* o_lo, const float* lse, const float* d_o, const float* do_hi,
                                  int64_t do_plane, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
-                                 float* dqkv_lo, float* dvec, bool simt, int* err_word, cudaStream_t s) {
+                                 float* dqkv_lo, float* dvec, bool simt, int* err_word, cudaStream_t s,
+                                 float* rg_sums, bool* rg_sums_written) {
+    if (rg_sums_written) *rg_sums_written = false;
     const bool tc = !simt && qkv_hi && do_hi && dqkv_hi && !dqkv && attention_tc_supports(C / H, C) &&
                     dqkv_lo == dqkv_hi + (int64_t)B * T * 3 * C;
     if (tc) {
         cudaError_t e = d_o ? launch_attention_dvec(o, o_lo, d_o, nullptr, B, T, C, H, dvec, s)
                             : launch_attention_dvec(o, o_lo, do_hi, do_hi + do_plane, B, T, C, H, dvec, s);
         if (e != cudaSuccess) return e;
+        if (rg_sums_written) *rg_sums_written = rg_sums != nullptr;
         return launch_attention_bwd_tc(qkv_hi, qkv_plane, do_hi, do_plane, lse, dvec, B, T, C, H, dqkv_hi,
-                                       (int64_t)B * T * 3 * C, err_word, s);
+                                       (int64_t)B * T * 3 * C, rg_sums, err_word, s);
     }
     if (!qkv || !d_o) return cudaErrorInvalidValue;
     if (simt || !attention_mma_supports(C / H))

@@ -84,25 +84,48 @@ __device__ __forceinline__ void row_to_tmem(const float* hi_row, const float* lo
     tmem_st_wait();
 }
 
+// Column sums over the 32 rows a warp owns: v[i] is column i of this lane's row; the result is the
+// sum of column `lane` over the 32 lanes (a halving butterfly: 31 shuffles, fixed order).
+__device__ __forceinline__ float warp_colsum32(float (&v)[32], int lane) {
+#pragma unroll
+    for (int off = 16; off >= 1; off >>= 1) {
+        const bool upper = (lane & off) != 0;
+#pragma unroll
+        for (int i = 0; i < off; ++i) {
+            const float send = upper ? v[i] : v[i + off];
+            const float keep = upper ? v[i + off] : v[i];
+            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
+        }
+    }
+    return v[0];
+}
+
 // Thread-owned accumulator row (64 tensor-memory columns) * mul -> hi/lo planes in global memory.
 // The tensor-memory loads are .sync.aligned: EVERY lane of the warp must call this; `store` says
 // whether this lane's row exists (rows past the end of the sequence are read and dropped).
+// sums (nullable): 64 floats that receive the column sums over the warp's existing rows.
 __device__ __forceinline__ void tmem_row_to_split(uint32_t t_row, float mul, float* hi_row, float* lo_row,
-                                                  bool store) {
+                                                  bool store, float* sums, int lane) {
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
         uint32_t r[32];
         tmem_ld32(t_row + half * 32, r);
         tmem_ld_wait();
-        if (!store) continue;
+        float v[32];
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-            float4 v = make_float4(__uint_as_float(r[i]) * mul, __uint_as_float(r[i + 1]) * mul,
-                                   __uint_as_float(r[i + 2]) * mul, __uint_as_float(r[i + 3]) * mul);
-            float4 h, l;
-            split_tf32(v, h, l);
-            *reinterpret_cast<float4*>(hi_row + half * 32 + i) = h;
-            *reinterpret_cast<float4*>(lo_row + half * 32 + i) = l;
+        for (int i = 0; i < 32; ++i) v[i] = store ? __uint_as_float(r[i]) * mul : 0.f;
+        if (store) {
+#pragma unroll
+            for (int i = 0; i < 32; i += 4) {
+                float4 h, l;
+                split_tf32(make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]), h, l);
+                *reinterpret_cast<float4*>(hi_row + half * 32 + i) = h;
+                *reinterpret_cast<float4*>(lo_row + half * 32 + i) = l;
+            }
+        }
+        if (sums) {   // warp-uniform
+            const float t = warp_colsum32(v, lane);
+            sums[half * 32 + lane] = t;
         }
     }
 }
@@ -129,6 +152,8 @@ struct BwdArgs {
     long long dqkv_plane;
     int* err;
     unsigned long long* trace;   // optional timing trace of CTA (0,0) (debug aid, normally null)
+    float* rg_sums;           // optional [B * nrg][3C]: column sums of dqkv over each 32-row group
+    int nrg;                  // 32-row groups per sequence (4 per 128-row block)
 };
 
 // trace record: (tag, SM clock) in the recording role's own region (no atomics, so a mark costs
@@ -376,8 +401,11 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             const int64_t off = (int64_t)(row_base + (valid ? key : 0)) * gs + h * HD;
             float* hi = g.dqkv_hi + off;
             float* lo = hi + g.dqkv_plane;
-            if (wg == 0) tmem_row_to_split(tdK + t_lane, scale, hi + g.C, lo + g.C, valid);
-            else tmem_row_to_split(tdV + t_lane, 1.0f, hi + 2 * g.C, lo + 2 * g.C, valid);
+            float* sums = g.rg_sums
+                              ? g.rg_sums + ((int64_t)b * g.nrg + (j0 >> 5) + lane_group) * gs + h * HD
+                              : nullptr;
+            if (wg == 0) tmem_row_to_split(tdK + t_lane, scale, hi + g.C, lo + g.C, valid, sums ? sums + g.C : nullptr, lane);
+            else tmem_row_to_split(tdV + t_lane, 1.0f, hi + 2 * g.C, lo + 2 * g.C, valid, sums ? sums + 2 * g.C : nullptr, lane);
         }
     }
     tc_fence_before();
@@ -589,7 +617,11 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
                 tc_fence_after();
                 const int64_t off = (int64_t)(row_base + rc) * gs + h * HD;
-                tmem_row_to_split(tdQ + t_lane, scale, g.dqkv_hi + off, g.dqkv_hi + g.dqkv_plane + off, row < g.T);
+                float* sums = g.rg_sums
+                                  ? g.rg_sums + ((int64_t)b * g.nrg + (q0 >> 5) + lane_group) * gs + h * HD
+                                  : nullptr;
+                tmem_row_to_split(tdQ + t_lane, scale, g.dqkv_hi + off, g.dqkv_hi + g.dqkv_plane + off, row < g.T, sums,
+                                  lane);
             }
         }
     }
@@ -619,10 +651,15 @@ bool enc3(CUtensorMap* tm, const float* base, int64_t cols, int64_t rows, int64_
 
 cudaError_t attention_tc_default_err(int** out);
 
+// Rows of the optional row-group sums array: one per 32 rows of every 128-row block.
+int64_t attention_bwd_rowgroups(int B, int T) { return (int64_t)B * 4 * ((T + BR - 1) / BR); }
+
 // dqkv (hi/lo planes) from qkv (hi/lo planes), dO (hi/lo planes), lse and dvec = rowsum(dO o O).
+// rg_sums (nullable, [attention_bwd_rowgroups][3C]): column sums of dqkv per 32-row group; summing
+// its rows gives the gradient of the QKV bias without another pass over dqkv.
 cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, const float* do_hi, int64_t do_plane,
                                     const float* lse, const float* dvec, int B, int T, int C, int H, float* dqkv_hi,
-                                    int64_t dqkv_plane, int* err_word, cudaStream_t s) {
+                                    int64_t dqkv_plane, float* rg_sums, int* err_word, cudaStream_t s) {
     static cudaError_t attr = []() {
         cudaError_t e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kDkvSmem);
@@ -647,7 +684,8 @@ cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, cons
     ok = ok && enc3(&qk64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, false) &&  // 64-row tiles for the dq kernel
          enc3(&qm64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, true);
     if (!ok) return cudaErrorInvalidValue;
-    BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dqkv_hi, dqkv_plane, err_word, attention_tc_get_trace()};
+    BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dqkv_hi, dqkv_plane, err_word, attention_tc_get_trace(), rg_sums,
+              4 * ((T + BR - 1) / BR)};
     dim3 gk(B * H, (T + BR - 1) / BR);
     attn_bwd_dkv_tc_kernel<<<gk, kThreads, kDkvSmem, s>>>(qk32, qm32, dok32, dom32, vres, g);
     BT_COUNT_LAUNCH();

@@ -97,7 +97,8 @@ cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float
 size_t layernorm_bwd_scratch_floats(int64_t N, int C);
 cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
                                  const float* rstd, const float* dres, int64_t N, int C, float* dx, float* dx_hi,
-                                 float* dx_lo, float* dgamma, float* dbeta, float* scratch, cudaStream_t s);
+                                 float* dx_lo, float* dgamma, float* dbeta, float* dx_colsum, float* scratch,
+                                 cudaStream_t s);   // dx_colsum (nullable): column sums of the dx written
 cudaError_t launch_gelu_fwd(const float* x, int64_t n, int tanh_form, float* y, float* y_hi, float* y_lo,
                             cudaStream_t s);
 cudaError_t launch_gelu_bwd(const float* x, const float* dy, int64_t n, int tanh_form, float* dx, float* dx_hi,
@@ -160,6 +161,11 @@ cudaError_t attention_tc_default_err(int** out);
 cudaError_t launch_attention_bwd(const float* qkv, const float* qkv_hi, int64_t qkv_plane, const float* o,
                                  const float* o_lo, const float* lse, const float* d_o, const float* do_hi,
                                  int64_t do_plane, int B, int T, int C, int H, float* dqkv, float* dqkv_hi,
-                                 float* dqkv_lo, float* dvec, bool simt, int* err_word, cudaStream_t s);
+                                 float* dqkv_lo, float* dvec, bool simt, int* err_word, cudaStream_t s,
+                                 float* rg_sums = nullptr, bool* rg_sums_written = nullptr);
+// rg_sums (nullable): [attention_bwd_rowgroups(B, T)][3C] floats; when the tcgen05 kernels run they
+// fill it with the column sums of dqkv per 32-row group (*rg_sums_written = true), so the QKV bias
+// gradient is the column sum of this small array.
+int64_t attention_bwd_rowgroups(int B, int T);
 
 }  // namespace bt

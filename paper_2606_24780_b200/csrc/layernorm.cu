@@ -88,15 +88,23 @@ static inline int ln_bwd_ctas(int64_t N) {
     if (g > 148 * 2) g = 148 * 2;  // two CTAs per SM, one wave
     return (int)g;
 }
-size_t layernorm_bwd_scratch_floats(int64_t N, int C) { return (size_t)ln_bwd_ctas(N) * 2 * C; }
+size_t layernorm_bwd_scratch_floats(int64_t N, int C) { return (size_t)ln_bwd_ctas(N) * 3 * C; }
 
-template <int VPL>
+// CS: also accumulate the column sums of the rows written to dx (the bias gradient of the linear
+// layer whose output this dx is the gradient of).  Those sums live in shared memory, one private
+// array per warp, so they cost no registers.
+template <int VPL, bool CS>
 __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     const float* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ gamma,
     const float* __restrict__ mean, const float* __restrict__ rstd, const float* dres, int64_t N, int C4,
     float* dx, float* dx_hi, float* dx_lo, float* __restrict__ partial) {
-    extern __shared__ float4 sm[];  // [2][C4]
+    extern __shared__ float4 sm[];  // [2][C4], then (CS) [kLnWarps][C4]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float4* cs = sm + 2 * C4 + warp * C4;
+    if (CS) {
+        for (int i = lane; i < C4; i += 32) cs[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+        __syncwarp();
+    }
     const float inv_c = 1.0f / (float)(C4 * 4);
     // Per-lane running sums of dy*xhat and dy for the columns this lane owns.  Only x, dy and
     // these sums stay in registers (gamma is re-read through L1 each row), which keeps the kernel
@@ -146,6 +154,7 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
                 r.w = rs * (dv[k].w - s1 - xv[k].w * s2);
                 if (dres) r = add4(r, ld4(dres, row * C4 + idx));
                 store_raw_split(r, dx, dx_hi, dx_lo, row * C4 + idx);
+                if (CS) cs[idx] = add4(cs[idx], r);
             }
         }
     }
@@ -168,48 +177,67 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
         }
         __syncthreads();
     }
-    float4* dst = reinterpret_cast<float4*>(partial) + (int64_t)blockIdx.x * 2 * C4;
+    constexpr int kParts = CS ? 3 : 2;
+    float4* dst = reinterpret_cast<float4*>(partial) + (int64_t)blockIdx.x * kParts * C4;
     for (int i = threadIdx.x; i < 2 * C4; i += blockDim.x) dst[i] = sm[i];
+    if (CS) {   // the loop above ended with a __syncthreads, so every warp's array is complete
+        for (int i = threadIdx.x; i < C4; i += blockDim.x) {
+            float4 t = sm[2 * C4 + i];
+#pragma unroll
+            for (int w = 1; w < kLnWarps; ++w) t = add4(t, sm[(2 + w) * C4 + i]);
+            dst[2 * C4 + i] = t;
+        }
+    }
 }
 
 // Sums the per-CTA partials in a fixed order: lane = float4 column, warp w takes partials
 // w, w+8, ... (four loads in flight), the eight warp sums are combined in warp order.
 __global__ void __launch_bounds__(256) ln_bwd_reduce_kernel(const float* __restrict__ partial, int nparts, int C4,
-                                                            float* __restrict__ dgamma, float* __restrict__ dbeta) {
+                                                            int kparts, float* __restrict__ dgamma,
+                                                            float* __restrict__ dbeta, float* __restrict__ dcolsum) {
     __shared__ float4 sm[8][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int c = blockIdx.x * 32 + lane;  // float4 column over [2*C4): first dgamma, then dbeta
+    const int c = blockIdx.x * 32 + lane;  // float4 column over [kparts*C4): dgamma, dbeta, column sums
+    const int W = kparts * C4;
     float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (c < 2 * C4) {
+    if (c < W) {
         int p = warp;
         for (; p + 24 < nparts; p += 32) {
-            float4 a0 = ld4(partial, (int64_t)p * 2 * C4 + c), a1 = ld4(partial, (int64_t)(p + 8) * 2 * C4 + c);
-            float4 a2 = ld4(partial, (int64_t)(p + 16) * 2 * C4 + c), a3 = ld4(partial, (int64_t)(p + 24) * 2 * C4 + c);
+            float4 a0 = ld4(partial, (int64_t)p * W + c), a1 = ld4(partial, (int64_t)(p + 8) * W + c);
+            float4 a2 = ld4(partial, (int64_t)(p + 16) * W + c), a3 = ld4(partial, (int64_t)(p + 24) * W + c);
             t = add4(add4(add4(add4(t, a0), a1), a2), a3);
         }
-        for (; p < nparts; p += 8) t = add4(t, ld4(partial, (int64_t)p * 2 * C4 + c));
+        for (; p < nparts; p += 8) t = add4(t, ld4(partial, (int64_t)p * W + c));
     }
     sm[warp][lane] = t;
     __syncthreads();
-    if (warp == 0 && c < 2 * C4) {
+    if (warp == 0 && c < W) {
         float4 r = sm[0][lane];
 #pragma unroll
         for (int w = 1; w < 8; ++w) r = add4(r, sm[w][lane]);
         if (c < C4) reinterpret_cast<float4*>(dgamma)[c] = r;
-        else reinterpret_cast<float4*>(dbeta)[c - C4] = r;
+        else if (c < 2 * C4) reinterpret_cast<float4*>(dbeta)[c - C4] = r;
+        else reinterpret_cast<float4*>(dcolsum)[c - 2 * C4] = r;
     }
 }
 
 cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
                                  const float* rstd, const float* dres, int64_t N, int C, float* dx, float* dx_hi,
-                                 float* dx_lo, float* dgamma, float* dbeta, float* scratch, cudaStream_t s) {
+                                 float* dx_lo, float* dgamma, float* dbeta, float* dx_colsum, float* scratch,
+                                 cudaStream_t s) {
     const int C4 = C / 4;
     const int vpl = (C4 + 31) / 32;
     const int grid = ln_bwd_ctas(N);
-    const size_t smem = (size_t)2 * C4 * sizeof(float4);
-#define BT_LN_BWD(V)                                                                                         \
-    ln_bwd_kernel<V><<<grid, kLnWarps * 32, smem, s>>>(dy, x, gamma, mean, rstd, dres, N, C4, dx, dx_hi, dx_lo, \
-                                                        scratch)
+    const size_t smem = (size_t)(dx_colsum ? 2 + kLnWarps : 2) * C4 * sizeof(float4);
+#define BT_LN_BWD(V)                                                                                          \
+    do {                                                                                                      \
+        if (dx_colsum)                                                                                        \
+            ln_bwd_kernel<V, true><<<grid, kLnWarps * 32, smem, s>>>(dy, x, gamma, mean, rstd, dres, N, C4, dx, \
+                                                                     dx_hi, dx_lo, scratch);                  \
+        else                                                                                                  \
+            ln_bwd_kernel<V, false><<<grid, kLnWarps * 32, smem, s>>>(dy, x, gamma, mean, rstd, dres, N, C4, dx, \
+                                                                      dx_hi, dx_lo, scratch);                 \
+    } while (0)
     if (vpl <= 1) BT_LN_BWD(1);
     else if (vpl <= 2) BT_LN_BWD(2);
     else if (vpl <= 4) BT_LN_BWD(4);
@@ -218,7 +246,8 @@ cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* g
     else return cudaErrorInvalidValue;
 #undef BT_LN_BWD
     BT_COUNT_LAUNCH();
-    ln_bwd_reduce_kernel<<<(2 * C4 + 31) / 32, 256, 0, s>>>(scratch, grid, C4, dgamma, dbeta);
+    const int kparts = dx_colsum ? 3 : 2;
+    ln_bwd_reduce_kernel<<<(kparts * C4 + 31) / 32, 256, 0, s>>>(scratch, grid, C4, kparts, dgamma, dbeta, dx_colsum);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }

@@ -98,6 +98,27 @@ def test_layernorm_bwd_in_place_residual():
     assert rel_l2(host(buf), rdx + dres) < 1e-5
 
 
+@pytest.mark.parametrize("N,C", [(1000, 768), (37, 132), (8192, 1024), (3, 4)])
+def test_layernorm_bwd_colsum(N, C):
+    """The variant with fused column sums: same dx / dgamma / dbeta, plus colsum(dx) incl. residual."""
+    x, dy, dres = si.normal_f32(31, (N, C), 1.5), si.normal_f32(32, (N, C), 1e-2), si.normal_f32(33, (N, C), 1e-2)
+    g = (1.0 + si.normal_f32(34, (C,), 0.1)).astype(np.float32)
+    rm, rr = oracle.layernorm_fwd(x, g, np.zeros(C, np.float32))[1:3]
+    mean, rstd = dev(rm, torch.float32), dev(rr, torch.float32)
+    nb = b.bt_op_layernorm_bwd_scratch_bytes(N, C)
+    dx0, dg0, db0 = empty(N, C), empty(C), empty(C)
+    b.bt_op_layernorm_bwd(dev(dy), dev(x), dev(g), mean, rstd, dev(dres), N, C, dx0, None, dg0, db0, scratch(nb), nb)
+    dx1, dxs, dg1, db1, cs = empty(N, C), empty(2, N, C), empty(C), empty(C), empty(C)
+    b.bt_op_layernorm_bwd_colsum(dev(dy), dev(x), dev(g), mean, rstd, dev(dres), N, C, dx1, dxs, dg1, db1, cs,
+                                 scratch(nb), nb)
+    assert np.array_equal(host(dx0), host(dx1)) and np.array_equal(host(dg0), host(dg1))
+    assert np.array_equal(host(db0), host(db1))
+    check_split(dxs, host(dx1))
+    rdx, _, _ = oracle.layernorm_bwd(dy, x, g, host(mean), host(rstd))
+    ref = (rdx.astype(np.float64) + dres).sum(0)
+    assert np.abs(host(cs) - ref).max() < 1e-5 * np.abs(rdx + dres).sum(0).max() + 1e-12
+
+
 # ------------------------------------------------------------------ GELU
 
 @pytest.mark.parametrize("tanh_form", [0, 1])
