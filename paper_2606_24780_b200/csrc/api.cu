@@ -76,8 +76,8 @@ enum ProfCat {
     kCatLnBwd, kCatGeluBwd, kCatAttnBwd, kCatColsum, kCatEmbedBwd, kCatGradNorm, kCatAdamW, kNumCats
 };
 const char* const kCatNames[kNumCats] = {
-    "split_weights", "embedding_fwd", "layernorm_fwd", "gemm_nt", "attention_fwd", "gelu_fwd", "softmax_xent",
-    "gemm_nn", "gemm_tn", "layernorm_bwd", "gelu_bwd", "attention_bwd", "colsum", "embedding_bwd", "grad_norm",
+    "split_weights", "embedding_fwd", "layernorm_fwd", "gemm_fwd", "attention_fwd", "gelu_fwd", "softmax_xent",
+    "gemm_dx", "gemm_dw", "layernorm_bwd", "gelu_bwd", "attention_bwd", "colsum", "embedding_bwd", "grad_norm",
     "adamw"};
 
 struct LayerAct {
@@ -105,7 +105,9 @@ struct bt_model {
     int L, C, H, T, V, Vp, F, maxB;
     std::vector<Tensor> tensors;
     int64_t P;  // padded parameter count (multiple of 1024)
-    float *params, *grads, *mom1, *mom2, *wsplit;
+    float *params, *grads, *mom1, *mom2, *wsplit, *wsplit_t;
+    MatDesc* mat_descs;   // device table of the weight matrices (for the split in both orientations)
+    int n_mats, n_mat_tiles;
     uint8_t* decay_flags;
     std::vector<LayerAct> act;
     float *xL, *meanf, *rstdf, *xf_s, *logits, *dlogits_s, *losses, *loss, *norm_out;
@@ -169,6 +171,7 @@ bt_status validate(const bt_config* c) {
         return fail(BT_ERR_UNSUPPORTED, "config: head_dim %d not in {16,32,64,128}", d);
     if (c->d_model % 32) return fail(BT_ERR_INVALID_ARG, "config: d_model %% 32 != 0");
     if (c->d_model > 1024) return fail(BT_ERR_UNSUPPORTED, "config: d_model > 1024 not compiled");
+    if (1 + 4 * (int64_t)c->n_layers > kMaxSplitMats) return fail(BT_ERR_UNSUPPORTED, "config: more than 63 layers");
     if (c->padded_vocab_size < c->vocab_size) return fail(BT_ERR_INVALID_ARG, "config: padded_vocab < vocab");
     if (c->padded_vocab_size % 32) return fail(BT_ERR_INVALID_ARG, "config: padded_vocab %% 32 != 0");
     if ((int64_t)c->max_batch * c->seq_len > (1 << 24))
@@ -185,6 +188,8 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->mom1 = b.take<float>(P);
     m->mom2 = b.take<float>(P);
     m->wsplit = b.take<float>(2 * P);
+    m->wsplit_t = b.take<float>(2 * P);
+    m->mat_descs = b.take<MatDesc>(kMaxSplitMats);
     m->decay_flags = b.take<uint8_t>(P / 1024);
     m->act.resize(m->L);
     for (int l = 0; l < m->L; ++l) {
@@ -257,6 +262,10 @@ enum { LN1G = 0, LN1B, QKVW, QKVB, PROJW, PROJB, LN2G, LN2B, FCW, FCB, PRW, PRB 
 inline SplitMat weight_mat(bt_model* m, const Tensor& t, int64_t rows, int64_t cols) {
     return SplitMat{m->wsplit + t.off, m->P, rows, cols, cols};
 }
+// The transposed copy of a [rows, cols] weight: [cols, rows] row-major.
+inline SplitMat weight_mat_t(bt_model* m, const Tensor& t, int64_t rows, int64_t cols) {
+    return SplitMat{m->wsplit_t + t.off, m->P, cols, rows, rows};
+}
 inline SplitMat act_mat(const float* hi, int64_t rows, int64_t cols, int64_t plane_rows) {
     return SplitMat{hi, plane_rows * cols, rows, cols, cols};
 }
@@ -309,13 +318,16 @@ cudaError_t gemm_raw(bt_model* m, int layout, int64_t M, int64_t N, int64_t K, S
                           m->stream, d_split, M * N);
 }
 
+// Timing category by role: the forward products (Y = X W^T, run as NN on the transposed weight
+// copy), the input gradients (NN on the weight) and the weight gradients (TN).
+#define BT_GEMM_CAT(fwd, layout) ((fwd) ? kCatGemmNT : (layout) == kTN ? kCatGemmTN : kCatGemmNN)
 #define BT_GEMM(layout, M, N, K, A, B, D, bias, res)                                                        \
-    BT_STEP((layout) == kNT ? kCatGemmNT : (layout) == kNN ? kCatGemmNN : kCatGemmTN, gemm_flops(M, N, K),     \
-            gemm_bytes(M, N, K), gemm_raw(m, layout, M, N, K, A, B, D, bias, res))
+    BT_STEP(BT_GEMM_CAT(gemm_is_fwd, layout), gemm_flops(M, N, K), gemm_bytes(M, N, K),                         \
+            gemm_raw(m, layout, M, N, K, A, B, D, bias, res))
 // same, the output also written as TF32 hi/lo planes at DS
 #define BT_GEMM_SPLIT_OUT(layout, M, N, K, A, B, D, DS, bias, res)                                           \
-    BT_STEP((layout) == kNT ? kCatGemmNT : (layout) == kNN ? kCatGemmNN : kCatGemmTN, gemm_flops(M, N, K),     \
-            gemm_bytes(M, N, K) + 8.0 * (M) * (N), gemm_raw(m, layout, M, N, K, A, B, D, bias, res, DS))
+    BT_STEP(BT_GEMM_CAT(gemm_is_fwd, layout), gemm_flops(M, N, K), gemm_bytes(M, N, K) + 8.0 * (M) * (N),       \
+            gemm_raw(m, layout, M, N, K, A, B, D, bias, res, DS))
 
 bt_status check_device_error(bt_model* m) {
     int err = 0;
@@ -370,7 +382,26 @@ extern "C" bt_status bt_model_create(const bt_config* cfg, void* d_workspace, si
     for (const Tensor& t : m->tensors)
         if (t.decay)
             for (int64_t c = t.off / 1024; c < (t.off + t.numel + 1023) / 1024; ++c) flags[(size_t)c] = 1;
+    // table of the GEMM weight matrices, with their 64x64 tiles numbered consecutively
+    std::vector<MatDesc> descs;
+    int tiles = 0;
+    auto add_mat = [&](const Tensor& t, int rows, int cols) {
+        MatDesc d{(long long)t.off, rows, cols, tiles, (cols + 63) / 64};
+        tiles += ((rows + 63) / 64) * d.tiles_c;
+        descs.push_back(d);
+    };
+    add_mat(m->tensors[0], m->Vp, m->C);
+    for (int l = 0; l < m->L; ++l) {
+        add_mat(layer_tensor(m, l, QKVW), 3 * m->C, m->C);
+        add_mat(layer_tensor(m, l, PROJW), m->C, m->C);
+        add_mat(layer_tensor(m, l, FCW), m->F, m->C);
+        add_mat(layer_tensor(m, l, PRW), m->C, m->F);
+    }
+    m->n_mats = (int)descs.size();
+    m->n_mat_tiles = tiles;
     cudaError_t e = cudaMemcpyAsync(m->decay_flags, flags.data(), flags.size(), cudaMemcpyHostToDevice, m->stream);
+    if (e == cudaSuccess)
+        e = cudaMemcpyAsync(m->mat_descs, descs.data(), descs.size() * sizeof(MatDesc), cudaMemcpyHostToDevice, m->stream);
     if (e == cudaSuccess) e = cudaMemsetAsync(m->params, 0, (size_t)m->P * 4 * sizeof(float), m->stream);  // p,g,m,v
     if (e == cudaSuccess) e = cudaMemsetAsync(m->err_word, 0, 4 * sizeof(int), m->stream);
     if (e == cudaSuccess) e = cudaStreamSynchronize(m->stream);
@@ -509,8 +540,7 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
     cudaStream_t s = m->stream;
     const int C = m->C, F = m->F, T = m->T, H = m->H, Vp = m->Vp;
     const int64_t N = (int64_t)B * T;
-    const int64_t Nmax = (int64_t)m->maxB * T;  // plane stride of split activations uses the current N
-    (void)Nmax;
+    constexpr bool gemm_is_fwd = true;   // timing category of this function's GEMMs
     const bool simt_attn = (m->cfg.flags & BT_FLAG_ATTN_SIMT) != 0;
     const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
     // the tcgen05 attention kernels read qkv only as hi/lo planes; the raw copy is written only
@@ -518,7 +548,8 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
     const bool raw_qkv = simt_attn || (C / H) != 64 || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
 
     // hi/lo planes of every parameter (weights are GEMM operands; one streaming pass)
-    BT_STEP(kCatSplit, 0, 12.0 * m->P, launch_split(m->params, m->wsplit, m->wsplit + m->P, m->P, s));
+    BT_STEP(kCatSplit, 0, 20.0 * m->P, launch_split_matrices(m->params, m->wsplit, m->wsplit_t, m->P, m->mat_descs, m->n_mats,
+                                  m->n_mat_tiles, s));
     BT_STEP(kCatEmbedFwd, N * C, 12.0 * N * C, launch_embedding_fwd(d_tokens, m->params + m->tensors[0].off, m->params + m->tensors[1].off, N, T, C,
                                  m->act[0].x, s));
     for (int l = 0; l < m->L; ++l) {
@@ -526,24 +557,24 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
         float* xout = (l + 1 < m->L) ? m->act[l + 1].x : m->xL;
         auto P = [&](int k) { return m->params + layer_tensor(m, l, k).off; };
         BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x, P(LN1G), P(LN1B), N, C, nullptr, a.a_s, a.a_s + N * C, a.mean1, a.rstd1, s));
-        BT_GEMM_SPLIT_OUT(kNT, N, 3 * C, C, act_mat(a.a_s, N, C, N), weight_mat(m, layer_tensor(m, l, QKVW), 3 * C, C),
+        BT_GEMM_SPLIT_OUT(kNN, N, 3 * C, C, act_mat(a.a_s, N, C, N), weight_mat_t(m, layer_tensor(m, l, QKVW), 3 * C, C),
                           raw_qkv ? a.qkv : nullptr, a.qkv_s, P(QKVB), nullptr);
         BT_STEP(kCatAttnFwd, attn_fwd_flops(B, H, T, C / H), 20.0 * N * C, launch_attention_fwd(raw_qkv ? a.qkv : nullptr, a.qkv_s, N * 3 * C, B, T, C, H, nullptr, a.o_s, a.o_s + N * C, a.lse, simt_attn,
                                      m->err_word, s));
-        BT_GEMM(kNT, N, C, C, act_mat(a.o_s, N, C, N), weight_mat(m, layer_tensor(m, l, PROJW), C, C), a.x1,
+        BT_GEMM(kNN, N, C, C, act_mat(a.o_s, N, C, N), weight_mat_t(m, layer_tensor(m, l, PROJW), C, C), a.x1,
                      P(PROJB), a.x);
         BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x1, P(LN2G), P(LN2B), N, C, nullptr, a.m_s, a.m_s + N * C, a.mean2, a.rstd2, s));
-        BT_GEMM(kNT, N, F, C, act_mat(a.m_s, N, C, N), weight_mat(m, layer_tensor(m, l, FCW), F, C), a.h,
+        BT_GEMM(kNN, N, F, C, act_mat(a.m_s, N, C, N), weight_mat_t(m, layer_tensor(m, l, FCW), F, C), a.h,
                      P(FCB), nullptr);
         BT_STEP(kCatGeluFwd, 0, 12.0 * N * F, launch_gelu_fwd(a.h, N * F, tanh_form, nullptr, a.g_s, a.g_s + N * F, s));
-        BT_GEMM(kNT, N, C, F, act_mat(a.g_s, N, F, N), weight_mat(m, layer_tensor(m, l, PRW), C, F), xout,
+        BT_GEMM(kNN, N, C, F, act_mat(a.g_s, N, F, N), weight_mat_t(m, layer_tensor(m, l, PRW), C, F), xout,
                      P(PRB), a.x1);
     }
     const Tensor& lnfg = m->tensors[m->tensors.size() - 2];
     const Tensor& lnfb = m->tensors[m->tensors.size() - 1];
     BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(m->xL, m->params + lnfg.off, m->params + lnfb.off, N, C, nullptr, m->xf_s,
                                  m->xf_s + N * C, m->meanf, m->rstdf, s));
-    BT_GEMM(kNT, N, Vp, C, act_mat(m->xf_s, N, C, N), weight_mat(m, m->tensors[0], Vp, C), m->logits, nullptr,
+    BT_GEMM(kNN, N, Vp, C, act_mat(m->xf_s, N, C, N), weight_mat_t(m, m->tensors[0], Vp, C), m->logits, nullptr,
                  nullptr);
     BT_STEP(kCatXent, 0, 12.0 * N * Vp, launch_softmax_xent(m->logits, d_targets, N, Vp, 1.0f / (float)N, m->losses, m->loss, nullptr,
                                 m->dlogits_s, m->dlogits_s + N * Vp, s));
@@ -564,6 +595,7 @@ extern "C" bt_status bt_backward(bt_model* m) {
     if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
     if (!m->have_forward) return fail(BT_ERR_INVALID_ARG, "bt_backward without a preceding bt_forward");
     cudaStream_t s = m->stream;
+    constexpr bool gemm_is_fwd = false;  // timing category of this function's GEMMs
     const int B = m->curB, C = m->C, F = m->F, T = m->T, H = m->H, Vp = m->Vp;
     const int64_t N = (int64_t)B * T;
     const bool simt_attn = (m->cfg.flags & BT_FLAG_ATTN_SIMT) != 0;

@@ -79,6 +79,19 @@ struct SplitMat {
 
 enum GemmLayout { kNT = 0, kNN = 1, kTN = 2 };
 
+// One weight matrix of the parameter arena ([rows, cols] row-major at float offset `off`) and the
+// index of its first 64x64 tile in the concatenated tile list of all matrices.
+struct MatDesc {
+    long long off;
+    int rows, cols;
+    int tile0, tiles_c;
+};
+constexpr int kMaxSplitMats = 256;
+// For every listed matrix: TF32 hi/lo planes in place (w_hi + off, lo at + plane) AND the hi/lo
+// planes of its transpose ([cols, rows] row-major at wt_hi + off), in one pass over the weights.
+cudaError_t launch_split_matrices(const float* params, float* w_hi, float* wt_hi, int64_t plane,
+                                  const MatDesc* descs_dev, int nmats, int ntiles, cudaStream_t s);
+
 struct AdamParams {
     float lr, beta1, beta2, eps, weight_decay;
     float inv_c1, inv_c2;  // 1 / (1 - beta^t), computed on the host in double

@@ -45,6 +45,65 @@ cudaError_t launch_split(const float* x, float* hi, float* lo, int64_t n, cudaSt
     return cudaGetLastError();
 }
 
+// Weight matrices -> split planes in both orientations.  A CTA takes 64x64 tiles: the tile is read
+// once with 128-bit loads, its hi/lo planes are written in place, the values pass through shared
+// memory and the transposed tile's hi/lo planes are written with 128-bit stores too.  The forward
+// GEMMs read the transposed copy (so that the weight is the tensor core's "N-contiguous" operand,
+// whose TMA boxes are 128-byte rows), the backward GEMMs the original orientation.
+__global__ void __launch_bounds__(256) split_matrices_kernel(const float* __restrict__ params, float* __restrict__ w_hi,
+                                                             float* __restrict__ wt_hi, int64_t plane,
+                                                             const MatDesc* __restrict__ descs, int nmats,
+                                                             int ntiles) {
+    __shared__ MatDesc sd[kMaxSplitMats];
+    __shared__ float tile[64][65];
+    for (int i = threadIdx.x; i < nmats; i += blockDim.x) sd[i] = descs[i];
+    __syncthreads();
+    for (int t = blockIdx.x; t < ntiles; t += gridDim.x) {
+        int mi = 0;
+        while (mi + 1 < nmats && sd[mi + 1].tile0 <= t) ++mi;   // few matrices: a linear scan
+        const MatDesc d = sd[mi];
+        const int lt = t - d.tile0, r0 = (lt / d.tiles_c) * 64, c0 = (lt % d.tiles_c) * 64;
+        const float* src = params + d.off;
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int idx = threadIdx.x + 256 * k, r = idx >> 4, c = (idx & 15) * 4;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (r0 + r < d.rows && c0 + c < d.cols) {
+                const int64_t i4 = ((int64_t)(r0 + r) * d.cols + c0 + c) >> 2;
+                v = ld4(src, i4);
+                float4 h, l;
+                split_tf32(v, h, l);
+                reinterpret_cast<float4*>(w_hi + d.off)[i4] = h;
+                reinterpret_cast<float4*>(w_hi + plane + d.off)[i4] = l;
+            }
+            tile[r][c] = v.x; tile[r][c + 1] = v.y; tile[r][c + 2] = v.z; tile[r][c + 3] = v.w;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const int idx = threadIdx.x + 256 * k, c = idx >> 4, r = (idx & 15) * 4;
+            if (c0 + c < d.cols && r0 + r < d.rows) {
+                const float4 v = make_float4(tile[r][c], tile[r + 1][c], tile[r + 2][c], tile[r + 3][c]);
+                float4 h, l;
+                split_tf32(v, h, l);
+                const int64_t i4 = ((int64_t)(c0 + c) * d.rows + r0 + r) >> 2;
+                reinterpret_cast<float4*>(wt_hi + d.off)[i4] = h;
+                reinterpret_cast<float4*>(wt_hi + plane + d.off)[i4] = l;
+            }
+        }
+        __syncthreads();
+    }
+}
+
+cudaError_t launch_split_matrices(const float* params, float* w_hi, float* wt_hi, int64_t plane,
+                                  const MatDesc* descs_dev, int nmats, int ntiles, cudaStream_t s) {
+    if (nmats < 1 || nmats > kMaxSplitMats) return cudaErrorInvalidValue;
+    const int grid = ntiles < 148 * 8 ? ntiles : 148 * 8;
+    split_matrices_kernel<<<grid, 256, 0, s>>>(params, w_hi, wt_hi, plane, descs_dev, nmats, ntiles);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ embedding forward
 
 // One thread per float4 of the output: x[n,:] = wte[tok[n],:] + wpe[n mod T,:].
