@@ -161,6 +161,33 @@ BT_API bt_status bt_train_step(bt_model* m, const int32_t* d_tokens, const int32
 BT_API bt_status bt_train_step_host(bt_model* m, const int32_t* h_tokens, const int32_t* h_targets,
                                     int32_t B, const bt_adamw_config* opt, float* h_loss);
 
+/* Gradient accumulation (Algorithm 1: grad_accum_steps micro-steps, then one optimizer step).
+ * bt_micro_step runs bt_forward + bt_backward on micro-batch micro_index of n_micro equally
+ * sized micro-batches and folds its gradient, weighted 1/n_micro, into an accumulator inside
+ * the workspace; after the call with micro_index == n_micro - 1 the gradient tensors hold the
+ * gradient of the mean loss over all n_micro * B sequences and the loss word holds that mean
+ * (reading: the paper does not say how micro-batch losses are weighted; the mean over the global
+ * batch is the definition that makes the result independent of the split).  Call the micro-steps
+ * in order 0 .. n_micro - 1, then bt_adamw_step.  h_loss (nullable, synchronises): this
+ * micro-batch's loss, on the last micro-step the mean over all of them. */
+BT_API bt_status bt_micro_step(bt_model* m, const int32_t* d_tokens, const int32_t* d_targets, int32_t B,
+                               int32_t micro_index, int32_t n_micro, float* h_loss);
+
+/* n_micro micro-steps over d_tokens / d_targets of shape [n_micro * B, seq_len] (device),
+ * then bt_adamw_step; h_loss (nullable) receives the mean loss. */
+BT_API bt_status bt_train_step_accum(bt_model* m, const int32_t* d_tokens, const int32_t* d_targets, int32_t B,
+                                     int32_t n_micro, const bt_adamw_config* opt, float* h_loss);
+
+/* Learning rate of optimizer step `step` (1-based) from the hyper-parameter table's max / min
+ * learning rate, warmup steps and training steps.  Reading (the paper gives the four numbers, not
+ * the curve): linear warmup max_lr * step / warmup_steps, then a half cosine from max_lr at
+ * step = warmup_steps to min_lr at step = max_steps, min_lr afterwards.  Host arithmetic only. */
+typedef struct {
+    float max_lr, min_lr;
+    int32_t warmup_steps, max_steps;
+} bt_lr_schedule;
+BT_API float bt_lr_at(const bt_lr_schedule* s, int64_t step);
+
 /* Synchronises and reads the loss of the last forward. */
 BT_API bt_status bt_get_loss(bt_model* m, float* h_loss);
 

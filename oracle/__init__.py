@@ -11,6 +11,7 @@ closed forms, invariants and library routines -- none is "parity unpinned".
 from __future__ import annotations
 
 import ctypes
+import math
 import hashlib
 import os
 import subprocess
@@ -249,6 +250,22 @@ def adamw(p, g, m, v, lr, beta1, beta2, eps, weight_decay, decay, t, scale=1.0):
 
 
 # ------------------------------------------------------------------------- model
+
+def lr_schedule(step: int, max_lr: float, min_lr: float, warmup_steps: int, max_steps: int) -> float:
+    """Learning rate of optimizer step `step` (first step = 1), from the four numbers of the
+    hyper-parameter table (max / min learning rate, warmup steps, training steps).  The paper gives
+    no curve; the reading taken: a straight line from 0 to max_lr over the warmup steps, then half
+    a cosine period from max_lr (at step = warmup_steps) down to min_lr (at step = max_steps),
+    min_lr from there on."""
+    if step < 1:
+        return 0.0
+    if warmup_steps > 0 and step <= warmup_steps:
+        return max_lr * step / warmup_steps
+    if step >= max_steps or max_steps <= warmup_steps:
+        return min_lr
+    progress = (step - warmup_steps) / (max_steps - warmup_steps)
+    return min_lr + 0.5 * (1.0 + math.cos(math.pi * progress)) * (max_lr - min_lr)
+
 
 class Model:
     """The whole training step in float64."""

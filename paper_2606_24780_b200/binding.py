@@ -35,6 +35,11 @@ class bt_adamw_config(ctypes.Structure):
     _fields_ = [(n, ctypes.c_float) for n in ("lr", "beta1", "beta2", "eps", "weight_decay", "grad_clip")]
 
 
+class bt_lr_schedule(ctypes.Structure):
+    _fields_ = [("max_lr", ctypes.c_float), ("min_lr", ctypes.c_float), ("warmup_steps", ctypes.c_int32),
+                ("max_steps", ctypes.c_int32)]
+
+
 _vp, _i32, _i64, _u32, _sz, _f = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int64, ctypes.c_uint32, ctypes.c_size_t,
                                   ctypes.c_float)
 _SIGNATURES = {
@@ -53,6 +58,9 @@ _SIGNATURES = {
     "bt_adamw_step": (_i32, [_vp, ctypes.POINTER(bt_adamw_config), ctypes.POINTER(_f)]),
     "bt_train_step": (_i32, [_vp, _vp, _vp, _i32, ctypes.POINTER(bt_adamw_config), ctypes.POINTER(_f)]),
     "bt_train_step_host": (_i32, [_vp, _vp, _vp, _i32, ctypes.POINTER(bt_adamw_config), ctypes.POINTER(_f)]),
+    "bt_micro_step": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, ctypes.POINTER(_f)]),
+    "bt_train_step_accum": (_i32, [_vp, _vp, _vp, _i32, _i32, ctypes.POINTER(bt_adamw_config), ctypes.POINTER(_f)]),
+    "bt_lr_at": (_f, [ctypes.POINTER(bt_lr_schedule), _i64]),
     "bt_get_loss": (_i32, [_vp, ctypes.POINTER(_f)]),
     "bt_launch_count": (_i64, [_vp]),
     "bt_last_error": (ctypes.c_char_p, []),
@@ -223,6 +231,25 @@ def bt_train_step_host(model, h_tokens, h_targets, B, opt, want_loss=True):
     _check(lib().bt_train_step_host(model, _ptr(h_tokens), _ptr(h_targets), B, ctypes.byref(opt),
                                     ctypes.byref(loss) if want_loss else None))
     return float(loss.value) if want_loss else None
+
+
+def bt_micro_step(model, tokens, targets, B, micro_index, n_micro, want_loss=True):
+    loss = _f()
+    _check(lib().bt_micro_step(model, _ptr(tokens), _ptr(targets), B, micro_index, n_micro,
+                               ctypes.byref(loss) if want_loss else None))
+    return float(loss.value) if want_loss else None
+
+
+def bt_train_step_accum(model, tokens, targets, B, n_micro, opt, want_loss=True):
+    """tokens / targets: device int32 [n_micro * B, seq_len]."""
+    loss = _f()
+    _check(lib().bt_train_step_accum(model, _ptr(tokens), _ptr(targets), B, n_micro, ctypes.byref(opt),
+                                     ctypes.byref(loss) if want_loss else None))
+    return float(loss.value) if want_loss else None
+
+
+def bt_lr_at(schedule, step):
+    return float(lib().bt_lr_at(ctypes.byref(schedule), step))
 
 
 def bt_get_loss(model):
@@ -437,6 +464,12 @@ class Model:
 
     def train_step(self, tokens, targets, opt, want_loss=True):
         return bt_train_step(self.h, tokens, targets, tokens.shape[0], opt, want_loss)
+
+    def micro_step(self, tokens, targets, micro_index, n_micro, want_loss=True):
+        return bt_micro_step(self.h, tokens, targets, tokens.shape[0], micro_index, n_micro, want_loss)
+
+    def train_step_accum(self, tokens, targets, n_micro, opt, want_loss=True):
+        return bt_train_step_accum(self.h, tokens, targets, tokens.shape[0] // n_micro, n_micro, opt, want_loss)
 
     def train_step_host(self, h_tokens, h_targets, opt, want_loss=True):
         return bt_train_step_host(self.h, h_tokens, h_targets, h_tokens.shape[0], opt, want_loss)

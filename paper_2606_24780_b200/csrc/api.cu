@@ -105,7 +105,7 @@ struct bt_model {
     int L, C, H, T, V, Vp, F, maxB;
     std::vector<Tensor> tensors;
     int64_t P;  // padded parameter count (multiple of 1024)
-    float *params, *grads, *mom1, *mom2, *wsplit, *wsplit_t;
+    float *params, *grads, *mom1, *mom2, *wsplit, *wsplit_t, *gacc, *loss_acc;
     MatDesc* mat_descs;   // device table of the weight matrices (for the split in both orientations)
     int n_mats, n_mat_tiles;
     uint8_t* decay_flags;
@@ -189,6 +189,8 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->mom2 = b.take<float>(P);
     m->wsplit = b.take<float>(2 * P);
     m->wsplit_t = b.take<float>(2 * P);
+    m->gacc = b.take<float>(P);      // gradient accumulator of the micro-step loop
+    m->loss_acc = b.take<float>(4);
     m->mat_descs = b.take<MatDesc>(kMaxSplitMats);
     m->decay_flags = b.take<uint8_t>(P / 1024);
     m->act.resize(m->L);
@@ -689,6 +691,47 @@ extern "C" bt_status bt_train_step(bt_model* m, const int32_t* d_tokens, const i
     if (st != BT_OK) return st;
     if (h_loss) return bt_get_loss(m, h_loss);
     return BT_OK;
+}
+
+extern "C" bt_status bt_micro_step(bt_model* m, const int32_t* d_tokens, const int32_t* d_targets, int32_t B,
+                                   int32_t micro_index, int32_t n_micro, float* h_loss) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    if (n_micro < 1 || micro_index < 0 || micro_index >= n_micro)
+        return fail(BT_ERR_INVALID_ARG, "micro step %d of %d", micro_index, n_micro);
+    bt_status st = bt_forward(m, d_tokens, d_targets, B, nullptr);
+    if (st != BT_OK) return st;
+    st = bt_backward(m);
+    if (st != BT_OK) return st;
+    if (n_micro > 1) {
+        const int mode = micro_index == 0 ? 0 : micro_index == n_micro - 1 ? 2 : 1;
+        BT_CUDA(launch_grad_accumulate(m->gacc, m->grads, m->P, 1.0f / (float)n_micro, mode, m->loss_acc, m->loss,
+                                       m->stream));
+    }
+    if (h_loss) return bt_get_loss(m, h_loss);
+    return BT_OK;
+}
+
+extern "C" bt_status bt_train_step_accum(bt_model* m, const int32_t* d_tokens, const int32_t* d_targets, int32_t B,
+                                         int32_t n_micro, const bt_adamw_config* opt, float* h_loss) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    if (n_micro < 1) return fail(BT_ERR_INVALID_ARG, "n_micro < 1");
+    for (int32_t i = 0; i < n_micro; ++i) {
+        const int64_t off = (int64_t)i * B * m->T;
+        bt_status st = bt_micro_step(m, d_tokens + off, d_targets + off, B, i, n_micro, nullptr);
+        if (st != BT_OK) return st;
+    }
+    bt_status st = bt_adamw_step(m, opt, nullptr);
+    if (st != BT_OK) return st;
+    if (h_loss) return bt_get_loss(m, h_loss);
+    return BT_OK;
+}
+
+extern "C" float bt_lr_at(const bt_lr_schedule* s, int64_t step) {
+    if (!s || step < 1) return 0.0f;
+    if (s->warmup_steps > 0 && step <= s->warmup_steps) return s->max_lr * (float)((double)step / (double)s->warmup_steps);
+    if (step >= s->max_steps || s->max_steps <= s->warmup_steps) return s->min_lr;
+    const double frac = (double)(step - s->warmup_steps) / (double)(s->max_steps - s->warmup_steps);
+    return (float)((double)s->min_lr + 0.5 * (1.0 + std::cos(3.14159265358979323846 * frac)) * ((double)s->max_lr - (double)s->min_lr));
 }
 
 extern "C" bt_status bt_train_step_host(bt_model* m, const int32_t* h_tokens, const int32_t* h_targets, int32_t B,

@@ -127,6 +127,9 @@ size_t colsum_scratch_floats(int64_t N, int C);
 // x_lo (nullable): second plane added to the first (sums a split array).
 cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, float* out, float* scratch,
                           cudaStream_t s);
+// Gradient accumulation over micro-steps (see the kernel): n % 4 == 0.
+cudaError_t launch_grad_accumulate(float* acc, float* g, int64_t n, float w, int mode, float* loss_acc, float* loss,
+                                   cudaStream_t s);
 size_t grad_norm_scratch_bytes(int64_t n);
 cudaError_t launch_grad_norm(const float* g, int64_t n, float clip, float* out2, void* scratch, cudaStream_t s);
 // Flat-arena AdamW: n floats (multiple of 1024), decay_flags[n / 1024].

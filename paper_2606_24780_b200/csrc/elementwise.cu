@@ -600,6 +600,39 @@ cudaError_t launch_adamw_multi(const AdamTensorList& tl, AdamParams hp, const fl
 }
 int adamw_chunk_elems() { return kAdamChunk; }
 
+// ------------------------------------------------------------------ gradient accumulation
+
+// Micro-step i of n with weight w = 1/n: mode 0 (first) acc = w g; mode 1 acc += w g; mode 2 (last)
+// g = acc + w g, so that after the last micro-step the gradient arena holds the gradient of the
+// mean loss over all micro-batches.  The scalar loss is averaged the same way.
+__global__ void __launch_bounds__(256) grad_accumulate_kernel(float* __restrict__ acc, float* __restrict__ g, int64_t n4,
+                                                              float w, int mode, float* loss_acc, float* loss) {
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        const float l = w * loss[0];
+        if (mode == 0) loss_acc[0] = l;
+        else if (mode == 1) loss_acc[0] += l;
+        else loss[0] = loss_acc[0] + l;
+    }
+    for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
+        float4 v = ld4(g, i);
+        v = make_float4(w * v.x, w * v.y, w * v.z, w * v.w);
+        if (mode == 0) {
+            reinterpret_cast<float4*>(acc)[i] = v;
+        } else {
+            const float4 a = ld4(acc, i);
+            v = add4(a, v);
+            if (mode == 1) reinterpret_cast<float4*>(acc)[i] = v;
+            else reinterpret_cast<float4*>(g)[i] = v;
+        }
+    }
+}
+cudaError_t launch_grad_accumulate(float* acc, float* g, int64_t n, float w, int mode, float* loss_acc, float* loss,
+                                   cudaStream_t s) {
+    grad_accumulate_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(acc, g, n / 4, w, mode, loss_acc, loss);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
 // ------------------------------------------------------------------ split-K reduction
 
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partials, int splits,

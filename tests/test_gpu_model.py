@@ -237,3 +237,68 @@ def test_model_init_distribution():
     assert np.all(host(gm.tensor("h0.ln1.g")) == 1.0) and not host(gm.tensor("h0.attn.qkv.b")).any()
     assert not host(gm.tensor("wte", 2)).any()
     gm.close()
+
+
+def test_gradient_accumulation_matches_one_large_batch():
+    """Algorithm 1's micro-step loop: n_micro micro-batches of B sequences accumulate to the gradient
+    of the mean loss over all n_micro * B sequences, which the oracle computes as one batch.  Both
+    the explicit bt_micro_step calls and bt_train_step_accum are checked, then the optimizer step."""
+    cfg = si.make_config(n_layers=2, d_model=64, n_heads=1, seq_len=96, vocab_size=300, padded_vocab_size=320,
+                         batch=2, tokens="zipf")          # head_dim 64: the tcgen05 attention path
+    B, n_micro = 2, 3
+    gm, om = make_pair(cfg, 5, 0, B)
+    tok, tgt = si.tokens_for(cfg, 77, B * n_micro)
+    dtok, dtgt = dev(tok), dev(tgt)
+    micro_losses = []
+    for i in range(n_micro):
+        sl = slice(i * B, (i + 1) * B)
+        micro_losses.append(gm.micro_step(dtok[sl], dtgt[sl], i, n_micro))
+    ref_loss = om.loss_and_grad(tok, tgt, chunk=B)
+    assert abs(micro_losses[-1] - ref_loss) < TOL_LOSS * ref_loss                    # last call: the mean
+    ref_micro0 = oracle.Model(cfg)
+    ref_micro0.set_params(si.init_params(cfg, 5, jitter=0.02))
+    assert abs(micro_losses[0] - ref_micro0.loss(tok[:B], tgt[:B])) < TOL_LOSS * ref_loss
+    worst = compare_gradients(gm, om, cfg)
+    print(f"accumulated gradient: worst relative L2 error {worst:.2e}")
+    adamw_step_and_compare(gm, om, 0)
+    # the one-call form, from the state both sides now share
+    tok2, tgt2 = si.tokens_for(cfg, 78, B * n_micro)
+    opt = b.make_adamw(**si.ADAMW)
+    p_before = {n: host(gm.tensor(n)) for n in om.names()}
+    loss2 = gm.train_step_accum(dev(tok2), dev(tgt2), n_micro, opt)
+    ref2 = om.loss_and_grad(tok2, tgt2, chunk=B)
+    assert abs(loss2 - ref2) < TOL_LOSS * ref2
+    compare_gradients(gm, om, cfg)
+    assert b.bt_get_step(gm.h) == 2
+    assert any(np.abs(host(gm.tensor(n)) - p_before[n]).max() > 0 for n in om.names())
+    gm.close()
+
+
+def test_training_trajectory_with_schedule_and_accumulation():
+    """100 optimizer steps of a small model on Zipf tokens, two micro-batches per step, learning rate
+    from the warmup + cosine schedule: the GPU and the oracle run independently from the same start
+    (no re-synchronisation) and must report the same falling loss curve."""
+    cfg = si.make_config(n_layers=2, d_model=64, n_heads=4, seq_len=64, vocab_size=512, padded_vocab_size=512,
+                         batch=4, tokens="zipf")
+    B, n_micro, steps = 4, 2, 100
+    gm, om = make_pair(cfg, 9, 0, B, jitter=0.0)
+    hp = dict(si.ADAMW)
+    sched = b.bt_lr_schedule(6e-3, 6e-4, 10, steps)       # a short schedule with a larger peak, same shape
+    gpu_curve, ref_curve = [], []
+    for step in range(1, steps + 1):
+        tok, tgt = si.tokens_for(cfg, 5000 + step, B * n_micro)
+        lr = b.bt_lr_at(sched, step)
+        assert abs(lr - oracle.lr_schedule(step, np.float32(6e-3), np.float32(6e-4), 10, steps)) < 1e-9
+        hp["lr"] = lr
+        gpu_curve.append(gm.train_step_accum(dev(tok), dev(tgt), n_micro, b.make_adamw(**hp)))
+        ref_curve.append(om.loss_and_grad(tok, tgt, chunk=B))
+        om.adamw_step(lr, hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], hp["grad_clip"])
+    gpu_curve, ref_curve = np.array(gpu_curve), np.array(ref_curve)
+    print("loss: start %.4f, step 50 %.4f, end %.4f (oracle %.4f)" % (gpu_curve[0], gpu_curve[49], gpu_curve[-1],
+                                                                   ref_curve[-1]))
+    print("largest loss difference along the trajectory: %.2e relative" % (np.abs(gpu_curve - ref_curve).max() /
+                                                                            ref_curve.max()))
+    assert np.abs(gpu_curve - ref_curve).max() < 5e-4 * ref_curve.max()   # measured 2e-5 on a B200; both sides run free
+    assert np.abs(gpu_curve[:10] - ref_curve[:10]).max() < TOL_LOSS * ref_curve.max()
+    assert gpu_curve[-10:].mean() < gpu_curve[0] - 0.5          # it learns the token frequencies
+    gm.close()

@@ -4,6 +4,7 @@ import ctypes
 import os
 import re
 
+import numpy as np
 import pytest
 
 from paper_2606_24780_b200 import binding as b
@@ -75,3 +76,14 @@ def test_null_and_misaligned_arguments_are_rejected(lib):
     assert e.value.status == 1
     assert b.bt_op_gemm_scratch_bytes(0, 128, 128, 128) > 0
     assert b.bt_op_layernorm_bwd_scratch_bytes(1000, 768) > 0
+
+
+def test_lr_schedule_matches_oracle():
+    """bt_lr_at is host arithmetic: compared with the oracle's schedule on the paper's four numbers
+    (max 6e-4, min 6e-5, warmup 715, 19,073 steps) and on degenerate schedules."""
+    import oracle
+    for mx, mn, wu, ms in [(6e-4, 6e-5, 715, 19073), (1e-3, 1e-4, 10, 100), (3e-4, 3e-4, 0, 50), (1e-3, 0.0, 5, 5)]:
+        sched = b.bt_lr_schedule(mx, mn, wu, ms)
+        for step in list(range(0, 25)) + [wu - 1, wu, wu + 1, (wu + ms) // 2, ms - 1, ms, ms + 1, 10 * ms + 3]:
+            want = oracle.lr_schedule(step, np.float32(mx), np.float32(mn), wu, ms)
+            assert abs(b.bt_lr_at(sched, step) - want) <= 1e-6 * mx, (mx, mn, wu, ms, step)

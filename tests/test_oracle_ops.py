@@ -330,3 +330,27 @@ def test_clip_matches_torch_clip_grad_norm():
             assert s == 1.0
         else:
             np.testing.assert_allclose(s * gn, gn / (gn + 1e-6), rtol=1e-13)
+
+
+def test_lr_schedule_pins():
+    """Learning-rate schedule against what the hyper-parameter table fixes (Table of GPT-2 124M
+    hyper-parameters: max 6e-4, min 6e-5, 715 warmup steps, 19,073 training steps) and the shape
+    of the reading: end points, the linear ramp, the cosine's midpoint and symmetry, monotonicity."""
+    mx, mn, wu, ms = 6e-4, 6e-5, 715, 19073
+    f = lambda t: oracle.lr_schedule(t, mx, mn, wu, ms)
+    assert f(0) == 0.0
+    assert f(wu) == mx and f(ms) == mn and f(ms + 1000) == mn
+    assert abs(f(1) - mx / wu) < 1e-18 and abs(f(wu // 5) - mx * (wu // 5) / wu) < 1e-18
+    mid = (wu + ms) // 2          # (715 + 19073) / 2 = 9894 exactly: cos(pi/2) = 0
+    assert (wu + ms) % 2 == 0 and abs(f(mid) - 0.5 * (mx + mn)) < 1e-15
+    for k in (1, 100, 5000):       # cos(pi - x) = -cos(x): the curve is point-symmetric about the midpoint
+        assert abs((f(mid - k) - 0.5 * (mx + mn)) + (f(mid + k) - 0.5 * (mx + mn))) < 1e-15
+    ramp = [f(t) for t in range(1, wu + 1)]
+    decay = [f(t) for t in range(wu, ms + 1)]
+    assert all(a < b for a, b in zip(ramp, ramp[1:]))
+    assert all(a > b for a, b in zip(decay, decay[1:]))
+    # a quarter of the way down the cosine: (1 + cos(pi/4)) / 2 of the range above min
+    q = wu + (ms - wu) // 4
+    assert (ms - wu) % 4 != 0 or abs(f(q) - (mn + 0.5 * (1 + 2 ** -0.5) * (mx - mn))) < 1e-15
+    # no warmup, no decay
+    assert oracle.lr_schedule(1, 1e-3, 1e-3, 0, 10) == 1e-3
