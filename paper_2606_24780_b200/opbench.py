@@ -53,7 +53,13 @@ def build_cases(B, T, C, H, Vp, n_params):
         cases[name] = dict(run=run, flops=2.0 * M * Nn * K, bytes=8.0 * (M * K + Nn * K) + 4.0 * M * Nn,
                            bound="tensor", keep=(A, Bm, D, bi, res), check=lambda: b.bt_op_gemm_check(gscratch))
 
-    # forward GEMMs of the block, the two backward layouts of each, and the LM head
+    # forward GEMMs of the block as the training step runs them (weight read from its transposed
+    # copy: layout NN, bias / residual in the epilogue), the same products in the NT layout, the two
+    # backward layouts of each, and the LM head
+    gemm_case("gemm_fwd_qkv", 1, N, 3 * C, C, bias=True)
+    gemm_case("gemm_fwd_attnproj", 1, N, C, C, bias=True, residual=True)
+    gemm_case("gemm_fwd_fc", 1, N, F, C, bias=True)
+    gemm_case("gemm_fwd_mlpproj", 1, N, C, F, bias=True, residual=True)
     gemm_case("gemm_nt_qkv", 0, N, 3 * C, C, bias=True)
     gemm_case("gemm_nt_attnproj", 0, N, C, C, bias=True, residual=True)
     gemm_case("gemm_nt_fc", 0, N, F, C, bias=True)
@@ -67,6 +73,7 @@ def build_cases(B, T, C, H, Vp, n_params):
     gemm_case("gemm_tn_wfc", 2, F, C, N)
     gemm_case("gemm_tn_wmlpproj", 2, C, F, N)
     if Vp:
+        gemm_case("gemm_fwd_lmhead", 1, N, Vp, C)
         gemm_case("gemm_nt_lmhead", 0, N, Vp, C)
         gemm_case("gemm_nn_dlmhead", 1, N, C, Vp)
         gemm_case("gemm_tn_wlmhead", 2, Vp, C, N)
@@ -194,7 +201,7 @@ def main(argv=None):
     args = ap.parse_args(argv)
     torch.cuda.set_device(0)
     only = [s for s in args.only.split(",") if s]
-    need_big = not only or any(s.startswith(("gemm_nt_lm", "gemm_nn_dlm", "gemm_tn_wlm", "softmax", "adamw", "grad"))
+    need_big = not only or any(s.startswith(("gemm_fwd_lm", "gemm_nt_lm", "gemm_nn_dlm", "gemm_tn_wlm", "softmax", "adamw", "grad"))
                                for s in only)
     cases = build_cases(args.batch, args.seq, args.d_model, args.heads, args.vocab if need_big else 0,
                         args.params if need_big else 0)
