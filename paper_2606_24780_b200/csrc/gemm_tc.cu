@@ -44,6 +44,10 @@ constexpr int BM = 128;
 constexpr int kThreads = 192;
 constexpr int kEpiWarps = 4;
 constexpr uint32_t kSmemBudget = 227u * 1024u;
+// Epilogue staging: each epilogue warp owns a 32 x 32 float tile with a 144-byte row pitch (both the
+// row-wise 128-bit writes and the transposed 128-bit reads are then bank-conflict free).
+constexpr uint32_t kEpiPitch = 144u;
+constexpr uint32_t kEpiStageBytes = kEpiWarps * 32u * kEpiPitch;
 
 // BN: tile width (128, 192 or 256).  BK: floats per k-block; 32 = one 128-byte swizzle row,
 // 16 = one 64-byte swizzle row (smaller stages, deeper ring).
@@ -52,11 +56,11 @@ struct Cfg {
     static constexpr uint32_t kATileBytes = 2u * BM * BK * 4u;  // hi + lo
     static constexpr uint32_t kBTileBytes = 2u * BN * BK * 4u;
     static constexpr uint32_t kStageBytes = kATileBytes + kBTileBytes;
-    static constexpr int kStagesFit = (int)((kSmemBudget - 2048u) / kStageBytes);
+    static constexpr int kStagesFit = (int)((kSmemBudget - 2048u - kEpiStageBytes) / kStageBytes);
     static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
     static constexpr uint32_t kAccStride = (BN <= 128) ? 128u : 256u;  // TMEM columns per accumulator
     static constexpr uint32_t kTmemCols = 2u * kAccStride;             // 256 or 512 (power of two)
-    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + 256;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + kEpiStageBytes + 256;
 };
 
 struct GemmArgs {
@@ -97,7 +101,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     constexpr uint32_t kMnAtomBytes = 2u * BK * 128u;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bars = smem_base + C::kStages * C::kStageBytes;  // 8-byte barriers
+    const uint32_t epi_stage = smem_base + C::kStages * C::kStageBytes;
+    const uint32_t bars = epi_stage + kEpiStageBytes;  // 8-byte barriers
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (C::kStages + s); };
     auto tfull_bar = [&](int a) { return bars + 8u * (2 * C::kStages + a); };
@@ -217,7 +222,6 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             const uint32_t aph = (ut >> 1) & 1u;
             if (!mbar_wait_warp(tfull_bar(acc), aph, g.err, 4)) { ok = false; break; }
             tc_fence_after();
-            const int row = tm * BM + lane_group * 32 + lane;
             float* Dp = g.D;
             long long ldd = g.ldd;
             if (g.splits > 1) {
@@ -225,6 +229,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 ldd = g.N;
             }
             const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)acc * C::kAccStride;
+            // A thread reads its accumulator row from tensor memory; the warp's 32 x 32 chunk goes
+            // through shared memory so that global memory is then touched a full 128-byte row
+            // segment at a time (8 lanes x 16 B): lane -> rows sub + 4i, columns 4*cq .. 4*cq+3.
+            float* my_stage = reinterpret_cast<float*>(smem_raw + (epi_stage - smem_u32(smem_raw)) +
+                                                       (uint32_t)(warp - 2) * 32u * kEpiPitch);
+            const int sub = lane >> 3, cq = lane & 7;
+            const int row0 = tm * BM + lane_group * 32;
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 const int col0 = tn * BN + c * 32;
@@ -232,27 +243,47 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                 uint32_t rr[32];
                 tmem_ld32(t_row + c * 32, rr);
                 tmem_ld_wait();
-                if (row < g.M) {
-                    float* drow = Dp + (long long)row * ldd + col0;
-                    const float* rrow = g.residual ? g.residual + (long long)row * g.ldd + col0 : nullptr;
+                float4* wr = reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(my_stage) + lane * kEpiPitch);
 #pragma unroll
-                    for (int q = 0; q < 8; ++q) {
-                        if (col0 + q * 4 < g.N) {
-                            float4 v = make_float4(__uint_as_float(rr[4 * q]), __uint_as_float(rr[4 * q + 1]),
-                                                   __uint_as_float(rr[4 * q + 2]), __uint_as_float(rr[4 * q + 3]));
-                            if (g.bias) v = add4(v, *reinterpret_cast<const float4*>(g.bias + col0 + q * 4));
-                            if (rrow) v = add4(v, *reinterpret_cast<const float4*>(rrow + q * 4));
-                            if (Dp) *reinterpret_cast<float4*>(drow + q * 4) = v;
+                for (int q = 0; q < 8; ++q)
+                    wr[q] = make_float4(__uint_as_float(rr[4 * q]), __uint_as_float(rr[4 * q + 1]),
+                                        __uint_as_float(rr[4 * q + 2]), __uint_as_float(rr[4 * q + 3]));
+                __syncwarp();
+                const int col = col0 + 4 * cq;
+                if (col < g.N) {
+                    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (g.bias) bv = *reinterpret_cast<const float4*>(g.bias + col);
+                    // all residual rows of the chunk are requested before the first store (the output
+                    // may alias the residual, so the compiler cannot hoist these loads itself)
+                    float4 rv[8];
+                    if (g.residual) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int row = row0 + sub + 4 * i;
+                            rv[i] = (row < g.M) ? *reinterpret_cast<const float4*>(g.residual + (long long)row * g.ldd + col)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int r = sub + 4 * i, row = row0 + r;
+                        if (row < g.M) {
+                            float4 v = *reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(my_stage) +
+                                                                        r * kEpiPitch + cq * 16);
+                            v = add4(v, bv);
+                            if (g.residual) v = add4(v, rv[i]);
+                            if (Dp) *reinterpret_cast<float4*>(Dp + (long long)row * ldd + col) = v;
                             if (g.d_hi) {
                                 float4 hh, ll;
                                 split_tf32(v, hh, ll);
-                                float* hrow = g.d_hi + (long long)row * g.ldd + col0 + q * 4;
+                                float* hrow = g.d_hi + (long long)row * g.ldd + col;
                                 *reinterpret_cast<float4*>(hrow) = hh;
                                 *reinterpret_cast<float4*>(hrow + g.d_plane) = ll;
                             }
                         }
                     }
                 }
+                __syncwarp();   // the staging tile is rewritten by the next chunk
             }
             tc_fence_before();
             __syncwarp();
