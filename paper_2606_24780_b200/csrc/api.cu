@@ -129,6 +129,14 @@ struct bt_model {
     size_t prof_used;
 };
 
+bool bt::pdl_enabled() {
+    static const bool on = []() {
+        const char* v = getenv("BT_PDL");
+        return !(v && v[0] == '0');
+    }();
+    return on;
+}
+
 namespace {
 
 void build_registry(const bt_config& c, std::vector<Tensor>& out, int64_t& P) {

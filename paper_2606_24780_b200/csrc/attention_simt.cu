@@ -29,6 +29,8 @@ template <int DPL>
 __global__ void __launch_bounds__(kAsWarps * 32) attn_fwd_simt_kernel(const float* __restrict__ qkv, int B, int T,
                                                                        int C, int H, float* o, float* o_hi,
                                                                        float* o_lo, float* __restrict__ lse) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     const int64_t gw = (int64_t)blockIdx.x * kAsWarps + (threadIdx.x >> 5);
     if (gw >= (int64_t)B * H * T) return;
@@ -79,6 +81,8 @@ __global__ void __launch_bounds__(kAsWarps * 32) attn_dvec_kernel(const float* _
                                                                    const float* __restrict__ d_o,
                                                                    const float* __restrict__ d_o_lo, int B, int T,
                                                                    int C, int H, float* __restrict__ dvec) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     const int64_t gw = (int64_t)blockIdx.x * kAsWarps + (threadIdx.x >> 5);
     if (gw >= (int64_t)B * H * T) return;
@@ -127,6 +131,8 @@ template <int DPL>
 __global__ void __launch_bounds__(kAsWarps * 32) attn_bwd_dq_simt_kernel(
     const float* __restrict__ qkv, const float* __restrict__ lse, const float* __restrict__ d_o,
     const float* __restrict__ dvec, int B, int T, int C, int H, float* dqkv, float* dqkv_hi, float* dqkv_lo) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     const int64_t gw = (int64_t)blockIdx.x * kAsWarps + (threadIdx.x >> 5);
     if (gw >= (int64_t)B * H * T) return;
@@ -156,6 +162,8 @@ template <int DPL>
 __global__ void __launch_bounds__(kAsWarps * 32) attn_bwd_dkv_simt_kernel(
     const float* __restrict__ qkv, const float* __restrict__ lse, const float* __restrict__ d_o,
     const float* __restrict__ dvec, int B, int T, int C, int H, float* dqkv, float* dqkv_hi, float* dqkv_lo) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     const int64_t gw = (int64_t)blockIdx.x * kAsWarps + (threadIdx.x >> 5);
     if (gw >= (int64_t)B * H * T) return;
@@ -190,9 +198,9 @@ cudaError_t launch_attention_fwd_simt(const float* qkv, int B, int T, int C, int
     const int d = C / H;
     const int64_t warps = (int64_t)B * H * T;
     const int grid = (int)((warps + kAsWarps - 1) / kAsWarps);
-    if (d <= 32) attn_fwd_simt_kernel<1><<<grid, kAsWarps * 32, 0, s>>>(qkv, B, T, C, H, o, o_hi, o_lo, lse);
-    else if (d <= 64) attn_fwd_simt_kernel<2><<<grid, kAsWarps * 32, 0, s>>>(qkv, B, T, C, H, o, o_hi, o_lo, lse);
-    else attn_fwd_simt_kernel<4><<<grid, kAsWarps * 32, 0, s>>>(qkv, B, T, C, H, o, o_hi, o_lo, lse);
+    if (d <= 32) BT_KERNEL_LAUNCH((attn_fwd_simt_kernel<1>), grid, kAsWarps * 32, 0, s, qkv, B, T, C, H, o, o_hi, o_lo, lse);
+    else if (d <= 64) BT_KERNEL_LAUNCH((attn_fwd_simt_kernel<2>), grid, kAsWarps * 32, 0, s, qkv, B, T, C, H, o, o_hi, o_lo, lse);
+    else BT_KERNEL_LAUNCH((attn_fwd_simt_kernel<4>), grid, kAsWarps * 32, 0, s, qkv, B, T, C, H, o, o_hi, o_lo, lse);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -202,9 +210,9 @@ cudaError_t launch_attention_dvec(const float* o, const float* o_lo, const float
     const int d = C / H;
     const int64_t warps = (int64_t)B * H * T;
     const int grid = (int)((warps + kAsWarps - 1) / kAsWarps);
-    if (d <= 32) attn_dvec_kernel<1><<<grid, kAsWarps * 32, 0, s>>>(o, o_lo, d_o, d_o_lo, B, T, C, H, dvec);
-    else if (d <= 64) attn_dvec_kernel<2><<<grid, kAsWarps * 32, 0, s>>>(o, o_lo, d_o, d_o_lo, B, T, C, H, dvec);
-    else attn_dvec_kernel<4><<<grid, kAsWarps * 32, 0, s>>>(o, o_lo, d_o, d_o_lo, B, T, C, H, dvec);
+    if (d <= 32) BT_KERNEL_LAUNCH((attn_dvec_kernel<1>), grid, kAsWarps * 32, 0, s, o, o_lo, d_o, d_o_lo, B, T, C, H, dvec);
+    else if (d <= 64) BT_KERNEL_LAUNCH((attn_dvec_kernel<2>), grid, kAsWarps * 32, 0, s, o, o_lo, d_o, d_o_lo, B, T, C, H, dvec);
+    else BT_KERNEL_LAUNCH((attn_dvec_kernel<4>), grid, kAsWarps * 32, 0, s, o, o_lo, d_o, d_o_lo, B, T, C, H, dvec);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -218,9 +226,9 @@ cudaError_t launch_attention_bwd_simt(const float* qkv, const float* o, const fl
     const int64_t warps = (int64_t)B * H * T;
     const int grid = (int)((warps + kAsWarps - 1) / kAsWarps);
 #define BT_AB(DPL)                                                                                                  \
-    attn_bwd_dq_simt_kernel<DPL><<<grid, kAsWarps * 32, 0, s>>>(qkv, lse, d_o, dvec, B, T, C, H, dqkv, dqkv_hi,     \
+    BT_KERNEL_LAUNCH((attn_bwd_dq_simt_kernel<DPL>), grid, kAsWarps * 32, 0, s, qkv, lse, d_o, dvec, B, T, C, H, dqkv, dqkv_hi,     \
                                                                  dqkv_lo);                                          \
-    attn_bwd_dkv_simt_kernel<DPL><<<grid, kAsWarps * 32, 0, s>>>(qkv, lse, d_o, dvec, B, T, C, H, dqkv, dqkv_hi,    \
+    BT_KERNEL_LAUNCH((attn_bwd_dkv_simt_kernel<DPL>), grid, kAsWarps * 32, 0, s, qkv, lse, d_o, dvec, B, T, C, H, dqkv, dqkv_hi,    \
                                                                   dqkv_lo)
     if (d <= 32) { BT_AB(1); } else if (d <= 64) { BT_AB(2); } else { BT_AB(4); }
 #undef BT_AB

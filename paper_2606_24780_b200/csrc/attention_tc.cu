@@ -123,6 +123,8 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
+    pdl_wait();      // set-up done; global memory is touched from here on
+    pdl_trigger();
 
     if (warp == 0) {
         // ------------------------------------------------------------ TMA producer
@@ -392,7 +394,7 @@ cudaError_t launch_attention_fwd_tc(const float* qkv_hi, int64_t qkv_plane, int 
     if (!ok) return cudaErrorInvalidValue;
     AttnArgs g{T, C, H, o, o_hi, o_lo, lse, err_word, g_trace_ptr};
     dim3 grid(B * H, (T + BQ - 1) / BQ);
-    attn_fwd_tc_kernel<<<grid, kThreads, kSmemBytes, s>>>(tmQ, tmK, tmV, g);
+    BT_KERNEL_LAUNCH((attn_fwd_tc_kernel), grid, kThreads, kSmemBytes, s, tmQ, tmK, tmV, g);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }

@@ -232,6 +232,8 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     }
 
     const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp);
+    pdl_wait();      // set-up done; global memory is touched from here on
+    pdl_trigger();
     // TMEM columns
     const uint32_t tK_hi = tmem, tK_lo = tmem + 64, tdK = tmem + 128, tdV = tmem + 192;
     auto tbuf = [&](int bb) { return tmem + 256u + 128u * (uint32_t)bb; };  // +0 S^T|P^T_hi, +32 P^T_lo, +64 dP^T|dS^T_hi, +96 dS^T_lo
@@ -468,6 +470,8 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
     }
 
     const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp);
+    pdl_wait();      // set-up done; global memory is touched from here on
+    pdl_trigger();
     const uint32_t tQ_hi = tmem, tQ_lo = tmem + 64, tdQ = tmem + 128;
     auto tbuf = [&](int bb) { return tmem + 192u + 128u * (uint32_t)bb; };   // +0 S -> dS_hi, +64 dP -> dS_lo
 
@@ -687,9 +691,9 @@ cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, cons
     BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dqkv_hi, dqkv_plane, err_word, attention_tc_get_trace(), rg_sums,
               4 * ((T + BR - 1) / BR)};
     dim3 gk(B * H, (T + BR - 1) / BR);
-    attn_bwd_dkv_tc_kernel<<<gk, kThreads, kDkvSmem, s>>>(qk32, qm32, dok32, dom32, vres, g);
+    BT_KERNEL_LAUNCH((attn_bwd_dkv_tc_kernel), gk, kThreads, kDkvSmem, s, qk32, qm32, dok32, dom32, vres, g);
     BT_COUNT_LAUNCH();
-    attn_bwd_dq_tc_kernel<<<gk, kThreads, kDqSmem, s>>>(qk64, qm64, qk64, dores, g);
+    BT_KERNEL_LAUNCH((attn_bwd_dq_tc_kernel), gk, kThreads, kDqSmem, s, qk64, qm64, qk64, dores, g);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }

@@ -77,6 +77,34 @@ struct SplitMat {
     int64_t rows, cols, ld;
 };
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// Every kernel of the step starts with pdl_wait() (returns once the kernels before it in the stream
+// have completed and their writes are visible) followed by pdl_trigger() (lets the NEXT launch be
+// scheduled), and is launched with the programmatic-stream-serialization attribute: the next
+// kernel's launch latency and block scheduling then overlap the tail of the current one instead of
+// following it.  BT_PDL=0 in the environment turns the attribute off (plain stream order).
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_trigger() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+#endif
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl_enabled() ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#define BT_KERNEL_LAUNCH(kernel, grid, block, smem, stream, ...) \
+    (void)bt::launch_k(kernel, dim3(grid), dim3(block), (size_t)(smem), stream, __VA_ARGS__)
+
 enum GemmLayout { kNT = 0, kNN = 1, kTN = 2 };
 
 // One weight matrix of the parameter arena ([rows, cols] row-major at float offset `off`) and the

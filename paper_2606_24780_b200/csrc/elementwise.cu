@@ -30,6 +30,8 @@ constexpr int kStreamGridCap = 148 * 16;
 
 __global__ void __launch_bounds__(256) split_kernel(const float* __restrict__ x, float* __restrict__ hi,
                                                     float* __restrict__ lo, int64_t n4) {
+    pdl_wait();
+    pdl_trigger();
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
         float4 v = ld4(x, i), h, l;
         split_tf32(v, h, l);
@@ -40,7 +42,7 @@ __global__ void __launch_bounds__(256) split_kernel(const float* __restrict__ x,
 
 cudaError_t launch_split(const float* x, float* hi, float* lo, int64_t n, cudaStream_t s) {
     int64_t n4 = n / 4;
-    split_kernel<<<grid_for(n4, 256, kStreamGridCap), 256, 0, s>>>(x, hi, lo, n4);
+    BT_KERNEL_LAUNCH((split_kernel), grid_for(n4, 256, kStreamGridCap), 256, 0, s, x, hi, lo, n4);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -54,6 +56,8 @@ __global__ void __launch_bounds__(256) split_matrices_kernel(const float* __rest
                                                              float* __restrict__ wt_hi, int64_t plane,
                                                              const MatDesc* __restrict__ descs, int nmats,
                                                              int ntiles) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ MatDesc sd[kMaxSplitMats];
     __shared__ float tile[64][65];
     for (int i = threadIdx.x; i < nmats; i += blockDim.x) sd[i] = descs[i];
@@ -99,7 +103,7 @@ cudaError_t launch_split_matrices(const float* params, float* w_hi, float* wt_hi
                                   const MatDesc* descs_dev, int nmats, int ntiles, cudaStream_t s) {
     if (nmats < 1 || nmats > kMaxSplitMats) return cudaErrorInvalidValue;
     const int grid = ntiles < 148 * 8 ? ntiles : 148 * 8;
-    split_matrices_kernel<<<grid, 256, 0, s>>>(params, w_hi, wt_hi, plane, descs_dev, nmats, ntiles);
+    BT_KERNEL_LAUNCH((split_matrices_kernel), grid, 256, 0, s, params, w_hi, wt_hi, plane, descs_dev, nmats, ntiles);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -111,6 +115,8 @@ __global__ void __launch_bounds__(256) embedding_fwd_kernel(const int32_t* __res
                                                             const float* __restrict__ wte,
                                                             const float* __restrict__ wpe, int64_t N, int T, int C4,
                                                             float* __restrict__ x) {
+    pdl_wait();
+    pdl_trigger();
     int64_t total = N * C4;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
@@ -129,7 +135,7 @@ __global__ void __launch_bounds__(256) embedding_fwd_kernel(const int32_t* __res
 
 cudaError_t launch_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int T, int C,
                                  float* x, cudaStream_t s) {
-    embedding_fwd_kernel<<<grid_for(N * (C / 4), 256, kStreamGridCap), 256, 0, s>>>(tok, wte, wpe, N, T, C / 4, x);
+    BT_KERNEL_LAUNCH((embedding_fwd_kernel), grid_for(N * (C / 4), 256, kStreamGridCap), 256, 0, s, tok, wte, wpe, N, T, C / 4, x);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -143,6 +149,8 @@ cudaError_t launch_embedding_fwd(const int32_t* tok, const float* wte, const flo
 __global__ void __launch_bounds__(256) embedding_bwd_wte_kernel(const int32_t* __restrict__ tok,
                                                                 const float* __restrict__ dx, int N, int C4,
                                                                 float* __restrict__ dwte) {
+    pdl_wait();
+    pdl_trigger();
     const int n = blockIdx.x;
     const int t = tok[n];
     int found = 0;
@@ -184,6 +192,8 @@ __global__ void __launch_bounds__(256) embedding_bwd_wte_kernel(const int32_t* _
 // dwpe[t,:] = sum over sequences b (ascending) of dx[b*T + t,:].
 __global__ void __launch_bounds__(256) embedding_bwd_wpe_kernel(const float* __restrict__ dx, int B, int T, int C4,
                                                                 float* __restrict__ dwpe) {
+    pdl_wait();
+    pdl_trigger();
     int64_t total = (int64_t)T * C4;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < total;
          i += (int64_t)gridDim.x * blockDim.x) {
@@ -195,9 +205,9 @@ __global__ void __launch_bounds__(256) embedding_bwd_wpe_kernel(const float* __r
 
 cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, float* dwte,
                                  float* dwpe, cudaStream_t s) {
-    embedding_bwd_wte_kernel<<<(int)N, 256, 0, s>>>(tok, dx, (int)N, C / 4, dwte);
+    BT_KERNEL_LAUNCH((embedding_bwd_wte_kernel), (int)N, 256, 0, s, tok, dx, (int)N, C / 4, dwte);
     BT_COUNT_LAUNCH();
-    embedding_bwd_wpe_kernel<<<grid_for((int64_t)T * (C / 4), 256, kStreamGridCap), 256, 0, s>>>(
+    BT_KERNEL_LAUNCH((embedding_bwd_wpe_kernel), grid_for((int64_t)T * (C / 4), 256, kStreamGridCap), 256, 0, s, 
         dx, (int)(N / T), T, C / 4, dwpe);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
@@ -225,6 +235,8 @@ __device__ __forceinline__ float gelu_grad_f(float x, bool tanh_form) {
 
 __global__ void __launch_bounds__(256) gelu_fwd_kernel(const float* __restrict__ x, int64_t n4, int tanh_form,
                                                        float* y, float* y_hi, float* y_lo) {
+    pdl_wait();
+    pdl_trigger();
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
         float4 v = ld4(x, i), r;
         r.x = gelu_f(v.x, tanh_form);
@@ -238,6 +250,8 @@ __global__ void __launch_bounds__(256) gelu_fwd_kernel(const float* __restrict__
 __global__ void __launch_bounds__(256) gelu_bwd_kernel(const float* __restrict__ x, const float* __restrict__ dy,
                                                        int64_t n4, int tanh_form, float* dx, float* dx_hi,
                                                        float* dx_lo) {
+    pdl_wait();
+    pdl_trigger();
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
         float4 v = ld4(x, i), d = ld4(dy, i), r;
         r.x = d.x * gelu_grad_f(v.x, tanh_form);
@@ -250,13 +264,13 @@ __global__ void __launch_bounds__(256) gelu_bwd_kernel(const float* __restrict__
 
 cudaError_t launch_gelu_fwd(const float* x, int64_t n, int tanh_form, float* y, float* y_hi, float* y_lo,
                             cudaStream_t s) {
-    gelu_fwd_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(x, n / 4, tanh_form, y, y_hi, y_lo);
+    BT_KERNEL_LAUNCH((gelu_fwd_kernel), grid_for(n / 4, 256, kStreamGridCap), 256, 0, s, x, n / 4, tanh_form, y, y_hi, y_lo);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
 cudaError_t launch_gelu_bwd(const float* x, const float* dy, int64_t n, int tanh_form, float* dx, float* dx_hi,
                             float* dx_lo, cudaStream_t s) {
-    gelu_bwd_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(x, dy, n / 4, tanh_form, dx, dx_hi, dx_lo);
+    BT_KERNEL_LAUNCH((gelu_bwd_kernel), grid_for(n / 4, 256, kStreamGridCap), 256, 0, s, x, dy, n / 4, tanh_form, dx, dx_hi, dx_lo);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -279,6 +293,8 @@ size_t colsum_scratch_floats(int64_t N, int C) { return (size_t)colsum_strips(N,
 __global__ void __launch_bounds__(256) colsum_stage1_kernel(const float* __restrict__ x,
                                                             const float* __restrict__ x_lo, int64_t N, int C4,
                                                             int strips, float* __restrict__ partial) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x * 32 + lane;
     const int st = blockIdx.y;
@@ -319,6 +335,8 @@ __global__ void __launch_bounds__(256) colsum_stage1_kernel(const float* __restr
 // warp sums are combined in warp order: a fixed summation order.
 __global__ void __launch_bounds__(256) colsum_stage2_kernel(const float* __restrict__ partial, int strips, int C4,
                                                             float* __restrict__ out) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ float4 sm[8][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x * 32 + lane;
@@ -349,6 +367,8 @@ __global__ void __launch_bounds__(256) gelu_bwd_colsum_kernel(const float* __res
                                                               const float* __restrict__ dy, int64_t N, int C4,
                                                               int strips, int tanh_form, float* dx, float* dx_hi,
                                                               float* dx_lo, float* __restrict__ partial) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x * 32 + lane;
     const int st = blockIdx.y;
@@ -392,9 +412,9 @@ cudaError_t launch_gelu_bwd_colsum(const float* x, const float* dy, int64_t N, i
                                    float* dx_hi, float* dx_lo, float* colsum, float* scratch, cudaStream_t s) {
     int C4 = C / 4, strips = colsum_strips(N, C);
     dim3 grid((C4 + 31) / 32, strips);
-    gelu_bwd_colsum_kernel<<<grid, 256, 0, s>>>(x, dy, N, C4, strips, tanh_form, dx, dx_hi, dx_lo, scratch);
+    BT_KERNEL_LAUNCH((gelu_bwd_colsum_kernel), grid, 256, 0, s, x, dy, N, C4, strips, tanh_form, dx, dx_hi, dx_lo, scratch);
     BT_COUNT_LAUNCH();
-    colsum_stage2_kernel<<<(C4 + 31) / 32, 256, 0, s>>>(scratch, strips, C4, colsum);
+    BT_KERNEL_LAUNCH((colsum_stage2_kernel), (C4 + 31) / 32, 256, 0, s, scratch, strips, C4, colsum);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -403,9 +423,9 @@ cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, f
                           cudaStream_t s) {
     int C4 = C / 4, strips = colsum_strips(N, C);
     dim3 grid((C4 + 31) / 32, strips);
-    colsum_stage1_kernel<<<grid, 256, 0, s>>>(x, x_lo, N, C4, strips, scratch);
+    BT_KERNEL_LAUNCH((colsum_stage1_kernel), grid, 256, 0, s, x, x_lo, N, C4, strips, scratch);
     BT_COUNT_LAUNCH();
-    colsum_stage2_kernel<<<(C4 + 31) / 32, 256, 0, s>>>(scratch, strips, C4, out);
+    BT_KERNEL_LAUNCH((colsum_stage2_kernel), (C4 + 31) / 32, 256, 0, s, scratch, strips, C4, out);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -467,6 +487,8 @@ size_t grad_norm_scratch_bytes(int64_t) { return kNormBlocks * sizeof(double); }
 
 __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ g, int64_t n4, int64_t n,
                                                     double* __restrict__ partial) {
+    pdl_wait();
+    pdl_trigger();
     float acc = 0.f;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
         float4 v = ld4(g, i);
@@ -490,6 +512,8 @@ __global__ void __launch_bounds__(256) sumsq_kernel(const float* __restrict__ g,
 
 __global__ void __launch_bounds__(256) norm_finalize_kernel(const double* __restrict__ partial, int nb, float clip,
                                                             float* __restrict__ out2) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ double sm[256];
     double t = 0.0;
     for (int i = threadIdx.x; i < nb; i += 256) t += partial[i];
@@ -513,9 +537,9 @@ __global__ void __launch_bounds__(256) norm_finalize_kernel(const double* __rest
 
 cudaError_t launch_grad_norm(const float* g, int64_t n, float clip, float* out2, void* scratch, cudaStream_t s) {
     int nb = grid_for(n / 4, 256, kNormBlocks);
-    sumsq_kernel<<<nb, 256, 0, s>>>(g, n / 4, n, (double*)scratch);
+    BT_KERNEL_LAUNCH((sumsq_kernel), nb, 256, 0, s, g, n / 4, n, (double*)scratch);
     BT_COUNT_LAUNCH();
-    norm_finalize_kernel<<<1, 256, 0, s>>>((const double*)scratch, nb, clip, out2);
+    BT_KERNEL_LAUNCH((norm_finalize_kernel), 1, 256, 0, s, (const double*)scratch, nb, clip, out2);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -546,6 +570,8 @@ __global__ void __launch_bounds__(256) adamw_flat_kernel(float* __restrict__ p, 
                                                          float* __restrict__ m, float* __restrict__ v, int64_t n4,
                                                          const uint8_t* __restrict__ decay_flags, AdamParams hp,
                                                          const float* __restrict__ d_scale) {
+    pdl_wait();
+    pdl_trigger();
     const float scale = d_scale ? *d_scale : 1.0f;
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
         float4 pv = ld4(p, i), gv = ld4(g, i), mv = ld4(m, i), vv = ld4(v, i);
@@ -558,7 +584,7 @@ __global__ void __launch_bounds__(256) adamw_flat_kernel(float* __restrict__ p, 
 
 cudaError_t launch_adamw_flat(float* p, const float* g, float* m, float* v, int64_t n, const uint8_t* decay_flags,
                               AdamParams hp, const float* d_scale, cudaStream_t s) {
-    adamw_flat_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(p, g, m, v, n / 4, decay_flags, hp,
+    BT_KERNEL_LAUNCH((adamw_flat_kernel), grid_for(n / 4, 256, kStreamGridCap), 256, 0, s, p, g, m, v, n / 4, decay_flags, hp,
                                                                             d_scale);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
@@ -569,6 +595,8 @@ cudaError_t launch_adamw_flat(float* p, const float* g, float* m, float* v, int6
 constexpr int kAdamChunk = 4096;
 __global__ void __launch_bounds__(256) adamw_multi_kernel(const __grid_constant__ AdamTensorList tl, AdamParams hp,
                                                           const float* __restrict__ d_scale) {
+    pdl_wait();
+    pdl_trigger();
     const float scale = d_scale ? *d_scale : 1.0f;
     int t = 0;
     while (t + 1 < tl.n && (int)blockIdx.x >= tl.chunk_begin[t + 1]) ++t;
@@ -594,7 +622,7 @@ __global__ void __launch_bounds__(256) adamw_multi_kernel(const __grid_constant_
 cudaError_t launch_adamw_multi(const AdamTensorList& tl, AdamParams hp, const float* d_scale, cudaStream_t s) {
     int chunks = tl.chunk_begin[tl.n];
     if (chunks <= 0) return cudaSuccess;
-    adamw_multi_kernel<<<chunks, 256, 0, s>>>(tl, hp, d_scale);
+    BT_KERNEL_LAUNCH((adamw_multi_kernel), chunks, 256, 0, s, tl, hp, d_scale);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -607,6 +635,8 @@ int adamw_chunk_elems() { return kAdamChunk; }
 // mean loss over all micro-batches.  The scalar loss is averaged the same way.
 __global__ void __launch_bounds__(256) grad_accumulate_kernel(float* __restrict__ acc, float* __restrict__ g, int64_t n4,
                                                               float w, int mode, float* loss_acc, float* loss) {
+    pdl_wait();
+    pdl_trigger();
     if (blockIdx.x == 0 && threadIdx.x == 0) {
         const float l = w * loss[0];
         if (mode == 0) loss_acc[0] = l;
@@ -628,7 +658,7 @@ __global__ void __launch_bounds__(256) grad_accumulate_kernel(float* __restrict_
 }
 cudaError_t launch_grad_accumulate(float* acc, float* g, int64_t n, float w, int mode, float* loss_acc, float* loss,
                                    cudaStream_t s) {
-    grad_accumulate_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(acc, g, n / 4, w, mode, loss_acc, loss);
+    BT_KERNEL_LAUNCH((grad_accumulate_kernel), grid_for(n / 4, 256, kStreamGridCap), 256, 0, s, acc, g, n / 4, w, mode, loss_acc, loss);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -637,6 +667,8 @@ cudaError_t launch_grad_accumulate(float* acc, float* g, int64_t n, float w, int
 
 __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restrict__ partials, int splits,
                                                             int64_t n4, float* __restrict__ out) {
+    pdl_wait();
+    pdl_trigger();
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n4; i += (int64_t)gridDim.x * blockDim.x) {
         float4 t = ld4(partials, i);
         for (int s = 1; s < splits; ++s) t = add4(t, ld4(partials, (int64_t)s * n4 + i));
@@ -644,7 +676,7 @@ __global__ void __launch_bounds__(256) splitk_reduce_kernel(const float* __restr
     }
 }
 cudaError_t launch_splitk_reduce(const float* partials, int splits, int64_t n, float* out, cudaStream_t s) {
-    splitk_reduce_kernel<<<grid_for(n / 4, 256, kStreamGridCap), 256, 0, s>>>(partials, splits, n / 4, out);
+    BT_KERNEL_LAUNCH((splitk_reduce_kernel), grid_for(n / 4, 256, kStreamGridCap), 256, 0, s, partials, splits, n / 4, out);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
@@ -661,6 +693,8 @@ __device__ __forceinline__ uint64_t splitmix64(uint64_t z) {
 }
 __global__ void __launch_bounds__(256) init_normal_kernel(float* __restrict__ p, int64_t n, float std, uint64_t seed,
                                                           uint64_t offset) {
+    pdl_wait();
+    pdl_trigger();
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x) {
         uint64_t r = splitmix64(splitmix64(seed) ^ (offset + (uint64_t)i));
         float u1 = ((float)(uint32_t)(r >> 40) + 0.5f) * (1.0f / 16777216.0f);
@@ -669,16 +703,18 @@ __global__ void __launch_bounds__(256) init_normal_kernel(float* __restrict__ p,
     }
 }
 __global__ void __launch_bounds__(256) fill_kernel(float* __restrict__ p, int64_t n, float v) {
+    pdl_wait();
+    pdl_trigger();
     for (int64_t i = blockIdx.x * (int64_t)blockDim.x + threadIdx.x; i < n; i += (int64_t)gridDim.x * blockDim.x)
         p[i] = v;
 }
 cudaError_t launch_init_normal(float* p, int64_t n, float std, uint64_t seed, uint64_t offset, cudaStream_t s) {
-    init_normal_kernel<<<grid_for(n, 256, kStreamGridCap), 256, 0, s>>>(p, n, std, seed, offset);
+    BT_KERNEL_LAUNCH((init_normal_kernel), grid_for(n, 256, kStreamGridCap), 256, 0, s, p, n, std, seed, offset);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
 cudaError_t launch_fill(float* p, int64_t n, float v, cudaStream_t s) {
-    fill_kernel<<<grid_for(n, 256, kStreamGridCap), 256, 0, s>>>(p, n, v);
+    BT_KERNEL_LAUNCH((fill_kernel), grid_for(n, 256, kStreamGridCap), 256, 0, s, p, n, v);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }

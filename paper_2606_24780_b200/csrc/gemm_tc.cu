@@ -134,6 +134,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot_ptr;
+    // barriers and tensor memory are set up; from here on global memory is read and written
+    pdl_wait();
+    pdl_trigger();
 
     const int units = g.tiles_m * g.tiles_n * g.splits;
 
@@ -452,7 +455,7 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     const int grid = (int)(units < sms ? units : sms);
 
 #define BT_LAUNCH(AM, BMN, BNV)                                                                              \
-    gemm_tc_kernel<AM, BMN, BNV, BK><<<grid, kThreads, Cfg<BNV, BK>::kSmemBytes, s>>>(tmA, tmB, g)
+    BT_KERNEL_LAUNCH((gemm_tc_kernel<AM, BMN, BNV, BK>), grid, kThreads, (Cfg<BNV, BK>::kSmemBytes), s, tmA, tmB, g)
 #define BT_LAUNCH_BN(BNV)                                                                                    \
     do {                                                                                                     \
         if (layout == kNT) BT_LAUNCH(false, false, BNV);                                                     \

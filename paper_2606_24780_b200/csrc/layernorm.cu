@@ -17,6 +17,8 @@ __global__ void __launch_bounds__(kLnWarps * 32) ln_fwd_kernel(const float* __re
                                                                const float* __restrict__ beta, int64_t N, int C4,
                                                                float* y, float* y_hi, float* y_lo,
                                                                float* __restrict__ mean, float* __restrict__ rstd) {
+    pdl_wait();
+    pdl_trigger();
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int64_t row = (int64_t)blockIdx.x * kLnWarps + warp;
     if (row >= N) return;
@@ -67,7 +69,7 @@ cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float
     const int vpl = (C4 + 31) / 32;
     const int grid = (int)((N + kLnWarps - 1) / kLnWarps);
 #define BT_LN_FWD(V)                                                                                     \
-    ln_fwd_kernel<V><<<grid, kLnWarps * 32, 0, s>>>(x, gamma, beta, N, C4, y, y_hi, y_lo, mean, rstd)
+    BT_KERNEL_LAUNCH((ln_fwd_kernel<V>), grid, kLnWarps * 32, 0, s, x, gamma, beta, N, C4, y, y_hi, y_lo, mean, rstd)
     if (vpl <= 1) BT_LN_FWD(1);
     else if (vpl <= 2) BT_LN_FWD(2);
     else if (vpl <= 4) BT_LN_FWD(4);
@@ -98,6 +100,8 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     const float* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ gamma,
     const float* __restrict__ mean, const float* __restrict__ rstd, const float* dres, int64_t N, int C4,
     float* dx, float* dx_hi, float* dx_lo, float* __restrict__ partial) {
+    pdl_wait();
+    pdl_trigger();
     extern __shared__ float4 sm[];  // [2][C4], then (CS) [kLnWarps][C4]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     float4* cs = sm + 2 * C4 + warp * C4;
@@ -195,6 +199,8 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
 __global__ void __launch_bounds__(256) ln_bwd_reduce_kernel(const float* __restrict__ partial, int nparts, int C4,
                                                             int kparts, float* __restrict__ dgamma,
                                                             float* __restrict__ dbeta, float* __restrict__ dcolsum) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ float4 sm[8][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int c = blockIdx.x * 32 + lane;  // float4 column over [kparts*C4): dgamma, dbeta, column sums
@@ -232,10 +238,10 @@ cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* g
 #define BT_LN_BWD(V)                                                                                          \
     do {                                                                                                      \
         if (dx_colsum)                                                                                        \
-            ln_bwd_kernel<V, true><<<grid, kLnWarps * 32, smem, s>>>(dy, x, gamma, mean, rstd, dres, N, C4, dx, \
+            BT_KERNEL_LAUNCH((ln_bwd_kernel<V, true>), grid, kLnWarps * 32, smem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, \
                                                                      dx_hi, dx_lo, scratch);                  \
         else                                                                                                  \
-            ln_bwd_kernel<V, false><<<grid, kLnWarps * 32, smem, s>>>(dy, x, gamma, mean, rstd, dres, N, C4, dx, \
+            BT_KERNEL_LAUNCH((ln_bwd_kernel<V, false>), grid, kLnWarps * 32, smem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, \
                                                                       dx_hi, dx_lo, scratch);                 \
     } while (0)
     if (vpl <= 1) BT_LN_BWD(1);
@@ -247,7 +253,7 @@ cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* g
 #undef BT_LN_BWD
     BT_COUNT_LAUNCH();
     const int kparts = dx_colsum ? 3 : 2;
-    ln_bwd_reduce_kernel<<<(kparts * C4 + 31) / 32, 256, 0, s>>>(scratch, grid, C4, kparts, dgamma, dbeta, dx_colsum);
+    BT_KERNEL_LAUNCH((ln_bwd_reduce_kernel), (kparts * C4 + 31) / 32, 256, 0, s, scratch, grid, C4, kparts, dgamma, dbeta, dx_colsum);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }

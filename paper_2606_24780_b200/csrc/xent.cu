@@ -28,6 +28,8 @@ __global__ void __launch_bounds__(kXentThreads) xent_kernel(const float* __restr
                                                             const int32_t* __restrict__ targets, int V4,
                                                             float inv_count, float* __restrict__ losses, float* dl,
                                                             float* dl_hi, float* dl_lo) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ float sm[kXentThreads / 32];
     const int64_t row = blockIdx.x;
     const int64_t base = row * V4;
@@ -82,6 +84,8 @@ __global__ void __launch_bounds__(kXentThreads) xent_generic_kernel(const float*
                                                                     const int32_t* __restrict__ targets, int V4,
                                                                     float inv_count, float* __restrict__ losses,
                                                                     float* dl, float* dl_hi, float* dl_lo) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ float sm[kXentThreads / 32];
     const int64_t row = blockIdx.x;
     const int64_t base = row * V4;
@@ -118,6 +122,8 @@ __global__ void __launch_bounds__(kXentThreads) xent_generic_kernel(const float*
 // loss_mean = inv_count * sum_n losses[n], summed in a fixed tree order by one CTA.
 __global__ void __launch_bounds__(1024) loss_mean_kernel(const float* __restrict__ losses, int64_t N, float inv_count,
                                                          float* __restrict__ loss_mean) {
+    pdl_wait();
+    pdl_trigger();
     __shared__ double sm[1024];
     double t = 0.0;
     for (int64_t i = threadIdx.x; i < N; i += 1024) t += (double)losses[i];
@@ -136,18 +142,18 @@ cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int
     const int V4 = Vp / 4;
     const int items = (V4 + kXentThreads - 1) / kXentThreads;
 #define BT_XENT(I)                                                                                              \
-    xent_kernel<I><<<(int)N, kXentThreads, 0, s>>>(logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo)
+    BT_KERNEL_LAUNCH((xent_kernel<I>), (int)N, kXentThreads, 0, s, logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo)
     if (items <= 1) BT_XENT(1);
     else if (items <= 2) BT_XENT(2);
     else if (items <= 4) BT_XENT(4);
     else if (items <= 8) BT_XENT(8);
     else if (items <= 16) BT_XENT(16);
     else if (items <= 25) BT_XENT(25);
-    else xent_generic_kernel<<<(int)N, kXentThreads, 0, s>>>(logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo);
+    else BT_KERNEL_LAUNCH((xent_generic_kernel), (int)N, kXentThreads, 0, s, logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo);
 #undef BT_XENT
     BT_COUNT_LAUNCH();
     if (loss_mean) {
-        loss_mean_kernel<<<1, 1024, 0, s>>>(losses, N, inv_count, loss_mean);
+        BT_KERNEL_LAUNCH((loss_mean_kernel), 1, 1024, 0, s, losses, N, inv_count, loss_mean);
         BT_COUNT_LAUNCH();
     }
     return cudaGetLastError();
