@@ -203,6 +203,40 @@ def attention_bwd(qkv, d_o, B, T, H):
     return dqkv
 
 
+def attention_dense(qkv, d_o, B, T, H):
+    """Causal attention forward and backward by its matrix definition, one (sequence, head) at a
+    time with float64 library matmuls: S = Q K^T / sqrt(d) with the strict upper triangle at -inf,
+    P = row softmax(S), O = P V; then dV = P^T dO, dP = dO V^T, dS = P o (dP - rowsum(dO o O)),
+    dQ = dS K / sqrt(d), dK = dS^T Q / sqrt(d).  It holds whole T x T matrices, so it serves where
+    the row-by-row C routine is too slow (long contexts); a test pins it to that routine.
+    Returns (o [B*T, C], lse [B, H, T], dqkv [B*T, 3C])."""
+    qkv, d_o = _d(qkv), _d(d_o)
+    C = qkv.shape[-1] // 3
+    d = C // H
+    o, lse, dqkv = np.empty((B * T, C)), np.empty((B, H, T)), np.empty((B * T, 3 * C))
+    upper = np.triu(np.ones((T, T), dtype=bool), k=1)
+    for b in range(B):
+        rows = slice(b * T, (b + 1) * T)
+        for h in range(H):
+            cq, ck, cv = (slice(p * C + h * d, p * C + (h + 1) * d) for p in range(3))
+            q, k, v, do = qkv[rows, cq], qkv[rows, ck], qkv[rows, cv], d_o[rows, h * d:(h + 1) * d]
+            s = (q @ k.T) / math.sqrt(d)
+            s[upper] = -np.inf
+            mx = s.max(axis=1, keepdims=True)
+            p = np.exp(s - mx)
+            den = p.sum(axis=1, keepdims=True)
+            p /= den
+            lse[b, h] = (mx + np.log(den)).ravel()
+            oh = p @ v
+            o[rows, h * d:(h + 1) * d] = oh
+            dp = do @ v.T
+            ds = p * (dp - (do * oh).sum(axis=1, keepdims=True))
+            dqkv[rows, cq] = (ds @ k) / math.sqrt(d)
+            dqkv[rows, ck] = (ds.T @ q) / math.sqrt(d)
+            dqkv[rows, cv] = p.T @ do
+    return o, lse, dqkv
+
+
 def gelu_fwd(x, tanh_form=False):
     x = _d(x)
     y = np.empty_like(x)

@@ -10,7 +10,11 @@
 //                 dV  += P^T  dO     A = P^T  (hi/lo written back to tensor memory),   B = dO tile
 //                 dK  += dS^T Q      A = dS^T (tensor memory),                          B = Q tile
 //               dK and dV accumulate in tensor memory over the whole walk (the backward needs no
-//               running-max rescaling).
+//               running-max rescaling).  The walk runs from the LAST query tile down to the diagonal:
+//               the tensor core adds into its FP32 accumulator with truncation, so a long chain of
+//               small additions to an already large sum drifts toward zero (about n * 2^-25 after
+//               n MMAs); probabilities of a key usually decay with the query's distance, and adding
+//               the small far-away terms first keeps that drift relative to a small sum.
 //   dq kernel   one CTA owns 128 query rows and walks the 32-key tiles up to the diagonal:
 //                 S  = Q' K^T (A = Q' in tensor memory),  dP = dO V^T (A = dO resident in smem),
 //                 dS = P o (dP - D),  dQ += dS K (A = dS in tensor memory).
@@ -245,7 +249,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 tma_load_3d(v_s + kb * (kResBytes / 2), &tmVres, v_full, 2 * g.C + h * HD + kb * 32, row_base + j0, 0);
             bool ok = true;
             for (int t = 0; t < n_t && ok; ++t) {
-                const int st = t & 1, q0 = (qt0 + t) * BT_;
+                const int st = t & 1, q0 = (n_qt - 1 - t) * BT_;   // walk from the last query tile down to the diagonal
                 const uint32_t ph = (t >> 1) & 1u;
                 if (!mbar_wait(kempty(st), ph ^ 1u, g.err, 21)) { ok = false; break; }
                 mbar_expect_tx(kfull(st), 2u * kTileBytes);
@@ -354,7 +358,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
         int tn = 0;
         const uint32_t tb = tbuf(wg) + t_lane;
         for (int t = wg; t < n_t && ok; t += 2) {
-            const int q0 = (qt0 + t) * BT_;
+            const int q0 = (n_qt - 1 - t) * BT_;
             // per-column softmax statistics of this query tile (same addresses in every thread:
             // broadcast loads, issued before the wait so their latency is hidden); rows past the
             // sequence end are clamped here and masked below

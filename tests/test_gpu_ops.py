@@ -338,3 +338,30 @@ def test_attention_bwd_tcgen05_kernels(B, T, H):
     for part in range(3):
         assert rel_l2(got[:, part * C:(part + 1) * C], rd[:, part * C:(part + 1) * C]) < 1e-4, part
     assert not (dqs[0].cpu().numpy().view(np.uint32) & 0x1FFF).any()
+
+
+def test_attention_long_context_16k():
+    """The long-context shape (T = 16,384, head_dim 64): 128 key tiles per query block in the forward,
+    512 query tiles per key block in the backward.  Two heads of one sequence against the
+    matrix-form float64 oracle."""
+    B, T, H, d = 1, 16384, 2, 64
+    C = H * d
+    qkv = si.normal_f32(85, (B * T, 3 * C))
+    d_o = si.normal_f32(86, (B * T, C), 1e-2)
+    dq, ddo = dev(qkv), dev(d_o)
+    qs, dos = empty(2, B * T, 3 * C), empty(2, B * T, C)
+    b.bt_op_split(dq, dq.numel(), qs)
+    b.bt_op_split(ddo, ddo.numel(), dos)
+    o, lse = empty(B * T, C), empty(B, H, T)
+    b.bt_op_attention_fwd(None, B, T, C, H, o, None, lse, 0, qkv_split=qs)
+    dqs = zeros(2, B * T, 3 * C)
+    nb = B * H * T * 4
+    b.bt_op_attention_bwd(None, o, lse, None, B, T, C, H, None, dqs, scratch(nb), nb, 0, qkv_split=qs, d_o_split=dos)
+    ro, rlse, rd = oracle.attention_dense(qkv, d_o, B, T, H)
+    assert rel_l2(host(o), ro) < 1e-4 and rel_max(host(o), ro) < 1e-4
+    assert np.abs(host(lse) - rlse).max() < 1e-4
+    got = host(dqs)
+    got = got[0] + got[1]
+    errs = [rel_l2(got[:, part * C:(part + 1) * C], rd[:, part * C:(part + 1) * C]) for part in range(3)]
+    print("T = 16384: o %.1e, dq %.1e, dk %.1e, dv %.1e (relative L2)" % (rel_l2(host(o), ro), *errs))
+    assert max(errs) < 1e-4, errs

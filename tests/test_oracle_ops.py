@@ -354,3 +354,16 @@ def test_lr_schedule_pins():
     assert (ms - wu) % 4 != 0 or abs(f(q) - (mn + 0.5 * (1 + 2 ** -0.5) * (mx - mn))) < 1e-15
     # no warmup, no decay
     assert oracle.lr_schedule(1, 1e-3, 1e-3, 0, 10) == 1e-3
+
+
+def test_dense_attention_route_equals_row_by_row_routine():
+    """The matrix-form attention (library matmuls, used for long contexts) against the row-by-row C
+    routine, which the tests above pin to the library, to finite differences and to special cases."""
+    B, T, H, d = 2, 150, 3, 16
+    qkv = si.normal_f32(901, (B * T, 3 * H * d)).astype(np.float64)
+    d_o = si.normal_f32(902, (B * T, H * d), 1e-2).astype(np.float64)
+    o, lse, dqkv = oracle.attention_dense(qkv, d_o, B, T, H)
+    ro, rlse = oracle.attention_fwd(qkv, B, T, H)
+    rd = oracle.attention_bwd(qkv, d_o, B, T, H)
+    assert np.abs(o - ro).max() < 1e-13 and np.abs(lse - rlse).max() < 1e-12
+    assert np.abs(dqkv - rd).max() < 1e-13 * max(1.0, np.abs(rd).max() / 1e-2)
