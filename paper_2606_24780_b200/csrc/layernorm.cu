@@ -92,9 +92,11 @@ static inline int ln_bwd_ctas(int64_t N) {
 }
 size_t layernorm_bwd_scratch_floats(int64_t N, int C) { return (size_t)ln_bwd_ctas(N) * 3 * C; }
 
-// CS: also accumulate the column sums of the rows written to dx (the bias gradient of the linear
-// layer whose output this dx is the gradient of).  Those sums live in shared memory, one private
-// array per warp, so they cost no registers.
+// Column accumulators (dgamma, dbeta and, with CS, the column sums of the dx written: the bias
+// gradient of the linear layer whose output this dx is the gradient of) live in shared memory, one
+// private array per warp, so the registers hold only the row being processed: x, dy and the
+// residual gradient are all requested before anything is consumed (18 128-bit loads in flight per
+// lane at C = 768), which is what keeps a two-CTA-per-SM kernel near the memory rate.
 template <int VPL, bool CS>
 __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     const float* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ gamma,
@@ -102,26 +104,16 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     float* dx, float* dx_hi, float* dx_lo, float* __restrict__ partial) {
     pdl_wait();
     pdl_trigger();
-    extern __shared__ float4 sm[];  // [2][C4], then (CS) [kLnWarps][C4]
+    constexpr int kParts = CS ? 3 : 2;
+    extern __shared__ float4 sm[];  // [kLnWarps][kParts][C4]
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float4* cs = sm + 2 * C4 + warp * C4;
-    if (CS) {
-        for (int i = lane; i < C4; i += 32) cs[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-        __syncwarp();
-    }
+    float4* acc = sm + (size_t)warp * kParts * C4;
+    for (int i = lane; i < kParts * C4; i += 32) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncwarp();
     const float inv_c = 1.0f / (float)(C4 * 4);
-    // Per-lane running sums of dy*xhat and dy for the columns this lane owns.  Only x, dy and
-    // these sums stay in registers (gamma is re-read through L1 each row), which keeps the kernel
-    // at two CTAs per SM.
-    float4 ag[VPL], ab[VPL];
-#pragma unroll
-    for (int k = 0; k < VPL; ++k) {
-        ag[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-        ab[k] = make_float4(0.f, 0.f, 0.f, 0.f);
-    }
     for (int64_t row = (int64_t)blockIdx.x * kLnWarps + warp; row < N; row += (int64_t)gridDim.x * kLnWarps) {
         const float mu = mean[row], rs = rstd[row];
-        float4 xv[VPL], dv[VPL];
+        float4 xv[VPL], dv[VPL], rv[VPL];
         float s1 = 0.f, s2 = 0.f;
 #pragma unroll
         for (int k = 0; k < VPL; ++k) {
@@ -129,6 +121,7 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
             if (idx < C4) {
                 xv[k] = ld4(x, row * C4 + idx);
                 dv[k] = ld4(dy, row * C4 + idx);
+                rv[k] = dres ? ld4(dres, row * C4 + idx) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
 #pragma unroll
@@ -137,9 +130,11 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
             if (idx < C4) {
                 const float4 gm = ld4(gamma, idx);
                 xv[k] = make_float4((xv[k].x - mu) * rs, (xv[k].y - mu) * rs, (xv[k].z - mu) * rs, (xv[k].w - mu) * rs);
-                ag[k].x += dv[k].x * xv[k].x; ag[k].y += dv[k].y * xv[k].y;
-                ag[k].z += dv[k].z * xv[k].z; ag[k].w += dv[k].w * xv[k].w;
-                ab[k] = add4(ab[k], dv[k]);
+                float4 a = acc[idx];
+                a.x += dv[k].x * xv[k].x; a.y += dv[k].y * xv[k].y;
+                a.z += dv[k].z * xv[k].z; a.w += dv[k].w * xv[k].w;
+                acc[idx] = a;
+                acc[C4 + idx] = add4(acc[C4 + idx], dv[k]);
                 dv[k] = make_float4(dv[k].x * gm.x, dv[k].y * gm.y, dv[k].z * gm.z, dv[k].w * gm.w);
                 s1 += (dv[k].x + dv[k].y) + (dv[k].z + dv[k].w);
                 s2 += (dv[k].x * xv[k].x + dv[k].y * xv[k].y) + (dv[k].z * xv[k].z + dv[k].w * xv[k].w);
@@ -156,41 +151,20 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
                 r.y = rs * (dv[k].y - s1 - xv[k].y * s2);
                 r.z = rs * (dv[k].z - s1 - xv[k].z * s2);
                 r.w = rs * (dv[k].w - s1 - xv[k].w * s2);
-                if (dres) r = add4(r, ld4(dres, row * C4 + idx));
+                r = add4(r, rv[k]);
                 store_raw_split(r, dx, dx_hi, dx_lo, row * C4 + idx);
-                if (CS) cs[idx] = add4(cs[idx], r);
+                if (CS) acc[2 * C4 + idx] = add4(acc[2 * C4 + idx], r);
             }
         }
     }
-    // combine the CTA's warps in warp order, then publish the CTA partial
-    for (int w = 0; w < kLnWarps; ++w) {
-        if (warp == w) {
-#pragma unroll
-            for (int k = 0; k < VPL; ++k) {
-                int idx = lane + 32 * k;
-                if (idx < C4) {
-                    if (w == 0) {
-                        sm[idx] = ag[k];
-                        sm[C4 + idx] = ab[k];
-                    } else {
-                        sm[idx] = add4(sm[idx], ag[k]);
-                        sm[C4 + idx] = add4(sm[C4 + idx], ab[k]);
-                    }
-                }
-            }
-        }
-        __syncthreads();
-    }
-    constexpr int kParts = CS ? 3 : 2;
+    // combine the CTA's warps in warp order and publish the CTA partial
+    __syncthreads();
     float4* dst = reinterpret_cast<float4*>(partial) + (int64_t)blockIdx.x * kParts * C4;
-    for (int i = threadIdx.x; i < 2 * C4; i += blockDim.x) dst[i] = sm[i];
-    if (CS) {   // the loop above ended with a __syncthreads, so every warp's array is complete
-        for (int i = threadIdx.x; i < C4; i += blockDim.x) {
-            float4 t = sm[2 * C4 + i];
+    for (int i = threadIdx.x; i < kParts * C4; i += blockDim.x) {
+        float4 t = sm[i];
 #pragma unroll
-            for (int w = 1; w < kLnWarps; ++w) t = add4(t, sm[(2 + w) * C4 + i]);
-            dst[2 * C4 + i] = t;
-        }
+        for (int w = 1; w < kLnWarps; ++w) t = add4(t, sm[(size_t)w * kParts * C4 + i]);
+        dst[i] = t;
     }
 }
 
@@ -227,6 +201,23 @@ __global__ void __launch_bounds__(256) ln_bwd_reduce_kernel(const float* __restr
     }
 }
 
+template <int V>
+static cudaError_t ln_bwd_set_smem_limit() {
+    constexpr int kMax = 160 * 1024;
+    cudaError_t e = cudaFuncSetAttribute(ln_bwd_kernel<V, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax);
+    if (e == cudaSuccess)
+        e = cudaFuncSetAttribute(ln_bwd_kernel<V, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kMax);
+    return e;
+}
+static cudaError_t ln_bwd_set_smem_limits() {
+    cudaError_t e = ln_bwd_set_smem_limit<1>();
+    if (e == cudaSuccess) e = ln_bwd_set_smem_limit<2>();
+    if (e == cudaSuccess) e = ln_bwd_set_smem_limit<4>();
+    if (e == cudaSuccess) e = ln_bwd_set_smem_limit<6>();
+    if (e == cudaSuccess) e = ln_bwd_set_smem_limit<8>();
+    return e;
+}
+
 cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
                                  const float* rstd, const float* dres, int64_t N, int C, float* dx, float* dx_hi,
                                  float* dx_lo, float* dgamma, float* dbeta, float* dx_colsum, float* scratch,
@@ -234,7 +225,9 @@ cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* g
     const int C4 = C / 4;
     const int vpl = (C4 + 31) / 32;
     const int grid = ln_bwd_ctas(N);
-    const size_t smem = (size_t)(dx_colsum ? 2 + kLnWarps : 2) * C4 * sizeof(float4);
+    const size_t smem = (size_t)kLnWarps * (dx_colsum ? 3 : 2) * C4 * sizeof(float4);   // 72 KB at C = 768 with sums
+    static const cudaError_t attr = ln_bwd_set_smem_limits();
+    if (attr != cudaSuccess) return attr;
 #define BT_LN_BWD(V)                                                                                          \
     do {                                                                                                      \
         if (dx_colsum)                                                                                        \
