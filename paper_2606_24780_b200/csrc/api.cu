@@ -178,7 +178,7 @@ bt_status validate(const bt_config* c) {
     if (d != 16 && d != 32 && d != 64 && d != 128)
         return fail(BT_ERR_UNSUPPORTED, "config: head_dim %d not in {16,32,64,128}", d);
     if (c->d_model % 32) return fail(BT_ERR_INVALID_ARG, "config: d_model %% 32 != 0");
-    if (c->d_model > 1024) return fail(BT_ERR_UNSUPPORTED, "config: d_model > 1024 not compiled");
+    if (c->d_model > 4096) return fail(BT_ERR_UNSUPPORTED, "config: d_model > 4096 not compiled");
     if (1 + 4 * (int64_t)c->n_layers > kMaxSplitMats) return fail(BT_ERR_UNSUPPORTED, "config: more than 63 layers");
     if (c->padded_vocab_size < c->vocab_size) return fail(BT_ERR_INVALID_ARG, "config: padded_vocab < vocab");
     if (c->padded_vocab_size % 32) return fail(BT_ERR_INVALID_ARG, "config: padded_vocab %% 32 != 0");
@@ -793,7 +793,7 @@ static bt_status layernorm_bwd_impl(const float* dy, const float* x, const float
     BT_PTR(dy); BT_PTR(x); BT_PTR(gamma); BT_PTR(mean); BT_PTR(rstd); BT_OPT_PTR(dres); BT_OPT_PTR(dx);
     BT_OPT_PTR(dx_split); BT_PTR(dgamma); BT_PTR(dbeta); BT_OPT_PTR(dx_colsum); BT_PTR(scratch);
     if (N < 1 || C < 4 || C % 4) return fail(BT_ERR_INVALID_ARG, "layernorm_bwd: bad sizes");
-    if (C > 1024) return fail(BT_ERR_UNSUPPORTED, "layernorm_bwd: C > 1024");
+    if (C > 4096) return fail(BT_ERR_UNSUPPORTED, "layernorm_bwd: C > 4096");
     if (scratch_bytes < bt_op_layernorm_bwd_scratch_bytes(N, C)) return fail(BT_ERR_OOM, "layernorm_bwd: scratch too small");
     BT_CUDA(launch_layernorm_bwd(dy, x, gamma, mean, rstd, dres, N, C, dx, dx_split,
                                  dx_split ? dx_split + N * C : nullptr, dgamma, dbeta, dx_colsum, (float*)scratch,

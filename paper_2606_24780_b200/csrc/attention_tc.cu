@@ -23,7 +23,7 @@
 // TMEM map (512 columns): per buffer b in {0,1}: S at 256b, P_hi at 256b+64, P_lo at 256b+128,
 // O_tile at 256b+192.  Shared memory: Q 64 KB, K 2 x 32 KB, V 2 x 32 KB.
 // Every mbarrier wait is bounded; a wait that runs out raises the device error word and the CTA
-// drains, frees its TMEM and exits.  No cluster multicast is used.
+// drains, frees its TMEM and exits.  Every TMA load targets this CTA's own shared memory only.
 #include "common.cuh"
 #include "tc_common.cuh"
 

@@ -21,7 +21,7 @@
 // Operand layouts.  "K-major" operands (rows of K contiguous: A of NT/NN, B of NT) use the
 // 128-byte swizzle; "MN-major" operands (K rows of M or N contiguous: A of TN, B of NN/TN) use
 // the 128-byte swizzle with 32-byte atoms, the only shared-memory layout the tensor core accepts
-// for transposed 32-bit operands.  No cluster multicast is used anywhere.
+// for transposed 32-bit operands.  Every TMA load targets the issuing CTA's own shared memory only.
 //
 // Every mbarrier wait is bounded: a wait that runs out raises a device error word and the CTA
 // drains and exits, still releasing its TMEM.

@@ -90,7 +90,13 @@ static inline int ln_bwd_ctas(int64_t N) {
     if (g > 148 * 2) g = 148 * 2;  // two CTAs per SM, one wave
     return (int)g;
 }
-size_t layernorm_bwd_scratch_floats(int64_t N, int C) { return (size_t)ln_bwd_ctas(N) * 3 * C; }
+static inline int ln_bwd_wide_ctas(int64_t N) {
+    int64_t g = (N + 3) / 4;   // four warps (rows) per CTA, one CTA per SM
+    return (int)(g < 148 ? g : 148);
+}
+size_t layernorm_bwd_scratch_floats(int64_t N, int C) {
+    return (size_t)(C > 1024 ? ln_bwd_wide_ctas(N) : ln_bwd_ctas(N)) * 3 * C;
+}
 
 // Column accumulators (dgamma, dbeta and, with CS, the column sums of the dx written: the bias
 // gradient of the linear layer whose output this dx is the gradient of) live in shared memory, one
@@ -168,6 +174,65 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     }
 }
 
+// Rows wider than the register-resident kernel takes (C > 1024): a warp walks its row twice, 32
+// float4 at a time -- once for the two row sums, once (the row now comes from L1/L2) for dx and
+// the column accumulators, which live in shared memory as above.  Four warps per CTA, one CTA per
+// SM: 3 x C floats of accumulators per warp.
+template <bool CS>
+__global__ void __launch_bounds__(128, 1) ln_bwd_wide_kernel(
+    const float* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ gamma,
+    const float* __restrict__ mean, const float* __restrict__ rstd, const float* dres, int64_t N, int C4,
+    float* dx, float* dx_hi, float* dx_lo, float* __restrict__ partial) {
+    pdl_wait();
+    pdl_trigger();
+    constexpr int kParts = CS ? 3 : 2;
+    constexpr int kWarps = 4;
+    extern __shared__ float4 sm[];  // [kWarps][kParts][C4]
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float4* acc = sm + (size_t)warp * kParts * C4;
+    for (int i = lane; i < kParts * C4; i += 32) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+    __syncwarp();
+    const float inv_c = 1.0f / (float)(C4 * 4);
+    for (int64_t row = (int64_t)blockIdx.x * kWarps + warp; row < N; row += (int64_t)gridDim.x * kWarps) {
+        const float mu = mean[row], rs = rstd[row];
+        float s1 = 0.f, s2 = 0.f;
+        for (int idx = lane; idx < C4; idx += 32) {
+            const float4 xv = ld4(x, row * C4 + idx), dv = ld4(dy, row * C4 + idx), gm = ld4(gamma, idx);
+            const float4 xh = make_float4((xv.x - mu) * rs, (xv.y - mu) * rs, (xv.z - mu) * rs, (xv.w - mu) * rs);
+            const float4 dg = make_float4(dv.x * gm.x, dv.y * gm.y, dv.z * gm.z, dv.w * gm.w);
+            s1 += (dg.x + dg.y) + (dg.z + dg.w);
+            s2 += (dg.x * xh.x + dg.y * xh.y) + (dg.z * xh.z + dg.w * xh.w);
+        }
+        s1 = warp_sum(s1) * inv_c;
+        s2 = warp_sum(s2) * inv_c;
+        for (int idx = lane; idx < C4; idx += 32) {
+            const float4 xv = ld4(x, row * C4 + idx), dv = ld4(dy, row * C4 + idx), gm = ld4(gamma, idx);
+            const float4 xh = make_float4((xv.x - mu) * rs, (xv.y - mu) * rs, (xv.z - mu) * rs, (xv.w - mu) * rs);
+            const float4 dg = make_float4(dv.x * gm.x, dv.y * gm.y, dv.z * gm.z, dv.w * gm.w);
+            float4 a = acc[idx];
+            a.x += dv.x * xh.x; a.y += dv.y * xh.y; a.z += dv.z * xh.z; a.w += dv.w * xh.w;
+            acc[idx] = a;
+            acc[C4 + idx] = add4(acc[C4 + idx], dv);
+            float4 r;
+            r.x = rs * (dg.x - s1 - xh.x * s2);
+            r.y = rs * (dg.y - s1 - xh.y * s2);
+            r.z = rs * (dg.z - s1 - xh.z * s2);
+            r.w = rs * (dg.w - s1 - xh.w * s2);
+            if (dres) r = add4(r, ld4(dres, row * C4 + idx));
+            store_raw_split(r, dx, dx_hi, dx_lo, row * C4 + idx);
+            if (CS) acc[2 * C4 + idx] = add4(acc[2 * C4 + idx], r);
+        }
+    }
+    __syncthreads();
+    float4* dst = reinterpret_cast<float4*>(partial) + (int64_t)blockIdx.x * kParts * C4;
+    for (int i = threadIdx.x; i < kParts * C4; i += blockDim.x) {
+        float4 t = sm[i];
+#pragma unroll
+        for (int w = 1; w < kWarps; ++w) t = add4(t, sm[(size_t)w * kParts * C4 + i]);
+        dst[i] = t;
+    }
+}
+
 // Sums the per-CTA partials in a fixed order: lane = float4 column, warp w takes partials
 // w, w+8, ... (four loads in flight), the eight warp sums are combined in warp order.
 __global__ void __launch_bounds__(256) ln_bwd_reduce_kernel(const float* __restrict__ partial, int nparts, int C4,
@@ -224,6 +289,27 @@ cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* g
                                  cudaStream_t s) {
     const int C4 = C / 4;
     const int vpl = (C4 + 31) / 32;
+    if (vpl > 8) {   // C > 1024: the two-pass kernel
+        if (C > 4096) return cudaErrorInvalidValue;
+        static const cudaError_t wattr = []() {
+            cudaError_t e = cudaFuncSetAttribute(ln_bwd_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            if (e == cudaSuccess)
+                e = cudaFuncSetAttribute(ln_bwd_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+            return e;
+        }();
+        if (wattr != cudaSuccess) return wattr;
+        const int kparts = dx_colsum ? 3 : 2;
+        const int wgrid = ln_bwd_wide_ctas(N);
+        const size_t wsmem = (size_t)4 * kparts * C4 * sizeof(float4);
+        if (dx_colsum)
+            BT_KERNEL_LAUNCH((ln_bwd_wide_kernel<true>), wgrid, 128, wsmem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, dx_hi, dx_lo, scratch);
+        else
+            BT_KERNEL_LAUNCH((ln_bwd_wide_kernel<false>), wgrid, 128, wsmem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, dx_hi, dx_lo, scratch);
+        BT_COUNT_LAUNCH();
+        BT_KERNEL_LAUNCH((ln_bwd_reduce_kernel), (kparts * C4 + 31) / 32, 256, 0, s, scratch, wgrid, C4, kparts, dgamma, dbeta, dx_colsum);
+        BT_COUNT_LAUNCH();
+        return cudaGetLastError();
+    }
     const int grid = ln_bwd_ctas(N);
     const size_t smem = (size_t)kLnWarps * (dx_colsum ? 3 : 2) * C4 * sizeof(float4);   // 72 KB at C = 768 with sums
     static const cudaError_t attr = ln_bwd_set_smem_limits();

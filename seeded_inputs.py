@@ -41,6 +41,8 @@ CONFIGS = {
             vocab_size=50257, padded_vocab_size=50304, batch=8, tokens="zipf"),
     5: dict(name="gpt2-124M-t16k-b2", n_layers=12, d_model=768, n_heads=12, seq_len=16384,
             vocab_size=50257, padded_vocab_size=50304, batch=2, tokens="zipf"),   # the long-context shape
+    6: dict(name="gpt2-2.42B-b2", n_layers=20, d_model=3072, n_heads=24, seq_len=1024,
+            vocab_size=50257, padded_vocab_size=50304, batch=2, tokens="zipf"),   # the paper's largest model
 }
 
 ADAMW = dict(lr=6e-4, beta1=0.9, beta2=0.95, eps=1e-8, weight_decay=0.1, grad_clip=1.0)

@@ -302,3 +302,11 @@ def test_training_trajectory_with_schedule_and_accumulation():
     assert np.abs(gpu_curve[:10] - ref_curve[:10]).max() < TOL_LOSS * ref_curve.max()
     assert gpu_curve[-10:].mean() < gpu_curve[0] - 0.5          # it learns the token frequencies
     gm.close()
+
+
+def test_wide_model_head_dim_128():
+    """One layer at the width of the paper's 2.42B configuration (d_model 3072, 24 heads of 128):
+    the wide LayerNorm backward, head_dim-128 attention and K = 12,288 GEMMs in one step."""
+    cfg = si.make_config(n_layers=1, d_model=3072, n_heads=24, seq_len=64, vocab_size=1000, padded_vocab_size=1024,
+                         batch=2, tokens="zipf")
+    run_steps(cfg, seed=6, flags=0, B=2, steps=1)

@@ -64,7 +64,8 @@ def test_layernorm_fwd(N, C):
     check_split(ys, host(y))
 
 
-@pytest.mark.parametrize("N,C,res", [(256, 64, True), (1000, 768, True), (4100, 768, False), (37, 1024, True)])
+@pytest.mark.parametrize("N,C,res", [(256, 64, True), (1000, 768, True), (4100, 768, False), (37, 1024, True),
+                                     (300, 3072, True), (9, 4096, False), (70, 1028, True)])
 def test_layernorm_bwd(N, C, res):
     x = si.normal_f32(13, (N, C), 1.5) - 0.2
     g = si.normal_f32(14, (C,), 0.3) + 1.0
@@ -98,7 +99,7 @@ def test_layernorm_bwd_in_place_residual():
     assert rel_l2(host(buf), rdx + dres) < 1e-5
 
 
-@pytest.mark.parametrize("N,C", [(1000, 768), (37, 132), (8192, 1024), (3, 4)])
+@pytest.mark.parametrize("N,C", [(1000, 768), (37, 132), (8192, 1024), (3, 4), (700, 3072), (5, 2052)])
 def test_layernorm_bwd_colsum(N, C):
     """The variant with fused column sums: same dx / dgamma / dbeta, plus colsum(dx) incl. residual."""
     x, dy, dres = si.normal_f32(31, (N, C), 1.5), si.normal_f32(32, (N, C), 1e-2), si.normal_f32(33, (N, C), 1e-2)
