@@ -72,7 +72,9 @@ typedef struct {
 enum {
     BT_FLAG_GELU_TANH = 1u,  /* tanh-form GELU instead of the exact erf form */
     BT_FLAG_GEMM_SIMT = 2u,  /* plain FP32 FMA GEMM (bring-up reference) instead of tcgen05 */
-    BT_FLAG_ATTN_SIMT = 4u   /* plain FP32 FMA attention (bring-up reference) */
+    BT_FLAG_ATTN_SIMT = 4u,  /* plain FP32 FMA attention (bring-up reference) */
+    BT_FLAG_GEMM_PAIR = 8u,  /* per-op GEMM calls: 256-row tiles on CTA pairs wherever M >= 256 */
+    BT_FLAG_GEMM_SINGLE = 16u /* per-op GEMM calls: 128-row tiles on single CTAs only (default: planner) */
 };
 
 /* AdamW hyper-parameters (hyper-parameter table, "Optimization" column).  grad_clip <= 0
@@ -252,7 +254,9 @@ BT_API bt_status bt_op_layernorm_bwd_colsum(const float* dy, const float* x, con
  *   BT_GEMM_NN: A [M,K], B [K,N]   (backward: dX = dY W)
  *   BT_GEMM_TN: A [K,M], B [K,N]   (backward: dW = dY^T X)
  * M, N, K multiples of 4 (NN/TN: the contiguous extents multiples of 32).
- * flags: BT_FLAG_GEMM_SIMT selects the FP32 FMA reference kernel. */
+ * flags: BT_FLAG_GEMM_SIMT selects the FP32 FMA reference kernel; BT_FLAG_GEMM_PAIR / BT_FLAG_GEMM_SINGLE
+ * pin the tensor-core tile (256 rows on a CTA pair / 128 rows on one CTA) instead of letting the
+ * wave-model planner choose. */
 enum { BT_GEMM_NT = 0, BT_GEMM_NN = 1, BT_GEMM_TN = 2 };
 
 /* x_split[0][i] = hi(x[i]), x_split[1][i] = lo(x[i]) for n values (n % 4 == 0). */

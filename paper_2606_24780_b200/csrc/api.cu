@@ -872,7 +872,9 @@ extern "C" bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int6
     float* partials = (float*)scratch;
     int* err = (int*)(partials + gemm_tc_partial_floats_bound());
     BT_CUDA(cudaMemsetAsync(err, 0, sizeof(int), s));
-    BT_CUDA(launch_gemm_tc(layout, M, N, K, Am, Bm, D, N, bias, residual, partials, gemm_tc_partial_floats_bound(), err, s));
+    const int two_cta_mode = (flags & BT_FLAG_GEMM_PAIR) ? 1 : (flags & BT_FLAG_GEMM_SINGLE) ? 0 : -1;
+    BT_CUDA(launch_gemm_tc(layout, M, N, K, Am, Bm, D, N, bias, residual, partials, gemm_tc_partial_floats_bound(), err, s,
+                           nullptr, 0, two_cta_mode));
     return BT_OK;
 }
 

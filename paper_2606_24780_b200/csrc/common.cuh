@@ -191,7 +191,9 @@ cudaError_t launch_gemm_simt(int layout, int64_t M, int64_t N, int64_t K, SplitM
 cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
                            int64_t ldd, const float* bias, const float* residual, float* partials,
                            size_t max_partial_floats, int* err_word, cudaStream_t s, float* d_hi = nullptr,
-                           int64_t d_plane = 0);
+                           int64_t d_plane = 0, int two_cta_mode = -1);
+// two_cta_mode: -1 the planner chooses between 128-row tiles on single CTAs and 256-row tiles on
+// CTA pairs (cta_group::2); 0 / 1 force the one or the other (1 applies where M >= 256).
 size_t gemm_tc_partial_floats_bound();
 bool gemm_tc_init(char* err, size_t errlen);  // resolves the tensor-map encoder
 

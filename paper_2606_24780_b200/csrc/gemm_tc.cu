@@ -302,12 +302,246 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
     }
 }
 
+// ------------------------------------------------------------------ CTA-pair variant
+//
+// The same GEMM on pairs of CTAs (a cluster of two on neighbouring SMs): the pair owns a 256 x BN
+// tile, one tcgen05.mma.cta_group::2 of M = 256 covers it, each CTA streams its own 128 rows of A
+// and only HALF of the B tile, so a third less operand data enters shared memory per MMA and the
+// ring gets deeper (32 KB stages instead of 48 KB).  The even CTA (leader) issues the MMAs and
+// owns the "stage full" and "accumulator drained" barriers; completion is broadcast to both CTAs'
+// "stage free" / "accumulator full" barriers by the commit.
+template <int BN, int BK>
+struct Cfg2 {
+    static constexpr uint32_t kATileBytes = 2u * BM * BK * 4u;          // this CTA's 128 rows, hi + lo
+    static constexpr uint32_t kBTileBytes = 2u * (BN / 2) * BK * 4u;    // this CTA's half of the columns
+    static constexpr uint32_t kStageBytes = kATileBytes + kBTileBytes;
+    static constexpr int kStagesFit = (int)((kSmemBudget - 2048u - kEpiStageBytes) / kStageBytes);
+    static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
+    static constexpr uint32_t kAccStride = 256u;
+    static constexpr uint32_t kTmemCols = 512u;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + kEpiStageBytes + 256;
+};
+
+template <bool A_MN, bool B_MN, int BN, int BK>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
+    using C = Cfg2<BN, BK>;
+    constexpr int BH = BN / 2;                         // B columns held by one CTA
+    constexpr uint32_t kMnAtomBytes = 2u * BK * 128u;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t epi_stage = smem_base + C::kStages * C::kStageBytes;
+    const uint32_t bars = epi_stage + kEpiStageBytes;
+    auto full_bar = [&](int s) { return bars + 8u * s; };
+    auto empty_bar = [&](int s) { return bars + 8u * (C::kStages + s); };
+    auto tfull_bar = [&](int a) { return bars + 8u * (2 * C::kStages + a); };
+    auto tempty_bar = [&](int a) { return bars + 8u * (2 * C::kStages + 2 + a); };
+    const uint32_t tmem_slot = bars + 8u * (2 * C::kStages + 4);
+    volatile uint32_t* tmem_slot_ptr =
+        reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_ctarank();          // 0 = leader
+    const int pair = blockIdx.x >> 1, n_pairs = gridDim.x >> 1;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < C::kStages; ++s) {
+            mbar_init(full_bar(s), 1);                 // used in the leader: its producer's expect_tx arrival
+            mbar_init(empty_bar(s), 1);                // one commit per use, delivered to both CTAs
+        }
+        for (int a = 0; a < 2; ++a) {
+            mbar_init(tfull_bar(a), 1);
+            mbar_init(tempty_bar(a), 2 * kEpiWarps);   // used in the leader: both CTAs' epilogue warps
+        }
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot),
+                     "r"(C::kTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();      // the partner's barriers exist before anything is signalled across the pair
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot_ptr;
+    pdl_wait();
+    pdl_trigger();
+
+    const int units = g.tiles_m * g.tiles_n * g.splits;   // tiles_m counts 256-row tiles here
+
+    if (warp == 0) {
+        // ---------------------------------------------------------------- TMA producer (both CTAs)
+        if (lane == 0) {
+            uint32_t it = 0;
+            bool ok = true;
+            for (int u = pair; u < units && ok; u += n_pairs) {
+                const int tm = u % g.tiles_m, r = u / g.tiles_m, tn = r % g.tiles_n, sp = r / g.tiles_n;
+                const int kb0 = sp * g.kb_per_split;
+                const int kb1 = min(g.kb_total, kb0 + g.kb_per_split);
+                const int a_row = tm * 2 * BM + (int)rank * BM;      // first A row (or column, if MN-major) of this CTA
+                const int b_col = tn * BN + (int)rank * BH;          // first B column of this CTA
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = it % C::kStages;
+                    const uint32_t ph = (it / C::kStages) & 1u;
+                    if (!mbar_wait(empty_bar(s), ph ^ 1u, g.err, 5)) { ok = false; break; }
+                    const uint32_t a_dst = smem_base + s * C::kStageBytes;
+                    const uint32_t b_dst = a_dst + C::kATileBytes;
+                    const uint32_t lbar = mapa_shared(full_bar(s), 0);   // the leader's barrier collects both halves
+                    if (rank == 0) mbar_expect_tx(full_bar(s), 2u * C::kStageBytes);
+                    if (A_MN) {
+#pragma unroll
+                        for (int a = 0; a < BM / 32; ++a)
+                            tma_load_3d_pair(a_dst + a * kMnAtomBytes, &tmA, lbar, a_row + 32 * a, kb * BK, 0);
+                    } else {
+                        tma_load_3d_pair(a_dst, &tmA, lbar, kb * BK, a_row, 0);
+                    }
+                    if (B_MN) {
+#pragma unroll
+                        for (int a = 0; a < BH / 32; ++a)
+                            tma_load_3d_pair(b_dst + a * kMnAtomBytes, &tmB, lbar, b_col + 32 * a, kb * BK, 0);
+                    } else {
+                        tma_load_3d_pair(b_dst, &tmB, lbar, kb * BK, b_col, 0);
+                    }
+                }
+            }
+            if (!ok)
+                for (int i = 0; i < 2000; ++i) __nanosleep(1000);
+        }
+    } else if (warp == 1) {
+        // ---------------------------------------------------------------- MMA issuer (leader only)
+        if (lane == 0 && rank == 0) {
+            constexpr uint32_t idesc = make_idesc_tf32(2 * BM, BN, A_MN, B_MN);
+            uint32_t it = 0, ut = 0;
+            bool ok = true;
+            for (int u = pair; u < units && ok; u += n_pairs, ++ut) {
+                const int r = u / g.tiles_m, sp = r / g.tiles_n;
+                const int kb0 = sp * g.kb_per_split;
+                const int kb1 = min(g.kb_total, kb0 + g.kb_per_split);
+                const int acc = ut & 1;
+                const uint32_t aph = (ut >> 1) & 1u;
+                if (!mbar_wait(tempty_bar(acc), aph ^ 1u, g.err, 6)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + (uint32_t)acc * C::kAccStride;
+                for (int kb = kb0; kb < kb1; ++kb, ++it) {
+                    const int s = it % C::kStages;
+                    const uint32_t ph = (it / C::kStages) & 1u;
+                    if (!mbar_wait(full_bar(s), ph, g.err, 7)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint32_t a_base = smem_base + s * C::kStageBytes;
+                    const uint32_t b_base = a_base + C::kATileBytes;
+#pragma unroll
+                    for (int j = 0; j < BK / 8; ++j) {
+                        const uint64_t a_hi = operand_desc<A_MN, BK>(a_base, BM, false, j);
+                        const uint64_t a_lo = operand_desc<A_MN, BK>(a_base, BM, true, j);
+                        const uint64_t b_hi = operand_desc<B_MN, BK>(b_base, BH, false, j);
+                        const uint64_t b_lo = operand_desc<B_MN, BK>(b_base, BH, true, j);
+                        umma2_tf32(d_tmem, a_lo, b_hi, idesc, (kb > kb0 || j > 0) ? 1u : 0u);
+                        umma2_tf32(d_tmem, a_hi, b_lo, idesc, 1u);
+                        umma2_tf32(d_tmem, a_hi, b_hi, idesc, 1u);
+                    }
+                    umma2_commit(empty_bar(s), (uint16_t)3);   // both CTAs may refill this stage
+                }
+                if (ok) umma2_commit(tfull_bar(acc), (uint16_t)3);
+            }
+        }
+    } else {
+        // ---------------------------------------------------------------- epilogue warps (both CTAs)
+        const int lane_group = warp & 3;
+        uint32_t ut = 0;
+        bool ok = true;
+        const uint32_t my_tempty0 = mapa_shared(tempty_bar(0), 0), my_tempty1 = mapa_shared(tempty_bar(1), 0);
+        for (int u = pair; u < units && ok; u += n_pairs, ++ut) {
+            const int tm = u % g.tiles_m, r = u / g.tiles_m, tn = r % g.tiles_n, sp = r / g.tiles_n;
+            const int acc = ut & 1;
+            const uint32_t aph = (ut >> 1) & 1u;
+            if (!mbar_wait_warp(tfull_bar(acc), aph, g.err, 8)) { ok = false; break; }
+            tc_fence_after();
+            float* Dp = g.D;
+            long long ldd = g.ldd;
+            if (g.splits > 1) {
+                Dp = g.partials + (long long)sp * g.M * g.N;
+                ldd = g.N;
+            }
+            const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)acc * C::kAccStride;
+            float* my_stage = reinterpret_cast<float*>(smem_raw + (epi_stage - smem_u32(smem_raw)) +
+                                                       (uint32_t)(warp - 2) * 32u * kEpiPitch);
+            const int sub = lane >> 3, cq = lane & 7;
+            const int row0 = tm * 2 * BM + (int)rank * BM + lane_group * 32;
+#pragma unroll 1
+            for (int c = 0; c < BN / 32; ++c) {
+                const int col0 = tn * BN + c * 32;
+                if (col0 >= g.N) break;  // warp-uniform
+                uint32_t rr[32];
+                tmem_ld32(t_row + c * 32, rr);
+                tmem_ld_wait();
+                float4* wr = reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(my_stage) + lane * kEpiPitch);
+#pragma unroll
+                for (int q = 0; q < 8; ++q)
+                    wr[q] = make_float4(__uint_as_float(rr[4 * q]), __uint_as_float(rr[4 * q + 1]),
+                                        __uint_as_float(rr[4 * q + 2]), __uint_as_float(rr[4 * q + 3]));
+                __syncwarp();
+                const int col = col0 + 4 * cq;
+                if (col < g.N) {
+                    float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
+                    if (g.bias) bv = *reinterpret_cast<const float4*>(g.bias + col);
+                    float4 rv[8];
+                    if (g.residual) {
+#pragma unroll
+                        for (int i = 0; i < 8; ++i) {
+                            const int row = row0 + sub + 4 * i;
+                            rv[i] = (row < g.M) ? *reinterpret_cast<const float4*>(g.residual + (long long)row * g.ldd + col)
+                                                : make_float4(0.f, 0.f, 0.f, 0.f);
+                        }
+                    }
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        const int rr_ = sub + 4 * i, row = row0 + rr_;
+                        if (row < g.M) {
+                            float4 v = *reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(my_stage) +
+                                                                        rr_ * kEpiPitch + cq * 16);
+                            v = add4(v, bv);
+                            if (g.residual) v = add4(v, rv[i]);
+                            if (Dp) *reinterpret_cast<float4*>(Dp + (long long)row * ldd + col) = v;
+                            if (g.d_hi) {
+                                float4 hh, ll;
+                                split_tf32(v, hh, ll);
+                                float* hrow = g.d_hi + (long long)row * g.ldd + col;
+                                *reinterpret_cast<float4*>(hrow) = hh;
+                                *reinterpret_cast<float4*>(hrow + g.d_plane) = ll;
+                            }
+                        }
+                    }
+                }
+                __syncwarp();
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(acc ? my_tempty1 : my_tempty0);   // on the leader's barrier
+        }
+    }
+
+    // The partner's shared and tensor memory stay in use by the pair's MMAs until both CTAs are done.
+    tc_fence_before();
+    __syncthreads();
+    cluster_sync_all();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(C::kTmemCols)
+                     : "memory");
+    }
+}
+
 // ------------------------------------------------------------------ host side
 
 EncodeTiledFn g_encode = nullptr;
 int g_num_sms = 0;
 int g_bk = 16;       // k-block depth in use (BT_GEMM_BK=32 selects the 128-byte-row variant)
 int g_force_bn = 0;  // BT_GEMM_BN=128|192|256 pins the tile width (tuning aid)
+// Measured time of a CTA-pair tile relative to two single-CTA tiles of the same width: 256-wide pair
+// tiles run about 5 % faster (a third less operand data into shared memory), 192-wide ones slower.
+double kTwoCtaFactor256 = 0.95, kTwoCtaFactor192 = 1.03;   // BT_GEMM_F256 / BT_GEMM_F192 override (tuning aid)
+int g_two_cta = -1;  // BT_GEMM_2CTA=0 never / 1 always (where the shape allows) / unset: the planner decides
 std::once_flag g_once;
 char g_init_err[256] = {0};
 
@@ -316,8 +550,20 @@ cudaError_t set_attr() {
     return cudaFuncSetAttribute(gemm_tc_kernel<A_MN, B_MN, BN, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                 (int)Cfg<BN, BK>::kSmemBytes);
 }
+template <bool A_MN, bool B_MN, int BN, int BK>
+cudaError_t set_attr2() {
+    return cudaFuncSetAttribute(gemm_tc2_kernel<A_MN, B_MN, BN, BK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                (int)Cfg2<BN, BK>::kSmemBytes);
+}
 template <bool A_MN, bool B_MN>
 cudaError_t set_attr_layout() {
+    {
+        cudaError_t b = set_attr2<A_MN, B_MN, 256, 16>();
+        if (b == cudaSuccess) b = set_attr2<A_MN, B_MN, 192, 16>();
+        if (b == cudaSuccess) b = set_attr2<A_MN, B_MN, 256, 32>();
+        if (b == cudaSuccess) b = set_attr2<A_MN, B_MN, 192, 32>();
+        if (b != cudaSuccess) return b;
+    }
     cudaError_t a = set_attr<A_MN, B_MN, 256, 16>();
     if (a == cudaSuccess) a = set_attr<A_MN, B_MN, 192, 16>();
     if (a == cudaSuccess) a = set_attr<A_MN, B_MN, 128, 16>();
@@ -339,6 +585,9 @@ void init_once() {
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (const char* v = getenv("BT_GEMM_BK")) g_bk = (atoi(v) == 32) ? 32 : 16;
+    if (const char* v = getenv("BT_GEMM_2CTA")) g_two_cta = atoi(v) ? 1 : 0;
+    if (const char* v = getenv("BT_GEMM_F256")) kTwoCtaFactor256 = atof(v);
+    if (const char* v = getenv("BT_GEMM_F192")) kTwoCtaFactor192 = atof(v);
     if (const char* v = getenv("BT_GEMM_BN")) {
         int bn = atoi(v);
         if (bn == 128 || bn == 192 || bn == 256) g_force_bn = bn;
@@ -367,36 +616,47 @@ bool encode_map(CUtensorMap* tm, const SplitMat& m, uint32_t box_cols, uint32_t 
 
 constexpr int kMaxUnitsForSplit = 4 * 148;
 
+
 struct Plan {
     int bn, splits, kb_per_split;
     double cost;
+    bool two_cta;   // 256-row tiles on CTA pairs
 };
 
 // Picks tile width and K-split by a simple wave model.  Every work unit of one launch costs the
 // same, so the launch takes ceil(units / SMs) unit times; a unit is (k-blocks + fixed overhead)
 // x tile width, narrower tiles pay a small efficiency penalty, and a K-split pays for writing
 // and re-reading its partial sums.
-Plan make_plan(int64_t M, int64_t N, int kb_total, int bk, int sms, bool can_split, size_t max_partial_floats) {
+Plan make_plan(int64_t M, int64_t N, int kb_total, int bk, int sms, bool can_split, size_t max_partial_floats,
+               int two_cta_mode) {   // -1: the planner decides, 0: single-CTA tiles only, 1: pair tiles where M >= 256
     const int tiles_m = (int)((M + BM - 1) / BM);
     const double kOverheadKb = 96.0 / bk;                     // pipeline fill + exposed epilogue, in k-blocks
     const double kb_seconds = 768.0 * (bk / 16.0) / 1.9e9;    // one 128x256 k-block of 3 MMAs at peak
     static const int kSplits[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 20, 24, 32};
-    Plan best{256, 1, kb_total, 1e300};
-    for (int bn : {256, 192, 128}) {
-        if (g_force_bn && bn != g_force_bn) continue;
-        if (bn > 128 && N <= bn - 64) continue;               // mostly padding
-        const double pen = bn == 256 ? 1.0 : bn == 192 ? 1.04 : 1.12;
-        const long long tiles = (long long)tiles_m * ((N + bn - 1) / bn);
-        for (int sp : kSplits) {
-            if (sp > 1 && (!can_split || kb_total / sp < 8 || (size_t)sp * M * N > max_partial_floats)) continue;
-            const int kbps = (kb_total + sp - 1) / sp;
-            const int real_sp = (kb_total + kbps - 1) / kbps;
-            if (real_sp != sp) continue;
-            const long long units = tiles * sp;
-            const long long rounds = (units + sms - 1) / sms;
-            double cost = (double)rounds * (kbps + kOverheadKb) * (bn / 256.0) * pen;
-            if (sp > 1) cost += (double)(sp + 1) * M * N * 4.0 / 6.0e12 / kb_seconds;
-            if (cost < best.cost) best = Plan{bn, sp, kbps, cost};
+    Plan best{256, 1, kb_total, 1e300, false};
+    for (int two = 0; two < 2; ++two) {
+        if (two && (two_cta_mode == 0 || M < 256)) continue;
+        if (!two && two_cta_mode == 1 && M >= 256) continue;
+        for (int bn : {256, 192, 128}) {
+            if (g_force_bn && bn != g_force_bn) continue;
+            if (two && bn == 128) continue;
+            if (bn > 128 && N <= bn - 64) continue;               // mostly padding
+            const double pen = (bn == 256 ? 1.0 : bn == 192 ? 1.04 : 1.12) *
+                               (two ? (bn == 256 ? kTwoCtaFactor256 : kTwoCtaFactor192) : 1.0);
+            const long long tm = two ? (M + 2 * BM - 1) / (2 * BM) : tiles_m;
+            const long long tiles = tm * ((N + bn - 1) / bn);
+            const int slots = two ? sms / 2 : sms;
+            for (int sp : kSplits) {
+                if (sp > 1 && (!can_split || kb_total / sp < 8 || (size_t)sp * M * N > max_partial_floats)) continue;
+                const int kbps = (kb_total + sp - 1) / sp;
+                const int real_sp = (kb_total + kbps - 1) / kbps;
+                if (real_sp != sp) continue;
+                const long long units = tiles * sp;
+                const long long rounds = (units + slots - 1) / slots;
+                double cost = (double)rounds * (kbps + kOverheadKb) * (bn / 256.0) * pen;
+                if (sp > 1) cost += (double)(sp + 1) * M * N * 4.0 / 6.0e12 / kb_seconds;
+                if (cost < best.cost) best = Plan{bn, sp, kbps, cost, two != 0};
+            }
         }
     }
     return best;
@@ -427,25 +687,27 @@ template <int BK>
 static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const SplitMat& A, const SplitMat& B,
                              float* D, int64_t ldd, const float* bias, const float* residual, float* partials,
                              size_t max_partial_floats, int* err_word, float* d_hi, int64_t d_plane,
-                             cudaStream_t s) {
+                             cudaStream_t s, int two_cta_mode) {
     const bool a_mn = (layout == kTN), b_mn = (layout != kNT);
     const int sms = g_num_sms > 0 ? g_num_sms : 148;
     const int kb_total = (int)((K + BK - 1) / BK);
     const bool can_split = !bias && !residual && partials && ldd == N && D && !d_hi;
-    const Plan plan = make_plan(M, N, kb_total, BK, sms, can_split, max_partial_floats);
+    const Plan plan = make_plan(M, N, kb_total, BK, sms, can_split, max_partial_floats,
+                                two_cta_mode >= 0 ? two_cta_mode : g_two_cta);
     const int bn = plan.bn;
 
     const CUtensorMapSwizzle sw_k = (BK == 32) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
     const CUtensorMapSwizzle sw_mn = CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B;
     CUtensorMap tmA, tmB;
     bool ok = a_mn ? encode_map(&tmA, A, 32, BK, sw_mn) : encode_map(&tmA, A, BK, BM, sw_k);
-    ok = ok && (b_mn ? encode_map(&tmB, B, 32, BK, sw_mn) : encode_map(&tmB, B, BK, (uint32_t)bn, sw_k));
+    ok = ok && (b_mn ? encode_map(&tmB, B, 32, BK, sw_mn)
+                     : encode_map(&tmB, B, BK, (uint32_t)(plan.two_cta ? bn / 2 : bn), sw_k));
     if (!ok) return cudaErrorInvalidValue;
 
     GemmArgs g;
     g.M = (int)M; g.N = (int)N; g.K = (int)K;
     g.D = D; g.ldd = ldd; g.bias = bias; g.residual = residual;
-    g.tiles_m = (int)((M + BM - 1) / BM);
+    g.tiles_m = plan.two_cta ? (int)((M + 2 * BM - 1) / (2 * BM)) : (int)((M + BM - 1) / BM);
     g.tiles_n = (int)((N + bn - 1) / bn);
     g.splits = plan.splits;
     g.kb_per_split = plan.kb_per_split; g.kb_total = kb_total;
@@ -453,6 +715,26 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     g.d_hi = d_hi; g.d_plane = d_plane;
     const long long units = (long long)g.tiles_m * g.tiles_n * g.splits;
     const int grid = (int)(units < sms ? units : sms);
+    if (plan.two_cta) {
+        const int pairs = (int)(units < sms / 2 ? units : sms / 2);
+#define BT_LAUNCH2(AM, BMN, BNV)                                                                             \
+    BT_KERNEL_LAUNCH((gemm_tc2_kernel<AM, BMN, BNV, BK>), 2 * pairs, kThreads, (Cfg2<BNV, BK>::kSmemBytes), s, tmA, tmB, g)
+#define BT_LAUNCH2_BN(BNV)                                                                                   \
+    do {                                                                                                     \
+        if (layout == kNT) BT_LAUNCH2(false, false, BNV);                                                    \
+        else if (layout == kNN) BT_LAUNCH2(false, true, BNV);                                                \
+        else BT_LAUNCH2(true, true, BNV);                                                                    \
+    } while (0)
+        if (bn == 256) BT_LAUNCH2_BN(256);
+        else BT_LAUNCH2_BN(192);
+#undef BT_LAUNCH2_BN
+#undef BT_LAUNCH2
+        BT_COUNT_LAUNCH();
+        cudaError_t e2 = cudaGetLastError();
+        if (e2 != cudaSuccess) return e2;
+        if (g.splits > 1) return launch_splitk_reduce(partials, g.splits, M * N, D, s);
+        return cudaSuccess;
+    }
 
 #define BT_LAUNCH(AM, BMN, BNV)                                                                              \
     BT_KERNEL_LAUNCH((gemm_tc_kernel<AM, BMN, BNV, BK>), grid, kThreads, (Cfg<BNV, BK>::kSmemBytes), s, tmA, tmB, g)
@@ -476,14 +758,14 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
 
 cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D, int64_t ldd,
                            const float* bias, const float* residual, float* partials, size_t max_partial_floats,
-                           int* err_word, cudaStream_t s, float* d_hi, int64_t d_plane) {
+                           int* err_word, cudaStream_t s, float* d_hi, int64_t d_plane, int two_cta_mode) {
     if (!gemm_tc_init(nullptr, 0)) return cudaErrorNotSupported;
     if (!D && !d_hi) return cudaErrorInvalidValue;
     if (g_bk == 32)
         return launch_bk<32>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word,
-                             d_hi, d_plane, s);
+                             d_hi, d_plane, s, two_cta_mode);
     return launch_bk<16>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word, d_hi,
-                         d_plane, s);
+                         d_plane, s, two_cta_mode);
 }
 
 }  // namespace bt

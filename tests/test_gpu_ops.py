@@ -234,10 +234,12 @@ GEMM_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("flags", [0, b.BT_FLAG_GEMM_SIMT])
+@pytest.mark.parametrize("flags", [0, b.BT_FLAG_GEMM_SIMT, b.BT_FLAG_GEMM_PAIR, b.BT_FLAG_GEMM_SINGLE])
 @pytest.mark.parametrize("layout,M,N,K", GEMM_SHAPES)
 def test_gemm(layout, M, N, K, flags):
-    if flags == 0 and ((layout == 2 and M % 32) or (layout != 0 and N % 32)):
+    """flags 0: the planner picks the tile; PAIR / SINGLE force the cta_group::2 (256-row tiles on
+    CTA pairs) or the single-CTA kernel; SIMT is the FP32 FMA reference kernel."""
+    if flags != b.BT_FLAG_GEMM_SIMT and ((layout == 2 and M % 32) or (layout != 0 and N % 32)):
         pytest.skip("transposed extents must be multiples of 32 on the tensor-core path")
     a_shape = (K, M) if layout == 2 else (M, K)
     b_shape = (N, K) if layout == 0 else (K, N)
@@ -254,7 +256,7 @@ def test_gemm(layout, M, N, K, flags):
         ref = A64 @ B64
         if use_epi:
             ref = ref + bias + res
-        assert rel_l2(host(D), ref) < 1e-5 if flags else rel_l2(host(D), ref) < 1e-4, (layout, M, N, K, use_epi)
+        assert rel_l2(host(D), ref) < (1e-5 if flags == b.BT_FLAG_GEMM_SIMT else 1e-4), (layout, M, N, K, use_epi)
         assert rel_max(host(D), ref) < 1e-4
 
 

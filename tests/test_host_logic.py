@@ -40,7 +40,7 @@ def test_workspace_bytes_and_config_validation(lib):
     for bad in [b.make_config(0, 64, 4, 64, 512, 512, 4), b.make_config(2, 66, 4, 64, 512, 512, 4),
                 b.make_config(2, 64, 4, 64, 512, 500, 4), b.make_config(2, 64, 4, 64, 512, 520, 4),
                 b.make_config(2, 96, 4, 64, 512, 512, 4), b.make_config(2, 64, 4, 64, 512, 512, 0),
-                b.make_config(2, 2048, 16, 64, 512, 512, 1)]:
+                b.make_config(2, 8192, 64, 64, 512, 512, 1)]:
         assert b.bt_workspace_bytes(bad) == 0
         assert lib.bt_last_error()
 
