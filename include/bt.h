@@ -271,6 +271,14 @@ BT_API size_t bt_op_gemm_split_scratch_bytes(void);
 BT_API bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
                                   const float* B_split, float* D, const float* bias, const float* residual,
                                   void* scratch, size_t scratch_bytes, uint32_t flags, void* stream);
+/* The same, and D_act_split [2][M][N] (device) receives the TF32 hi/lo planes of act(D) from the
+ * same epilogue: act 0 = D itself, 1 = GELU(D) in the exact erf form, 2 = the tanh form.  The
+ * training step uses it for the MLP up-projection (Section 2: h = m Wfc^T + b is kept for the
+ * backward, g = GELU(h) is the next GEMM's operand). */
+BT_API bt_status bt_op_gemm_split_act(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
+                                      const float* B_split, float* D, float* D_act_split, int32_t act,
+                                      const float* bias, const float* residual, void* scratch,
+                                      size_t scratch_bytes, uint32_t flags, void* stream);
 BT_API bt_status bt_op_gemm_check(const void* scratch, void* stream);
 
 /* Convenience form on raw FP32 operands: bt_op_split of A and B into `scratch`, then

@@ -79,6 +79,7 @@ _SIGNATURES = {
     "bt_op_split": (_i32, [_vp, _i64, _vp, _vp]),
     "bt_op_gemm_split_scratch_bytes": (_sz, []),
     "bt_op_gemm_split": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
+    "bt_op_gemm_split_act": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 4 + [_i32] + [_vp] * 3 + [_sz, _u32, _vp]),
     "bt_op_gemm_check": (_i32, [_vp, _vp]),
     "bt_op_gemm": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
     "bt_op_attention_fwd": (_i32, [_vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _u32, _vp]),
@@ -329,6 +330,12 @@ def bt_op_split(x, n, x_split, stream=None):
 
 def bt_op_gemm_split_scratch_bytes():
     return int(lib().bt_op_gemm_split_scratch_bytes())
+
+
+def bt_op_gemm_split_act(layout, M, N, K, A_split, B_split, D, D_act_split, act, bias, residual, scratch,
+                         scratch_bytes, flags=0, stream=None):
+    _check(lib().bt_op_gemm_split_act(layout, M, N, K, _ptr(A_split), _ptr(B_split), _ptr(D), _ptr(D_act_split), act,
+                                      _ptr(bias), _ptr(residual), _ptr(scratch), scratch_bytes, flags, _stream(stream)))
 
 
 def bt_op_gemm_split(layout, M, N, K, A_split, B_split, D, bias, residual, scratch, scratch_bytes, flags=0,

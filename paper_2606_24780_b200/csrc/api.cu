@@ -317,15 +317,18 @@ inline double attn_fwd_flops(int64_t B, int64_t H, int64_t T, int64_t d) {
 
 // D = op(A) op(B) (+bias)(+residual) through the tensor-core kernel or the FMA reference.
 cudaError_t gemm_raw(bt_model* m, int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
-                 const float* bias, const float* residual, float* d_split = nullptr) {
+                 const float* bias, const float* residual, float* d_split = nullptr, int act = 0) {
     if (m->cfg.flags & BT_FLAG_GEMM_SIMT) {
         // the FMA reference writes the raw output; the planes are made by a separate pass
         cudaError_t e = launch_gemm_simt(layout, M, N, K, A, B, D, N, bias, residual, m->stream);
-        if (e == cudaSuccess && d_split) e = launch_split(D, d_split, d_split + M * N, M * N, m->stream);
+        if (e == cudaSuccess && d_split) {
+            if (act) e = launch_gelu_fwd(D, M * N, act == 2, nullptr, d_split, d_split + M * N, m->stream);
+            else e = launch_split(D, d_split, d_split + M * N, M * N, m->stream);
+        }
         return e;
     }
     return launch_gemm_tc(layout, M, N, K, A, B, D, N, bias, residual, m->partials, m->partial_floats, m->err_word,
-                          m->stream, d_split, M * N);
+                          m->stream, d_split, M * N, -1, act);
 }
 
 // Timing category by role: the forward products (Y = X W^T, run as NN on the transposed weight
@@ -574,9 +577,10 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
         BT_GEMM(kNN, N, C, C, act_mat(a.o_s, N, C, N), weight_mat_t(m, layer_tensor(m, l, PROJW), C, C), a.x1,
                      P(PROJB), a.x);
         BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x1, P(LN2G), P(LN2B), N, C, nullptr, a.m_s, a.m_s + N * C, a.mean2, a.rstd2, s));
-        BT_GEMM(kNN, N, F, C, act_mat(a.m_s, N, C, N), weight_mat_t(m, layer_tensor(m, l, FCW), F, C), a.h,
-                     P(FCB), nullptr);
-        BT_STEP(kCatGeluFwd, 0, 12.0 * N * F, launch_gelu_fwd(a.h, N * F, tanh_form, nullptr, a.g_s, a.g_s + N * F, s));
+        // h = m Wfc^T + bfc is kept (the backward needs it); g = GELU(h) leaves the same epilogue as hi/lo planes
+        BT_STEP(kCatGemmNT, gemm_flops(N, F, C), gemm_bytes(N, F, C) + 8.0 * N * F,
+                gemm_raw(m, kNN, N, F, C, act_mat(a.m_s, N, C, N), weight_mat_t(m, layer_tensor(m, l, FCW), F, C), a.h,
+                         P(FCB), nullptr, a.g_s, tanh_form ? 2 : 1));
         BT_GEMM(kNN, N, C, F, act_mat(a.g_s, N, F, N), weight_mat_t(m, layer_tensor(m, l, PRW), C, F), xout,
                      P(PRB), a.x1);
     }
@@ -848,10 +852,13 @@ extern "C" bt_status bt_op_split(const float* x, int64_t n, float* x_split, void
     return BT_OK;
 }
 
-extern "C" bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
-                                      const float* B_split, float* D, const float* bias, const float* residual,
-                                      void* scratch, size_t scratch_bytes, uint32_t flags, void* stream) {
-    BT_PTR(A_split); BT_PTR(B_split); BT_PTR(D); BT_OPT_PTR(bias); BT_OPT_PTR(residual); BT_PTR(scratch);
+static bt_status gemm_split_impl(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
+                                 const float* B_split, float* D, float* D_act_split, int32_t act, const float* bias,
+                                 const float* residual, void* scratch, size_t scratch_bytes, uint32_t flags,
+                                 void* stream) {
+    BT_PTR(A_split); BT_PTR(B_split); BT_PTR(D); BT_OPT_PTR(D_act_split); BT_OPT_PTR(bias); BT_OPT_PTR(residual);
+    BT_PTR(scratch);
+    if (act < 0 || act > 2) return fail(BT_ERR_INVALID_ARG, "gemm: act %d", act);
     if (layout < 0 || layout > 2) return fail(BT_ERR_INVALID_ARG, "gemm: layout %d", layout);
     if (M < 1 || N < 1 || K < 1 || M % 4 || N % 4 || K % 4) return fail(BT_ERR_INVALID_ARG, "gemm: M, N, K must be positive multiples of 4");
     if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return fail(BT_ERR_INVALID_ARG, "gemm: size too large");
@@ -863,6 +870,10 @@ extern "C" bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int6
     SplitMat Am{A_split, na, sh.a_rows, sh.a_cols, sh.a_cols}, Bm{B_split, nb, sh.b_rows, sh.b_cols, sh.b_cols};
     if (flags & BT_FLAG_GEMM_SIMT) {
         BT_CUDA(launch_gemm_simt(layout, M, N, K, Am, Bm, D, N, bias, residual, s));
+        if (D_act_split) {
+            if (act) BT_CUDA(launch_gelu_fwd(D, M * N, act == 2, nullptr, D_act_split, D_act_split + M * N, s));
+            else BT_CUDA(launch_split(D, D_act_split, D_act_split + M * N, M * N, s));
+        }
         return BT_OK;
     }
     if ((layout == BT_GEMM_TN && M % 32) || (layout != BT_GEMM_NT && N % 32))
@@ -874,8 +885,24 @@ extern "C" bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int6
     BT_CUDA(cudaMemsetAsync(err, 0, sizeof(int), s));
     const int two_cta_mode = (flags & BT_FLAG_GEMM_PAIR) ? 1 : (flags & BT_FLAG_GEMM_SINGLE) ? 0 : -1;
     BT_CUDA(launch_gemm_tc(layout, M, N, K, Am, Bm, D, N, bias, residual, partials, gemm_tc_partial_floats_bound(), err, s,
-                           nullptr, 0, two_cta_mode));
+                           D_act_split, M * N, two_cta_mode, act));
     return BT_OK;
+}
+
+extern "C" bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
+                                      const float* B_split, float* D, const float* bias, const float* residual,
+                                      void* scratch, size_t scratch_bytes, uint32_t flags, void* stream) {
+    return gemm_split_impl(layout, M, N, K, A_split, B_split, D, nullptr, 0, bias, residual, scratch, scratch_bytes,
+                           flags, stream);
+}
+
+extern "C" bt_status bt_op_gemm_split_act(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
+                                          const float* B_split, float* D, float* D_act_split, int32_t act,
+                                          const float* bias, const float* residual, void* scratch,
+                                          size_t scratch_bytes, uint32_t flags, void* stream) {
+    if (!D_act_split) return fail(BT_ERR_INVALID_ARG, "gemm_split_act: D_act_split is NULL");
+    return gemm_split_impl(layout, M, N, K, A_split, B_split, D, D_act_split, act, bias, residual, scratch,
+                           scratch_bytes, flags, stream);
 }
 
 extern "C" bt_status bt_op_gemm_check(const void* scratch, void* stream) {

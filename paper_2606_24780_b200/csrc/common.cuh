@@ -77,6 +77,17 @@ struct SplitMat {
     int64_t rows, cols, ld;
 };
 
+#ifdef __CUDACC__
+// GELU (exact erf form, or the tanh form): shared by the GELU kernels and the GEMM epilogue.
+__device__ __forceinline__ float gelu_f(float x, bool tanh_form) {
+    if (tanh_form) {
+        float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
+        return 0.5f * x * (1.0f + tanhf(u));
+    }
+    return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f));
+}
+#endif
+
 // ---------------------------------------------------------------- programmatic dependent launch
 // Every kernel of the step starts with pdl_wait() (returns once the kernels before it in the stream
 // have completed and their writes are visible) followed by pdl_trigger() (lets the NEXT launch be
@@ -191,7 +202,8 @@ cudaError_t launch_gemm_simt(int layout, int64_t M, int64_t N, int64_t K, SplitM
 cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
                            int64_t ldd, const float* bias, const float* residual, float* partials,
                            size_t max_partial_floats, int* err_word, cudaStream_t s, float* d_hi = nullptr,
-                           int64_t d_plane = 0, int two_cta_mode = -1);
+                           int64_t d_plane = 0, int two_cta_mode = -1, int act = 0);
+// act: 1 / 2 = the hi/lo planes receive GELU(output) (erf / tanh form) while D keeps the output itself.
 // two_cta_mode: -1 the planner chooses between 128-row tiles on single CTAs and 256-row tiles on
 // CTA pairs (cta_group::2); 0 / 1 force the one or the other (1 applies where M >= 256).
 size_t gemm_tc_partial_floats_bound();

@@ -215,13 +215,6 @@ cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N,
 
 // ------------------------------------------------------------------ GELU
 
-__device__ __forceinline__ float gelu_f(float x, bool tanh_form) {
-    if (tanh_form) {
-        float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-        return 0.5f * x * (1.0f + tanhf(u));
-    }
-    return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f));
-}
 __device__ __forceinline__ float gelu_grad_f(float x, bool tanh_form) {
     if (tanh_form) {
         float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);

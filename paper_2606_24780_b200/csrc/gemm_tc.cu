@@ -74,6 +74,7 @@ struct GemmArgs {
     int* err;
     float* d_hi;        // optional TF32 hi/lo planes of the output (lo = d_hi + d_plane)
     long long d_plane;
+    int act;            // 0: the planes hold the output; 1 / 2: they hold GELU(output), erf / tanh form
 };
 
 // Descriptor of one 8-deep k-step of an operand tile.
@@ -277,6 +278,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             if (g.residual) v = add4(v, rv[i]);
                             if (Dp) *reinterpret_cast<float4*>(Dp + (long long)row * ldd + col) = v;
                             if (g.d_hi) {
+                                if (g.act) {   // the raw output above stays pre-activation (the backward needs it)
+                                    const bool th = g.act == 2;
+                                    v = make_float4(gelu_f(v.x, th), gelu_f(v.y, th), gelu_f(v.z, th), gelu_f(v.w, th));
+                                }
                                 float4 hh, ll;
                                 split_tf32(v, hh, ll);
                                 float* hrow = g.d_hi + (long long)row * g.ldd + col;
@@ -505,6 +510,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             if (g.residual) v = add4(v, rv[i]);
                             if (Dp) *reinterpret_cast<float4*>(Dp + (long long)row * ldd + col) = v;
                             if (g.d_hi) {
+                                if (g.act) {   // the raw output above stays pre-activation (the backward needs it)
+                                    const bool th = g.act == 2;
+                                    v = make_float4(gelu_f(v.x, th), gelu_f(v.y, th), gelu_f(v.z, th), gelu_f(v.w, th));
+                                }
                                 float4 hh, ll;
                                 split_tf32(v, hh, ll);
                                 float* hrow = g.d_hi + (long long)row * g.ldd + col;
@@ -687,7 +696,7 @@ template <int BK>
 static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const SplitMat& A, const SplitMat& B,
                              float* D, int64_t ldd, const float* bias, const float* residual, float* partials,
                              size_t max_partial_floats, int* err_word, float* d_hi, int64_t d_plane,
-                             cudaStream_t s, int two_cta_mode) {
+                             cudaStream_t s, int two_cta_mode, int act) {
     const bool a_mn = (layout == kTN), b_mn = (layout != kNT);
     const int sms = g_num_sms > 0 ? g_num_sms : 148;
     const int kb_total = (int)((K + BK - 1) / BK);
@@ -712,7 +721,7 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     g.splits = plan.splits;
     g.kb_per_split = plan.kb_per_split; g.kb_total = kb_total;
     g.partials = partials; g.err = err_word;
-    g.d_hi = d_hi; g.d_plane = d_plane;
+    g.d_hi = d_hi; g.d_plane = d_plane; g.act = d_hi ? act : 0;
     const long long units = (long long)g.tiles_m * g.tiles_n * g.splits;
     const int grid = (int)(units < sms ? units : sms);
     if (plan.two_cta) {
@@ -758,14 +767,14 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
 
 cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D, int64_t ldd,
                            const float* bias, const float* residual, float* partials, size_t max_partial_floats,
-                           int* err_word, cudaStream_t s, float* d_hi, int64_t d_plane, int two_cta_mode) {
+                           int* err_word, cudaStream_t s, float* d_hi, int64_t d_plane, int two_cta_mode, int act) {
     if (!gemm_tc_init(nullptr, 0)) return cudaErrorNotSupported;
     if (!D && !d_hi) return cudaErrorInvalidValue;
     if (g_bk == 32)
         return launch_bk<32>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word,
-                             d_hi, d_plane, s, two_cta_mode);
+                             d_hi, d_plane, s, two_cta_mode, act);
     return launch_bk<16>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word, d_hi,
-                         d_plane, s, two_cta_mode);
+                         d_plane, s, two_cta_mode, act);
 }
 
 }  // namespace bt

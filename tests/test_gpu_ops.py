@@ -368,3 +368,27 @@ def test_attention_long_context_16k():
     errs = [rel_l2(got[:, part * C:(part + 1) * C], rd[:, part * C:(part + 1) * C]) for part in range(3)]
     print("T = 16384: o %.1e, dq %.1e, dk %.1e, dv %.1e (relative L2)" % (rel_l2(host(o), ro), *errs))
     assert max(errs) < 1e-4, errs
+
+
+@pytest.mark.parametrize("flags", [b.BT_FLAG_GEMM_PAIR, b.BT_FLAG_GEMM_SINGLE, b.BT_FLAG_GEMM_SIMT])
+@pytest.mark.parametrize("act", [0, 1, 2])
+def test_gemm_epilogue_activation_planes(act, flags):
+    """The MLP up-projection as the step runs it: weight given transposed (layout NN), bias in the
+    epilogue, the raw output kept and GELU(output) emitted as TF32 hi/lo planes by the same kernel."""
+    N, cin, cout = 520, 256, 768
+    x, w, bias = si.normal_f32(91, (N, cin)), si.normal_f32(92, (cout, cin), 0.1), si.normal_f32(93, (cout,), 0.5)
+    xs, wts = empty(2, N, cin), empty(2, cin, cout)
+    b.bt_op_split(dev(x), N * cin, xs)
+    b.bt_op_split(dev(np.ascontiguousarray(w.T)), cin * cout, wts)
+    h, gs = empty(N, cout), empty(2, N, cout)
+    nb = b.bt_op_gemm_split_scratch_bytes()
+    b.bt_op_gemm_split_act(1, N, cout, cin, xs, wts, h, gs, act, dev(bias), None, scratch(nb), nb, flags)
+    rh = oracle.linear_fwd(x, w, bias)
+    assert rel_l2(host(h), rh) < 1e-4
+    want = rh if act == 0 else oracle.gelu_fwd(rh.ravel(), act == 2).reshape(N, cout)
+    got = host(gs)
+    assert rel_l2(got[0] + got[1], want) < 1e-4
+    # the planes are the split of the kernel's own FP32 value of act(h)
+    ref32 = host(h) if act == 0 else oracle.gelu_fwd(host(h).ravel(), act == 2).reshape(N, cout)
+    assert np.abs((got[0].astype(np.float64) + got[1]) - ref32).max() < 1e-5 * np.abs(ref32).max()
+    assert not (gs[0].cpu().numpy().view(np.uint32) & 0x1FFF).any()
