@@ -32,7 +32,7 @@ METRIC = "GPT-2 124M FP32 train tokens/s on 1 B200"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 TF32_OVER_BF16 = 0.5          # nominal dense ratio (1.1 / 2.25 PFLOP/s)
 MMA_PER_PRODUCT = 3.0         # 3xTF32: three tensor-core products per FP32 product
-NCU_GEMM_FC_DRAM_BYTES = 127.1e6 + 71.2e6   # read + write of one forward fc GEMM launch (ncu summary in profiles/)
+NCU_GEMM_QKV_DRAM_BYTES = 109.6e6 + 46.0e6   # read + write of one forward QKV GEMM launch (ncu summary in profiles/)
 
 
 def load_peaks():
@@ -267,15 +267,15 @@ def run_ours(args, cfg):
     gemm_ms = sum(v["ms_per_step"] for v in gemm.values())
     gemm_flops = sum(v["tflops"] * v["ms_per_step"] for v in gemm.values())  # TFLOP/s * ms
     achieved = gemm_flops / gemm_ms if gemm_ms > 0 else 0.0
-    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel (forward, dX and dW products, 3xTF32)", "achieved": achieved,
+    roofline = {"bound": "tensor", "kernel": "gemm_tc_kernel / gemm_tc2_kernel (forward, dX and dW products, 3xTF32)", "achieved": achieved,
                 "peak": tf32x3_peak, "unit": "TFLOP/s", "frac": achieved / tf32x3_peak,
                 "peak_kind": f"{peak_kind} bf16 sustained x {TF32_OVER_BF16} (tf32) / {MMA_PER_PRODUCT:g} (3xTF32)",
                 "share_of_step": gemm_ms / sum(v["ms_per_step"] for v in kernels.values()),
-                # DRAM bytes of ONE launch of the forward fc GEMM (8192 x 3072 x 768) from the committed
+                # DRAM bytes of ONE launch of the forward QKV GEMM (8192 x 2304 x 768) from the committed
                 # ncu capture under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum), beside
                 # its algorithmic bytes 8(MK + NK) + 4MN; other launches scale with their own sizes
-                "traffic": NCU_GEMM_FC_DRAM_BYTES, "traffic_launch": "gemm forward fc, M=8192 N=3072 K=768",
-                "traffic_algorithmic": 8.0 * (8192 * 768 + 3072 * 768) + 4.0 * 8192 * 3072}
+                "traffic": NCU_GEMM_QKV_DRAM_BYTES, "traffic_launch": "gemm forward qkv, M=8192 N=2304 K=768",
+                "traffic_algorithmic": 8.0 * (8192 * 768 + 2304 * 768) + 4.0 * 8192 * 2304}
 
     flop_per_token = si_flops_per_token(cfg)
     step_frac = value / world * flop_per_token / 1e12 / tf32x3_peak
