@@ -190,6 +190,31 @@ typedef struct {
 } bt_lr_schedule;
 BT_API float bt_lr_at(const bt_lr_schedule* s, int64_t step);
 
+/* Double-buffered batch production (Algorithm 2).  The token stream is a list of shards (host
+ * int32 arrays the caller keeps alive, e.g. memory-mapped files); rank r of `world` starts at
+ * position B*T*r of shard 0, each batch is the window [pos, pos + B*T) as tokens and
+ * [pos + 1, pos + B*T + 1) as targets, pos advances by B*T*world, and the next shard is opened when
+ * fewer than B*T + 1 tokens remain at pos (checked before a window is taken) or fewer than
+ * B*T*world + 1 remain after the advance.  Every shard must hold at least B*T*world + 1 tokens.
+ *   d_buffers: device, 4*B*T int32 (tokens/targets of the two channels), caller-owned;
+ *   h_pinned:  page-locked host memory of the same size, or NULL: then windows are copied straight
+ *              from the shards, synchronously, with identical results;
+ *   compute_stream: the stream the consumer (bt_train_step ...) runs on.
+ * bt_loader_next returns device pointers to the next batch; the pointers stay valid until the
+ * second following call.  The copy for the batch after next is already in flight on the loader's
+ * own stream; events order the two streams in both directions.  Unlike the algorithm as printed,
+ * the host also waits for the previous copy out of a pinned buffer before rewriting it (the host
+ * may run ahead of the GPU).  bt_loader_plan is the cursor alone (host only): the shard index and
+ * position of the first n_batches windows. */
+typedef struct bt_loader bt_loader;
+BT_API bt_status bt_loader_plan(const int64_t* shard_lens, int32_t n_shards, int32_t B, int32_t T, int32_t rank,
+                                int32_t world, int32_t n_batches, int32_t* out_shard, int64_t* out_pos);
+BT_API bt_status bt_loader_create(const int32_t* const* shards, const int64_t* shard_lens, int32_t n_shards,
+                                  int32_t B, int32_t T, int32_t rank, int32_t world, int32_t* d_buffers,
+                                  int32_t* h_pinned, void* compute_stream, bt_loader** out);
+BT_API bt_status bt_loader_next(bt_loader* loader, const int32_t** d_tokens, const int32_t** d_targets);
+BT_API void bt_loader_destroy(bt_loader* loader);
+
 /* Synchronises and reads the loss of the last forward. */
 BT_API bt_status bt_get_loss(bt_model* m, float* h_loss);
 

@@ -285,6 +285,26 @@ def adamw(p, g, m, v, lr, beta1, beta2, eps, weight_decay, decay, t, scale=1.0):
 
 # ------------------------------------------------------------------------- model
 
+def loader_windows(shard_lens, B, T, rank, world, n_batches):
+    """The batch cursor of Algorithm 2 (double-buffered batch production), without any copying:
+    the (shard, position) of each of the first n_batches windows a rank reads.  A window is B*T
+    tokens at `position` (the targets are the same window one token later); the rank starts at
+    B*T*rank, moves on by B*T*world after each window, and opens the next shard (positions start
+    again at B*T*rank) when the current one has fewer than B*T + 1 tokens left at the position --
+    tested before a window is taken -- or fewer than B*T*world + 1 left after moving on."""
+    bt = B * T
+    cur, pos = 0, bt * rank
+    out = []
+    for _ in range(n_batches):
+        if pos + bt + 1 > shard_lens[cur]:
+            cur, pos = (cur + 1) % len(shard_lens), bt * rank
+        out.append((cur, pos))
+        pos += bt * world
+        if pos + bt * world + 1 > shard_lens[cur]:
+            cur, pos = (cur + 1) % len(shard_lens), bt * rank
+    return out
+
+
 def lr_schedule(step: int, max_lr: float, min_lr: float, warmup_steps: int, max_steps: int) -> float:
     """Learning rate of optimizer step `step` (first step = 1), from the four numbers of the
     hyper-parameter table (max / min learning rate, warmup steps, training steps).  The paper gives

@@ -61,6 +61,12 @@ _SIGNATURES = {
     "bt_micro_step": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, ctypes.POINTER(_f)]),
     "bt_train_step_accum": (_i32, [_vp, _vp, _vp, _i32, _i32, ctypes.POINTER(bt_adamw_config), ctypes.POINTER(_f)]),
     "bt_lr_at": (_f, [ctypes.POINTER(bt_lr_schedule), _i64]),
+    "bt_loader_plan": (_i32, [ctypes.POINTER(_i64), _i32, _i32, _i32, _i32, _i32, _i32, ctypes.POINTER(_i32),
+                              ctypes.POINTER(_i64)]),
+    "bt_loader_create": (_i32, [ctypes.POINTER(_vp), ctypes.POINTER(_i64), _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp,
+                                ctypes.POINTER(_vp)]),
+    "bt_loader_next": (_i32, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp)]),
+    "bt_loader_destroy": (None, [_vp]),
     "bt_get_loss": (_i32, [_vp, ctypes.POINTER(_f)]),
     "bt_launch_count": (_i64, [_vp]),
     "bt_last_error": (ctypes.c_char_p, []),
@@ -251,6 +257,47 @@ def bt_train_step_accum(model, tokens, targets, B, n_micro, opt, want_loss=True)
 
 def bt_lr_at(schedule, step):
     return float(lib().bt_lr_at(ctypes.byref(schedule), step))
+
+
+def bt_loader_plan(shard_lens, B, T, rank, world, n_batches):
+    """Host only: [(shard, position)] of the first n_batches windows of this rank."""
+    n = len(shard_lens)
+    lens = (_i64 * n)(*shard_lens)
+    out_s, out_p = (_i32 * n_batches)(), (_i64 * n_batches)()
+    _check(lib().bt_loader_plan(lens, n, B, T, rank, world, n_batches, out_s, out_p))
+    return [(int(out_s[i]), int(out_p[i])) for i in range(n_batches)]
+
+
+class Loader:
+    """Double-buffered batch production over host int32 token shards (CPU torch tensors, kept alive
+    here).  `next()` returns (tokens, targets) as device int32 tensors of shape [B, T]."""
+
+    def __init__(self, shards, B, T, rank=0, world=1, pinned=True, device="cuda", stream=None):
+        self.shards = [s.contiguous() for s in shards]
+        self.B, self.T = B, T
+        n = len(self.shards)
+        ptrs = (_vp * n)(*[s.data_ptr() for s in self.shards])
+        lens = (_i64 * n)(*[s.numel() for s in self.shards])
+        self.d_buffers = torch.empty(4 * B * T, dtype=torch.int32, device=device)
+        self.h_pinned = torch.empty(4 * B * T, dtype=torch.int32).pin_memory() if pinned else None
+        self.h = _vp()
+        _check(lib().bt_loader_create(ptrs, lens, n, B, T, rank, world, _ptr(self.d_buffers), _ptr(self.h_pinned),
+                                      _stream(stream), ctypes.byref(self.h)))
+
+    def next(self):
+        x, y = _vp(), _vp()
+        _check(lib().bt_loader_next(self.h, ctypes.byref(x), ctypes.byref(y)))
+        base, n = self.d_buffers.data_ptr(), self.B * self.T
+        ox, oy = (x.value - base) // 4, (y.value - base) // 4
+        return (self.d_buffers[ox:ox + n].view(self.B, self.T), self.d_buffers[oy:oy + n].view(self.B, self.T))
+
+    def close(self):
+        if self.h:
+            lib().bt_loader_destroy(self.h)
+            self.h = None
+
+    def __del__(self):
+        self.close()
 
 
 def bt_get_loss(model):

@@ -310,3 +310,39 @@ def test_wide_model_head_dim_128():
     cfg = si.make_config(n_layers=1, d_model=3072, n_heads=24, seq_len=64, vocab_size=1000, padded_vocab_size=1024,
                          batch=2, tokens="zipf")
     run_steps(cfg, seed=6, flags=0, B=2, steps=1)
+
+
+@pytest.mark.parametrize("pinned", [True, False])
+def test_double_buffered_loader_feeds_the_step(pinned):
+    """Algorithm 2 on the GPU: batches arrive through the copy stream two channels deep; every batch
+    is bit-identical to the window the oracle's cursor names, for two interleaved ranks over three
+    shards with wrap-around, and the training step can consume them directly."""
+    cfg = si.config(0)
+    B, T, world = 2, cfg["seq_len"], 2
+    bt_ = B * T
+    rng = np.random.Generator(np.random.PCG64(11))
+    lens = [bt_ * world * 3 + 1, bt_ * world + 7, bt_ * world * 2 + 1]
+    shards = [rng.integers(0, cfg["vocab_size"], n).astype(np.int32) for n in lens]
+    tshards = [torch.from_numpy(s) for s in shards]
+    loaders = [b.Loader(tshards, B, T, rank=r, world=world, pinned=pinned) for r in range(world)]
+    want = [oracle.loader_windows(lens, B, T, r, world, 14) for r in range(world)]
+    gm, om = make_pair(cfg, 3, 0, B)
+    opt = b.make_adamw(**si.ADAMW)
+    for i in range(14):
+        for r in range(world):
+            x, y = loaders[r].next()
+            s, p = want[r][i]
+            assert np.array_equal(x.cpu().numpy().ravel(), shards[s][p:p + bt_])
+            assert np.array_equal(y.cpu().numpy().ravel(), shards[s][p + 1:p + bt_ + 1])
+            if r == 0 and i < 3:
+                loss = gm.train_step(x, y, opt)
+                ref = om.loss_and_grad(x.cpu().numpy(), y.cpu().numpy())
+                assert abs(loss - ref) < TOL_LOSS * ref
+                hp = si.ADAMW
+                om.adamw_step(hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], hp["grad_clip"])
+                for n in om.names():
+                    for kind in (0, 2, 3):
+                        om.set_tensor(n, host(gm.tensor(n, kind)), kind)
+    for L in loaders:
+        L.close()
+    gm.close()

@@ -87,3 +87,18 @@ def test_lr_schedule_matches_oracle():
         for step in list(range(0, 25)) + [wu - 1, wu, wu + 1, (wu + ms) // 2, ms - 1, ms, ms + 1, 10 * ms + 3]:
             want = oracle.lr_schedule(step, np.float32(mx), np.float32(mn), wu, ms)
             assert abs(b.bt_lr_at(sched, step) - want) <= 1e-6 * mx, (mx, mn, wu, ms, step)
+
+
+def test_loader_plan_matches_oracle_cursor():
+    """bt_loader_plan is host arithmetic (the cursor of Algorithm 2): same windows as the oracle's."""
+    import oracle
+    B, T = 2, 8
+    for world in (1, 2, 3):
+        for lens in ([B * T * world * 4 + 1, B * T * world * 2 + 5, B * T * world + 1], [B * T * world + 1],
+                     [1000, 517, 999]):
+            if min(lens) < B * T * world + 1:
+                continue
+            for rank in range(world):
+                assert b.bt_loader_plan(lens, B, T, rank, world, 50) == oracle.loader_windows(lens, B, T, rank, world, 50)
+    with pytest.raises(b.BtError):
+        b.bt_loader_plan([10], B, T, 0, 1, 1)            # shorter than one batch + 1

@@ -367,3 +367,30 @@ def test_dense_attention_route_equals_row_by_row_routine():
     rd = oracle.attention_bwd(qkv, d_o, B, T, H)
     assert np.abs(o - ro).max() < 1e-13 and np.abs(lse - rlse).max() < 1e-12
     assert np.abs(dqkv - rd).max() < 1e-13 * max(1.0, np.abs(rd).max() / 1e-2)
+
+
+def test_loader_windows_pins():
+    """Batch cursor of Algorithm 2 against what the algorithm fixes: rank r starts at B*T*r, windows of
+    one rank are B*T*world apart, the ranks' windows tile a shard without gaps or overlap, a window
+    (plus its one-token-later target window) never crosses a shard's end, and shards are visited
+    cyclically."""
+    B, T = 2, 8
+    bt = B * T
+    world = 3
+    lens = [bt * world * 4 + 1, bt * world * 2 + 5, bt * world + 1]
+    per_rank = [oracle.loader_windows(lens, B, T, r, world, 40) for r in range(world)]
+    for r, wins in enumerate(per_rank):
+        assert wins[0] == (0, bt * r)
+        for (s0, p0), (s1, p1) in zip(wins, wins[1:]):
+            assert p0 + bt + 1 <= lens[s0]                       # tokens and targets fit
+            if s1 == s0 and p1 > p0:
+                assert p1 - p0 == bt * world                     # the global rank stride
+            else:
+                assert s1 == (s0 + 1) % len(lens) and p1 == bt * r
+    # inside one pass over shard 0 the ranks interleave into a gap-free tiling
+    first = sorted(p for wins in per_rank for (s, p) in wins[:4] if s == 0)
+    assert first == [bt * k for k in range(len(first))]
+    # shard 0 holds exactly 4 global batches + 1 token: every rank takes 4 windows there, then moves on
+    assert [s for s, _ in per_rank[0][:8]] == [0, 0, 0, 0, 1, 1, 2, 0]
+    # one rank, one shard of exactly one batch + 1: the same window for ever
+    assert oracle.loader_windows([bt + 1], B, T, 0, 1, 3) == [(0, 0)] * 3
