@@ -34,6 +34,16 @@ def make_pair(cfg, seed, flags, max_batch, jitter=0.02):
     return gm, om
 
 
+def grad_error(got, ref, scale=0.0):
+    """Relative L2 error of a gradient (part); a gradient that is mathematically zero (oracle norm
+    below 1e-12 sqrt(numel)) is held to an absolute bound instead -- 1e-9 per element, or 1e-5 of
+    `scale`, the size of a neighbouring non-zero gradient -- and counts as error 0."""
+    if np.linalg.norm(ref) < 1e-12 * math.sqrt(ref.size):
+        assert np.linalg.norm(got) <= max(1e-9, 1e-5 * scale) * math.sqrt(ref.size), np.linalg.norm(got)
+        return 0.0
+    return rel_l2(got, ref)
+
+
 def compare_gradients(gm, om, cfg):
     C = cfg["d_model"]
     worst = 0.0
@@ -42,14 +52,15 @@ def compare_gradients(gm, om, cfg):
         got = host(gm.tensor(name, 1))
         if name.endswith("attn.qkv.b"):
             # q and v parts relative; the k part is exactly zero in exact arithmetic
+            vscale = np.abs(ref[2 * C:]).max()
             for lo, hi in ((0, C), (2 * C, 3 * C)):
-                e = rel_l2(got[lo:hi], ref[lo:hi])
+                e = grad_error(got[lo:hi], ref[lo:hi], vscale)
                 assert e < TOL_GRAD, (name, lo, e)
                 worst = max(worst, e)
             assert np.abs(ref[C:2 * C]).max() < 1e-12
-            assert np.abs(got[C:2 * C]).max() < 1e-3 * np.abs(ref[:C]).max(), name
+            assert np.abs(got[C:2 * C]).max() <= max(1e-3 * np.abs(ref[:C]).max(), 1e-5 * vscale) + 1e-9, name
             continue
-        e = rel_l2(got, ref)
+        e = grad_error(got, ref)
         assert e < TOL_GRAD, (name, e)
         worst = max(worst, e)
     return worst
@@ -346,3 +357,13 @@ def test_double_buffered_loader_feeds_the_step(pinned):
     for L in loaders:
         L.close()
     gm.close()
+
+
+@pytest.mark.parametrize("L,C,H,T,V,B", [(1, 64, 4, 5, 40, 3), (1, 64, 1, 7, 36, 1), (2, 128, 2, 1, 32, 2),
+                                         (1, 64, 4, 64, 512, 1), (1, 32, 2, 3, 8, 1)])
+def test_ragged_and_degenerate_shapes(L, C, H, T, V, B):
+    """Token counts that are no multiple of anything (15, 7, 3 rows), a single sequence, and context
+    length 1, where attention is the identity on v and the query / key gradients vanish exactly."""
+    cfg = si.make_config(n_layers=L, d_model=C, n_heads=H, seq_len=T, vocab_size=V,
+                         padded_vocab_size=(V + 31) // 32 * 32, batch=B, tokens="uniform")
+    run_steps(cfg, seed=4, flags=0, B=B, steps=2)
