@@ -392,3 +392,22 @@ def test_gemm_epilogue_activation_planes(act, flags):
     ref32 = host(h) if act == 0 else oracle.gelu_fwd(host(h).ravel(), act == 2).reshape(N, cout)
     assert np.abs((got[0].astype(np.float64) + got[1]) - ref32).max() < 1e-5 * np.abs(ref32).max()
     assert not (gs[0].cpu().numpy().view(np.uint32) & 0x1FFF).any()
+
+
+def test_empty_inputs_are_no_ops_or_rejected():
+    """Zero-length calls: the element-wise entry points accept n = 0 and launch nothing; calls whose
+    result is undefined for no rows (reductions, GEMM) refuse them on the host."""
+    x = empty(4)
+    b.bt_op_gelu_fwd(x, 0, 0, x, None)
+    b.bt_op_gelu_bwd(x, x, 0, 0, x, None)
+    b.bt_op_embedding_fwd(dev(np.zeros(1, np.int32)), x, x, 0, 1, 4, x)
+    b.bt_op_layernorm_fwd(x, x, x, 0, 4, x, None, x, x)
+    for call in (lambda: b.bt_op_colsum(x, 0, 4, x, x, 1024),
+                 lambda: b.bt_op_softmax_xent(x, dev(np.zeros(1, np.int32)), 0, 4, 1.0, x, None, None, None),
+                 lambda: b.bt_op_grad_norm(x, 0, 1.0, x, x, 1024),
+                 lambda: b.bt_op_gemm_split(0, 0, 4, 4, x, x, x, None, None, scratch(b.bt_op_gemm_split_scratch_bytes()),
+                                            b.bt_op_gemm_split_scratch_bytes())):
+        with pytest.raises(b.BtError) as e:
+            call()
+        assert e.value.status == 1
+    torch.cuda.synchronize()
