@@ -193,8 +193,25 @@ __device__ __forceinline__ uint32_t setup(uint32_t bars, int n_bars_count1, uint
 }
 
 // ------------------------------------------------------------------------------------------ dkv
-
-constexpr uint32_t kDkvSmem = 1024u + kResBytes + 2u * 4u * kTileBytes + 1024u;
+//
+// 64-row query tiles, single score buffers, and an issue order that still keeps the tensor pipe fed:
+//     ... dV(t) | S^T(t+1) | dK(t) | dP^T(t+1) | dV(t+1) | S^T(t+2) | ...
+// S^T/P^T live in one pair of tensor-memory regions, dP^T/dS^T in another; the group that
+// overwrites a region is issued right after the group that last read it, and while the pipe
+// runs the two groups of the other region the 256 element-wise threads turn S^T into P^T (or
+// dP^T into dS^T).  N = 64 for every product (an MMA costs the same ~50 clocks for N = 32), so a
+// 64 x 128 tile takes 96 MMAs where two 32-row tiles took 144.
+//   tensor memory: K' hi|lo 0-127, dK 128-191, dV 192-255, S^T -> P^T_hi 256-319, P^T_lo 320-383,
+//                  dP^T -> dS^T_hi 384-447, dS^T_lo 448-511
+//   shared memory: V (128 keys, K-major, resident) 64 KB; one 32 KB buffer each for the query
+//                  tile's Q and dO in the K-major layout (B of S^T, dP^T) and in the MN-major layout
+//                  (B of dK, dV); every buffer has its own full/empty barriers and is refilled as
+//                  soon as the one product that reads it has completed.
+constexpr int BT64 = 64;
+constexpr uint32_t kTile64 = 2u * 2u * BT64 * 128u;   // one 64-row tile in one layout (32 KB)
+constexpr uint32_t kDkvSmem = 1024u + kResBytes + 4u * kTile64 + 256u;
+__device__ __forceinline__ constexpr uint32_t mn64_off(int ks, bool lo) { return (lo ? BT64 * 128u : 0u) + (uint32_t)ks * 1024u; }
+__device__ __forceinline__ DescBase mn64_base(uint32_t tile) { return make_desc_base(tile, 2u * BT64 * 128u, 512u, 1u); }
 
 __global__ void __launch_bounds__(kThreads, 1)
 attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_constant__ CUtensorMap tmQm,
@@ -203,23 +220,12 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     extern __shared__ uint8_t smem_raw[];
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t v_s = base;                                  // resident V (A operand of dP^T)
-    auto qk_s = [&](int st) { return base + kResBytes + (uint32_t)st * 4u * kTileBytes; };
-    auto dok_s = [&](int st) { return qk_s(st) + kTileBytes; };
-    auto qm_s = [&](int st) { return qk_s(st) + 2u * kTileBytes; };
-    auto dom_s = [&](int st) { return qk_s(st) + 3u * kTileBytes; };
-    const uint32_t bars = base + kResBytes + 8u * kTileBytes;
-    // count-1 barriers: 0 v_full, 1-2 kfull, 3-4 kempty, 5-6 mfull, 7-8 mempty, 9-10 sdp_full, 11 acc_full
-    const uint32_t v_full = bars;
-    auto kfull = [&](int s) { return bars + 8u * (1 + s); };
-    auto kempty = [&](int s) { return bars + 8u * (3 + s); };
-    auto mfull = [&](int s) { return bars + 8u * (5 + s); };
-    auto mempty = [&](int s) { return bars + 8u * (7 + s); };
-    auto sdp_full = [&](int b) { return bars + 8u * (9 + b); };
-    const uint32_t acc_full = bars + 8u * 11;
-    // count-4 barriers: 12-13 pds_full, 14 k_ready
-    auto pds_full = [&](int b) { return bars + 8u * (12 + b); };
-    const uint32_t k_ready = bars + 8u * 14;
-    const uint32_t tmem_slot = bars + 8u * 15;
+    const uint32_t qk_s = base + kResBytes, dok_s = qk_s + kTile64, dom_s = dok_s + kTile64, qm_s = dom_s + kTile64;
+    const uint32_t bars = qm_s + kTile64;
+    enum { V_FULL = 0, QK_FULL, QK_EMPTY, DOK_FULL, DOK_EMPTY, DOM_FULL, DOM_EMPTY, QM_FULL, QM_EMPTY, S_FULL,
+           DP_FULL, ACC_FULL, P_READY, DS_READY, K_READY, N_BARS };
+    auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+    const uint32_t tmem_slot = bars + 8u * N_BARS;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // grid = (sequence x head, key block): blocks are dispatched x-fastest, so all the key blocks
@@ -227,7 +233,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     const int b = blockIdx.x / g.H, h = blockIdx.x % g.H;
     const int j0 = blockIdx.y * BR;
     const int row_base = b * g.T;
-    const int n_qt = (g.T + BT_ - 1) / BT_, qt0 = j0 / BT_;
+    const int n_qt = (g.T + BT64 - 1) / BT64, qt0 = j0 / BT64;
     const int n_t = n_qt - qt0;
     if (threadIdx.x == 0) {
         trace_cta(g.trace, 0, 0, globaltimer_ns());
@@ -235,113 +241,140 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
         trace_cta(g.trace, 0, 3, n_t);
     }
 
-    const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp);
+    if (threadIdx.x == 0) {
+        for (int i = 0; i < P_READY; ++i) mbar_init(bar(i), 1);
+        mbar_init(bar(P_READY), 8);      // both element-wise warpgroups (8 warps) write every tile
+        mbar_init(bar(DS_READY), 8);
+        mbar_init(bar(K_READY), 4);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
     pdl_wait();      // set-up done; global memory is touched from here on
     pdl_trigger();
-    // TMEM columns
     const uint32_t tK_hi = tmem, tK_lo = tmem + 64, tdK = tmem + 128, tdV = tmem + 192;
-    auto tbuf = [&](int bb) { return tmem + 256u + 128u * (uint32_t)bb; };  // +0 S^T|P^T_hi, +32 P^T_lo, +64 dP^T|dS^T_hi, +96 dS^T_lo
+    const uint32_t tS = tmem + 256, tPlo = tmem + 320, tdP = tmem + 384, tdSlo = tmem + 448;
+    // tile t of the walk is query tile n_qt - 1 - t: from the last query tile down to the diagonal
+    // (the tensor core adds into its FP32 accumulator with truncation; adding the small far-away
+    // terms first keeps the drift of a long accumulation relative to a small sum)
+    auto q_row0 = [&](int t) { return (n_qt - 1 - t) * BT64; };
 
     if (warp == 0) {
         if (lane == 0) {
-            mbar_expect_tx(v_full, kResBytes);
+            mbar_expect_tx(bar(V_FULL), kResBytes);
             for (int kb = 0; kb < 2; ++kb)
-                tma_load_3d(v_s + kb * (kResBytes / 2), &tmVres, v_full, 2 * g.C + h * HD + kb * 32, row_base + j0, 0);
+                tma_load_3d(v_s + kb * (kResBytes / 2), &tmVres, bar(V_FULL), 2 * g.C + h * HD + kb * 32, row_base + j0, 0);
             bool ok = true;
+            // one buffer per (tensor, layout); t = the tile whose data goes in
+            auto load = [&](uint32_t dst, const CUtensorMap* tm, int full, int empty, int t) -> bool {
+                if (!mbar_wait(bar(empty), (uint32_t)(t & 1) ^ 1u, g.err, 21)) return false;
+                mbar_expect_tx(bar(full), kTile64);
+                for (int part = 0; part < 2; ++part)
+                    tma_load_3d(dst + part * (kTile64 / 2), tm, bar(full), h * HD + part * 32, row_base + q_row0(t), 0);
+                return true;
+            };
+            // in the order the products consume them: S^T(0), dP^T(0), then per tile dV(t), S^T(t+1), dK(t), dP^T(t+1)
+            if (n_t > 0) ok = load(qk_s, &tmQk, QK_FULL, QK_EMPTY, 0) && load(dok_s, &tmDOk, DOK_FULL, DOK_EMPTY, 0);
             for (int t = 0; t < n_t && ok; ++t) {
-                const int st = t & 1, q0 = (n_qt - 1 - t) * BT_;   // walk from the last query tile down to the diagonal
-                const uint32_t ph = (t >> 1) & 1u;
-                if (!mbar_wait(kempty(st), ph ^ 1u, g.err, 21)) { ok = false; break; }
-                mbar_expect_tx(kfull(st), 2u * kTileBytes);
-                for (int kb = 0; kb < 2; ++kb) {
-                    tma_load_3d(qk_s(st) + kb * (kTileBytes / 2), &tmQk, kfull(st), h * HD + kb * 32, row_base + q0, 0);
-                    tma_load_3d(dok_s(st) + kb * (kTileBytes / 2), &tmDOk, kfull(st), h * HD + kb * 32, row_base + q0, 0);
-                }
-                if (!mbar_wait(mempty(st), ph ^ 1u, g.err, 22)) { ok = false; break; }
-                mbar_expect_tx(mfull(st), 2u * kTileBytes);
-                for (int grp = 0; grp < 2; ++grp) {
-                    tma_load_3d(qm_s(st) + grp * (kTileBytes / 2), &tmQm, mfull(st), h * HD + grp * 32, row_base + q0, 0);
-                    tma_load_3d(dom_s(st) + grp * (kTileBytes / 2), &tmDOm, mfull(st), h * HD + grp * 32, row_base + q0, 0);
-                }
+                ok = load(dom_s, &tmDOm, DOM_FULL, DOM_EMPTY, t);
+                if (ok && t + 1 < n_t) ok = load(qk_s, &tmQk, QK_FULL, QK_EMPTY, t + 1);
+                if (ok) ok = load(qm_s, &tmQm, QM_FULL, QM_EMPTY, t);
+                if (ok && t + 1 < n_t) ok = load(dok_s, &tmDOk, DOK_FULL, DOK_EMPTY, t + 1);
             }
             if (!ok)
                 for (int i = 0; i < 2000; ++i) __nanosleep(1000);
         }
     } else if (warp == 1) {
         if (lane == 0) {
-            constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT_, false, false);   // 128 x 32, B K-major
+            constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT64, false, false);  // 128 x 64, B K-major
             constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
-            bool ok = mbar_wait(v_full, 0, g.err, 23) && mbar_wait(k_ready, 0, g.err, 24);
+            bool ok = mbar_wait(bar(V_FULL), 0, g.err, 23) && mbar_wait(bar(K_READY), 0, g.err, 24);
             int tn = 0;
-            const DescBase vd = kmaj_base(v_s);
-            auto issue_a = [&](int t) -> bool {
-                const int st = t & 1, bb = t & 1;
-                trace_mark(g.trace, 0, tn, 100 + t);
-                if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 25)) return false;
-                trace_mark(g.trace, 0, tn, 200 + t);
+            const DescBase vd = kmaj_base(v_s), qd = kmaj_base(qk_s), od = kmaj_base(dok_s);
+            const DescBase omd = mn64_base(dom_s), qmd = mn64_base(qm_s);
+            auto issue_s = [&](int t) -> bool {      // S^T(t) = K' Q^T
+                if (!mbar_wait(bar(QK_FULL), (uint32_t)(t & 1), g.err, 25)) return false;
                 tc_fence_after();
-                const uint32_t dS = tbuf(bb), dP = tbuf(bb) + 64u;
-                const DescBase qd = kmaj_base(qk_s(st)), od = kmaj_base(dok_s(st));
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t q_hi = qd.at(kmaj_off(BT_, ks, false)), q_lo = qd.at(kmaj_off(BT_, ks, true));
-                    umma_tf32_ts(dS, tK_lo + ks * 8, q_hi, idesc_a, ks > 0 ? 1u : 0u);
-                    umma_tf32_ts(dS, tK_hi + ks * 8, q_lo, idesc_a, 1u);
-                    umma_tf32_ts(dS, tK_hi + ks * 8, q_hi, idesc_a, 1u);
+                    const uint64_t q_hi = qd.at(kmaj_off(BT64, ks, false)), q_lo = qd.at(kmaj_off(BT64, ks, true));
+                    umma_tf32_ts(tS, tK_lo + ks * 8, q_hi, idesc_a, ks > 0 ? 1u : 0u);
+                    umma_tf32_ts(tS, tK_hi + ks * 8, q_lo, idesc_a, 1u);
+                    umma_tf32_ts(tS, tK_hi + ks * 8, q_hi, idesc_a, 1u);
                 }
+                umma_commit(bar(QK_EMPTY));
+                umma_commit(bar(S_FULL));
+                trace_mark(g.trace, 0, tn, 100 + t);
+                return true;
+            };
+            auto issue_dp = [&](int t) -> bool {     // dP^T(t) = V dO^T
+                if (!mbar_wait(bar(DOK_FULL), (uint32_t)(t & 1), g.err, 26)) return false;
+                tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t v_hi = vd.at(kmaj_off(BR, ks, false)), v_lo = vd.at(kmaj_off(BR, ks, true));
-                    const uint64_t o_hi = od.at(kmaj_off(BT_, ks, false)), o_lo = od.at(kmaj_off(BT_, ks, true));
-                    umma_tf32(dP, v_lo, o_hi, idesc_a, ks > 0 ? 1u : 0u);
-                    umma_tf32(dP, v_hi, o_lo, idesc_a, 1u);
-                    umma_tf32(dP, v_hi, o_hi, idesc_a, 1u);
+                    const uint64_t o_hi = od.at(kmaj_off(BT64, ks, false)), o_lo = od.at(kmaj_off(BT64, ks, true));
+                    umma_tf32(tdP, v_lo, o_hi, idesc_a, ks > 0 ? 1u : 0u);
+                    umma_tf32(tdP, v_hi, o_lo, idesc_a, 1u);
+                    umma_tf32(tdP, v_hi, o_hi, idesc_a, 1u);
                 }
-                umma_commit(kempty(st));
-                umma_commit(sdp_full(bb));
+                umma_commit(bar(DOK_EMPTY));
+                umma_commit(bar(DP_FULL));
+                trace_mark(g.trace, 0, tn, 200 + t);
+                return true;
+            };
+            auto issue_dv = [&](int t) -> bool {     // dV += P^T(t) dO
+                if (!mbar_wait(bar(P_READY), (uint32_t)(t & 1), g.err, 27)) return false;
+                if (!mbar_wait(bar(DOM_FULL), (uint32_t)(t & 1), g.err, 28)) return false;
+                tc_fence_after();
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t o_hi = omd.at(mn64_off(ks, false)), o_lo = omd.at(mn64_off(ks, true));
+                    const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
+                    umma_tf32_ts(tdV, tPlo + ks * 8, o_hi, idesc_b, acc);
+                    umma_tf32_ts(tdV, tS + ks * 8, o_lo, idesc_b, 1u);
+                    umma_tf32_ts(tdV, tS + ks * 8, o_hi, idesc_b, 1u);
+                }
+                umma_commit(bar(DOM_EMPTY));
                 trace_mark(g.trace, 0, tn, 300 + t);
                 return true;
             };
-            auto issue_b = [&](int t) -> bool {
-                const int st = t & 1, bb = t & 1;
-                if (!mbar_wait(pds_full(bb), (t >> 1) & 1u, g.err, 26)) return false;
-                trace_mark(g.trace, 0, tn, 400 + t);
-                if (!mbar_wait(mfull(st), (t >> 1) & 1u, g.err, 27)) return false;
-                trace_mark(g.trace, 0, tn, 500 + t);
+            auto issue_dk = [&](int t) -> bool {     // dK += dS^T(t) Q
+                if (!mbar_wait(bar(DS_READY), (uint32_t)(t & 1), g.err, 29)) return false;
+                if (!mbar_wait(bar(QM_FULL), (uint32_t)(t & 1), g.err, 30)) return false;
                 tc_fence_after();
-                const uint32_t p_hi = tbuf(bb), p_lo = tbuf(bb) + 32u, s_hi = tbuf(bb) + 64u, s_lo = tbuf(bb) + 96u;
-                const DescBase omd = mnmaj_base(dom_s(st)), qmd = mnmaj_base(qm_s(st));
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t o_hi = omd.at(mnmaj_off(ks, false)), o_lo = omd.at(mnmaj_off(ks, true));
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint64_t q_hi = qmd.at(mn64_off(ks, false)), q_lo = qmd.at(mn64_off(ks, true));
                     const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
-                    umma_tf32_ts(tdV, p_lo + ks * 8, o_hi, idesc_b, acc);
-                    umma_tf32_ts(tdV, p_hi + ks * 8, o_lo, idesc_b, 1u);
-                    umma_tf32_ts(tdV, p_hi + ks * 8, o_hi, idesc_b, 1u);
+                    umma_tf32_ts(tdK, tdSlo + ks * 8, q_hi, idesc_b, acc);
+                    umma_tf32_ts(tdK, tdP + ks * 8, q_lo, idesc_b, 1u);
+                    umma_tf32_ts(tdK, tdP + ks * 8, q_hi, idesc_b, 1u);
                 }
-#pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t q_hi = qmd.at(mnmaj_off(ks, false)), q_lo = qmd.at(mnmaj_off(ks, true));
-                    const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
-                    umma_tf32_ts(tdK, s_lo + ks * 8, q_hi, idesc_b, acc);
-                    umma_tf32_ts(tdK, s_hi + ks * 8, q_lo, idesc_b, 1u);
-                    umma_tf32_ts(tdK, s_hi + ks * 8, q_hi, idesc_b, 1u);
-                }
-                umma_commit(mempty(st));
-                trace_mark(g.trace, 0, tn, 600 + t);
+                umma_commit(bar(QM_EMPTY));
+                trace_mark(g.trace, 0, tn, 400 + t);
                 return true;
             };
-            if (ok && n_t > 0) ok = issue_a(0);
+            if (ok && n_t > 0) ok = issue_s(0) && issue_dp(0);
             for (int t = 0; t < n_t && ok; ++t) {
-                if (t + 1 < n_t) ok = issue_a(t + 1);
-                if (ok) ok = issue_b(t);
+                ok = issue_dv(t);                              // frees the S^T / P^T regions ...
+                if (ok && t + 1 < n_t) ok = issue_s(t + 1);    // ... which the next scores overwrite
+                if (ok) ok = issue_dk(t);                      // frees the dP^T / dS^T regions ...
+                if (ok && t + 1 < n_t) ok = issue_dp(t + 1);   // ... which the next dP^T overwrites
             }
-            if (ok) umma_commit(acc_full);
+            if (ok) umma_commit(bar(ACC_FULL));
         }
     } else {
-        const int wg = (warp - 2) >> 2;                   // 0 or 1: takes tiles t with (t & 1) == wg, buffer wg
+        const int wg = (warp - 2) >> 2;                   // 0 or 1: columns (query rows) 32 wg .. 32 wg + 31 of every tile
         const int lane_group = warp & 3;
-        const int etid = lane_group * 32 + lane;          // 0..127: row owned inside the CTA
+        const int etid = lane_group * 32 + lane;          // 0..127: key row owned inside the CTA
         const int key = j0 + etid;
         const uint32_t t_lane = ((uint32_t)(lane_group * 32) << 16);
         const float scale = 1.0f / sqrtf((float)HD);
@@ -352,55 +385,63 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             row_to_tmem(g.qkv_hi + off, g.qkv_hi + g.qkv_plane + off, scale * kLog2e, tK_hi + t_lane, tK_lo + t_lane);
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(k_ready);
+            if (lane == 0) mbar_arrive(bar(K_READY));
         }
         bool ok = true;
         int tn = 0;
-        const uint32_t tb = tbuf(wg) + t_lane;
-        for (int t = wg; t < n_t && ok; t += 2) {
-            const int q0 = (n_qt - 1 - t) * BT_;
-            // per-column softmax statistics of this query tile (same addresses in every thread:
+        const uint32_t c0 = 32u * (uint32_t)wg;
+        for (int t = 0; t < n_t && ok; ++t) {
+            const int q0 = q_row0(t) + 32 * wg;
+            // softmax statistics of this warpgroup's 32 query rows (same addresses in every thread:
             // broadcast loads, issued before the wait so their latency is hidden); rows past the
             // sequence end are clamped here and masked below
-            const int nvalid = min(BT_, g.T - q0);
-            const float* lse_t = g.lse + lb + q0;
-            const float* d_t = g.dvec + lb + q0;
+            const int nvalid = min(32, g.T - q0);
             float Lc[32], Dc[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-                const int ic = min(i, nvalid - 1);
-                Lc[i] = __ldg(lse_t + ic) * kLog2e;
-                Dc[i] = __ldg(d_t + ic);
+                const int r = min(q0 + i, g.T - 1);     // clamped: rows past the end are masked below
+                Lc[i] = __ldg(g.lse + lb + r) * kLog2e;
+                Dc[i] = __ldg(g.dvec + lb + r);
             }
             if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 700 + t);
-            if (!mbar_wait_warp(sdp_full(wg), (t >> 1) & 1u, g.err, 28)) { ok = false; break; }
-            if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 800 + t);
+            if (!mbar_wait_warp(bar(S_FULL), (uint32_t)(t & 1), g.err, 31)) { ok = false; break; }
             tc_fence_after();
-            uint32_t s[32], dp[32];
-            tmem_ld32(tb, s);
-            tmem_ld32(tb + 64u, dp);
+            uint32_t s[32];
+            tmem_ld32(tS + t_lane + c0, s);
             tmem_ld_wait();
-            if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 900 + t);
-            uint32_t p_hi[32], p_lo[32];
+            float p[32];
+            uint32_t lo[32];
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const bool live = (i < nvalid) && (q0 + i >= key);   // in the sequence and not before this key
-                const float p = live ? ex2_approx(__uint_as_float(s[i]) - Lc[i]) : 0.f;
-                const float ds = p * (__uint_as_float(dp[i]) - Dc[i]);
-                split_tf32_int(p, p_hi[i], p_lo[i]);
-                split_tf32_int(ds, s[i], dp[i]);                     // reuse: dS^T hi, lo
+                p[i] = live ? ex2_approx(__uint_as_float(s[i]) - Lc[i]) : 0.f;
+                split_tf32_int(p[i], s[i], lo[i]);
             }
-            tmem_st32(tb, p_hi);
-            tmem_st32(tb + 32u, p_lo);
-            tmem_st32(tb + 64u, s);
-            tmem_st32(tb + 96u, dp);
+            tmem_st32(tS + t_lane + c0, s);          // P^T hi over S^T
+            tmem_st32(tPlo + t_lane + c0, lo);
             tmem_st_wait();
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive(pds_full(wg));
-            if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 1000 + t);
+            if (lane == 0) mbar_arrive(bar(P_READY));
+            if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 800 + t);
+            if (!mbar_wait_warp(bar(DP_FULL), (uint32_t)(t & 1), g.err, 32)) { ok = false; break; }
+            tc_fence_after();
+            tmem_ld32(tdP + t_lane + c0, s);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) {
+                const float ds = p[i] * (__uint_as_float(s[i]) - Dc[i]);
+                split_tf32_int(ds, s[i], lo[i]);
+            }
+            tmem_st32(tdP + t_lane + c0, s);         // dS^T hi over dP^T
+            tmem_st32(tdSlo + t_lane + c0, lo);
+            tmem_st_wait();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(bar(DS_READY));
+            if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 900 + t);
         }
-        if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 29);
+        if (ok) ok = mbar_wait_warp(bar(ACC_FULL), 0, g.err, 33);
         if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
             tc_fence_after();
             const bool valid = key < g.T;
@@ -681,21 +722,19 @@ cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, cons
         if (e != cudaSuccess) return e;
     }
     const int64_t rows = (int64_t)B * T;
-    CUtensorMap qk32, qm32, dok32, dom32, vres, kres_unused, dores;
-    (void)kres_unused;
-    bool ok = enc3(&qk32, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BT_, false) &&   // 32-row K-major tiles of qkv
-              enc3(&qm32, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BT_, true) &&    // 32-row MN-major tiles of qkv
-              enc3(&dok32, do_hi, C, rows, do_plane, BT_, false) && enc3(&dom32, do_hi, C, rows, do_plane, BT_, true) &&
+    CUtensorMap dok64, dom64, vres, dores;
+    bool ok = enc3(&dok64, do_hi, C, rows, do_plane, BT64, false) &&                // 64-row K-major / MN-major tiles of dO
+              enc3(&dom64, do_hi, C, rows, do_plane, BT64, true) &&
               enc3(&vres, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BR, false) &&    // 128-row resident tiles
               enc3(&dores, do_hi, C, rows, do_plane, BR, false);
     CUtensorMap qk64, qm64;
-    ok = ok && enc3(&qk64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, false) &&  // 64-row tiles for the dq kernel
+    ok = ok && enc3(&qk64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, false) &&  // 64-row K-major / MN-major tiles of qkv
          enc3(&qm64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, true);
     if (!ok) return cudaErrorInvalidValue;
     BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dqkv_hi, dqkv_plane, err_word, attention_tc_get_trace(), rg_sums,
               4 * ((T + BR - 1) / BR)};
     dim3 gk(B * H, (T + BR - 1) / BR);
-    BT_KERNEL_LAUNCH((attn_bwd_dkv_tc_kernel), gk, kThreads, kDkvSmem, s, qk32, qm32, dok32, dom32, vres, g);
+    BT_KERNEL_LAUNCH((attn_bwd_dkv_tc_kernel), gk, kThreads, kDkvSmem, s, qk64, qm64, dok64, dom64, vres, g);
     BT_COUNT_LAUNCH();
     BT_KERNEL_LAUNCH((attn_bwd_dq_tc_kernel), gk, kThreads, kDqSmem, s, qk64, qm64, qk64, dores, g);
     BT_COUNT_LAUNCH();
