@@ -327,17 +327,22 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 m = mm;
 #pragma unroll
                 for (int i = 0; i < HD; ++i) o_reg[i] = o_reg[i] * f0 + src[i] * f1;
-                if (row < g.T) {
-                    const float inv = 1.0f / l;
-                    const int64_t off = ((int64_t)(row_base + row)) * g.C + h * HD;
+                // the rows leave in full 128-byte segments through a slice of the idle V buffers
+                const float inv = 1.0f / l;
+                const int wrow0 = q0 + lane_group * 32;                 // first query row of this warp
+                const int nvalid = max(0, min(32, g.T - wrow0));
+                const int64_t off0 = ((int64_t)(row_base + wrow0)) * g.C + h * HD;
+                float* tile = reinterpret_cast<float*>(smem_raw + (v_s - smem_u32(smem_raw)) + (uint32_t)lane_group * kRowTileBytes);
 #pragma unroll
-                    for (int i = 0; i < HD; i += 4) {
-                        float4 v = make_float4(o_reg[i] * inv, o_reg[i + 1] * inv, o_reg[i + 2] * inv, o_reg[i + 3] * inv);
-                        store_raw_split(v, g.o ? g.o + off : nullptr, g.o_hi ? g.o_hi + off : nullptr,
-                                        g.o_lo ? g.o_lo + off : nullptr, i / 4);
-                    }
-                    if (g.lse) g.lse[((int64_t)b * g.H + h) * g.T + row] = (m * c + log2f(l)) * kLn2;
+                for (int half = 0; half < 2; ++half) {
+                    float v[32];
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) v[i] = o_reg[half * 32 + i] * inv;
+                    warp_rows_store(v, tile, lane, nvalid, g.o ? g.o + off0 + half * 32 : nullptr,
+                                    g.o_hi ? g.o_hi + off0 + half * 32 : nullptr, g.o_lo ? g.o_lo + off0 + half * 32 : nullptr,
+                                    g.C, nullptr);
                 }
+                if (row < g.T && g.lse) g.lse[((int64_t)b * g.H + h) * g.T + row] = (m * c + log2f(l)) * kLn2;
             }
         }
     }

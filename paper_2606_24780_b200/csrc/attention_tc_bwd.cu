@@ -88,28 +88,13 @@ __device__ __forceinline__ void row_to_tmem(const float* hi_row, const float* lo
     tmem_st_wait();
 }
 
-// Column sums over the 32 rows a warp owns: v[i] is column i of this lane's row; the result is the
-// sum of column `lane` over the 32 lanes (a halving butterfly: 31 shuffles, fixed order).
-__device__ __forceinline__ float warp_colsum32(float (&v)[32], int lane) {
-#pragma unroll
-    for (int off = 16; off >= 1; off >>= 1) {
-        const bool upper = (lane & off) != 0;
-#pragma unroll
-        for (int i = 0; i < off; ++i) {
-            const float send = upper ? v[i] : v[i + off];
-            const float keep = upper ? v[i + off] : v[i];
-            v[i] = keep + __shfl_xor_sync(0xffffffffu, send, off);
-        }
-    }
-    return v[0];
-}
-
-// Thread-owned accumulator row (64 tensor-memory columns) * mul -> hi/lo planes in global memory.
-// The tensor-memory loads are .sync.aligned: EVERY lane of the warp must call this; `store` says
-// whether this lane's row exists (rows past the end of the sequence are read and dropped).
-// sums (nullable): 64 floats that receive the column sums over the warp's existing rows.
-__device__ __forceinline__ void tmem_row_to_split(uint32_t t_row, float mul, float* hi_row, float* lo_row,
-                                                  bool store, float* sums, int lane) {
+// The 64 accumulator columns of the warp's 32 rows (times mul) -> hi/lo planes in global memory,
+// in full 128-byte row segments (see warp_rows_store).  The tensor-memory loads are .sync.aligned:
+// EVERY lane of the warp must call this.  hi0 / lo0: row 0 of the warp, column 0 of the head;
+// nvalid: rows of the warp inside the sequence; sums (nullable): 64 column sums over those rows.
+__device__ __forceinline__ void tmem_rows_to_split(uint32_t t_row, float mul, float* hi0, float* lo0,
+                                                   long long row_stride, int nvalid, float* sums, float* tile,
+                                                   int lane) {
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
         uint32_t r[32];
@@ -117,20 +102,9 @@ __device__ __forceinline__ void tmem_row_to_split(uint32_t t_row, float mul, flo
         tmem_ld_wait();
         float v[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = store ? __uint_as_float(r[i]) * mul : 0.f;
-        if (store) {
-#pragma unroll
-            for (int i = 0; i < 32; i += 4) {
-                float4 h, l;
-                split_tf32(make_float4(v[i], v[i + 1], v[i + 2], v[i + 3]), h, l);
-                *reinterpret_cast<float4*>(hi_row + half * 32 + i) = h;
-                *reinterpret_cast<float4*>(lo_row + half * 32 + i) = l;
-            }
-        }
-        if (sums) {   // warp-uniform
-            const float t = warp_colsum32(v, lane);
-            sums[half * 32 + lane] = t;
-        }
+        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * mul;
+        warp_rows_store(v, tile, lane, nvalid, nullptr, hi0 + half * 32, lo0 + half * 32, row_stride,
+                        sums ? sums + half * 32 : nullptr);
     }
 }
 
@@ -444,15 +418,17 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
         if (ok) ok = mbar_wait_warp(bar(ACC_FULL), 0, g.err, 33);
         if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
             tc_fence_after();
-            const bool valid = key < g.T;
-            const int64_t off = (int64_t)(row_base + (valid ? key : 0)) * gs + h * HD;
-            float* hi = g.dqkv_hi + off;
+            const int wrow0 = j0 + lane_group * 32;                    // first key row of this warp
+            const int nvalid = max(0, min(32, g.T - wrow0));
+            float* hi = g.dqkv_hi + (int64_t)(row_base + wrow0) * gs + h * HD;   // dereferenced for valid rows only
             float* lo = hi + g.dqkv_plane;
             float* sums = g.rg_sums
                               ? g.rg_sums + ((int64_t)b * g.nrg + (j0 >> 5) + lane_group) * gs + h * HD
                               : nullptr;
-            if (wg == 0) tmem_row_to_split(tdK + t_lane, scale, hi + g.C, lo + g.C, valid, sums ? sums + g.C : nullptr, lane);
-            else tmem_row_to_split(tdV + t_lane, 1.0f, hi + 2 * g.C, lo + 2 * g.C, valid, sums ? sums + 2 * g.C : nullptr, lane);
+            // the streamed-tile buffers are idle by now: each warp stages its rows in a slice of them
+            float* tile = reinterpret_cast<float*>(smem_raw + (qk_s - smem_u32(smem_raw)) + (uint32_t)(warp - 2) * kRowTileBytes);
+            if (wg == 0) tmem_rows_to_split(tdK + t_lane, scale, hi + g.C, lo + g.C, gs, nvalid, sums ? sums + g.C : nullptr, tile, lane);
+            else tmem_rows_to_split(tdV + t_lane, 1.0f, hi + 2 * g.C, lo + 2 * g.C, gs, nvalid, sums ? sums + 2 * g.C : nullptr, tile, lane);
         }
     }
     tc_fence_before();
@@ -665,12 +641,14 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 39);
             if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
                 tc_fence_after();
-                const int64_t off = (int64_t)(row_base + rc) * gs + h * HD;
+                const int wrow0 = q0 + lane_group * 32;                // first query row of this warp
+                const int nvalid = max(0, min(32, g.T - wrow0));
+                float* hi = g.dqkv_hi + (int64_t)(row_base + wrow0) * gs + h * HD;
                 float* sums = g.rg_sums
                                   ? g.rg_sums + ((int64_t)b * g.nrg + (q0 >> 5) + lane_group) * gs + h * HD
                                   : nullptr;
-                tmem_row_to_split(tdQ + t_lane, scale, g.dqkv_hi + off, g.dqkv_hi + g.dqkv_plane + off, row < g.T, sums,
-                                  lane);
+                float* tile = reinterpret_cast<float*>(smem_raw + (kk_s(0) - smem_u32(smem_raw)) + (uint32_t)(warp - 2) * kRowTileBytes);
+                tmem_rows_to_split(tdQ + t_lane, scale, hi, hi + g.dqkv_plane, gs, nvalid, sums, tile, lane);
             }
         }
     }

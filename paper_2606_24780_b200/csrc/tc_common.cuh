@@ -6,6 +6,8 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include "common.cuh"
+
 namespace bt {
 namespace tc {
 
@@ -176,6 +178,52 @@ __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.
 __host__ __device__ constexpr uint32_t make_idesc_tf32(int m, int n, bool a_mn_major, bool b_mn_major) {
     return (1u << 4) | (2u << 7) | (2u << 10) | ((a_mn_major ? 1u : 0u) << 15) | ((b_mn_major ? 1u : 0u) << 16) |
            ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
+// ---------------------------------------------------------------- row-owner results -> global memory
+// In the attention kernels a thread owns a row (its tensor-memory lane).  Written straight out,
+// one warp store would touch 32 rows x 16 bytes; instead the warp's 32 x 32 chunk goes through a
+// shared-memory tile (144-byte pitch: conflict-free both ways) and leaves as full 128-byte row
+// segments: lane -> rows (lane >> 3) + 4 i, columns 4 (lane & 7) .. + 3.
+//   v        this lane's 32 columns of the chunk (lane = row inside the warp's 32 rows)
+//   tile     the warp's own 32 x 144-byte shared-memory tile
+//   nvalid   how many of the warp's 32 rows exist (rows >= nvalid are neither stored nor summed)
+//   raw/hi/lo  destination of row 0, column 0 of the chunk (any may be null); row_stride in floats
+//   sums     nullable: 32 floats receiving the column sums over the valid rows (fixed order)
+constexpr uint32_t kRowTilePitch = 144u;
+constexpr uint32_t kRowTileBytes = 32u * kRowTilePitch;
+__device__ __forceinline__ void warp_rows_store(const float (&v)[32], float* tile, int lane, int nvalid, float* raw,
+                                                float* hi, float* lo, long long row_stride, float* sums) {
+    float4* wr = reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(tile) + lane * kRowTilePitch);
+#pragma unroll
+    for (int q = 0; q < 8; ++q) wr[q] = make_float4(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
+    __syncwarp();
+    const int sub = lane >> 3, cq = lane & 7;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = sub + 4 * i;
+        if (r < nvalid) {
+            const float4 x = *reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(tile) + r * kRowTilePitch + cq * 16);
+            const long long off = (long long)r * row_stride + 4 * cq;
+            if (raw) *reinterpret_cast<float4*>(raw + off) = x;
+            if (hi) {
+                float4 h, l;
+                bt::split_tf32(x, h, l);
+                *reinterpret_cast<float4*>(hi + off) = h;
+                *reinterpret_cast<float4*>(lo + off) = l;
+            }
+            acc.x += x.x; acc.y += x.y; acc.z += x.z; acc.w += x.w;
+        }
+    }
+    if (sums) {   // warp-uniform
+        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, 8);  acc.y += __shfl_xor_sync(0xffffffffu, acc.y, 8);
+        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, 8);  acc.w += __shfl_xor_sync(0xffffffffu, acc.w, 8);
+        acc.x += __shfl_xor_sync(0xffffffffu, acc.x, 16); acc.y += __shfl_xor_sync(0xffffffffu, acc.y, 16);
+        acc.z += __shfl_xor_sync(0xffffffffu, acc.z, 16); acc.w += __shfl_xor_sync(0xffffffffu, acc.w, 16);
+        if (sub == 0) *reinterpret_cast<float4*>(sums + 4 * cq) = acc;
+    }
+    __syncwarp();   // the tile is rewritten by the next chunk
 }
 
 // ---------------------------------------------------------------- CTA pairs (cta_group::2)
