@@ -63,27 +63,48 @@ __device__ __forceinline__ unsigned smid() {
     return r;
 }
 
-// Thread-owned row (64 floats given as hi/lo planes) -> x * mul -> hi/lo columns of tensor memory.
-__device__ __forceinline__ void row_to_tmem(const float* hi_row, const float* lo_row, float mul, uint32_t t_hi,
-                                            uint32_t t_lo) {
+// The warp's 32 rows x 64 floats (given as hi/lo planes; row r of the warp at src + r * row_stride)
+// -> (hi + lo) * mul -> re-split -> hi/lo columns of tensor memory, lane = row.  The rows are read
+// the way they lie in memory (8 lanes x 16 bytes = one 128-byte row segment, all loads of a chunk in
+// flight together) and turned so that every lane ends up with its own row through the warp's
+// shared-memory tile.  Rows >= nvalid are read as the last valid row (their results are never used).
+__device__ __forceinline__ void rows_to_tmem(const float* src_hi, const float* src_lo, long long row_stride, int nvalid,
+                                             float mul, uint32_t t_hi, uint32_t t_lo, float* tile, int lane) {
+    const int sub = lane >> 3, cq = lane & 7;
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
-        uint32_t h[32], l[32];
+        float4 a[8], b[8];
 #pragma unroll
-        for (int i = 0; i < 32; i += 4) {
-            const float4 a = *reinterpret_cast<const float4*>(hi_row + half * 32 + i);
-            const float4 b = *reinterpret_cast<const float4*>(lo_row + half * 32 + i);
-            const float x[4] = {(a.x + b.x) * mul, (a.y + b.y) * mul, (a.z + b.z) * mul, (a.w + b.w) * mul};
+        for (int i = 0; i < 8; ++i) {
+            const int r = max(0, min(sub + 4 * i, nvalid - 1));
+            const long long off = (long long)r * row_stride + half * 32 + 4 * cq;
+            a[i] = *reinterpret_cast<const float4*>(src_hi + off);
+            b[i] = *reinterpret_cast<const float4*>(src_lo + off);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 x = make_float4((a[i].x + b[i].x) * mul, (a[i].y + b[i].y) * mul, (a[i].z + b[i].z) * mul,
+                                         (a[i].w + b[i].w) * mul);
+            *reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(tile) + (sub + 4 * i) * kRowTilePitch + cq * 16) = x;
+        }
+        __syncwarp();
+        uint32_t h[32], l[32];
+        const float4* rd = reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(tile) + lane * kRowTilePitch);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float4 x = rd[q];
+            const float xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
                 float fh, fl;
-                split_tf32(x[e], fh, fl);
-                h[i + e] = __float_as_uint(fh);
-                l[i + e] = __float_as_uint(fl);
+                split_tf32(xs[e], fh, fl);
+                h[4 * q + e] = __float_as_uint(fh);
+                l[4 * q + e] = __float_as_uint(fl);
             }
         }
         tmem_st32(t_hi + half * 32, h);
         tmem_st32(t_lo + half * 32, l);
+        __syncwarp();   // the tile is rewritten by the next half
     }
     tmem_st_wait();
 }
@@ -183,7 +204,7 @@ __device__ __forceinline__ uint32_t setup(uint32_t bars, int n_bars_count1, uint
 //                  soon as the one product that reads it has completed.
 constexpr int BT64 = 64;
 constexpr uint32_t kTile64 = 2u * 2u * BT64 * 128u;   // one 64-row tile in one layout (32 KB)
-constexpr uint32_t kDkvSmem = 1024u + kResBytes + 4u * kTile64 + 256u;
+constexpr uint32_t kDkvSmem = 1024u + kResBytes + 4u * kTile64 + 256u + 4u * kRowTileBytes;   // + K' staging tiles
 __device__ __forceinline__ constexpr uint32_t mn64_off(int ks, bool lo) { return (lo ? BT64 * 128u : 0u) + (uint32_t)ks * 1024u; }
 __device__ __forceinline__ DescBase mn64_base(uint32_t tile) { return make_desc_base(tile, 2u * BT64 * 128u, 512u, 1u); }
 
@@ -355,8 +376,11 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
         const int64_t gs = 3 * (int64_t)g.C;
         const int64_t lb = ((int64_t)b * g.H + h) * g.T;
         if (wg == 0) {   // K' = K * scale * log2(e) into tensor memory
-            const int64_t off = (int64_t)(row_base + min(key, g.T - 1)) * gs + g.C + h * HD;
-            row_to_tmem(g.qkv_hi + off, g.qkv_hi + g.qkv_plane + off, scale * kLog2e, tK_hi + t_lane, tK_lo + t_lane);
+            const int wrow0 = min(j0 + lane_group * 32, g.T - 1);
+            const int64_t off = (int64_t)(row_base + wrow0) * gs + g.C + h * HD;
+            float* tile = reinterpret_cast<float*>(smem_raw + (bars + 256u - smem_u32(smem_raw)) + (uint32_t)lane_group * kRowTileBytes);
+            rows_to_tmem(g.qkv_hi + off, g.qkv_hi + g.qkv_plane + off, gs, max(1, min(32, g.T - wrow0)), scale * kLog2e,
+                         tK_hi + t_lane, tK_lo + t_lane, tile, lane);
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(K_READY));
@@ -464,6 +488,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
     auto kk_s = [&](int st) { return base + kResBytes + (uint32_t)st * 2u * kTileQ; };
     auto vk_s = [&](int st) { return kk_s(st) + kTileQ; };
     const uint32_t km_s = base + kResBytes + 4u * kTileQ;       // single stage
+    const uint32_t qstage = km_s;                               // staging of the query rows before the first fill
     const uint32_t bars = base + kResBytes + 5u * kTileQ;
     // count-1: 0 do_full, 1-2 kfull, 3-4 kempty, 5 mfull, 7 mempty, 9-10 sdp_full, 11 acc_full
     const uint32_t do_full = bars;
@@ -518,6 +543,8 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             for (int t = 0; t < n_t && ok; ++t) {
                 if (t + 1 < n_t) ok = load_kmajor(t + 1);
                 if (!ok) break;
+                // the MN-major buffer doubles as the staging area of the query rows: first fill after that
+                if (t == 0 && !mbar_wait(q_ready, 0, g.err, 40)) { ok = false; break; }
                 if (!mbar_wait(mempty, (t & 1u) ^ 1u, g.err, 32)) { ok = false; break; }
                 mbar_expect_tx(mfull, kTileQ);
                 for (int grp = 0; grp < 2; ++grp)
@@ -599,8 +626,14 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
         const int64_t lb = ((int64_t)b * g.H + h) * g.T;
         const int rc = min(row, g.T - 1);
         if (wg == 0) {
-            const int64_t off = (int64_t)(row_base + rc) * gs + h * HD;
-            row_to_tmem(g.qkv_hi + off, g.qkv_hi + g.qkv_plane + off, scale * kLog2e, tQ_hi + t_lane, tQ_lo + t_lane);
+            // the MN-major K buffer is not filled before the first score products are under way: its
+            // first 18 KB stage the query rows on their way into tensor memory
+            const int wrow0 = min(q0 + lane_group * 32, g.T - 1);
+            const int64_t off = (int64_t)(row_base + wrow0) * gs + h * HD;
+            float* tile = reinterpret_cast<float*>(smem_raw + (qstage - smem_u32(smem_raw)) + (uint32_t)lane_group * kRowTileBytes);
+            rows_to_tmem(g.qkv_hi + off, g.qkv_hi + g.qkv_plane + off, gs, max(1, min(32, g.T - wrow0)), scale * kLog2e,
+                         tQ_hi + t_lane, tQ_lo + t_lane, tile, lane);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tile is next written by TMA
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(q_ready);
