@@ -369,7 +369,7 @@ BT_API bt_status bt_op_colsum(const float* x, int64_t N, int32_t C, float* out, 
  * sums live in a fixed array inside the library image: 98,304 floats (384 KB) that every GPU
  * loading the library holds until the process exits.  The call allocates nothing (no cudaMalloc,
  * cudaFree or allocating library routine) and returns BT_ERR_UNSUPPORTED when
- * bt_op_colsum_scratch_bytes(N, C) exceeds that size (roughly C > 22,000).
+ * bt_op_colsum_scratch_bytes(N, C) exceeds that size (C > 98,304).
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
  * that device current) and caches it; make that first call before starting any stream capture.
  * Every call on a device shares the one array and overwrites the part it uses, so calls that

@@ -558,7 +558,7 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
     const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
     // the tcgen05 attention kernels read qkv only as hi/lo planes; the raw copy is written only
     // for the kernels that need it
-    const bool raw_qkv = simt_attn || (C / H) != 64 || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
+    const bool raw_qkv = simt_attn || ((C / H) != 64 && (C / H) != 128) || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
 
     // hi/lo planes of every parameter (weights are GEMM operands; one streaming pass)
     BT_STEP(kCatSplit, 0, 20.0 * m->P, launch_split_matrices(m->params, m->wsplit, m->wsplit_t, m->P, m->mat_descs, m->n_mats,
@@ -614,7 +614,7 @@ extern "C" bt_status bt_backward(bt_model* m) {
     const int64_t N = (int64_t)B * T;
     const bool simt_attn = (m->cfg.flags & BT_FLAG_ATTN_SIMT) != 0;
     const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
-    const bool raw_qkv = simt_attn || (C / H) != 64 || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
+    const bool raw_qkv = simt_attn || ((C / H) != 64 && (C / H) != 128) || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
     auto G = [&](const Tensor& t) { return m->grads + t.off; };
 
     // LM head: dxf = dlogits . wte ; dwte = dlogits^T . xf
@@ -947,10 +947,10 @@ extern "C" bt_status bt_op_attention_fwd(const float* qkv, const float* qkv_spli
     int d = C / H;
     if (d != 16 && d != 32 && d != 64 && d != 128) return fail(BT_ERR_UNSUPPORTED, "attention: head_dim %d", d);
     const bool simt = (flags & BT_FLAG_ATTN_SIMT) != 0;
-    if (!qkv && (simt || d != 64))
+    if (!qkv && (simt || (d != 64 && d != 128)))
         return fail(BT_ERR_INVALID_ARG, "attention_fwd: this kernel needs the raw qkv array");
     int* err = nullptr;
-    if (qkv_split && d == 64 && !simt) {
+    if (qkv_split && (d == 64 || d == 128) && !simt) {
         char msg[256];
         if (!gemm_tc_init(msg, sizeof(msg))) return fail(BT_ERR_CUDA, "tensor-core attention unavailable: %s", msg);
         BT_CUDA(attention_tc_default_err(&err));
@@ -980,7 +980,7 @@ extern "C" bt_status bt_op_attention_bwd(const float* qkv, const float* qkv_spli
     if (scratch_bytes < (size_t)B * H * T * sizeof(float)) return fail(BT_ERR_OOM, "attention_bwd: scratch too small");
     if (!dqkv && !dqkv_split) return fail(BT_ERR_INVALID_ARG, "attention_bwd: no output requested");
     const bool simt = (flags & BT_FLAG_ATTN_SIMT) != 0;
-    const bool tc = !simt && qkv_split && d_o_split && dqkv_split && !dqkv && d == 64;
+    const bool tc = !simt && qkv_split && d_o_split && dqkv_split && !dqkv && (d == 64 || d == 128);
     if (!tc && (!qkv || !d_o)) return fail(BT_ERR_INVALID_ARG, "attention_bwd: this kernel needs the raw qkv and d_o arrays");
     int* err = nullptr;
     cudaStream_t s = (cudaStream_t)stream;

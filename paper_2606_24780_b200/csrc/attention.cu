@@ -1,5 +1,5 @@
-// Attention dispatch: tensor-core kernels by default, the FP32 FMA reference on request (and
-// for head_dim 128, which the tensor-core kernels are not instantiated for).
+// Attention dispatch: tcgen05 kernels for head_dim 64 and 128 when the inputs come as hi/lo
+// planes, warp-MMA kernels for head_dim 16 / 32 / 64 on raw inputs, the FP32 FMA reference on request.
 #include "common.cuh"
 
 namespace bt {
@@ -22,22 +22,30 @@ cudaError_t launch_attention_bwd_mma(const float* qkv, const float* lse, const f
                                      cudaStream_t s);
 
 bool attention_tc_supports(int head_dim, int C);
+bool attention_tc128_supports(int head_dim, int C);
+cudaError_t launch_attention_fwd_tc128(const float* qkv_hi, int64_t qkv_plane, int B, int T, int C, int H, float* o,
+                                       float* o_hi, float* o_lo, float* lse, int* err_word, cudaStream_t s);
+cudaError_t launch_attention_bwd_tc128(const float* qkv_hi, int64_t qkv_plane, const float* do_hi, int64_t do_plane,
+                                       const float* lse, const float* dvec, int B, int T, int C, int H, float* dqkv_hi,
+                                       int64_t dqkv_plane, float* rg_sums, int* err_word, cudaStream_t s);
 cudaError_t launch_attention_fwd_tc(const float* qkv_hi, int64_t qkv_plane, int B, int T, int C, int H, float* o,
                                     float* o_hi, float* o_lo, float* lse, int* err_word, cudaStream_t s);
 
 // qkv_hi (nullable): the same qkv as TF32 hi/lo planes (lo at qkv_hi + qkv_plane); with it and
-// head_dim 64 the tcgen05 kernel runs, otherwise the warp-MMA kernel on the raw array.
+// head_dim 64 or 128 the tcgen05 kernels run, otherwise the warp-MMA kernel on the raw array.
 cudaError_t launch_attention_fwd(const float* qkv, const float* qkv_hi, int64_t qkv_plane, int B, int T, int C, int H,
                                  float* o, float* o_hi, float* o_lo, float* lse, bool simt, int* err_word,
                                  cudaStream_t s) {
     if (!simt && qkv_hi && attention_tc_supports(C / H, C))
         return launch_attention_fwd_tc(qkv_hi, qkv_plane, B, T, C, H, o, o_hi, o_lo, lse, err_word, s);
+    if (!simt && qkv_hi && lse && attention_tc128_supports(C / H, C))
+        return launch_attention_fwd_tc128(qkv_hi, qkv_plane, B, T, C, H, o, o_hi, o_lo, lse, err_word, s);
     if (!qkv) return cudaErrorInvalidValue;
     if (simt || !attention_mma_supports(C / H)) return launch_attention_fwd_simt(qkv, B, T, C, H, o, o_hi, o_lo, lse, s);
     return launch_attention_fwd_mma(qkv, B, T, C, H, o, o_hi, o_lo, lse, s);
 }
 
-// Inputs may be given raw and/or as hi/lo planes (qkv_hi, do_hi; lo at +plane).  With head_dim 64,
+// Inputs may be given raw and/or as hi/lo planes (qkv_hi, do_hi; lo at +plane).  With head_dim 64 or 128,
 // both split inputs and only the split output requested, the tcgen05 kernels run; otherwise the
 // warp-MMA kernels run on the raw arrays.
 cudaError_t launch_attention_bwd(const float* qkv, const float* qkv_hi, int64_t qkv_plane, const float* o,
@@ -46,13 +54,17 @@ cudaError_t launch_attention_bwd(const float* qkv, const float* qkv_hi, int64_t 
                                  float* dqkv_lo, float* dvec, bool simt, int* err_word, cudaStream_t s,
                                  float* rg_sums, bool* rg_sums_written) {
     if (rg_sums_written) *rg_sums_written = false;
-    const bool tc = !simt && qkv_hi && do_hi && dqkv_hi && !dqkv && attention_tc_supports(C / H, C) &&
+    const bool tc128 = attention_tc128_supports(C / H, C);
+    const bool tc = !simt && qkv_hi && do_hi && dqkv_hi && !dqkv && (attention_tc_supports(C / H, C) || tc128) &&
                     dqkv_lo == dqkv_hi + (int64_t)B * T * 3 * C;
     if (tc) {
         cudaError_t e = d_o ? launch_attention_dvec(o, o_lo, d_o, nullptr, B, T, C, H, dvec, s)
                             : launch_attention_dvec(o, o_lo, do_hi, do_hi + do_plane, B, T, C, H, dvec, s);
         if (e != cudaSuccess) return e;
         if (rg_sums_written) *rg_sums_written = rg_sums != nullptr;
+        if (tc128)
+            return launch_attention_bwd_tc128(qkv_hi, qkv_plane, do_hi, do_plane, lse, dvec, B, T, C, H, dqkv_hi,
+                                              (int64_t)B * T * 3 * C, rg_sums, err_word, s);
         return launch_attention_bwd_tc(qkv_hi, qkv_plane, do_hi, do_plane, lse, dvec, B, T, C, H, dqkv_hi,
                                        (int64_t)B * T * 3 * C, rg_sums, err_word, s);
     }

@@ -275,7 +275,7 @@ cudaError_t launch_gelu_bwd(const float* x, const float* dy, int64_t n, int tanh
 // warp order.  Stage 2 adds the strips in strip order.
 static inline int colsum_strips(int64_t N, int C) {
     int cblocks = (C + 127) / 128;
-    int64_t strips = (4 * 148 + cblocks - 1) / cblocks;
+    int64_t strips = (4 * 148) / cblocks;  // 4 resident CTAs per SM: one wave
     int64_t max_strips = (N + 63) / 64;
     if (strips > max_strips) strips = max_strips;
     if (strips < 1) strips = 1;
@@ -403,8 +403,20 @@ __global__ void __launch_bounds__(256) gelu_bwd_colsum_kernel(const float* __res
 
 cudaError_t launch_gelu_bwd_colsum(const float* x, const float* dy, int64_t N, int C, int tanh_form, float* dx,
                                    float* dx_hi, float* dx_lo, float* colsum, float* scratch, cudaStream_t s) {
+    // One wave: no more strips than the CTAs that are resident at once (the kernel's register
+    // count decides that, so it is asked for), and never more than the scratch was sized for.
+    static int resident = 0;
+    if (resident == 0) {
+        int per_sm = 0, sms = 0, dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, gelu_bwd_colsum_kernel, 256, 0);
+        resident = (per_sm > 0 && sms > 0) ? per_sm * sms : 296;
+    }
     int C4 = C / 4, strips = colsum_strips(N, C);
-    dim3 grid((C4 + 31) / 32, strips);
+    const int cblocks = (C4 + 31) / 32;
+    if (strips * cblocks > resident && resident / cblocks >= 1) strips = resident / cblocks;
+    dim3 grid(cblocks, strips);
     BT_KERNEL_LAUNCH((gelu_bwd_colsum_kernel), grid, 256, 0, s, x, dy, N, C4, strips, tanh_form, dx, dx_hi, dx_lo, scratch);
     BT_COUNT_LAUNCH();
     BT_KERNEL_LAUNCH((colsum_stage2_kernel), (C4 + 31) / 32, 256, 0, s, scratch, strips, C4, colsum);

@@ -298,10 +298,15 @@ def test_attention_fwd_bwd(B, T, H, d, flags):
     check_split(dqs, host(dqkv))
 
 
-@pytest.mark.parametrize("B,T,H", [(2, 200, 3), (1, 1024, 2), (1, 1, 2), (3, 129, 1), (1, 130, 12), (2, 64, 1), (1, 65, 1)])
-def test_attention_fwd_tcgen05_kernel(B, T, H):
-    """head_dim 64 with the qkv array given as hi/lo planes: the TMA + tcgen05 + TMEM kernel."""
-    d = 64
+TC_ATTN_SHAPES = [(2, 200, 3, 64), (1, 1024, 2, 64), (1, 1, 2, 64), (3, 129, 1, 64), (1, 130, 12, 64), (2, 64, 1, 64),
+                  (1, 65, 1, 64), (1, 33, 1, 64),
+                  (2, 200, 2, 128), (1, 1024, 1, 128), (1, 1, 2, 128), (2, 129, 1, 128), (1, 130, 3, 128),
+                  (2, 64, 1, 128), (1, 33, 1, 128), (1, 300, 2, 128)]
+
+
+@pytest.mark.parametrize("B,T,H,d", TC_ATTN_SHAPES)
+def test_attention_fwd_tcgen05_kernel(B, T, H, d):
+    """head_dim 64 / 128 with the qkv array given as hi/lo planes: the TMA + tcgen05 + TMEM kernels."""
     C = H * d
     qkv = si.normal_f32(82, (B * T, 3 * C))
     dq = dev(qkv)
@@ -313,16 +318,15 @@ def test_attention_fwd_tcgen05_kernel(B, T, H):
     assert rel_l2(host(o), ro) < 1e-4 and rel_max(host(o), ro) < 1e-4
     assert np.abs(host(lse) - rlse).max() < 1e-4
     check_split(os_, host(o))
-    # and it agrees with the warp-MMA kernel on the raw array
+    # and it agrees with the kernel that takes the raw array (warp-MMA; FMA for head_dim 128)
     o2, lse2 = empty(B * T, C), empty(B, H, T)
     b.bt_op_attention_fwd(dq, B, T, C, H, o2, None, lse2, 0)
     assert rel_max(host(o), host(o2)) < 1e-5
 
 
-@pytest.mark.parametrize("B,T,H", [(2, 200, 3), (1, 1024, 2), (1, 1, 2), (3, 129, 1), (1, 130, 12), (2, 64, 1), (1, 33, 1)])
-def test_attention_bwd_tcgen05_kernels(B, T, H):
-    """head_dim 64, qkv and d_o given as hi/lo planes, only the split gradient requested."""
-    d = 64
+@pytest.mark.parametrize("B,T,H,d", TC_ATTN_SHAPES)
+def test_attention_bwd_tcgen05_kernels(B, T, H, d):
+    """head_dim 64 / 128, qkv and d_o given as hi/lo planes, only the split gradient requested."""
     C = H * d
     qkv = si.normal_f32(83, (B * T, 3 * C))
     d_o = si.normal_f32(84, (B * T, C), 1e-2)

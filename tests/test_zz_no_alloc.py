@@ -47,10 +47,10 @@ def test_static_scratch_colsum_matches_scratch_entry_point_twice():
 
 def test_static_scratch_colsum_rejects_oversized_and_bad_arguments():
     assert b.bt_op_colsum_static_max_floats() == 96 * 1024
-    x = empty(640, 65536)            # needs 2 strips x 65536 floats of partial sums: over the limit
-    assert b.bt_op_colsum_scratch_bytes(640, 65536) > 4 * b.bt_op_colsum_static_max_floats()
+    x = empty(64, 131072)            # one strip x 131072 floats of partial sums: over the limit
+    assert b.bt_op_colsum_scratch_bytes(64, 131072) > 4 * b.bt_op_colsum_static_max_floats()
     with pytest.raises(b.BtError) as e:
-        b.bt_op_colsum_static(x, 640, 65536, empty(65536))
+        b.bt_op_colsum_static(x, 64, 131072, empty(131072))
     assert e.value.status == 2 and "scratch" in str(e.value)
     with pytest.raises(b.BtError) as e:
         b.bt_op_colsum_static(x, 64, 6, empty(8))
