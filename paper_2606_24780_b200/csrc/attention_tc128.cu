@@ -151,9 +151,15 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
     const uint32_t a2_s = base;
     const uint32_t b1_s = base + kRes, b2_s = b1_s + kTile, b3_s = b2_s + kTile;
     const uint32_t bars = b3_s + kTile;
-    enum { A2_FULL = 0, B1_FULL, B1_EMPTY, B2_FULL, B2_EMPTY, B3_FULL, B3_EMPTY, XY_FULL0, XY_FULL1, ACC_FULL,
-           Z_READY0, Z_READY1, A1_READY, N_BARS };
+    // Passes without a resident A2 spend its 128 KB on the streams: B1 three stages deep (its own
+    // buffer and two A2 slots), B3 two stages (the other two A2 slots); the B2 / B3 buffers then only
+    // stage the CTA's own rows on their way into tensor memory.
+    constexpr int S1 = kHasY ? 1 : 3, S3 = kHasY ? 1 : 2;
+    enum { A2_FULL = 0, B1_FULL, B1_EMPTY = B1_FULL + 3, B2_FULL = B1_EMPTY + 3, B2_EMPTY, B3_FULL, B3_EMPTY = B3_FULL + 2,
+           XY_FULL0 = B3_EMPTY + 2, XY_FULL1, ACC_FULL, Z_READY0, Z_READY1, A1_READY, N_BARS };
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
+    auto b1_stage = [&](int st) { return (kHasY || st == 0) ? b1_s : a2_s + (uint32_t)(st - 1) * kTile; };
+    auto b3_stage = [&](int st) { return kHasY ? b3_s : a2_s + (uint32_t)(2 + st) * kTile; };
     const uint32_t tmem_slot = bars + 8u * N_BARS;
     auto smem_ptr = [&](uint32_t addr) { return smem_raw + (addr - smem_u32(smem_raw)); };
 
@@ -199,24 +205,28 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
                     tma_load_3d(a2_s + kb * (kRes / 4), &tmA2, bar(A2_FULL), g.a2_col + h * HD + kb * 32, row_base + r0, 0);
             }
             bool ok = true;
-            // one buffer per stream; t = the tile whose rows go in
-            auto load = [&](uint32_t dst, const CUtensorMap* tm, int full, int empty, int col, int t) -> bool {
-                if (!mbar_wait(bar(empty), (uint32_t)(t & 1) ^ 1u, g.err, 51)) return false;
-                mbar_expect_tx(bar(full), kTile);
+            // t = the tile whose rows go in; a stream of S stages keeps tile t in stage t % S
+            auto load = [&](uint32_t dst, const CUtensorMap* tm, int full, int empty, int col, int t, int stages) -> bool {
+                const int st = t % stages;
+                const uint32_t round = (uint32_t)(t / stages);
+                if (!mbar_wait(bar(empty + st), (round & 1u) ^ 1u, g.err, 51)) return false;
+                mbar_expect_tx(bar(full + st), kTile);
                 for (int part = 0; part < 4; ++part)
-                    tma_load_3d(dst + part * (kTile / 4), tm, bar(full), col + h * HD + part * 32, row_base + o0(t), 0);
+                    tma_load_3d(dst + part * (kTile / 4), tm, bar(full + st), col + h * HD + part * 32, row_base + o0(t), 0);
                 return true;
             };
-            ok = load(b1_s, &tmB1, B1_FULL, B1_EMPTY, g.b1_col, 0);
-            // the B2 / B3 buffers stage the CTA's own rows on their way into tensor memory first
-            if (ok) ok = mbar_wait(bar(A1_READY), 0, g.err, 52);
-            if (ok && kHasY) ok = load(b2_s, &tmB2, B2_FULL, B2_EMPTY, g.b2_col, 0);
+            ok = load(b1_stage(0), &tmB1, B1_FULL, B1_EMPTY, g.b1_col, 0, S1);
+            if (kHasY) {
+                // here the B2 / B3 buffers stage the CTA's own rows on their way into tensor memory first
+                if (ok) ok = mbar_wait(bar(A1_READY), 0, g.err, 52);
+                if (ok) ok = load(b2_s, &tmB2, B2_FULL, B2_EMPTY, g.b2_col, 0, 1);
+            }
             for (int t = 0; t < n_t && ok; ++t) {
                 if (t + 1 < n_t) {
-                    ok = load(b1_s, &tmB1, B1_FULL, B1_EMPTY, g.b1_col, t + 1);
-                    if (ok && kHasY) ok = load(b2_s, &tmB2, B2_FULL, B2_EMPTY, g.b2_col, t + 1);
+                    ok = load(b1_stage((t + 1) % S1), &tmB1, B1_FULL, B1_EMPTY, g.b1_col, t + 1, S1);
+                    if (ok && kHasY) ok = load(b2_s, &tmB2, B2_FULL, B2_EMPTY, g.b2_col, t + 1, 1);
                 }
-                if (ok && kHasOut) ok = load(b3_s, &tmB3, B3_FULL, B3_EMPTY, g.b3_col, t);
+                if (ok && kHasOut) ok = load(b3_stage(t % S3), &tmB3, B3_FULL, B3_EMPTY, g.b3_col, t, S3);
             }
             if (!ok)
                 for (int i = 0; i < 2000; ++i) __nanosleep(1000);   // let loads in flight land
@@ -228,12 +238,13 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
             constexpr uint32_t idesc_o = make_idesc_tf32(BR, HD, false, true);     // 128 x 128, B MN-major
             bool ok = mbar_wait(bar(A1_READY), 0, g.err, 53);
             if (ok && kHasY) ok = mbar_wait(bar(A2_FULL), 0, g.err, 54);
-            const DescBase a2d = kmaj_base(a2_s), b1d = kmaj_base(b1_s), b2d = kmaj_base(b2_s);
-            const DescBase b3d = mnmaj_base(b3_s);
+            const DescBase a2d = kmaj_base(a2_s), b2d = kmaj_base(b2_s);
             auto issue_xy = [&](int t) -> bool {
                 const uint32_t tX = tbuf(t & 1), tY = tX + 32u;
-                if (!mbar_wait(bar(B1_FULL), (uint32_t)(t & 1), g.err, 55)) return false;
+                const int st1 = t % S1;
+                if (!mbar_wait(bar(B1_FULL + st1), (uint32_t)((t / S1) & 1), g.err, 55)) return false;
                 tc_fence_after();
+                const DescBase b1d = kmaj_base(b1_stage(st1));
 #pragma unroll
                 for (int ks = 0; ks < 16; ++ks) {
                     const uint64_t b_hi = b1d.at(kmaj_off(BT_, ks, false)), b_lo = b1d.at(kmaj_off(BT_, ks, true));
@@ -241,7 +252,7 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
                     umma_tf32_ts(tX, tA1_hi + ks * 8, b_lo, idesc_x, 1u);
                     umma_tf32_ts(tX, tA1_hi + ks * 8, b_hi, idesc_x, 1u);
                 }
-                umma_commit(bar(B1_EMPTY));
+                umma_commit(bar(B1_EMPTY + st1));
                 if (kHasY) {
                     if (!mbar_wait(bar(B2_FULL), (uint32_t)(t & 1), g.err, 56)) return false;
                     tc_fence_after();
@@ -263,8 +274,10 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
             auto issue_out = [&](int t) -> bool {
                 if (!mbar_wait(bar(Z_READY0 + (t & 1)), (uint32_t)((t >> 1) & 1), g.err, 57)) return false;
                 if (kHasOut) {
-                    if (!mbar_wait(bar(B3_FULL), (uint32_t)(t & 1), g.err, 58)) return false;
+                    const int st3 = t % S3;
+                    if (!mbar_wait(bar(B3_FULL + st3), (uint32_t)((t / S3) & 1), g.err, 58)) return false;
                     tc_fence_after();
+                    const DescBase b3d = mnmaj_base(b3_stage(st3));
                     const uint32_t z_hi = tbuf(t & 1), z_lo = z_hi + 32u;
 #pragma unroll
                     for (int ks = 0; ks < 4; ++ks) {
@@ -274,7 +287,7 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
                         umma_tf32_ts(tOut, z_hi + ks * 8, b_lo, idesc_o, 1u);
                         umma_tf32_ts(tOut, z_hi + ks * 8, b_hi, idesc_o, 1u);
                     }
-                    umma_commit(bar(B3_EMPTY));
+                    umma_commit(bar(B3_EMPTY + st3));
                 }
                 return true;
             };

@@ -116,12 +116,12 @@ def build_cases(B, T, C, H, Vp, n_params):
     cases["attention_fwd"] = dict(run=lambda: b.bt_op_attention_fwd(qkv, B, T, C, H, o, os_, lse), flops=afl,
                                   bytes=24.0 * N * C, bound="tensor", keep=(qkv, o, os_, lse))
     b.bt_op_attention_fwd(qkv, B, T, C, H, o, os_, lse)
-    if C // H == 64:
+    if C // H in (64, 128):
         qkv_s = _split(qkv)
         cases["attention_fwd_tcgen05"] = dict(
             run=lambda: b.bt_op_attention_fwd(None, B, T, C, H, None, os_, lse, qkv_split=qkv_s), flops=afl,
             bytes=32.0 * N * C, bound="tensor", keep=(qkv_s,))
-    if C // H == 64:
+    if C // H in (64, 128):
         do_s, dqs2 = _split(d_o), torch.empty(2, N, 3 * C, device="cuda")
         cases["attention_bwd_tcgen05"] = dict(
             run=lambda: b.bt_op_attention_bwd(None, o, lse, None, B, T, C, H, None, dqs2, dv, dv.numel() * 4,
