@@ -41,12 +41,6 @@ constexpr uint32_t kSmemBytes = 1024u + kQBytes + 4u * kKVBytes + 256u;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
 struct AttnArgs {
     int T, C, H;
     float* o;

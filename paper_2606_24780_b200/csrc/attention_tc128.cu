@@ -53,12 +53,6 @@ constexpr uint32_t kSmem = 1024u + kRes + 3u * kTile + 256u;
 
 enum Pass { P_LSE = 0, P_FWD = 1, P_DQ = 2, P_DK = 3, P_DV = 4 };
 
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
 struct Args128 {
     int T, C, H;
     const float* a1_hi;       // hi plane of the array the CTA's own rows come from (lo at + a1_plane)
@@ -80,63 +74,11 @@ struct Args128 {
     int* err;
 };
 
-// Byte offset of k-step ks (8 contraction values) in a K-major tile of `rows` rows: k-blocks of
-// [hi | lo][rows][128 B].
-__device__ __forceinline__ constexpr uint32_t kmaj_off(int rows, int ks, bool lo) {
-    return (uint32_t)(ks >> 2) * 2u * (uint32_t)rows * 128u + (lo ? (uint32_t)rows * 128u : 0u) + (uint32_t)(ks & 3) * 32u;
-}
-__device__ __forceinline__ DescBase kmaj_base(uint32_t tile) { return make_desc_base(tile, 16u, 1024u, 2u); }
 // MN-major 32-row tile: 4 column groups of [hi | lo][32 rows][128 B]; k-step = 8 rows.
 __device__ __forceinline__ constexpr uint32_t mnmaj_off(int ks, bool lo) {
     return (lo ? BT_ * 128u : 0u) + (uint32_t)ks * 1024u;
 }
 __device__ __forceinline__ DescBase mnmaj_base(uint32_t tile) { return make_desc_base(tile, 2u * BT_ * 128u, 512u, 1u); }
-
-// The warp's 32 rows x 64 floats (hi/lo planes; row r of the warp at src + r * row_stride) ->
-// (hi + lo) * mul -> re-split -> 64 hi and 64 lo columns of tensor memory, lane = row.  Rows are
-// read as they lie in memory (8 lanes x 16 bytes = one 128-byte segment, all loads of a chunk in
-// flight) and turned through the warp's shared-memory tile.  Rows >= nvalid read the last valid row.
-__device__ __forceinline__ void rows64_to_tmem(const float* src_hi, const float* src_lo, long long row_stride,
-                                               int nvalid, float mul, uint32_t t_hi, uint32_t t_lo, float* tile,
-                                               int lane) {
-    const int sub = lane >> 3, cq = lane & 7;
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        float4 a[8], b[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int r = max(0, min(sub + 4 * i, nvalid - 1));
-            const long long off = (long long)r * row_stride + half * 32 + 4 * cq;
-            a[i] = *reinterpret_cast<const float4*>(src_hi + off);
-            b[i] = *reinterpret_cast<const float4*>(src_lo + off);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float4 x = make_float4((a[i].x + b[i].x) * mul, (a[i].y + b[i].y) * mul, (a[i].z + b[i].z) * mul,
-                                         (a[i].w + b[i].w) * mul);
-            *reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(tile) + (sub + 4 * i) * kRowTilePitch + cq * 16) = x;
-        }
-        __syncwarp();
-        uint32_t h[32], l[32];
-        const float4* rd = reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(tile) + lane * kRowTilePitch);
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const float4 x = rd[q];
-            const float xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                float fh, fl;
-                split_tf32(xs[e], fh, fl);
-                h[4 * q + e] = __float_as_uint(fh);
-                l[4 * q + e] = __float_as_uint(fl);
-            }
-        }
-        tmem_st32(t_hi + half * 32, h);
-        tmem_st32(t_lo + half * 32, l);
-        __syncwarp();   // the tile is rewritten by the next half
-    }
-    tmem_st_wait();
-}
 
 template <int PASS>
 __global__ void __launch_bounds__(kThreads, 1)
@@ -315,7 +257,7 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
             const int wrow0 = min(r0 + lane_group * 32, g.T - 1);
             const long long off = (long long)(row_base + wrow0) * g.a1_stride + g.a1_col + h * HD + 64 * wg;
             float* tile = reinterpret_cast<float*>(smem_ptr(b2_s) + (uint32_t)(warp - 2) * kRowTileBytes);
-            rows64_to_tmem(g.a1_hi + off, g.a1_hi + g.a1_plane + off, g.a1_stride, max(1, min(32, g.T - wrow0)),
+            rows_to_tmem(g.a1_hi + off, g.a1_hi + g.a1_plane + off, g.a1_stride, max(1, min(32, g.T - wrow0)),
                            kLog2e / sqrtf((float)HD), tA1_hi + t_lane + 64u * wg, tA1_lo + t_lane + 64u * wg, tile, lane);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the staging tiles are next written by TMA
             tc_fence_before();

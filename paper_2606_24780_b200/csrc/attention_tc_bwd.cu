@@ -44,12 +44,6 @@ constexpr float kLog2e = 1.4426950408889634f;
 constexpr uint32_t kResBytes = 2u * 2u * BR * 128u;   // resident 128-row operand: 2 k-blocks x (hi,lo)
 constexpr uint32_t kTileBytes = 2u * 2u * BT_ * 128u; // one streamed 32-row tile in one layout (16 KB)
 
-__device__ __forceinline__ float ex2_approx(float x) {
-    float y;
-    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-    return y;
-}
-
 // Per-CTA (start, end, SM, tiles) record behind the mark regions of the trace buffer (debug aid).
 __device__ __forceinline__ void trace_cta(unsigned long long* tr, int kernel_index, int slot, unsigned long long v) {
     if (tr == nullptr) return;
@@ -61,52 +55,6 @@ __device__ __forceinline__ unsigned smid() {
     unsigned r;
     asm volatile("mov.u32 %0, %%smid;" : "=r"(r));
     return r;
-}
-
-// The warp's 32 rows x 64 floats (given as hi/lo planes; row r of the warp at src + r * row_stride)
-// -> (hi + lo) * mul -> re-split -> hi/lo columns of tensor memory, lane = row.  The rows are read
-// the way they lie in memory (8 lanes x 16 bytes = one 128-byte row segment, all loads of a chunk in
-// flight together) and turned so that every lane ends up with its own row through the warp's
-// shared-memory tile.  Rows >= nvalid are read as the last valid row (their results are never used).
-__device__ __forceinline__ void rows_to_tmem(const float* src_hi, const float* src_lo, long long row_stride, int nvalid,
-                                             float mul, uint32_t t_hi, uint32_t t_lo, float* tile, int lane) {
-    const int sub = lane >> 3, cq = lane & 7;
-#pragma unroll
-    for (int half = 0; half < 2; ++half) {
-        float4 a[8], b[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const int r = max(0, min(sub + 4 * i, nvalid - 1));
-            const long long off = (long long)r * row_stride + half * 32 + 4 * cq;
-            a[i] = *reinterpret_cast<const float4*>(src_hi + off);
-            b[i] = *reinterpret_cast<const float4*>(src_lo + off);
-        }
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-            const float4 x = make_float4((a[i].x + b[i].x) * mul, (a[i].y + b[i].y) * mul, (a[i].z + b[i].z) * mul,
-                                         (a[i].w + b[i].w) * mul);
-            *reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(tile) + (sub + 4 * i) * kRowTilePitch + cq * 16) = x;
-        }
-        __syncwarp();
-        uint32_t h[32], l[32];
-        const float4* rd = reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(tile) + lane * kRowTilePitch);
-#pragma unroll
-        for (int q = 0; q < 8; ++q) {
-            const float4 x = rd[q];
-            const float xs[4] = {x.x, x.y, x.z, x.w};
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                float fh, fl;
-                split_tf32(xs[e], fh, fl);
-                h[4 * q + e] = __float_as_uint(fh);
-                l[4 * q + e] = __float_as_uint(fl);
-            }
-        }
-        tmem_st32(t_hi + half * 32, h);
-        tmem_st32(t_lo + half * 32, l);
-        __syncwarp();   // the tile is rewritten by the next half
-    }
-    tmem_st_wait();
 }
 
 // The 64 accumulator columns of the warp's 32 rows (times mul) -> hi/lo planes in global memory,
@@ -130,11 +78,6 @@ __device__ __forceinline__ void tmem_rows_to_split(uint32_t t_row, float mul, fl
 }
 
 // Byte offsets of one 8-deep k-step inside an operand tile (compile-time after unrolling).
-//  K-major tile (rows x 64 floats as 2 k-blocks of [hi|lo][rows][128 B]), contraction over d.
-__device__ __forceinline__ constexpr uint32_t kmaj_off(int rows, int ks, bool lo) {
-    return (uint32_t)(ks >> 2) * 2u * (uint32_t)rows * 128u + (lo ? (uint32_t)rows * 128u : 0u) + (uint32_t)(ks & 3) * 32u;
-}
-__device__ __forceinline__ DescBase kmaj_base(uint32_t tile) { return make_desc_base(tile, 16u, 1024u, 2u); }
 //  MN-major 32-row tile (2 column groups of [hi|lo][32 rows][128 B]), contraction over the rows.
 __device__ __forceinline__ constexpr uint32_t mnmaj_off(int ks, bool lo) {
     return (lo ? BT_ * 128u : 0u) + (uint32_t)ks * 1024u;

@@ -226,6 +226,66 @@ __device__ __forceinline__ void warp_rows_store(const float (&v)[32], float* til
     __syncwarp();   // the tile is rewritten by the next chunk
 }
 
+// ---------------------------------------------------------------- helpers of the attention kernels
+__device__ __forceinline__ float ex2_approx(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Byte offset of k-step ks (8 contraction values) in a K-major operand tile of `rows` rows held as
+// k-blocks of [hi | lo][rows][128 B] (32 floats of the contraction index per block).
+__device__ __forceinline__ constexpr uint32_t kmaj_off(int rows, int ks, bool lo) {
+    return (uint32_t)(ks >> 2) * 2u * (uint32_t)rows * 128u + (lo ? (uint32_t)rows * 128u : 0u) + (uint32_t)(ks & 3) * 32u;
+}
+__device__ __forceinline__ DescBase kmaj_base(uint32_t tile) { return make_desc_base(tile, 16u, 1024u, 2u); }
+
+// The warp's 32 rows x 64 floats (given as hi/lo planes; row r of the warp at src + r * row_stride)
+// -> (hi + lo) * mul -> re-split -> hi/lo columns of tensor memory, lane = row.  The rows are read
+// the way they lie in memory (8 lanes x 16 bytes = one 128-byte row segment, all loads of a chunk in
+// flight together) and turned so that every lane ends up with its own row through the warp's
+// shared-memory tile.  Rows >= nvalid are read as the last valid row (their results are never used).
+__device__ __forceinline__ void rows_to_tmem(const float* src_hi, const float* src_lo, long long row_stride, int nvalid,
+                                             float mul, uint32_t t_hi, uint32_t t_lo, float* tile, int lane) {
+    const int sub = lane >> 3, cq = lane & 7;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+        float4 a[8], b[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const int r = max(0, min(sub + 4 * i, nvalid - 1));
+            const long long off = (long long)r * row_stride + half * 32 + 4 * cq;
+            a[i] = *reinterpret_cast<const float4*>(src_hi + off);
+            b[i] = *reinterpret_cast<const float4*>(src_lo + off);
+        }
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const float4 x = make_float4((a[i].x + b[i].x) * mul, (a[i].y + b[i].y) * mul, (a[i].z + b[i].z) * mul,
+                                         (a[i].w + b[i].w) * mul);
+            *reinterpret_cast<float4*>(reinterpret_cast<uint8_t*>(tile) + (sub + 4 * i) * kRowTilePitch + cq * 16) = x;
+        }
+        __syncwarp();
+        uint32_t h[32], l[32];
+        const float4* rd = reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(tile) + lane * kRowTilePitch);
+#pragma unroll
+        for (int q = 0; q < 8; ++q) {
+            const float4 x = rd[q];
+            const float xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                float fh, fl;
+                split_tf32(xs[e], fh, fl);
+                h[4 * q + e] = __float_as_uint(fh);
+                l[4 * q + e] = __float_as_uint(fl);
+            }
+        }
+        tmem_st32(t_hi + half * 32, h);
+        tmem_st32(t_lo + half * 32, l);
+        __syncwarp();   // the tile is rewritten by the next half
+    }
+    tmem_st_wait();
+}
+
 // ---------------------------------------------------------------- CTA pairs (cta_group::2)
 // A cluster of two CTAs on neighbouring SMs issues one MMA of M = 256: each CTA supplies its own
 // 128 rows of A and HALF of the B tile from its own shared memory and holds its own 128 rows of
