@@ -63,10 +63,92 @@ __global__ void __launch_bounds__(kLnWarps * 32) ln_fwd_kernel(const float* __re
     }
 }
 
+// Rows wider than 1024 floats: the whole CTA works on a row (thread i = float4 column i), two
+// rows per round; the mean and then the centred sum of squares go through block reductions.
+template <int R>
+__global__ void __launch_bounds__(1024, 1) ln_fwd_wide_kernel(const float* __restrict__ x,
+                                                              const float* __restrict__ gamma,
+                                                              const float* __restrict__ beta, int64_t N, int C4,
+                                                              float* y, float* y_hi, float* y_lo,
+                                                              float* __restrict__ mean, float* __restrict__ rstd) {
+    pdl_wait();
+    pdl_trigger();
+    __shared__ float red[32][R];
+    __shared__ float tot[R];
+    const int idx = threadIdx.x, lane = idx & 31, warp = idx >> 5, nwarps = blockDim.x >> 5;
+    const bool active = idx < C4;
+    const float inv_c = 1.0f / (float)(C4 * 4);
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4 g = active ? ld4(gamma, idx) : zero, b = active ? ld4(beta, idx) : zero;
+    // block-wide sums of R values (one per row of the round), warps combined in warp order
+    auto block_sums = [&](float (&v)[R]) {
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            const float w = warp_sum(v[j]);
+            if (lane == 0) red[warp][j] = w;
+        }
+        __syncthreads();
+        if (idx < R) {
+            float t = 0.f;
+            for (int w = 0; w < nwarps; ++w) t += red[w][idx];
+            tot[idx] = t;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < R; ++j) v[j] = tot[j];
+        __syncthreads();   // tot and red are rewritten by the next reduction
+    };
+    for (int64_t row0 = (int64_t)blockIdx.x * R; row0 < N; row0 += (int64_t)gridDim.x * R) {
+        float4 v[R];
+        float s[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            v[j] = (row0 + j < N && active) ? ld4(x, (row0 + j) * C4 + idx) : zero;
+            s[j] = (v[j].x + v[j].y) + (v[j].z + v[j].w);
+        }
+        block_sums(s);
+        float mu[R], q[R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            mu[j] = s[j] * inv_c;
+            const float a = v[j].x - mu[j], c = v[j].y - mu[j], d = v[j].z - mu[j], e = v[j].w - mu[j];
+            q[j] = active ? (a * a + c * c) + (d * d + e * e) : 0.f;
+        }
+        block_sums(q);
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            const int64_t row = row0 + j;
+            if (row >= N) continue;
+            const float rs = 1.0f / sqrtf(q[j] * inv_c + kLnEps);
+            if (active) {
+                float4 r;
+                r.x = g.x * ((v[j].x - mu[j]) * rs) + b.x;
+                r.y = g.y * ((v[j].y - mu[j]) * rs) + b.y;
+                r.z = g.z * ((v[j].z - mu[j]) * rs) + b.z;
+                r.w = g.w * ((v[j].w - mu[j]) * rs) + b.w;
+                store_raw_split(r, y, y_hi, y_lo, row * C4 + idx);
+            }
+            if (idx == 0) {
+                if (mean) mean[row] = mu[j];
+                if (rstd) rstd[row] = rs;
+            }
+        }
+    }
+}
+
 cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float* beta, int64_t N, int C, float* y,
                                  float* y_hi, float* y_lo, float* mean, float* rstd, cudaStream_t s) {
     const int C4 = C / 4;
     const int vpl = (C4 + 31) / 32;
+    if (vpl > 8) {   // C > 1024: CTA per row
+        if (C > 4096) return cudaErrorInvalidValue;
+        constexpr int R = 2;
+        const int64_t rounds = (N + R - 1) / R;
+        const int wgrid = (int)(rounds < 2 * 148 ? rounds : 2 * 148);
+        BT_KERNEL_LAUNCH((ln_fwd_wide_kernel<R>), wgrid, vpl * 32, 0, s, x, gamma, beta, N, C4, y, y_hi, y_lo, mean, rstd);
+        BT_COUNT_LAUNCH();
+        return cudaGetLastError();
+    }
     const int grid = (int)((N + kLnWarps - 1) / kLnWarps);
 #define BT_LN_FWD(V)                                                                                     \
     BT_KERNEL_LAUNCH((ln_fwd_kernel<V>), grid, kLnWarps * 32, 0, s, x, gamma, beta, N, C4, y, y_hi, y_lo, mean, rstd)
@@ -75,8 +157,6 @@ cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float
     else if (vpl <= 4) BT_LN_FWD(4);
     else if (vpl <= 6) BT_LN_FWD(6);
     else if (vpl <= 8) BT_LN_FWD(8);
-    else if (vpl <= 16) BT_LN_FWD(16);
-    else if (vpl <= 32) BT_LN_FWD(32);
     else return cudaErrorInvalidValue;
 #undef BT_LN_FWD
     BT_COUNT_LAUNCH();
@@ -91,7 +171,7 @@ static inline int ln_bwd_ctas(int64_t N) {
     return (int)g;
 }
 static inline int ln_bwd_wide_ctas(int64_t N) {
-    int64_t g = (N + 3) / 4;   // four warps (rows) per CTA, one CTA per SM
+    int64_t g = (N + 1) / 2;   // two rows per round, one CTA per SM
     return (int)(g < 148 ? g : 148);
 }
 size_t layernorm_bwd_scratch_floats(int64_t N, int C) {
@@ -174,67 +254,98 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     }
 }
 
-// Rows wider than the register-resident kernel takes (C > 1024): a warp walks its row twice, 32
-// float4 at a time -- once for the two row sums, once (the row now comes from L1/L2) for dx and
-// the column accumulators, which live in shared memory as above.  Four warps per CTA, one CTA per
-// SM: 3 x C floats of accumulators per warp.
+// Rows wider than the register-resident kernel takes (C > 1024): the whole CTA works on a row.
+// Thread i owns float4 column i (C / 4 <= 1024 threads), keeps that column's dgamma, dbeta and
+// column-sum accumulators in registers, and the two row sums go through a block reduction; two
+// rows are in flight per round (6 128-bit loads per thread, two barriers).  One CTA per SM, rows
+// dealt to the CTAs two at a time.
+constexpr int kWideRows = 2;
 template <bool CS>
-__global__ void __launch_bounds__(128, 1) ln_bwd_wide_kernel(
+__global__ void __launch_bounds__(1024, 1) ln_bwd_wide_kernel(
     const float* __restrict__ dy, const float* __restrict__ x, const float* __restrict__ gamma,
     const float* __restrict__ mean, const float* __restrict__ rstd, const float* dres, int64_t N, int C4,
     float* dx, float* dx_hi, float* dx_lo, float* __restrict__ partial) {
     pdl_wait();
     pdl_trigger();
     constexpr int kParts = CS ? 3 : 2;
-    constexpr int kWarps = 4;
-    extern __shared__ float4 sm[];  // [kWarps][kParts][C4]
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float4* acc = sm + (size_t)warp * kParts * C4;
-    for (int i = lane; i < kParts * C4; i += 32) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-    __syncwarp();
+    constexpr int R = kWideRows;
+    __shared__ float red[32][2 * R];
+    __shared__ float tot[2 * R];
+    const int idx = threadIdx.x, lane = idx & 31, warp = idx >> 5, nwarps = blockDim.x >> 5;
+    const bool active = idx < C4;
     const float inv_c = 1.0f / (float)(C4 * 4);
-    for (int64_t row = (int64_t)blockIdx.x * kWarps + warp; row < N; row += (int64_t)gridDim.x * kWarps) {
-        const float mu = mean[row], rs = rstd[row];
-        float s1 = 0.f, s2 = 0.f;
-        for (int idx = lane; idx < C4; idx += 32) {
-            const float4 xv = ld4(x, row * C4 + idx), dv = ld4(dy, row * C4 + idx), gm = ld4(gamma, idx);
-            const float4 xh = make_float4((xv.x - mu) * rs, (xv.y - mu) * rs, (xv.z - mu) * rs, (xv.w - mu) * rs);
-            const float4 dg = make_float4(dv.x * gm.x, dv.y * gm.y, dv.z * gm.z, dv.w * gm.w);
-            s1 += (dg.x + dg.y) + (dg.z + dg.w);
-            s2 += (dg.x * xh.x + dg.y * xh.y) + (dg.z * xh.z + dg.w * xh.w);
+    const float4 zero = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float4 gm = active ? ld4(gamma, idx) : zero;
+    float4 a_g = zero, a_b = zero, a_c = zero;
+    for (int64_t row0 = (int64_t)blockIdx.x * R; row0 < N; row0 += (int64_t)gridDim.x * R) {
+        float4 xh[R], dg[R], rv[R];
+        float rs[R], part[2 * R];
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            const int64_t row = row0 + j;
+            xh[j] = dg[j] = rv[j] = zero;
+            rs[j] = 0.f;
+            if (row < N && active) {
+                xh[j] = ld4(x, row * C4 + idx);
+                dg[j] = ld4(dy, row * C4 + idx);
+                if (dres) rv[j] = ld4(dres, row * C4 + idx);
+            }
         }
-        s1 = warp_sum(s1) * inv_c;
-        s2 = warp_sum(s2) * inv_c;
-        for (int idx = lane; idx < C4; idx += 32) {
-            const float4 xv = ld4(x, row * C4 + idx), dv = ld4(dy, row * C4 + idx), gm = ld4(gamma, idx);
-            const float4 xh = make_float4((xv.x - mu) * rs, (xv.y - mu) * rs, (xv.z - mu) * rs, (xv.w - mu) * rs);
-            const float4 dg = make_float4(dv.x * gm.x, dv.y * gm.y, dv.z * gm.z, dv.w * gm.w);
-            float4 a = acc[idx];
-            a.x += dv.x * xh.x; a.y += dv.y * xh.y; a.z += dv.z * xh.z; a.w += dv.w * xh.w;
-            acc[idx] = a;
-            acc[C4 + idx] = add4(acc[C4 + idx], dv);
-            float4 r;
-            r.x = rs * (dg.x - s1 - xh.x * s2);
-            r.y = rs * (dg.y - s1 - xh.y * s2);
-            r.z = rs * (dg.z - s1 - xh.z * s2);
-            r.w = rs * (dg.w - s1 - xh.w * s2);
-            if (dres) r = add4(r, ld4(dres, row * C4 + idx));
-            store_raw_split(r, dx, dx_hi, dx_lo, row * C4 + idx);
-            if (CS) acc[2 * C4 + idx] = add4(acc[2 * C4 + idx], r);
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            const int64_t row = row0 + j;
+            part[2 * j] = part[2 * j + 1] = 0.f;
+            if (row < N) {
+                const float mu = mean[row];
+                rs[j] = rstd[row];
+                if (active) {
+                    xh[j] = make_float4((xh[j].x - mu) * rs[j], (xh[j].y - mu) * rs[j], (xh[j].z - mu) * rs[j], (xh[j].w - mu) * rs[j]);
+                    a_g.x += dg[j].x * xh[j].x; a_g.y += dg[j].y * xh[j].y; a_g.z += dg[j].z * xh[j].z; a_g.w += dg[j].w * xh[j].w;
+                    a_b = add4(a_b, dg[j]);
+                    dg[j] = make_float4(dg[j].x * gm.x, dg[j].y * gm.y, dg[j].z * gm.z, dg[j].w * gm.w);
+                    part[2 * j] = (dg[j].x + dg[j].y) + (dg[j].z + dg[j].w);
+                    part[2 * j + 1] = (dg[j].x * xh[j].x + dg[j].y * xh[j].y) + (dg[j].z * xh[j].z + dg[j].w * xh[j].w);
+                }
+            }
+        }
+#pragma unroll
+        for (int v = 0; v < 2 * R; ++v) {
+            const float w = warp_sum(part[v]);
+            if (lane == 0) red[warp][v] = w;
+        }
+        __syncthreads();
+        if (idx < 2 * R) {   // warps are combined in warp order
+            float t = 0.f;
+            for (int w = 0; w < nwarps; ++w) t += red[w][idx];
+            tot[idx] = t * inv_c;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int j = 0; j < R; ++j) {
+            const int64_t row = row0 + j;
+            if (row < N && active) {
+                const float s1 = tot[2 * j], s2 = tot[2 * j + 1];
+                float4 r;
+                r.x = rs[j] * (dg[j].x - s1 - xh[j].x * s2);
+                r.y = rs[j] * (dg[j].y - s1 - xh[j].y * s2);
+                r.z = rs[j] * (dg[j].z - s1 - xh[j].z * s2);
+                r.w = rs[j] * (dg[j].w - s1 - xh[j].w * s2);
+                r = add4(r, rv[j]);
+                store_raw_split(r, dx, dx_hi, dx_lo, row * C4 + idx);
+                if (CS) a_c = add4(a_c, r);
+            }
         }
     }
-    __syncthreads();
-    float4* dst = reinterpret_cast<float4*>(partial) + (int64_t)blockIdx.x * kParts * C4;
-    for (int i = threadIdx.x; i < kParts * C4; i += blockDim.x) {
-        float4 t = sm[i];
-#pragma unroll
-        for (int w = 1; w < kWarps; ++w) t = add4(t, sm[(size_t)w * kParts * C4 + i]);
-        dst[i] = t;
+    if (active) {
+        float4* dst = reinterpret_cast<float4*>(partial) + (int64_t)blockIdx.x * kParts * C4;
+        dst[idx] = a_g;
+        dst[C4 + idx] = a_b;
+        if (CS) dst[2 * C4 + idx] = a_c;
     }
 }
 
 // Sums the per-CTA partials in a fixed order: lane = float4 column, warp w takes partials
-// w, w+8, ... (four loads in flight), the eight warp sums are combined in warp order.
+// w, w+8, ... (twelve, then four loads in flight), the eight warp sums are combined in warp order.
 __global__ void __launch_bounds__(256) ln_bwd_reduce_kernel(const float* __restrict__ partial, int nparts, int C4,
                                                             int kparts, float* __restrict__ dgamma,
                                                             float* __restrict__ dbeta, float* __restrict__ dcolsum) {
@@ -247,6 +358,13 @@ __global__ void __launch_bounds__(256) ln_bwd_reduce_kernel(const float* __restr
     float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
     if (c < W) {
         int p = warp;
+        for (; p + 88 < nparts; p += 96) {   // twelve loads in flight: the grid is small, latency is the cost
+            float4 a[12];
+#pragma unroll
+            for (int j = 0; j < 12; ++j) a[j] = ld4(partial, (int64_t)(p + 8 * j) * W + c);
+#pragma unroll
+            for (int j = 0; j < 12; ++j) t = add4(t, a[j]);
+        }
         for (; p + 24 < nparts; p += 32) {
             float4 a0 = ld4(partial, (int64_t)p * W + c), a1 = ld4(partial, (int64_t)(p + 8) * W + c);
             float4 a2 = ld4(partial, (int64_t)(p + 16) * W + c), a3 = ld4(partial, (int64_t)(p + 24) * W + c);
@@ -291,20 +409,13 @@ cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* g
     const int vpl = (C4 + 31) / 32;
     if (vpl > 8) {   // C > 1024: the two-pass kernel
         if (C > 4096) return cudaErrorInvalidValue;
-        static const cudaError_t wattr = []() {
-            cudaError_t e = cudaFuncSetAttribute(ln_bwd_wide_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            if (e == cudaSuccess)
-                e = cudaFuncSetAttribute(ln_bwd_wide_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-            return e;
-        }();
-        if (wattr != cudaSuccess) return wattr;
         const int kparts = dx_colsum ? 3 : 2;
         const int wgrid = ln_bwd_wide_ctas(N);
-        const size_t wsmem = (size_t)4 * kparts * C4 * sizeof(float4);
+        const int wblock = ((C4 + 31) / 32) * 32;
         if (dx_colsum)
-            BT_KERNEL_LAUNCH((ln_bwd_wide_kernel<true>), wgrid, 128, wsmem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, dx_hi, dx_lo, scratch);
+            BT_KERNEL_LAUNCH((ln_bwd_wide_kernel<true>), wgrid, wblock, 0, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, dx_hi, dx_lo, scratch);
         else
-            BT_KERNEL_LAUNCH((ln_bwd_wide_kernel<false>), wgrid, 128, wsmem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, dx_hi, dx_lo, scratch);
+            BT_KERNEL_LAUNCH((ln_bwd_wide_kernel<false>), wgrid, wblock, 0, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, dx_hi, dx_lo, scratch);
         BT_COUNT_LAUNCH();
         BT_KERNEL_LAUNCH((ln_bwd_reduce_kernel), (kparts * C4 + 31) / 32, 256, 0, s, scratch, wgrid, C4, kparts, dgamma, dbeta, dx_colsum);
         BT_COUNT_LAUNCH();

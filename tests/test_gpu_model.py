@@ -323,6 +323,15 @@ def test_wide_model_head_dim_128():
     run_steps(cfg, seed=6, flags=0, B=2, steps=1)
 
 
+def test_head_dim_128_model_with_several_query_blocks():
+    """Two layers with two heads of 128 at T = 200: the head_dim-128 attention passes walk several
+    128-row blocks and a ragged last tile inside a whole training step (loss, every gradient, the
+    AdamW update against the oracle)."""
+    cfg = si.make_config(n_layers=2, d_model=256, n_heads=2, seq_len=200, vocab_size=500, padded_vocab_size=512,
+                         batch=2, tokens="zipf")
+    run_steps(cfg, seed=8, flags=0, B=2, steps=2)
+
+
 @pytest.mark.parametrize("pinned", [True, False])
 def test_double_buffered_loader_feeds_the_step(pinned):
     """Algorithm 2 on the GPU: batches arrive through the copy stream two channels deep; every batch
