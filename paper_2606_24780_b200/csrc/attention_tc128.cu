@@ -21,9 +21,10 @@
 // then FWD: with the row's log-sum-exp known, P is final when it is formed and O accumulates in
 // tensor memory like the backward's outputs, with no running-maximum rescaling.  The streamed
 // tiles B1, B2 (K-major, 128-byte swizzle) and B3 (MN-major, 128-byte swizzle with 32-byte atoms)
-// are 32 rows x 128 columns x (hi, lo) = 32 KB each, one buffer per stream, each refilled as soon
-// as the one product that reads it has completed; X / Y live in two tensor-memory buffers that
-// the two element-wise warpgroups take alternately, and Z overwrites X / Y in place.
+// are 32 rows x 128 columns x (hi, lo) = 32 KB each.  With A2 resident (DQ, DK) every stream has
+// one buffer, refilled as soon as the one product that reads it has completed; the passes without
+// A2 spend its 128 KB on three B1 stages and two B3 stages.  X / Y live in two tensor-memory
+// buffers that the two element-wise warpgroups take alternately, and Z overwrites X / Y in place.
 //
 //   warp 0 (one lane)   TMA producer
 //   warp 1 (one lane)   MMA issuer: X(0) Y(0), then per tile t: X(t+1) Y(t+1) | Out(t)
@@ -31,7 +32,7 @@
 //
 //   tensor memory: A1 hi 0-127, A1 lo 128-255, Out 256-383, buffer b: X -> Z_hi at 384 + 64 b,
 //                  Y -> Z_lo at 416 + 64 b
-//   shared memory: A2 128 KB, B1 / B2 / B3 32 KB each
+//   shared memory: A2 128 KB (or stream stages), B1 / B2 / B3 32 KB each
 // Every mbarrier wait is bounded and reports through the device error word; a CTA whose wait ran
 // out stops issuing, lets loads in flight land, frees its tensor memory and exits.
 #include "common.cuh"
