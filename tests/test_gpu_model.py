@@ -323,6 +323,16 @@ def test_wide_model_head_dim_128():
     run_steps(cfg, seed=6, flags=0, B=2, steps=1)
 
 
+def test_wide_model_full_width_full_context():
+    """Two layers at the full width of the paper's 2.42B configuration (d_model 3072, 24 heads of
+    128) and its full context (T = 1024, one sequence): eight query blocks per head in the
+    head_dim-128 attention passes, K = 12,288 GEMMs, CTA-per-row LayerNorm.  About half a minute
+    of oracle time."""
+    cfg = si.make_config(n_layers=2, d_model=3072, n_heads=24, seq_len=1024, vocab_size=2000, padded_vocab_size=2048,
+                         batch=1, tokens="zipf")
+    run_steps(cfg, seed=9, flags=0, B=1, steps=1)
+
+
 def test_head_dim_128_model_with_several_query_blocks():
     """Two layers with two heads of 128 at T = 200: the head_dim-128 attention passes walk several
     128-row blocks and a ragged last tile inside a whole training step (loss, every gradient, the
