@@ -323,6 +323,14 @@ def test_wide_model_head_dim_128():
     run_steps(cfg, seed=6, flags=0, B=2, steps=1)
 
 
+def test_350m_width_two_layers():
+    """The width of BASELINE config 4 (d_model 1024, 16 heads of 64, MLP 4096) at reduced depth and
+    context: the VPL = 8 LayerNorm instantiations and the 1024 / 4096-wide GEMM tilings in a step."""
+    cfg = si.make_config(n_layers=2, d_model=1024, n_heads=16, seq_len=256, vocab_size=3000, padded_vocab_size=3072,
+                         batch=2, tokens="zipf")
+    run_steps(cfg, seed=10, flags=0, B=2, steps=1)
+
+
 def test_wide_model_full_width_full_context():
     """Two layers at the full width of the paper's 2.42B configuration (d_model 3072, 24 heads of
     128) and its full context (T = 1024, one sequence): eight query blocks per head in the
