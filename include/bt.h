@@ -123,7 +123,7 @@ BT_API bt_status bt_tensor_info(const bt_model* m, int32_t index, const char** n
 BT_API bt_status bt_tensor_ptr(bt_model* m, const char* name, int32_t kind, float** d_ptr);
 
 /* Activations of the last forward/backward, for tests: per-layer "x", "qkv" (raw; written only
- * when head_dim != 64 or a reference-kernel flag is set), "x1", "h",
+ * when head_dim is neither 64 nor 128 or a reference-kernel flag is set), "x1", "h",
  * "ln1.mean", "ln1.rstd", "ln2.mean", "ln2.rstd", "lse"; split per-layer "qkv_split", "a", "o", "m", "g"
  * (pointer to the hi plane; lo plane follows at +numel); global "xL", "logits", "losses",
  * split "xf", "dlogits".  `numel` (nullable) receives the element count of one plane for
@@ -316,17 +316,17 @@ BT_API bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K, con
 /* Causal multi-head self-attention over fused qkv [B*T, 3C] (columns q | k | v, head h at
  * columns h*d..(h+1)*d-1 of each part): o = softmax(q k^T / sqrt(d) + causal mask) v,
  * lse [B,H,T] = log of the softmax normaliser.  d = C/H in {16, 32, 64, 128}.
- * qkv_split (nullable) is the same array as hi/lo planes [2][B*T][3C]; when it is given and d = 64
- * the tcgen05 kernel runs (TMA-fed, scores and probabilities in tensor memory; synchronises to
- * report a device timeout), otherwise the warp-MMA kernel runs on the raw array.  One of qkv,
- * qkv_split may be NULL. */
+ * qkv_split (nullable) is the same array as hi/lo planes [2][B*T][3C]; when it is given and d is
+ * 64 or 128 the tcgen05 kernels run (TMA-fed, scores and probabilities in tensor memory;
+ * synchronises to report a device timeout), otherwise the warp-MMA kernel (d <= 64) or the FMA
+ * kernel (d = 128) runs on the raw array.  One of qkv, qkv_split may be NULL. */
 BT_API bt_status bt_op_attention_fwd(const float* qkv, const float* qkv_split, int32_t B, int32_t T, int32_t C,
                                      int32_t H, float* o, float* o_split, float* lse, uint32_t flags, void* stream);
 
 /* Backward of the above with recomputed probabilities: dV = P^T do, dP = do V^T,
  * dS = P o (dP - rowsum(do o o)), dq = dS k / sqrt(d), dk = dS^T q / sqrt(d).
  * scratch: B*H*T floats.  qkv and d_o may be given raw and/or as hi/lo planes (qkv_split
- * [2][B*T][3C], d_o_split [2][B*T][C]); with both split inputs, d = 64 and only dqkv_split
+ * [2][B*T][3C], d_o_split [2][B*T][C]); with both split inputs, d = 64 or 128 and only dqkv_split
  * requested (dqkv NULL) the tcgen05 kernels run (they synchronise to report a device timeout),
  * otherwise the warp-MMA kernels run on the raw arrays, which must then be given. */
 BT_API bt_status bt_op_attention_bwd(const float* qkv, const float* qkv_split, const float* o, const float* lse,
