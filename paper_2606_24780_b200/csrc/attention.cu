@@ -12,8 +12,9 @@ cudaError_t launch_attention_bwd_simt(const float* qkv, const float* o, const fl
 cudaError_t launch_attention_dvec(const float* o, const float* o_lo, const float* d_o, const float* d_o_lo, int B,
                                   int T, int C, int H, float* dvec, cudaStream_t s);
 cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, const float* do_hi, int64_t do_plane,
-                                    const float* lse, const float* dvec, int B, int T, int C, int H, float* dqkv_hi,
-                                    int64_t dqkv_plane, float* rg_sums, int* err_word, cudaStream_t s);
+                                    const float* o, const float* o_lo, const float* lse, float* dvec, int B, int T,
+                                    int C, int H, float* dqkv_hi, int64_t dqkv_plane, float* rg_sums, int* err_word,
+                                    cudaStream_t s);
 bool attention_mma_supports(int head_dim);
 cudaError_t launch_attention_fwd_mma(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi,
                                      float* o_lo, float* lse, cudaStream_t s);
@@ -58,15 +59,15 @@ cudaError_t launch_attention_bwd(const float* qkv, const float* qkv_hi, int64_t 
     const bool tc = !simt && qkv_hi && do_hi && dqkv_hi && !dqkv && (attention_tc_supports(C / H, C) || tc128) &&
                     dqkv_lo == dqkv_hi + (int64_t)B * T * 3 * C;
     if (tc) {
+        if (rg_sums_written) *rg_sums_written = rg_sums != nullptr;
+        if (!tc128)   // head_dim 64: the dq kernel forms rowsum(dO o O) itself
+            return launch_attention_bwd_tc(qkv_hi, qkv_plane, do_hi, do_plane, o, o_lo, lse, dvec, B, T, C, H, dqkv_hi,
+                                           (int64_t)B * T * 3 * C, rg_sums, err_word, s);
         cudaError_t e = d_o ? launch_attention_dvec(o, o_lo, d_o, nullptr, B, T, C, H, dvec, s)
                             : launch_attention_dvec(o, o_lo, do_hi, do_hi + do_plane, B, T, C, H, dvec, s);
         if (e != cudaSuccess) return e;
-        if (rg_sums_written) *rg_sums_written = rg_sums != nullptr;
-        if (tc128)
-            return launch_attention_bwd_tc128(qkv_hi, qkv_plane, do_hi, do_plane, lse, dvec, B, T, C, H, dqkv_hi,
-                                              (int64_t)B * T * 3 * C, rg_sums, err_word, s);
-        return launch_attention_bwd_tc(qkv_hi, qkv_plane, do_hi, do_plane, lse, dvec, B, T, C, H, dqkv_hi,
-                                       (int64_t)B * T * 3 * C, rg_sums, err_word, s);
+        return launch_attention_bwd_tc128(qkv_hi, qkv_plane, do_hi, do_plane, lse, dvec, B, T, C, H, dqkv_hi,
+                                          (int64_t)B * T * 3 * C, rg_sums, err_word, s);
     }
     if (!qkv || !d_o) return cudaErrorInvalidValue;
     if (simt || !attention_mma_supports(C / H))

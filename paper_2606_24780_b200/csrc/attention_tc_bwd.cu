@@ -84,12 +84,59 @@ __device__ __forceinline__ constexpr uint32_t mnmaj_off(int ks, bool lo) {
 }
 __device__ __forceinline__ DescBase mnmaj_base(uint32_t tile) { return make_desc_base(tile, 2u * BT_ * 128u, 512u, 1u); }
 
+// D = rowsum(dO o O) over one head's 64 columns for the warp's 32 rows; lane r returns row r's value.
+// The rows are read as they lie in memory (8 lanes x 16 bytes = one 128-byte segment), four rows of
+// all planes in flight per lane; a 3-step butterfly adds the 8 column slices of a row, 8 shuffles
+// bring row r's sum to lane r.  a = O (a_lo nullable), b = dO as hi/lo planes; rows >= nvalid read
+// the last valid row.
+__device__ __forceinline__ float warp_rows_dot64(const float* a_hi, const float* a_lo, const float* b_hi,
+                                                 const float* b_lo, long long row_stride, int nvalid, int lane) {
+    const int sub = lane >> 3, cq = lane & 7;
+    float acc[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) acc[i] = 0.f;
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+#pragma unroll
+        for (int g4 = 0; g4 < 2; ++g4) {
+            float4 x[4], y[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int r = max(0, min(sub + 4 * (4 * g4 + j), nvalid - 1));
+                const long long off = (long long)r * row_stride + half * 32 + 4 * cq;
+                x[j] = *reinterpret_cast<const float4*>(a_hi + off);
+                if (a_lo) x[j] = add4(x[j], *reinterpret_cast<const float4*>(a_lo + off));
+                y[j] = add4(*reinterpret_cast<const float4*>(b_hi + off), *reinterpret_cast<const float4*>(b_lo + off));
+            }
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                acc[4 * g4 + j] += (x[j].x * y[j].x + x[j].y * y[j].y) + (x[j].z * y[j].z + x[j].w * y[j].w);
+        }
+    }
+    float d = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        float v = acc[i];
+        v += __shfl_xor_sync(0xffffffffu, v, 1);
+        v += __shfl_xor_sync(0xffffffffu, v, 2);
+        v += __shfl_xor_sync(0xffffffffu, v, 4);
+        v = __shfl_sync(0xffffffffu, v, 8 * (lane & 3));     // row sub + 4 i lives in the lanes of slice `sub`
+        if ((lane >> 2) == i) d = v;                          // lane r wants row r = (r & 3) + 4 (r >> 2)
+    }
+    return d;
+}
+
 struct BwdArgs {
     int T, C, H;
     const float* qkv_hi;      // split qkv [2][B*T][3C]
     long long qkv_plane;
     const float* lse;
-    const float* dvec;
+    const float* dvec;        // [B, H, T] rowsum(dO o O): written by the dq kernel, read by the dkv kernel
+    float* dvec_out;          // the same array, for the dq kernel
+    const float* o_hi;        // attention output [B*T][C] (raw, or the hi plane with o_lo the lo plane)
+    const float* o_lo;        // nullable
+    const float* do_hi;       // split output gradient [2][B*T][C]
+    long long do_plane;
     float* dqkv_hi;           // split output [2][B*T][3C]
     long long dqkv_plane;
     int* err;
@@ -414,7 +461,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
 // K-major K and V tiles (4 x 32 KB) and ONE stage of the MN-major K tile (32 KB): 224 KB.
 constexpr int BKT = 64;
 constexpr uint32_t kTileQ = 2u * 2u * BKT * 128u;   // one streamed 64-row tile in one layout (32 KB)
-constexpr uint32_t kDqSmem = 1024u + kResBytes + 5u * kTileQ + 256u;
+constexpr uint32_t kDqSmem = 1024u + kResBytes + 5u * kTileQ + 256u + 512u;   // + the 128 row sums D
 //  MN-major 64-row tile (2 column groups of [hi|lo][64 rows][128 B]), contraction over the rows.
 __device__ __forceinline__ constexpr uint32_t mnmaj64_off(int ks, bool lo) {
     return (lo ? BKT * 128u : 0u) + (uint32_t)ks * 1024u;
@@ -581,7 +628,20 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             __syncwarp();
             if (lane == 0) mbar_arrive(q_ready);
         }
-        const float L = g.lse[lb + rc] * kLog2e, D = g.dvec[lb + rc];
+        // D = rowsum(dO o O) of the CTA's 128 rows: formed here by warpgroup 1, which has nothing
+        // else to do until its first tile, handed to warpgroup 0 through shared memory and left in
+        // global memory for the dkv kernel
+        float* dsm = reinterpret_cast<float*>(smem_raw + (bars + 256u - smem_u32(smem_raw)));
+        if (wg == 1) {
+            const int wrow0 = min(q0 + lane_group * 32, g.T - 1);
+            const long long off = (long long)(row_base + wrow0) * g.C + h * HD;
+            const float d = warp_rows_dot64(g.o_hi + off, g.o_lo ? g.o_lo + off : nullptr, g.do_hi + off,
+                                            g.do_hi + g.do_plane + off, g.C, max(1, min(32, g.T - wrow0)), lane);
+            dsm[lane_group * 32 + lane] = d;
+            if (row < g.T) g.dvec_out[lb + row] = d;
+        }
+        asm volatile("bar.sync 2, 256;" ::: "memory");    // the eight element-wise warps, exactly once
+        const float L = g.lse[lb + rc] * kLog2e, D = dsm[lane_group * 32 + lane];
         bool ok = true;
         int tn = 0;
         const uint32_t tb = tbuf(wg) + t_lane;
@@ -657,12 +717,14 @@ cudaError_t attention_tc_default_err(int** out);
 // Rows of the optional row-group sums array: one per 32 rows of every 128-row block.
 int64_t attention_bwd_rowgroups(int B, int T) { return (int64_t)B * 4 * ((T + BR - 1) / BR); }
 
-// dqkv (hi/lo planes) from qkv (hi/lo planes), dO (hi/lo planes), lse and dvec = rowsum(dO o O).
+// dqkv (hi/lo planes) from qkv (hi/lo planes), dO (hi/lo planes), O (raw, or hi/lo planes) and lse;
+// dvec [B, H, T] receives rowsum(dO o O) on the way.
 // rg_sums (nullable, [attention_bwd_rowgroups][3C]): column sums of dqkv per 32-row group; summing
 // its rows gives the gradient of the QKV bias without another pass over dqkv.
 cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, const float* do_hi, int64_t do_plane,
-                                    const float* lse, const float* dvec, int B, int T, int C, int H, float* dqkv_hi,
-                                    int64_t dqkv_plane, float* rg_sums, int* err_word, cudaStream_t s) {
+                                    const float* o, const float* o_lo, const float* lse, float* dvec, int B, int T,
+                                    int C, int H, float* dqkv_hi, int64_t dqkv_plane, float* rg_sums, int* err_word,
+                                    cudaStream_t s) {
     static cudaError_t attr = []() {
         cudaError_t e = cudaFuncSetAttribute(attn_bwd_dkv_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)kDkvSmem);
@@ -685,12 +747,13 @@ cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, cons
     ok = ok && enc3(&qk64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, false) &&  // 64-row K-major / MN-major tiles of qkv
          enc3(&qm64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, true);
     if (!ok) return cudaErrorInvalidValue;
-    BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dqkv_hi, dqkv_plane, err_word, attention_tc_get_trace(), rg_sums,
-              4 * ((T + BR - 1) / BR)};
+    BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dvec, o, o_lo, do_hi, do_plane, dqkv_hi, dqkv_plane, err_word,
+              attention_tc_get_trace(), rg_sums, 4 * ((T + BR - 1) / BR)};
     dim3 gk(B * H, (T + BR - 1) / BR);
-    BT_KERNEL_LAUNCH((attn_bwd_dkv_tc_kernel), gk, kThreads, kDkvSmem, s, qk64, qm64, dok64, dom64, vres, g);
-    BT_COUNT_LAUNCH();
+    // the dq kernel goes first: it also forms D = rowsum(dO o O), which the dkv kernel reads
     BT_KERNEL_LAUNCH((attn_bwd_dq_tc_kernel), gk, kThreads, kDqSmem, s, qk64, qm64, qk64, dores, g);
+    BT_COUNT_LAUNCH();
+    BT_KERNEL_LAUNCH((attn_bwd_dkv_tc_kernel), gk, kThreads, kDkvSmem, s, qk64, qm64, dok64, dom64, vres, g);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
