@@ -146,39 +146,75 @@ cudaError_t launch_embedding_fwd(const int32_t* tok, const float* wte, const flo
 // later positions with that id, in ascending order, and adds the row sum to dwte[id,:]; all
 // other CTAs exit.  One writer per row and a fixed order: deterministic, no atomics, and the
 // heavy-tailed (Zipf) token distribution costs one long row sum instead of contended atomics.
+// Both scans read the token array four ids per thread (128-bit loads); a round of 1024 positions
+// without a match -- nearly all of them for a rare token -- costs one load and one barrier.
+constexpr int kEmbRound = 1024;   // positions per round: 256 threads x 4
+__device__ __forceinline__ int4 load_tok4(const int32_t* __restrict__ tok, int j, int lo, int hi, int fill, bool vec) {
+    // ids at positions j .. j+3; positions outside [lo, hi) read as `fill`
+    if (vec && j >= lo && j + 3 < hi) return *reinterpret_cast<const int4*>(tok + j);
+    int4 v;
+    v.x = (j >= lo && j < hi) ? tok[j] : fill;
+    v.y = (j + 1 >= lo && j + 1 < hi) ? tok[j + 1] : fill;
+    v.z = (j + 2 >= lo && j + 2 < hi) ? tok[j + 2] : fill;
+    v.w = (j + 3 >= lo && j + 3 < hi) ? tok[j + 3] : fill;
+    return v;
+}
 __global__ void __launch_bounds__(256) embedding_bwd_wte_kernel(const int32_t* __restrict__ tok,
                                                                 const float* __restrict__ dx, int N, int C4,
-                                                                float* __restrict__ dwte) {
+                                                                float* __restrict__ dwte, int vec) {
     pdl_wait();
     pdl_trigger();
     const int n = blockIdx.x;
     const int t = tok[n];
     int found = 0;
-    for (int j = threadIdx.x; j < n; j += blockDim.x) found |= (tok[j] == t);
+    for (int j = 4 * threadIdx.x; j < n; j += kEmbRound) {
+        const int4 v = load_tok4(tok, j, 0, n, ~t, vec != 0);
+        found |= (v.x == t) | (v.y == t) | (v.z == t) | (v.w == t);
+    }
     if (__syncthreads_or(found)) return;
 
-    __shared__ int list[256];
+    __shared__ int list[kEmbRound];
     __shared__ int wcount[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int a0 = n & ~3;   // rounds start on a multiple of four so that the 128-bit loads stay aligned
     for (int c0 = 0; c0 < C4; c0 += 256) {
         const int c = c0 + threadIdx.x;
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int base = n; base < N; base += 256) {
-            int j = base + threadIdx.x;
-            bool flag = (j < N) && (tok[j] == t);
-            unsigned b = __ballot_sync(0xffffffffu, flag);
-            if (lane == 0) wcount[warp] = __popc(b);
+        for (int base = a0; base < N; base += kEmbRound) {
+            const int j = base + 4 * threadIdx.x;
+            const int4 v = load_tok4(tok, j, n, N, ~t, vec != 0);
+            const int m = (v.x == t ? 1 : 0) | (v.y == t ? 2 : 0) | (v.z == t ? 4 : 0) | (v.w == t ? 8 : 0);
+            if (!__syncthreads_or(m)) continue;
+            // ordered list of the round's matches: thread order, then position inside the thread
+            const int cnt = __popc(m);
+            int pre = cnt;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const int y = __shfl_up_sync(0xffffffffu, pre, d);
+                if (lane >= d) pre += y;
+            }
+            if (lane == 31) wcount[warp] = pre;
             __syncthreads();
-            int off = 0, total = 0;
+            int off = pre - cnt, total = 0;
 #pragma unroll
             for (int k = 0; k < 8; ++k) {
                 if (k < warp) off += wcount[k];
                 total += wcount[k];
             }
-            if (flag) list[off + __popc(b & ((1u << lane) - 1u))] = j;
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (m & (1 << q)) list[off++] = j + q;
             __syncthreads();
-            if (c < C4) {
-                for (int k = 0; k < total; ++k) acc = add4(acc, ld4(dx, (int64_t)list[k] * C4 + c));
+            if (c < C4) {   // eight rows in flight (a frequent token has dozens per round), added in list order
+                int k = 0;
+                for (; k + 8 <= total; k += 8) {
+                    float4 r[8];
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) r[q] = ld4(dx, (int64_t)list[k + q] * C4 + c);
+#pragma unroll
+                    for (int q = 0; q < 8; ++q) acc = add4(acc, r[q]);
+                }
+                for (; k < total; ++k) acc = add4(acc, ld4(dx, (int64_t)list[k] * C4 + c));
             }
             __syncthreads();
         }
@@ -205,7 +241,8 @@ __global__ void __launch_bounds__(256) embedding_bwd_wpe_kernel(const float* __r
 
 cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, float* dwte,
                                  float* dwpe, cudaStream_t s) {
-    BT_KERNEL_LAUNCH((embedding_bwd_wte_kernel), (int)N, 256, 0, s, tok, dx, (int)N, C / 4, dwte);
+    const int vec = (reinterpret_cast<uintptr_t>(tok) & 15u) == 0 ? 1 : 0;
+    BT_KERNEL_LAUNCH((embedding_bwd_wte_kernel), (int)N, 256, 0, s, tok, dx, (int)N, C / 4, dwte, vec);
     BT_COUNT_LAUNCH();
     BT_KERNEL_LAUNCH((embedding_bwd_wpe_kernel), grid_for((int64_t)T * (C / 4), 256, kStreamGridCap), 256, 0, s, 
         dx, (int)(N / T), T, C / 4, dwpe);
