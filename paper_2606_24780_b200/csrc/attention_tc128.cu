@@ -11,15 +11,18 @@
 //     Out += Z B3            Z hi/lo written back to tensor memory, Out accumulates there
 //
 //   pass   rows (lanes)  A1   B1  A2   B2   f                          B3   Out
-//   LSE    queries       Q'   K   -    -    running max / sum -> lse   -    -
-//   FWD    queries       Q'   K   -    -    P = exp2(X - lse)          V    O
+//   MAX    queries       Q'   K   -    -    row maximum m (X in 1xTF32) -    -
+//   FWD    queries       Q'   K   -    -    P = exp2(X - m), l = sum P V    O = (P V) / l, lse = m + log l
 //   DQ     queries       Q'   K   dO   V    dS = P o (Y - D)           K    dQ (x 1/sqrt d)
 //   DK     keys          K'   Q   V    dO   dS^T = P^T o (Y - D)       Q    dK (x 1/sqrt d)
 //   DV     keys          K'   Q   -    -    P^T                        dO   dV
 //
-// (Q' = Q log2(e)/sqrt(d), K' likewise: X is the score in base-2 units.)  The forward runs LSE and
-// then FWD: with the row's log-sum-exp known, P is final when it is formed and O accumulates in
-// tensor memory like the backward's outputs, with no running-maximum rescaling.  The streamed
+// (Q' = Q log2(e)/sqrt(d), K' likewise: X is the score in base-2 units.)  The forward runs MAX and
+// then FWD.  MAX only has to find a reference value near each row's maximum, so it forms the scores
+// from the hi planes alone (one MMA per k-step instead of three); FWD then uses that reference for
+// every tile -- P needs no running-maximum rescaling, O accumulates in tensor memory like the
+// backward's outputs -- and normalises with the sum of the P it actually formed, so the result does
+// not depend on how exact the reference is.  The streamed
 // tiles B1, B2 (K-major, 128-byte swizzle) and B3 (MN-major, 128-byte swizzle with 32-byte atoms)
 // are 32 rows x 128 columns x (hi, lo) = 32 KB each.  With A2 resident (DQ, DK) every stream has
 // one buffer, refilled as soon as the one product that reads it has completed; the passes without
@@ -61,9 +64,9 @@ struct Args128 {
     long long a1_stride;      // row stride of that array in floats
     int a1_col;               // column of head 0 in it
     int a2_col, b1_col, b2_col, b3_col;   // column of head 0 in the arrays behind the tensor maps
-    const float* lse;         // [B, H, T], natural log (input of every pass but LSE)
+    const float* lse;         // [B, H, T], natural log (backward passes); FWD reads the MAX pass's reference
     const float* dvec;        // [B, H, T] rowsum(dO o O) (DQ, DK)
-    float* lse_out;           // LSE
+    float* lse_out;           // MAX: the row reference (base-2 units); FWD: the log-sum-exp
     float* out_raw;           // row-major outputs [B*T][out_stride], any may be null
     float* out_hi;
     float* out_lo;
@@ -191,9 +194,13 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
 #pragma unroll
                 for (int ks = 0; ks < 16; ++ks) {
                     const uint64_t b_hi = b1d.at(kmaj_off(BT_, ks, false)), b_lo = b1d.at(kmaj_off(BT_, ks, true));
-                    umma_tf32_ts(tX, tA1_lo + ks * 8, b_hi, idesc_x, ks > 0 ? 1u : 0u);
-                    umma_tf32_ts(tX, tA1_hi + ks * 8, b_lo, idesc_x, 1u);
-                    umma_tf32_ts(tX, tA1_hi + ks * 8, b_hi, idesc_x, 1u);
+                    if (PASS == P_LSE) {   // a reference near the row maximum: the hi planes suffice
+                        umma_tf32_ts(tX, tA1_hi + ks * 8, b_hi, idesc_x, ks > 0 ? 1u : 0u);
+                    } else {
+                        umma_tf32_ts(tX, tA1_lo + ks * 8, b_hi, idesc_x, ks > 0 ? 1u : 0u);
+                        umma_tf32_ts(tX, tA1_hi + ks * 8, b_lo, idesc_x, 1u);
+                        umma_tf32_ts(tX, tA1_hi + ks * 8, b_hi, idesc_x, 1u);
+                    }
                 }
                 umma_commit(bar(B1_EMPTY + st1));
                 if (kHasY) {
@@ -267,9 +274,10 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
         }
         const int rc = min(own, g.T - 1);
         float L = 0.f, D = 0.f;                           // query passes: this row's statistics
-        if (!kKeys && PASS != P_LSE) L = g.lse[lb + rc] * kLog2e;
+        if (PASS == P_FWD) L = g.lse[lb + rc];            // the MAX pass left the reference there, in base-2 units
+        if (PASS == P_DQ) L = g.lse[lb + rc] * kLog2e;
         if (PASS == P_DQ) D = g.dvec[lb + rc];
-        float m_run = -INFINITY, l_run = 0.f;             // LSE pass: running maximum / sum of this warpgroup's tiles
+        float m_run = -INFINITY, l_run = 0.f;             // MAX: maximum, FWD: sum of P, over this warpgroup's tiles
         bool ok = true;
         const uint32_t tb = tbuf(wg) + t_lane;
         for (int t = wg; t < n_t && ok; t += 2) {
@@ -296,13 +304,7 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
                     if (s0 + i > own) x[i] = 0xff800000u;            // key follows this query: -inf
                     mx = fmaxf(mx, __uint_as_float(x[i]));
                 }
-                const float m_new = fmaxf(m_run, mx);
-                const float m_use = (m_new == -INFINITY) ? 0.f : m_new;   // a fully masked tile keeps the arithmetic finite
-                float sum = 0.f;
-#pragma unroll
-                for (int i = 0; i < 32; ++i) sum += ex2_approx(__uint_as_float(x[i]) - m_use);
-                l_run = fmaf(l_run, ex2_approx(m_run - m_use), sum);
-                m_run = m_new;
+                m_run = fmaxf(m_run, mx);
             } else {
 #pragma unroll
                 for (int i = 0; i < 32; ++i) {
@@ -316,6 +318,7 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
                         p = live ? ex2_approx(__uint_as_float(x[i]) - L) : 0.f;
                     }
                     float z = p;
+                    if (PASS == P_FWD) l_run += p;
                     if (PASS == P_DQ) z = p * (__uint_as_float(y[i]) - D);
                     if (PASS == P_DK) z = p * (__uint_as_float(y[i]) - Dc[i]);
                     split_tf32_int(z, x[i], y[i]);
@@ -330,18 +333,23 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
         }
         // every product has completed, every load has landed: the stream buffers are free
         if (ok) ok = mbar_wait_warp(bar(ACC_FULL), 0, g.err, 60);
-        if (PASS == P_LSE) {
-            // warpgroup 1 hands its (max, sum) to warpgroup 0 through shared memory
-            float2* xch = reinterpret_cast<float2*>(smem_ptr(b1_s));
-            if (wg == 1 && ok) xch[rloc] = make_float2(m_run, l_run);
+        float out_mul = g.out_mul;
+        if (PASS == P_LSE || PASS == P_FWD) {
+            // the two warpgroups combine their maxima (MAX) or their sums of P (FWD) through shared memory
+            float* xch = reinterpret_cast<float*>(smem_ptr(b3_s));
+            xch[wg * BR + rloc] = (PASS == P_LSE) ? m_run : l_run;
             asm volatile("bar.sync 1, 256;" ::: "memory");             // all eight element-wise warps, exactly once
-            if (wg == 0 && ok && own < g.T) {
-                const float2 o = xch[rloc];
-                const float mm = fmaxf(m_run, o.x);                    // finite: tile 0 (key 0) belongs to warpgroup 0
-                const float l = l_run * ex2_approx(m_run - mm) + o.y * ex2_approx(o.x - mm);
-                g.lse_out[lb + own] = (mm + log2f(l)) * kLn2;
+            const float v0 = xch[rloc], v1 = xch[BR + rloc];
+            if (PASS == P_LSE) {
+                // finite: tile 0 (key 0) belongs to warpgroup 0
+                if (wg == 0 && ok && own < g.T) g.lse_out[lb + own] = fmaxf(v0, v1);
+            } else {
+                const float l = v0 + v1;                               // > 0: the diagonal term
+                out_mul *= 1.0f / l;
+                if (wg == 0 && ok && own < g.T) g.lse_out[lb + own] = (L + log2f(l)) * kLn2;
             }
-        } else if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
+        }
+        if (PASS != P_LSE && ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
             tc_fence_after();
             const int wrow0 = r0 + lane_group * 32;                    // first row of this warp
             const int nvalid = max(0, min(32, g.T - wrow0));
@@ -357,7 +365,7 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
                 tmem_ld_wait();
                 float v[32];
 #pragma unroll
-                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * g.out_mul;
+                for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * out_mul;
                 warp_rows_store(v, tile, lane, nvalid, g.out_raw ? g.out_raw + off0 + 32 * half : nullptr,
                                 g.out_hi ? g.out_hi + off0 + 32 * half : nullptr,
                                 g.out_lo ? g.out_lo + off0 + 32 * half : nullptr, g.out_stride,
@@ -427,7 +435,7 @@ cudaError_t launch_attention_fwd_tc128(const float* qkv_hi, int64_t qkv_plane, i
     dim3 grid(B * H, (T + BR - 1) / BR);
     BT_KERNEL_LAUNCH((attn128_kernel<P_LSE>), grid, kThreads, kSmem, s, kk, kk, kk, vm, g);
     BT_COUNT_LAUNCH();
-    g.lse = lse; g.lse_out = nullptr;
+    g.lse = lse;   // read (the reference) when a CTA starts, overwritten with the log-sum-exp when it ends
     g.out_raw = o; g.out_hi = o_hi; g.out_lo = o_lo; g.out_stride = C; g.out_col = 0; g.out_mul = 1.0f;
     BT_KERNEL_LAUNCH((attn128_kernel<P_FWD>), grid, kThreads, kSmem, s, kk, kk, kk, vm, g);
     BT_COUNT_LAUNCH();
