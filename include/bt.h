@@ -23,15 +23,22 @@
  *           a thread-local description of the last failure.  Kernels that wait on
  *           hardware barriers bound every wait; a wait that runs out sets a device
  *           error word that the next synchronising call reports as
- *           BT_ERR_DEVICE_TIMEOUT.
+ *           BT_ERR_DEVICE_TIMEOUT.  An error word is reported once and then cleared.
  * Split     The tensor-core GEMMs compute FP32 products as three TF32 products
  *           (a_hi*b_hi + a_hi*b_lo + a_lo*b_hi, FP32 accumulate).  Operands are therefore
  *           stored as two FP32 planes, `hi` = the value rounded to the nearest TF32 number
  *           (low 13 mantissa bits zero) and `lo` = value - hi (exact).  A "split" array of R x C values is
  *           [2][R][C]: plane 0 = hi, plane 1 = lo.  Kernels that produce GEMM operands
  *           can write the split form directly.
- * Tokens    Token and target ids must lie in [0, vocab_size); this is not checked on
- *           the device.
+ * Tokens    Token and target ids must lie in [0, vocab_size).  No kernel ever indexes
+ *           with an id outside that range: such an id is treated as id 0 and its
+ *           position is recorded in a device error word, which the next synchronising
+ *           call of the model (h_loss, h_grad_norm, bt_get_loss) reports as
+ *           BT_ERR_INVALID_ARG.  Entry points that receive the ids in HOST memory
+ *           (bt_train_step_host, the loader) check them before anything is enqueued.
+ *           With BT_FLAG_DEBUG in the configuration, or BT_DEBUG=1 in the environment,
+ *           bt_forward, bt_backward and bt_adamw_step synchronise before returning and
+ *           report any device error at the call that caused it.
  */
 #ifndef BT_H_
 #define BT_H_
@@ -74,7 +81,8 @@ enum {
     BT_FLAG_GEMM_SIMT = 2u,  /* plain FP32 FMA GEMM (bring-up reference) instead of tcgen05 */
     BT_FLAG_ATTN_SIMT = 4u,  /* plain FP32 FMA attention (bring-up reference) */
     BT_FLAG_GEMM_PAIR = 8u,  /* per-op GEMM calls: 256-row tiles on CTA pairs wherever M >= 256 */
-    BT_FLAG_GEMM_SINGLE = 16u /* per-op GEMM calls: 128-row tiles on single CTAs only (default: planner) */
+    BT_FLAG_GEMM_SINGLE = 16u, /* per-op GEMM calls: 128-row tiles on single CTAs only (default: planner) */
+    BT_FLAG_DEBUG = 32u       /* every step call synchronises and reports device errors (ids, waits) itself */
 };
 
 /* AdamW hyper-parameters (hyper-parameter table, "Optimization" column).  grad_clip <= 0
@@ -159,7 +167,9 @@ BT_API bt_status bt_train_step(bt_model* m, const int32_t* d_tokens, const int32
                                const bt_adamw_config* opt, float* h_loss);
 
 /* Same step with HOST token / target buffers (int32 [B, seq_len], pinned for a truly
- * asynchronous copy): the ids are copied into the workspace on the model's stream first. */
+ * asynchronous copy): the ids are checked against [0, vocab_size) on the host
+ * (BT_ERR_INVALID_ARG names the first offender; nothing is enqueued), then copied into the
+ * workspace on the model's stream. */
 BT_API bt_status bt_train_step_host(bt_model* m, const int32_t* h_tokens, const int32_t* h_targets,
                                     int32_t B, const bt_adamw_config* opt, float* h_loss);
 
@@ -190,30 +200,69 @@ typedef struct {
 } bt_lr_schedule;
 BT_API float bt_lr_at(const bt_lr_schedule* s, int64_t step);
 
-/* Double-buffered batch production (Algorithm 2).  The token stream is a list of shards (host
- * int32 arrays the caller keeps alive, e.g. memory-mapped files); rank r of `world` starts at
- * position B*T*r of shard 0, each batch is the window [pos, pos + B*T) as tokens and
- * [pos + 1, pos + B*T + 1) as targets, pos advances by B*T*world, and the next shard is opened when
- * fewer than B*T + 1 tokens remain at pos (checked before a window is taken) or fewer than
- * B*T*world + 1 remain after the advance.  Every shard must hold at least B*T*world + 1 tokens.
- *   d_buffers: device, 4*B*T int32 (tokens/targets of the two channels), caller-owned;
+/* Prefetching batch production (Implementation, "Data Loader", Algorithm 2 "Double-Buffered Batch
+ * Production").  The token stream is a list of shards (host int32 arrays the caller keeps alive,
+ * e.g. memory-mapped files).  The algorithm fixes which windows a rank sees: rank r of `world`
+ * starts at position B*T*r of shard 0; each batch is the window [pos, pos + B*T) as tokens and
+ * [pos + 1, pos + B*T + 1) as targets; pos advances by B*T*world; the next shard is opened when
+ * fewer than B*T*world + 1 tokens remain after the advance.  Every shard must hold at least
+ * B*T*world + 1 tokens.  Here that sequence is computed in closed form (a rank takes
+ * max(1, floor((len - 1 - B*T*r) / (B*T*world))) windows from a shard of `len` tokens), and the
+ * two buffers of the algorithm are a ring of n_slots slots (2 <= n_slots <= 8; 2 is the paper's
+ * double buffering) with one "copy landed" and one "consumer done" event per slot:
+ *   d_buffers: device, n_slots * 2 * B*T int32 (tokens and targets of every slot), caller-owned;
  *   h_pinned:  page-locked host memory of the same size, or NULL: then windows are copied straight
  *              from the shards, synchronously, with identical results;
+ *   vocab_size: if > 0, every id is checked against [0, vocab_size) while it is staged; a window
+ *              with an id outside makes the staging call return BT_ERR_INVALID_ARG (shard and
+ *              position in bt_last_error()) and the loader unusable; 0 = unchecked;
  *   compute_stream: the stream the consumer (bt_train_step ...) runs on.
- * bt_loader_next returns device pointers to the next batch; the pointers stay valid until the
- * second following call.  The copy for the batch after next is already in flight on the loader's
- * own stream; events order the two streams in both directions.  Unlike the algorithm as printed,
- * the host also waits for the previous copy out of a pinned buffer before rewriting it (the host
- * may run ahead of the GPU).  bt_loader_plan is the cursor alone (host only): the shard index and
- * position of the first n_batches windows. */
+ * bt_loader_next hands out the oldest filled slot: device pointers to its tokens and targets and
+ * the slot number; the compute stream is made to wait for the slot's copy.  The first call stages
+ * all n_slots slots.  The pointers stay valid until the slot is released.
+ * bt_loader_release(slot): call it after the LAST kernel that reads the slot has been enqueued on
+ * the compute stream.  It records the slot's "consumer done" event there and immediately stages
+ * the next window into the slot on the loader's own stream, which waits for that event: a slot is
+ * never overwritten before its readers have finished, however far the host runs ahead, and the host
+ * never rewrites a staging buffer before the copy out of it has run.  With every slot lent out and
+ * none released, bt_loader_next returns BT_ERR_INVALID_ARG.
+ * bt_loader_plan is the window sequence alone (host only): the shard index and position of the
+ * first n_batches windows. */
 typedef struct bt_loader bt_loader;
 BT_API bt_status bt_loader_plan(const int64_t* shard_lens, int32_t n_shards, int32_t B, int32_t T, int32_t rank,
                                 int32_t world, int32_t n_batches, int32_t* out_shard, int64_t* out_pos);
 BT_API bt_status bt_loader_create(const int32_t* const* shards, const int64_t* shard_lens, int32_t n_shards,
-                                  int32_t B, int32_t T, int32_t rank, int32_t world, int32_t* d_buffers,
-                                  int32_t* h_pinned, void* compute_stream, bt_loader** out);
-BT_API bt_status bt_loader_next(bt_loader* loader, const int32_t** d_tokens, const int32_t** d_targets);
+                                  int32_t B, int32_t T, int32_t rank, int32_t world, int32_t vocab_size,
+                                  int32_t n_slots, int32_t* d_buffers, int32_t* h_pinned, void* compute_stream,
+                                  bt_loader** out);
+BT_API bt_status bt_loader_next(bt_loader* loader, const int32_t** d_tokens, const int32_t** d_targets,
+                                int32_t* slot);
+BT_API bt_status bt_loader_release(bt_loader* loader, int32_t slot);
 BT_API void bt_loader_destroy(bt_loader* loader);
+
+/* Position of the first id outside [0, vocab_size) in a HOST array of n ids, -1 if all are valid,
+ * -2 for bad arguments.  Host arithmetic only (what bt_train_step_host and the loader run). */
+BT_API int64_t bt_first_invalid_id(const int32_t* h_ids, int64_t n, int32_t vocab_size);
+
+/* Self-test of the error path of the bounded device-side waits (the paper's fault-handling layer
+ * is an operations subsystem; this covers only the library's own promise that a kernel never
+ * waits forever).  One warp runs the library's barrier wait, with limit_ms (0 < limit_ms <= 1000)
+ * as its limit, on a barrier nothing arrives at -- no copy or tensor-memory operation is in
+ * flight, the kernel returns normally -- and the call returns what the next synchronising call
+ * of a real step would: BT_ERR_DEVICE_TIMEOUT (bt_last_error() names code 900).  The model stays
+ * usable.  Synchronises the stream. */
+BT_API bt_status bt_selftest_bounded_wait(bt_model* m, float limit_ms);
+
+/* Measurement aid (Appendix "Hardware and Benchmarking Methodology" asks for measured, not
+ * nominal, peaks): n_ctas CTAs each issue `iters` tcgen05.mma.kind::tf32 instructions of
+ * M = 128, N = 256, K = 8 (operands in shared memory, two alternating accumulators) and store the
+ * SM clocks from first issue to last completion in d_clocks[cta] (device int64, -1 if the bounded
+ * completion wait ran out, which also sets *d_err (device int32, zeroed by the caller) to 901).
+ * 262,144 MACs per instruction / (clocks / iters) is the dense TF32 rate of one SM in MAC per
+ * clock; times 2 x SMs x SM clock it is the TF32 peak, and a third of that the 3xTF32 peak the
+ * GEMM roofline is scaled with.  Asynchronous; one CTA per SM when n_ctas <= the SM count. */
+BT_API bt_status bt_probe_tf32_mma_rate(int32_t n_ctas, int32_t iters, int64_t* d_clocks, int32_t* d_err,
+                                        void* stream);
 
 /* Synchronises and reads the loss of the last forward. */
 BT_API bt_status bt_get_loss(bt_model* m, float* h_loss);
@@ -242,22 +291,37 @@ BT_API bt_status bt_profile_read(bt_model* m, int32_t category, double* ms_total
  * -------------------------------------------------------------------------------- */
 
 /* x[n,:] = wte[tok[n],:] + wpe[n mod T,:], one IEEE single-precision add per element
- * (architecture caption: token + learned position embedding). */
+ * (Evaluation, GPT-2 architecture figure: token embedding plus learned position embedding feed the
+ * first decoder block).  wte has V rows; an id outside [0, V) is read as id 0 and its position + 1
+ * is stored in *d_bad (device int32, nullable, zeroed by the caller; first writer wins). */
 BT_API bt_status bt_op_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N,
-                                     int32_t T, int32_t C, float* x, void* stream);
+                                     int32_t T, int32_t C, int32_t V, float* x, int32_t* d_bad, void* stream);
 
-/* dwte[tok[n],:] += dx[n,:] summed in ascending n (deterministic); dwpe[t,:] = sum_b dx[b*T+t,:].
- * dwte is accumulated into (the tied LM-head gradient is already there), dwpe overwritten. */
+/* Backward of the above (Evaluation, GPT-2 architecture figure caption: the embeddings are
+ * weight-tied, so the gradient of the tied matrix is the LM-head part plus this scatter-add):
+ * dwte[tok[n],:] += dx[n,:] summed in ascending n; dwpe[t,:] = sum_b dx[b*T+t,:].
+ * dwte (V rows) is accumulated into (the tied LM-head gradient is already there), dwpe is
+ * overwritten.  Deterministic and free of atomics: positions are grouped by id inside chunks of
+ * 128 positions, one partial row per (chunk, id) is written to scratch, and the partial rows of an
+ * id are added in chunk order.  Ids outside [0, V) count as id 0 (as in the forward).
+ * scratch: device, bt_op_embedding_bwd_scratch_bytes(N, C, V) bytes, 256-byte aligned, caller-owned,
+ * contents irrelevant on entry.  N % T == 0, N <= 2^24. */
+BT_API size_t bt_op_embedding_bwd_scratch_bytes(int64_t N, int32_t C, int32_t V);
 BT_API bt_status bt_op_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int32_t T, int32_t C,
-                                     float* dwte, float* dwpe, void* stream);
+                                     int32_t V, float* dwte, float* dwpe, void* scratch, size_t scratch_bytes,
+                                     void* stream);
 
-/* y = gamma * (x - mean) * rstd + beta over the C features of each of N rows; biased
+/* LayerNorm forward (Kernel Design and Optimization: the memory-bound kernels, reductions kept
+ * inside a warp; Appendix "Performance Benchmarks", LayerNorm Forward):
+ * y = gamma * (x - mean) * rstd + beta over the C features of each of N rows; biased
  * variance, eps = 1e-5.  C % 4 == 0. */
 BT_API bt_status bt_op_layernorm_fwd(const float* x, const float* gamma, const float* beta, int64_t N,
                                      int32_t C, float* y, float* y_split, float* mean, float* rstd,
                                      void* stream);
 
-/* dx = rstd * (dxhat - mean_c dxhat - xhat * mean_c(dxhat * xhat)) [+ dres], dxhat = dy * gamma;
+/* LayerNorm backward (Appendix "Performance Benchmarks", LayerNorm Backward; the residual add is
+ * the pre-normalised block's skip connection of the GPT-2 architecture figure):
+ * dx = rstd * (dxhat - mean_c dxhat - xhat * mean_c(dxhat * xhat)) [+ dres], dxhat = dy * gamma;
  * dgamma = sum_n dy * xhat, dbeta = sum_n dy (overwritten, fixed summation order). */
 BT_API size_t bt_op_layernorm_bwd_scratch_bytes(int64_t N, int32_t C);
 BT_API bt_status bt_op_layernorm_bwd(const float* dy, const float* x, const float* gamma, const float* mean,
@@ -265,16 +329,17 @@ BT_API bt_status bt_op_layernorm_bwd(const float* dy, const float* x, const floa
                                      float* dx_split, float* dgamma, float* dbeta, void* scratch,
                                      size_t scratch_bytes, void* stream);
 /* The same, plus dx_colsum[C] (device) = the column sums of the dx written (residual included):
- * in the pre-LN block (Section 2) that dx is the gradient at a residual-stream position, so its
+ * in the pre-normalised decoder block (Evaluation, GPT-2 architecture figure caption) that dx is
+ * the gradient at a residual-stream position, so its
  * column sums are the bias gradient of the projection that wrote to that position.  Same scratch. */
 BT_API bt_status bt_op_layernorm_bwd_colsum(const float* dy, const float* x, const float* gamma, const float* mean,
                                             const float* rstd, const float* dres, int64_t N, int32_t C, float* dx,
                                             float* dx_split, float* dgamma, float* dbeta, float* dx_colsum,
                                             void* scratch, size_t scratch_bytes, void* stream);
 
-/* Dense FP32 GEMM with 3xTF32 split accumulation on the tensor cores (the paper's GEMM
- * library serves QKV, attention-output and MLP projections in all forward and backward
- * layouts):  D[M,N] = op(A) op(B) (+ bias[N]) (+ residual[M,N]).
+/* Dense FP32 GEMM with 3xTF32 split accumulation on the tensor cores (Implementation, "Native
+ * GEMM Library": one library serves the QKV, attention-output and MLP projections in all forward
+ * and backward layouts, including the irregular weight-gradient shapes):  D[M,N] = op(A) op(B) (+ bias[N]) (+ residual[M,N]).
  *   BT_GEMM_NT: A [M,K], B [N,K]   (forward:  Y  = X W^T)
  *   BT_GEMM_NN: A [M,K], B [K,N]   (backward: dX = dY W)
  *   BT_GEMM_TN: A [K,M], B [K,N]   (backward: dW = dY^T X)
@@ -284,7 +349,8 @@ BT_API bt_status bt_op_layernorm_bwd_colsum(const float* dy, const float* x, con
  * wave-model planner choose. */
 enum { BT_GEMM_NT = 0, BT_GEMM_NN = 1, BT_GEMM_TN = 2 };
 
-/* x_split[0][i] = hi(x[i]), x_split[1][i] = lo(x[i]) for n values (n % 4 == 0). */
+/* x_split[0][i] = hi(x[i]), x_split[1][i] = lo(x[i]) for n values (n % 4 == 0).  The paper has no
+ * counterpart: this is the operand format of the 3xTF32 products above. */
 BT_API bt_status bt_op_split(const float* x, int64_t n, float* x_split, void* stream);
 
 /* The GEMM as the training step calls it: operands already stored as hi/lo planes
@@ -298,8 +364,9 @@ BT_API bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int64_t 
                                   void* scratch, size_t scratch_bytes, uint32_t flags, void* stream);
 /* The same, and D_act_split [2][M][N] (device) receives the TF32 hi/lo planes of act(D) from the
  * same epilogue: act 0 = D itself, 1 = GELU(D) in the exact erf form, 2 = the tanh form.  The
- * training step uses it for the MLP up-projection (Section 2: h = m Wfc^T + b is kept for the
- * backward, g = GELU(h) is the next GEMM's operand). */
+ * training step uses it for the MLP up-projection (the GELU feed-forward sublayer of the GPT-2
+ * architecture figure: h = m Wfc^T + b is kept for the backward, g = GELU(h) is the next GEMM's
+ * operand). */
 BT_API bt_status bt_op_gemm_split_act(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
                                       const float* B_split, float* D, float* D_act_split, int32_t act,
                                       const float* bias, const float* residual, void* scratch,
@@ -313,7 +380,9 @@ BT_API bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K, con
                             float* D, const float* bias, const float* residual, void* scratch,
                             size_t scratch_bytes, uint32_t flags, void* stream);
 
-/* Causal multi-head self-attention over fused qkv [B*T, 3C] (columns q | k | v, head h at
+/* Attention forward (Kernel Design and Optimization: the compute-bound kernels, tensor cores with
+ * on-chip reuse of the score tiles; Appendix "Performance Benchmarks", Attention Forward, Causal=1).
+ * Causal multi-head self-attention over fused qkv [B*T, 3C] (columns q | k | v, head h at
  * columns h*d..(h+1)*d-1 of each part): o = softmax(q k^T / sqrt(d) + causal mask) v,
  * lse [B,H,T] = log of the softmax normaliser.  d = C/H in {16, 32, 64, 128}.
  * qkv_split (nullable) is the same array as hi/lo planes [2][B*T][3C]; when it is given and d is
@@ -323,7 +392,8 @@ BT_API bt_status bt_op_gemm(int32_t layout, int64_t M, int64_t N, int64_t K, con
 BT_API bt_status bt_op_attention_fwd(const float* qkv, const float* qkv_split, int32_t B, int32_t T, int32_t C,
                                      int32_t H, float* o, float* o_split, float* lse, uint32_t flags, void* stream);
 
-/* Backward of the above with recomputed probabilities: dV = P^T do, dP = do V^T,
+/* Attention backward (Appendix "Performance Benchmarks", Attention Backward, Causal=1), with
+ * recomputed probabilities: dV = P^T do, dP = do V^T,
  * dS = P o (dP - rowsum(do o o)), dq = dS k / sqrt(d), dk = dS^T q / sqrt(d).
  * scratch: B*H*T floats.  qkv and d_o may be given raw and/or as hi/lo planes (qkv_split
  * [2][B*T][3C], d_o_split [2][B*T][C]); with both split inputs, d = 64 or 128 and only dqkv_split
@@ -334,29 +404,36 @@ BT_API bt_status bt_op_attention_bwd(const float* qkv, const float* qkv_split, c
                                      int32_t H, float* dqkv, float* dqkv_split, void* scratch, size_t scratch_bytes,
                                      uint32_t flags, void* stream);
 
-/* y = GELU(x) (exact erf form, or tanh form), n % 4 == 0. */
+/* GELU forward (Appendix "Performance Benchmarks", GELU Forward; Kernel Design and Optimization:
+ * 128-bit accesses, one pass, no lossy approximation): y = GELU(x) in the exact erf form (or the
+ * tanh form), n % 4 == 0. */
 BT_API bt_status bt_op_gelu_fwd(const float* x, int64_t n, int32_t tanh_form, float* y, float* y_split,
                                 void* stream);
-/* dx = dy * GELU'(x). */
+/* GELU backward (Appendix "Performance Benchmarks", GELU Backward): dx = dy * GELU'(x). */
 BT_API bt_status bt_op_gelu_bwd(const float* x, const float* dy, int64_t n, int32_t tanh_form, float* dx,
                                 float* dx_split, void* stream);
 
 /* The same dx for x, dy of shape [N, C] (device), plus colsum[C] (device) = the column sums of
- * dx: the bias gradient of the linear layer that produced x (Section 2, backward of the MLP's
- * up-projection), taken in the pass that writes dx.  scratch: device,
+ * dx: the bias gradient of the linear layer that produced x (the MLP up-projection of the GELU
+ * feed-forward sublayer; Appendix "Performance Benchmarks", Reduce Sum Kernel, is the paper's
+ * stand-alone form of that sum), taken in the pass that writes dx.  scratch: device,
  * bt_op_colsum_scratch_bytes(N, C) bytes, caller-owned.  C % 4 == 0; summation order fixed. */
 BT_API bt_status bt_op_gelu_bwd_colsum(const float* x, const float* dy, int64_t N, int32_t C, int32_t tanh_form,
                                        float* dx, float* dx_split, float* colsum, void* scratch,
                                        size_t scratch_bytes, void* stream);
 
-/* Fused softmax cross-entropy over all Vp columns: losses[n] = logsumexp(logits[n,:]) -
- * logits[n, y_n]; dlogits = (softmax - onehot) * inv_count; loss_mean (1 float) =
- * inv_count * sum_n losses[n] in fixed order.  Vp % 4 == 0. */
+/* Fused softmax cross-entropy over all Vp columns (Appendix "Performance Benchmarks", Sparse
+ * Cross-Entropy Loss Forward and Backward, here one kernel; Algorithm 1's "cross-entropy against
+ * target"): losses[n] = logsumexp(logits[n,:]) - logits[n, y_n]; dlogits = (softmax - onehot) *
+ * inv_count; loss_mean (1 float) = inv_count * sum_n losses[n] in fixed order.  Vp % 4 == 0.
+ * A target outside [0, Vp) counts as class 0 and its row + 1 is stored in *d_bad (device int32,
+ * nullable, zeroed by the caller; first writer wins). */
 BT_API bt_status bt_op_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int32_t Vp,
                                     float inv_count, float* losses, float* loss_mean, float* dlogits,
-                                    float* dlogits_split, void* stream);
+                                    float* dlogits_split, int32_t* d_bad, void* stream);
 
-/* out[c] = sum_n x[n,c] (bias gradients), fixed summation order. */
+/* Column sums (Appendix "Performance Benchmarks", Reduce Sum Kernel; in the step: the bias
+ * gradients): out[c] = sum_n x[n,c], fixed summation order. */
 BT_API size_t bt_op_colsum_scratch_bytes(int64_t N, int32_t C);
 BT_API bt_status bt_op_colsum(const float* x, int64_t N, int32_t C, float* out, void* scratch,
                               size_t scratch_bytes, void* stream);
@@ -371,20 +448,24 @@ BT_API bt_status bt_op_colsum(const float* x, int64_t N, int32_t C, float* out, 
  * cudaFree or allocating library routine) and returns BT_ERR_UNSUPPORTED when
  * bt_op_colsum_scratch_bytes(N, C) exceeds that size (C > 98,304).
  * The first call on each device looks up the array's device address (cudaGetSymbolAddress, with
- * that device current) and caches it; make that first call before starting any stream capture.
+ * that device current) and caches it; that lookup may make the CUDA runtime load the library's
+ * device code onto the device, so make that first call at start-up, before any stream capture.
  * Every call on a device shares the one array and overwrites the part it uses, so calls that
  * may overlap on the GPU (different streams, no ordering between them) race; keep them on one
  * stream or order them with events.  Same result as bt_op_colsum, bit for bit. */
 BT_API size_t bt_op_colsum_static_max_floats(void);
 BT_API bt_status bt_op_colsum_static(const float* x, int64_t N, int32_t C, float* out, void* stream);
 
-/* out[0] = sqrt(sum g^2), out[1] = clip > 0 ? min(1, clip / (out[0] + 1e-6)) : 1. */
+/* Global gradient norm and clip factor (hyper-parameter table: "Gradient clip 1.0"; a reduce-sum
+ * over the whole gradient arena): out[0] = sqrt(sum g^2), out[1] = clip > 0 ?
+ * min(1, clip / (out[0] + 1e-6)) : 1. */
 BT_API size_t bt_op_grad_norm_scratch_bytes(int64_t n);
 BT_API bt_status bt_op_grad_norm(const float* g, int64_t n, float clip, float* out2, void* scratch,
                                  size_t scratch_bytes, void* stream);
 
-/* One AdamW update at step t >= 1 of n_tensors tensors in one launch (the paper's
- * horizontally fused multi-tensor optimizer).  h_p/h_g/h_m/h_v are HOST arrays of device
+/* One AdamW update at step t >= 1 of n_tensors tensors in one launch (Implementation,
+ * "Horizontal Tensor Fusion": the multi-tensor optimizer; Appendix "Performance Benchmarks", AdamW
+ * Optimizer Kernel).  h_p/h_g/h_m/h_v are HOST arrays of device
  * pointers, h_numel/h_decay host arrays; d_scale (nullable) is a device float multiplying
  * every gradient (the clip factor).  n_tensors <= 64 per call. */
 BT_API bt_status bt_op_adamw_multi(int32_t n_tensors, float* const* h_p, const float* const* h_g,

@@ -15,6 +15,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libbt.so")
 
 BT_FLAG_GELU_TANH, BT_FLAG_GEMM_SIMT, BT_FLAG_ATTN_SIMT, BT_FLAG_GEMM_PAIR, BT_FLAG_GEMM_SINGLE = 1, 2, 4, 8, 16
+BT_FLAG_DEBUG = 32
 BT_GEMM_NT, BT_GEMM_NN, BT_GEMM_TN = 0, 1, 2
 STATUS = {0: "BT_OK", 1: "BT_ERR_INVALID_ARG", 2: "BT_ERR_UNSUPPORTED", 3: "BT_ERR_OOM", 4: "BT_ERR_CUDA",
           5: "BT_ERR_DEVICE_TIMEOUT", 6: "BT_ERR_NOT_FOUND"}
@@ -63,9 +64,10 @@ _SIGNATURES = {
     "bt_lr_at": (_f, [ctypes.POINTER(bt_lr_schedule), _i64]),
     "bt_loader_plan": (_i32, [ctypes.POINTER(_i64), _i32, _i32, _i32, _i32, _i32, _i32, ctypes.POINTER(_i32),
                               ctypes.POINTER(_i64)]),
-    "bt_loader_create": (_i32, [ctypes.POINTER(_vp), ctypes.POINTER(_i64), _i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp,
-                                ctypes.POINTER(_vp)]),
-    "bt_loader_next": (_i32, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp)]),
+    "bt_loader_create": (_i32, [ctypes.POINTER(_vp), ctypes.POINTER(_i64), _i32, _i32, _i32, _i32, _i32, _i32, _i32,
+                                _vp, _vp, _vp, ctypes.POINTER(_vp)]),
+    "bt_loader_next": (_i32, [_vp, ctypes.POINTER(_vp), ctypes.POINTER(_vp), ctypes.POINTER(_i32)]),
+    "bt_loader_release": (_i32, [_vp, _i32]),
     "bt_loader_destroy": (None, [_vp]),
     "bt_get_loss": (_i32, [_vp, ctypes.POINTER(_f)]),
     "bt_launch_count": (_i64, [_vp]),
@@ -75,8 +77,12 @@ _SIGNATURES = {
     "bt_profile_category_name": (ctypes.c_char_p, [_i32]),
     "bt_profile_read": (_i32, [_vp, _i32, ctypes.POINTER(ctypes.c_double), ctypes.POINTER(_i64),
                                ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double)]),
-    "bt_op_embedding_fwd": (_i32, [_vp, _vp, _vp, _i64, _i32, _i32, _vp, _vp]),
-    "bt_op_embedding_bwd": (_i32, [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp]),
+    "bt_op_embedding_fwd": (_i32, [_vp, _vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp]),
+    "bt_op_embedding_bwd_scratch_bytes": (_sz, [_i64, _i32, _i32]),
+    "bt_op_embedding_bwd": (_i32, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _sz, _vp]),
+    "bt_first_invalid_id": (_i64, [_vp, _i64, _i32]),
+    "bt_selftest_bounded_wait": (_i32, [_vp, _f]),
+    "bt_probe_tf32_mma_rate": (_i32, [_i32, _i32, _vp, _vp, _vp]),
     "bt_op_layernorm_fwd": (_i32, [_vp, _vp, _vp, _i64, _i32, _vp, _vp, _vp, _vp, _vp]),
     "bt_op_layernorm_bwd_scratch_bytes": (_sz, [_i64, _i32]),
     "bt_op_layernorm_bwd": (_i32, [_vp] * 6 + [_i64, _i32] + [_vp] * 5 + [_sz, _vp]),
@@ -93,7 +99,7 @@ _SIGNATURES = {
     "bt_op_gelu_fwd": (_i32, [_vp, _i64, _i32, _vp, _vp, _vp]),
     "bt_op_gelu_bwd": (_i32, [_vp, _vp, _i64, _i32, _vp, _vp, _vp]),
     "bt_op_gelu_bwd_colsum": (_i32, [_vp, _vp, _i64, _i32, _i32, _vp, _vp, _vp, _vp, _sz, _vp]),
-    "bt_op_softmax_xent": (_i32, [_vp, _vp, _i64, _i32, _f, _vp, _vp, _vp, _vp, _vp]),
+    "bt_op_softmax_xent": (_i32, [_vp, _vp, _i64, _i32, _f, _vp, _vp, _vp, _vp, _vp, _vp]),
     "bt_op_colsum_scratch_bytes": (_sz, [_i64, _i32]),
     "bt_op_colsum": (_i32, [_vp, _i64, _i32, _vp, _vp, _sz, _vp]),
     "bt_op_colsum_static_max_floats": (_sz, []),
@@ -269,27 +275,33 @@ def bt_loader_plan(shard_lens, B, T, rank, world, n_batches):
 
 
 class Loader:
-    """Double-buffered batch production over host int32 token shards (CPU torch tensors, kept alive
-    here).  `next()` returns (tokens, targets) as device int32 tensors of shape [B, T]."""
+    """Prefetching batch production over host int32 token shards (CPU torch tensors, kept alive
+    here).  `next()` returns (tokens, targets, slot): device int32 tensors of shape [B, T] and the
+    ring slot they live in; call `release(slot)` after enqueuing the last kernel that reads them."""
 
-    def __init__(self, shards, B, T, rank=0, world=1, pinned=True, device="cuda", stream=None):
+    def __init__(self, shards, B, T, rank=0, world=1, pinned=True, vocab_size=0, n_slots=2, device="cuda",
+                 stream=None):
         self.shards = [s.contiguous() for s in shards]
         self.B, self.T = B, T
         n = len(self.shards)
         ptrs = (_vp * n)(*[s.data_ptr() for s in self.shards])
         lens = (_i64 * n)(*[s.numel() for s in self.shards])
-        self.d_buffers = torch.empty(4 * B * T, dtype=torch.int32, device=device)
-        self.h_pinned = torch.empty(4 * B * T, dtype=torch.int32).pin_memory() if pinned else None
+        self.d_buffers = torch.empty(2 * n_slots * B * T, dtype=torch.int32, device=device)
+        self.h_pinned = torch.empty(2 * n_slots * B * T, dtype=torch.int32).pin_memory() if pinned else None
         self.h = _vp()
-        _check(lib().bt_loader_create(ptrs, lens, n, B, T, rank, world, _ptr(self.d_buffers), _ptr(self.h_pinned),
-                                      _stream(stream), ctypes.byref(self.h)))
+        _check(lib().bt_loader_create(ptrs, lens, n, B, T, rank, world, vocab_size, n_slots, _ptr(self.d_buffers),
+                                      _ptr(self.h_pinned), _stream(stream), ctypes.byref(self.h)))
 
     def next(self):
-        x, y = _vp(), _vp()
-        _check(lib().bt_loader_next(self.h, ctypes.byref(x), ctypes.byref(y)))
+        x, y, slot = _vp(), _vp(), _i32()
+        _check(lib().bt_loader_next(self.h, ctypes.byref(x), ctypes.byref(y), ctypes.byref(slot)))
         base, n = self.d_buffers.data_ptr(), self.B * self.T
         ox, oy = (x.value - base) // 4, (y.value - base) // 4
-        return (self.d_buffers[ox:ox + n].view(self.B, self.T), self.d_buffers[oy:oy + n].view(self.B, self.T))
+        return (self.d_buffers[ox:ox + n].view(self.B, self.T), self.d_buffers[oy:oy + n].view(self.B, self.T),
+                int(slot.value))
+
+    def release(self, slot):
+        _check(lib().bt_loader_release(self.h, slot))
 
     def close(self):
         if self.h:
@@ -331,12 +343,44 @@ def bt_profile_read(model, cat):
 
 # ------------------------------------------------------------------ per-op calls
 
-def bt_op_embedding_fwd(tok, wte, wpe, N, T, C, x, stream=None):
-    _check(lib().bt_op_embedding_fwd(_ptr(tok), _ptr(wte), _ptr(wpe), N, T, C, _ptr(x), _stream(stream)))
+def bt_op_embedding_fwd(tok, wte, wpe, N, T, C, V, x, d_bad=None, stream=None):
+    _check(lib().bt_op_embedding_fwd(_ptr(tok), _ptr(wte), _ptr(wpe), N, T, C, V, _ptr(x), _ptr(d_bad), _stream(stream)))
 
 
-def bt_op_embedding_bwd(tok, dx, N, T, C, dwte, dwpe, stream=None):
-    _check(lib().bt_op_embedding_bwd(_ptr(tok), _ptr(dx), N, T, C, _ptr(dwte), _ptr(dwpe), _stream(stream)))
+def bt_op_embedding_bwd_scratch_bytes(N, C, V):
+    return int(lib().bt_op_embedding_bwd_scratch_bytes(N, C, V))
+
+
+def bt_op_embedding_bwd(tok, dx, N, T, C, V, dwte, dwpe, scratch, scratch_bytes, stream=None):
+    _check(lib().bt_op_embedding_bwd(_ptr(tok), _ptr(dx), N, T, C, V, _ptr(dwte), _ptr(dwpe), _ptr(scratch),
+                                     scratch_bytes, _stream(stream)))
+
+
+def bt_first_invalid_id(h_ids, vocab_size):
+    """Position of the first id outside [0, vocab_size) in a host int32 tensor, or -1 (host only)."""
+    if not isinstance(h_ids, torch.Tensor) or h_ids.is_cuda or h_ids.dtype != torch.int32 or not h_ids.is_contiguous():
+        raise TypeError("h_ids must be a contiguous int32 host tensor")
+    return int(lib().bt_first_invalid_id(h_ids.data_ptr(), h_ids.numel(), vocab_size))
+
+
+def bt_probe_tf32_mma_rate(n_ctas=148, iters=4000, stream=None):
+    """Clocks per tcgen05.mma.kind::tf32 (128 x 256 x 8) on every CTA's SM: (min, median, max) over
+    the CTAs.  262144 / clocks = dense TF32 MAC per clock per SM."""
+    clocks = torch.zeros(n_ctas, dtype=torch.int64, device="cuda")
+    err = torch.zeros(4, dtype=torch.int32, device="cuda")
+    for _ in range(2):                       # the first launch also loads the kernel
+        _check(lib().bt_probe_tf32_mma_rate(n_ctas, iters, _ptr(clocks), _ptr(err), _stream(stream)))
+    torch.cuda.synchronize()
+    if int(err[0]) != 0 or int(clocks.min()) < 0:
+        raise BtError(5, f"rate probe: a bounded wait ran out (code {int(err[0])})")
+    c = clocks.double() / iters
+    return float(c.min()), float(c.median()), float(c.max())
+
+
+def bt_selftest_bounded_wait(model, limit_ms):
+    """Runs the library's bounded barrier wait on a barrier nobody arrives at; raises BtError with
+    status BT_ERR_DEVICE_TIMEOUT once the limit has passed (the expected outcome)."""
+    _check(lib().bt_selftest_bounded_wait(model, limit_ms))
 
 
 def bt_op_layernorm_fwd(x, gamma, beta, N, C, y, y_split, mean, rstd, stream=None):
@@ -420,9 +464,10 @@ def bt_op_gelu_bwd_colsum(x, dy, N, C, tanh_form, dx, dx_split, colsum, scratch,
                                        _ptr(scratch), scratch_bytes, _stream(stream)))
 
 
-def bt_op_softmax_xent(logits, targets, N, Vp, inv_count, losses, loss_mean, dlogits, dlogits_split, stream=None):
+def bt_op_softmax_xent(logits, targets, N, Vp, inv_count, losses, loss_mean, dlogits, dlogits_split, d_bad=None,
+                       stream=None):
     _check(lib().bt_op_softmax_xent(_ptr(logits), _ptr(targets), N, Vp, inv_count, _ptr(losses), _ptr(loss_mean),
-                                    _ptr(dlogits), _ptr(dlogits_split), _stream(stream)))
+                                    _ptr(dlogits), _ptr(dlogits_split), _ptr(d_bad), _stream(stream)))
 
 
 def bt_op_colsum_scratch_bytes(N, C):

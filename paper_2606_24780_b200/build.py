@@ -12,8 +12,7 @@ BUILD = os.path.join(_HERE, "build")
 LIB = os.path.join(_HERE, "libbt.so")
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
-              "-Xcompiler", "-fPIC,-fvisibility=hidden", "--use_fast_math=false"]
-NVCC_FLAGS = [f for f in NVCC_FLAGS if f != "--use_fast_math=false"]
+              "-Xcompiler", "-fPIC,-fvisibility=hidden"]
 
 
 def _sources():

@@ -117,6 +117,8 @@ struct bt_model {
     size_t partial_floats;
     int* err_word;
     int32_t *tok_stage, *tgt_stage;
+    uint8_t* emb_table;   // [Vp][chunks] byte table of the embedding backward
+    bool debug_sync;      // BT_FLAG_DEBUG or BT_DEBUG=1: every step call synchronises and reports device errors
     int64_t step;
     int curB;
     const int32_t* cur_tok;
@@ -250,6 +252,7 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->err_word = b.take<int>(4);
     m->tok_stage = b.take<int32_t>(N);
     m->tgt_stage = b.take<int32_t>(N);
+    m->emb_table = b.take<uint8_t>(embedding_bwd_scratch_bytes(N, 0, (int)Vp));
     return (b.off + 255) & ~(size_t)255;
 }
 
@@ -342,12 +345,35 @@ cudaError_t gemm_raw(bt_model* m, int layout, int64_t M, int64_t N, int64_t K, S
     BT_STEP(BT_GEMM_CAT(gemm_is_fwd, layout), gemm_flops(M, N, K), gemm_bytes(M, N, K) + 8.0 * (M) * (N),       \
             gemm_raw(m, layout, M, N, K, A, B, D, bias, res, DS))
 
+// The device error words: [0] code of the first bounded wait that ran out, [1] position + 1 of a
+// token id outside [0, vocab_size), [2] row + 1 of a target id outside it.  Reading them
+// synchronises the stream; words that were set are reported once and cleared, so that the model
+// stays usable after the caller has dealt with the error.
 bt_status check_device_error(bt_model* m) {
-    int err = 0;
-    BT_CUDA(cudaMemcpyAsync(&err, m->err_word, sizeof(int), cudaMemcpyDeviceToHost, m->stream));
+    int err[4] = {0, 0, 0, 0};
+    BT_CUDA(cudaMemcpyAsync(err, m->err_word, sizeof(err), cudaMemcpyDeviceToHost, m->stream));
     BT_CUDA(cudaStreamSynchronize(m->stream));
-    if (err != 0) return fail(BT_ERR_DEVICE_TIMEOUT, "a bounded device-side wait ran out (code %d)", err);
-    return BT_OK;
+    if (err[0] == 0 && err[1] == 0 && err[2] == 0) return BT_OK;
+    BT_CUDA(cudaMemsetAsync(m->err_word, 0, sizeof(err), m->stream));
+    if (err[0] != 0) return fail(BT_ERR_DEVICE_TIMEOUT, "a bounded device-side wait ran out (code %d)", err[0]);
+    if (err[1] != 0)
+        return fail(BT_ERR_INVALID_ARG, "token id outside [0, %d) at position %d (treated as id 0)", m->V, err[1] - 1);
+    return fail(BT_ERR_INVALID_ARG, "target id outside [0, %d) at position %d (treated as id 0)", m->V, err[2] - 1);
+}
+
+// Position of the first id outside [0, vocab) in a host array, or -1.
+int64_t first_bad_id(const int32_t* ids, int64_t n, int32_t vocab) {
+    for (int64_t i = 0; i < n; ++i)
+        if ((uint32_t)ids[i] >= (uint32_t)vocab) return i;
+    return -1;
+}
+
+bool debug_env() {
+    static const bool on = []() {
+        const char* v = getenv("BT_DEBUG");
+        return v && v[0] != '\0' && v[0] != '0';
+    }();
+    return on;
 }
 
 }  // namespace
@@ -391,6 +417,7 @@ extern "C" bt_status bt_model_create(const bt_config* cfg, void* d_workspace, si
     m->launches_at_create = g_launches.load();
     m->prof_on = false;
     m->prof_used = 0;
+    m->debug_sync = (cfg->flags & BT_FLAG_DEBUG) != 0 || debug_env();
     std::vector<uint8_t> flags((size_t)(m->P / 1024), 0);
     for (const Tensor& t : m->tensors)
         if (t.decay)
@@ -564,7 +591,7 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
     BT_STEP(kCatSplit, 0, 20.0 * m->P, launch_split_matrices(m->params, m->wsplit, m->wsplit_t, m->P, m->mat_descs, m->n_mats,
                                   m->n_mat_tiles, s));
     BT_STEP(kCatEmbedFwd, N * C, 12.0 * N * C, launch_embedding_fwd(d_tokens, m->params + m->tensors[0].off, m->params + m->tensors[1].off, N, T, C,
-                                 m->act[0].x, s));
+                                 m->V, m->act[0].x, m->err_word + 1, s));
     for (int l = 0; l < m->L; ++l) {
         LayerAct& a = m->act[l];
         float* xout = (l + 1 < m->L) ? m->act[l + 1].x : m->xL;
@@ -591,11 +618,12 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
     BT_GEMM(kNN, N, Vp, C, act_mat(m->xf_s, N, C, N), weight_mat_t(m, m->tensors[0], Vp, C), m->logits, nullptr,
                  nullptr);
     BT_STEP(kCatXent, 0, 12.0 * N * Vp, launch_softmax_xent(m->logits, d_targets, N, Vp, 1.0f / (float)N, m->losses, m->loss, nullptr,
-                                m->dlogits_s, m->dlogits_s + N * Vp, s));
+                                m->dlogits_s, m->dlogits_s + N * Vp, m->V, m->err_word + 2, s));
     m->curB = B;
     m->cur_tok = d_tokens;
     m->have_forward = true;
     if (h_loss) return bt_get_loss(m, h_loss);
+    if (m->debug_sync) return check_device_error(m);
     return BT_OK;
 }
 
@@ -670,7 +698,9 @@ extern "C" bt_status bt_backward(bt_model* m) {
                                      l > 0 ? G(layer_tensor(m, l - 1, PRB)) : nullptr, m->ln_scratch, s));
     }
     // embeddings: dwte (already holding the LM-head part) += gather-transpose, dwpe = sum over sequences
-    BT_STEP(kCatEmbedBwd, 0, 8.0 * N * C, launch_embedding_bwd(m->cur_tok, m->dres, N, T, C, G(m->tensors[0]), G(m->tensors[1]), s));
+    BT_STEP(kCatEmbedBwd, 0, 8.0 * N * C, launch_embedding_bwd(m->cur_tok, m->dres, N, T, C, m->V, Vp, G(m->tensors[0]), G(m->tensors[1]),
+                                                              m->dtmp, m->emb_table, s));
+    if (m->debug_sync) return check_device_error(m);
     return BT_OK;
 }
 
@@ -690,6 +720,7 @@ extern "C" bt_status bt_adamw_step(bt_model* m, const bt_adamw_config* opt, floa
         BT_CUDA(cudaMemcpyAsync(h_grad_norm, m->norm_out, sizeof(float), cudaMemcpyDeviceToHost, s));
         return check_device_error(m);
     }
+    if (m->debug_sync) return check_device_error(m);
     return BT_OK;
 }
 
@@ -751,28 +782,64 @@ extern "C" bt_status bt_train_step_host(bt_model* m, const int32_t* h_tokens, co
     if (!m || !h_tokens || !h_targets) return fail(BT_ERR_INVALID_ARG, "NULL argument");
     if (B < 1 || B > m->maxB) return fail(BT_ERR_INVALID_ARG, "batch %d not in [1, %d]", B, m->maxB);
     const size_t bytes = (size_t)B * m->T * sizeof(int32_t);
+    // the ids are on the host here: check them before anything is enqueued
+    int64_t bad = first_bad_id(h_tokens, (int64_t)B * m->T, m->V);
+    if (bad >= 0) return fail(BT_ERR_INVALID_ARG, "token id %d outside [0, %d) at position %lld", h_tokens[bad], m->V, (long long)bad);
+    bad = first_bad_id(h_targets, (int64_t)B * m->T, m->V);
+    if (bad >= 0) return fail(BT_ERR_INVALID_ARG, "target id %d outside [0, %d) at position %lld", h_targets[bad], m->V, (long long)bad);
     BT_CUDA(cudaMemcpyAsync(m->tok_stage, h_tokens, bytes, cudaMemcpyHostToDevice, m->stream));
     BT_CUDA(cudaMemcpyAsync(m->tgt_stage, h_targets, bytes, cudaMemcpyHostToDevice, m->stream));
     return bt_train_step(m, m->tok_stage, m->tgt_stage, B, opt, h_loss);
 }
 
-// =============================================================================== per-op entry points
+extern "C" bt_status bt_selftest_bounded_wait(bt_model* m, float limit_ms) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    if (!(limit_ms > 0.f) || limit_ms > 1000.f) return fail(BT_ERR_INVALID_ARG, "limit_ms must lie in (0, 1000]");
+    BT_CUDA(launch_bounded_wait_probe(m->err_word, (unsigned long long)((double)limit_ms * 1e6), kSelftestWaitCode, m->stream));
+    return check_device_error(m);
+}
 
-extern "C" bt_status bt_op_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int32_t T,
-                                         int32_t C, float* x, void* stream) {
-    BT_PTR(tok); BT_PTR(wte); BT_PTR(wpe); BT_PTR(x);
-    if (N < 0 || T < 1 || C < 4 || C % 4) return fail(BT_ERR_INVALID_ARG, "embedding_fwd: bad sizes");
-    if (N == 0) return BT_OK;
-    BT_CUDA(launch_embedding_fwd(tok, wte, wpe, N, T, C, x, (cudaStream_t)stream));
+extern "C" bt_status bt_probe_tf32_mma_rate(int32_t n_ctas, int32_t iters, int64_t* d_clocks, int32_t* d_err,
+                                            void* stream) {
+    if (!d_clocks || !d_err) return fail(BT_ERR_INVALID_ARG, "probe: NULL argument");
+    if (reinterpret_cast<uintptr_t>(d_clocks) & 7u) return fail(BT_ERR_INVALID_ARG, "probe: d_clocks not 8-byte aligned");
+    if (n_ctas < 1 || n_ctas > 4096 || iters < 16 || iters > (1 << 20))
+        return fail(BT_ERR_INVALID_ARG, "probe: n_ctas in [1, 4096], iters in [16, 2^20]");
+    BT_CUDA(launch_tf32_rate_probe(n_ctas, iters, reinterpret_cast<long long*>(d_clocks), d_err, (cudaStream_t)stream));
     return BT_OK;
 }
 
-extern "C" bt_status bt_op_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int32_t T, int32_t C,
-                                         float* dwte, float* dwpe, void* stream) {
-    BT_PTR(tok); BT_PTR(dx); BT_PTR(dwte); BT_PTR(dwpe);
-    if (N < 1 || T < 1 || C < 4 || C % 4 || N % T || N > (1 << 24)) return fail(BT_ERR_INVALID_ARG, "embedding_bwd: bad sizes");
-    BT_CUDA(launch_embedding_bwd(tok, dx, N, T, C, dwte, dwpe, (cudaStream_t)stream));
+// =============================================================================== per-op entry points
+
+extern "C" bt_status bt_op_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int32_t T,
+                                         int32_t C, int32_t V, float* x, int32_t* d_bad, void* stream) {
+    BT_PTR(tok); BT_PTR(wte); BT_PTR(wpe); BT_PTR(x);
+    if (N < 0 || T < 1 || C < 4 || C % 4 || V < 1) return fail(BT_ERR_INVALID_ARG, "embedding_fwd: bad sizes");
+    if (N == 0) return BT_OK;
+    BT_CUDA(launch_embedding_fwd(tok, wte, wpe, N, T, C, V, x, d_bad, (cudaStream_t)stream));
     return BT_OK;
+}
+
+extern "C" size_t bt_op_embedding_bwd_scratch_bytes(int64_t N, int32_t C, int32_t V) {
+    if (N < 1 || C < 4 || V < 1) return 0;
+    return embedding_bwd_scratch_bytes(N, C, V);
+}
+
+extern "C" bt_status bt_op_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int32_t T, int32_t C, int32_t V,
+                                         float* dwte, float* dwpe, void* scratch, size_t scratch_bytes, void* stream) {
+    BT_PTR(tok); BT_PTR(dx); BT_PTR(dwte); BT_PTR(dwpe); BT_PTR(scratch);
+    if (N < 1 || T < 1 || C < 4 || C % 4 || N % T || N > (1 << 24) || V < 1)
+        return fail(BT_ERR_INVALID_ARG, "embedding_bwd: bad sizes");
+    if (scratch_bytes < embedding_bwd_scratch_bytes(N, C, V)) return fail(BT_ERR_OOM, "embedding_bwd: scratch too small");
+    const size_t partial_bytes = embedding_bwd_scratch_bytes(N, C, V) - (size_t)V * (size_t)((N + 127) / 128);
+    BT_CUDA(launch_embedding_bwd(tok, dx, N, T, C, V, V, dwte, dwpe, (float*)scratch, (uint8_t*)scratch + partial_bytes,
+                                 (cudaStream_t)stream));
+    return BT_OK;
+}
+
+extern "C" int64_t bt_first_invalid_id(const int32_t* h_ids, int64_t n, int32_t vocab_size) {
+    if ((!h_ids && n > 0) || n < 0 || vocab_size < 1) return -2;
+    return first_bad_id(h_ids, n, vocab_size);
 }
 
 extern "C" bt_status bt_op_layernorm_fwd(const float* x, const float* gamma, const float* beta, int64_t N, int32_t C,
@@ -1033,11 +1100,11 @@ extern "C" bt_status bt_op_gelu_bwd_colsum(const float* x, const float* dy, int6
 
 extern "C" bt_status bt_op_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int32_t Vp,
                                         float inv_count, float* losses, float* loss_mean, float* dlogits,
-                                        float* dlogits_split, void* stream) {
+                                        float* dlogits_split, int32_t* d_bad, void* stream) {
     BT_PTR(logits); BT_PTR(targets); BT_PTR(losses); BT_OPT_PTR(dlogits); BT_OPT_PTR(dlogits_split);
     if (N < 1 || Vp < 4 || Vp % 4 || N > (1 << 30)) return fail(BT_ERR_INVALID_ARG, "softmax_xent: bad sizes");
     BT_CUDA(launch_softmax_xent(logits, targets, N, Vp, inv_count, losses, loss_mean, dlogits, dlogits_split,
-                                dlogits_split ? dlogits_split + N * Vp : nullptr, (cudaStream_t)stream));
+                                dlogits_split ? dlogits_split + N * Vp : nullptr, Vp, d_bad, (cudaStream_t)stream));
     return BT_OK;
 }
 

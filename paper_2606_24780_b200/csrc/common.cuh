@@ -140,10 +140,13 @@ struct AdamParams {
 // All return cudaGetLastError() of their launches.
 
 cudaError_t launch_split(const float* x, float* hi, float* lo, int64_t n, cudaStream_t s);
+// Ids outside [0, V) are treated as id 0; position + 1 of one of them is left in *bad (nullable).
 cudaError_t launch_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int T,
-                                 int C, float* x, cudaStream_t s);
-cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, float* dwte,
-                                 float* dwpe, cudaStream_t s);
+                                 int C, int V, float* x, int* bad, cudaStream_t s);
+// partial: N*C floats; table: Vp * ceil(N / 128) bytes (both scratch, contents irrelevant on entry).
+size_t embedding_bwd_scratch_bytes(int64_t N, int C, int Vp);
+cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, int V, int Vp,
+                                 float* dwte, float* dwpe, float* partial, uint8_t* table, cudaStream_t s);
 cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float* beta, int64_t N, int C,
                                  float* y, float* y_hi, float* y_lo, float* mean, float* rstd, cudaStream_t s);
 size_t layernorm_bwd_scratch_floats(int64_t N, int C);
@@ -160,8 +163,8 @@ cudaError_t launch_gelu_bwd(const float* x, const float* dy, int64_t n, int tanh
 cudaError_t launch_gelu_bwd_colsum(const float* x, const float* dy, int64_t N, int C, int tanh_form, float* dx,
                                    float* dx_hi, float* dx_lo, float* colsum, float* scratch, cudaStream_t s);
 cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int Vp, float inv_count,
-                                float* losses, float* loss_mean, float* dl, float* dl_hi, float* dl_lo,
-                                cudaStream_t s);
+                                float* losses, float* loss_mean, float* dl, float* dl_hi, float* dl_lo, int V,
+                                int* bad, cudaStream_t s);
 size_t colsum_scratch_floats(int64_t N, int C);
 // x_lo (nullable): second plane added to the first (sums a split array).
 cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, float* out, float* scratch,
@@ -189,6 +192,11 @@ cudaError_t launch_adamw_multi(const AdamTensorList& tl, AdamParams hp, const fl
 cudaError_t launch_splitk_reduce(const float* partials, int splits, int64_t n, float* out, cudaStream_t s);
 cudaError_t launch_init_normal(float* p, int64_t n, float std, uint64_t seed, uint64_t offset, cudaStream_t s);
 cudaError_t launch_fill(float* p, int64_t n, float v, cudaStream_t s);
+// One warp waits (bounded by limit_ns) on a barrier nobody arrives at, then raises *err = code.
+constexpr int kSelftestWaitCode = 900;
+cudaError_t launch_bounded_wait_probe(int* err, unsigned long long limit_ns, int code, cudaStream_t s);
+// clocks[cta] = SM clocks that `iters` tcgen05.mma.kind::tf32 (128 x 256 x 8) took on that CTA's SM (-1: wait ran out).
+cudaError_t launch_tf32_rate_probe(int n_ctas, int iters, long long* clocks, int* err, cudaStream_t s);
 
 // SIMT reference GEMM: D = op(A) op(B) (+bias) (+residual), operands given as split planes
 // (lo may be absent: plane == 0 means "hi only").

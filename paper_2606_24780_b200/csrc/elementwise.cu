@@ -110,11 +110,19 @@ cudaError_t launch_split_matrices(const float* params, float* w_hi, float* wt_hi
 
 // ------------------------------------------------------------------ embedding forward
 
+// An id outside [0, V) is never used as an index: it is treated as id 0 and position + 1 is
+// recorded in *bad (first writer wins; bad may be null).
+__device__ __forceinline__ int checked_id(int id, int V, int64_t position, int* bad) {
+    if ((unsigned)id < (unsigned)V) return id;
+    if (bad) atomicCAS(bad, 0, (int)position + 1);
+    return 0;
+}
+
 // One thread per float4 of the output: x[n,:] = wte[tok[n],:] + wpe[n mod T,:].
 __global__ void __launch_bounds__(256) embedding_fwd_kernel(const int32_t* __restrict__ tok,
                                                             const float* __restrict__ wte,
                                                             const float* __restrict__ wpe, int64_t N, int T, int C4,
-                                                            float* __restrict__ x) {
+                                                            int V, float* __restrict__ x, int* bad) {
     pdl_wait();
     pdl_trigger();
     int64_t total = N * C4;
@@ -122,7 +130,8 @@ __global__ void __launch_bounds__(256) embedding_fwd_kernel(const int32_t* __res
          i += (int64_t)gridDim.x * blockDim.x) {
         int64_t n = i / C4;
         int c = (int)(i - n * C4);
-        float4 e = ld4(wte, (int64_t)tok[n] * C4 + c);
+        const int id = checked_id(tok[n], V, n, bad);
+        float4 e = ld4(wte, (int64_t)id * C4 + c);
         float4 p = ld4(wpe, (n % T) * C4 + c);
         float4 r;
         r.x = __fadd_rn(e.x, p.x);
@@ -134,93 +143,144 @@ __global__ void __launch_bounds__(256) embedding_fwd_kernel(const int32_t* __res
 }
 
 cudaError_t launch_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int T, int C,
-                                 float* x, cudaStream_t s) {
-    BT_KERNEL_LAUNCH((embedding_fwd_kernel), grid_for(N * (C / 4), 256, kStreamGridCap), 256, 0, s, tok, wte, wpe, N, T, C / 4, x);
+                                 int V, float* x, int* bad, cudaStream_t s) {
+    BT_KERNEL_LAUNCH((embedding_fwd_kernel), grid_for(N * (C / 4), 256, kStreamGridCap), 256, 0, s, tok, wte, wpe, N, T,
+                     C / 4, V, x, bad);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
 
 // ------------------------------------------------------------------ embedding backward
+//
+// dwte[id,:] += sum over the positions n with tok[n] == id of dx[n,:], in ascending n, without
+// atomics and with the work spread evenly although the ids are heavy-tailed (under a Zipf law one id
+// owns a seventh of all positions).  Two stages over chunks of kEmbChunk consecutive positions:
+//   1. one CTA per chunk groups the chunk's positions by id (all in shared memory), reads every row
+//      of dx exactly once, eight rows in flight, and writes one partial row per (chunk, id) group to
+//      `partial` at the slot of the group's first position; a byte table [Vp][chunks] records that
+//      position (offset in the chunk + 1, 0 = the id does not occur in the chunk);
+//   2. one CTA per eight ids reads their table rows; for an id that occurs it adds the partial rows
+//      of its chunks in ascending chunk order and then the sum to dwte[id,:].
+// Every CTA of stage 1 moves the same number of bytes; the longest serial chain of stage 2 is one
+// row per chunk.  The order of every addition is fixed by the positions alone.
+constexpr int kEmbChunk = 128;
 
-// One CTA per position n.  The CTA owning the FIRST occurrence of a token id gathers all
-// later positions with that id, in ascending order, and adds the row sum to dwte[id,:]; all
-// other CTAs exit.  One writer per row and a fixed order: deterministic, no atomics, and the
-// heavy-tailed (Zipf) token distribution costs one long row sum instead of contended atomics.
-// Both scans read the token array four ids per thread (128-bit loads); a round of 1024 positions
-// without a match -- nearly all of them for a rare token -- costs one load and one barrier.
-constexpr int kEmbRound = 1024;   // positions per round: 256 threads x 4
-__device__ __forceinline__ int4 load_tok4(const int32_t* __restrict__ tok, int j, int lo, int hi, int fill, bool vec) {
-    // ids at positions j .. j+3; positions outside [lo, hi) read as `fill`
-    if (vec && j >= lo && j + 3 < hi) return *reinterpret_cast<const int4*>(tok + j);
-    int4 v;
-    v.x = (j >= lo && j < hi) ? tok[j] : fill;
-    v.y = (j + 1 >= lo && j + 1 < hi) ? tok[j + 1] : fill;
-    v.z = (j + 2 >= lo && j + 2 < hi) ? tok[j + 2] : fill;
-    v.w = (j + 3 >= lo && j + 3 < hi) ? tok[j + 3] : fill;
-    return v;
-}
-__global__ void __launch_bounds__(256) embedding_bwd_wte_kernel(const int32_t* __restrict__ tok,
-                                                                const float* __restrict__ dx, int N, int C4,
-                                                                float* __restrict__ dwte, int vec) {
+__global__ void __launch_bounds__(256) embedding_bwd_group_kernel(const int32_t* __restrict__ tok,
+                                                                  const float* __restrict__ dx, int N, int C4, int V,
+                                                                  int n_chunks, float* __restrict__ partial,
+                                                                  uint8_t* __restrict__ table) {
     pdl_wait();
     pdl_trigger();
-    const int n = blockIdx.x;
-    const int t = tok[n];
-    int found = 0;
-    for (int j = 4 * threadIdx.x; j < n; j += kEmbRound) {
-        const int4 v = load_tok4(tok, j, 0, n, ~t, vec != 0);
-        found |= (v.x == t) | (v.y == t) | (v.z == t) | (v.w == t);
+    __shared__ int ids[kEmbChunk];      // id of position p of the chunk (-1 beyond N)
+    __shared__ int lead[kEmbChunk];     // first position of the chunk with the same id
+    __shared__ int order[kEmbChunk];    // positions sorted by (lead, position): the groups, concatenated
+    __shared__ int ends[kEmbChunk];     // 1 where a group ends in `order`
+    const int chunk = blockIdx.x, base = chunk * kEmbChunk, p = threadIdx.x;
+    const int nvalid = min(kEmbChunk, N - base);
+    if (p < kEmbChunk) ids[p] = p < nvalid ? checked_id(tok[base + p], V, base + p, nullptr) : -1;
+    __syncthreads();
+    if (p < kEmbChunk) {
+        int g = p;
+        const int id = ids[p];
+        for (int j = 0; j < p; ++j)
+            if (ids[j] == id) { g = j; break; }
+        lead[p] = g;
+        if (g == p && p < nvalid) table[(int64_t)id * n_chunks + chunk] = (uint8_t)(p + 1);
     }
-    if (__syncthreads_or(found)) return;
-
-    __shared__ int list[kEmbRound];
-    __shared__ int wcount[8];
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int a0 = n & ~3;   // rounds start on a multiple of four so that the 128-bit loads stay aligned
-    for (int c0 = 0; c0 < C4; c0 += 256) {
-        const int c = c0 + threadIdx.x;
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-        for (int base = a0; base < N; base += kEmbRound) {
-            const int j = base + 4 * threadIdx.x;
-            const int4 v = load_tok4(tok, j, n, N, ~t, vec != 0);
-            const int m = (v.x == t ? 1 : 0) | (v.y == t ? 2 : 0) | (v.z == t ? 4 : 0) | (v.w == t ? 8 : 0);
-            if (!__syncthreads_or(m)) continue;
-            // ordered list of the round's matches: thread order, then position inside the thread
-            const int cnt = __popc(m);
-            int pre = cnt;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const int y = __shfl_up_sync(0xffffffffu, pre, d);
-                if (lane >= d) pre += y;
-            }
-            if (lane == 31) wcount[warp] = pre;
-            __syncthreads();
-            int off = pre - cnt, total = 0;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) {
-                if (k < warp) off += wcount[k];
-                total += wcount[k];
-            }
-#pragma unroll
-            for (int q = 0; q < 4; ++q)
-                if (m & (1 << q)) list[off++] = j + q;
-            __syncthreads();
-            if (c < C4) {   // eight rows in flight (a frequent token has dozens per round), added in list order
-                int k = 0;
-                for (; k + 8 <= total; k += 8) {
-                    float4 r[8];
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) r[q] = ld4(dx, (int64_t)list[k + q] * C4 + c);
-#pragma unroll
-                    for (int q = 0; q < 8; ++q) acc = add4(acc, r[q]);
-                }
-                for (; k < total; ++k) acc = add4(acc, ld4(dx, (int64_t)list[k] * C4 + c));
-            }
-            __syncthreads();
+    __syncthreads();
+    if (p < nvalid) {
+        const int g = lead[p];
+        int slot = 0;
+        for (int q = 0; q < nvalid; ++q) {
+            const int gq = lead[q];
+            slot += (gq < g || (gq == g && q < p)) ? 1 : 0;
         }
-        if (c < C4) {
-            float4* dst = reinterpret_cast<float4*>(dwte) + (int64_t)t * C4 + c;
-            *dst = add4(*dst, acc);
+        order[slot] = p;
+    }
+    __syncthreads();
+    if (p < nvalid) ends[p] = (p == nvalid - 1 || lead[order[p + 1]] != lead[order[p]]) ? 1 : 0;
+    __syncthreads();
+    for (int c = threadIdx.x; c < C4; c += 256) {
+        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int i0 = 0; i0 < nvalid; i0 += 8) {
+            float4 r[8];
+#pragma unroll
+            for (int q = 0; q < 8; ++q)
+                if (i0 + q < nvalid) r[q] = ld4(dx, (int64_t)(base + order[i0 + q]) * C4 + c);
+#pragma unroll
+            for (int q = 0; q < 8; ++q) {
+                if (i0 + q < nvalid) {
+                    acc = add4(acc, r[q]);
+                    if (ends[i0 + q]) {
+                        reinterpret_cast<float4*>(partial)[(int64_t)(base + lead[order[i0 + q]]) * C4 + c] = acc;
+                        acc = make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                }
+            }
+        }
+    }
+}
+
+constexpr int kEmbIdsPerCta = 8;
+__global__ void __launch_bounds__(256) embedding_bwd_combine_kernel(const uint8_t* __restrict__ table, int n_chunks,
+                                                                    const float* __restrict__ partial, int C4, int Vp,
+                                                                    float* __restrict__ dwte) {
+    pdl_wait();
+    pdl_trigger();
+    __shared__ int present[kEmbIdsPerCta];
+    __shared__ int list[256];
+    __shared__ int wcount[8];
+    const int id0 = blockIdx.x * kEmbIdsPerCta;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (threadIdx.x < kEmbIdsPerCta) present[threadIdx.x] = 0;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < kEmbIdsPerCta; ++w) {
+        const int id = id0 + w;
+        if (id >= Vp) break;
+        int any = 0;
+        for (int k = threadIdx.x; k < n_chunks; k += 256) any |= table[(int64_t)id * n_chunks + k];
+        if (any) present[w] = 1;
+    }
+    __syncthreads();
+    for (int w = 0; w < kEmbIdsPerCta; ++w) {
+        if (!present[w]) continue;   // uniform over the CTA
+        const int id = id0 + w;
+        for (int c0 = 0; c0 < C4; c0 += 256) {
+            const int c = c0 + threadIdx.x;
+            float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int k0 = 0; k0 < n_chunks; k0 += 256) {
+                const int k = k0 + threadIdx.x;
+                const int b = k < n_chunks ? table[(int64_t)id * n_chunks + k] : 0;
+                // ordered list of the round's partial rows: chunk order = thread order
+                const unsigned bal = __ballot_sync(0xffffffffu, b != 0);
+                if (lane == 0) wcount[warp] = __popc(bal);
+                __syncthreads();
+                int off = __popc(bal & ((1u << lane) - 1u)), total = 0;
+#pragma unroll
+                for (int q = 0; q < 8; ++q) {
+                    if (q < warp) off += wcount[q];
+                    total += wcount[q];
+                }
+                if (b) list[off] = k * kEmbChunk + (b - 1);
+                __syncthreads();
+                if (c < C4) {
+                    int i = 0;
+                    for (; i + 8 <= total; i += 8) {
+                        float4 r[8];
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) r[q] = ld4(partial, (int64_t)list[i + q] * C4 + c);
+#pragma unroll
+                        for (int q = 0; q < 8; ++q) acc = add4(acc, r[q]);
+                    }
+                    for (; i < total; ++i) acc = add4(acc, ld4(partial, (int64_t)list[i] * C4 + c));
+                }
+                __syncthreads();
+            }
+            if (c < C4) {
+                float4* dst = reinterpret_cast<float4*>(dwte) + (int64_t)id * C4 + c;
+                *dst = add4(*dst, acc);
+            }
         }
     }
 }
@@ -239,12 +299,23 @@ __global__ void __launch_bounds__(256) embedding_bwd_wpe_kernel(const float* __r
     }
 }
 
-cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, float* dwte,
-                                 float* dwpe, cudaStream_t s) {
-    const int vec = (reinterpret_cast<uintptr_t>(tok) & 15u) == 0 ? 1 : 0;
-    BT_KERNEL_LAUNCH((embedding_bwd_wte_kernel), (int)N, 256, 0, s, tok, dx, (int)N, C / 4, dwte, vec);
+size_t embedding_bwd_scratch_bytes(int64_t N, int C, int Vp) {
+    const int64_t chunks = (N + kEmbChunk - 1) / kEmbChunk;
+    const size_t partial = ((size_t)N * C * sizeof(float) + 255) & ~(size_t)255;
+    return partial + (size_t)Vp * (size_t)chunks;
+}
+
+cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, int V, int Vp,
+                                 float* dwte, float* dwpe, float* partial, uint8_t* table, cudaStream_t s) {
+    const int chunks = (int)((N + kEmbChunk - 1) / kEmbChunk);
+    cudaError_t e = cudaMemsetAsync(table, 0, (size_t)Vp * chunks, s);
+    if (e != cudaSuccess) return e;
+    BT_KERNEL_LAUNCH((embedding_bwd_group_kernel), chunks, 256, 0, s, tok, dx, (int)N, C / 4, V, chunks, partial, table);
     BT_COUNT_LAUNCH();
-    BT_KERNEL_LAUNCH((embedding_bwd_wpe_kernel), grid_for((int64_t)T * (C / 4), 256, kStreamGridCap), 256, 0, s, 
+    BT_KERNEL_LAUNCH((embedding_bwd_combine_kernel), (Vp + kEmbIdsPerCta - 1) / kEmbIdsPerCta, 256, 0, s,
+                     (const uint8_t*)table, chunks, (const float*)partial, C / 4, Vp, dwte);
+    BT_COUNT_LAUNCH();
+    BT_KERNEL_LAUNCH((embedding_bwd_wpe_kernel), grid_for((int64_t)T * (C / 4), 256, kStreamGridCap), 256, 0, s,
         dx, (int)(N / T), T, C / 4, dwpe);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();

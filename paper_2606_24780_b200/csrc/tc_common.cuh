@@ -44,14 +44,17 @@ __device__ __forceinline__ unsigned long long globaltimer_ns() {
     asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
     return t;
 }
-// Bounded wait (about one second).  Returns false after raising the error word.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, int code) {
+// Bounded wait: gives up after limit_ns nanoseconds of the global timer (one second unless the
+// caller passes another limit).  Returns false after raising the error word.
+constexpr unsigned long long kWaitLimitNs = 1000000000ull;
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* err, int code,
+                                          unsigned long long limit_ns = kWaitLimitNs) {
     if (mbar_try_wait(bar, parity)) return true;
     const unsigned long long t0 = globaltimer_ns();
     for (;;) {
         for (int i = 0; i < 256; ++i)
             if (mbar_try_wait(bar, parity)) return true;
-        if (globaltimer_ns() - t0 > 1000000000ull) {
+        if (globaltimer_ns() - t0 > limit_ns) {
             atomicCAS(err, 0, code);  // the first wait that ran out is the one reported
             return false;
         }
@@ -60,8 +63,9 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
 
 // The same wait made by a whole warp, with a warp-uniform result: the callers go on to issue
 // .sync.aligned tensor-memory instructions, which every lane of the warp must reach together.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* err, int code) {
-    const bool ok = mbar_wait(bar, parity, err, code);
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* err, int code,
+                                               unsigned long long limit_ns = kWaitLimitNs) {
+    const bool ok = mbar_wait(bar, parity, err, code, limit_ns);
     return __all_sync(0xffffffffu, ok);
 }
 

@@ -23,11 +23,19 @@ __device__ __forceinline__ float block_reduce(float v, bool is_max, float* sm) {
     return r;
 }
 
+// A target outside [0, V) is never used as an index: it is treated as class 0 and row + 1 is
+// recorded in *bad (first writer wins; bad may be null).
+__device__ __forceinline__ int checked_target(int t, int V, int64_t row, int* bad) {
+    if ((unsigned)t < (unsigned)V) return t;
+    if (bad && threadIdx.x == 0) atomicCAS(bad, 0, (int)row + 1);
+    return 0;
+}
+
 template <int ITEMS>
 __global__ void __launch_bounds__(kXentThreads) xent_kernel(const float* __restrict__ logits,
                                                             const int32_t* __restrict__ targets, int V4,
                                                             float inv_count, float* __restrict__ losses, float* dl,
-                                                            float* dl_hi, float* dl_lo) {
+                                                            float* dl_hi, float* dl_lo, int V, int* bad) {
     pdl_wait();
     pdl_trigger();
     __shared__ float sm[kXentThreads / 32];
@@ -57,7 +65,7 @@ __global__ void __launch_bounds__(kXentThreads) xent_kernel(const float* __restr
         }
     }
     sum = block_reduce(sum, false, sm);
-    const int t = targets[row];
+    const int t = checked_target(targets[row], V, row, bad);
     if (threadIdx.x == 0) losses[row] = (mx + logf(sum)) - logits[row * V4 * 4 + t];
     if (dl == nullptr && dl_hi == nullptr) return;
     const float sc = inv_count / sum;
@@ -83,7 +91,8 @@ __global__ void __launch_bounds__(kXentThreads) xent_kernel(const float* __restr
 __global__ void __launch_bounds__(kXentThreads) xent_generic_kernel(const float* __restrict__ logits,
                                                                     const int32_t* __restrict__ targets, int V4,
                                                                     float inv_count, float* __restrict__ losses,
-                                                                    float* dl, float* dl_hi, float* dl_lo) {
+                                                                    float* dl, float* dl_hi, float* dl_lo, int V,
+                                                                    int* bad) {
     pdl_wait();
     pdl_trigger();
     __shared__ float sm[kXentThreads / 32];
@@ -101,7 +110,7 @@ __global__ void __launch_bounds__(kXentThreads) xent_generic_kernel(const float*
         sum += (expf(a.x - mx) + expf(a.y - mx)) + (expf(a.z - mx) + expf(a.w - mx));
     }
     sum = block_reduce(sum, false, sm);
-    const int t = targets[row];
+    const int t = checked_target(targets[row], V, row, bad);
     if (threadIdx.x == 0) losses[row] = (mx + logf(sum)) - logits[row * V4 * 4 + t];
     if (dl == nullptr && dl_hi == nullptr) return;
     const float sc = inv_count / sum;
@@ -137,19 +146,19 @@ __global__ void __launch_bounds__(1024) loss_mean_kernel(const float* __restrict
 }
 
 cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int Vp, float inv_count,
-                                float* losses, float* loss_mean, float* dl, float* dl_hi, float* dl_lo,
-                                cudaStream_t s) {
+                                float* losses, float* loss_mean, float* dl, float* dl_hi, float* dl_lo, int V,
+                                int* bad, cudaStream_t s) {
     const int V4 = Vp / 4;
     const int items = (V4 + kXentThreads - 1) / kXentThreads;
 #define BT_XENT(I)                                                                                              \
-    BT_KERNEL_LAUNCH((xent_kernel<I>), (int)N, kXentThreads, 0, s, logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo)
+    BT_KERNEL_LAUNCH((xent_kernel<I>), (int)N, kXentThreads, 0, s, logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo, V, bad)
     if (items <= 1) BT_XENT(1);
     else if (items <= 2) BT_XENT(2);
     else if (items <= 4) BT_XENT(4);
     else if (items <= 8) BT_XENT(8);
     else if (items <= 16) BT_XENT(16);
     else if (items <= 25) BT_XENT(25);
-    else BT_KERNEL_LAUNCH((xent_generic_kernel), (int)N, kXentThreads, 0, s, logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo);
+    else BT_KERNEL_LAUNCH((xent_generic_kernel), (int)N, kXentThreads, 0, s, logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo, V, bad);
 #undef BT_XENT
     BT_COUNT_LAUNCH();
     if (loss_mean) {

@@ -93,6 +93,28 @@ def build_cases(B, T, C, H, Vp, n_params):
         run=lambda: b.bt_op_layernorm_bwd(dy, x, g, mean, rstd, dres, N, C, dres, dxs, dg, db, lscr, lnb),
         bytes=24.0 * N * C, bound="hbm", keep=(dy, dres, dxs, dg, db, lscr))
 
+    dcs = torch.empty(C, device="cuda")
+    cases["layernorm_bwd_colsum"] = dict(          # the variant the training step runs (projection bias sums fused)
+        run=lambda: b.bt_op_layernorm_bwd_colsum(dy, x, g, mean, rstd, dres, N, C, dres, dxs, dg, db, dcs, lscr, lnb),
+        bytes=24.0 * N * C, bound="hbm", keep=(dcs,))
+
+    # embedding gather and its scatter-add backward on Zipf ids (the 124M vocabulary)
+    if Vp:
+        import seeded_inputs as si
+        V = 50257 if Vp == 50304 else Vp
+        tok = torch.as_tensor(si.zipf_tokens(7, B, T, V)[0].ravel()).cuda()
+        wte, wpe = _rand(Vp, C, std=0.02), _rand(T, C, std=0.02)
+        x0, dx0 = torch.empty(N, C, device="cuda"), _rand(N, C, std=1e-2)
+        dwte, dwpe = torch.zeros(Vp, C, device="cuda"), torch.empty(T, C, device="cuda")
+        esb = b.bt_op_embedding_bwd_scratch_bytes(N, C, Vp)
+        escr = torch.empty(esb + 256, dtype=torch.uint8, device="cuda")
+        escr = escr[(-escr.data_ptr()) % 256:]
+        cases["embedding_fwd"] = dict(run=lambda: b.bt_op_embedding_fwd(tok, wte, wpe, N, T, C, Vp, x0),
+                                      bytes=12.0 * N * C, bound="hbm", keep=(tok, wte, wpe, x0))
+        cases["embedding_bwd"] = dict(
+            run=lambda: b.bt_op_embedding_bwd(tok, dx0, N, T, C, Vp, dwte, dwpe, escr, esb),
+            bytes=8.0 * N * C, bound="hbm", keep=(dx0, dwte, dwpe, escr))
+
     # GELU
     h, dgl = _rand(N, F), _rand(N, F, std=1e-2)
     gs, dhs = torch.empty(2, N, F, device="cuda"), torch.empty(2, N, F, device="cuda")
@@ -163,7 +185,27 @@ def build_cases(B, T, C, H, Vp, n_params):
         out2 = torch.empty(2, device="cuda")
         cases["grad_norm"] = dict(run=lambda: b.bt_op_grad_norm(gr[0], shapes[0], 1.0, out2, nscr, gnb),
                                   bytes=4.0 * shapes[0], bound="hbm", keep=(nscr, out2))
+    if n_params:
+        # the optimizer and the weight split as the training step runs them (flat arenas of a model):
+        # one GPT-2-small layer plus the 50304-row embedding, 46 M parameters, batch 1 x 64 tokens so
+        # that the activations stay small
+        mdl = b.Model(1, C, H, 64, 50257 if Vp == 50304 else Vp, Vp, 1)
+        mdl.init(7)
+        opt2 = b.make_adamw()
+        tk = torch.zeros(1, 64, dtype=torch.int32, device="cuda")
+        mdl.train_step(tk, tk, opt2)
+        P = sum(-(-n // 1024) * 1024 for _, n, _ in mdl.names)
+        cases["model_adamw_step"] = dict(run=lambda: mdl.adamw_step(opt2, want_norm=False), bytes=(28.0 + 4.0) * P,
+                                         bound="hbm", keep=(mdl, tk))
+        cases["model_forward_64_tokens"] = dict(run=lambda: mdl.forward(tk, tk, want_loss=False), bytes=20.0 * P,
+                                                bound="hbm", keep=())
     return cases
+
+
+def tf32_rate(sm_mhz=None):
+    """The tensor pipe's measured dense TF32 rate (one SM): clocks per 128 x 256 x 8 MMA and MAC per clock."""
+    lo, med, hi = b.bt_probe_tf32_mma_rate(torch.cuda.get_device_properties(0).multi_processor_count, 4000)
+    return {"clocks_per_mma_128x256x8": med, "clocks_min_max": [lo, hi], "mac_per_clk_per_sm": 128 * 256 * 8 / med}
 
 
 def time_case(case, iters, warmup, flush_buf):
@@ -201,12 +243,21 @@ def main(argv=None):
     args = ap.parse_args(argv)
     torch.cuda.set_device(0)
     only = [s for s in args.only.split(",") if s]
-    need_big = not only or any(s.startswith(("gemm_fwd_lm", "gemm_nt_lm", "gemm_nn_dlm", "gemm_tn_wlm", "softmax", "adamw", "grad"))
+    need_big = not only or any(s.startswith(("gemm_fwd_lm", "gemm_nt_lm", "gemm_nn_dlm", "gemm_tn_wlm", "softmax", "adamw", "grad",
+                                          "embedding", "model_"))
                                for s in only)
     cases = build_cases(args.batch, args.seq, args.d_model, args.heads, args.vocab if need_big else 0,
                         args.params if need_big else 0)
     flush = None if args.no_flush else torch.zeros(64 * 1024 * 1024, device="cuda")  # 256 MB > 126 MB L2
     results = {}
+    if not only or "tf32_rate" in only:
+        r = tf32_rate()
+        sms = torch.cuda.get_device_properties(0).multi_processor_count
+        r["tf32_tflops_at_1965_mhz"] = r["mac_per_clk_per_sm"] * 2 * sms * 1.965e9 / 1e12
+        results["tf32_rate"] = r
+        print(f"tf32_rate              {r['clocks_per_mma_128x256x8']:10.1f} clk per 128x256x8 MMA  "
+              f"{r['mac_per_clk_per_sm']:7.0f} MAC/clk/SM  (x 2 x {sms} SMs x clock = dense TF32 peak; / 3 for 3xTF32)",
+              flush=True)
     for name, case in cases.items():
         if only and name not in only:
             continue

@@ -22,6 +22,10 @@ from gpu_util import dev, host, rel_l2, rel_max
 pytestmark = pytest.mark.gpu
 
 TOL_LOGITS, TOL_LOSS, TOL_GRAD, TOL_PARAM = 1e-4, 1e-4, 1e-3, 1e-5
+# an element whose parameter misses 1e-5 after AdamW must still have an accurate gradient: its difference from
+# the oracle's, relative to the RMS of the oracle's gradient over its tensor (the scale of the 1e-3 gradient
+# tolerance, applied here to single elements; the largest value measured on a B200 is 7.1e-4)
+OUTLIER_GRAD_TOL = 3e-3
 
 
 def make_pair(cfg, seed, flags, max_batch, jitter=0.02):
@@ -66,35 +70,61 @@ def compare_gradients(gm, om, cfg):
     return worst
 
 
-def adamw_step_and_compare(gm, om, step, max_outside=0.02):
+def adam_slope_bound(G1, G2, m0, v0, hp, t):
+    """Upper bound, per element, of |d u / d G| for u(G) = mhat / (sqrt(vhat) + eps) over every G
+    between G1 and G2 (m = b1 m0 + (1-b1) G, v = b2 v0 + (1-b2) G^2, bias-corrected), so that by the
+    mean-value theorem |u(G1) - u(G2)| <= bound * |G1 - G2|.
+
+    du/dG = [(1-b1)/c1 - R(G) * dsqrt(vhat)/dG] / (sqrt(vhat) + eps) with R = mhat / (sqrt(vhat) + eps);
+    dsqrt(vhat)/dG = (1-b2) G / (c2 sqrt(vhat)) <= sqrt((1-b2)/c2) because vhat >= (1-b2) G^2 / c2;
+    |R| <= b1 |m0| / (c1 (sqrt(b2 v0 / c2) + eps)) + (1-b1) sqrt(c2) / (c1 sqrt(1-b2)) for every G;
+    sqrt(vhat) is smallest at the G of the interval nearest to zero.  At t = 1 (m0 = v0 = 0) this
+    is 2 / (|G| + eps): the update lr * G / (|G| + eps) has slope lr / eps at G = 0."""
+    b1, b2, eps = hp["beta1"], hp["beta2"], hp["eps"]
+    c1, c2 = 1.0 - b1 ** t, 1.0 - b2 ** t
+    g_near = np.where(G1 * G2 > 0, np.minimum(np.abs(G1), np.abs(G2)), 0.0)
+    den = np.sqrt((b2 * v0 + (1 - b2) * g_near ** 2) / c2) + eps
+    r_max = b1 * np.abs(m0) / (c1 * (np.sqrt(b2 * v0 / c2) + eps)) + (1 - b1) * math.sqrt(c2) / (c1 * math.sqrt(1 - b2))
+    return ((1 - b1) / c1 + r_max * math.sqrt((1 - b2) / c2)) / den
+
+
+def adamw_step_and_compare(gm, om, step, max_outside=1e-4, stats=None):
     """One optimizer step on both sides from IDENTICAL state (p, m, v, t), two comparisons.
 
     (A) optimizer exactness: the oracle's AdamW applied to the GPU's own gradient must give the
         GPU's new parameters within 1e-5 absolute on EVERY element (and the moments within 1e-5
         relative L2).  This is the post-AdamW tolerance for the update itself.
-    (B) end to end against the oracle's own gradient: the update lr * mhat / (sqrt(vhat) + eps)
-        is ill-conditioned where an element's gradient history is ~0 (at t = 1 it is
-        lr * g / (|g| + eps): slope lr / eps = 6e4 at g = 0, so an FP32-rounding-sized gradient
-        error flips the whole +-lr step).  Elements outside 1e-5 must therefore be rare and
-        bounded by 2.2 lr; their count is reported.
+    (B) end to end against the oracle's own gradient, element by element.  The update
+        lr * mhat / (sqrt(vhat) + eps) is ill-conditioned where an element's gradient history is
+        ~0 (at t = 1 it is lr * G / (|G| + eps): slope lr / eps = 6e4 at G = 0, so an
+        FP32-rounding-sized gradient difference flips the whole +-lr step).  Every element must
+        satisfy |dp| <= 1e-5 + lr * slope * |G_gpu - G_ref| with `slope` the mean-value bound of
+        adam_slope_bound (G = clip scale * gradient): a parameter may miss 1e-5 only by what the
+        conditioning of ITS update explains.  For the elements that do miss it, the gradient
+        difference itself must be small against the RMS of the oracle's gradient over the
+        element's tensor (OUTLIER_GRAD_TOL), their fraction must stay under `max_outside` (about
+        ten times what was measured on a B200), and none moves by more than 2.2 lr.
     """
     hp = si.ADAMW
+    lr = hp["lr"]
     opt = b.make_adamw(**hp)
     names = om.names()
     g_gpu = {n: host(gm.tensor(n, 1)) for n in names}
+    g_ref = {n: om.get(n, 1).copy() for n in names}
     state = {n: (om.get(n, 0), om.get(n, 2), om.get(n, 3)) for n in names}
     gn_gpu_ref = oracle.grad_norm(list(g_gpu.values()))
     scale = oracle.clip_scale(gn_gpu_ref, hp["grad_clip"])
     gn = gm.adamw_step(opt)
-    ref_gn = om.adamw_step(hp["lr"], hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], hp["grad_clip"])
+    ref_gn = om.adamw_step(lr, hp["beta1"], hp["beta2"], hp["eps"], hp["weight_decay"], hp["grad_clip"])
+    ref_scale = oracle.clip_scale(ref_gn, hp["grad_clip"])
     # the norm is a gradient quantity: held to the gradient tolerance against the oracle's own
     # gradient, and to FP32 accuracy against the norm of the GPU's gradient
     assert abs(gn - ref_gn) < TOL_GRAD * ref_gn and abs(gn - gn_gpu_ref) < 1e-5 * gn_gpu_ref
     print(f"grad norm {gn:.6f} (oracle {ref_gn:.6f}, rel diff {(gn - ref_gn) / ref_gn:+.2e})")
-    total, outside, worst_a = 0, 0, 0.0
+    total, outside, worst_a, worst_used, worst_dg, worst_name = 0, 0, 0.0, 0.0, 0.0, "-"
     for n in names:
         p0, m0, v0 = state[n]
-        pb, mb, vb = oracle.adamw(p0, g_gpu[n], m0, v0, hp["lr"], hp["beta1"], hp["beta2"], hp["eps"],
+        pb, mb, vb = oracle.adamw(p0, g_gpu[n], m0, v0, lr, hp["beta1"], hp["beta2"], hp["eps"],
                                   hp["weight_decay"], om.decay(n), step + 1, scale)
         got = host(gm.tensor(n))
         da = np.abs(got - pb).max()
@@ -102,10 +132,31 @@ def adamw_step_and_compare(gm, om, step, max_outside=0.02):
         assert da < TOL_PARAM, (step, n, da)                                   # (A)
         assert rel_l2(host(gm.tensor(n, 2)), mb) < 1e-5 and rel_l2(host(gm.tensor(n, 3)), vb) < 1e-5, n
         db = np.abs(got - om.get(n))                                           # (B)
+        G1, G2 = scale * g_gpu[n], ref_scale * g_ref[n]
+        dG = np.abs(G1 - G2)
+        allowed = TOL_PARAM + lr * adam_slope_bound(G1, G2, m0, v0, hp, step + 1) * dG
+        bad = db > allowed
+        assert not bad.any(), (step, n, int(bad.sum()), float((db / allowed).max()))
+        out = db >= TOL_PARAM
         total += db.size
-        outside += int((db >= TOL_PARAM).sum())
-        assert db.max() <= 2.2 * hp["lr"], (step, n, db.max())
+        outside += int(out.sum())
+        assert db.max() <= 2.2 * lr, (step, n, db.max())
+        if out.any():
+            rms = math.sqrt(float((G2 ** 2).mean()))
+            assert rms > 0.0, (step, n)
+            rel = dG[out] / rms
+            if rel.max() > worst_dg:
+                k = int(rel.argmax())
+                worst_dg = float(rel.max())
+                worst_name = f"{n}[{np.flatnonzero(out)[k]}], |G| = {np.abs(G2[out][k]) / rms:.1e} RMS"
+            assert rel.max() <= OUTLIER_GRAD_TOL, (step, n, float(rel.max()))
+            worst_used = max(worst_used, float(((db[out] - TOL_PARAM) / (allowed[out] - TOL_PARAM)).max()))
+    print(f"post-AdamW: {outside} of {total} elements ({100.0 * outside / total:.4f}%) outside 1e-5, each within its "
+          f"conditioning bound (largest share of the bound used {worst_used:.2f}); their gradient differences are "
+          f"at most {worst_dg:.1e} of their tensor's RMS gradient ({worst_name})")
     assert outside <= max_outside * total, (step, outside, total)
+    if stats is not None:
+        stats.update(outside=outside, total=total, worst_bound_share=worst_used, worst_outlier_grad=worst_dg)
     # continue from identical state: the oracle adopts the GPU's FP32 parameters and moments
     for n in names:
         for kind in (0, 2, 3):
@@ -113,7 +164,7 @@ def adamw_step_and_compare(gm, om, step, max_outside=0.02):
     return outside / total, worst_a
 
 
-def run_steps(cfg, seed, flags, B, steps, chunk=0):
+def run_steps(cfg, seed, flags, B, steps, chunk=0, max_outside=1e-4):
     gm, om = make_pair(cfg, seed, flags, B)
     Vp = cfg["padded_vocab_size"]
     for step in range(steps):
@@ -128,7 +179,7 @@ def run_steps(cfg, seed, flags, B, steps, chunk=0):
             assert rel_max(got_logits, ref_logits) < TOL_LOGITS and rel_l2(got_logits, ref_logits) < TOL_LOGITS
         gm.backward()
         compare_gradients(gm, om, cfg)
-        frac, worst = adamw_step_and_compare(gm, om, step)
+        frac, worst = adamw_step_and_compare(gm, om, step, max_outside=max_outside)
         print(f"step {step}: loss {loss:.6f} (oracle {ref_loss:.6f}); AdamW exactness {worst:.2e}; "
               f"{100 * frac:.3f}% of parameters ill-conditioned")
         assert b.bt_get_step(gm.h) == step + 1
@@ -160,7 +211,7 @@ def test_medium_config_spans_tiles_and_ragged_tails():
     dimension, ragged M (B*T = 3*200 = 600 rows), Zipf tokens, head_dim 64."""
     cfg = si.make_config(n_layers=2, d_model=768, n_heads=12, seq_len=200, vocab_size=4000,
                          padded_vocab_size=4032, batch=3, tokens="zipf")
-    run_steps(cfg, seed=3, flags=0, B=3, steps=2)
+    run_steps(cfg, seed=3, flags=0, B=3, steps=2, max_outside=1e-3)     # measured 0.009 %
 
 
 def test_gpt2_124m_full_size_step():
@@ -189,7 +240,7 @@ def test_gpt2_124m_full_size_step():
     got_logits = host(gm.activation("logits")).reshape(-1, Vp)[(B - 1) * T:]
     assert rel_max(got_logits, ref_logits) < TOL_LOGITS and rel_l2(got_logits, ref_logits) < TOL_LOGITS
     worst = compare_gradients(gm, om, cfg)
-    frac, exact = adamw_step_and_compare(gm, om, 0, max_outside=0.05)
+    frac, exact = adamw_step_and_compare(gm, om, 0, max_outside=1e-3)
     print(f"worst gradient rel-L2 {worst:.2e}; AdamW exactness {exact:.2e}; {100 * frac:.2f}% of parameters "
           f"ill-conditioned at t = 1")
     gm.close()
@@ -218,6 +269,73 @@ def test_partial_batch_and_host_tokens():
     om.set_params(params)
     ref = om.loss_and_grad(tok, tgt)
     assert abs(results[0][0] - ref) < TOL_LOSS * ref
+
+
+def test_out_of_range_ids_surface_as_a_status():
+    """An id outside [0, vocab) never indexes memory: the host entry point refuses it before
+    anything is enqueued; the device-pointer entry points treat it as id 0 and the next
+    synchronising call returns BT_ERR_INVALID_ARG once (with BT_FLAG_DEBUG: the call that ran the
+    offending kernel does).  The model stays usable."""
+    cfg = si.config(0)
+    params = si.init_params(cfg, 5, jitter=0.02)
+    opt = b.make_adamw(**si.ADAMW)
+    tok, tgt = si.tokens_for(cfg, 5)
+    bad_tok, bad_tgt = tok.copy(), tgt.copy()
+    bad_tok[1, 7] = cfg["vocab_size"]
+    bad_tgt[2, 3] = -5
+    zero_tok = bad_tok.copy()
+    zero_tok[1, 7] = 0
+    for flags in (0, b.BT_FLAG_DEBUG):
+        gm = b.Model(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["seq_len"], cfg["vocab_size"],
+                     cfg["padded_vocab_size"], cfg["batch"], flags)
+        gm.load_params(params)
+        for ht, hy in ((bad_tok, tgt), (tok, bad_tgt)):
+            with pytest.raises(b.BtError) as e:
+                gm.train_step_host(torch.as_tensor(ht).pin_memory(), torch.as_tensor(hy).pin_memory(), opt)
+            assert e.value.status == 1 and "outside" in str(e.value)
+        assert b.bt_get_step(gm.h) == 0                      # nothing ran
+        with pytest.raises(b.BtError) as e:
+            if flags:
+                gm.forward(dev(bad_tok), dev(tgt), want_loss=False)     # debug: reported by the call itself
+            else:
+                gm.forward(dev(bad_tok), dev(tgt), want_loss=False)
+                gm.backward()
+                b.bt_get_loss(gm.h)                                      # release: by the next synchronising call
+        assert e.value.status == 1 and "token id" in str(e.value) and "position 71" in str(e.value)
+        loss_bad = b.bt_get_loss(gm.h)                                   # reported once, then cleared
+        assert loss_bad == gm.forward(dev(zero_tok), dev(tgt))           # the bad id was read as id 0
+        with pytest.raises(b.BtError) as e:
+            gm.forward(dev(tok), dev(bad_tgt))
+        assert e.value.status == 1 and "target id" in str(e.value)
+        om = oracle.Model(cfg)
+        om.set_params(params)
+        loss = gm.train_step(dev(tok), dev(tgt), opt)                    # and the model still trains
+        assert abs(loss - om.loss_and_grad(tok, tgt)) < TOL_LOSS * loss
+        gm.close()
+
+
+def test_bounded_wait_times_out_with_a_status():
+    """The path bounded wait -> device error word -> BT_ERR_DEVICE_TIMEOUT, driven by a kernel
+    that waits (for 2 ms) on a barrier nothing arrives at and then returns normally; the next step
+    on the same stream runs as usual."""
+    import time
+    cfg = si.config(0)
+    gm, om = make_pair(cfg, 5, 0, cfg["batch"])
+    tok, tgt = si.tokens_for(cfg, 5)
+    opt = b.make_adamw(**si.ADAMW)
+    t0 = time.time()
+    with pytest.raises(b.BtError) as e:
+        b.bt_selftest_bounded_wait(gm.h, 2.0)
+    assert e.value.status == 5 and "code 900" in str(e.value), str(e.value)
+    assert time.time() - t0 < 5.0
+    loss = gm.train_step(dev(tok), dev(tgt), opt)
+    assert abs(loss - om.loss_and_grad(tok, tgt)) < TOL_LOSS * loss
+    b.bt_get_loss(gm.h)                                                  # no stale error
+    for bad in (0.0, -1.0, 5000.0):
+        with pytest.raises(b.BtError) as e:
+            b.bt_selftest_bounded_wait(gm.h, bad)
+        assert e.value.status == 1
+    gm.close()
 
 
 def test_step_is_deterministic():
@@ -320,7 +438,7 @@ def test_wide_model_head_dim_128():
     the wide LayerNorm backward, head_dim-128 attention and K = 12,288 GEMMs in one step."""
     cfg = si.make_config(n_layers=1, d_model=3072, n_heads=24, seq_len=64, vocab_size=1000, padded_vocab_size=1024,
                          batch=2, tokens="zipf")
-    run_steps(cfg, seed=6, flags=0, B=2, steps=1)
+    run_steps(cfg, seed=6, flags=0, B=2, steps=1, max_outside=3e-3)     # measured 0.032 % (128 tokens, 117 M parameters)
 
 
 def test_350m_width_two_layers():
@@ -328,7 +446,26 @@ def test_350m_width_two_layers():
     context: the VPL = 8 LayerNorm instantiations and the 1024 / 4096-wide GEMM tilings in a step."""
     cfg = si.make_config(n_layers=2, d_model=1024, n_heads=16, seq_len=256, vocab_size=3000, padded_vocab_size=3072,
                          batch=2, tokens="zipf")
-    run_steps(cfg, seed=10, flags=0, B=2, steps=1)
+    run_steps(cfg, seed=10, flags=0, B=2, steps=1, max_outside=1.5e-3)    # measured 0.014 %
+
+
+def test_batch_32_full_context_zipf():
+    """The row count of BASELINE config 3 (B = 32 x T = 1024 = 32,768 token rows, Zipf ids) on one
+    GPT-2-small layer with a small vocabulary: the GEMM planner's choices for 32,768-row products,
+    a K = 32,768 weight-gradient reduction, and thousands of positions colliding on the rank-1
+    token's row in the embedding backward, in one step against the oracle (about a minute of
+    oracle time, processed eight sequences at a time)."""
+    cfg = si.make_config(n_layers=1, d_model=768, n_heads=12, seq_len=1024, vocab_size=4000, padded_vocab_size=4032,
+                         batch=32, tokens="zipf")
+    run_steps(cfg, seed=12, flags=0, B=32, steps=1, chunk=8, max_outside=1.5e-3)    # measured 0.013 %
+
+
+def test_350m_width_full_context():
+    """BASELINE config 4's width at its real context: d_model 1024, 16 heads of 64, MLP 4096,
+    T = 1024 (eight query blocks per head, 16 key tiles), one layer, one sequence."""
+    cfg = si.make_config(n_layers=1, d_model=1024, n_heads=16, seq_len=1024, vocab_size=3000, padded_vocab_size=3072,
+                         batch=1, tokens="zipf")
+    run_steps(cfg, seed=13, flags=0, B=1, steps=1, max_outside=1e-3)      # measured 0.008 %
 
 
 def test_wide_model_full_width_full_context():
@@ -338,7 +475,7 @@ def test_wide_model_full_width_full_context():
     of oracle time."""
     cfg = si.make_config(n_layers=2, d_model=3072, n_heads=24, seq_len=1024, vocab_size=2000, padded_vocab_size=2048,
                          batch=1, tokens="zipf")
-    run_steps(cfg, seed=9, flags=0, B=1, steps=1)
+    run_steps(cfg, seed=9, flags=0, B=1, steps=1, max_outside=5e-3)       # measured 0.057 % (1,024 tokens, 236 M parameters)
 
 
 def test_head_dim_128_model_with_several_query_blocks():
@@ -347,14 +484,16 @@ def test_head_dim_128_model_with_several_query_blocks():
     AdamW update against the oracle)."""
     cfg = si.make_config(n_layers=2, d_model=256, n_heads=2, seq_len=200, vocab_size=500, padded_vocab_size=512,
                          batch=2, tokens="zipf")
-    run_steps(cfg, seed=8, flags=0, B=2, steps=2)
+    run_steps(cfg, seed=8, flags=0, B=2, steps=2, max_outside=3e-4)       # measured 0.002 %
 
 
-@pytest.mark.parametrize("pinned", [True, False])
-def test_double_buffered_loader_feeds_the_step(pinned):
-    """Algorithm 2 on the GPU: batches arrive through the copy stream two channels deep; every batch
-    is bit-identical to the window the oracle's cursor names, for two interleaved ranks over three
-    shards with wrap-around, and the training step can consume them directly."""
+@pytest.mark.parametrize("pinned,n_slots", [(True, 2), (False, 2), (True, 4)])
+def test_prefetching_loader_feeds_the_step(pinned, n_slots):
+    """Algorithm 2 on the GPU: batches arrive through the copy stream, n_slots deep; every batch is
+    bit-identical to the window the oracle's step-by-step cursor names, for two interleaved ranks
+    over three shards with wrap-around; the training step consumes them directly; a slot is
+    rewritten only after its release, and asking for more than n_slots batches without a release
+    is refused."""
     cfg = si.config(0)
     B, T, world = 2, cfg["seq_len"], 2
     bt_ = B * T
@@ -362,13 +501,14 @@ def test_double_buffered_loader_feeds_the_step(pinned):
     lens = [bt_ * world * 3 + 1, bt_ * world + 7, bt_ * world * 2 + 1]
     shards = [rng.integers(0, cfg["vocab_size"], n).astype(np.int32) for n in lens]
     tshards = [torch.from_numpy(s) for s in shards]
-    loaders = [b.Loader(tshards, B, T, rank=r, world=world, pinned=pinned) for r in range(world)]
+    loaders = [b.Loader(tshards, B, T, rank=r, world=world, pinned=pinned, vocab_size=cfg["vocab_size"],
+                        n_slots=n_slots) for r in range(world)]
     want = [oracle.loader_windows(lens, B, T, r, world, 14) for r in range(world)]
     gm, om = make_pair(cfg, 3, 0, B)
     opt = b.make_adamw(**si.ADAMW)
     for i in range(14):
         for r in range(world):
-            x, y = loaders[r].next()
+            x, y, slot = loaders[r].next()
             s, p = want[r][i]
             assert np.array_equal(x.cpu().numpy().ravel(), shards[s][p:p + bt_])
             assert np.array_equal(y.cpu().numpy().ravel(), shards[s][p + 1:p + bt_ + 1])
@@ -381,9 +521,43 @@ def test_double_buffered_loader_feeds_the_step(pinned):
                 for n in om.names():
                     for kind in (0, 2, 3):
                         om.set_tensor(n, host(gm.tensor(n, kind)), kind)
+            loaders[r].release(slot)
+    # a lent slot keeps its contents until it is released, whatever else is produced meanwhile
+    held = [loaders[0].next() for _ in range(n_slots)]
+    kept = [(x.clone(), y.clone()) for x, y, _ in held]
+    with pytest.raises(b.BtError) as e:
+        loaders[0].next()
+    assert e.value.status == 1 and "release" in str(e.value)
+    for (x, y, slot), (kx, ky) in zip(held[1:], kept[1:]):
+        loaders[0].release(slot)
+    torch.cuda.synchronize()
+    assert torch.equal(held[0][0], kept[0][0]) and torch.equal(held[0][1], kept[0][1])
+    with pytest.raises(b.BtError):
+        loaders[0].release(held[1][2] if n_slots > 2 else 7)      # not lent out (refilled) / no such slot
     for L in loaders:
         L.close()
     gm.close()
+
+
+def test_loader_checks_ids_on_the_host():
+    """With a vocabulary size the loader validates every id while staging it: the window holding an
+    id outside [0, vocab) is never copied to the device and the call names shard and position."""
+    B, T = 2, 8
+    shard = np.arange(0, 200, dtype=np.int32) % 50
+    shard[70] = 50
+    ld = b.Loader([torch.from_numpy(shard)], B, T, vocab_size=50, n_slots=2)
+    x, y, slot = ld.next()                      # stages windows 0 and 1: positions 0..32, clean
+    assert np.array_equal(x.cpu().numpy().ravel(), shard[:16])
+    ld.release(slot)                            # stages window 2: positions 32..48, clean
+    x, y, slot = ld.next()
+    ld.release(slot)                            # window 3: 48..64 (+1), clean
+    x, y, slot = ld.next()
+    with pytest.raises(b.BtError) as e:
+        ld.release(slot)                        # window 4: 64..80 holds position 70
+    assert e.value.status == 1 and "position 70 of shard 0" in str(e.value)
+    with pytest.raises(b.BtError):
+        ld.next()                               # unusable from here on
+    ld.close()
 
 
 @pytest.mark.parametrize("L,C,H,T,V,B", [(1, 64, 4, 5, 40, 3), (1, 64, 1, 7, 36, 1), (2, 128, 2, 1, 32, 2),
@@ -393,4 +567,4 @@ def test_ragged_and_degenerate_shapes(L, C, H, T, V, B):
     length 1, where attention is the identity on v and the query / key gradients vanish exactly."""
     cfg = si.make_config(n_layers=L, d_model=C, n_heads=H, seq_len=T, vocab_size=V,
                          padded_vocab_size=(V + 31) // 32 * 32, batch=B, tokens="uniform")
-    run_steps(cfg, seed=4, flags=0, B=B, steps=2)
+    run_steps(cfg, seed=4, flags=0, B=B, steps=2, max_outside=1e-3)       # models of 14 K - 55 K parameters: a handful of elements

@@ -25,19 +25,26 @@ def test_embedding_fwd_bit_exact(B, T, C, V, zipf):
     wte, wpe = si.normal_f32(1, (V, C), 0.02), si.normal_f32(2, (T, C), 0.02)
     tok = (si.zipf_tokens(3, B, T, V) if zipf else si.uniform_tokens(3, B, T, V))[0]
     x = empty(B * T, C)
-    b.bt_op_embedding_fwd(dev(tok), dev(wte), dev(wpe), B * T, T, C, x)
+    b.bt_op_embedding_fwd(dev(tok), dev(wte), dev(wpe), B * T, T, C, V, x)
     ref = oracle.embedding_fwd(tok, wte, wpe, T, round_fp32=True).astype(np.float32)
     got = x.cpu().numpy()
     assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
 
 
-@pytest.mark.parametrize("B,T,C,V,zipf", [(4, 64, 64, 512, False), (8, 300, 768, 50257, True), (2, 513, 128, 7, False)])
+@pytest.mark.parametrize("B,T,C,V,zipf", [(4, 64, 64, 512, False), (8, 300, 768, 50257, True), (2, 513, 128, 7, False),
+                                          (32, 1024, 768, 50257, True), (1, 5, 2048, 3, False), (3, 128, 64, 1, False)])
 def test_embedding_bwd(B, T, C, V, zipf):
+    """Chunks of 128 positions with a ragged last chunk, ids that collide inside a chunk and across
+    chunks (V = 7, 3, 1), more than 256 float4 columns (C = 2048), and BASELINE config 3's token
+    count with Zipf ids (thousands of positions on the most frequent id's row)."""
     tok = (si.zipf_tokens(5, B, T, V) if zipf else si.uniform_tokens(5, B, T, V))[0]
     dx = si.normal_f32(6, (B * T, C), 1e-2)
     base = si.normal_f32(7, (V, C), 1e-2)          # the LM-head gradient already in dwte
     dwte, dwpe = dev(base), empty(T, C)
-    b.bt_op_embedding_bwd(dev(tok), dev(dx), B * T, T, C, dwte, dwpe)
+    nbytes = b.bt_op_embedding_bwd_scratch_bytes(B * T, C, V)
+    sc = scratch(nbytes)
+    sc.fill_(0xAB)                                  # the scratch's previous contents must not matter
+    b.bt_op_embedding_bwd(dev(tok), dev(dx), B * T, T, C, V, dwte, dwpe, sc, nbytes)
     rw, rp = oracle.embedding_bwd(tok, dx, T, V)
     assert rel_l2(host(dwte), rw + base) < 1e-5
     assert rel_l2(host(dwpe), rp) < 1e-5
@@ -46,8 +53,47 @@ def test_embedding_bwd(B, T, C, V, zipf):
         assert np.array_equal(dwte.cpu().numpy()[untouched], base[untouched])
     # deterministic: a second run gives identical bits
     dwte2, dwpe2 = dev(base), empty(T, C)
-    b.bt_op_embedding_bwd(dev(tok), dev(dx), B * T, T, C, dwte2, dwpe2)
+    b.bt_op_embedding_bwd(dev(tok), dev(dx), B * T, T, C, V, dwte2, dwpe2, sc, nbytes)
     assert torch.equal(dwte, dwte2) and torch.equal(dwpe, dwpe2)
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_embedding_bwd(dev(tok), dev(dx), B * T, T, C, V, dwte2, dwpe2, sc, nbytes - 1)
+    assert e.value.status == 3
+
+
+def test_out_of_range_ids_are_reported_and_never_used_as_an_index():
+    """Ids outside [0, V) (negative, V itself, far beyond) are read as id 0 by the gather, by its
+    backward and by the loss, and their position is left in the caller's error word."""
+    B, T, C, V = 2, 70, 64, 50
+    wte, wpe = si.normal_f32(1, (V, C), 0.02), si.normal_f32(2, (T, C), 0.02)
+    tok = si.uniform_tokens(3, B, T, V)[0]
+    bad_tok = tok.copy().ravel()
+    bad_tok[[5, 77, 139]] = [V, -1, 2 ** 30]
+    clean = bad_tok.copy()
+    clean[[5, 77, 139]] = 0
+    x, x_ref = empty(B * T, C), empty(B * T, C)
+    flag = zeros(4, dtype=torch.int32)
+    b.bt_op_embedding_fwd(dev(bad_tok), dev(wte), dev(wpe), B * T, T, C, V, x, flag)
+    b.bt_op_embedding_fwd(dev(clean), dev(wte), dev(wpe), B * T, T, C, V, x_ref, flag[1:])
+    assert torch.equal(x, x_ref)
+    assert int(flag[0]) - 1 in (5, 77, 139) and int(flag[1]) == 0
+    dx = si.normal_f32(6, (B * T, C), 1e-2)
+    nbytes = b.bt_op_embedding_bwd_scratch_bytes(B * T, C, V)
+    outs = []
+    for ids in (bad_tok, clean):
+        dwte, dwpe = zeros(V, C), empty(T, C)
+        b.bt_op_embedding_bwd(dev(ids), dev(dx), B * T, T, C, V, dwte, dwpe, scratch(nbytes), nbytes)
+        outs.append(dwte)
+    assert torch.equal(outs[0], outs[1])
+    z = si.normal_f32(23, (4, 64), 3.0)
+    y_bad, y_clean = np.array([3, 64, -7, 9], np.int32), np.array([3, 0, 0, 9], np.int32)
+    res = []
+    flag.zero_()
+    for i, y in enumerate((y_bad, y_clean)):
+        losses, dl = empty(4), empty(4, 64)
+        b.bt_op_softmax_xent(dev(z), dev(y), 4, 64, 0.25, losses, None, dl, None, flag[i:])
+        res.append((losses, dl))
+    assert torch.equal(res[0][0], res[1][0]) and torch.equal(res[0][1], res[1][1])
+    assert int(flag[0]) - 1 in (1, 2) and int(flag[1]) == 0
 
 
 # ------------------------------------------------------------------ LayerNorm
@@ -404,7 +450,7 @@ def test_empty_inputs_are_no_ops_or_rejected():
     x = empty(4)
     b.bt_op_gelu_fwd(x, 0, 0, x, None)
     b.bt_op_gelu_bwd(x, x, 0, 0, x, None)
-    b.bt_op_embedding_fwd(dev(np.zeros(1, np.int32)), x, x, 0, 1, 4, x)
+    b.bt_op_embedding_fwd(dev(np.zeros(1, np.int32)), x, x, 0, 1, 4, 1, x)
     b.bt_op_layernorm_fwd(x, x, x, 0, 4, x, None, x, x)
     for call in (lambda: b.bt_op_colsum(x, 0, 4, x, x, 1024),
                  lambda: b.bt_op_softmax_xent(x, dev(np.zeros(1, np.int32)), 0, 4, 1.0, x, None, None, None),

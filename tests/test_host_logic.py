@@ -78,6 +78,22 @@ def test_null_and_misaligned_arguments_are_rejected(lib):
     assert b.bt_op_layernorm_bwd_scratch_bytes(1000, 768) > 0
 
 
+def test_host_id_check(lib):
+    """bt_first_invalid_id is what bt_train_step_host and the loader run on ids that are still on the
+    host: the position of the first id outside [0, vocab), or -1."""
+    import torch
+    ids = torch.arange(0, 100, dtype=torch.int32)
+    assert b.bt_first_invalid_id(ids, 100) == -1
+    assert b.bt_first_invalid_id(ids, 99) == 99
+    assert b.bt_first_invalid_id(ids, 1) == 1
+    ids[17] = -1
+    assert b.bt_first_invalid_id(ids, 1000) == 17
+    ids[3] = 2 ** 31 - 1
+    assert b.bt_first_invalid_id(ids, 2 ** 31 - 1) == 3
+    assert b.bt_first_invalid_id(ids[:0], 5) == -1
+    assert lib.bt_first_invalid_id(None, 4, 5) == -2 and lib.bt_first_invalid_id(ids.data_ptr(), 4, 0) == -2
+
+
 def test_lr_schedule_matches_oracle():
     """bt_lr_at is host arithmetic: compared with the oracle's schedule on the paper's four numbers
     (max 6e-4, min 6e-5, warmup 715, 19,073 steps) and on degenerate schedules."""

@@ -40,6 +40,15 @@ def test_static_scratch_colsum_matches_scratch_entry_point_twice():
         ref = _reference(x, N, C)
         assert torch.equal(out, ref)                           # same kernels, same order: same bits
         assert rel_l2(host(out), host(x).sum(0)) < 1e-5
+        # torch's counter cannot see an allocation made inside the library; the driver's count of
+        # free device bytes can.  From the second call on (the first one on a device may load the
+        # library's module) a call must leave it exactly where it was.
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
+        b.bt_op_colsum_static(x, N, C, out)
+        torch.cuda.synchronize()
+        assert torch.cuda.mem_get_info()[0] == free_before
+        assert torch.equal(out, ref)
     # a repeat of the first shape after the second
     x = dev(si.normal_f32(99, (8192, 768), 1e-2))
     out = empty(768)
@@ -54,6 +63,15 @@ def test_static_scratch_colsum_rejects_oversized_and_bad_arguments():
     with pytest.raises(b.BtError) as e:
         b.bt_op_colsum_static(x, 64, 131072, empty(131072))
     assert e.value.status == 2 and "scratch" in str(e.value)
+    # the edge itself: 98,304 columns is the largest accepted width, the next multiple of four is refused
+    edge = b.bt_op_colsum_static_max_floats()
+    xe = dev(si.normal_f32(97, (64, edge), 1e-2))
+    oute = empty(edge)
+    b.bt_op_colsum_static(xe, 64, edge, oute)
+    assert torch.equal(oute, _reference(xe, 64, edge))
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_colsum_static(empty(64, edge + 4), 64, edge + 4, empty(edge + 4))
+    assert e.value.status == 2
     with pytest.raises(b.BtError) as e:
         b.bt_op_colsum_static(x, 64, 6, empty(8))
     assert e.value.status == 1
