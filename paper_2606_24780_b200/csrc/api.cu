@@ -831,7 +831,7 @@ extern "C" bt_status bt_op_embedding_bwd(const int32_t* tok, const float* dx, in
     if (N < 1 || T < 1 || C < 4 || C % 4 || N % T || N > (1 << 24) || V < 1)
         return fail(BT_ERR_INVALID_ARG, "embedding_bwd: bad sizes");
     if (scratch_bytes < embedding_bwd_scratch_bytes(N, C, V)) return fail(BT_ERR_OOM, "embedding_bwd: scratch too small");
-    const size_t partial_bytes = embedding_bwd_scratch_bytes(N, C, V) - (size_t)V * (size_t)((N + 127) / 128);
+    const size_t partial_bytes = embedding_bwd_partial_bytes(N, C);
     BT_CUDA(launch_embedding_bwd(tok, dx, N, T, C, V, V, dwte, dwpe, (float*)scratch, (uint8_t*)scratch + partial_bytes,
                                  (cudaStream_t)stream));
     return BT_OK;

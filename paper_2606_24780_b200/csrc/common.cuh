@@ -143,7 +143,9 @@ cudaError_t launch_split(const float* x, float* hi, float* lo, int64_t n, cudaSt
 // Ids outside [0, V) are treated as id 0; position + 1 of one of them is left in *bad (nullable).
 cudaError_t launch_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int T,
                                  int C, int V, float* x, int* bad, cudaStream_t s);
-// partial: N*C floats; table: Vp * ceil(N / 128) bytes (both scratch, contents irrelevant on entry).
+// partial: N*C floats (embedding_bwd_partial_bytes); table: Vp bytes per chunk of 128 positions, the rest of
+// embedding_bwd_scratch_bytes (both scratch, contents irrelevant on entry).
+size_t embedding_bwd_partial_bytes(int64_t N, int C);
 size_t embedding_bwd_scratch_bytes(int64_t N, int C, int Vp);
 cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, int V, int Vp,
                                  float* dwte, float* dwpe, float* partial, uint8_t* table, cudaStream_t s);

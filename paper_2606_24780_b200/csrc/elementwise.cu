@@ -154,7 +154,7 @@ cudaError_t launch_embedding_fwd(const int32_t* tok, const float* wte, const flo
 //
 // dwte[id,:] += sum over the positions n with tok[n] == id of dx[n,:], in ascending n, without
 // atomics and with the work spread evenly although the ids are heavy-tailed (under a Zipf law one id
-// owns a seventh of all positions).  Two stages over chunks of kEmbChunk consecutive positions:
+// owns a seventh of all positions).  Two stages over chunks of kEmbChunk (128) consecutive positions:
 //   1. one CTA per chunk groups the chunk's positions by id (all in shared memory), reads every row
 //      of dx exactly once, eight rows in flight, and writes one partial row per (chunk, id) group to
 //      `partial` at the slot of the group's first position; a byte table [Vp][chunks] records that
@@ -230,28 +230,35 @@ __global__ void __launch_bounds__(256) embedding_bwd_combine_kernel(const uint8_
     __shared__ int present[kEmbIdsPerCta];
     __shared__ int list[256];
     __shared__ int wcount[8];
-    const int id0 = blockIdx.x * kEmbIdsPerCta;
+    // the CTA's ids are blockIdx.x, blockIdx.x + gridDim.x, ...: frequent ids are neighbours under a
+    // rank-ordered vocabulary (id = frequency rank), and every one of them has a partial row in
+    // every chunk, so consecutive ids must not share a CTA
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     if (threadIdx.x < kEmbIdsPerCta) present[threadIdx.x] = 0;
     __syncthreads();
+    int any[kEmbIdsPerCta];      // all table reads are issued before any of them is looked at
 #pragma unroll
     for (int w = 0; w < kEmbIdsPerCta; ++w) {
-        const int id = id0 + w;
-        if (id >= Vp) break;
-        int any = 0;
-        for (int k = threadIdx.x; k < n_chunks; k += 256) any |= table[(int64_t)id * n_chunks + k];
-        if (any) present[w] = 1;
+        const int id = blockIdx.x + w * gridDim.x;
+        any[w] = 0;
+        if (id < Vp)
+            for (int k = threadIdx.x; k < n_chunks; k += 256) any[w] |= table[(int64_t)id * n_chunks + k];
     }
+#pragma unroll
+    for (int w = 0; w < kEmbIdsPerCta; ++w)
+        if (any[w]) present[w] = 1;
     __syncthreads();
+#pragma unroll
     for (int w = 0; w < kEmbIdsPerCta; ++w) {
         if (!present[w]) continue;   // uniform over the CTA
-        const int id = id0 + w;
+        const int id = blockIdx.x + w * gridDim.x;
         for (int c0 = 0; c0 < C4; c0 += 256) {
             const int c = c0 + threadIdx.x;
             float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
             for (int k0 = 0; k0 < n_chunks; k0 += 256) {
                 const int k = k0 + threadIdx.x;
-                const int b = k < n_chunks ? table[(int64_t)id * n_chunks + k] : 0;
+                // up to 256 chunks the byte read during the presence test is this thread's entry
+                const int b = n_chunks <= 256 ? any[w] : (k < n_chunks ? table[(int64_t)id * n_chunks + k] : 0);
                 // ordered list of the round's partial rows: chunk order = thread order
                 const unsigned bal = __ballot_sync(0xffffffffu, b != 0);
                 if (lane == 0) wcount[warp] = __popc(bal);
@@ -299,10 +306,10 @@ __global__ void __launch_bounds__(256) embedding_bwd_wpe_kernel(const float* __r
     }
 }
 
+size_t embedding_bwd_partial_bytes(int64_t N, int C) { return ((size_t)N * C * sizeof(float) + 255) & ~(size_t)255; }
 size_t embedding_bwd_scratch_bytes(int64_t N, int C, int Vp) {
     const int64_t chunks = (N + kEmbChunk - 1) / kEmbChunk;
-    const size_t partial = ((size_t)N * C * sizeof(float) + 255) & ~(size_t)255;
-    return partial + (size_t)Vp * (size_t)chunks;
+    return embedding_bwd_partial_bytes(N, C) + (size_t)Vp * (size_t)chunks;
 }
 
 cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N, int T, int C, int V, int Vp,

@@ -8,7 +8,25 @@
 
 namespace bt {
 
-constexpr int kLnWarps = 8;
+constexpr int kLnWarps = 8;   // most warps a CTA of the warp-per-row kernels has
+
+// Launch shape of the warp-per-row kernels: ctas_per_sm * 148 CTAs of w warps, every warp walking
+// rows warp, warp + total, ...  All warps are resident at once and the kernel is memory-bound, so
+// its time goes like (rounds per warp) x (warps per SM); w in 4..8 is chosen to minimise
+// ceil(N / total warps) * w, i.e. the work lost to a last, partly filled round (N = 8192 rows on
+// 148 SMs: eight warps per CTA leave a fourth round 46 % full, seven fill it to 99 %).
+struct LnShape { int ctas, warps; };
+static inline LnShape ln_shape(int64_t N, int ctas_per_sm) {
+    const int64_t slots = 148LL * ctas_per_sm;
+    if (N <= slots * 4) return LnShape{(int)((N + 3) / 4), 4};   // fewer rows than one round of the smallest shape
+    int best_w = kLnWarps;
+    int64_t best = -1;
+    for (int w = kLnWarps; w >= 4; --w) {
+        const int64_t cost = ((N + slots * w - 1) / (slots * w)) * w;
+        if (best < 0 || cost < best) { best = cost; best_w = w; }
+    }
+    return LnShape{(int)slots, best_w};
+}
 
 // VPL = float4 values per lane (C <= 128 * VPL).
 template <int VPL>
@@ -19,10 +37,9 @@ __global__ void __launch_bounds__(kLnWarps * 32) ln_fwd_kernel(const float* __re
                                                                float* __restrict__ mean, float* __restrict__ rstd) {
     pdl_wait();
     pdl_trigger();
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t row = (int64_t)blockIdx.x * kLnWarps + warp;
-    if (row >= N) return;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     const float inv_c = 1.0f / (float)(C4 * 4);
+    for (int64_t row = (int64_t)blockIdx.x * nwarps + warp; row < N; row += (int64_t)gridDim.x * nwarps) {
     float4 v[VPL];
     float s = 0.f;
 #pragma unroll
@@ -60,6 +77,7 @@ __global__ void __launch_bounds__(kLnWarps * 32) ln_fwd_kernel(const float* __re
     if (lane == 0) {
         if (mean) mean[row] = mu;
         if (rstd) rstd[row] = rs;
+    }
     }
 }
 
@@ -149,9 +167,9 @@ cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float
         BT_COUNT_LAUNCH();
         return cudaGetLastError();
     }
-    const int grid = (int)((N + kLnWarps - 1) / kLnWarps);
+    const LnShape shape = ln_shape(N, 4);
 #define BT_LN_FWD(V)                                                                                     \
-    BT_KERNEL_LAUNCH((ln_fwd_kernel<V>), grid, kLnWarps * 32, 0, s, x, gamma, beta, N, C4, y, y_hi, y_lo, mean, rstd)
+    BT_KERNEL_LAUNCH((ln_fwd_kernel<V>), shape.ctas, shape.warps * 32, 0, s, x, gamma, beta, N, C4, y, y_hi, y_lo, mean, rstd)
     if (vpl <= 1) BT_LN_FWD(1);
     else if (vpl <= 2) BT_LN_FWD(2);
     else if (vpl <= 4) BT_LN_FWD(4);
@@ -165,11 +183,7 @@ cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float
 
 // ------------------------------------------------------------------ backward
 
-static inline int ln_bwd_ctas(int64_t N) {
-    int64_t g = (N + kLnWarps - 1) / kLnWarps;
-    if (g > 148 * 2) g = 148 * 2;  // two CTAs per SM, one wave
-    return (int)g;
-}
+static inline int ln_bwd_ctas(int64_t N) { return ln_shape(N, 2).ctas; }   // two CTAs per SM, one wave
 static inline int ln_bwd_wide_ctas(int64_t N) {
     int64_t g = (N + 1) / 2;   // two rows per round, one CTA per SM
     return (int)(g < 148 ? g : 148);
@@ -192,12 +206,12 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     pdl_trigger();
     constexpr int kParts = CS ? 3 : 2;
     extern __shared__ float4 sm[];  // [kLnWarps][kParts][C4]
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
     float4* acc = sm + (size_t)warp * kParts * C4;
     for (int i = lane; i < kParts * C4; i += 32) acc[i] = make_float4(0.f, 0.f, 0.f, 0.f);
     __syncwarp();
     const float inv_c = 1.0f / (float)(C4 * 4);
-    for (int64_t row = (int64_t)blockIdx.x * kLnWarps + warp; row < N; row += (int64_t)gridDim.x * kLnWarps) {
+    for (int64_t row = (int64_t)blockIdx.x * nwarps + warp; row < N; row += (int64_t)gridDim.x * nwarps) {
         const float mu = mean[row], rs = rstd[row];
         float4 xv[VPL], dv[VPL], rv[VPL];
         float s1 = 0.f, s2 = 0.f;
@@ -248,8 +262,7 @@ __global__ void __launch_bounds__(kLnWarps * 32, 2) ln_bwd_kernel(
     float4* dst = reinterpret_cast<float4*>(partial) + (int64_t)blockIdx.x * kParts * C4;
     for (int i = threadIdx.x; i < kParts * C4; i += blockDim.x) {
         float4 t = sm[i];
-#pragma unroll
-        for (int w = 1; w < kLnWarps; ++w) t = add4(t, sm[(size_t)w * kParts * C4 + i]);
+        for (int w = 1; w < nwarps; ++w) t = add4(t, sm[(size_t)w * kParts * C4 + i]);
         dst[i] = t;
     }
 }
@@ -421,17 +434,18 @@ cudaError_t launch_layernorm_bwd(const float* dy, const float* x, const float* g
         BT_COUNT_LAUNCH();
         return cudaGetLastError();
     }
-    const int grid = ln_bwd_ctas(N);
-    const size_t smem = (size_t)kLnWarps * (dx_colsum ? 3 : 2) * C4 * sizeof(float4);   // 72 KB at C = 768 with sums
+    const LnShape shape = ln_shape(N, 2);
+    const int grid = shape.ctas;
+    const size_t smem = (size_t)shape.warps * (dx_colsum ? 3 : 2) * C4 * sizeof(float4);   // 72 KB at C = 768, 8 warps, with sums
     static const cudaError_t attr = ln_bwd_set_smem_limits();
     if (attr != cudaSuccess) return attr;
 #define BT_LN_BWD(V)                                                                                          \
     do {                                                                                                      \
         if (dx_colsum)                                                                                        \
-            BT_KERNEL_LAUNCH((ln_bwd_kernel<V, true>), grid, kLnWarps * 32, smem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, \
+            BT_KERNEL_LAUNCH((ln_bwd_kernel<V, true>), grid, shape.warps * 32, smem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, \
                                                                      dx_hi, dx_lo, scratch);                  \
         else                                                                                                  \
-            BT_KERNEL_LAUNCH((ln_bwd_kernel<V, false>), grid, kLnWarps * 32, smem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, \
+            BT_KERNEL_LAUNCH((ln_bwd_kernel<V, false>), grid, shape.warps * 32, smem, s, dy, x, gamma, mean, rstd, dres, N, C4, dx, \
                                                                       dx_hi, dx_lo, scratch);                 \
     } while (0)
     if (vpl <= 1) BT_LN_BWD(1);
