@@ -190,6 +190,64 @@ BT_API bt_status bt_micro_step(bt_model* m, const int32_t* d_tokens, const int32
 BT_API bt_status bt_train_step_accum(bt_model* m, const int32_t* d_tokens, const int32_t* d_targets, int32_t B,
                                      int32_t n_micro, const bt_adamw_config* opt, float* h_loss);
 
+/* ----------------------------------------------------------------------------------
+ * Data-parallel gradient exchange (Distributed Execution, "Data-Parallel Orchestration",
+ * Algorithm 1 "Distributed Data Parallel Training Step")
+ * --------------------------------------------------------------------------------
+ * Every rank holds a replica and its own batch rows; on the synchronising micro-step the
+ * gradients are averaged over the ranks in buckets, each bucket as soon as the backward pass has
+ * finished it, on a second stream, ordered against the compute stream by events only (the host
+ * never blocks), and the optimizer step waits for the last bucket.
+ *
+ * The gradients of a model lie in ONE flat arena in registry order and the backward pass finishes
+ * them in the reverse of that order, so a bucket is a contiguous range of the arena and is reduced
+ * in place: there is no copy into bucket memory and no scatter back.  bt_ddp_plan_* is the host-only
+ * part -- which range each bucket covers, which tensors it waits for, and the in-order launch gate
+ * -- usable (and tested) without a GPU:
+ *   bt_ddp_plan_create    buckets for `cfg` under a cap of bucket_cap_bytes (the paper uses 25 MB):
+ *                         tensors are taken in gradient-ready order (last registry entry first) and
+ *                         a bucket is closed when the next tensor would exceed the cap; a tensor
+ *                         larger than the cap is cut into equal ranges under the cap.  Bucket 0 is ready first.
+ *   bt_ddp_plan_bucket    range (offset and count, in floats, inside the arena) of bucket b and the
+ *                         number of tensors it waits for.
+ *   bt_ddp_plan_tensor    arena offset and padded length of registry tensor i (every tensor starts
+ *                         on a multiple of 1024 floats; the padding is zero and stays zero).
+ *   bt_ddp_plan_reset     before a backward pass: every bucket pending again, next bucket = 0.
+ *   bt_ddp_plan_mark_ready  "the gradient of tensor i is final" (the hook of Algorithm 1): returns
+ *                         how many buckets may be launched NOW, in order, and writes their indices
+ *                         to `launch` (room for bt_ddp_plan_num_buckets entries).  A bucket is
+ *                         launched only after all buckets before it, whatever order the marks
+ *                         arrive in; marking a tensor twice is an error (-1).
+ * bt_ddp_attach connects a model to an all-reduce: during bt_backward the library marks tensors
+ * ready as the kernels that finish them are enqueued; for every released bucket it records an
+ * event on the model's stream, makes `comm_stream` wait for it and calls
+ *     fn(user, d_grads + offset, count, bucket, comm_stream)
+ * which must ENQUEUE on comm_stream an in-place all-reduce of `count` floats that leaves the
+ * AVERAGE over the ranks (for example ncclAllReduce with ncclAvg), must not block the host, and
+ * returns 0 on success.  After the last bucket the model's stream is made to wait for
+ * comm_stream, so bt_adamw_step sees the averaged gradients.  With bt_micro_step /
+ * bt_train_step_accum only the last micro-step exchanges gradients (the others run without any
+ * communication), and its accumulation is folded in bucket by bucket so that the exchange still
+ * overlaps the backward pass.  The loss every rank reports stays its own.  Start every rank from
+ * the same parameters (bt_arena_ptr gives the parameter arena as one range to broadcast).
+ * bt_ddp_detach returns the model to single-replica operation. */
+typedef struct bt_ddp_plan bt_ddp_plan;
+typedef int32_t (*bt_allreduce_fn)(void* user, float* d_buf, int64_t count, int32_t bucket, void* comm_stream);
+BT_API bt_status bt_ddp_plan_create(const bt_config* cfg, int64_t bucket_cap_bytes, bt_ddp_plan** out);
+BT_API void bt_ddp_plan_destroy(bt_ddp_plan* plan);
+BT_API int32_t bt_ddp_plan_num_buckets(const bt_ddp_plan* plan);
+BT_API bt_status bt_ddp_plan_bucket(const bt_ddp_plan* plan, int32_t b, int64_t* offset, int64_t* count,
+                                    int32_t* n_tensors);
+BT_API bt_status bt_ddp_plan_tensor(const bt_ddp_plan* plan, int32_t tensor, int64_t* offset, int64_t* padded_len);
+BT_API void bt_ddp_plan_reset(bt_ddp_plan* plan);
+BT_API int32_t bt_ddp_plan_mark_ready(bt_ddp_plan* plan, int32_t tensor, int32_t* launch);
+BT_API bt_status bt_ddp_attach(bt_model* m, int64_t bucket_cap_bytes, bt_allreduce_fn fn, void* user,
+                               void* comm_stream);
+BT_API bt_status bt_ddp_detach(bt_model* m);
+/* The four flat arenas (kind: 0 parameters, 1 gradients, 2 / 3 moments): device pointer and length
+ * in floats, padding included. */
+BT_API bt_status bt_arena_ptr(bt_model* m, int32_t kind, float** d_ptr, int64_t* count);
+
 /* Learning rate of optimizer step `step` (1-based) from the hyper-parameter table's max / min
  * learning rate, warmup steps and training steps.  Reading (the paper gives the four numbers, not
  * the curve): linear warmup max_lr * step / warmup_steps, then a half cosine from max_lr at

@@ -62,6 +62,16 @@ _SIGNATURES = {
     "bt_micro_step": (_i32, [_vp, _vp, _vp, _i32, _i32, _i32, ctypes.POINTER(_f)]),
     "bt_train_step_accum": (_i32, [_vp, _vp, _vp, _i32, _i32, ctypes.POINTER(bt_adamw_config), ctypes.POINTER(_f)]),
     "bt_lr_at": (_f, [ctypes.POINTER(bt_lr_schedule), _i64]),
+    "bt_ddp_plan_create": (_i32, [ctypes.POINTER(bt_config), _i64, ctypes.POINTER(_vp)]),
+    "bt_ddp_plan_destroy": (None, [_vp]),
+    "bt_ddp_plan_num_buckets": (_i32, [_vp]),
+    "bt_ddp_plan_bucket": (_i32, [_vp, _i32, ctypes.POINTER(_i64), ctypes.POINTER(_i64), ctypes.POINTER(_i32)]),
+    "bt_ddp_plan_tensor": (_i32, [_vp, _i32, ctypes.POINTER(_i64), ctypes.POINTER(_i64)]),
+    "bt_ddp_plan_reset": (None, [_vp]),
+    "bt_ddp_plan_mark_ready": (_i32, [_vp, _i32, ctypes.POINTER(_i32)]),
+    "bt_ddp_attach": (_i32, [_vp, _i64, _vp, _vp, _vp]),
+    "bt_ddp_detach": (_i32, [_vp]),
+    "bt_arena_ptr": (_i32, [_vp, _i32, ctypes.POINTER(_vp), ctypes.POINTER(_i64)]),
     "bt_loader_plan": (_i32, [ctypes.POINTER(_i64), _i32, _i32, _i32, _i32, _i32, _i32, ctypes.POINTER(_i32),
                               ctypes.POINTER(_i64)]),
     "bt_loader_create": (_i32, [ctypes.POINTER(_vp), ctypes.POINTER(_i64), _i32, _i32, _i32, _i32, _i32, _i32, _i32,
@@ -272,6 +282,57 @@ def bt_loader_plan(shard_lens, B, T, rank, world, n_batches):
     out_s, out_p = (_i32 * n_batches)(), (_i64 * n_batches)()
     _check(lib().bt_loader_plan(lens, n, B, T, rank, world, n_batches, out_s, out_p))
     return [(int(out_s[i]), int(out_p[i])) for i in range(n_batches)]
+
+
+ALLREDUCE_FN = ctypes.CFUNCTYPE(ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
+                                ctypes.c_void_p)
+
+
+class DdpPlan:
+    """Host-only view of the gradient buckets of a configuration (no GPU needed): ranges of the flat
+    gradient arena in gradient-ready order, the arena offsets of the registry tensors, and the
+    in-order launch gate."""
+
+    def __init__(self, cfg, bucket_cap_bytes=25 * 1000 * 1000):
+        self.h = _vp()
+        _check(lib().bt_ddp_plan_create(ctypes.byref(cfg), bucket_cap_bytes, ctypes.byref(self.h)))
+        self.n_buckets = int(lib().bt_ddp_plan_num_buckets(self.h))
+
+    def bucket(self, b):
+        """(offset, count, n_tensors) of bucket b, offsets and counts in floats."""
+        off, cnt, nt = _i64(), _i64(), _i32()
+        _check(lib().bt_ddp_plan_bucket(self.h, b, ctypes.byref(off), ctypes.byref(cnt), ctypes.byref(nt)))
+        return int(off.value), int(cnt.value), int(nt.value)
+
+    def tensor(self, i):
+        """(offset, padded length) of registry tensor i inside the arena, in floats."""
+        off, ln = _i64(), _i64()
+        _check(lib().bt_ddp_plan_tensor(self.h, i, ctypes.byref(off), ctypes.byref(ln)))
+        return int(off.value), int(ln.value)
+
+    def reset(self):
+        lib().bt_ddp_plan_reset(self.h)
+
+    def mark_ready(self, tensor):
+        """Buckets the gate releases now that `tensor`'s gradient is final (in launch order)."""
+        out = (_i32 * max(1, self.n_buckets))()
+        n = int(lib().bt_ddp_plan_mark_ready(self.h, tensor, out))
+        if n < 0:
+            raise BtError(1, f"tensor {tensor} out of range or marked ready twice")
+        return [int(out[i]) for i in range(n)]
+
+    def close(self):
+        if self.h and _lib is not None:
+            _lib.bt_ddp_plan_destroy(self.h)
+        self.h = None
+
+    __del__ = close
+
+
+def bt_arena_ptr(model, kind):
+    p, n = _vp(), _i64()
+    _check(lib().bt_arena_ptr(model, kind, ctypes.byref(p), ctypes.byref(n)))
+    return p.value, int(n.value)
 
 
 class Loader:
@@ -544,6 +605,31 @@ class Model:
     def activation(self, name, layer=0, planes=1):
         ptr, numel = bt_activation_ptr(self.h, name, layer)
         return self._view(ptr, numel * planes)
+
+    def arena(self, kind=0):
+        """One of the four flat arenas (0 parameters, 1 gradients, 2 / 3 moments) as a float32 view."""
+        ptr, n = bt_arena_ptr(self.h, kind)
+        return self._view(ptr, n)
+
+    def ddp_attach(self, allreduce, comm_stream, bucket_cap_bytes=25 * 1000 * 1000):
+        """allreduce(buf, bucket): must enqueue, on comm_stream, an in-place all-reduce of the float32
+        tensor view `buf` (a range of the gradient arena) that leaves the average over the ranks."""
+        def trampoline(_user, d_buf, count, bucket, _stream):
+            try:
+                with torch.cuda.stream(comm_stream):
+                    allreduce(self._view(d_buf, count), int(bucket))
+                return 0
+            except Exception as exc:          # an exception must not cross the C frames
+                self._ddp_error = exc
+                return 1
+        self._ddp_cb = ALLREDUCE_FN(trampoline)     # kept alive with the model
+        self._ddp_stream = comm_stream
+        _check(lib().bt_ddp_attach(self.h, bucket_cap_bytes, ctypes.cast(self._ddp_cb, _vp), None,
+                                   comm_stream.cuda_stream))
+
+    def ddp_detach(self):
+        _check(lib().bt_ddp_detach(self.h))
+        self._ddp_cb = None
 
     def load_params(self, params):
         for name, a in params.items():

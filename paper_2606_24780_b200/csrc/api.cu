@@ -99,6 +99,23 @@ struct Bump {
 
 }  // namespace
 
+// Gradient buckets of the data-parallel step (Algorithm 1).  The gradients of one model lie in one
+// flat arena in registry order, and the backward pass finishes them in (almost exactly) the reverse
+// of that order, so a bucket needs no memory of its own: it is a contiguous range of the arena,
+// bucket 0 at the arena's end (first ready), the last bucket at its start (the tied embedding, ready
+// last).  Ranges are cut at tensor boundaries while a tensor fits under the cap; a larger tensor is
+// cut into equal ranges under the cap (all of them ready together).  `pending` counts the tensors that overlap
+// a bucket and are not ready yet; buckets are released strictly in order (the launch gate).
+struct bt_ddp_plan {
+    struct Bucket { int64_t offset, count; int n_tensors, pending; };
+    std::vector<Bucket> buckets;
+    std::vector<int64_t> t_off, t_len;          // arena range of every tensor (padded length)
+    std::vector<int> t_first, t_last;           // buckets a tensor overlaps
+    std::vector<uint8_t> t_ready;
+    int next_bucket = 0;
+    int64_t P = 0;
+};
+
 struct bt_model {
     bt_config cfg;
     cudaStream_t stream;
@@ -125,6 +142,15 @@ struct bt_model {
     bool have_forward;
     long long launches_at_create;
     // optional per-kernel timing (CUDA events around every launch of the step)
+    // data-parallel gradient exchange (null: single replica)
+    bt_ddp_plan* ddp;
+    bt_allreduce_fn ddp_fn;
+    void* ddp_user;
+    cudaStream_t ddp_stream;
+    std::vector<cudaEvent_t> ddp_ready_ev;   // one per bucket, recorded on the compute stream
+    cudaEvent_t ddp_done_ev;                 // recorded on the communication stream after the last bucket
+    bool ddp_sync;                           // this backward exchanges gradients (false on all but the last micro-step)
+    float ddp_acc_weight;                    // > 0: the last micro-step's accumulation is folded in per bucket
     bool prof_on;
     std::vector<ProfRec> prof_recs;
     std::vector<cudaEvent_t> prof_events;
@@ -376,7 +402,139 @@ bool debug_env() {
     return on;
 }
 
+// ------------------------------------------------------------------ data-parallel buckets
+bt_status build_ddp_plan(const bt_config* cfg, int64_t cap_bytes, bt_ddp_plan** out) {
+    if (!out) return fail(BT_ERR_INVALID_ARG, "ddp plan: out is NULL");
+    *out = nullptr;
+    bt_status st = validate(cfg);
+    if (st != BT_OK) return st;
+    if (cap_bytes < 4096) return fail(BT_ERR_INVALID_ARG, "ddp plan: bucket cap below 4096 bytes");
+    std::vector<Tensor> reg;
+    int64_t P = 0;
+    build_registry(*cfg, reg, P);
+    bt_ddp_plan* plan = new bt_ddp_plan();
+    plan->P = P;
+    const int n = (int)reg.size();
+    plan->t_off.resize(n); plan->t_len.resize(n); plan->t_first.assign(n, -1); plan->t_last.assign(n, -1);
+    plan->t_ready.assign(n, 0);
+    for (int i = 0; i < n; ++i) {
+        plan->t_off[i] = reg[i].off;
+        plan->t_len[i] = (i + 1 < n ? reg[i + 1].off : P) - reg[i].off;
+    }
+    const int64_t cap = cap_bytes / 4 / 1024 * 1024;          // floats, a multiple of the tensor alignment
+    // walk the registry backwards = gradient-ready order; `lo` is the start of the open bucket
+    int64_t hi = P;          // end of the open bucket
+    int64_t lo = P;
+    int open_tensors = 0;
+    auto close = [&]() {
+        if (hi > lo) plan->buckets.push_back(bt_ddp_plan::Bucket{lo, hi - lo, open_tensors, open_tensors});
+        hi = lo;
+        open_tensors = 0;
+    };
+    for (int i = n - 1; i >= 0; --i) {
+        const int64_t len = plan->t_len[i];
+        if (len > cap) {                                      // larger than a bucket: equal ranges of its own, each under the cap
+            close();
+            plan->t_first[i] = (int)plan->buckets.size();
+            int64_t end = plan->t_off[i] + len;
+            const int64_t pieces = (len + cap - 1) / cap;
+            const int64_t piece = ((len + pieces - 1) / pieces + 1023) / 1024 * 1024;   // equal ranges, each under the cap
+            while (end > plan->t_off[i]) {
+                const int64_t start = std::max(plan->t_off[i], end - piece);
+                plan->buckets.push_back(bt_ddp_plan::Bucket{start, end - start, 1, 1});
+                end = start;
+            }
+            plan->t_last[i] = (int)plan->buckets.size() - 1;
+            hi = lo = plan->t_off[i];
+            continue;
+        }
+        if (open_tensors > 0 && (hi - lo) + len > cap) close();
+        lo = plan->t_off[i];
+        ++open_tensors;
+        plan->t_first[i] = plan->t_last[i] = (int)plan->buckets.size();   // index the open bucket will get
+    }
+    close();
+    *out = plan;
+    return BT_OK;
+}
+
+// The hook of Algorithm 1 on the host side of one model: marks a tensor ready and launches the
+// exchange of every bucket the gate releases.
+bt_status ddp_launch_bucket(bt_model* m, int b) {
+    const bt_ddp_plan::Bucket& bk = m->ddp->buckets[(size_t)b];
+    float* g = m->grads + bk.offset;
+    if (m->ddp_acc_weight > 0.f)     // last micro-step: g = acc + w g for this range (the loss is handled by the caller)
+        BT_CUDA(launch_grad_accumulate(m->gacc + bk.offset, g, bk.count, m->ddp_acc_weight, 2, nullptr, nullptr, m->stream));
+    BT_CUDA(cudaEventRecord(m->ddp_ready_ev[(size_t)b], m->stream));
+    BT_CUDA(cudaStreamWaitEvent(m->ddp_stream, m->ddp_ready_ev[(size_t)b], 0));
+    if (m->ddp_fn(m->ddp_user, g, bk.count, b, (void*)m->ddp_stream) != 0)
+        return fail(BT_ERR_CUDA, "ddp: the all-reduce callback failed on bucket %d", b);
+    if (b + 1 == (int)m->ddp->buckets.size()) {   // the optimizer step must see every averaged bucket
+        BT_CUDA(cudaEventRecord(m->ddp_done_ev, m->ddp_stream));
+        BT_CUDA(cudaStreamWaitEvent(m->stream, m->ddp_done_ev, 0));
+    }
+    return BT_OK;
+}
+bt_status ddp_ready(bt_model* m, std::initializer_list<int> tensors) {
+    if (!m->ddp || !m->ddp_sync) return BT_OK;
+    std::vector<int32_t> launch(m->ddp->buckets.size());
+    for (int t : tensors) {
+        const int32_t n = bt_ddp_plan_mark_ready(m->ddp, t, launch.data());
+        if (n < 0) return fail(BT_ERR_INVALID_ARG, "ddp: tensor %d marked ready twice", t);
+        for (int32_t i = 0; i < n; ++i) {
+            bt_status st = ddp_launch_bucket(m, launch[(size_t)i]);
+            if (st != BT_OK) return st;
+        }
+    }
+    return BT_OK;
+}
+#define BT_DDP_READY(...)                                  \
+    do {                                                   \
+        bt_status st__ = ddp_ready(m, {__VA_ARGS__});      \
+        if (st__ != BT_OK) return st__;                    \
+    } while (0)
+
 }  // namespace
+
+// =============================================================================== data-parallel plan (host only)
+
+extern "C" bt_status bt_ddp_plan_create(const bt_config* cfg, int64_t bucket_cap_bytes, bt_ddp_plan** out) {
+    return build_ddp_plan(cfg, bucket_cap_bytes, out);
+}
+extern "C" void bt_ddp_plan_destroy(bt_ddp_plan* plan) { delete plan; }
+extern "C" int32_t bt_ddp_plan_num_buckets(const bt_ddp_plan* plan) { return plan ? (int32_t)plan->buckets.size() : 0; }
+extern "C" bt_status bt_ddp_plan_bucket(const bt_ddp_plan* plan, int32_t b, int64_t* offset, int64_t* count,
+                                        int32_t* n_tensors) {
+    if (!plan) return fail(BT_ERR_INVALID_ARG, "ddp plan is NULL");
+    if (b < 0 || b >= (int32_t)plan->buckets.size()) return fail(BT_ERR_NOT_FOUND, "bucket %d out of range", b);
+    if (offset) *offset = plan->buckets[(size_t)b].offset;
+    if (count) *count = plan->buckets[(size_t)b].count;
+    if (n_tensors) *n_tensors = plan->buckets[(size_t)b].n_tensors;
+    return BT_OK;
+}
+extern "C" bt_status bt_ddp_plan_tensor(const bt_ddp_plan* plan, int32_t tensor, int64_t* offset, int64_t* padded_len) {
+    if (!plan) return fail(BT_ERR_INVALID_ARG, "ddp plan is NULL");
+    if (tensor < 0 || tensor >= (int32_t)plan->t_off.size()) return fail(BT_ERR_NOT_FOUND, "tensor %d out of range", tensor);
+    if (offset) *offset = plan->t_off[(size_t)tensor];
+    if (padded_len) *padded_len = plan->t_len[(size_t)tensor];
+    return BT_OK;
+}
+extern "C" void bt_ddp_plan_reset(bt_ddp_plan* plan) {
+    if (!plan) return;
+    for (auto& b : plan->buckets) b.pending = b.n_tensors;
+    std::fill(plan->t_ready.begin(), plan->t_ready.end(), (uint8_t)0);
+    plan->next_bucket = 0;
+}
+extern "C" int32_t bt_ddp_plan_mark_ready(bt_ddp_plan* plan, int32_t tensor, int32_t* launch) {
+    if (!plan || !launch || tensor < 0 || tensor >= (int32_t)plan->t_off.size()) return -1;
+    if (plan->t_ready[(size_t)tensor]) return -1;
+    plan->t_ready[(size_t)tensor] = 1;
+    for (int b = plan->t_first[(size_t)tensor]; b <= plan->t_last[(size_t)tensor]; ++b) plan->buckets[(size_t)b].pending -= 1;
+    int32_t n = 0;
+    while (plan->next_bucket < (int)plan->buckets.size() && plan->buckets[(size_t)plan->next_bucket].pending == 0)
+        launch[n++] = plan->next_bucket++;      // the in-order launch gate
+    return n;
+}
 
 // =============================================================================== model lifetime
 
@@ -417,6 +575,13 @@ extern "C" bt_status bt_model_create(const bt_config* cfg, void* d_workspace, si
     m->launches_at_create = g_launches.load();
     m->prof_on = false;
     m->prof_used = 0;
+    m->ddp = nullptr;
+    m->ddp_fn = nullptr;
+    m->ddp_user = nullptr;
+    m->ddp_stream = nullptr;
+    m->ddp_done_ev = nullptr;
+    m->ddp_sync = false;
+    m->ddp_acc_weight = 0.f;
     m->debug_sync = (cfg->flags & BT_FLAG_DEBUG) != 0 || debug_env();
     std::vector<uint8_t> flags((size_t)(m->P / 1024), 0);
     for (const Tensor& t : m->tensors)
@@ -456,7 +621,57 @@ extern "C" bt_status bt_model_create(const bt_config* cfg, void* d_workspace, si
 extern "C" void bt_model_destroy(bt_model* m) {
     if (!m) return;
     for (cudaEvent_t e : m->prof_events) cudaEventDestroy(e);
+    bt_ddp_detach(m);
     delete m;
+}
+
+extern "C" bt_status bt_ddp_attach(bt_model* m, int64_t bucket_cap_bytes, bt_allreduce_fn fn, void* user,
+                                   void* comm_stream) {
+    if (!m || !fn) return fail(BT_ERR_INVALID_ARG, "ddp_attach: NULL argument");
+    if ((cudaStream_t)comm_stream == m->stream)
+        return fail(BT_ERR_INVALID_ARG, "ddp_attach: the communication stream must differ from the model's stream");
+    bt_ddp_detach(m);
+    bt_ddp_plan* plan = nullptr;
+    bt_status st = build_ddp_plan(&m->cfg, bucket_cap_bytes, &plan);
+    if (st != BT_OK) return st;
+    std::vector<cudaEvent_t> evs(plan->buckets.size(), nullptr);
+    cudaError_t e = cudaEventCreateWithFlags(&m->ddp_done_ev, cudaEventDisableTiming);
+    for (size_t i = 0; i < evs.size() && e == cudaSuccess; ++i) e = cudaEventCreateWithFlags(&evs[i], cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+        for (cudaEvent_t ev : evs) if (ev) cudaEventDestroy(ev);
+        if (m->ddp_done_ev) cudaEventDestroy(m->ddp_done_ev);
+        m->ddp_done_ev = nullptr;
+        delete plan;
+        return fail(BT_ERR_CUDA, "ddp_attach: event creation failed: %s", cudaGetErrorString(e));
+    }
+    m->ddp = plan;
+    m->ddp_ready_ev = evs;
+    m->ddp_fn = fn;
+    m->ddp_user = user;
+    m->ddp_stream = (cudaStream_t)comm_stream;
+    return BT_OK;
+}
+
+extern "C" bt_status bt_ddp_detach(bt_model* m) {
+    if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    if (!m->ddp) return BT_OK;
+    for (cudaEvent_t ev : m->ddp_ready_ev) cudaEventDestroy(ev);
+    m->ddp_ready_ev.clear();
+    if (m->ddp_done_ev) cudaEventDestroy(m->ddp_done_ev);
+    m->ddp_done_ev = nullptr;
+    delete m->ddp;
+    m->ddp = nullptr;
+    m->ddp_fn = nullptr;
+    return BT_OK;
+}
+
+extern "C" bt_status bt_arena_ptr(bt_model* m, int32_t kind, float** d_ptr, int64_t* count) {
+    if (!m || !d_ptr) return fail(BT_ERR_INVALID_ARG, "NULL argument");
+    float* base = kind == 0 ? m->params : kind == 1 ? m->grads : kind == 2 ? m->mom1 : kind == 3 ? m->mom2 : nullptr;
+    if (!base) return fail(BT_ERR_INVALID_ARG, "kind %d not in 0..3", kind);
+    *d_ptr = base;
+    if (count) *count = m->P;
+    return BT_OK;
 }
 
 extern "C" bt_status bt_model_init(bt_model* m, uint64_t seed) {
@@ -633,8 +848,16 @@ extern "C" bt_status bt_get_loss(bt_model* m, float* h_loss) {
     return check_device_error(m);
 }
 
+static bt_status backward_impl(bt_model* m);
+
 extern "C" bt_status bt_backward(bt_model* m) {
     if (!m) return fail(BT_ERR_INVALID_ARG, "model is NULL");
+    m->ddp_sync = true;          // a plain backward always exchanges gradients when ranks are attached
+    m->ddp_acc_weight = 0.f;
+    return backward_impl(m);
+}
+
+static bt_status backward_impl(bt_model* m) {
     if (!m->have_forward) return fail(BT_ERR_INVALID_ARG, "bt_backward without a preceding bt_forward");
     cudaStream_t s = m->stream;
     constexpr bool gemm_is_fwd = false;  // timing category of this function's GEMMs
@@ -644,6 +867,10 @@ extern "C" bt_status bt_backward(bt_model* m) {
     const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
     const bool raw_qkv = simt_attn || ((C / H) != 64 && (C / H) != 128) || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
     auto G = [&](const Tensor& t) { return m->grads + t.off; };
+    // data-parallel exchange: registry indices of the tensors whose gradients each launch group finishes
+    const int nT = (int)m->tensors.size();
+    auto LI = [&](int l, int k) { return 2 + 12 * l + k; };
+    if (m->ddp && m->ddp_sync) bt_ddp_plan_reset(m->ddp);
 
     // LM head: dxf = dlogits . wte ; dwte = dlogits^T . xf
     SplitMat dlog = act_mat(m->dlogits_s, N, Vp, N);
@@ -655,6 +882,7 @@ extern "C" bt_status bt_backward(bt_model* m) {
     // the bias gradient of the projection whose output this residual stream position is.
     BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, m->xL, m->params + lnfg.off, m->meanf, m->rstdf, nullptr, N, C, m->dres,
                                  m->dres_s, m->dres_s + N * C, G(lnfg), G(lnfb), G(layer_tensor(m, m->L - 1, PRB)), m->ln_scratch, s));
+    BT_DDP_READY(nT - 1, nT - 2, LI(m->L - 1, PRB));
     SplitMat dres = act_mat(m->dres_s, N, C, N);
     for (int l = m->L - 1; l >= 0; --l) {
         LayerAct& a = m->act[l];
@@ -662,21 +890,26 @@ extern "C" bt_status bt_backward(bt_model* m) {
         // MLP down-projection: x_out = x1 + g . Wpr^T + bpr
         BT_GEMM(kNN, N, F, C, dres, weight_mat(m, LT(PRW), C, F), m->dg, nullptr, nullptr);
         BT_GEMM(kTN, C, F, N, dres, act_mat(a.g_s, N, F, N), G(LT(PRW)), nullptr, nullptr);
+        BT_DDP_READY(LI(l, PRW));
         // d h, with its column sums (the gradient of bfc) taken in the same pass
         BT_STEP(kCatGeluBwd, 0, 16.0 * N * F, launch_gelu_bwd_colsum(a.h, m->dg, N, F, tanh_form, nullptr, m->dh_s, m->dh_s + N * F,
                                        G(LT(FCB)), m->colsum_scratch, s));
+        BT_DDP_READY(LI(l, FCB));
         // MLP up-projection: h = m . Wfc^T + bfc
         SplitMat dh = act_mat(m->dh_s, N, F, N);
         BT_GEMM(kNN, N, C, F, dh, weight_mat(m, LT(FCW), F, C), m->dtmp, nullptr, nullptr);
         BT_GEMM(kTN, F, C, N, dh, act_mat(a.m_s, N, C, N), G(LT(FCW)), nullptr, nullptr);
+        BT_DDP_READY(LI(l, FCW));
         // LN2 and the residual: d x1 = d x_out + LN2'(dm)
         BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, a.x1, m->params + LT(LN2G).off, a.mean2, a.rstd2, m->dres, N, C, m->dres,
                                      m->dres_s, m->dres_s + N * C, G(LT(LN2G)), G(LT(LN2B)), G(LT(PROJB)), m->ln_scratch, s));
+        BT_DDP_READY(LI(l, LN2B), LI(l, LN2G), LI(l, PROJB));
         // attention output projection: x1 = x + o . Wo^T + bo
         // d o, raw for the FMA / warp-MMA attention kernels, as hi/lo planes for the tcgen05 ones
         BT_GEMM_SPLIT_OUT(kNN, N, C, C, dres, weight_mat(m, LT(PROJW), C, C), raw_qkv ? m->dtmp : nullptr, m->do_s, nullptr,
                           nullptr);
         BT_GEMM(kTN, C, C, N, dres, act_mat(a.o_s, N, C, N), G(LT(PROJW)), nullptr, nullptr);
+        BT_DDP_READY(LI(l, PROJW));
         bool rg_written = false;
         BT_STEP(kCatAttnBwd, 2.5 * attn_fwd_flops(B, H, T, C / H), 48.0 * N * C, launch_attention_bwd(raw_qkv ? a.qkv : nullptr, a.qkv_s, N * 3 * C, a.o_s, a.o_s + N * C, a.lse,
                                      raw_qkv ? m->dtmp : nullptr, m->do_s, N * C, B, T,
@@ -692,14 +925,18 @@ extern "C" bt_status bt_backward(bt_model* m) {
                     launch_colsum(m->attn_rg, nullptr, attention_bwd_rowgroups(B, T), 3 * C, G(LT(QKVB)), m->colsum_scratch, s));
         else
             BT_STEP(kCatColsum, 0, 24.0 * N * C, launch_colsum(m->dqkv_s, m->dqkv_s + N * 3 * C, N, 3 * C, G(LT(QKVB)), m->colsum_scratch, s));
+        BT_DDP_READY(LI(l, QKVB), LI(l, QKVW));
         // LN1 and the residual: d x = d x1 + LN1'(da)
         BT_STEP(kCatLnBwd, 0, 24.0 * N * C, launch_layernorm_bwd(m->dtmp, a.x, m->params + LT(LN1G).off, a.mean1, a.rstd1, m->dres, N, C, m->dres,
                                      m->dres_s, m->dres_s + N * C, G(LT(LN1G)), G(LT(LN1B)),
                                      l > 0 ? G(layer_tensor(m, l - 1, PRB)) : nullptr, m->ln_scratch, s));
+        BT_DDP_READY(LI(l, LN1B), LI(l, LN1G));
+        if (l > 0) BT_DDP_READY(LI(l - 1, PRB));
     }
     // embeddings: dwte (already holding the LM-head part) += gather-transpose, dwpe = sum over sequences
     BT_STEP(kCatEmbedBwd, 0, 8.0 * N * C, launch_embedding_bwd(m->cur_tok, m->dres, N, T, C, m->V, Vp, G(m->tensors[0]), G(m->tensors[1]),
                                                               m->dtmp, m->emb_table, s));
+    BT_DDP_READY(1, 0);
     if (m->debug_sync) return check_device_error(m);
     return BT_OK;
 }
@@ -743,12 +980,20 @@ extern "C" bt_status bt_micro_step(bt_model* m, const int32_t* d_tokens, const i
         return fail(BT_ERR_INVALID_ARG, "micro step %d of %d", micro_index, n_micro);
     bt_status st = bt_forward(m, d_tokens, d_targets, B, nullptr);
     if (st != BT_OK) return st;
-    st = bt_backward(m);
+    // Algorithm 1: gradients are exchanged on the last micro-step only; there the accumulation
+    // g = acc + g / n is applied bucket by bucket, just before each bucket's all-reduce
+    const bool last = micro_index == n_micro - 1;
+    const bool per_bucket = m->ddp != nullptr && last && n_micro > 1;
+    m->ddp_sync = last;
+    m->ddp_acc_weight = per_bucket ? 1.0f / (float)n_micro : 0.f;
+    st = backward_impl(m);
+    m->ddp_acc_weight = 0.f;
     if (st != BT_OK) return st;
     if (n_micro > 1) {
-        const int mode = micro_index == 0 ? 0 : micro_index == n_micro - 1 ? 2 : 1;
-        BT_CUDA(launch_grad_accumulate(m->gacc, m->grads, m->P, 1.0f / (float)n_micro, mode, m->loss_acc, m->loss,
-                                       m->stream));
+        const int mode = micro_index == 0 ? 0 : last ? 2 : 1;
+        // with buckets the gradient ranges are already folded in: only the loss word is left (n = 0)
+        BT_CUDA(launch_grad_accumulate(m->gacc, m->grads, per_bucket ? 0 : m->P, 1.0f / (float)n_micro, mode, m->loss_acc,
+                                       m->loss, m->stream));
     }
     if (h_loss) return bt_get_loss(m, h_loss);
     return BT_OK;

@@ -757,7 +757,7 @@ __global__ void __launch_bounds__(256) grad_accumulate_kernel(float* __restrict_
                                                               float w, int mode, float* loss_acc, float* loss) {
     pdl_wait();
     pdl_trigger();
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (loss != nullptr && blockIdx.x == 0 && threadIdx.x == 0) {
         const float l = w * loss[0];
         if (mode == 0) loss_acc[0] = l;
         else if (mode == 1) loss_acc[0] += l;

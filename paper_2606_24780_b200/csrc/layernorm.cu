@@ -167,7 +167,9 @@ cudaError_t launch_layernorm_fwd(const float* x, const float* gamma, const float
         BT_COUNT_LAUNCH();
         return cudaGetLastError();
     }
-    const LnShape shape = ln_shape(N, 4);
+    // forward: one row per warp, every row's loads in flight from the start (measured faster inside the
+    // training step, where the input was just written and is largely in L2, than a balanced row loop)
+    const LnShape shape{(int)((N + kLnWarps - 1) / kLnWarps), kLnWarps};
 #define BT_LN_FWD(V)                                                                                     \
     BT_KERNEL_LAUNCH((ln_fwd_kernel<V>), shape.ctas, shape.warps * 32, 0, s, x, gamma, beta, N, C4, y, y_hi, y_lo, mean, rstd)
     if (vpl <= 1) BT_LN_FWD(1);
