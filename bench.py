@@ -32,7 +32,26 @@ METRIC = "GPT-2 124M FP32 train tokens/s on 1 B200"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 TF32_OVER_BF16 = 0.5          # nominal dense ratio (1.1 / 2.25 PFLOP/s)
 MMA_PER_PRODUCT = 3.0         # 3xTF32: three tensor-core products per FP32 product
-NCU_GEMM_QKV_DRAM_BYTES = 109.6e6 + 46.0e6   # read + write of one forward QKV GEMM launch (ncu summary in profiles/)
+GEMM_PROFILE = os.path.join(ROOT, "profiles", "gemm_tc_kernel_gpt2small_block.txt")
+
+
+def ncu_qkv_gemm_dram_bytes():
+    """dram__bytes_read.sum + dram__bytes_write.sum of the forward QKV GEMM launch (the first kernel of
+    the committed ncu summary), in bytes; None if the summary is missing or unreadable."""
+    try:
+        total, seen = 0.0, 0
+        with open(GEMM_PROFILE) as f:
+            for line in f:
+                parts = line.split()
+                if len(parts) >= 3 and parts[0] in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+                    scale = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}[parts[2]]
+                    total += float(parts[1]) * scale
+                    seen += 1
+                    if seen == 2:
+                        return total
+    except (OSError, KeyError, ValueError):
+        pass
+    return None
 
 
 def load_peaks():
@@ -261,6 +280,11 @@ def run_ours(args, cfg):
                 "gbs": (by / (ms * 1e-3) / 1e9) if ms > 0 else None}
     b.bt_profile_enable(model.h, 0)
 
+    # the tensor pipe's own rate: clocks per 128 x 256 x 8 TF32 MMA on every SM (run after the timed regions)
+    _, probe_clk, _ = b.bt_probe_tf32_mma_rate(torch.cuda.get_device_properties(local).multi_processor_count, 4000)
+    mac_per_clk_sm = 128 * 256 * 8 / probe_clk
+    n_sms = torch.cuda.get_device_properties(local).multi_processor_count
+
     peaks, peak_kind = load_peaks()
     tf32x3_peak = peaks["bf16_tflops_sustained"] * TF32_OVER_BF16 / MMA_PER_PRODUCT
     gemm = {k: v for k, v in kernels.items() if k.startswith("gemm_")}
@@ -274,8 +298,17 @@ def run_ours(args, cfg):
                 # DRAM bytes of ONE launch of the forward QKV GEMM (8192 x 2304 x 768) from the committed
                 # ncu capture under profiles/ (dram__bytes_read.sum + dram__bytes_write.sum), beside
                 # its algorithmic bytes 8(MK + NK) + 4MN; other launches scale with their own sizes
-                "traffic": NCU_GEMM_QKV_DRAM_BYTES, "traffic_launch": "gemm forward qkv, M=8192 N=2304 K=768",
+                "traffic": ncu_qkv_gemm_dram_bytes(), "traffic_launch": "gemm forward qkv, M=8192 N=2304 K=768",
                 "traffic_algorithmic": 8.0 * (8192 * 768 + 2304 * 768) + 4.0 * 8192 * 2304}
+    # the same achieved rate against the pipe's own measured peak at the clock this run held:
+    # (MAC per clock per SM from the probe) x 2 x SMs x median sampled SM clock / 3
+    if clocks.get("sm_mhz"):
+        clock_peak = mac_per_clk_sm * 2.0 * n_sms * clocks["sm_mhz"] * 1e6 / 1e12 / MMA_PER_PRODUCT
+        roofline["tf32_probe"] = {"clocks_per_mma_128x256x8": probe_clk, "mac_per_clk_per_sm": mac_per_clk_sm,
+                                  "peak_3xtf32_at_sampled_clock": clock_peak}
+        roofline["frac_clock_scaled"] = achieved / clock_peak
+        for v in kernels.values():
+            v["mcycles"] = v["ms_per_step"] * clocks["sm_mhz"] / 1e3      # millions of SM clocks per step
 
     flop_per_token = si_flops_per_token(cfg)
     step_frac = value / world * flop_per_token / 1e12 / tf32x3_peak
@@ -289,7 +322,8 @@ def run_ours(args, cfg):
                    "padded_vocab": cfg["padded_vocab_size"], "tokens": "Zipf(1.1), seeded",
                    "parallelism": "replicas only" if world > 1 else "1 GPU",
                    "l2": "working set per step (>10 GB) exceeds L2; no explicit flush",
-                   "workspace_gib": model.workspace_bytes / 2 ** 30},
+                   "workspace_gib": model.workspace_bytes / 2 ** 30,
+                   "workspace_parts_gib": {k: v / 2 ** 30 for k, v in b.bt_workspace_parts(model.cfg).items()}},
         "clocks": clocks,
         "e2e": {"value": e2e_value, "unit": "tokens/s", "ms_per_step": e2e_ms,
                 "h2d_bytes_per_step": 2 * B * T * 4 * world, "d2h_bytes_per_step": 4 * world},
@@ -303,12 +337,14 @@ def run_ours(args, cfg):
 
     if rank == 0:
         if world == 1 and not args.no_cpu_baseline:
-            # bounded oracle sample: one full-length sequence of the same workload if it fits ~30 s
-            dt64, cores, _ = oracle_step_seconds(cfg, 64, 1)
-            seq = 64
-            while seq * 2 <= T and dt64 * (seq * 2 / 64.0) * 1.3 < 30.0:
-                seq *= 2
+            # bounded oracle sample (10 - 30 s of CPU work): one sequence of the same workload, as long
+            # as fits; the time of a half-length sequence predicts the full one (attention grows with
+            # the square of the length, the rest linearly: at most 4x)
+            seq = max(64, T // 2)
             dt, cores, _ = oracle_step_seconds(cfg, seq, 2)
+            while seq * 2 <= T and dt * 3.0 < 30.0:
+                seq *= 2
+                dt, cores, _ = oracle_step_seconds(cfg, seq, 2)
             line["cpu_baseline"] = {"value": seq / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                                     "sample": f"1 sequence of {seq} tokens, full model, fwd+bwd+AdamW, {dt:.1f} s"}
         print(json.dumps(line), flush=True)

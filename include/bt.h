@@ -99,6 +99,14 @@ typedef struct {
  * both moments, split weight copies, activations for max_batch sequences, scratch).
  * Returns 0 for an invalid configuration. */
 BT_API size_t bt_workspace_bytes(const bt_config* cfg);
+/* The same total by section (the paper's Evaluation reports the memory footprint beside the
+ * throughput): part 0 parameters + gradients + both moments, 1 TF32 hi/lo planes of the weights in
+ * both orientations, 2 gradient accumulator of the micro-step loop and small tables, 3 activations
+ * kept for the backward pass (max_batch sequences), 4 logits, their gradient planes and per-row
+ * losses, 5 backward temporaries reused by every layer, 6 scratch (split-K partial sums, reduction
+ * partials, id staging, embedding table).  The seven parts add up to bt_workspace_bytes; 0 for an
+ * invalid configuration or part. */
+BT_API size_t bt_workspace_part_bytes(const bt_config* cfg, int32_t part);
 
 /* Builds the host-side model over a caller-allocated device workspace of at least
  * bt_workspace_bytes(cfg) bytes, 256-byte aligned.  Moments and the step counter start

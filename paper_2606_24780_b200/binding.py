@@ -45,6 +45,7 @@ _vp, _i32, _i64, _u32, _sz, _f = (ctypes.c_void_p, ctypes.c_int32, ctypes.c_int6
                                   ctypes.c_float)
 _SIGNATURES = {
     "bt_workspace_bytes": (_sz, [ctypes.POINTER(bt_config)]),
+    "bt_workspace_part_bytes": (_sz, [ctypes.POINTER(bt_config), _i32]),
     "bt_model_create": (_i32, [ctypes.POINTER(bt_config), _vp, _sz, _vp, ctypes.POINTER(_vp)]),
     "bt_model_destroy": (None, [_vp]),
     "bt_model_init": (_i32, [_vp, ctypes.c_uint64]),
@@ -286,6 +287,15 @@ def bt_loader_plan(shard_lens, B, T, rank, world, n_batches):
 
 ALLREDUCE_FN = ctypes.CFUNCTYPE(ctypes.c_int32, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32,
                                 ctypes.c_void_p)
+
+
+WORKSPACE_PARTS = ("params_grads_moments", "weight_planes", "grad_accumulator", "activations", "logits",
+                   "backward_temporaries", "scratch")
+
+
+def bt_workspace_parts(cfg):
+    """{section: bytes} of the workspace of a configuration; the values add up to bt_workspace_bytes."""
+    return {name: int(lib().bt_workspace_part_bytes(ctypes.byref(cfg), i)) for i, name in enumerate(WORKSPACE_PARTS)}
 
 
 class DdpPlan:

@@ -122,6 +122,7 @@ struct bt_model {
     int L, C, H, T, V, Vp, F, maxB;
     std::vector<Tensor> tensors;
     int64_t P;  // padded parameter count (multiple of 1024)
+    size_t part_bytes[7];   // workspace sections, see bt_workspace_part_bytes
     float *params, *grads, *mom1, *mom2, *wsplit, *wsplit_t, *gacc, *loss_acc;
     MatDesc* mat_descs;   // device table of the weight matrices (for the split in both orientations)
     int n_mats, n_mat_tiles;
@@ -219,16 +220,25 @@ bt_status validate(const bt_config* c) {
 size_t layout(bt_model* m, uint8_t* base) {
     Bump b{base};
     const int64_t C = m->C, F = m->F, N = (int64_t)m->maxB * m->T, Vp = m->Vp, P = m->P;
+    // the raw (single-plane) qkv exists only for the attention kernels that read it: the warp-MMA
+    // kernels of head_dim 16 / 32 and the reference kernels behind the test flags
+    const int hd = (int)(C / m->H);
+    const bool raw_qkv = (m->cfg.flags & (BT_FLAG_ATTN_SIMT | BT_FLAG_GEMM_SIMT)) != 0 || (hd != 64 && hd != 128);
+    size_t mark = 0;
+    auto section = [&](int part) { m->part_bytes[part] = b.off - mark; mark = b.off; };
     m->params = b.take<float>(P);
     m->grads = b.take<float>(P);
     m->mom1 = b.take<float>(P);
     m->mom2 = b.take<float>(P);
+    section(0);                      // parameters, gradients, both moments
     m->wsplit = b.take<float>(2 * P);
     m->wsplit_t = b.take<float>(2 * P);
+    section(1);                      // TF32 hi/lo planes of the weights, both orientations
     m->gacc = b.take<float>(P);      // gradient accumulator of the micro-step loop
     m->loss_acc = b.take<float>(4);
     m->mat_descs = b.take<MatDesc>(kMaxSplitMats);
     m->decay_flags = b.take<uint8_t>(P / 1024);
+    section(2);                      // gradient accumulator, tables
     m->act.resize(m->L);
     for (int l = 0; l < m->L; ++l) {
         LayerAct& a = m->act[l];
@@ -236,7 +246,7 @@ size_t layout(bt_model* m, uint8_t* base) {
         a.mean1 = b.take<float>(N);
         a.rstd1 = b.take<float>(N);
         a.a_s = b.take<float>(2 * N * C);
-        a.qkv = b.take<float>(N * 3 * C);
+        a.qkv = raw_qkv ? b.take<float>(N * 3 * C) : nullptr;
         a.qkv_s = b.take<float>(2 * N * 3 * C);
         a.o_s = b.take<float>(2 * N * C);
         a.lse = b.take<float>((int64_t)m->maxB * m->H * m->T);
@@ -251,11 +261,13 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->meanf = b.take<float>(N);
     m->rstdf = b.take<float>(N);
     m->xf_s = b.take<float>(2 * N * C);
+    section(3);                      // activations kept for the backward pass
     m->logits = b.take<float>(N * Vp);
     m->dlogits_s = b.take<float>(2 * N * Vp);
     m->losses = b.take<float>(N);
     m->loss = b.take<float>(4);
     m->norm_out = b.take<float>(4);
+    section(4);                      // logits, their gradient planes, per-row losses
     m->dres = b.take<float>(N * C);
     m->dres_s = b.take<float>(2 * N * C);
     m->dtmp = b.take<float>(N * C);
@@ -265,6 +277,7 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->dg = b.take<float>(N * F);
     m->dvec = b.take<float>((int64_t)m->maxB * m->H * m->T);
     m->attn_rg = b.take<float>(attention_bwd_rowgroups(m->maxB, m->T) * 3 * m->C);
+    section(5);                      // backward temporaries (reused by every layer)
     m->partial_floats = gemm_tc_partial_floats_bound();
     m->partials = b.take<float>(m->partial_floats);
     m->ln_scratch = b.take<float>(layernorm_bwd_scratch_floats(N, (int)C));
@@ -279,7 +292,9 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->tok_stage = b.take<int32_t>(N);
     m->tgt_stage = b.take<int32_t>(N);
     m->emb_table = b.take<uint8_t>(embedding_bwd_scratch_bytes(N, 0, (int)Vp));
-    return (b.off + 255) & ~(size_t)255;
+    b.off = (b.off + 255) & ~(size_t)255;
+    section(6);                      // split-K partial sums, reduction scratch, id staging, embedding table
+    return b.off;
 }
 
 void fill_dims(bt_model* m, const bt_config* cfg) {
@@ -545,6 +560,14 @@ extern "C" size_t bt_workspace_bytes(const bt_config* cfg) {
     return layout(&tmp, nullptr);
 }
 
+extern "C" size_t bt_workspace_part_bytes(const bt_config* cfg, int32_t part) {
+    if (part < 0 || part > 6 || validate(cfg) != BT_OK) return 0;
+    bt_model tmp{};
+    fill_dims(&tmp, cfg);
+    layout(&tmp, nullptr);
+    return tmp.part_bytes[part];
+}
+
 extern "C" bt_status bt_model_create(const bt_config* cfg, void* d_workspace, size_t workspace_bytes, void* stream,
                                      bt_model** out) {
     if (!out) return fail(BT_ERR_INVALID_ARG, "out is NULL");
@@ -726,7 +749,10 @@ extern "C" bt_status bt_activation_ptr(bt_model* m, const char* name, int32_t la
         if (n == "x") { p = a.x; ne = N * C; }
         else if (n == "qkv_split") { p = a.qkv_s; ne = N * 3 * C; }
         else if (n == "a") { p = a.a_s; ne = N * C; }
-        else if (n == "qkv") { p = a.qkv; ne = N * 3 * C; }
+        else if (n == "qkv") {
+            if (!a.qkv) return fail(BT_ERR_NOT_FOUND, "the raw qkv array is not kept in this configuration (use qkv_split)");
+            p = a.qkv; ne = N * 3 * C;
+        }
         else if (n == "o") { p = a.o_s; ne = N * C; }
         else if (n == "lse") { p = a.lse; ne = (int64_t)m->curB * m->H * m->T; }
         else if (n == "x1") { p = a.x1; ne = N * C; }

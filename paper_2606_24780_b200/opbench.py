@@ -243,11 +243,11 @@ def main(argv=None):
     args = ap.parse_args(argv)
     torch.cuda.set_device(0)
     only = [s for s in args.only.split(",") if s]
-    need_big = not only or any(s.startswith(("gemm_fwd_lm", "gemm_nt_lm", "gemm_nn_dlm", "gemm_tn_wlm", "softmax", "adamw", "grad",
-                                          "embedding", "model_"))
+    need_big = not only or any(s.startswith(("gemm_fwd_lm", "gemm_nt_lm", "gemm_nn_dlm", "gemm_tn_wlm", "softmax", "embedding"))
                                for s in only)
-    cases = build_cases(args.batch, args.seq, args.d_model, args.heads, args.vocab if need_big else 0,
-                        args.params if need_big else 0)
+    need_params = not only or any(s.startswith(("adamw", "grad", "model_")) for s in only)
+    cases = build_cases(args.batch, args.seq, args.d_model, args.heads, args.vocab if (need_big or need_params) else 0,
+                        args.params if need_params else 0)
     flush = None if args.no_flush else torch.zeros(64 * 1024 * 1024, device="cuda")  # 256 MB > 126 MB L2
     results = {}
     if not only or "tf32_rate" in only:

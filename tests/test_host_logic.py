@@ -37,6 +37,10 @@ def test_workspace_bytes_and_config_validation(lib):
     assert n > 0 and n % 256 == 0
     bigger = b.make_config(2, 64, 4, 64, 512, 512, 8)
     assert b.bt_workspace_bytes(bigger) > n
+    parts = b.bt_workspace_parts(good)
+    assert sum(parts.values()) == n and all(v > 0 for v in parts.values())
+    assert b.bt_workspace_parts(bigger)["params_grads_moments"] == parts["params_grads_moments"]
+    assert b.bt_workspace_parts(bigger)["activations"] > parts["activations"]
     for bad in [b.make_config(0, 64, 4, 64, 512, 512, 4), b.make_config(2, 66, 4, 64, 512, 512, 4),
                 b.make_config(2, 64, 4, 64, 512, 500, 4), b.make_config(2, 64, 4, 64, 512, 520, 4),
                 b.make_config(2, 96, 4, 64, 512, 512, 4), b.make_config(2, 64, 4, 64, 512, 512, 0),
