@@ -208,6 +208,28 @@ def tf32_rate(sm_mhz=None):
     return {"clocks_per_mma_128x256x8": med, "clocks_min_max": [lo, hi], "mac_per_clk_per_sm": 128 * 256 * 8 / med}
 
 
+def hbm_rates(n_bytes=1 << 30, iters=10):
+    """Measured HBM rates for the roofline denominators of the memory-bound kernels (harness-side torch
+    kernels, best of `iters`): a copy (read + write bytes), a pure write (fill) and a pure read (sum).
+    A kernel that writes more than it reads is bound by the write rate, not by the copy rate."""
+    a = torch.empty(n_bytes // 4, device="cuda")
+    c = torch.empty_like(a)
+    a.fill_(1.0)
+    out = {}
+    for name, fn, moved in (("copy", lambda: c.copy_(a), 2 * n_bytes), ("write", lambda: c.fill_(2.0), n_bytes),
+                            ("read", lambda: a.sum(), n_bytes)):
+        best = 1e30
+        for _ in range(iters):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            best = min(best, e0.elapsed_time(e1))
+        out[name + "_gbs"] = moved / best / 1e6
+    return out
+
+
 def time_case(case, iters, warmup, flush_buf):
     for _ in range(warmup):
         case["run"]()
@@ -258,6 +280,11 @@ def main(argv=None):
         print(f"tf32_rate              {r['clocks_per_mma_128x256x8']:10.1f} clk per 128x256x8 MMA  "
               f"{r['mac_per_clk_per_sm']:7.0f} MAC/clk/SM  (x 2 x {sms} SMs x clock = dense TF32 peak; / 3 for 3xTF32)",
               flush=True)
+    if not only or "hbm_rates" in only:
+        r = hbm_rates()
+        results["hbm_rates"] = r
+        print(f"hbm_rates              copy {r['copy_gbs']:.0f} GB/s (read + write bytes), write only {r['write_gbs']:.0f} GB/s, "
+              f"read only {r['read_gbs']:.0f} GB/s  (1 GiB each, best of 10)", flush=True)
     for name, case in cases.items():
         if only and name not in only:
             continue
