@@ -61,17 +61,29 @@ __device__ __forceinline__ unsigned smid() {
 // in full 128-byte row segments (see warp_rows_store).  The tensor-memory loads are .sync.aligned:
 // EVERY lane of the warp must call this.  hi0 / lo0: row 0 of the warp, column 0 of the head;
 // nvalid: rows of the warp inside the sequence; sums (nullable): 64 column sums over those rows.
+// PAIRS: the accumulator is 128 columns wide and output columns 32 h .. 32 h + 31 are the sum of its
+// columns 64 h .. 64 h + 31 and 64 h + 32 .. 64 h + 63 (the halves of a split product, see the dq kernel).
+template <bool PAIRS = false>
 __device__ __forceinline__ void tmem_rows_to_split(uint32_t t_row, float mul, float* hi0, float* lo0,
                                                    long long row_stride, int nvalid, float* sums, float* tile,
                                                    int lane) {
 #pragma unroll
     for (int half = 0; half < 2; ++half) {
         uint32_t r[32];
-        tmem_ld32(t_row + half * 32, r);
-        tmem_ld_wait();
         float v[32];
+        if (PAIRS) {
+            uint32_t r2[32];
+            tmem_ld32(t_row + half * 64, r);
+            tmem_ld32(t_row + half * 64 + 32, r2);
+            tmem_ld_wait();
 #pragma unroll
-        for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * mul;
+            for (int i = 0; i < 32; ++i) v[i] = (__uint_as_float(r[i]) + __uint_as_float(r2[i])) * mul;
+        } else {
+            tmem_ld32(t_row + half * 32, r);
+            tmem_ld_wait();
+#pragma unroll
+            for (int i = 0; i < 32; ++i) v[i] = __uint_as_float(r[i]) * mul;
+        }
         warp_rows_store(v, tile, lane, nvalid, nullptr, hi0 + half * 32, lo0 + half * 32, row_stride,
                         sums ? sums + half * 32 : nullptr);
     }
@@ -279,6 +291,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     } else if (warp == 1) {
         if (lane == 0) {
             constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT64, false, false);  // 128 x 64, B K-major
+            constexpr uint32_t idesc_a2 = make_idesc_tf32(BR, 2 * BT64, false, false);  // 128 x 128: B = [hi rows | lo rows]
             constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
             bool ok = mbar_wait(bar(V_FULL), 0, g.err, 23) && mbar_wait(bar(K_READY), 0, g.err, 24);
             int tn = 0;
@@ -289,10 +302,11 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t q_hi = qd.at(kmaj_off(BT64, ks, false)), q_lo = qd.at(kmaj_off(BT64, ks, true));
-                    umma_tf32_ts(tS, tK_lo + ks * 8, q_hi, idesc_a, ks > 0 ? 1u : 0u);
-                    umma_tf32_ts(tS, tK_hi + ks * 8, q_lo, idesc_a, 1u);
-                    umma_tf32_ts(tS, tK_hi + ks * 8, q_hi, idesc_a, 1u);
+                    // the tile's lo rows follow its hi rows: [Q_hi | Q_lo] is one 128-row operand, and the
+                    // product's two halves land in the S^T and the P^T_lo columns (added when they are read)
+                    const uint64_t q_hl = qd.at(kmaj_off(BT64, ks, false));
+                    umma_tf32_ts(tS, tK_hi + ks * 8, q_hl, idesc_a2, ks > 0 ? 1u : 0u);   // K'_hi Q_hi | K'_hi Q_lo
+                    umma_tf32_ts(tS, tK_lo + ks * 8, q_hl, idesc_a, 1u);                  // + K'_lo Q_hi
                 }
                 umma_commit(bar(QK_EMPTY));
                 umma_commit(bar(S_FULL));
@@ -305,10 +319,9 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint64_t v_hi = vd.at(kmaj_off(BR, ks, false)), v_lo = vd.at(kmaj_off(BR, ks, true));
-                    const uint64_t o_hi = od.at(kmaj_off(BT64, ks, false)), o_lo = od.at(kmaj_off(BT64, ks, true));
-                    umma_tf32(tdP, v_lo, o_hi, idesc_a, ks > 0 ? 1u : 0u);
-                    umma_tf32(tdP, v_hi, o_lo, idesc_a, 1u);
-                    umma_tf32(tdP, v_hi, o_hi, idesc_a, 1u);
+                    const uint64_t o_hl = od.at(kmaj_off(BT64, ks, false));
+                    umma_tf32(tdP, v_hi, o_hl, idesc_a2, ks > 0 ? 1u : 0u);   // V_hi dO_hi | V_hi dO_lo
+                    umma_tf32(tdP, v_lo, o_hl, idesc_a, 1u);                  // + V_lo dO_hi
                 }
                 umma_commit(bar(DOK_EMPTY));
                 umma_commit(bar(DP_FULL));
@@ -395,14 +408,15 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             if (!mbar_wait_warp(bar(S_FULL), (uint32_t)(t & 1), g.err, 31)) { ok = false; break; }
             tc_fence_after();
             uint32_t s[32];
-            tmem_ld32(tS + t_lane + c0, s);
-            tmem_ld_wait();
             float p[32];
             uint32_t lo[32];
+            tmem_ld32(tS + t_lane + c0, s);
+            tmem_ld32(tPlo + t_lane + c0, lo);        // the second half of the split score product
+            tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
                 const bool live = (i < nvalid) && (q0 + i >= key);   // in the sequence and not before this key
-                p[i] = live ? ex2_approx(__uint_as_float(s[i]) - Lc[i]) : 0.f;
+                p[i] = live ? ex2_approx((__uint_as_float(s[i]) + __uint_as_float(lo[i])) - Lc[i]) : 0.f;
                 split_tf32_int(p[i], s[i], lo[i]);
             }
             tmem_st32(tS + t_lane + c0, s);          // P^T hi over S^T
@@ -415,10 +429,11 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             if (!mbar_wait_warp(bar(DP_FULL), (uint32_t)(t & 1), g.err, 32)) { ok = false; break; }
             tc_fence_after();
             tmem_ld32(tdP + t_lane + c0, s);
+            tmem_ld32(tdSlo + t_lane + c0, lo);
             tmem_ld_wait();
 #pragma unroll
             for (int i = 0; i < 32; ++i) {
-                const float ds = p[i] * (__uint_as_float(s[i]) - Dc[i]);
+                const float ds = p[i] * ((__uint_as_float(s[i]) + __uint_as_float(lo[i])) - Dc[i]);
                 split_tf32_int(ds, s[i], lo[i]);
             }
             tmem_st32(tdP + t_lane + c0, s);         // dS^T hi over dP^T
@@ -508,8 +523,9 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
     const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp);
     pdl_wait();      // set-up done; global memory is touched from here on
     pdl_trigger();
+    // dQ is 128 columns: the halves of the split product dS . [K_hi | K_lo] by 32-column groups (see issue_b)
     const uint32_t tQ_hi = tmem, tQ_lo = tmem + 64, tdQ = tmem + 128;
-    auto tbuf = [&](int bb) { return tmem + 192u + 128u * (uint32_t)bb; };   // +0 S -> dS_hi, +64 dP -> dS_lo
+    auto tbuf = [&](int bb) { return tmem + 256u + 128u * (uint32_t)bb; };   // +0 S -> dS_hi, +64 dP -> dS_lo
 
     if (warp == 0) {
         if (lane == 0) {
@@ -547,6 +563,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
         if (lane == 0) {
             constexpr uint32_t idesc_a = make_idesc_tf32(BR, BKT, false, false);   // 128 x 64, B K-major
             constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
+            constexpr uint32_t idesc_b2 = make_idesc_tf32(BR, 2 * HD, false, true);   // 128 x 128, B = four column groups
             bool ok = mbar_wait(do_full, 0, g.err, 33) && mbar_wait(q_ready, 0, g.err, 34);
             int tn = 0;
             const DescBase dod = kmaj_base(do_s);
@@ -586,14 +603,19 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
                 trace_mark(g.trace, 0, tn, 500 + t);
                 tc_fence_after();
                 const uint32_t s_hi = tbuf(bb), s_lo = tbuf(bb) + 64u;
+                // Two instructions per k-step.  The MN-major K tile lies in shared memory as the column
+                // groups [K_hi g0 | K_lo g0 | K_hi g1 | K_lo g1] (g = 32 head columns), 8 KB apart: seen
+                // with that stride it is one operand of N = 128, and dS_hi times it fills the four
+                // 32-column groups of dQ in that order.  dS_lo . K_hi (groups g0, g1, 16 KB apart, N = 64)
+                // is accumulated 32 columns further, so that its halves land on the second and third group:
+                // head columns 0-31 = dQ[0:32) + dQ[32:64), 32-63 = dQ[64:96) + dQ[96:128).
                 const DescBase kmd = mnmaj64_base(km_s);
+                const DescBase kmd4 = make_desc_base(km_s, BKT * 128u, 512u, 1u);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t k_hi = kmd.at(mnmaj64_off(ks, false)), k_lo = kmd.at(mnmaj64_off(ks, true));
                     const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
-                    umma_tf32_ts(tdQ, s_lo + ks * 8, k_hi, idesc_b, acc);
-                    umma_tf32_ts(tdQ, s_hi + ks * 8, k_lo, idesc_b, 1u);
-                    umma_tf32_ts(tdQ, s_hi + ks * 8, k_hi, idesc_b, 1u);
+                    umma_tf32_ts(tdQ, s_hi + ks * 8, kmd4.at(mnmaj64_off(ks, false)), idesc_b2, acc);
+                    umma_tf32_ts(tdQ + 32u, s_lo + ks * 8, kmd.at(mnmaj64_off(ks, false)), idesc_b, 1u);
                 }
                 umma_commit(mempty);
                 trace_mark(g.trace, 0, tn, 600 + t);
@@ -684,7 +706,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
                                   ? g.rg_sums + ((int64_t)b * g.nrg + (q0 >> 5) + lane_group) * gs + h * HD
                                   : nullptr;
                 float* tile = reinterpret_cast<float*>(smem_raw + (kk_s(0) - smem_u32(smem_raw)) + (uint32_t)(warp - 2) * kRowTileBytes);
-                tmem_rows_to_split(tdQ + t_lane, scale, hi, hi + g.dqkv_plane, gs, nvalid, sums, tile, lane);
+                tmem_rows_to_split<true>(tdQ + t_lane, scale, hi, hi + g.dqkv_plane, gs, nvalid, sums, tile, lane);
             }
         }
     }
