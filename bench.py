@@ -54,6 +54,26 @@ def ncu_qkv_gemm_dram_bytes():
     return None
 
 
+_RESULT_OUT = None
+
+
+def claim_stdout():
+    """Standard output carries exactly one JSON line.  Libraries underneath write there too (NCCL prints
+    its version banner on the first communicator), so file descriptor 1 is pointed at standard error
+    for the rest of the process and the result goes to a private copy of the original descriptor."""
+    global _RESULT_OUT
+    if _RESULT_OUT is None:
+        sys.stdout.flush()
+        _RESULT_OUT = os.fdopen(os.dup(1), "w")
+        os.dup2(2, 1)
+
+
+def emit(line: dict):
+    out = _RESULT_OUT if _RESULT_OUT is not None else sys.stdout
+    out.write(json.dumps(line) + "\n")
+    out.flush()
+
+
 def load_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
     try:
@@ -165,7 +185,7 @@ def run_reference(args, cfg):
         "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }
-    print(json.dumps(line), flush=True)
+    emit(line)
 
 
 class RankSync:
@@ -213,11 +233,27 @@ def run_ours(args, cfg):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    elif args.ddp:
+        import socket
+        import torch.distributed as dist
+        with socket.socket() as sk:
+            sk.bind(("127.0.0.1", 0))
+            port = sk.getsockname()[1]
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                                device_id=torch.device(f"cuda:{local}"))
 
     B, T = cfg["batch"], cfg["seq_len"]
     model = b.Model(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], T, cfg["vocab_size"],
                     cfg["padded_vocab_size"], B, device=f"cuda:{local}")
     model.init(1234 + rank)
+    if args.ddp:
+        # Algorithm 1 instead of independent replicas: identical start weights from rank 0, then every
+        # backward pass averages the gradients bucket by bucket on a second stream (NCCL through
+        # torch.distributed; the library only orders the two streams with events)
+        torch.cuda.synchronize()
+        dist.broadcast(model.arena(0), src=0)
+        comm_stream = torch.cuda.Stream()
+        model.ddp_attach(lambda buf, bucket: dist.all_reduce(buf, op=dist.ReduceOp.AVG), comm_stream)
     opt = b.make_adamw(**si.ADAMW)
     n_batches = 4
     batches = [si.tokens_for(cfg, 10 * rank + i) for i in range(n_batches)]
@@ -320,7 +356,8 @@ def run_ours(args, cfg):
         "config": {"workload": cfg["name"], "n_layers": cfg["n_layers"], "d_model": cfg["d_model"],
                    "n_heads": cfg["n_heads"], "seq_len": T, "batch_per_gpu": B, "vocab": cfg["vocab_size"],
                    "padded_vocab": cfg["padded_vocab_size"], "tokens": "Zipf(1.1), seeded",
-                   "parallelism": "replicas only" if world > 1 else "1 GPU",
+                   "parallelism": (f"ddp{world}: bucketed gradient all-reduce (Algorithm 1)" if args.ddp else
+                                   "replicas only" if world > 1 else "1 GPU"),
                    "l2": "working set per step (>10 GB) exceeds L2; no explicit flush",
                    "workspace_gib": model.workspace_bytes / 2 ** 30,
                    "workspace_parts_gib": {k: v / 2 ** 30 for k, v in b.bt_workspace_parts(model.cfg).items()}},
@@ -347,7 +384,7 @@ def run_ours(args, cfg):
                 dt, cores, _ = oracle_step_seconds(cfg, seq, 2)
             line["cpu_baseline"] = {"value": seq / dt, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                                     "sample": f"1 sequence of {seq} tokens, full model, fwd+bwd+AdamW, {dt:.1f} s"}
-        print(json.dumps(line), flush=True)
+        emit(line)
     model.close()
     if dist is not None:
         dist.destroy_process_group()
@@ -370,8 +407,12 @@ def main():
     ap.add_argument("--config", type=int, default=2)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--ddp", action="store_true",
+                    help="average the gradients over the ranks (bucketed all-reduce overlapped with the backward "
+                         "pass) instead of running independent replicas")
     args = ap.parse_args()
     cfg = si.config(args.config)
+    claim_stdout()
     if args.impl == "reference":
         run_reference(args, cfg)
     else:
