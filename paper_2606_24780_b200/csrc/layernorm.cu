@@ -12,9 +12,9 @@ constexpr int kLnWarps = 8;   // most warps a CTA of the warp-per-row kernels ha
 
 // Launch shape of the warp-per-row kernels: ctas_per_sm * 148 CTAs of w warps, every warp walking
 // rows warp, warp + total, ...  All warps are resident at once and the kernel is memory-bound, so
-// its time goes like (rounds per warp) x (warps per SM); w in 4..8 is chosen to minimise
-// ceil(N / total warps) * w, i.e. the work lost to a last, partly filled round (N = 8192 rows on
-// 148 SMs: eight warps per CTA leave a fourth round 46 % full, seven fill it to 99 %).
+// its time goes like (rows per warp) x (warps per SM); w in 4..8 is chosen to minimise
+// ceil(N / total warps) * w, i.e. the work lost to a last, partly filled pass over the warps
+// (N = 8192 rows on 148 SMs: with eight warps per CTA the fourth pass is 46 % full, with seven 99 %).
 struct LnShape { int ctas, warps; };
 static inline LnShape ln_shape(int64_t N, int ctas_per_sm) {
     const int64_t slots = 148LL * ctas_per_sm;
