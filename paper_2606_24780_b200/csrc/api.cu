@@ -240,12 +240,17 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->decay_flags = b.take<uint8_t>(P / 1024);
     section(2);                      // gradient accumulator, tables
     m->act.resize(m->L);
+    // BT_FLAG_RECOMPUTE_LN: the LayerNorm outputs (hi/lo planes) are not kept per layer; one buffer
+    // serves every layer and the backward pass re-runs the LayerNorm forward from the saved input
+    // and statistics where a weight-gradient product needs them
+    const bool recompute_ln = (m->cfg.flags & BT_FLAG_RECOMPUTE_LN) != 0;
+    float* ln_shared = recompute_ln ? b.take<float>(2 * N * C) : nullptr;
     for (int l = 0; l < m->L; ++l) {
         LayerAct& a = m->act[l];
         a.x = b.take<float>(N * C);
         a.mean1 = b.take<float>(N);
         a.rstd1 = b.take<float>(N);
-        a.a_s = b.take<float>(2 * N * C);
+        a.a_s = recompute_ln ? ln_shared : b.take<float>(2 * N * C);
         a.qkv = raw_qkv ? b.take<float>(N * 3 * C) : nullptr;
         a.qkv_s = b.take<float>(2 * N * 3 * C);
         a.o_s = b.take<float>(2 * N * C);
@@ -253,7 +258,7 @@ size_t layout(bt_model* m, uint8_t* base) {
         a.x1 = b.take<float>(N * C);
         a.mean2 = b.take<float>(N);
         a.rstd2 = b.take<float>(N);
-        a.m_s = b.take<float>(2 * N * C);
+        a.m_s = recompute_ln ? ln_shared : b.take<float>(2 * N * C);
         a.h = b.take<float>(N * F);
         a.g_s = b.take<float>(2 * N * F);
     }
@@ -892,6 +897,7 @@ static bt_status backward_impl(bt_model* m) {
     const bool simt_attn = (m->cfg.flags & BT_FLAG_ATTN_SIMT) != 0;
     const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
     const bool raw_qkv = simt_attn || ((C / H) != 64 && (C / H) != 128) || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
+    const bool recompute_ln = (m->cfg.flags & BT_FLAG_RECOMPUTE_LN) != 0;
     auto G = [&](const Tensor& t) { return m->grads + t.off; };
     // data-parallel exchange: registry indices of the tensors whose gradients each launch group finishes
     const int nT = (int)m->tensors.size();
@@ -924,6 +930,9 @@ static bt_status backward_impl(bt_model* m) {
         // MLP up-projection: h = m . Wfc^T + bfc
         SplitMat dh = act_mat(m->dh_s, N, F, N);
         BT_GEMM(kNN, N, C, F, dh, weight_mat(m, LT(FCW), F, C), m->dtmp, nullptr, nullptr);
+        if (recompute_ln)   // m = LN2(x1) again (bit-identical to the forward's: same kernel, same inputs)
+            BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x1, m->params + LT(LN2G).off, m->params + LT(LN2B).off, N, C, nullptr,
+                                                                       a.m_s, a.m_s + N * C, nullptr, nullptr, s));
         BT_GEMM(kTN, F, C, N, dh, act_mat(a.m_s, N, C, N), G(LT(FCW)), nullptr, nullptr);
         BT_DDP_READY(LI(l, FCW));
         // LN2 and the residual: d x1 = d x_out + LN2'(dm)
@@ -944,6 +953,9 @@ static bt_status backward_impl(bt_model* m) {
         // QKV projection: qkv = a . Wqkv^T + bqkv
         SplitMat dqkv = act_mat(m->dqkv_s, N, 3 * C, N);
         BT_GEMM(kNN, N, C, 3 * C, dqkv, weight_mat(m, LT(QKVW), 3 * C, C), m->dtmp, nullptr, nullptr);
+        if (recompute_ln)   // a = LN1(x) again
+            BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x, m->params + LT(LN1G).off, m->params + LT(LN1B).off, N, C, nullptr,
+                                                                       a.a_s, a.a_s + N * C, nullptr, nullptr, s));
         BT_GEMM(kTN, 3 * C, C, N, dqkv, act_mat(a.a_s, N, C, N), G(LT(QKVW)), nullptr, nullptr);
         // d bqkv: from the attention kernels' per-row-group sums when they wrote them, else a pass over dqkv
         if (rg_written)
