@@ -83,9 +83,11 @@ enum {
     BT_FLAG_GEMM_PAIR = 8u,  /* per-op GEMM calls: 256-row tiles on CTA pairs wherever M >= 256 */
     BT_FLAG_GEMM_SINGLE = 16u, /* per-op GEMM calls: 128-row tiles on single CTAs only (default: planner) */
     BT_FLAG_DEBUG = 32u,      /* every step call synchronises and reports device errors (ids, waits) itself */
-    BT_FLAG_RECOMPUTE_LN = 64u /* do not keep the LayerNorm outputs of every layer (2 x 8 B per token and feature):
+    BT_FLAG_RECOMPUTE_LN = 64u, /* do not keep the LayerNorm outputs of every layer (2 x 8 B per token and feature):
                                   the backward pass re-runs the LayerNorm forward from the saved input and statistics
                                   before the two weight-gradient products that read them (same bits, about 1 % more time) */
+    BT_FLAG_LOGITS_IN_PLACE = 128u /* the hi plane of the logit gradient is written over the logits (4 B per token and
+                                  vocabulary entry less); the "logits" activation is then unavailable.  padded_vocab <= 51200 */
 };
 
 /* AdamW hyper-parameters (hyper-parameter table, "Optimization" column).  grad_clip <= 0

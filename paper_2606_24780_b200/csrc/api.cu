@@ -211,6 +211,8 @@ bt_status validate(const bt_config* c) {
     if (1 + 4 * (int64_t)c->n_layers > kMaxSplitMats) return fail(BT_ERR_UNSUPPORTED, "config: more than 63 layers");
     if (c->padded_vocab_size < c->vocab_size) return fail(BT_ERR_INVALID_ARG, "config: padded_vocab < vocab");
     if (c->padded_vocab_size % 32) return fail(BT_ERR_INVALID_ARG, "config: padded_vocab %% 32 != 0");
+    if ((c->flags & BT_FLAG_LOGITS_IN_PLACE) && c->padded_vocab_size > softmax_xent_max_in_place_columns())
+        return fail(BT_ERR_UNSUPPORTED, "config: BT_FLAG_LOGITS_IN_PLACE needs padded_vocab <= %d", softmax_xent_max_in_place_columns());
     if ((int64_t)c->max_batch * c->seq_len > (1 << 24))
         return fail(BT_ERR_UNSUPPORTED, "config: more than 2^24 tokens per step");
     return BT_OK;
@@ -267,8 +269,10 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->rstdf = b.take<float>(N);
     m->xf_s = b.take<float>(2 * N * C);
     section(3);                      // activations kept for the backward pass
-    m->logits = b.take<float>(N * Vp);
+    // BT_FLAG_LOGITS_IN_PLACE: the hi plane of the logit gradient overwrites the logits (the loss kernel
+    // holds a whole row in registers before it writes anything)
     m->dlogits_s = b.take<float>(2 * N * Vp);
+    m->logits = (m->cfg.flags & BT_FLAG_LOGITS_IN_PLACE) ? m->dlogits_s : b.take<float>(N * Vp);
     m->losses = b.take<float>(N);
     m->loss = b.take<float>(4);
     m->norm_out = b.take<float>(4);
@@ -745,7 +749,11 @@ extern "C" bt_status bt_activation_ptr(bt_model* m, const char* name, int32_t la
     int64_t ne = 0;
     if (n == "xL") { p = m->xL; ne = N * C; }
     else if (n == "xf") { p = m->xf_s; ne = N * C; }
-    else if (n == "logits") { p = m->logits; ne = N * m->Vp; }
+    else if (n == "logits") {
+        if (m->cfg.flags & BT_FLAG_LOGITS_IN_PLACE)
+            return fail(BT_ERR_NOT_FOUND, "the logits are not kept with BT_FLAG_LOGITS_IN_PLACE (their gradient overwrites them)");
+        p = m->logits; ne = N * m->Vp;
+    }
     else if (n == "dlogits") { p = m->dlogits_s; ne = N * m->Vp; }
     else if (n == "losses") { p = m->losses; ne = N; }
     else {

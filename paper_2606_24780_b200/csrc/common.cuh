@@ -167,6 +167,7 @@ cudaError_t launch_gelu_bwd_colsum(const float* x, const float* dy, int64_t N, i
 cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int Vp, float inv_count,
                                 float* losses, float* loss_mean, float* dl, float* dl_hi, float* dl_lo, int V,
                                 int* bad, cudaStream_t s);
+int softmax_xent_max_in_place_columns();
 size_t colsum_scratch_floats(int64_t N, int C);
 // x_lo (nullable): second plane added to the first (sums a split array).
 cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, float* out, float* scratch,

@@ -32,7 +32,7 @@ __device__ __forceinline__ int checked_target(int t, int V, int64_t row, int* ba
 }
 
 template <int ITEMS>
-__global__ void __launch_bounds__(kXentThreads) xent_kernel(const float* __restrict__ logits,
+__global__ void __launch_bounds__(kXentThreads) xent_kernel(const float* logits,   // may alias dl_hi (in place)
                                                             const int32_t* __restrict__ targets, int V4,
                                                             float inv_count, float* __restrict__ losses, float* dl,
                                                             float* dl_hi, float* dl_lo, int V, int* bad) {
@@ -68,6 +68,9 @@ __global__ void __launch_bounds__(kXentThreads) xent_kernel(const float* __restr
     const int t = checked_target(targets[row], V, row, bad);
     if (threadIdx.x == 0) losses[row] = (mx + logf(sum)) - logits[row * V4 * 4 + t];
     if (dl == nullptr && dl_hi == nullptr) return;
+    // the gradient may be written over the logits themselves (in place): every thread has its part of
+    // the row in registers by now, and the target's logit has been read before anyone stores
+    __syncthreads();
     const float sc = inv_count / sum;
 #pragma unroll
     for (int k = 0; k < ITEMS; ++k) {
@@ -144,6 +147,9 @@ __global__ void __launch_bounds__(1024) loss_mean_kernel(const float* __restrict
     }
     if (threadIdx.x == 0) *loss_mean = (float)(sm[0] * (double)inv_count);
 }
+
+// Rows up to this many columns take the one-pass kernel, which may write its output over its input.
+int softmax_xent_max_in_place_columns() { return 25 * kXentThreads * 4; }
 
 cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int Vp, float inv_count,
                                 float* losses, float* loss_mean, float* dl, float* dl_hi, float* dl_lo, int V,
