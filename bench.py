@@ -245,7 +245,8 @@ def run_ours(args, cfg):
     B, T = cfg["batch"], cfg["seq_len"]
     model = b.Model(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], T, cfg["vocab_size"],
                     cfg["padded_vocab_size"], B, flags=(b.BT_FLAG_RECOMPUTE_LN if args.recompute_ln else 0) |
-                    (b.BT_FLAG_LOGITS_IN_PLACE if args.logits_in_place else 0),
+                    (b.BT_FLAG_LOGITS_IN_PLACE if args.logits_in_place else 0) |
+                    (b.BT_FLAG_RECOMPUTE_GELU if args.recompute_gelu else 0),
                     device=f"cuda:{local}")
     model.init(1234 + rank)
     if args.ddp:
@@ -363,6 +364,7 @@ def run_ours(args, cfg):
                    "l2": "working set per step (>10 GB) exceeds L2; no explicit flush",
                    "layernorm_outputs": "recomputed in the backward pass" if args.recompute_ln else "kept",
                    "logits": "overwritten by their gradient" if args.logits_in_place else "kept",
+                   "gelu_outputs": "recomputed in the backward pass" if args.recompute_gelu else "kept",
                    "workspace_gib": model.workspace_bytes / 2 ** 30,
                    "workspace_parts_gib": {k: v / 2 ** 30 for k, v in b.bt_workspace_parts(model.cfg).items()}},
         "clocks": clocks,
@@ -413,6 +415,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--recompute-ln", action="store_true",
                     help="BT_FLAG_RECOMPUTE_LN: smaller workspace, the LayerNorm forward runs again in the backward pass")
+    ap.add_argument("--recompute-gelu", action="store_true",
+                    help="BT_FLAG_RECOMPUTE_GELU: the GELU output planes are formed again in the backward pass")
     ap.add_argument("--logits-in-place", action="store_true",
                     help="BT_FLAG_LOGITS_IN_PLACE: the logit gradient's hi plane overwrites the logits")
     ap.add_argument("--ddp", action="store_true",

@@ -86,8 +86,10 @@ enum {
     BT_FLAG_RECOMPUTE_LN = 64u, /* do not keep the LayerNorm outputs of every layer (2 x 8 B per token and feature):
                                   the backward pass re-runs the LayerNorm forward from the saved input and statistics
                                   before the two weight-gradient products that read them (same bits, about 1 % more time) */
-    BT_FLAG_LOGITS_IN_PLACE = 128u /* the hi plane of the logit gradient is written over the logits (4 B per token and
+    BT_FLAG_LOGITS_IN_PLACE = 128u, /* the hi plane of the logit gradient is written over the logits (4 B per token and
                                   vocabulary entry less); the "logits" activation is then unavailable.  padded_vocab <= 51200 */
+    BT_FLAG_RECOMPUTE_GELU = 256u /* do not keep the GELU output planes of every layer (8 B per token and MLP feature):
+                                  the backward pass forms them again from the kept pre-activation (same bits, about 2 % more time) */
 };
 
 /* AdamW hyper-parameters (hyper-parameter table, "Optimization" column).  grad_clip <= 0

@@ -18,6 +18,7 @@ BT_FLAG_GELU_TANH, BT_FLAG_GEMM_SIMT, BT_FLAG_ATTN_SIMT, BT_FLAG_GEMM_PAIR, BT_F
 BT_FLAG_DEBUG = 32
 BT_FLAG_RECOMPUTE_LN = 64
 BT_FLAG_LOGITS_IN_PLACE = 128
+BT_FLAG_RECOMPUTE_GELU = 256
 BT_GEMM_NT, BT_GEMM_NN, BT_GEMM_TN = 0, 1, 2
 STATUS = {0: "BT_OK", 1: "BT_ERR_INVALID_ARG", 2: "BT_ERR_UNSUPPORTED", 3: "BT_ERR_OOM", 4: "BT_ERR_CUDA",
           5: "BT_ERR_DEVICE_TIMEOUT", 6: "BT_ERR_NOT_FOUND"}

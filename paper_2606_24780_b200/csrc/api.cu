@@ -247,6 +247,10 @@ size_t layout(bt_model* m, uint8_t* base) {
     // and statistics where a weight-gradient product needs them
     const bool recompute_ln = (m->cfg.flags & BT_FLAG_RECOMPUTE_LN) != 0;
     float* ln_shared = recompute_ln ? b.take<float>(2 * N * C) : nullptr;
+    // BT_FLAG_RECOMPUTE_GELU: likewise for the GELU output planes (the largest saved activation); the
+    // backward pass forms them again from the pre-activation h, which is kept anyway
+    const bool recompute_gelu = (m->cfg.flags & BT_FLAG_RECOMPUTE_GELU) != 0;
+    float* gelu_shared = recompute_gelu ? b.take<float>(2 * N * F) : nullptr;
     for (int l = 0; l < m->L; ++l) {
         LayerAct& a = m->act[l];
         a.x = b.take<float>(N * C);
@@ -262,7 +266,7 @@ size_t layout(bt_model* m, uint8_t* base) {
         a.rstd2 = b.take<float>(N);
         a.m_s = recompute_ln ? ln_shared : b.take<float>(2 * N * C);
         a.h = b.take<float>(N * F);
-        a.g_s = b.take<float>(2 * N * F);
+        a.g_s = recompute_gelu ? gelu_shared : b.take<float>(2 * N * F);
     }
     m->xL = b.take<float>(N * C);
     m->meanf = b.take<float>(N);
@@ -906,6 +910,7 @@ static bt_status backward_impl(bt_model* m) {
     const int tanh_form = (m->cfg.flags & BT_FLAG_GELU_TANH) ? 1 : 0;
     const bool raw_qkv = simt_attn || ((C / H) != 64 && (C / H) != 128) || (m->cfg.flags & BT_FLAG_GEMM_SIMT);
     const bool recompute_ln = (m->cfg.flags & BT_FLAG_RECOMPUTE_LN) != 0;
+    const bool recompute_gelu = (m->cfg.flags & BT_FLAG_RECOMPUTE_GELU) != 0;
     auto G = [&](const Tensor& t) { return m->grads + t.off; };
     // data-parallel exchange: registry indices of the tensors whose gradients each launch group finishes
     const int nT = (int)m->tensors.size();
@@ -929,6 +934,8 @@ static bt_status backward_impl(bt_model* m) {
         auto LT = [&](int k) -> Tensor& { return layer_tensor(m, l, k); };
         // MLP down-projection: x_out = x1 + g . Wpr^T + bpr
         BT_GEMM(kNN, N, F, C, dres, weight_mat(m, LT(PRW), C, F), m->dg, nullptr, nullptr);
+        if (recompute_gelu)   // g = GELU(h) again, as hi/lo planes (the same function of the same values as the epilogue's)
+            BT_STEP(kCatGeluFwd, 0, 12.0 * N * F, launch_gelu_fwd(a.h, N * F, tanh_form, nullptr, a.g_s, a.g_s + N * F, s));
         BT_GEMM(kTN, C, F, N, dres, act_mat(a.g_s, N, F, N), G(LT(PRW)), nullptr, nullptr);
         BT_DDP_READY(LI(l, PRW));
         // d h, with its column sums (the gradient of bfc) taken in the same pass

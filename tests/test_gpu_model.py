@@ -199,8 +199,9 @@ def test_tiny_config_three_steps(flags):
 
 def test_recomputed_layernorm_outputs_give_the_same_step():
     """BT_FLAG_RECOMPUTE_LN keeps one LayerNorm output buffer instead of two per layer and re-runs the
-    LayerNorm forward in the backward pass; BT_FLAG_LOGITS_IN_PLACE writes the logit gradient's hi
-    plane over the logits.  Same kernels on the same inputs, so the whole step is bit-identical to
+    LayerNorm forward in the backward pass; BT_FLAG_RECOMPUTE_GELU does the same for the GELU output
+    planes; BT_FLAG_LOGITS_IN_PLACE writes the logit gradient's hi plane over the logits.  Same
+    functions of the same inputs, so the whole step is bit-identical to
     the default layout, with a smaller workspace; and it matches the oracle."""
     cfg = si.make_config(n_layers=2, d_model=768, n_heads=12, seq_len=200, vocab_size=4000, padded_vocab_size=4032,
                          batch=3, tokens="zipf")
@@ -208,7 +209,7 @@ def test_recomputed_layernorm_outputs_give_the_same_step():
     tok, tgt = si.tokens_for(cfg, 3000, 3)
     opt = b.make_adamw(**si.ADAMW)
     outs, sizes = [], []
-    for flags in (0, b.BT_FLAG_RECOMPUTE_LN | b.BT_FLAG_LOGITS_IN_PLACE):
+    for flags in (0, b.BT_FLAG_RECOMPUTE_LN | b.BT_FLAG_LOGITS_IN_PLACE | b.BT_FLAG_RECOMPUTE_GELU):
         gm = b.Model(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["seq_len"], cfg["vocab_size"],
                      cfg["padded_vocab_size"], 3, flags)
         gm.load_params(params)
@@ -219,8 +220,9 @@ def test_recomputed_layernorm_outputs_give_the_same_step():
     assert outs[0][0] == outs[1][0]
     assert torch.equal(outs[0][1], outs[1][1]) and torch.equal(outs[0][2], outs[1][2])
     N, C, L = 3 * 200, 768, 2
-    assert sizes[0] - sizes[1] >= (2 * L - 1) * 2 * N * C * 4 + N * 4032 * 4   # 2L - 1 plane pairs and one logits array fewer
-    run_steps(cfg, seed=3, flags=b.BT_FLAG_RECOMPUTE_LN, B=3, steps=1, max_outside=1e-3)
+    # 2L - 1 LayerNorm plane pairs, L - 1 GELU plane pairs and one logits array fewer
+    assert sizes[0] - sizes[1] >= (2 * L - 1) * 2 * N * C * 4 + (L - 1) * 2 * N * 4 * C * 4 + N * 4032 * 4
+    run_steps(cfg, seed=3, flags=b.BT_FLAG_RECOMPUTE_LN | b.BT_FLAG_RECOMPUTE_GELU, B=3, steps=1, max_outside=1e-3)
     gm = b.Model(cfg["n_layers"], cfg["d_model"], cfg["n_heads"], cfg["seq_len"], cfg["vocab_size"],
                  cfg["padded_vocab_size"], 3, b.BT_FLAG_LOGITS_IN_PLACE)
     gm.load_params(params)
