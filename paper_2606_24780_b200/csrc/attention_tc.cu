@@ -34,10 +34,22 @@ using namespace tc;
 namespace {
 
 constexpr int HD = 64, BQ = 128, BKV = 64;
-constexpr int kThreads = 384;   // TMA warp, two MMA-issuing warps, a spare, two softmax warpgroups
+// Warps 0-7: the two softmax warpgroups (a warp's TMEM lane quadrant is its index mod 4); warp 8: TMA
+// producer; warps 9, 10: the two MMA issuers.  Eleven warps leave 184 registers per thread.
+constexpr int kThreads = 352;
+constexpr int kWarpProducer = 8, kWarpMmaS = 9, kWarpMmaO = 10;
 constexpr uint32_t kQBytes = 2u * 2u * BQ * 128u;      // 2 k-blocks x (hi, lo) x 128 rows x 128 B
-constexpr uint32_t kKVBytes = 2u * 2u * BKV * 128u;    // per buffer
-constexpr uint32_t kSmemBytes = 1024u + kQBytes + 4u * kKVBytes + 256u;
+constexpr uint32_t kKVBytes = 2u * 2u * BKV * 128u;    // one K or V tile (hi, lo)
+// K and V tiles share one ring of five slots, filled in the order K0 K1 V0 K2 V1 K3 V2 ...: the load
+// at position p goes to slot p mod 5 once the load at position p - 5 has been consumed.  K(t) then
+// takes over the slot of V(t-4) and V(t) the slot of K(t-1), so a K tile is requested three tile
+// periods before its product and a V tile more than one period before its own: a tile load takes
+// about 1.5 tile periods to arrive, which a two-deep ring per operand cannot cover.
+constexpr int kSlots = 5;
+constexpr uint32_t kSmemBytes = 1024u + kQBytes + kSlots * kKVBytes + 256u;
+static_assert(kSmemBytes <= 232448u, "shared memory");
+__device__ __forceinline__ int pos_k(int t) { return t == 0 ? 0 : 2 * t - 1; }
+__device__ __forceinline__ int pos_v(int t) { return 2 * t + 2; }
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr float kLn2 = 0.6931471805599453f;
 
@@ -67,21 +79,18 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t q_s = smem_base;
-    const uint32_t k_s = q_s + kQBytes;            // two buffers
-    const uint32_t v_s = k_s + 2u * kKVBytes;      // two buffers
-    const uint32_t bars = v_s + 2u * kKVBytes;
+    const uint32_t ring_s = q_s + kQBytes;         // kSlots tiles
+    const uint32_t bars = ring_s + kSlots * kKVBytes;
     // barrier slots
     const uint32_t q_full = bars;
-    auto k_full = [&](int b) { return bars + 8u * (1 + b); };
-    auto k_empty = [&](int b) { return bars + 8u * (3 + b); };
-    auto v_full = [&](int b) { return bars + 8u * (5 + b); };
-    auto v_empty = [&](int b) { return bars + 8u * (7 + b); };
-    auto s_full = [&](int b) { return bars + 8u * (9 + b); };
-    auto p_full = [&](int b) { return bars + 8u * (11 + b); };
-    auto o_full = [&](int b) { return bars + 8u * (13 + b); };
-    const uint32_t merge_full = bars + 8u * 15;
-    const uint32_t all_done = bars + 8u * 16;
-    const uint32_t tmem_slot = bars + 8u * 17;
+    auto slot_full = [&](int i) { return bars + 8u * (1 + i); };
+    auto slot_empty = [&](int i) { return bars + 8u * (6 + i); };
+    auto s_full = [&](int b) { return bars + 8u * (11 + b); };
+    auto p_full = [&](int b) { return bars + 8u * (13 + b); };
+    auto o_full = [&](int b) { return bars + 8u * (15 + b); };
+    const uint32_t merge_full = bars + 8u * 17;
+    const uint32_t all_done = bars + 8u * 18;
+    const uint32_t tmem_slot = bars + 8u * 19;
     volatile uint32_t* tmem_slot_ptr =
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
@@ -95,11 +104,11 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
     if (threadIdx.x == 0) {
         mbar_init(q_full, 1);
+        for (int i = 0; i < kSlots; ++i) {
+            mbar_init(slot_full(i), 1);
+            mbar_init(slot_empty(i), 1);
+        }
         for (int i = 0; i < 2; ++i) {
-            mbar_init(k_full(i), 1);
-            mbar_init(k_empty(i), 1);
-            mbar_init(v_full(i), 1);
-            mbar_init(v_empty(i), 1);
             mbar_init(s_full(i), 1);
             mbar_init(p_full(i), 4);
             mbar_init(o_full(i), 1);
@@ -108,7 +117,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         mbar_init(all_done, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    if (warp == 1) {
+    if (warp == kWarpMmaS) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(tmem_slot), "r"(512u)
                      : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -120,31 +129,33 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
     pdl_wait();      // set-up done; global memory is touched from here on
     pdl_trigger();
 
-    if (warp == 0) {
+    if (warp == kWarpProducer) {
         // ------------------------------------------------------------ TMA producer
         if (lane == 0) {
             mbar_expect_tx(q_full, kQBytes);
             for (int kb = 0; kb < 2; ++kb)
                 tma_load_3d(q_s + kb * (kQBytes / 2), &tmQ, q_full, h * HD + kb * 32, row_base + q0, 0);
             bool ok = true;
-            for (int kt = 0; kt < n_kt && ok; ++kt) {
-                const int buf = kt & 1;
-                const uint32_t ph = (kt >> 1) & 1u;
-                if (!mbar_wait(k_empty(buf), ph ^ 1u, g.err, 11)) { ok = false; break; }
-                mbar_expect_tx(k_full(buf), kKVBytes);
-                for (int kb = 0; kb < 2; ++kb)
-                    tma_load_3d(k_s + buf * kKVBytes + kb * (kKVBytes / 2), &tmK, k_full(buf),
-                                g.C + h * HD + kb * 32, row_base + kt * BKV, 0);
-                if (!mbar_wait(v_empty(buf), ph ^ 1u, g.err, 12)) { ok = false; break; }
-                mbar_expect_tx(v_full(buf), kKVBytes);
-                for (int grp = 0; grp < 2; ++grp)
-                    tma_load_3d(v_s + buf * kKVBytes + grp * (kKVBytes / 2), &tmV, v_full(buf),
-                                2 * g.C + h * HD + grp * 32, row_base + kt * BKV, 0);
+            const int n_pos = pos_v(n_kt - 1) + 1;
+            int slot = 0;
+            uint32_t round = 0;                          // p / kSlots
+            for (int p = 0; p < n_pos && ok; ++p) {
+                const bool is_k = p == 0 || (p & 1);
+                const int t = p == 0 ? 0 : (is_k ? (p + 1) >> 1 : (p - 2) >> 1);
+                if (t < n_kt) {                          // only K(n_kt) near the end falls outside
+                    if (!mbar_wait(slot_empty(slot), (round & 1u) ^ 1u, g.err, is_k ? 11 : 12)) { ok = false; break; }
+                    mbar_expect_tx(slot_full(slot), kKVBytes);
+                    const uint32_t dst = ring_s + (uint32_t)slot * kKVBytes;
+                    for (int kb = 0; kb < 2; ++kb)
+                        tma_load_3d(dst + kb * (kKVBytes / 2), is_k ? &tmK : &tmV, slot_full(slot),
+                                    (is_k ? g.C : 2 * g.C) + h * HD + kb * 32, row_base + t * BKV, 0);
+                }
+                if (++slot == kSlots) { slot = 0; ++round; }
             }
             if (!ok)
                 for (int i = 0; i < 2000; ++i) __nanosleep(1000);  // let loads in flight land
         }
-    } else if (warp == 1) {
+    } else if (warp == kWarpMmaS) {
         // ------------------------------------------------------------ MMA issuer 1: S = Q K^T
         if (lane == 0) {
             constexpr uint32_t idesc_s = make_idesc_tf32(BQ, BKV, false, false);
@@ -152,13 +163,14 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
             const DescBase qd = make_desc_base(q_s, 16u, 1024u, 2u);
             for (int kt = 0; kt < n_kt && ok; ++kt) {
                 const int buf = kt & 1;
-                if (!mbar_wait(k_full(buf), (kt >> 1) & 1u, g.err, 14)) { ok = false; break; }
+                const int pk = pos_k(kt), slot = pk % kSlots;
+                if (!mbar_wait(slot_full(slot), (uint32_t)(pk / kSlots) & 1u, g.err, 14)) { ok = false; break; }
                 // S[buf] is free once the softmax of tile kt-2 has read it (it then publishes P)
                 if (kt >= 2 && !mbar_wait(p_full(buf), ((kt - 2) >> 1) & 1u, g.err, 20)) { ok = false; break; }
                 tc_fence_after();
                 trace_mark(g.trace, 100 + kt);
                 const uint32_t d = tmem_base + (uint32_t)buf * 256u;
-                const DescBase kd = make_desc_base(k_s + buf * kKVBytes, 16u, 1024u, 2u);
+                const DescBase kd = make_desc_base(ring_s + (uint32_t)slot * kKVBytes, 16u, 1024u, 2u);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint32_t qo = (uint32_t)(ks >> 2) * (kQBytes / 2) + (uint32_t)(ks & 3) * 32u;
@@ -169,12 +181,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     umma_tf32(d, a_hi, b_lo, idesc_s, 1u);
                     umma_tf32(d, a_hi, b_hi, idesc_s, 1u);
                 }
-                umma_commit(k_empty(buf));
+                umma_commit(slot_empty(slot));
                 umma_commit(s_full(buf));
                 trace_mark(g.trace, 200 + kt);
             }
         }
-    } else if (warp == 2) {
+    } else if (warp == kWarpMmaO) {
         // ------------------------------------------------------------ MMA issuer 2: O_tile = P V
         // A second issuing thread: the two products of a tile go to different accumulators and are
         // ordered only through the barriers, so their instruction streams can be issued in parallel.
@@ -185,12 +197,13 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 const int buf = kt & 1;
                 // P(kt) published; the softmax warps read O[buf] of tile kt-2 before publishing it
                 if (!mbar_wait(p_full(buf), (kt >> 1) & 1u, g.err, 15)) { ok = false; break; }
-                if (!mbar_wait(v_full(buf), (kt >> 1) & 1u, g.err, 16)) { ok = false; break; }
+                const int pv = pos_v(kt), slot = pv % kSlots;
+                if (!mbar_wait(slot_full(slot), (uint32_t)(pv / kSlots) & 1u, g.err, 16)) { ok = false; break; }
                 tc_fence_after();
                 trace_mark(g.trace, 300 + kt);
                 const uint32_t t0 = tmem_base + (uint32_t)buf * 256u;
                 const uint32_t d = t0 + 192u;
-                const DescBase vd = make_desc_base(v_s + buf * kKVBytes, kKVBytes / 2, 512u, 1u);
+                const DescBase vd = make_desc_base(ring_s + (uint32_t)slot * kKVBytes, kKVBytes / 2, 512u, 1u);
 #pragma unroll
                 for (int j = 0; j < 8; ++j) {
                     const uint64_t b_hi = vd.at(j * 1024u), b_lo = vd.at(BKV * 128u + j * 1024u);
@@ -198,20 +211,18 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                     umma_tf32_ts(d, t0 + 64u + j * 8u, b_lo, idesc_o, 1u);                // P_hi V_lo
                     umma_tf32_ts(d, t0 + 64u + j * 8u, b_hi, idesc_o, 1u);                // P_hi V_hi
                 }
-                umma_commit(v_empty(buf));
+                umma_commit(slot_empty(slot));
                 umma_commit(o_full(buf));
                 trace_mark(g.trace, 400 + kt);
             }
             if (ok) umma_commit(all_done);
         }
-    } else if (warp == 3) {
-        // idle (keeps the softmax warps' TMEM lane quadrants aligned with warp index mod 4)
-    } else {
+    } else if (warp < 8) {
         // ------------------------------------------------------------ softmax / correction warps
-        // Two warpgroups (warps 4-7 and 8-11) take alternate key tiles, each with its own running
+        // Two warpgroups (warps 0-3 and 4-7) take alternate key tiles, each with its own running
         // maximum, sum and output; they are merged at the end.  Two warps per scheduler hide each
         // other's instruction latencies.
-        const int wg = (warp - 4) >> 2;                              // 0 or 1; owns TMEM buffer wg
+        const int wg = warp >> 2;                                    // 0 or 1; owns TMEM buffer wg
         const int lane_group = warp & 3;
         const int rloc = lane_group * 32 + lane;                    // row inside the CTA
         const int row = q0 + rloc;                                   // query row of this thread
@@ -297,9 +308,9 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         }
         if (ok && last >= 0) ok = add_output(last, corr_prev);
 
-        // merge: warpgroup 1 hands (m, l, O) of its rows to warpgroup 0 through the K buffers, which
-        // are idle once every tile's products have completed
-        float* xch = reinterpret_cast<float*>(smem_raw + (k_s - smem_u32(smem_raw)));   // [128][66]
+        // merge: warpgroup 1 hands (m, l, O) of its rows to warpgroup 0 through the first ring slots,
+        // which are idle once every tile's products have completed
+        float* xch = reinterpret_cast<float*>(smem_raw + (ring_s - smem_u32(smem_raw)));   // [128][66]
         if (wg == 1) {
             if (ok) ok = mbar_wait_warp(all_done, 0, g.err, 21);   // no product still reads the K buffers
             float* dst = xch + rloc * 66;
@@ -321,12 +332,12 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
                 m = mm;
 #pragma unroll
                 for (int i = 0; i < HD; ++i) o_reg[i] = o_reg[i] * f0 + src[i] * f1;
-                // the rows leave in full 128-byte segments through a slice of the idle V buffers
+                // the rows leave in full 128-byte segments through a slice of the idle third ring slot
                 const float inv = 1.0f / l;
                 const int wrow0 = q0 + lane_group * 32;                 // first query row of this warp
                 const int nvalid = max(0, min(32, g.T - wrow0));
                 const int64_t off0 = ((int64_t)(row_base + wrow0)) * g.C + h * HD;
-                float* tile = reinterpret_cast<float*>(smem_raw + (v_s - smem_u32(smem_raw)) + (uint32_t)lane_group * kRowTileBytes);
+                float* tile = reinterpret_cast<float*>(smem_raw + (ring_s + 2u * kKVBytes - smem_u32(smem_raw)) + (uint32_t)lane_group * kRowTileBytes);
 #pragma unroll
                 for (int half = 0; half < 2; ++half) {
                     float v[32];
@@ -343,7 +354,7 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
 
     tc_fence_before();
     __syncthreads();
-    if (warp == 1) {
+    if (warp == kWarpMmaS) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
 }
