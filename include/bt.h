@@ -146,7 +146,9 @@ BT_API bt_status bt_tensor_info(const bt_model* m, int32_t index, const char** n
 BT_API bt_status bt_tensor_ptr(bt_model* m, const char* name, int32_t kind, float** d_ptr);
 
 /* Activations of the last forward/backward, for tests: per-layer "x", "qkv" (raw; written only
- * when head_dim is neither 64 nor 128 or a reference-kernel flag is set), "x1", "h",
+ * when head_dim is neither 64 nor 128 or a reference-kernel flag is set), "x1", "h" (the MLP
+ * pre-activation; without BT_FLAG_RECOMPUTE_GELU and BT_FLAG_GEMM_SIMT the array holds GELU'(h),
+ * all the backward pass needs of it),
  * "ln1.mean", "ln1.rstd", "ln2.mean", "ln2.rstd", "lse"; split per-layer "qkv_split", "a", "o", "m", "g"
  * (pointer to the hi plane; lo plane follows at +numel); global "xL", "logits", "losses",
  * split "xf", "dlogits".  `numel` (nullable) receives the element count of one plane for
@@ -445,6 +447,21 @@ BT_API bt_status bt_op_gemm_split_act(int32_t layout, int64_t M, int64_t N, int6
                                       const float* bias, const float* residual, void* scratch,
                                       size_t scratch_bytes, uint32_t flags, void* stream);
 BT_API bt_status bt_op_gemm_check(const void* scratch, void* stream);
+/* The input-gradient product of the MLP down-projection with the GELU backward in its epilogue
+ * (Kernel Design, fused element-wise epilogues; Appendix B "GELU Backward"): with dy_split
+ * [2][M][K] (hi/lo planes of the gradient at the projection's output), w_split [2][K][N] (the
+ * projection's weight, [out, in] = [K, N]) and h [M][N] (the pre-activation kept by the forward),
+ *   dh_split [2][M][N] = hi/lo planes of (dy . W) o GELU'(h)     (tanh_form 0: erf form, 1: tanh form)
+ *   colsum [N]          = the column sums of that product over the M rows, added per 32-row
+ *                         group in row order (the bias gradient of the up-projection).
+ * All pointers device, 16-byte aligned; N a multiple of 32, M and K multiples of 4.  `scratch`
+ * (256-byte aligned, bt_op_gemm_gelu_bwd_scratch_bytes(M, N) bytes) holds the group sums and the
+ * error word bt_op_gemm_check reads.  Asynchronous.  flags as for bt_op_gemm_split
+ * (BT_FLAG_GEMM_SIMT is not supported here: BT_ERR_UNSUPPORTED). */
+BT_API size_t bt_op_gemm_gelu_bwd_scratch_bytes(int64_t M, int64_t N);
+BT_API bt_status bt_op_gemm_gelu_bwd(int64_t M, int64_t N, int64_t K, const float* dy_split, const float* w_split,
+                                     const float* h, int32_t tanh_form, float* dh_split, float* colsum,
+                                     void* scratch, size_t scratch_bytes, uint32_t flags, void* stream);
 
 /* Convenience form on raw FP32 operands: bt_op_split of A and B into `scratch`, then
  * bt_op_gemm_split, then bt_op_gemm_check (synchronises). */

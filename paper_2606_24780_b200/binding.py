@@ -106,6 +106,8 @@ _SIGNATURES = {
     "bt_op_gemm_split_scratch_bytes": (_sz, []),
     "bt_op_gemm_split": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
     "bt_op_gemm_split_act": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 4 + [_i32] + [_vp] * 3 + [_sz, _u32, _vp]),
+    "bt_op_gemm_gelu_bwd_scratch_bytes": (_sz, [_i64, _i64]),
+    "bt_op_gemm_gelu_bwd": (_i32, [_i64, _i64, _i64] + [_vp] * 3 + [_i32] + [_vp] * 3 + [_sz, _u32, _vp]),
     "bt_op_gemm_check": (_i32, [_vp, _vp]),
     "bt_op_gemm": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
     "bt_op_attention_fwd": (_i32, [_vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _u32, _vp]),
@@ -507,6 +509,16 @@ def bt_op_gemm_split(layout, M, N, K, A_split, B_split, D, bias, residual, scrat
                      stream=None):
     _check(lib().bt_op_gemm_split(layout, M, N, K, _ptr(A_split), _ptr(B_split), _ptr(D), _ptr(bias), _ptr(residual),
                                   _ptr(scratch), scratch_bytes, flags, _stream(stream)))
+
+
+def bt_op_gemm_gelu_bwd_scratch_bytes(M, N):
+    return lib().bt_op_gemm_gelu_bwd_scratch_bytes(M, N)
+
+
+def bt_op_gemm_gelu_bwd(M, N, K, dy_split, w_split, h, tanh_form, dh_split, colsum, scratch, scratch_bytes, flags=0,
+                        stream=None):
+    _check(lib().bt_op_gemm_gelu_bwd(M, N, K, _ptr(dy_split), _ptr(w_split), _ptr(h), int(tanh_form), _ptr(dh_split),
+                                     _ptr(colsum), _ptr(scratch), scratch_bytes, flags, _stream(stream)))
 
 
 def bt_op_gemm_check(scratch, stream=None):

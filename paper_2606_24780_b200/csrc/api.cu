@@ -129,7 +129,7 @@ struct bt_model {
     uint8_t* decay_flags;
     std::vector<LayerAct> act;
     float *xL, *meanf, *rstdf, *xf_s, *logits, *dlogits_s, *losses, *loss, *norm_out;
-    float *dres, *dres_s, *dtmp, *do_s, *dqkv_s, *dh_s, *dg, *dvec, *attn_rg;
+    float *dres, *dres_s, *dtmp, *do_s, *dqkv_s, *dh_s, *dg, *dh_groups, *dvec, *attn_rg;
     float *partials, *ln_scratch, *colsum_scratch;
     void* norm_scratch;
     size_t partial_floats;
@@ -287,7 +287,11 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->do_s = b.take<float>(2 * N * C);
     m->dqkv_s = b.take<float>(2 * N * 3 * C);
     m->dh_s = b.take<float>(2 * N * F);
-    m->dg = b.take<float>(N * F);
+    // d g (the GELU output's gradient) exists as an array only with the FMA reference GEMM; the
+    // tensor-core GEMM applies GELU' in its epilogue and leaves column sums per 32-row group instead
+    const bool simt_gemm = (m->cfg.flags & BT_FLAG_GEMM_SIMT) != 0;
+    m->dg = simt_gemm ? b.take<float>(N * F) : nullptr;
+    m->dh_groups = simt_gemm ? nullptr : b.take<float>(((N + 31) / 32) * F);
     m->dvec = b.take<float>((int64_t)m->maxB * m->H * m->T);
     m->attn_rg = b.take<float>(attention_bwd_rowgroups(m->maxB, m->T) * 3 * m->C);
     section(5);                      // backward temporaries (reused by every layer)
@@ -372,9 +376,16 @@ inline double attn_fwd_flops(int64_t B, int64_t H, int64_t T, int64_t d) {
     return 4.0 * (double)B * H * d * ((double)T * (T + 1) / 2.0);
 }
 
+// The forward pass keeps GELU'(h) in the place of h = m Wfc^T + bfc unless h is needed again (GELU
+// recomputed in the backward pass) or the FMA reference GEMM, which has no fused epilogues, runs.
+inline bool h_holds_gelu_grad(const bt_model* m) {
+    return !(m->cfg.flags & (BT_FLAG_GEMM_SIMT | BT_FLAG_RECOMPUTE_GELU));
+}
+
 // D = op(A) op(B) (+bias)(+residual) through the tensor-core kernel or the FMA reference.
 cudaError_t gemm_raw(bt_model* m, int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
-                 const float* bias, const float* residual, float* d_split = nullptr, int act = 0) {
+                 const float* bias, const float* residual, float* d_split = nullptr, int act = 0,
+                 float* col_partial = nullptr) {
     if (m->cfg.flags & BT_FLAG_GEMM_SIMT) {
         // the FMA reference writes the raw output; the planes are made by a separate pass
         cudaError_t e = launch_gemm_simt(layout, M, N, K, A, B, D, N, bias, residual, m->stream);
@@ -385,7 +396,7 @@ cudaError_t gemm_raw(bt_model* m, int layout, int64_t M, int64_t N, int64_t K, S
         return e;
     }
     return launch_gemm_tc(layout, M, N, K, A, B, D, N, bias, residual, m->partials, m->partial_floats, m->err_word,
-                          m->stream, d_split, M * N, -1, act);
+                          m->stream, d_split, M * N, -1, act, col_partial);
 }
 
 // Timing category by role: the forward products (Y = X W^T, run as NN on the transposed weight
@@ -862,10 +873,11 @@ extern "C" bt_status bt_forward(bt_model* m, const int32_t* d_tokens, const int3
         BT_GEMM(kNN, N, C, C, act_mat(a.o_s, N, C, N), weight_mat_t(m, layer_tensor(m, l, PROJW), C, C), a.x1,
                      P(PROJB), a.x);
         BT_STEP(kCatLnFwd, 0, 12.0 * N * C, launch_layernorm_fwd(a.x1, P(LN2G), P(LN2B), N, C, nullptr, a.m_s, a.m_s + N * C, a.mean2, a.rstd2, s));
-        // h = m Wfc^T + bfc is kept (the backward needs it); g = GELU(h) leaves the same epilogue as hi/lo planes
+        // g = GELU(h), h = m Wfc^T + bfc, leaves the epilogue as hi/lo planes; what the backward needs of h
+        // is GELU'(h), which the same epilogue writes in its place (h itself when GELU is recomputed later)
         BT_STEP(kCatGemmNT, gemm_flops(N, F, C), gemm_bytes(N, F, C) + 8.0 * N * F,
                 gemm_raw(m, kNN, N, F, C, act_mat(a.m_s, N, C, N), weight_mat_t(m, layer_tensor(m, l, FCW), F, C), a.h,
-                         P(FCB), nullptr, a.g_s, tanh_form ? 2 : 1));
+                         P(FCB), nullptr, a.g_s, (tanh_form ? 2 : 1) + (h_holds_gelu_grad(m) ? 2 : 0)));
         BT_GEMM(kNN, N, C, F, act_mat(a.g_s, N, F, N), weight_mat_t(m, layer_tensor(m, l, PRW), C, F), xout,
                      P(PRB), a.x1);
     }
@@ -933,14 +945,25 @@ static bt_status backward_impl(bt_model* m) {
         LayerAct& a = m->act[l];
         auto LT = [&](int k) -> Tensor& { return layer_tensor(m, l, k); };
         // MLP down-projection: x_out = x1 + g . Wpr^T + bpr
-        BT_GEMM(kNN, N, F, C, dres, weight_mat(m, LT(PRW), C, F), m->dg, nullptr, nullptr);
+        // d h = (d x_out . Wpr) o GELU'(h): the GELU backward runs in the product's epilogue (a plain
+        // multiplication where the forward pass left GELU'(h)), which also leaves the column sums of
+        // d h per 32-row group (added up below: the gradient of bfc)
+        const bool fused_gelu_bwd = m->dg == nullptr;
+        if (fused_gelu_bwd)
+            BT_STEP(kCatGemmNN, gemm_flops(N, F, C), gemm_bytes(N, F, C) + 8.0 * N * F,
+                    gemm_raw(m, kNN, N, F, C, dres, weight_mat(m, LT(PRW), C, F), nullptr, nullptr, a.h, m->dh_s,
+                             h_holds_gelu_grad(m) ? 7 : tanh_form ? 6 : 5, m->dh_groups));
+        else
+            BT_GEMM(kNN, N, F, C, dres, weight_mat(m, LT(PRW), C, F), m->dg, nullptr, nullptr);
         if (recompute_gelu)   // g = GELU(h) again, as hi/lo planes (the same function of the same values as the epilogue's)
             BT_STEP(kCatGeluFwd, 0, 12.0 * N * F, launch_gelu_fwd(a.h, N * F, tanh_form, nullptr, a.g_s, a.g_s + N * F, s));
         BT_GEMM(kTN, C, F, N, dres, act_mat(a.g_s, N, F, N), G(LT(PRW)), nullptr, nullptr);
         BT_DDP_READY(LI(l, PRW));
-        // d h, with its column sums (the gradient of bfc) taken in the same pass
-        BT_STEP(kCatGeluBwd, 0, 16.0 * N * F, launch_gelu_bwd_colsum(a.h, m->dg, N, F, tanh_form, nullptr, m->dh_s, m->dh_s + N * F,
-                                       G(LT(FCB)), m->colsum_scratch, s));
+        if (fused_gelu_bwd)
+            BT_STEP(kCatColsum, 0, 4.0 * ((N + 31) / 32) * F, launch_colsum_stage2(m->dh_groups, (int)((N + 31) / 32), (int)F, G(LT(FCB)), s));
+        else   // d h, with its column sums taken in the same pass
+            BT_STEP(kCatGeluBwd, 0, 16.0 * N * F, launch_gelu_bwd_colsum(a.h, m->dg, N, F, tanh_form, nullptr, m->dh_s, m->dh_s + N * F,
+                                           G(LT(FCB)), m->colsum_scratch, s));
         BT_DDP_READY(LI(l, FCB));
         // MLP up-projection: h = m . Wfc^T + bfc
         SplitMat dh = act_mat(m->dh_s, N, F, N);
@@ -1268,6 +1291,35 @@ extern "C" bt_status bt_op_gemm_split_act(int32_t layout, int64_t M, int64_t N, 
     if (!D_act_split) return fail(BT_ERR_INVALID_ARG, "gemm_split_act: D_act_split is NULL");
     return gemm_split_impl(layout, M, N, K, A_split, B_split, D, D_act_split, act, bias, residual, scratch,
                            scratch_bytes, flags, stream);
+}
+
+extern "C" size_t bt_op_gemm_gelu_bwd_scratch_bytes(int64_t M, int64_t N) {
+    if (M < 1 || N < 1) return 0;
+    return bt_op_gemm_split_scratch_bytes() + pad256(((M + 31) / 32) * N) * sizeof(float);
+}
+
+extern "C" bt_status bt_op_gemm_gelu_bwd(int64_t M, int64_t N, int64_t K, const float* dy_split, const float* w_split,
+                                         const float* h, int32_t tanh_form, float* dh_split, float* colsum,
+                                         void* scratch, size_t scratch_bytes, uint32_t flags, void* stream) {
+    BT_PTR(dy_split); BT_PTR(w_split); BT_PTR(h); BT_PTR(dh_split); BT_PTR(colsum); BT_PTR(scratch);
+    if (M < 1 || N < 1 || K < 1 || M % 4 || N % 32 || K % 4) return fail(BT_ERR_INVALID_ARG, "gemm_gelu_bwd: bad sizes");
+    if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return fail(BT_ERR_INVALID_ARG, "gemm_gelu_bwd: size too large");
+    if (flags & BT_FLAG_GEMM_SIMT) return fail(BT_ERR_UNSUPPORTED, "gemm_gelu_bwd: tensor-core kernels only");
+    if (scratch_bytes < bt_op_gemm_gelu_bwd_scratch_bytes(M, N)) return fail(BT_ERR_OOM, "gemm_gelu_bwd: scratch too small");
+    if (reinterpret_cast<uintptr_t>(scratch) & 255u) return fail(BT_ERR_INVALID_ARG, "gemm_gelu_bwd: scratch not 256-byte aligned");
+    char msg[256];
+    if (!gemm_tc_init(msg, sizeof(msg))) return fail(BT_ERR_CUDA, "tensor-core GEMM unavailable: %s", msg);
+    cudaStream_t s = (cudaStream_t)stream;
+    float* partials = (float*)scratch;
+    int* err = (int*)(partials + gemm_tc_partial_floats_bound());
+    float* groups = (float*)((uint8_t*)scratch + bt_op_gemm_split_scratch_bytes());
+    BT_CUDA(cudaMemsetAsync(err, 0, sizeof(int), s));
+    SplitMat Am{dy_split, M * K, M, K, K}, Bm{w_split, K * N, K, N, N};
+    const int two_cta_mode = (flags & BT_FLAG_GEMM_PAIR) ? 1 : (flags & BT_FLAG_GEMM_SINGLE) ? 0 : -1;
+    BT_CUDA(launch_gemm_tc(BT_GEMM_NN, M, N, K, Am, Bm, nullptr, N, nullptr, h, partials, gemm_tc_partial_floats_bound(), err,
+                           s, dh_split, M * N, two_cta_mode, tanh_form ? 6 : 5, groups));
+    BT_CUDA(launch_colsum_stage2(groups, (int)((M + 31) / 32), (int)N, colsum, s));
+    return BT_OK;
 }
 
 extern "C" bt_status bt_op_gemm_check(const void* scratch, void* stream) {

@@ -78,13 +78,55 @@ struct SplitMat {
 };
 
 #ifdef __CUDACC__
-// GELU (exact erf form, or the tanh form): shared by the GELU kernels and the GEMM epilogue.
-__device__ __forceinline__ float gelu_f(float x, bool tanh_form) {
+// GELU and its derivative (erf form, or the tanh form): shared by the GELU kernels and the GEMM
+// epilogues, where four warps per SM evaluate them for a whole output tile -- hence branch-free and
+// about twenty instructions for both values together.
+//   erf form:  GELU(x) = x Phi(x),  GELU'(x) = Phi(x) + x phi(x), with one exponential
+//              E = exp(-x^2 / 2) shared by phi and by the complementary error function, which is
+//              the five-term rational approximation of Abramowitz & Stegun 7.1.26 (absolute error
+//              1.5e-7 on erf: about one FP32 rounding of Phi);
+//   tanh form: tanh(u) = 1 - 2 / (1 + exp(2u)),  u = sqrt(2 / pi) (x + 0.044715 x^3).
+__device__ __forceinline__ float ex2_fast(float x) {
+    float y;
+    asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_fast(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ void gelu_both_f(float x, bool tanh_form, float& g, float& gp) {
     if (tanh_form) {
-        float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-        return 0.5f * x * (1.0f + tanhf(u));
+        const float x2 = x * x;
+        const float u = 0.7978845608028654f * fmaf(0.044715f * x2, x, x);
+        const float t = 1.0f - 2.0f * rcp_fast(1.0f + ex2_fast(2.8853900817779268f * u));   // exp(2u) = 2^(2u log2 e)
+        const float du = 0.7978845608028654f * fmaf(3.0f * 0.044715f, x2, 1.0f);
+        const float half = 0.5f * (1.0f + t);
+        g = x * half;
+        gp = fmaf(0.5f * x * du, fmaf(-t, t, 1.0f), half);
+        return;
     }
-    return 0.5f * x * (1.0f + erff(x * 0.7071067811865476f));
+    const float E = ex2_fast(-0.7213475204444817f * x * x);                  // exp(-x^2 / 2)
+    const float r = rcp_fast(fmaf(0.3275911f * 0.7071067811865476f, fabsf(x), 1.0f));
+    float q = fmaf(r, 1.061405429f, -1.453152027f);
+    q = fmaf(q, r, 1.421413741f);
+    q = fmaf(q, r, -0.284496736f);
+    q = fmaf(q, r, 0.254829592f);
+    const float half_erfc = 0.5f * q * r * E;                                // erfc(|x| / sqrt 2) / 2
+    const float Phi = x >= 0.f ? 1.0f - half_erfc : half_erfc;
+    g = x * Phi;
+    gp = fmaf(x * 0.3989422804014327f, E, Phi);
+}
+__device__ __forceinline__ float gelu_f(float x, bool tanh_form) {
+    float g, gp;
+    gelu_both_f(x, tanh_form, g, gp);
+    return g;
+}
+__device__ __forceinline__ float gelu_grad_f(float x, bool tanh_form) {
+    float g, gp;
+    gelu_both_f(x, tanh_form, g, gp);
+    return gp;
 }
 #endif
 
@@ -170,6 +212,7 @@ cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int
 int softmax_xent_max_in_place_columns();
 size_t colsum_scratch_floats(int64_t N, int C);
 // x_lo (nullable): second plane added to the first (sums a split array).
+cudaError_t launch_colsum_stage2(const float* partial, int groups, int C, float* out, cudaStream_t s);
 cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, float* out, float* scratch,
                           cudaStream_t s);
 // Gradient accumulation over micro-steps (see the kernel): n % 4 == 0.
@@ -213,8 +256,16 @@ cudaError_t launch_gemm_simt(int layout, int64_t M, int64_t N, int64_t K, SplitM
 cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D,
                            int64_t ldd, const float* bias, const float* residual, float* partials,
                            size_t max_partial_floats, int* err_word, cudaStream_t s, float* d_hi = nullptr,
-                           int64_t d_plane = 0, int two_cta_mode = -1, int act = 0);
-// act: 1 / 2 = the hi/lo planes receive GELU(output) (erf / tanh form) while D keeps the output itself.
+                           int64_t d_plane = 0, int two_cta_mode = -1, int act = 0, float* col_partial = nullptr);
+// act: 1 / 2 = the hi/lo planes receive GELU(output) (erf / tanh form) while D keeps the output itself;
+//      3 / 4 = the same planes, and D receives GELU'(output) instead of the output (what the backward
+//      pass needs of it);
+//      5 / 6 = GELU backward in the epilogue: `residual` holds the pre-activation h [M, N] and the
+//      output is (A B) o GELU'(h) (erf / tanh form) -- the input gradient of the GELU whose output
+//      fed the product that A B back-propagates through;  7 = the same with GELU'(h) already in
+//      `residual`.  In 5 - 7 col_partial (nullable) receives the column sums of the output per 32-row
+//      group, [ceil(M / 32)][N]: launch_colsum_stage2 adds the groups in order (the bias gradient of
+//      the layer that produced h); no bias, no K-split.
 // two_cta_mode: -1 the planner chooses between 128-row tiles on single CTAs and 256-row tiles on
 // CTA pairs (cta_group::2); 0 / 1 force the one or the other (1 applies where M >= 256).
 size_t gemm_tc_partial_floats_bound();

@@ -330,17 +330,6 @@ cudaError_t launch_embedding_bwd(const int32_t* tok, const float* dx, int64_t N,
 
 // ------------------------------------------------------------------ GELU
 
-__device__ __forceinline__ float gelu_grad_f(float x, bool tanh_form) {
-    if (tanh_form) {
-        float u = 0.7978845608028654f * (x + 0.044715f * x * x * x);
-        float t = tanhf(u);
-        float du = 0.7978845608028654f * (1.0f + 3.0f * 0.044715f * x * x);
-        return 0.5f * (1.0f + t) + 0.5f * x * (1.0f - t * t) * du;
-    }
-    // Phi(x) + x phi(x)
-    return 0.5f * (1.0f + erff(x * 0.7071067811865476f)) + x * 0.3989422804014327f * expf(-0.5f * x * x);
-}
-
 __global__ void __launch_bounds__(256) gelu_fwd_kernel(const float* __restrict__ x, int64_t n4, int tanh_form,
                                                        float* y, float* y_hi, float* y_lo) {
     pdl_wait();
@@ -451,6 +440,13 @@ __global__ void __launch_bounds__(256) colsum_stage2_kernel(const float* __restr
     float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
     if (c < C4) {
         int s = warp;
+        for (; s + 120 < strips; s += 128) {   // sixteen rows in flight per lane, added in the same (ascending) order
+            float4 a[16];
+#pragma unroll
+            for (int j = 0; j < 16; ++j) a[j] = ld4(partial, (int64_t)(s + 8 * j) * C4 + c);
+#pragma unroll
+            for (int j = 0; j < 16; ++j) t = add4(t, a[j]);
+        }
         for (; s + 24 < strips; s += 32) {
             float4 a0 = ld4(partial, (int64_t)s * C4 + c), a1 = ld4(partial, (int64_t)(s + 8) * C4 + c);
             float4 a2 = ld4(partial, (int64_t)(s + 16) * C4 + c), a3 = ld4(partial, (int64_t)(s + 24) * C4 + c);
@@ -546,6 +542,15 @@ cudaError_t launch_colsum(const float* x, const float* x_lo, int64_t N, int C, f
     BT_KERNEL_LAUNCH((colsum_stage1_kernel), grid, 256, 0, s, x, x_lo, N, C4, strips, scratch);
     BT_COUNT_LAUNCH();
     BT_KERNEL_LAUNCH((colsum_stage2_kernel), (C4 + 31) / 32, 256, 0, s, scratch, strips, C4, out);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+// Stage 2 alone: out[c] = the sum over the `groups` rows of partial [groups][C], in row order (for
+// producers that leave per-row-group column sums themselves).
+cudaError_t launch_colsum_stage2(const float* partial, int groups, int C, float* out, cudaStream_t s) {
+    const int C4 = C / 4;
+    BT_KERNEL_LAUNCH((colsum_stage2_kernel), (C4 + 31) / 32, 256, 0, s, partial, groups, C4, out);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }

@@ -74,7 +74,11 @@ struct GemmArgs {
     int* err;
     float* d_hi;        // optional TF32 hi/lo planes of the output (lo = d_hi + d_plane)
     long long d_plane;
-    int act;            // 0: the planes hold the output; 1 / 2: they hold GELU(output), erf / tanh form
+    int act;            // 0: the planes hold the output; 1 / 2: they hold GELU(output), erf / tanh form;
+                        // 3 / 4: as 1 / 2, and D holds GELU'(output) instead of the output;
+                        // 5 / 6: `residual` is a pre-activation h and the output is (A B) o GELU'(h);
+                        // 7: `residual` holds GELU'(h) itself and the output is (A B) o residual
+    float* col_partial; // act 5 - 7: column sums of the output per 32-row group, [ceil(M / 32)][N] (nullable)
 };
 
 // Descriptor of one 8-deep k-step of an operand tile.
@@ -256,6 +260,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                                         __uint_as_float(rr[4 * q + 2]), __uint_as_float(rr[4 * q + 3]));
                 __syncwarp();
                 const int col = col0 + 4 * cq;
+                float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);   // this lane's 8 rows of its 4 columns (act 3 / 4)
                 if (col < g.N) {
                     float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (g.bias) bv = *reinterpret_cast<const float4*>(g.bias + col);
@@ -269,6 +274,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             rv[i] = (row < g.M) ? *reinterpret_cast<const float4*>(g.residual + (long long)row * g.ldd + col)
                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
+                        if (g.act == 5 || g.act == 6) {   // h -> GELU'(h): 32 independent evaluations, none behind a store
+                            const bool th = g.act == 6;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                rv[i] = make_float4(gelu_grad_f(rv[i].x, th), gelu_grad_f(rv[i].y, th),
+                                                    gelu_grad_f(rv[i].z, th), gelu_grad_f(rv[i].w, th));
+                        }
                     }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
@@ -277,21 +289,40 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
                             float4 v = *reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(my_stage) +
                                                                         r * kEpiPitch + cq * 16);
                             v = add4(v, bv);
-                            if (g.residual) v = add4(v, rv[i]);
+                            if (g.act >= 5) {   // GELU backward: the product times GELU'(h), and its column sums
+                                v = make_float4(v.x * rv[i].x, v.y * rv[i].y, v.z * rv[i].z, v.w * rv[i].w);
+                                csum = add4(csum, v);
+                            } else if (g.residual) {
+                                v = add4(v, rv[i]);
+                            }
+                            float4 pv = v;      // what the hi/lo planes receive
+                            if (g.act >= 1 && g.act <= 4) {   // GELU forward: the planes hold GELU(output) ...
+                                const bool th = !(g.act & 1);
+                                float4 gp;
+                                gelu_both_f(v.x, th, pv.x, gp.x);
+                                gelu_both_f(v.y, th, pv.y, gp.y);
+                                gelu_both_f(v.z, th, pv.z, gp.z);
+                                gelu_both_f(v.w, th, pv.w, gp.w);
+                                if (g.act >= 3) v = gp;       // ... and D holds GELU'(output) instead of the output
+                            }
                             if (Dp) *reinterpret_cast<float4*>(Dp + (long long)row * ldd + col) = v;
                             if (g.d_hi) {
-                                if (g.act) {   // the raw output above stays pre-activation (the backward needs it)
-                                    const bool th = g.act == 2;
-                                    v = make_float4(gelu_f(v.x, th), gelu_f(v.y, th), gelu_f(v.z, th), gelu_f(v.w, th));
-                                }
                                 float4 hh, ll;
-                                split_tf32(v, hh, ll);
+                                split_tf32(pv, hh, ll);
                                 float* hrow = g.d_hi + (long long)row * g.ldd + col;
                                 *reinterpret_cast<float4*>(hrow) = hh;
                                 *reinterpret_cast<float4*>(hrow + g.d_plane) = ll;
                             }
                         }
                     }
+                }
+                if (g.act >= 5 && g.col_partial) {   // warp-uniform: the 32 rows of this warp, rows sub + 4 i in lane order
+                    csum.x += __shfl_xor_sync(0xffffffffu, csum.x, 8);  csum.y += __shfl_xor_sync(0xffffffffu, csum.y, 8);
+                    csum.z += __shfl_xor_sync(0xffffffffu, csum.z, 8);  csum.w += __shfl_xor_sync(0xffffffffu, csum.w, 8);
+                    csum.x += __shfl_xor_sync(0xffffffffu, csum.x, 16); csum.y += __shfl_xor_sync(0xffffffffu, csum.y, 16);
+                    csum.z += __shfl_xor_sync(0xffffffffu, csum.z, 16); csum.w += __shfl_xor_sync(0xffffffffu, csum.w, 16);
+                    if (sub == 0 && col < g.N && row0 < g.M)
+                        *reinterpret_cast<float4*>(g.col_partial + (long long)(row0 >> 5) * g.N + col) = csum;
                 }
                 __syncwarp();   // the staging tile is rewritten by the next chunk
             }
@@ -492,6 +523,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                         __uint_as_float(rr[4 * q + 2]), __uint_as_float(rr[4 * q + 3]));
                 __syncwarp();
                 const int col = col0 + 4 * cq;
+                float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);   // this lane's 8 rows of its 4 columns (act 3 / 4)
                 if (col < g.N) {
                     float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
                     if (g.bias) bv = *reinterpret_cast<const float4*>(g.bias + col);
@@ -503,6 +535,13 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             rv[i] = (row < g.M) ? *reinterpret_cast<const float4*>(g.residual + (long long)row * g.ldd + col)
                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
+                        if (g.act == 5 || g.act == 6) {   // h -> GELU'(h): 32 independent evaluations, none behind a store
+                            const bool th = g.act == 6;
+#pragma unroll
+                            for (int i = 0; i < 8; ++i)
+                                rv[i] = make_float4(gelu_grad_f(rv[i].x, th), gelu_grad_f(rv[i].y, th),
+                                                    gelu_grad_f(rv[i].z, th), gelu_grad_f(rv[i].w, th));
+                        }
                     }
 #pragma unroll
                     for (int i = 0; i < 8; ++i) {
@@ -511,21 +550,40 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             float4 v = *reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(my_stage) +
                                                                         rr_ * kEpiPitch + cq * 16);
                             v = add4(v, bv);
-                            if (g.residual) v = add4(v, rv[i]);
+                            if (g.act >= 5) {   // GELU backward: the product times GELU'(h), and its column sums
+                                v = make_float4(v.x * rv[i].x, v.y * rv[i].y, v.z * rv[i].z, v.w * rv[i].w);
+                                csum = add4(csum, v);
+                            } else if (g.residual) {
+                                v = add4(v, rv[i]);
+                            }
+                            float4 pv = v;      // what the hi/lo planes receive
+                            if (g.act >= 1 && g.act <= 4) {   // GELU forward: the planes hold GELU(output) ...
+                                const bool th = !(g.act & 1);
+                                float4 gp;
+                                gelu_both_f(v.x, th, pv.x, gp.x);
+                                gelu_both_f(v.y, th, pv.y, gp.y);
+                                gelu_both_f(v.z, th, pv.z, gp.z);
+                                gelu_both_f(v.w, th, pv.w, gp.w);
+                                if (g.act >= 3) v = gp;       // ... and D holds GELU'(output) instead of the output
+                            }
                             if (Dp) *reinterpret_cast<float4*>(Dp + (long long)row * ldd + col) = v;
                             if (g.d_hi) {
-                                if (g.act) {   // the raw output above stays pre-activation (the backward needs it)
-                                    const bool th = g.act == 2;
-                                    v = make_float4(gelu_f(v.x, th), gelu_f(v.y, th), gelu_f(v.z, th), gelu_f(v.w, th));
-                                }
                                 float4 hh, ll;
-                                split_tf32(v, hh, ll);
+                                split_tf32(pv, hh, ll);
                                 float* hrow = g.d_hi + (long long)row * g.ldd + col;
                                 *reinterpret_cast<float4*>(hrow) = hh;
                                 *reinterpret_cast<float4*>(hrow + g.d_plane) = ll;
                             }
                         }
                     }
+                }
+                if (g.act >= 5 && g.col_partial) {   // warp-uniform: the 32 rows of this warp, rows sub + 4 i in lane order
+                    csum.x += __shfl_xor_sync(0xffffffffu, csum.x, 8);  csum.y += __shfl_xor_sync(0xffffffffu, csum.y, 8);
+                    csum.z += __shfl_xor_sync(0xffffffffu, csum.z, 8);  csum.w += __shfl_xor_sync(0xffffffffu, csum.w, 8);
+                    csum.x += __shfl_xor_sync(0xffffffffu, csum.x, 16); csum.y += __shfl_xor_sync(0xffffffffu, csum.y, 16);
+                    csum.z += __shfl_xor_sync(0xffffffffu, csum.z, 16); csum.w += __shfl_xor_sync(0xffffffffu, csum.w, 16);
+                    if (sub == 0 && col < g.N && row0 < g.M)
+                        *reinterpret_cast<float4*>(g.col_partial + (long long)(row0 >> 5) * g.N + col) = csum;
                 }
                 __syncwarp();
             }
@@ -700,7 +758,7 @@ template <int BK>
 static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const SplitMat& A, const SplitMat& B,
                              float* D, int64_t ldd, const float* bias, const float* residual, float* partials,
                              size_t max_partial_floats, int* err_word, float* d_hi, int64_t d_plane,
-                             cudaStream_t s, int two_cta_mode, int act) {
+                             cudaStream_t s, int two_cta_mode, int act, float* col_partial) {
     const bool a_mn = (layout == kTN), b_mn = (layout != kNT);
     const int sms = g_num_sms > 0 ? g_num_sms : 148;
     const int kb_total = (int)((K + BK - 1) / BK);
@@ -725,7 +783,8 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     g.splits = plan.splits;
     g.kb_per_split = plan.kb_per_split; g.kb_total = kb_total;
     g.partials = partials; g.err = err_word;
-    g.d_hi = d_hi; g.d_plane = d_plane; g.act = d_hi ? act : 0;
+    g.d_hi = d_hi; g.d_plane = d_plane; g.act = (d_hi || act >= 5) ? act : 0;
+    g.col_partial = act >= 5 ? col_partial : nullptr;
     const long long units = (long long)g.tiles_m * g.tiles_n * g.splits;
     const int grid = (int)(units < sms ? units : sms);
     if (plan.two_cta) {
@@ -771,14 +830,16 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
 
 cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat A, SplitMat B, float* D, int64_t ldd,
                            const float* bias, const float* residual, float* partials, size_t max_partial_floats,
-                           int* err_word, cudaStream_t s, float* d_hi, int64_t d_plane, int two_cta_mode, int act) {
+                           int* err_word, cudaStream_t s, float* d_hi, int64_t d_plane, int two_cta_mode, int act,
+                           float* col_partial) {
     if (!gemm_tc_init(nullptr, 0)) return cudaErrorNotSupported;
     if (!D && !d_hi) return cudaErrorInvalidValue;
+    if (act >= 5 && (!residual || bias)) return cudaErrorInvalidValue;   // the gate operand travels as `residual`
     if (g_bk == 32)
         return launch_bk<32>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word,
-                             d_hi, d_plane, s, two_cta_mode, act);
+                             d_hi, d_plane, s, two_cta_mode, act, col_partial);
     return launch_bk<16>(layout, M, N, K, A, B, D, ldd, bias, residual, partials, max_partial_floats, err_word, d_hi,
-                         d_plane, s, two_cta_mode, act);
+                         d_plane, s, two_cta_mode, act, col_partial);
 }
 
 }  // namespace bt

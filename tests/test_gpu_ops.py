@@ -444,6 +444,50 @@ def test_gemm_epilogue_activation_planes(act, flags):
     assert not (gs[0].cpu().numpy().view(np.uint32) & 0x1FFF).any()
 
 
+_GELU_BWD_CASES = [(M, N, K, t, f) for (M, N, K) in [(520, 768, 256), (8, 32, 4), (1000, 352, 132)] for t in (0, 1)
+                   for f in (0, b.BT_FLAG_GEMM_SINGLE, b.BT_FLAG_GEMM_PAIR)] + [(4096, 3072, 768, 0, 0)]
+
+
+@pytest.mark.parametrize("M,N,K,tanh_form,flags", _GELU_BWD_CASES)
+def test_gemm_gelu_bwd_epilogue(M, N, K, tanh_form, flags):
+    """The input-gradient product of the MLP down-projection with the GELU backward in its epilogue:
+    dh = (dy W) o GELU'(h) as hi/lo planes, and the column sums of dh (ragged row and column tiles,
+    rows that do not fill a 32-row group, several tiles per CTA)."""
+    dy, w, h = si.normal_f32(95, (M, K), 1e-2), si.normal_f32(96, (K, N), 0.1), si.normal_f32(97, (M, N), 2.0)
+    dys, ws = empty(2, M, K), empty(2, K, N)
+    b.bt_op_split(dev(dy), M * K, dys)
+    b.bt_op_split(dev(w), K * N, ws)
+    dh, cs = empty(2, M, N), empty(N)
+    nb = b.bt_op_gemm_gelu_bwd_scratch_bytes(M, N)
+    sc = scratch(nb)
+    b.bt_op_gemm_gelu_bwd(M, N, K, dys, ws, dev(h), tanh_form, dh, cs, sc, nb, flags)
+    b.bt_op_gemm_check(sc)
+    dg = dy.astype(np.float64) @ w.astype(np.float64)
+    want = oracle.gelu_bwd(h.ravel(), dg.ravel(), tanh_form).reshape(M, N)
+    got = host(dh)
+    assert rel_l2(got[0].astype(np.float64) + got[1], want) < 1e-5
+    assert not (dh[0].cpu().numpy().view(np.uint32) & 0x1FFF).any()
+    assert np.abs(host(cs) - want.sum(0)).max() < 1e-5 * np.abs(want).sum(0).max() + 1e-12
+    # the column sums are those of the planes the kernel wrote, group by group
+    assert np.abs(host(cs) - (got[0].astype(np.float64) + got[1]).sum(0)).max() < 2e-6 * np.abs(want).sum(0).max() + 1e-12
+
+
+def test_gemm_gelu_bwd_rejects_bad_arguments():
+    x = empty(64)
+    nb = b.bt_op_gemm_gelu_bwd_scratch_bytes(8, 32)
+    sc = scratch(nb)
+    for args, status in [((8, 30, 4), 1), ((0, 32, 4), 1), ((8, 32, 6), 1)]:
+        with pytest.raises(b.BtError) as e:
+            b.bt_op_gemm_gelu_bwd(*args, x, x, x, 0, x, x, sc, nb)
+        assert e.value.status == status
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_gemm_gelu_bwd(8, 32, 4, x, x, x, 0, x, x, sc, 16)
+    assert e.value.status == 3
+    with pytest.raises(b.BtError) as e:
+        b.bt_op_gemm_gelu_bwd(8, 32, 4, x, x, x, 0, x, x, sc, nb, b.BT_FLAG_GEMM_SIMT)
+    assert e.value.status == 2
+
+
 def test_empty_inputs_are_no_ops_or_rejected():
     """Zero-length calls: the element-wise entry points accept n = 0 and launch nothing; calls whose
     result is undefined for no rows (reductions, GEMM) refuse them on the host."""
