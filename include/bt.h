@@ -438,10 +438,11 @@ BT_API bt_status bt_op_gemm_split(int32_t layout, int64_t M, int64_t N, int64_t 
                                   const float* B_split, float* D, const float* bias, const float* residual,
                                   void* scratch, size_t scratch_bytes, uint32_t flags, void* stream);
 /* The same, and D_act_split [2][M][N] (device) receives the TF32 hi/lo planes of act(D) from the
- * same epilogue: act 0 = D itself, 1 = GELU(D) in the exact erf form, 2 = the tanh form.  The
- * training step uses it for the MLP up-projection (the GELU feed-forward sublayer of the GPT-2
- * architecture figure: h = m Wfc^T + b is kept for the backward, g = GELU(h) is the next GEMM's
- * operand). */
+ * same epilogue: act 0 = D itself, 1 = GELU(D) in the erf form, 2 = the tanh form; 3 / 4 = as
+ * 1 / 2, and D receives GELU'(output) instead of the output (tensor-core kernels only).  The
+ * training step uses 3 / 4 for the MLP up-projection (the GELU feed-forward sublayer of the GPT-2
+ * architecture figure: g = GELU(h), h = m Wfc^T + b, is the next GEMM's operand, and GELU'(h) is
+ * all the backward pass needs of h), 1 / 2 where h itself is needed again. */
 BT_API bt_status bt_op_gemm_split_act(int32_t layout, int64_t M, int64_t N, int64_t K, const float* A_split,
                                       const float* B_split, float* D, float* D_act_split, int32_t act,
                                       const float* bias, const float* residual, void* scratch,
@@ -451,7 +452,8 @@ BT_API bt_status bt_op_gemm_check(const void* scratch, void* stream);
  * (Kernel Design, fused element-wise epilogues; Appendix B "GELU Backward"): with dy_split
  * [2][M][K] (hi/lo planes of the gradient at the projection's output), w_split [2][K][N] (the
  * projection's weight, [out, in] = [K, N]) and h [M][N] (the pre-activation kept by the forward),
- *   dh_split [2][M][N] = hi/lo planes of (dy . W) o GELU'(h)     (tanh_form 0: erf form, 1: tanh form)
+ *   dh_split [2][M][N] = hi/lo planes of (dy . W) o GELU'(h)     (form 0: erf form, 1: tanh form,
+ *                         2: `h` already holds GELU'(h), as bt_op_gemm_split_act with act 3 / 4 leaves it)
  *   colsum [N]          = the column sums of that product over the M rows, added per 32-row
  *                         group in row order (the bias gradient of the up-projection).
  * All pointers device, 16-byte aligned; N a multiple of 32, M and K multiples of 4.  `scratch`
@@ -460,7 +462,7 @@ BT_API bt_status bt_op_gemm_check(const void* scratch, void* stream);
  * (BT_FLAG_GEMM_SIMT is not supported here: BT_ERR_UNSUPPORTED). */
 BT_API size_t bt_op_gemm_gelu_bwd_scratch_bytes(int64_t M, int64_t N);
 BT_API bt_status bt_op_gemm_gelu_bwd(int64_t M, int64_t N, int64_t K, const float* dy_split, const float* w_split,
-                                     const float* h, int32_t tanh_form, float* dh_split, float* colsum,
+                                     const float* h, int32_t form, float* dh_split, float* colsum,
                                      void* scratch, size_t scratch_bytes, uint32_t flags, void* stream);
 
 /* Convenience form on raw FP32 operands: bt_op_split of A and B into `scratch`, then

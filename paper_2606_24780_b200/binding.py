@@ -515,9 +515,9 @@ def bt_op_gemm_gelu_bwd_scratch_bytes(M, N):
     return lib().bt_op_gemm_gelu_bwd_scratch_bytes(M, N)
 
 
-def bt_op_gemm_gelu_bwd(M, N, K, dy_split, w_split, h, tanh_form, dh_split, colsum, scratch, scratch_bytes, flags=0,
+def bt_op_gemm_gelu_bwd(M, N, K, dy_split, w_split, h, form, dh_split, colsum, scratch, scratch_bytes, flags=0,
                         stream=None):
-    _check(lib().bt_op_gemm_gelu_bwd(M, N, K, _ptr(dy_split), _ptr(w_split), _ptr(h), int(tanh_form), _ptr(dh_split),
+    _check(lib().bt_op_gemm_gelu_bwd(M, N, K, _ptr(dy_split), _ptr(w_split), _ptr(h), int(form), _ptr(dh_split),
                                      _ptr(colsum), _ptr(scratch), scratch_bytes, flags, _stream(stream)))
 
 

@@ -1246,7 +1246,7 @@ static bt_status gemm_split_impl(int32_t layout, int64_t M, int64_t N, int64_t K
                                  void* stream) {
     BT_PTR(A_split); BT_PTR(B_split); BT_PTR(D); BT_OPT_PTR(D_act_split); BT_OPT_PTR(bias); BT_OPT_PTR(residual);
     BT_PTR(scratch);
-    if (act < 0 || act > 2) return fail(BT_ERR_INVALID_ARG, "gemm: act %d", act);
+    if (act < 0 || act > 4) return fail(BT_ERR_INVALID_ARG, "gemm: act %d", act);
     if (layout < 0 || layout > 2) return fail(BT_ERR_INVALID_ARG, "gemm: layout %d", layout);
     if (M < 1 || N < 1 || K < 1 || M % 4 || N % 4 || K % 4) return fail(BT_ERR_INVALID_ARG, "gemm: M, N, K must be positive multiples of 4");
     if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return fail(BT_ERR_INVALID_ARG, "gemm: size too large");
@@ -1258,6 +1258,7 @@ static bt_status gemm_split_impl(int32_t layout, int64_t M, int64_t N, int64_t K
     SplitMat Am{A_split, na, sh.a_rows, sh.a_cols, sh.a_cols}, Bm{B_split, nb, sh.b_rows, sh.b_cols, sh.b_cols};
     if (flags & BT_FLAG_GEMM_SIMT) {
         BT_CUDA(launch_gemm_simt(layout, M, N, K, Am, Bm, D, N, bias, residual, s));
+        if (act > 2) return fail(BT_ERR_UNSUPPORTED, "gemm: act %d needs the tensor-core kernels", act);
         if (D_act_split) {
             if (act) BT_CUDA(launch_gelu_fwd(D, M * N, act == 2, nullptr, D_act_split, D_act_split + M * N, s));
             else BT_CUDA(launch_split(D, D_act_split, D_act_split + M * N, M * N, s));
@@ -1299,11 +1300,12 @@ extern "C" size_t bt_op_gemm_gelu_bwd_scratch_bytes(int64_t M, int64_t N) {
 }
 
 extern "C" bt_status bt_op_gemm_gelu_bwd(int64_t M, int64_t N, int64_t K, const float* dy_split, const float* w_split,
-                                         const float* h, int32_t tanh_form, float* dh_split, float* colsum,
+                                         const float* h, int32_t form, float* dh_split, float* colsum,
                                          void* scratch, size_t scratch_bytes, uint32_t flags, void* stream) {
     BT_PTR(dy_split); BT_PTR(w_split); BT_PTR(h); BT_PTR(dh_split); BT_PTR(colsum); BT_PTR(scratch);
     if (M < 1 || N < 1 || K < 1 || M % 4 || N % 32 || K % 4) return fail(BT_ERR_INVALID_ARG, "gemm_gelu_bwd: bad sizes");
     if (M > (1 << 30) || N > (1 << 30) || K > (1 << 30)) return fail(BT_ERR_INVALID_ARG, "gemm_gelu_bwd: size too large");
+    if (form < 0 || form > 2) return fail(BT_ERR_INVALID_ARG, "gemm_gelu_bwd: form %d", form);
     if (flags & BT_FLAG_GEMM_SIMT) return fail(BT_ERR_UNSUPPORTED, "gemm_gelu_bwd: tensor-core kernels only");
     if (scratch_bytes < bt_op_gemm_gelu_bwd_scratch_bytes(M, N)) return fail(BT_ERR_OOM, "gemm_gelu_bwd: scratch too small");
     if (reinterpret_cast<uintptr_t>(scratch) & 255u) return fail(BT_ERR_INVALID_ARG, "gemm_gelu_bwd: scratch not 256-byte aligned");
@@ -1317,7 +1319,7 @@ extern "C" bt_status bt_op_gemm_gelu_bwd(int64_t M, int64_t N, int64_t K, const 
     SplitMat Am{dy_split, M * K, M, K, K}, Bm{w_split, K * N, K, N, N};
     const int two_cta_mode = (flags & BT_FLAG_GEMM_PAIR) ? 1 : (flags & BT_FLAG_GEMM_SINGLE) ? 0 : -1;
     BT_CUDA(launch_gemm_tc(BT_GEMM_NN, M, N, K, Am, Bm, nullptr, N, nullptr, h, partials, gemm_tc_partial_floats_bound(), err,
-                           s, dh_split, M * N, two_cta_mode, tanh_form ? 6 : 5, groups));
+                           s, dh_split, M * N, two_cta_mode, 5 + form, groups));
     BT_CUDA(launch_colsum_stage2(groups, (int)((M + 31) / 32), (int)N, colsum, s));
     return BT_OK;
 }

@@ -53,6 +53,26 @@ def build_cases(B, T, C, H, Vp, n_params):
         cases[name] = dict(run=run, flops=2.0 * M * Nn * K, bytes=8.0 * (M * K + Nn * K) + 4.0 * M * Nn,
                            bound="tensor", keep=(A, Bm, D, bi, res), check=lambda: b.bt_op_gemm_check(gscratch))
 
+    def fused_gelu_cases():
+        # the MLP up-projection with GELU in its epilogue (planes of GELU(h), GELU'(h) kept for the
+        # backward) and the down-projection's input gradient with the GELU backward in its epilogue
+        x_s, wt_s = _split(_rand(N, C)), _split(_rand(C, F, std=0.02))
+        hD, g_s, bi = torch.empty(N, F, device="cuda"), torch.empty(2, N, F, device="cuda"), _rand(F)
+        cases["gemm_fwd_fc_gelu"] = dict(
+            run=lambda: b.bt_op_gemm_split_act(1, N, F, C, x_s, wt_s, hD, g_s, 3, bi, None, gscratch, gsb),
+            flops=2.0 * N * F * C, bytes=8.0 * (N * C + F * C) + 12.0 * N * F, bound="tensor",
+            keep=(x_s, wt_s, hD, g_s, bi), check=lambda: b.bt_op_gemm_check(gscratch))
+        dy_s, w_s = _split(_rand(N, C)), _split(_rand(C, F, std=0.02))
+        gp, dh_s, cs = _rand(N, F), torch.empty(2, N, F, device="cuda"), torch.empty(F, device="cuda")
+        nb = b.bt_op_gemm_gelu_bwd_scratch_bytes(N, F)
+        sc = torch.empty(nb + 512, dtype=torch.uint8, device="cuda")
+        sc = sc[(-sc.data_ptr()) % 256:]
+        cases["gemm_nn_dmlpproj_gelu_bwd"] = dict(
+            run=lambda: b.bt_op_gemm_gelu_bwd(N, F, C, dy_s, w_s, gp, 2, dh_s, cs, sc, nb),
+            flops=2.0 * N * F * C, bytes=8.0 * (N * C + F * C) + 12.0 * N * F, bound="tensor",
+            keep=(dy_s, w_s, gp, dh_s, cs, sc), check=lambda: b.bt_op_gemm_check(sc))
+
+    fused_gelu_cases()
     # forward GEMMs of the block as the training step runs them (weight read from its transposed
     # copy: layout NN, bias / residual in the epilogue), the same products in the NT layout, the two
     # backward layouts of each, and the LM head

@@ -420,8 +420,9 @@ def test_attention_long_context_16k():
     assert max(errs) < 1e-4, errs
 
 
-@pytest.mark.parametrize("flags", [b.BT_FLAG_GEMM_PAIR, b.BT_FLAG_GEMM_SINGLE, b.BT_FLAG_GEMM_SIMT])
-@pytest.mark.parametrize("act", [0, 1, 2])
+@pytest.mark.parametrize("act,flags", [(a, f) for a in (0, 1, 2, 3, 4)
+                                       for f in (b.BT_FLAG_GEMM_PAIR, b.BT_FLAG_GEMM_SINGLE, b.BT_FLAG_GEMM_SIMT)
+                                       if not (a > 2 and f == b.BT_FLAG_GEMM_SIMT)])
 def test_gemm_epilogue_activation_planes(act, flags):
     """The MLP up-projection as the step runs it: weight given transposed (layout NN), bias in the
     epilogue, the raw output kept and GELU(output) emitted as TF32 hi/lo planes by the same kernel."""
@@ -434,14 +435,19 @@ def test_gemm_epilogue_activation_planes(act, flags):
     nb = b.bt_op_gemm_split_scratch_bytes()
     b.bt_op_gemm_split_act(1, N, cout, cin, xs, wts, h, gs, act, dev(bias), None, scratch(nb), nb, flags)
     rh = oracle.linear_fwd(x, w, bias)
-    assert rel_l2(host(h), rh) < 1e-4
-    want = rh if act == 0 else oracle.gelu_fwd(rh.ravel(), act == 2).reshape(N, cout)
+    tanh_form = act in (2, 4)
+    want = rh if act == 0 else oracle.gelu_fwd(rh.ravel(), tanh_form).reshape(N, cout)
     got = host(gs)
     assert rel_l2(got[0] + got[1], want) < 1e-4
-    # the planes are the split of the kernel's own FP32 value of act(h)
-    ref32 = host(h) if act == 0 else oracle.gelu_fwd(host(h).ravel(), act == 2).reshape(N, cout)
-    assert np.abs((got[0].astype(np.float64) + got[1]) - ref32).max() < 1e-5 * np.abs(ref32).max()
     assert not (gs[0].cpu().numpy().view(np.uint32) & 0x1FFF).any()
+    if act >= 3:   # D holds GELU'(h): the derivative the oracle's backward applies to a gradient of ones
+        want_d = oracle.gelu_bwd(rh.ravel(), np.ones(rh.size), tanh_form).reshape(N, cout)
+        assert rel_l2(host(h), want_d) < 1e-4
+        return
+    assert rel_l2(host(h), rh) < 1e-4
+    # the planes are the split of the kernel's own FP32 value of act(h)
+    ref32 = host(h) if act == 0 else oracle.gelu_fwd(host(h).ravel(), tanh_form).reshape(N, cout)
+    assert np.abs((got[0].astype(np.float64) + got[1]) - ref32).max() < 1e-5 * np.abs(ref32).max()
 
 
 _GELU_BWD_CASES = [(M, N, K, t, f) for (M, N, K) in [(520, 768, 256), (8, 32, 4), (1000, 352, 132)] for t in (0, 1)
@@ -470,6 +476,14 @@ def test_gemm_gelu_bwd_epilogue(M, N, K, tanh_form, flags):
     assert np.abs(host(cs) - want.sum(0)).max() < 1e-5 * np.abs(want).sum(0).max() + 1e-12
     # the column sums are those of the planes the kernel wrote, group by group
     assert np.abs(host(cs) - (got[0].astype(np.float64) + got[1]).sum(0)).max() < 2e-6 * np.abs(want).sum(0).max() + 1e-12
+    # the same with GELU'(h) handed over instead of h (what the forward epilogue leaves): bit-identical
+    # when the derivative is the library's own FP32 value
+    gp = empty(M, N)
+    b.bt_op_gelu_bwd(dev(h), dev(np.ones((M, N), np.float32)), M * N, tanh_form, gp, None)
+    dh2, cs2 = empty(2, M, N), empty(N)
+    b.bt_op_gemm_gelu_bwd(M, N, K, dys, ws, gp, 2, dh2, cs2, sc, nb, flags)
+    b.bt_op_gemm_check(sc)
+    assert torch.equal(dh2, dh) and torch.equal(cs2, cs)
 
 
 def test_gemm_gelu_bwd_rejects_bad_arguments():
