@@ -35,7 +35,8 @@ namespace {
 
 constexpr int HD = 64, BQ = 128, BKV = 64;
 // Warps 0-7: the two softmax warpgroups (a warp's TMEM lane quadrant is its index mod 4); warp 8: TMA
-// producer; warps 9, 10: the two MMA issuers.  Eleven warps leave 184 registers per thread.
+// producer; warps 9, 10: the two MMA issuers.  (Registers are handed out per four warps: eleven warps
+// get the 168 registers per thread that twelve would.)
 constexpr int kThreads = 352;
 constexpr int kWarpProducer = 8, kWarpMmaS = 9, kWarpMmaO = 10;
 constexpr uint32_t kQBytes = 2u * 2u * BQ * 128u;      // 2 k-blocks x (hi, lo) x 128 rows x 128 B
