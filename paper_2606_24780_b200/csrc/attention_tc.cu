@@ -4,24 +4,25 @@
 // One CTA owns 128 query rows of one (sequence, head) -- one row per TMEM lane -- and walks the
 // 64-key tiles up to the diagonal:
 //
-//   warp 0 (one lane)  TMA producer: Q once, then double-buffered K tiles (K-major, 128-byte
-//                      swizzle) and V tiles (MN-major, 128-byte swizzle with 32-byte atoms), each as
-//                      hi/lo planes straight from the split qkv array the QKV GEMM wrote.
-//   warp 1 (one lane)  MMA issuer.  S = Q K^T: 24 tcgen05.mma.kind::tf32 (8 k-steps x 3 split
-//                      terms) with both operands in shared memory, accumulator S[buf] in TMEM.
-//                      O_tile = P V: 24 MMAs with A = P (hi/lo) read from TENSOR MEMORY and B = V
-//                      from shared memory, accumulator O[buf] in TMEM.  S of tile t+1 is issued
-//                      before P V of tile t, so the tensor pipe works while the softmax runs.
-//   warps 2-5, 6-9     two softmax / correction warpgroups taking alternate key tiles (buffer b
+//   warps 0-3, 4-7     two softmax / correction warpgroups taking alternate key tiles (buffer b
 //                      belongs to warpgroup b), merged at the end; in each, thread i owns query row i.  It reads its 64 scores
 //                      with tcgen05.ld (the row maximum and sum need no shuffles), forms
 //                      p = exp2((s - m) * scale*log2e), splits p into hi/lo and writes both back to
 //                      TMEM with tcgen05.st as the A operand of P V.  The running output is kept in
 //                      registers: O_reg = O_reg * corr + O_tile, so no accumulator in TMEM is ever
 //                      rescaled.
+//   warp 8 (one lane)  TMA producer: Q once, then the K tiles (K-major, 128-byte swizzle) and V
+//                      tiles (MN-major, 128-byte swizzle with 32-byte atoms) through one ring of five
+//                      slots, each as hi/lo planes straight from the split qkv array the QKV GEMM wrote.
+//   warp 9 (one lane)  MMA issuer.  S = Q K^T: 24 tcgen05.mma.kind::tf32 (8 k-steps x 3 split
+//                      terms) with both operands in shared memory, accumulator S[buf] in TMEM.
+//                      S of tile t+1 is issued before P V of tile t, so the tensor pipe works
+//                      while the softmax runs.
+//   warp 10 (one lane) second MMA issuer.  O_tile = P V: 24 MMAs with A = P (hi/lo) read from
+//                      TENSOR MEMORY and B = V from shared memory, accumulator O[buf] in TMEM.
 //
 // TMEM map (512 columns): per buffer b in {0,1}: S at 256b, P_hi at 256b+64, P_lo at 256b+128,
-// O_tile at 256b+192.  Shared memory: Q 64 KB, K 2 x 32 KB, V 2 x 32 KB.
+// O_tile at 256b+192.  Shared memory: Q 64 KB, five 32 KB tile slots.
 // Every mbarrier wait is bounded; a wait that runs out raises the device error word and the CTA
 // drains, frees its TMEM and exits.  Every TMA load targets this CTA's own shared memory only.
 #include "common.cuh"
