@@ -40,6 +40,13 @@ namespace {
 
 constexpr int HD = 64, BR = 128, BT_ = 32;  // head dim, rows owned by the CTA, streamed tile rows
 constexpr int kThreads = 320;   // TMA warp, MMA warp, two element-wise warpgroups (alternate tiles)
+// One thread issues a tcgen05.mma about every 55-59 clocks, whatever its shape; an N = 64 product
+// whose A operand comes from tensor memory occupies the pipe for 32.  The kernels below therefore
+// spread their products over several issuing threads (one lane each of warps 1, 10 and, in the dq
+// kernel, 11), every thread owning whole products and a chain of regions of its own, ordered
+// against the others only through mbarriers.
+constexpr int kThreadsDkv = 352, kThreadsDq = 384;
+constexpr int kWarpMma2 = 10, kWarpMma3 = 11;
 constexpr float kLog2e = 1.4426950408889634f;
 constexpr uint32_t kResBytes = 2u * 2u * BR * 128u;   // resident 128-row operand: 2 k-blocks x (hi,lo)
 constexpr uint32_t kTileBytes = 2u * 2u * BT_ * 128u; // one streamed 32-row tile in one layout (16 KB)
@@ -172,9 +179,9 @@ __device__ __forceinline__ void trace_mark(unsigned long long* tr, int role, int
 
 // Shared prologue: barriers + TMEM allocation.  Returns the TMEM base address.
 __device__ __forceinline__ uint32_t setup(uint32_t bars, int n_bars_count1, uint32_t p_bar0, int n_p_bars,
-                                          uint32_t tmem_slot, uint8_t* smem_raw, int warp) {
+                                          uint32_t tmem_slot, uint8_t* smem_raw, int warp, uint32_t two_mask = 0u) {
     if (threadIdx.x == 0) {
-        for (int i = 0; i < n_bars_count1; ++i) mbar_init(bars + 8u * i, 1);
+        for (int i = 0; i < n_bars_count1; ++i) mbar_init(bars + 8u * i, ((two_mask >> i) & 1u) ? 2 : 1);
         for (int i = 0; i < n_p_bars; ++i) mbar_init(p_bar0 + 8u * i, 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -206,11 +213,11 @@ __device__ __forceinline__ uint32_t setup(uint32_t bars, int n_bars_count1, uint
 //                  soon as the one product that reads it has completed.
 constexpr int BT64 = 64;
 constexpr uint32_t kTile64 = 2u * 2u * BT64 * 128u;   // one 64-row tile in one layout (32 KB)
-constexpr uint32_t kDkvSmem = 1024u + kResBytes + 4u * kTile64 + 256u + 4u * kRowTileBytes;   // + K' staging tiles
+constexpr uint32_t kDkvSmem = 1024u + kResBytes + 4u * kTile64 + 256u + 4u * kRowTileBytes + 1024u;   // + K' staging tiles, + row statistics
 __device__ __forceinline__ constexpr uint32_t mn64_off(int ks, bool lo) { return (lo ? BT64 * 128u : 0u) + (uint32_t)ks * 1024u; }
 __device__ __forceinline__ DescBase mn64_base(uint32_t tile) { return make_desc_base(tile, 2u * BT64 * 128u, 512u, 1u); }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsDkv, 1)
 attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_constant__ CUtensorMap tmQm,
                        const __grid_constant__ CUtensorMap tmDOk, const __grid_constant__ CUtensorMap tmDOm,
                        const __grid_constant__ CUtensorMap tmVres, const BwdArgs g) {
@@ -220,7 +227,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     const uint32_t qk_s = base + kResBytes, dok_s = qk_s + kTile64, dom_s = dok_s + kTile64, qm_s = dom_s + kTile64;
     const uint32_t bars = qm_s + kTile64;
     enum { V_FULL = 0, QK_FULL, QK_EMPTY, DOK_FULL, DOK_EMPTY, DOM_FULL, DOM_EMPTY, QM_FULL, QM_EMPTY, S_FULL,
-           DP_FULL, ACC_FULL, P_READY, DS_READY, K_READY, N_BARS };
+           DP_FULL, ACC_FULL, P_READY, DS_READY, K_READY, STAT_READY, N_BARS };
     auto bar = [&](int i) { return bars + 8u * (uint32_t)i; };
     const uint32_t tmem_slot = bars + 8u * N_BARS;
 
@@ -239,10 +246,11 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     }
 
     if (threadIdx.x == 0) {
-        for (int i = 0; i < P_READY; ++i) mbar_init(bar(i), 1);
+        for (int i = 0; i < P_READY; ++i) mbar_init(bar(i), i == ACC_FULL ? 2 : 1);   // both issuing threads commit at the end
         mbar_init(bar(P_READY), 8);      // both element-wise warpgroups (8 warps) write every tile
         mbar_init(bar(DS_READY), 8);
         mbar_init(bar(K_READY), 4);
+        mbar_init(bar(STAT_READY), 4);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -288,12 +296,15 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             if (!ok)
                 for (int i = 0; i < 2000; ++i) __nanosleep(1000);
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == kWarpMma2) {
         if (lane == 0) {
             constexpr uint32_t idesc_a = make_idesc_tf32(BR, BT64, false, false);  // 128 x 64, B K-major
             constexpr uint32_t idesc_a2 = make_idesc_tf32(BR, 2 * BT64, false, false);  // 128 x 128: B = [hi rows | lo rows]
             constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
-            bool ok = mbar_wait(bar(V_FULL), 0, g.err, 23) && mbar_wait(bar(K_READY), 0, g.err, 24);
+            // warp 1: the S^T -> P^T -> dV chain (regions tS, tPlo, tdV); warp 10: dP^T -> dS^T -> dK
+            const bool score_chain = warp == 1;
+            const int trole = score_chain ? 0 : 3;   // region of the debug trace
+            bool ok = score_chain ? mbar_wait(bar(K_READY), 0, g.err, 24) : mbar_wait(bar(V_FULL), 0, g.err, 23);
             int tn = 0;
             const DescBase vd = kmaj_base(v_s), qd = kmaj_base(qk_s), od = kmaj_base(dok_s);
             const DescBase omd = mn64_base(dom_s), qmd = mn64_base(qm_s);
@@ -310,7 +321,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 }
                 umma_commit(bar(QK_EMPTY));
                 umma_commit(bar(S_FULL));
-                trace_mark(g.trace, 0, tn, 100 + t);
+                trace_mark(g.trace, trole, tn, 100 + t);
                 return true;
             };
             auto issue_dp = [&](int t) -> bool {     // dP^T(t) = V dO^T
@@ -325,7 +336,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 }
                 umma_commit(bar(DOK_EMPTY));
                 umma_commit(bar(DP_FULL));
-                trace_mark(g.trace, 0, tn, 200 + t);
+                trace_mark(g.trace, trole, tn, 200 + t);
                 return true;
             };
             auto issue_dv = [&](int t) -> bool {     // dV += P^T(t) dO
@@ -341,7 +352,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                     umma_tf32_ts(tdV, tS + ks * 8, o_hi, idesc_b, 1u);
                 }
                 umma_commit(bar(DOM_EMPTY));
-                trace_mark(g.trace, 0, tn, 300 + t);
+                trace_mark(g.trace, trole, tn, 300 + t);
                 return true;
             };
             auto issue_dk = [&](int t) -> bool {     // dK += dS^T(t) Q
@@ -357,19 +368,28 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                     umma_tf32_ts(tdK, tdP + ks * 8, q_hi, idesc_b, 1u);
                 }
                 umma_commit(bar(QM_EMPTY));
-                trace_mark(g.trace, 0, tn, 400 + t);
+                trace_mark(g.trace, trole, tn, 400 + t);
                 return true;
             };
-            if (ok && n_t > 0) ok = issue_s(0) && issue_dp(0);
-            for (int t = 0; t < n_t && ok; ++t) {
-                ok = issue_dv(t);                              // frees the S^T / P^T regions ...
-                if (ok && t + 1 < n_t) ok = issue_s(t + 1);    // ... which the next scores overwrite
-                if (ok) ok = issue_dk(t);                      // frees the dP^T / dS^T regions ...
-                if (ok && t + 1 < n_t) ok = issue_dp(t + 1);   // ... which the next dP^T overwrites
+            // Within a chain the product that overwrites a region follows the product that last read it
+            // in this thread's own program order (the pipe executes a thread's MMAs in order); the two
+            // chains share no region.
+            if (score_chain) {
+                if (ok && n_t > 0) ok = issue_s(0);
+                for (int t = 0; t < n_t && ok; ++t) {
+                    ok = issue_dv(t);                              // frees the S^T / P^T regions ...
+                    if (ok && t + 1 < n_t) ok = issue_s(t + 1);    // ... which the next scores overwrite
+                }
+            } else {
+                if (ok && n_t > 0) ok = issue_dp(0);
+                for (int t = 0; t < n_t && ok; ++t) {
+                    ok = issue_dk(t);                              // frees the dP^T / dS^T regions ...
+                    if (ok && t + 1 < n_t) ok = issue_dp(t + 1);   // ... which the next dP^T overwrites
+                }
             }
             if (ok) umma_commit(bar(ACC_FULL));
         }
-    } else {
+    } else if (warp < kWarpMma2) {
         const int wg = (warp - 2) >> 2;                   // 0 or 1: columns (query rows) 32 wg .. 32 wg + 31 of every tile
         const int lane_group = warp & 3;
         const int etid = lane_group * 32 + lane;          // 0..127: key row owned inside the CTA
@@ -391,18 +411,44 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
         bool ok = true;
         int tn = 0;
         const uint32_t c0 = 32u * (uint32_t)wg;
+        // Softmax statistics of a tile's 64 query rows (log-sum-exp in base-2 units, D = rowsum(dO o O)):
+        // every thread needs the 32 values of its warpgroup's columns.  128 threads fetch one value each
+        // for the NEXT tile while the current one is worked on and leave it in shared memory
+        // ([2][L 0-63 | D 64-127], double-buffered by tile parity), from where it is read with
+        // 128-bit broadcast loads.  (Each thread loading its 64 values itself -- 512 load instructions
+        // per tile and SM -- took 3,000 of a tile's 7,000 clocks.)  A buffer is rewritten at the end of
+        // tile t for tile t + 1: every warp read tile t - 1's values before the products of tile t could start.
+        float* stat = reinterpret_cast<float*>(smem_raw + (bars + 256u + 4u * kRowTileBytes - smem_u32(smem_raw)));
+        const int sidx = (warp - 2) * 32 + lane;          // 0..255; the first 128 threads stage values
+        auto fetch_stat = [&](int t) -> float {
+            const int r = min(q_row0(t) + (sidx & 63), g.T - 1);   // clamped: rows past the end are masked below
+            return sidx < 64 ? __ldg(g.lse + lb + r) * kLog2e : __ldg(g.dvec + lb + r);
+        };
+        auto publish_stat = [&](int t, float v) {          // warps 2-5: value of tile t into its buffer
+            if (sidx < 128) {
+                stat[(t & 1) * 128 + sidx] = v;
+                __threadfence_block();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(bar(STAT_READY));
+            }
+        };
+        if (n_t > 0) publish_stat(0, sidx < 128 ? fetch_stat(0) : 0.f);
         for (int t = 0; t < n_t && ok; ++t) {
             const int q0 = q_row0(t) + 32 * wg;
-            // softmax statistics of this warpgroup's 32 query rows (same addresses in every thread:
-            // broadcast loads, issued before the wait so their latency is hidden); rows past the
-            // sequence end are clamped here and masked below
             const int nvalid = min(32, g.T - q0);
+            float next_stat = 0.f;
+            if (sidx < 128 && t + 1 < n_t) next_stat = fetch_stat(t + 1);   // in flight during this tile
+            if (!mbar_wait_warp(bar(STAT_READY), (uint32_t)(t & 1), g.err, 42)) { ok = false; break; }
             float Lc[32], Dc[32];
+            {
+                const float4* Ls = reinterpret_cast<const float4*>(stat + (t & 1) * 128 + 32 * wg);
+                const float4* Ds = reinterpret_cast<const float4*>(stat + (t & 1) * 128 + 64 + 32 * wg);
 #pragma unroll
-            for (int i = 0; i < 32; ++i) {
-                const int r = min(q0 + i, g.T - 1);     // clamped: rows past the end are masked below
-                Lc[i] = __ldg(g.lse + lb + r) * kLog2e;
-                Dc[i] = __ldg(g.dvec + lb + r);
+                for (int i = 0; i < 8; ++i) {
+                    const float4 l4 = Ls[i], d4 = Ds[i];
+                    Lc[4 * i] = l4.x; Lc[4 * i + 1] = l4.y; Lc[4 * i + 2] = l4.z; Lc[4 * i + 3] = l4.w;
+                    Dc[4 * i] = d4.x; Dc[4 * i + 1] = d4.y; Dc[4 * i + 2] = d4.z; Dc[4 * i + 3] = d4.w;
+                }
             }
             if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 700 + t);
             if (!mbar_wait_warp(bar(S_FULL), (uint32_t)(t & 1), g.err, 31)) { ok = false; break; }
@@ -443,6 +489,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(DS_READY));
             if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 900 + t);
+            if (t + 1 < n_t) publish_stat(t + 1, next_stat);
         }
         if (ok) ok = mbar_wait_warp(bar(ACC_FULL), 0, g.err, 33);
         if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
@@ -483,7 +530,7 @@ __device__ __forceinline__ constexpr uint32_t mnmaj64_off(int ks, bool lo) {
 }
 __device__ __forceinline__ DescBase mnmaj64_base(uint32_t tile) { return make_desc_base(tile, 2u * BKT * 128u, 512u, 1u); }
 
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreadsDq, 1)
 attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_constant__ CUtensorMap tmKm,
                       const __grid_constant__ CUtensorMap tmVk, const __grid_constant__ CUtensorMap tmDOres,
                       const BwdArgs g) {
@@ -495,13 +542,15 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
     const uint32_t km_s = base + kResBytes + 4u * kTileQ;       // single stage
     const uint32_t qstage = km_s;                               // staging of the query rows before the first fill
     const uint32_t bars = base + kResBytes + 5u * kTileQ;
-    // count-1: 0 do_full, 1-2 kfull, 3-4 kempty, 5 mfull, 7 mempty, 9-10 sdp_full, 11 acc_full
+    // count-1: 0 do_full, 1-2 kfull, 5 mfull, 6 / 8 dq_done, 7 mempty, 11 acc_full; count-2 (the S and the dP
+    // issuing threads both commit): 3-4 kempty, 9-10 sdp_full
     const uint32_t do_full = bars;
     auto kfull = [&](int s) { return bars + 8u * (1 + s); };
     auto kempty = [&](int s) { return bars + 8u * (3 + s); };
     const uint32_t mfull = bars + 8u * 5;
     const uint32_t mempty = bars + 8u * 7;
     auto sdp_full = [&](int b) { return bars + 8u * (9 + b); };
+    auto dq_done = [&](int b) { return bars + 8u * (6 + 2 * b); };   // dQ(t) has read buffer b: it may be overwritten
     const uint32_t acc_full = bars + 8u * 11;
     // count-4: 12-13 ds_full, 14 q_ready
     auto ds_full = [&](int b) { return bars + 8u * (12 + b); };
@@ -520,7 +569,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
         trace_cta(g.trace, 1, 3, n_t);
     }
 
-    const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp);
+    const uint32_t tmem = setup(bars, 12, bars + 8u * 12, 3, tmem_slot, smem_raw, warp, 0x618u);   // bars 3, 4, 9, 10: two arrivals
     pdl_wait();      // set-up done; global memory is touched from here on
     pdl_trigger();
     // dQ is 128 columns: the halves of the split product dS . [K_hi | K_lo] by 32-column groups (see issue_b)
@@ -559,58 +608,73 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             if (!ok)
                 for (int i = 0; i < 2000; ++i) __nanosleep(1000);
         }
-    } else if (warp == 1) {
+    } else if (warp == 1 || warp == kWarpMma2) {
+        // ---- the two score products, one issuing thread each: warp 1 S = Q' K^T (A in tensor memory),
+        // warp 10 dP = dO V^T (A resident in shared memory).  Both write into buffer t & 1, which the
+        // dQ product of tile t - 2 must have read.
         if (lane == 0) {
             constexpr uint32_t idesc_a = make_idesc_tf32(BR, BKT, false, false);   // 128 x 64, B K-major
-            constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
-            constexpr uint32_t idesc_b2 = make_idesc_tf32(BR, 2 * HD, false, true);   // 128 x 128, B = four column groups
-            bool ok = mbar_wait(do_full, 0, g.err, 33) && mbar_wait(q_ready, 0, g.err, 34);
+            const bool s_product = warp == 1;
+            bool ok = s_product ? mbar_wait(q_ready, 0, g.err, 34) : mbar_wait(do_full, 0, g.err, 33);
             int tn = 0;
             const DescBase dod = kmaj_base(do_s);
-            auto issue_a = [&](int t) -> bool {
+            for (int t = 0; t < n_t && ok; ++t) {
                 const int st = t & 1, bb = t & 1;
                 trace_mark(g.trace, 0, tn, 100 + t);
-                if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 35)) return false;
+                if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 35)) { ok = false; break; }
+                if (t >= 2 && !mbar_wait(dq_done(bb), ((t - 2) >> 1) & 1u, g.err, 41)) { ok = false; break; }
                 trace_mark(g.trace, 0, tn, 200 + t);
                 tc_fence_after();
-                const uint32_t dS = tbuf(bb), dP = tbuf(bb) + 64u;
-                const DescBase kd = kmaj_base(kk_s(st)), vkd = kmaj_base(vk_s(st));
+                if (s_product) {
+                    const uint32_t dS = tbuf(bb);
+                    const DescBase kd = kmaj_base(kk_s(st));
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t k_hi = kd.at(kmaj_off(BKT, ks, false)), k_lo = kd.at(kmaj_off(BKT, ks, true));
-                    umma_tf32_ts(dS, tQ_lo + ks * 8, k_hi, idesc_a, ks > 0 ? 1u : 0u);
-                    umma_tf32_ts(dS, tQ_hi + ks * 8, k_lo, idesc_a, 1u);
-                    umma_tf32_ts(dS, tQ_hi + ks * 8, k_hi, idesc_a, 1u);
-                }
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t k_hi = kd.at(kmaj_off(BKT, ks, false)), k_lo = kd.at(kmaj_off(BKT, ks, true));
+                        umma_tf32_ts(dS, tQ_lo + ks * 8, k_hi, idesc_a, ks > 0 ? 1u : 0u);
+                        umma_tf32_ts(dS, tQ_hi + ks * 8, k_lo, idesc_a, 1u);
+                        umma_tf32_ts(dS, tQ_hi + ks * 8, k_hi, idesc_a, 1u);
+                    }
+                } else {
+                    const uint32_t dP = tbuf(bb) + 64u;
+                    const DescBase vkd = kmaj_base(vk_s(st));
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint64_t o_hi = dod.at(kmaj_off(BR, ks, false)), o_lo = dod.at(kmaj_off(BR, ks, true));
-                    const uint64_t v_hi = vkd.at(kmaj_off(BKT, ks, false)), v_lo = vkd.at(kmaj_off(BKT, ks, true));
-                    umma_tf32(dP, o_lo, v_hi, idesc_a, ks > 0 ? 1u : 0u);
-                    umma_tf32(dP, o_hi, v_lo, idesc_a, 1u);
-                    umma_tf32(dP, o_hi, v_hi, idesc_a, 1u);
+                    for (int ks = 0; ks < 8; ++ks) {
+                        const uint64_t o_hi = dod.at(kmaj_off(BR, ks, false)), o_lo = dod.at(kmaj_off(BR, ks, true));
+                        const uint64_t v_hi = vkd.at(kmaj_off(BKT, ks, false)), v_lo = vkd.at(kmaj_off(BKT, ks, true));
+                        umma_tf32(dP, o_lo, v_hi, idesc_a, ks > 0 ? 1u : 0u);
+                        umma_tf32(dP, o_hi, v_lo, idesc_a, 1u);
+                        umma_tf32(dP, o_hi, v_hi, idesc_a, 1u);
+                    }
                 }
                 umma_commit(kempty(st));
                 umma_commit(sdp_full(bb));
                 trace_mark(g.trace, 0, tn, 300 + t);
-                return true;
-            };
-            auto issue_b = [&](int t) -> bool {
+            }
+        }
+    } else if (warp == kWarpMma3) {
+        // ---- the accumulating product dQ += dS K, a third issuing thread
+        if (lane == 0) {
+            constexpr uint32_t idesc_b = make_idesc_tf32(BR, HD, false, true);     // 128 x 64, B MN-major
+            constexpr uint32_t idesc_b2 = make_idesc_tf32(BR, 2 * HD, false, true);   // 128 x 128, B = four column groups
+            bool ok = true;
+            int tn = 0;
+            // Two instructions per k-step.  The MN-major K tile lies in shared memory as the column
+            // groups [K_hi g0 | K_lo g0 | K_hi g1 | K_lo g1] (g = 32 head columns), 8 KB apart: seen
+            // with that stride it is one operand of N = 128, and dS_hi times it fills the four
+            // 32-column groups of dQ in that order.  dS_lo . K_hi (groups g0, g1, 16 KB apart, N = 64)
+            // is accumulated 32 columns further, so that its halves land on the second and third group:
+            // head columns 0-31 = dQ[0:32) + dQ[32:64), 32-63 = dQ[64:96) + dQ[96:128).
+            const DescBase kmd = mnmaj64_base(km_s);
+            const DescBase kmd4 = make_desc_base(km_s, BKT * 128u, 512u, 1u);
+            for (int t = 0; t < n_t && ok; ++t) {
                 const int bb = t & 1;
-                if (!mbar_wait(ds_full(bb), (t >> 1) & 1u, g.err, 36)) return false;
+                if (!mbar_wait(ds_full(bb), (t >> 1) & 1u, g.err, 36)) { ok = false; break; }
                 trace_mark(g.trace, 0, tn, 400 + t);
-                if (!mbar_wait(mfull, t & 1u, g.err, 37)) return false;
+                if (!mbar_wait(mfull, t & 1u, g.err, 37)) { ok = false; break; }
                 trace_mark(g.trace, 0, tn, 500 + t);
                 tc_fence_after();
                 const uint32_t s_hi = tbuf(bb), s_lo = tbuf(bb) + 64u;
-                // Two instructions per k-step.  The MN-major K tile lies in shared memory as the column
-                // groups [K_hi g0 | K_lo g0 | K_hi g1 | K_lo g1] (g = 32 head columns), 8 KB apart: seen
-                // with that stride it is one operand of N = 128, and dS_hi times it fills the four
-                // 32-column groups of dQ in that order.  dS_lo . K_hi (groups g0, g1, 16 KB apart, N = 64)
-                // is accumulated 32 columns further, so that its halves land on the second and third group:
-                // head columns 0-31 = dQ[0:32) + dQ[32:64), 32-63 = dQ[64:96) + dQ[96:128).
-                const DescBase kmd = mnmaj64_base(km_s);
-                const DescBase kmd4 = make_desc_base(km_s, BKT * 128u, 512u, 1u);
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
                     const uint32_t acc = (t > 0 || ks > 0) ? 1u : 0u;
@@ -618,17 +682,12 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
                     umma_tf32_ts(tdQ + 32u, s_lo + ks * 8, kmd.at(mnmaj64_off(ks, false)), idesc_b, 1u);
                 }
                 umma_commit(mempty);
+                umma_commit(dq_done(bb));
                 trace_mark(g.trace, 0, tn, 600 + t);
-                return true;
-            };
-            if (ok) ok = issue_a(0);
-            for (int t = 0; t < n_t && ok; ++t) {
-                if (t + 1 < n_t) ok = issue_a(t + 1);
-                if (ok) ok = issue_b(t);
             }
             if (ok) umma_commit(acc_full);
         }
-    } else {
+    } else if (warp < kWarpMma2) {
         const int wg = (warp - 2) >> 2;
         const int lane_group = warp & 3;
         const int row = q0 + lane_group * 32 + lane;
@@ -773,9 +832,9 @@ cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, cons
               attention_tc_get_trace(), rg_sums, 4 * ((T + BR - 1) / BR)};
     dim3 gk(B * H, (T + BR - 1) / BR);
     // the dq kernel goes first: it also forms D = rowsum(dO o O), which the dkv kernel reads
-    BT_KERNEL_LAUNCH((attn_bwd_dq_tc_kernel), gk, kThreads, kDqSmem, s, qk64, qm64, qk64, dores, g);
+    BT_KERNEL_LAUNCH((attn_bwd_dq_tc_kernel), gk, kThreadsDq, kDqSmem, s, qk64, qm64, qk64, dores, g);
     BT_COUNT_LAUNCH();
-    BT_KERNEL_LAUNCH((attn_bwd_dkv_tc_kernel), gk, kThreads, kDkvSmem, s, qk64, qm64, dok64, dom64, vres, g);
+    BT_KERNEL_LAUNCH((attn_bwd_dkv_tc_kernel), gk, kThreadsDkv, kDkvSmem, s, qk64, qm64, dok64, dom64, vres, g);
     BT_COUNT_LAUNCH();
     return cudaGetLastError();
 }
