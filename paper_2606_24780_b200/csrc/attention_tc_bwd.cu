@@ -74,7 +74,7 @@ template <bool PAIRS = false>
 __device__ __forceinline__ void tmem_rows_to_split(uint32_t t_row, float mul, float* hi0, float* lo0,
                                                    long long row_stride, int nvalid, float* sums, float* tile,
                                                    int lane) {
-#pragma unroll
+#pragma unroll 1   // the body is long and runs once per CTA: keep one copy of it
     for (int half = 0; half < 2; ++half) {
         uint32_t r[32];
         float v[32];
@@ -167,7 +167,7 @@ struct BwdArgs {
 // trace record: (tag, SM clock) in the recording role's own region (no atomics, so a mark costs
 // a few instructions); only block (0,0) records
 constexpr int kTraceRegion = 500;
-__device__ __forceinline__ void trace_mark(unsigned long long* tr, int role, int& n, unsigned long long tag) {
+static __device__ __noinline__ void trace_mark(unsigned long long* tr, int role, int& n, unsigned long long tag) {
     if (tr == nullptr || blockIdx.x != 0 || blockIdx.y != 0) return;
     if (n < kTraceRegion) {
         unsigned long long* p = tr + 2 + 2 * (role * kTraceRegion + n);
@@ -279,19 +279,23 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             bool ok = true;
             // one buffer per (tensor, layout); t = the tile whose data goes in
             auto load = [&](uint32_t dst, const CUtensorMap* tm, int full, int empty, int t) -> bool {
-                if (!mbar_wait(bar(empty), (uint32_t)(t & 1) ^ 1u, g.err, 21)) return false;
+                if (!mbar_wait_ool(bar(empty), (uint32_t)(t & 1) ^ 1u, g.err, 21)) return false;
                 mbar_expect_tx(bar(full), kTile64);
                 for (int part = 0; part < 2; ++part)
                     tma_load_3d(dst + part * (kTile64 / 2), tm, bar(full), h * HD + part * 32, row_base + q_row0(t), 0);
                 return true;
             };
-            // in the order the products consume them: S^T(0), dP^T(0), then per tile dV(t), S^T(t+1), dK(t), dP^T(t+1)
-            if (n_t > 0) ok = load(qk_s, &tmQk, QK_FULL, QK_EMPTY, 0) && load(dok_s, &tmDOk, DOK_FULL, DOK_EMPTY, 0);
-            for (int t = 0; t < n_t && ok; ++t) {
-                ok = load(dom_s, &tmDOm, DOM_FULL, DOM_EMPTY, t);
-                if (ok && t + 1 < n_t) ok = load(qk_s, &tmQk, QK_FULL, QK_EMPTY, t + 1);
-                if (ok) ok = load(qm_s, &tmQm, QM_FULL, QM_EMPTY, t);
-                if (ok && t + 1 < n_t) ok = load(dok_s, &tmDOk, DOK_FULL, DOK_EMPTY, t + 1);
+            // in the order the products consume them: S^T(0), dP^T(0), then per tile dV(t), S^T(t+1), dK(t),
+            // dP^T(t+1) -- as a schedule walked by one loop, so that the load sequence exists once
+            for (int i = 0; i < 4 * n_t + 2 && ok; ++i) {
+                // j: 0 dO MN-major (t), 1 Q K-major (t+1), 2 Q MN-major (t), 3 dO K-major (t+1); first Q(0), dO(0) K-major
+                const int j = i == 0 ? 1 : i == 1 ? 3 : (i - 2) & 3;
+                const int tt = i < 2 ? 0 : ((i - 2) >> 2) + (j & 1);
+                if (tt >= n_t) continue;
+                const uint32_t dst = j == 0 ? dom_s : j == 1 ? qk_s : j == 2 ? qm_s : dok_s;
+                const CUtensorMap* tm = j == 0 ? &tmDOm : j == 1 ? &tmQk : j == 2 ? &tmQm : &tmDOk;
+                const int full = j == 0 ? DOM_FULL : j == 1 ? QK_FULL : j == 2 ? QM_FULL : DOK_FULL;
+                ok = load(dst, tm, full, full + 1, tt);      // every EMPTY barrier follows its FULL barrier
             }
             if (!ok)
                 for (int i = 0; i < 2000; ++i) __nanosleep(1000);
@@ -304,12 +308,12 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             // warp 1: the S^T -> P^T -> dV chain (regions tS, tPlo, tdV); warp 10: dP^T -> dS^T -> dK
             const bool score_chain = warp == 1;
             const int trole = score_chain ? 0 : 3;   // region of the debug trace
-            bool ok = score_chain ? mbar_wait(bar(K_READY), 0, g.err, 24) : mbar_wait(bar(V_FULL), 0, g.err, 23);
+            bool ok = score_chain ? mbar_wait_ool(bar(K_READY), 0, g.err, 24) : mbar_wait_ool(bar(V_FULL), 0, g.err, 23);
             int tn = 0;
             const DescBase vd = kmaj_base(v_s), qd = kmaj_base(qk_s), od = kmaj_base(dok_s);
             const DescBase omd = mn64_base(dom_s), qmd = mn64_base(qm_s);
             auto issue_s = [&](int t) -> bool {      // S^T(t) = K' Q^T
-                if (!mbar_wait(bar(QK_FULL), (uint32_t)(t & 1), g.err, 25)) return false;
+                if (!mbar_wait_ool(bar(QK_FULL), (uint32_t)(t & 1), g.err, 25)) return false;
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -325,7 +329,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 return true;
             };
             auto issue_dp = [&](int t) -> bool {     // dP^T(t) = V dO^T
-                if (!mbar_wait(bar(DOK_FULL), (uint32_t)(t & 1), g.err, 26)) return false;
+                if (!mbar_wait_ool(bar(DOK_FULL), (uint32_t)(t & 1), g.err, 26)) return false;
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -340,8 +344,8 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 return true;
             };
             auto issue_dv = [&](int t) -> bool {     // dV += P^T(t) dO
-                if (!mbar_wait(bar(P_READY), (uint32_t)(t & 1), g.err, 27)) return false;
-                if (!mbar_wait(bar(DOM_FULL), (uint32_t)(t & 1), g.err, 28)) return false;
+                if (!mbar_wait_ool(bar(P_READY), (uint32_t)(t & 1), g.err, 27)) return false;
+                if (!mbar_wait_ool(bar(DOM_FULL), (uint32_t)(t & 1), g.err, 28)) return false;
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -356,8 +360,8 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 return true;
             };
             auto issue_dk = [&](int t) -> bool {     // dK += dS^T(t) Q
-                if (!mbar_wait(bar(DS_READY), (uint32_t)(t & 1), g.err, 29)) return false;
-                if (!mbar_wait(bar(QM_FULL), (uint32_t)(t & 1), g.err, 30)) return false;
+                if (!mbar_wait_ool(bar(DS_READY), (uint32_t)(t & 1), g.err, 29)) return false;
+                if (!mbar_wait_ool(bar(QM_FULL), (uint32_t)(t & 1), g.err, 30)) return false;
                 tc_fence_after();
 #pragma unroll
                 for (int ks = 0; ks < 8; ++ks) {
@@ -374,17 +378,16 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             // Within a chain the product that overwrites a region follows the product that last read it
             // in this thread's own program order (the pipe executes a thread's MMAs in order); the two
             // chains share no region.
+            // (one call site per product: the unrolled issue sequences are large)
             if (score_chain) {
-                if (ok && n_t > 0) ok = issue_s(0);
-                for (int t = 0; t < n_t && ok; ++t) {
-                    ok = issue_dv(t);                              // frees the S^T / P^T regions ...
-                    if (ok && t + 1 < n_t) ok = issue_s(t + 1);    // ... which the next scores overwrite
+                for (int t = 0; t <= n_t && ok; ++t) {
+                    if (t > 0) ok = issue_dv(t - 1);               // frees the S^T / P^T regions ...
+                    if (ok && t < n_t) ok = issue_s(t);            // ... which the next scores overwrite
                 }
             } else {
-                if (ok && n_t > 0) ok = issue_dp(0);
-                for (int t = 0; t < n_t && ok; ++t) {
-                    ok = issue_dk(t);                              // frees the dP^T / dS^T regions ...
-                    if (ok && t + 1 < n_t) ok = issue_dp(t + 1);   // ... which the next dP^T overwrites
+                for (int t = 0; t <= n_t && ok; ++t) {
+                    if (t > 0) ok = issue_dk(t - 1);               // frees the dP^T / dS^T regions ...
+                    if (ok && t < n_t) ok = issue_dp(t);           // ... which the next dP^T overwrites
                 }
             }
             if (ok) umma_commit(bar(ACC_FULL));
@@ -438,7 +441,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             const int nvalid = min(32, g.T - q0);
             float next_stat = 0.f;
             if (sidx < 128 && t + 1 < n_t) next_stat = fetch_stat(t + 1);   // in flight during this tile
-            if (!mbar_wait_warp(bar(STAT_READY), (uint32_t)(t & 1), g.err, 42)) { ok = false; break; }
+            if (!mbar_wait_warp_ool(bar(STAT_READY), (uint32_t)(t & 1), g.err, 42)) { ok = false; break; }
             float Lc[32], Dc[32];
             {
                 const float4* Ls = reinterpret_cast<const float4*>(stat + (t & 1) * 128 + 32 * wg);
@@ -451,7 +454,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                 }
             }
             if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 700 + t);
-            if (!mbar_wait_warp(bar(S_FULL), (uint32_t)(t & 1), g.err, 31)) { ok = false; break; }
+            if (!mbar_wait_warp_ool(bar(S_FULL), (uint32_t)(t & 1), g.err, 31)) { ok = false; break; }
             tc_fence_after();
             uint32_t s[32];
             float p[32];
@@ -472,7 +475,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             __syncwarp();
             if (lane == 0) mbar_arrive(bar(P_READY));
             if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 800 + t);
-            if (!mbar_wait_warp(bar(DP_FULL), (uint32_t)(t & 1), g.err, 32)) { ok = false; break; }
+            if (!mbar_wait_warp_ool(bar(DP_FULL), (uint32_t)(t & 1), g.err, 32)) { ok = false; break; }
             tc_fence_after();
             tmem_ld32(tdP + t_lane + c0, s);
             tmem_ld32(tdSlo + t_lane + c0, lo);
@@ -491,7 +494,7 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
             if (etid == 0) trace_mark(g.trace, 1 + wg, tn, 900 + t);
             if (t + 1 < n_t) publish_stat(t + 1, next_stat);
         }
-        if (ok) ok = mbar_wait_warp(bar(ACC_FULL), 0, g.err, 33);
+        if (ok) ok = mbar_wait_warp_ool(bar(ACC_FULL), 0, g.err, 33);
         if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
             tc_fence_after();
             const int wrow0 = j0 + lane_group * 32;                    // first key row of this warp
@@ -503,8 +506,10 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
                               : nullptr;
             // the streamed-tile buffers are idle by now: each warp stages its rows in a slice of them
             float* tile = reinterpret_cast<float*>(smem_raw + (qk_s - smem_u32(smem_raw)) + (uint32_t)(warp - 2) * kRowTileBytes);
-            if (wg == 0) tmem_rows_to_split(tdK + t_lane, scale, hi + g.C, lo + g.C, gs, nvalid, sums ? sums + g.C : nullptr, tile, lane);
-            else tmem_rows_to_split(tdV + t_lane, 1.0f, hi + 2 * g.C, lo + 2 * g.C, gs, nvalid, sums ? sums + 2 * g.C : nullptr, tile, lane);
+            // warpgroup 0 writes dK (columns C .. 2C of the row), warpgroup 1 dV (2C .. 3C): one call site
+            const int64_t col = (int64_t)(1 + wg) * g.C;
+            tmem_rows_to_split((wg == 0 ? tdK : tdV) + t_lane, wg == 0 ? scale : 1.0f, hi + col, lo + col, gs, nvalid,
+                               sums ? sums + col : nullptr, tile, lane);
         }
     }
     tc_fence_before();
@@ -584,7 +589,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             bool ok = true;
             auto load_kmajor = [&](int t) -> bool {
                 const int st = t & 1, k0 = t * BKT;
-                if (!mbar_wait(kempty(st), ((t >> 1) & 1u) ^ 1u, g.err, 31)) return false;
+                if (!mbar_wait_ool(kempty(st), ((t >> 1) & 1u) ^ 1u, g.err, 31)) return false;
                 mbar_expect_tx(kfull(st), 2u * kTileQ);
                 for (int kb = 0; kb < 2; ++kb) {
                     tma_load_3d(kk_s(st) + kb * (kTileQ / 2), &tmKk, kfull(st), g.C + h * HD + kb * 32, row_base + k0, 0);
@@ -599,8 +604,8 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
                 if (t + 1 < n_t) ok = load_kmajor(t + 1);
                 if (!ok) break;
                 // the MN-major buffer doubles as the staging area of the query rows: first fill after that
-                if (t == 0 && !mbar_wait(q_ready, 0, g.err, 40)) { ok = false; break; }
-                if (!mbar_wait(mempty, (t & 1u) ^ 1u, g.err, 32)) { ok = false; break; }
+                if (t == 0 && !mbar_wait_ool(q_ready, 0, g.err, 40)) { ok = false; break; }
+                if (!mbar_wait_ool(mempty, (t & 1u) ^ 1u, g.err, 32)) { ok = false; break; }
                 mbar_expect_tx(mfull, kTileQ);
                 for (int grp = 0; grp < 2; ++grp)
                     tma_load_3d(km_s + grp * (kTileQ / 2), &tmKm, mfull, g.C + h * HD + grp * 32, row_base + t * BKT, 0);
@@ -615,14 +620,14 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
         if (lane == 0) {
             constexpr uint32_t idesc_a = make_idesc_tf32(BR, BKT, false, false);   // 128 x 64, B K-major
             const bool s_product = warp == 1;
-            bool ok = s_product ? mbar_wait(q_ready, 0, g.err, 34) : mbar_wait(do_full, 0, g.err, 33);
+            bool ok = s_product ? mbar_wait_ool(q_ready, 0, g.err, 34) : mbar_wait_ool(do_full, 0, g.err, 33);
             int tn = 0;
             const DescBase dod = kmaj_base(do_s);
             for (int t = 0; t < n_t && ok; ++t) {
                 const int st = t & 1, bb = t & 1;
                 trace_mark(g.trace, 0, tn, 100 + t);
-                if (!mbar_wait(kfull(st), (t >> 1) & 1u, g.err, 35)) { ok = false; break; }
-                if (t >= 2 && !mbar_wait(dq_done(bb), ((t - 2) >> 1) & 1u, g.err, 41)) { ok = false; break; }
+                if (!mbar_wait_ool(kfull(st), (t >> 1) & 1u, g.err, 35)) { ok = false; break; }
+                if (t >= 2 && !mbar_wait_ool(dq_done(bb), ((t - 2) >> 1) & 1u, g.err, 41)) { ok = false; break; }
                 trace_mark(g.trace, 0, tn, 200 + t);
                 tc_fence_after();
                 if (s_product) {
@@ -669,9 +674,9 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             const DescBase kmd4 = make_desc_base(km_s, BKT * 128u, 512u, 1u);
             for (int t = 0; t < n_t && ok; ++t) {
                 const int bb = t & 1;
-                if (!mbar_wait(ds_full(bb), (t >> 1) & 1u, g.err, 36)) { ok = false; break; }
+                if (!mbar_wait_ool(ds_full(bb), (t >> 1) & 1u, g.err, 36)) { ok = false; break; }
                 trace_mark(g.trace, 0, tn, 400 + t);
-                if (!mbar_wait(mfull, t & 1u, g.err, 37)) { ok = false; break; }
+                if (!mbar_wait_ool(mfull, t & 1u, g.err, 37)) { ok = false; break; }
                 trace_mark(g.trace, 0, tn, 500 + t);
                 tc_fence_after();
                 const uint32_t s_hi = tbuf(bb), s_lo = tbuf(bb) + 64u;
@@ -729,7 +734,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
         for (int t = wg; t < n_t && ok; t += 2) {
             const int k0 = t * BKT;
             if (lane_group == 0 && lane == 0) trace_mark(g.trace, 1 + wg, tn, 700 + t);
-            if (!mbar_wait_warp(sdp_full(wg), (t >> 1) & 1u, g.err, 38)) { ok = false; break; }
+            if (!mbar_wait_warp_ool(sdp_full(wg), (t >> 1) & 1u, g.err, 38)) { ok = false; break; }
             if (lane_group == 0 && lane == 0) trace_mark(g.trace, 1 + wg, tn, 800 + t);
             tc_fence_after();
 #pragma unroll
@@ -755,7 +760,7 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
             if (lane_group == 0 && lane == 0) trace_mark(g.trace, 1 + wg, tn, 1000 + t);
         }
         if (wg == 0) {
-            if (ok) ok = mbar_wait_warp(acc_full, 0, g.err, 39);
+            if (ok) ok = mbar_wait_warp_ool(acc_full, 0, g.err, 39);
             if (ok) {   // warp-uniform: the tensor-memory loads below need the whole warp
                 tc_fence_after();
                 const int wrow0 = q0 + lane_group * 32;                // first query row of this warp

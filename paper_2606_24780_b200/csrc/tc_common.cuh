@@ -61,6 +61,34 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, int* er
     }
 }
 
+// The same wait with its polling loop out of line.  The attention kernels wait at dozens of sites and
+// their code has to stay within the instruction cache (every CTA start fetches it again: 175 KB of
+// inlined code cost the backward kernels 8 % of their time against 123 KB); a wait that did not
+// succeed at once has the time for a call.  Roles whose live registers are at the limit keep the
+// inline form (a call spills them).
+static __device__ __noinline__ bool mbar_wait_poll(uint32_t bar, uint32_t parity, int* err, int code,
+                                                   unsigned long long limit_ns) {
+    const unsigned long long t0 = globaltimer_ns();
+    for (;;) {
+        for (int i = 0; i < 256; ++i)
+            if (mbar_try_wait(bar, parity)) return true;
+        if (globaltimer_ns() - t0 > limit_ns) {
+            atomicCAS(err, 0, code);  // the first wait that ran out is the one reported
+            return false;
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait_ool(uint32_t bar, uint32_t parity, int* err, int code,
+                                              unsigned long long limit_ns = kWaitLimitNs) {
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_poll(bar, parity, err, code, limit_ns);
+}
+__device__ __forceinline__ bool mbar_wait_warp_ool(uint32_t bar, uint32_t parity, int* err, int code,
+                                                   unsigned long long limit_ns = kWaitLimitNs) {
+    const bool ok = mbar_wait_ool(bar, parity, err, code, limit_ns);
+    return __all_sync(0xffffffffu, ok);
+}
+
 // The same wait made by a whole warp, with a warp-uniform result: the callers go on to issue
 // .sync.aligned tensor-memory instructions, which every lane of the warp must reach together.
 __device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, int* err, int code,
@@ -258,7 +286,7 @@ __device__ __forceinline__ DescBase kmaj_base(uint32_t tile) { return make_desc_
 __device__ __forceinline__ void rows_to_tmem(const float* src_hi, const float* src_lo, long long row_stride, int nvalid,
                                              float mul, uint32_t t_hi, uint32_t t_lo, float* tile, int lane) {
     const int sub = lane >> 3, cq = lane & 7;
-#pragma unroll
+#pragma unroll 1   // runs once per CTA: one copy of the body (the kernels' code has to fit the instruction cache)
     for (int half = 0; half < 2; ++half) {
         float4 a[8], b[8];
 #pragma unroll
