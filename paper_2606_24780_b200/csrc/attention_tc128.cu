@@ -284,11 +284,26 @@ attn128_kernel(const __grid_constant__ CUtensorMap tmA2, const __grid_constant__
             const int s0 = o0(t);                         // first streamed row of the tile
             float Lc[32], Dc[32];
             if (kKeys) {   // the tile's 32 queries: same addresses in every thread (broadcast loads)
+                if (s0 + 32 <= g.T && ((lb + s0) & 3) == 0) {   // whole tile inside the sequence, 16-byte aligned: 128-bit loads
+                    const float4* lp = reinterpret_cast<const float4*>(g.lse + lb + s0);
+                    const float4* dp = reinterpret_cast<const float4*>(g.dvec + lb + s0);
 #pragma unroll
-                for (int i = 0; i < 32; ++i) {
-                    const int r = min(s0 + i, g.T - 1);   // rows past the end are masked below
-                    Lc[i] = __ldg(g.lse + lb + r) * kLog2e;
-                    if (PASS == P_DK) Dc[i] = __ldg(g.dvec + lb + r);
+                    for (int i = 0; i < 8; ++i) {
+                        const float4 l4 = __ldg(lp + i);
+                        Lc[4 * i] = l4.x * kLog2e; Lc[4 * i + 1] = l4.y * kLog2e;
+                        Lc[4 * i + 2] = l4.z * kLog2e; Lc[4 * i + 3] = l4.w * kLog2e;
+                        if (PASS == P_DK) {
+                            const float4 d4 = __ldg(dp + i);
+                            Dc[4 * i] = d4.x; Dc[4 * i + 1] = d4.y; Dc[4 * i + 2] = d4.z; Dc[4 * i + 3] = d4.w;
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < 32; ++i) {
+                        const int r = min(s0 + i, g.T - 1);   // rows past the end are masked below
+                        Lc[i] = __ldg(g.lse + lb + r) * kLog2e;
+                        if (PASS == P_DK) Dc[i] = __ldg(g.dvec + lb + r);
+                    }
                 }
             }
             if (!mbar_wait_warp(bar(XY_FULL0 + wg), (uint32_t)((t >> 1) & 1), g.err, 59)) { ok = false; break; }
