@@ -3,7 +3,7 @@
 // Two deterministic kernels (no atomics) that recompute the probabilities from (q, k, lse):
 //
 //   dkv kernel  one CTA owns 128 keys (one per TMEM lane) of one (sequence, head) and walks the
-//               32-row query tiles at or below the diagonal:
+//               64-row query tiles at or below the diagonal:
 //                 S^T  = K' Q^T      A = K' (pre-scaled, hi/lo) held in TENSOR MEMORY, B = Q tile (smem)
 //                 dP^T = V  dO^T     A = V (smem, resident),                           B = dO tile
 //                 P^T  = exp2(S^T - lse),  dS^T = P^T o (dP^T - D)       (thread = key row)
@@ -15,7 +15,7 @@
 //               small additions to an already large sum drifts toward zero (about n * 2^-25 after
 //               n MMAs); probabilities of a key usually decay with the query's distance, and adding
 //               the small far-away terms first keeps that drift relative to a small sum.
-//   dq kernel   one CTA owns 128 query rows and walks the 32-key tiles up to the diagonal:
+//   dq kernel   one CTA owns 128 query rows and walks the 64-key tiles up to the diagonal:
 //                 S  = Q' K^T (A = Q' in tensor memory),  dP = dO V^T (A = dO resident in smem),
 //                 dS = P o (dP - D),  dQ += dS K (A = dS in tensor memory).
 //
@@ -23,10 +23,19 @@
 // needs: K-major (128-byte swizzle) where the tile is the B operand of a "row . row" product, and
 // MN-major (128-byte swizzle, 32-byte atoms) where its rows are the contraction index.  The two
 // layouts have their own full/empty barriers, so a tile's K-major half is refilled as soon as the
-// first pair of products has consumed it.  Score/gradient buffers in tensor memory are double
-// buffered: the products of tile t+1 are issued before the accumulating products of tile t, so
-// the tensor pipe runs while the 128 element-wise threads work.
-// Every mbarrier wait is bounded and reports through the device error word.
+// first pair of products has consumed it.
+//
+// Issuing threads.  One thread issues a tcgen05.mma about every 57 clocks whatever its shape, while
+// an N = 64 product occupies the pipe for 32 clocks when its A operand comes from tensor memory
+// (48 from shared memory).  The products are therefore spread over several issuing threads, each
+// owning whole products and a chain of tensor-memory regions of its own: in the dkv kernel warp 1
+// issues S^T(t+1) right behind dV(t) (same regions: the pipe runs one thread's MMAs in order) and
+// warp 10 dP^T(t+1) behind dK(t); in the dq kernel warps 1, 10 and 11 issue S, dP and dQ, and the
+// two score products of tile t + 2 wait on a barrier for the dQ product of tile t to have read the
+// buffer they overwrite.  The chains meet only in mbarriers.
+// Every mbarrier wait is bounded and reports through the device error word; the polling loop is
+// out of line and the long run-once sequences have one copy each, because these kernels are
+// large (90 and 101 KB of code) and every CTA start runs through them with a cold instruction cache.
 #include "common.cuh"
 #include "tc_common.cuh"
 
