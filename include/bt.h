@@ -339,6 +339,17 @@ BT_API bt_status bt_selftest_bounded_wait(bt_model* m, float limit_ms);
 BT_API bt_status bt_probe_tf32_mma_rate(int32_t n_ctas, int32_t iters, int64_t* d_clocks, int32_t* d_err,
                                         void* stream);
 
+/* The same kind of measurement for the ISSUE rate: in each of n_ctas CTAs, `issuers` threads (1-4,
+ * in different warps) each issue `iters` MMAs of M = 128, N = n (64, 128 or 256), K = 8 with the A
+ * operand in shared memory or (a_in_tmem, n <= 128) in tensor memory; d_clocks[4 * cta + i] (device
+ * int64, 4 * n_ctas entries) receives thread i's clocks from its first issue to the completion of
+ * its last MMA (-1 and *d_err = 902 if the bounded wait ran out).  max_i clocks / (iters x issuers)
+ * is the cost of one MMA with that many issuing threads: the attention kernels' division of their
+ * products among issuing threads rests on it (Appendix "Hardware and Benchmarking Methodology").
+ * Asynchronous. */
+BT_API bt_status bt_probe_mma_issue_rate(int32_t n, int32_t a_in_tmem, int32_t issuers, int32_t n_ctas, int32_t iters,
+                                         int64_t* d_clocks, int32_t* d_err, void* stream);
+
 /* Synchronises and reads the loss of the last forward. */
 BT_API bt_status bt_get_loss(bt_model* m, float* h_loss);
 

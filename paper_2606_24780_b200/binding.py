@@ -97,6 +97,7 @@ _SIGNATURES = {
     "bt_first_invalid_id": (_i64, [_vp, _i64, _i32]),
     "bt_selftest_bounded_wait": (_i32, [_vp, _f]),
     "bt_probe_tf32_mma_rate": (_i32, [_i32, _i32, _vp, _vp, _vp]),
+    "bt_probe_mma_issue_rate": (_i32, [_i32, _i32, _i32, _i32, _i32, _vp, _vp, _vp]),
     "bt_op_layernorm_fwd": (_i32, [_vp, _vp, _vp, _i64, _i32, _vp, _vp, _vp, _vp, _vp]),
     "bt_op_layernorm_bwd_scratch_bytes": (_sz, [_i64, _i32]),
     "bt_op_layernorm_bwd": (_i32, [_vp] * 6 + [_i64, _i32] + [_vp] * 5 + [_sz, _vp]),
@@ -451,6 +452,21 @@ def bt_probe_tf32_mma_rate(n_ctas=148, iters=4000, stream=None):
         raise BtError(5, f"rate probe: a bounded wait ran out (code {int(err[0])})")
     c = clocks.double() / iters
     return float(c.min()), float(c.median()), float(c.max())
+
+
+def bt_probe_mma_issue_rate(n, a_in_tmem, issuers, n_ctas=148, iters=4096, stream=None):
+    """Clocks per tcgen05.mma (128 x n x 8) with `issuers` issuing threads per CTA: median over the CTAs of
+    (slowest thread's clocks) / (iters x issuers)."""
+    clocks = torch.zeros(4 * n_ctas, dtype=torch.int64, device="cuda")
+    err = torch.zeros(4, dtype=torch.int32, device="cuda")
+    for _ in range(2):                       # the first launch also loads the kernel
+        _check(lib().bt_probe_mma_issue_rate(n, int(a_in_tmem), issuers, n_ctas, iters, _ptr(clocks), _ptr(err),
+                                             _stream(stream)))
+    torch.cuda.synchronize()
+    c = clocks.view(n_ctas, 4)[:, :issuers]
+    if int(err[0]) != 0 or int(c.min()) < 0:
+        raise BtError(5, f"issue-rate probe: a bounded wait ran out (code {int(err[0])})")
+    return float((c.max(dim=1).values.double() / (iters * issuers)).median())
 
 
 def bt_selftest_bounded_wait(model, limit_ms):

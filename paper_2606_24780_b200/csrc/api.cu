@@ -1130,6 +1130,19 @@ extern "C" bt_status bt_probe_tf32_mma_rate(int32_t n_ctas, int32_t iters, int64
     return BT_OK;
 }
 
+extern "C" bt_status bt_probe_mma_issue_rate(int32_t n, int32_t a_in_tmem, int32_t issuers, int32_t n_ctas, int32_t iters,
+                                             int64_t* d_clocks, int32_t* d_err, void* stream) {
+    if (!d_clocks || !d_err) return fail(BT_ERR_INVALID_ARG, "probe: NULL argument");
+    if (reinterpret_cast<uintptr_t>(d_clocks) & 7u) return fail(BT_ERR_INVALID_ARG, "probe: d_clocks not 8-byte aligned");
+    if ((n != 64 && n != 128 && n != 256) || (n == 256 && a_in_tmem) || issuers < 1 || issuers > 4)
+        return fail(BT_ERR_INVALID_ARG, "probe: n in {64, 128, 256} (256: A in shared memory only), issuers in [1, 4]");
+    if (n_ctas < 1 || n_ctas > 4096 || iters < 16 || iters > (1 << 20))
+        return fail(BT_ERR_INVALID_ARG, "probe: n_ctas in [1, 4096], iters in [16, 2^20]");
+    BT_CUDA(launch_mma_issue_probe(n, a_in_tmem ? 1 : 0, issuers, n_ctas, iters, reinterpret_cast<long long*>(d_clocks), d_err,
+                                   (cudaStream_t)stream));
+    return BT_OK;
+}
+
 // =============================================================================== per-op entry points
 
 extern "C" bt_status bt_op_embedding_fwd(const int32_t* tok, const float* wte, const float* wpe, int64_t N, int32_t T,

@@ -243,6 +243,8 @@ constexpr int kSelftestWaitCode = 900;
 cudaError_t launch_bounded_wait_probe(int* err, unsigned long long limit_ns, int code, cudaStream_t s);
 // clocks[cta] = SM clocks that `iters` tcgen05.mma.kind::tf32 (128 x 256 x 8) took on that CTA's SM (-1: wait ran out).
 cudaError_t launch_tf32_rate_probe(int n_ctas, int iters, long long* clocks, int* err, cudaStream_t s);
+cudaError_t launch_mma_issue_probe(int n, int a_in_tmem, int issuers, int n_ctas, int iters, long long* clocks, int* err,
+                                   cudaStream_t s);
 
 // SIMT reference GEMM: D = op(A) op(B) (+bias) (+residual), operands given as split planes
 // (lo may be absent: plane == 0 means "hi only").

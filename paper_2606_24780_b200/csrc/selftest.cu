@@ -85,6 +85,74 @@ __global__ void __launch_bounds__(128) tf32_rate_probe_kernel(int iters, long lo
     if (tid == 0) clocks[blockIdx.x] = dt;
 }
 
+// The issue-rate probe: `issuers` threads (lane 0 of warps 0 .. issuers - 1) each issue `iters`
+// MMAs of M = 128, N, K = 8 -- A from shared memory or (TS) from tensor memory -- into an accumulator
+// of their own where the columns allow (N = 64) or a shared one, and record the clocks from their
+// first issue to the completion of their last MMA.
+template <int N, bool TS>
+__global__ void __launch_bounds__(128) mma_issue_probe_kernel(int iters, int issuers, long long* __restrict__ clocks, int* err) {
+    extern __shared__ uint8_t probe_smem[];
+    __shared__ uint32_t tmem_base_s;
+    __shared__ __align__(8) unsigned long long bar[4];
+    const uint32_t sm0 = (smem_u32(probe_smem) + 1023u) & ~1023u;
+    float* smf = reinterpret_cast<float*>(probe_smem + (sm0 - smem_u32(probe_smem)));
+    const int tid = threadIdx.x, w = tid >> 5;
+    for (int i = tid; i < (48 * 1024) / 4; i += 128) smf[i] = 0.001f * (float)(i & 255);
+    if (tid < 32) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512u)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if (tid == 0) {
+        for (int i = 0; i < 4; ++i) mbar_init(smem_u32(&bar[i]), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tm = tmem_base_s;
+    if ((tid & 31) == 0 && w < issuers) {
+        const DescBase ad = kmaj_base(sm0), bd = kmaj_base(sm0 + 16u * 1024u);   // A: 128 rows, B: up to 256 rows of 128 B
+        constexpr uint32_t idesc = make_idesc_tf32(128, N, false, false);
+        const uint32_t d = tm + 256u + (N <= 64 ? (uint32_t)w * 64u : 0u);         // columns 0-63 serve as the TMEM A operand
+        long long dt = -1;
+        const long long t0 = clock64();
+        for (int it = 0; it < iters; ++it) {
+            const uint32_t koff = (uint32_t)(it & 3) * 32u;
+            if (TS) umma_tf32_ts(d, tm + (uint32_t)(it & 7) * 8u, bd.at(koff), idesc, 1u);
+            else umma_tf32(d, ad.at(koff), bd.at(koff), idesc, 1u);
+        }
+        umma_commit(smem_u32(&bar[w]));
+        if (mbar_wait(smem_u32(&bar[w]), 0u, err, 902)) dt = clock64() - t0;
+        clocks[blockIdx.x * 4 + w] = dt;
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (tid < 32) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tm), "r"(512u) : "memory");
+}
+
+template <int N, bool TS>
+static cudaError_t launch_issue_probe_t(int n_ctas, int iters, int issuers, long long* clocks, int* err, cudaStream_t s) {
+    constexpr int kSmem = 49 * 1024 + 1024;
+    cudaError_t e = cudaFuncSetAttribute(mma_issue_probe_kernel<N, TS>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem);
+    if (e != cudaSuccess) return e;
+    mma_issue_probe_kernel<N, TS><<<n_ctas, 128, kSmem, s>>>(iters, issuers, clocks, err);
+    BT_COUNT_LAUNCH();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_mma_issue_probe(int n, int a_in_tmem, int issuers, int n_ctas, int iters, long long* clocks, int* err,
+                                   cudaStream_t s) {
+    if (n == 64) return a_in_tmem ? launch_issue_probe_t<64, true>(n_ctas, iters, issuers, clocks, err, s)
+                                  : launch_issue_probe_t<64, false>(n_ctas, iters, issuers, clocks, err, s);
+    if (n == 128) return a_in_tmem ? launch_issue_probe_t<128, true>(n_ctas, iters, issuers, clocks, err, s)
+                                   : launch_issue_probe_t<128, false>(n_ctas, iters, issuers, clocks, err, s);
+    if (n == 256 && !a_in_tmem) return launch_issue_probe_t<256, false>(n_ctas, iters, issuers, clocks, err, s);
+    return cudaErrorInvalidValue;
+}
+
 cudaError_t launch_tf32_rate_probe(int n_ctas, int iters, long long* clocks, int* err, cudaStream_t s) {
     constexpr int kSmem = 49 * 1024 + 1024;
     static cudaError_t attr =

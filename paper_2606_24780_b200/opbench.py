@@ -228,6 +228,14 @@ def tf32_rate(sm_mhz=None):
     return {"clocks_per_mma_128x256x8": med, "clocks_min_max": [lo, hi], "mac_per_clk_per_sm": 128 * 256 * 8 / med}
 
 
+def issue_rates():
+    """Clocks per MMA (M = 128, K = 8) by width, operand source and number of issuing threads."""
+    out = {}
+    for n, tmem in ((64, 0), (64, 1), (128, 0), (256, 0)):
+        out[f"n{n}_{'tmem' if tmem else 'smem'}"] = [round(b.bt_probe_mma_issue_rate(n, tmem, k), 1) for k in (1, 2, 3)]
+    return out
+
+
 def hbm_rates(n_bytes=1 << 30, iters=10):
     """Measured HBM rates for the roofline denominators of the memory-bound kernels (harness-side torch
     kernels, best of `iters`): a copy (read + write bytes), a pure write (fill) and a pure read (sum).
@@ -300,6 +308,11 @@ def main(argv=None):
         print(f"tf32_rate              {r['clocks_per_mma_128x256x8']:10.1f} clk per 128x256x8 MMA  "
               f"{r['mac_per_clk_per_sm']:7.0f} MAC/clk/SM  (x 2 x {sms} SMs x clock = dense TF32 peak; / 3 for 3xTF32)",
               flush=True)
+    if not only or "issue_rates" in only:
+        r = issue_rates()
+        results["issue_rates"] = r
+        print("issue_rates            clocks per 128 x N x 8 MMA with 1 / 2 / 3 issuing threads: " +
+              ", ".join(f"{k} {v[0]} / {v[1]} / {v[2]}" for k, v in r.items()), flush=True)
     if not only or "hbm_rates" in only:
         r = hbm_rates()
         results["hbm_rates"] = r

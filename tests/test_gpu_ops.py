@@ -519,3 +519,22 @@ def test_empty_inputs_are_no_ops_or_rejected():
             call()
         assert e.value.status == 1
     torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ rate probes (measurement aids)
+
+def test_mma_rate_probes_give_the_rates_the_kernels_are_planned_with():
+    """The probes behind the roofline's TF32 peak and behind the attention kernels' division of their
+    products among issuing threads: a 128 x 256 x 8 MMA occupies the pipe for 128 clocks (2048 MAC per
+    clock and SM); one thread cannot issue N = 64 MMAs as fast as the pipe executes them with the A
+    operand in tensor memory (32 clocks), two can; bad arguments are refused on the host."""
+    lo, med, hi = b.bt_probe_tf32_mma_rate(8, 2000)
+    assert 120.0 < med < 140.0 and hi < 160.0
+    one = b.bt_probe_mma_issue_rate(64, True, 1, n_ctas=8, iters=2048)
+    two = b.bt_probe_mma_issue_rate(64, True, 2, n_ctas=8, iters=2048)
+    assert 45.0 < one < 75.0 and 30.0 < two < 40.0 and two < 0.75 * one
+    assert 120.0 < b.bt_probe_mma_issue_rate(256, False, 2, n_ctas=8, iters=1024) < 140.0
+    for args in [(96, 0, 1), (256, 1, 1), (64, 0, 0), (64, 0, 5)]:
+        with pytest.raises(b.BtError) as e:
+            b.bt_probe_mma_issue_rate(*args, n_ctas=1, iters=16)
+        assert e.value.status == 1
