@@ -155,11 +155,11 @@ def run_reference(args, cfg):
         return
     import oracle
     total_steps = args.steps + args.warmup
-    budget = 150.0 / max(1, total_steps)
-    # calibrate on a 64-token sequence, then pick the longest sample that fits the per-step budget
+    allowance = 150.0 / max(1, total_steps)
+    # calibrate on a 64-token sequence, then pick the longest sample that fits the per-step allowance
     dt64, cores, _ = oracle_step_seconds(cfg, 64, 1)
     seq = 64
-    while seq * 2 <= cfg["seq_len"] and dt64 * (seq * 2 / 64.0) * 1.3 < budget:
+    while seq * 2 <= cfg["seq_len"] and dt64 * (seq * 2 / 64.0) * 1.3 < allowance:
         seq *= 2
     c = dict(cfg)
     c["seq_len"] = seq
