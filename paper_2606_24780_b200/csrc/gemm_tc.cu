@@ -71,6 +71,11 @@ struct GemmArgs {
     const float* residual;
     int tiles_m, tiles_n, splits, kb_per_split, kb_total;
     float* partials;
+    // Tail split (pair kernel, splits == 1): the tiles of the complete rounds run with the whole K; the
+    // tail_tiles tiles of the last, partly filled round are cut into tail_splits K ranges, so that this
+    // round costs 1 / tail_splits of a tile's time.  Their partial tiles go to `partials`, compact,
+    // [split][tail tile][256 x BN]; a second kernel adds them in split order and runs the output path.
+    int full_units, tail_tiles, tail_splits, tail_kbps;
     int* err;
     float* d_hi;        // optional TF32 hi/lo planes of the output (lo = d_hi + d_plane)
     long long d_plane;
@@ -80,6 +85,39 @@ struct GemmArgs {
                         // 7: `residual` holds GELU'(h) itself and the output is (A B) o residual
     float* col_partial; // act 5 - 7: column sums of the output per 32-row group, [ceil(M / 32)][N] (nullable)
 };
+
+// One work unit of the pair kernel: its tile, its k-block range and, for a partial result, the slot of
+// its partial tile (-1: the unit produces the output itself).
+struct PairUnit {
+    int tm, tn, kb0, kb1, partial;
+};
+__device__ __forceinline__ PairUnit decode_pair_unit(const GemmArgs& g, int u) {
+    PairUnit w;
+    if (g.tail_splits > 1) {
+        int tile = u, sp = 0;
+        w.partial = -1;
+        w.kb0 = 0;
+        w.kb1 = g.kb_total;
+        if (u >= g.full_units) {
+            const int v = u - g.full_units;
+            sp = v / g.tail_tiles;                       // all tiles' first range, then all second ranges, ...
+            tile = g.full_units + v % g.tail_tiles;
+            w.kb0 = sp * g.tail_kbps;
+            w.kb1 = min(g.kb_total, w.kb0 + g.tail_kbps);
+            w.partial = sp * g.tail_tiles + v % g.tail_tiles;
+        }
+        w.tm = tile % g.tiles_m;
+        w.tn = tile / g.tiles_m;
+        return w;
+    }
+    const int r = u / g.tiles_m, sp = r / g.tiles_n;
+    w.tm = u % g.tiles_m;
+    w.tn = r % g.tiles_n;
+    w.kb0 = sp * g.kb_per_split;
+    w.kb1 = min(g.kb_total, w.kb0 + g.kb_per_split);
+    w.partial = g.splits > 1 ? sp : -1;
+    return w;
+}
 
 // Descriptor of one 8-deep k-step of an operand tile.
 //   K-major (rows of BK floats): [plane][rows][BK]; BK = 32 -> 128B swizzle (mode 2, SBO 1024),
@@ -409,7 +447,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     pdl_wait();
     pdl_trigger();
 
-    const int units = g.tiles_m * g.tiles_n * g.splits;   // tiles_m counts 256-row tiles here
+    // tiles_m counts 256-row tiles here
+    const int units = g.tail_splits > 1 ? g.full_units + g.tail_tiles * g.tail_splits : g.tiles_m * g.tiles_n * g.splits;
 
     if (warp == 0) {
         // ---------------------------------------------------------------- TMA producer (both CTAs)
@@ -417,11 +456,10 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             uint32_t it = 0;
             bool ok = true;
             for (int u = pair; u < units && ok; u += n_pairs) {
-                const int tm = u % g.tiles_m, r = u / g.tiles_m, tn = r % g.tiles_n, sp = r / g.tiles_n;
-                const int kb0 = sp * g.kb_per_split;
-                const int kb1 = min(g.kb_total, kb0 + g.kb_per_split);
-                const int a_row = tm * 2 * BM + (int)rank * BM;      // first A row (or column, if MN-major) of this CTA
-                const int b_col = tn * BN + (int)rank * BH;          // first B column of this CTA
+                const PairUnit w = decode_pair_unit(g, u);
+                const int kb0 = w.kb0, kb1 = w.kb1;
+                const int a_row = w.tm * 2 * BM + (int)rank * BM;    // first A row (or column, if MN-major) of this CTA
+                const int b_col = w.tn * BN + (int)rank * BH;        // first B column of this CTA
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
                     const int s = it % C::kStages;
                     const uint32_t ph = (it / C::kStages) & 1u;
@@ -456,9 +494,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             uint32_t it = 0, ut = 0;
             bool ok = true;
             for (int u = pair; u < units && ok; u += n_pairs, ++ut) {
-                const int r = u / g.tiles_m, sp = r / g.tiles_n;
-                const int kb0 = sp * g.kb_per_split;
-                const int kb1 = min(g.kb_total, kb0 + g.kb_per_split);
+                const PairUnit w = decode_pair_unit(g, u);
+                const int kb0 = w.kb0, kb1 = w.kb1;
                 const int acc = ut & 1;
                 const uint32_t aph = (ut >> 1) & 1u;
                 if (!mbar_wait(tempty_bar(acc), aph ^ 1u, g.err, 6)) { ok = false; break; }
@@ -493,7 +530,8 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         bool ok = true;
         const uint32_t my_tempty0 = mapa_shared(tempty_bar(0), 0), my_tempty1 = mapa_shared(tempty_bar(1), 0);
         for (int u = pair; u < units && ok; u += n_pairs, ++ut) {
-            const int tm = u % g.tiles_m, r = u / g.tiles_m, tn = r % g.tiles_n, sp = r / g.tiles_n;
+            const PairUnit w = decode_pair_unit(g, u);
+            const int tm = w.tm, tn = w.tn;
             const int acc = ut & 1;
             const uint32_t aph = (ut >> 1) & 1u;
             if (!mbar_wait_warp(tfull_bar(acc), aph, g.err, 8)) { ok = false; break; }
@@ -501,8 +539,15 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             float* Dp = g.D;
             long long ldd = g.ldd;
             if (g.splits > 1) {
-                Dp = g.partials + (long long)sp * g.M * g.N;
+                Dp = g.partials + (long long)w.partial * g.M * g.N;
                 ldd = g.N;
+            }
+            // a K range of a tail tile: the raw sums go to the tile's compact partial slot (addressed so
+            // that the global row / column arithmetic below lands inside it); no bias, residual or planes
+            const bool tail_partial = g.tail_splits > 1 && w.partial >= 0;
+            if (tail_partial) {
+                ldd = BN;
+                Dp = g.partials + ((long long)w.partial * (2 * BM) - (long long)tm * (2 * BM)) * BN - (long long)tn * BN;
             }
             const uint32_t t_row = tmem_base + ((uint32_t)(lane_group * 32) << 16) + (uint32_t)acc * C::kAccStride;
             float* my_stage = reinterpret_cast<float*>(smem_raw + (epi_stage - smem_u32(smem_raw)) +
@@ -526,9 +571,9 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                 float4 csum = make_float4(0.f, 0.f, 0.f, 0.f);   // this lane's 8 rows of its 4 columns (act 3 / 4)
                 if (col < g.N) {
                     float4 bv = make_float4(0.f, 0.f, 0.f, 0.f);
-                    if (g.bias) bv = *reinterpret_cast<const float4*>(g.bias + col);
+                    if (g.bias && !tail_partial) bv = *reinterpret_cast<const float4*>(g.bias + col);
                     float4 rv[8];
-                    if (g.residual) {
+                    if (g.residual && !tail_partial) {
 #pragma unroll
                         for (int i = 0; i < 8; ++i) {
                             const int row = row0 + sub + 4 * i;
@@ -553,7 +598,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             if (g.act >= 5) {   // GELU backward: the product times GELU'(h), and its column sums
                                 v = make_float4(v.x * rv[i].x, v.y * rv[i].y, v.z * rv[i].z, v.w * rv[i].w);
                                 csum = add4(csum, v);
-                            } else if (g.residual) {
+                            } else if (g.residual && !tail_partial) {
                                 v = add4(v, rv[i]);
                             }
                             float4 pv = v;      // what the hi/lo planes receive
@@ -567,7 +612,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                                 if (g.act >= 3) v = gp;       // ... and D holds GELU'(output) instead of the output
                             }
                             if (Dp) *reinterpret_cast<float4*>(Dp + (long long)row * ldd + col) = v;
-                            if (g.d_hi) {
+                            if (g.d_hi && !tail_partial) {
                                 float4 hh, ll;
                                 split_tf32(pv, hh, ll);
                                 float* hrow = g.d_hi + (long long)row * g.ldd + col;
@@ -611,6 +656,7 @@ int g_bk = 16;       // k-block depth in use (BT_GEMM_BK=32 selects the 128-byte
 int g_force_bn = 0;  // BT_GEMM_BN=128|192|256 pins the tile width (tuning aid)
 // Measured time of a CTA-pair tile relative to two single-CTA tiles of the same width: 256-wide pair
 // tiles run about 5 % faster (a third less operand data into shared memory), 192-wide ones slower.
+int g_tail_split = 1;   // BT_GEMM_TAIL=0 turns the tail split off (tuning aid)
 double kTwoCtaFactor256 = 0.95, kTwoCtaFactor192 = 1.03;   // BT_GEMM_F256 / BT_GEMM_F192 override (tuning aid)
 int g_two_cta = -1;  // BT_GEMM_2CTA=0 never / 1 always (where the shape allows) / unset: the planner decides
 std::once_flag g_once;
@@ -657,6 +703,7 @@ void init_once() {
     cudaDeviceGetAttribute(&g_num_sms, cudaDevAttrMultiProcessorCount, dev);
     if (const char* v = getenv("BT_GEMM_BK")) g_bk = (atoi(v) == 32) ? 32 : 16;
     if (const char* v = getenv("BT_GEMM_2CTA")) g_two_cta = atoi(v) ? 1 : 0;
+    if (const char* v = getenv("BT_GEMM_TAIL")) g_tail_split = atoi(v) ? 1 : 0;
     if (const char* v = getenv("BT_GEMM_F256")) kTwoCtaFactor256 = atof(v);
     if (const char* v = getenv("BT_GEMM_F192")) kTwoCtaFactor192 = atof(v);
     if (const char* v = getenv("BT_GEMM_BN")) {
@@ -688,10 +735,43 @@ bool encode_map(CUtensorMap* tm, const SplitMat& m, uint32_t box_cols, uint32_t 
 constexpr int kMaxUnitsForSplit = 4 * 148;
 
 
+// The tail split's second pass: out = sum over the K ranges (in range order) of a tail tile's partial
+// tiles, then bias, residual and the hi/lo planes exactly as the GEMM's own epilogue writes them.
+__global__ void __launch_bounds__(256) tail_reduce_kernel(const float* __restrict__ partials, int splits, int tail_tiles,
+                                                          int first_tile, int tiles_m, int bn, int M, int N, float* D,
+                                                          long long ldd, const float* __restrict__ bias,
+                                                          const float* residual, float* d_hi, long long d_plane) {
+    pdl_wait();
+    pdl_trigger();
+    const int bn4 = bn / 4;
+    const long long per_tile4 = 256LL * bn4, total = (long long)tail_tiles * per_tile4;
+    for (long long i = blockIdx.x * (long long)blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+        const int j = (int)(i / per_tile4);
+        const long long r = i - (long long)j * per_tile4;
+        const int lr = (int)(r / bn4), c4 = (int)(r - (long long)lr * bn4);
+        const int tile = first_tile + j, tm = tile % tiles_m, tn = tile / tiles_m;
+        const int row = tm * 256 + lr, col = tn * bn + 4 * c4;
+        if (row >= M || col >= N) continue;
+        float4 t = ld4(partials, (long long)j * per_tile4 + r);
+        for (int sp = 1; sp < splits; ++sp) t = add4(t, ld4(partials, ((long long)sp * tail_tiles + j) * per_tile4 + r));
+        if (bias) t = add4(t, *reinterpret_cast<const float4*>(bias + col));
+        const long long off = (long long)row * ldd + col;
+        if (residual) t = add4(t, *reinterpret_cast<const float4*>(residual + off));
+        if (D) *reinterpret_cast<float4*>(D + off) = t;
+        if (d_hi) {
+            float4 hh, ll;
+            split_tf32(t, hh, ll);
+            *reinterpret_cast<float4*>(d_hi + off) = hh;
+            *reinterpret_cast<float4*>(d_hi + d_plane + off) = ll;
+        }
+    }
+}
+
 struct Plan {
     int bn, splits, kb_per_split;
     double cost;
     bool two_cta;   // 256-row tiles on CTA pairs
+    int tail_tiles, tail_splits, tail_kbps;   // pair tiles only: the last, partly filled round cut along K (0: not used)
 };
 
 // Picks tile width and K-split by a simple wave model.  Every work unit of one launch costs the
@@ -699,12 +779,13 @@ struct Plan {
 // x tile width, narrower tiles pay a small efficiency penalty, and a K-split pays for writing
 // and re-reading its partial sums.
 Plan make_plan(int64_t M, int64_t N, int kb_total, int bk, int sms, bool can_split, size_t max_partial_floats,
-               int two_cta_mode) {   // -1: the planner decides, 0: single-CTA tiles only, 1: pair tiles where M >= 256
+               int two_cta_mode,     // -1: the planner decides, 0: single-CTA tiles only, 1: pair tiles where M >= 256
+               bool can_tail) {      // a tail split may be used (a partial buffer exists, no activation in the epilogue)
     const int tiles_m = (int)((M + BM - 1) / BM);
     const double kOverheadKb = 96.0 / bk;                     // pipeline fill + exposed epilogue, in k-blocks
     const double kb_seconds = 768.0 * (bk / 16.0) / 1.9e9;    // one 128x256 k-block of 3 MMAs at peak
     static const int kSplits[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 20, 24, 32};
-    Plan best{256, 1, kb_total, 1e300, false};
+    Plan best{256, 1, kb_total, 1e300, false, 0, 0, 0};
     for (int two = 0; two < 2; ++two) {
         if (two && (two_cta_mode == 0 || M < 256)) continue;
         if (!two && two_cta_mode == 1 && M >= 256) continue;
@@ -726,7 +807,24 @@ Plan make_plan(int64_t M, int64_t N, int kb_total, int bk, int sms, bool can_spl
                 const long long rounds = (units + slots - 1) / slots;
                 double cost = (double)rounds * (kbps + kOverheadKb) * (bn / 256.0) * pen;
                 if (sp > 1) cost += (double)(sp + 1) * M * N * 4.0 / 6.0e12 / kb_seconds;
-                if (cost < best.cost) best = Plan{bn, sp, kbps, cost, two != 0};
+                if (cost < best.cost) best = Plan{bn, sp, kbps, cost, two != 0, 0, 0, 0};
+            }
+            // Tail split: with few tiles per slot the last round is the expensive one (96 pair tiles on 74
+            // pairs: two rounds for 1.3 rounds of work).  Its tiles are cut into as many K ranges as fill
+            // the idle slots, so the round costs a fraction of a tile's time plus a small reduction pass.
+            const long long full_rounds = tiles / slots, tail = tiles % slots;
+            if (two && can_tail && g_tail_split && full_rounds >= 1 && tail > 0 && 2 * tail <= slots) {
+                int sp = (int)(slots / tail);
+                if (sp > 8) sp = 8;
+                while (sp > 1 && kb_total / sp < 8) --sp;
+                const int kbps = (kb_total + sp - 1) / sp;
+                const int real_sp = (kb_total + kbps - 1) / kbps;
+                const size_t need = (size_t)real_sp * (size_t)tail * 256u * (size_t)bn;
+                if (real_sp > 1 && need <= max_partial_floats) {
+                    double cost = ((double)full_rounds * (kb_total + kOverheadKb) + (kbps + kOverheadKb)) * (bn / 256.0) * pen;
+                    cost += ((double)(real_sp + 2) * tail * 256.0 * bn * 4.0 / 6.0e12 + 3.0e-6) / kb_seconds;   // the reduction pass and its launch
+                    if (cost < best.cost) best = Plan{bn, 1, kb_total, cost, true, (int)tail, real_sp, kbps};
+                }
             }
         }
     }
@@ -763,8 +861,9 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     const int sms = g_num_sms > 0 ? g_num_sms : 148;
     const int kb_total = (int)((K + BK - 1) / BK);
     const bool can_split = !bias && !residual && partials && ldd == N && D && !d_hi;
+    const bool can_tail = partials && act == 0 && (D || d_hi);
     const Plan plan = make_plan(M, N, kb_total, BK, sms, can_split, max_partial_floats,
-                                two_cta_mode >= 0 ? two_cta_mode : g_two_cta);
+                                two_cta_mode >= 0 ? two_cta_mode : g_two_cta, can_tail);
     const int bn = plan.bn;
 
     const CUtensorMapSwizzle sw_k = (BK == 32) ? CU_TENSOR_MAP_SWIZZLE_128B : CU_TENSOR_MAP_SWIZZLE_64B;
@@ -783,9 +882,12 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     g.splits = plan.splits;
     g.kb_per_split = plan.kb_per_split; g.kb_total = kb_total;
     g.partials = partials; g.err = err_word;
+    g.tail_tiles = plan.tail_tiles; g.tail_splits = plan.tail_splits; g.tail_kbps = plan.tail_kbps;
+    g.full_units = g.tiles_m * g.tiles_n - plan.tail_tiles;
     g.d_hi = d_hi; g.d_plane = d_plane; g.act = (d_hi || act >= 5) ? act : 0;
     g.col_partial = act >= 5 ? col_partial : nullptr;
-    const long long units = (long long)g.tiles_m * g.tiles_n * g.splits;
+    const long long units = plan.tail_splits > 1 ? (long long)g.full_units + (long long)plan.tail_tiles * plan.tail_splits
+                                                 : (long long)g.tiles_m * g.tiles_n * g.splits;
     const int grid = (int)(units < sms ? units : sms);
     if (plan.two_cta) {
         const int pairs = (int)(units < sms / 2 ? units : sms / 2);
@@ -805,6 +907,16 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
         cudaError_t e2 = cudaGetLastError();
         if (e2 != cudaSuccess) return e2;
         if (g.splits > 1) return launch_splitk_reduce(partials, g.splits, M * N, D, s);
+        if (g.tail_splits > 1) {
+            const long long n4 = (long long)g.tail_tiles * 256 * (bn / 4);
+            const long long want = (n4 + 255) / 256;
+            const int rgrid = (int)(want < 148 * 16 ? want : 148 * 16);
+            BT_KERNEL_LAUNCH((tail_reduce_kernel), rgrid, 256, 0, s, (const float*)partials, g.tail_splits,
+                             g.tail_tiles, g.full_units, g.tiles_m, bn, g.M, g.N, D, (long long)ldd, bias, residual, d_hi,
+                             (long long)d_plane);
+            BT_COUNT_LAUNCH();
+            return cudaGetLastError();
+        }
         return cudaSuccess;
     }
 
