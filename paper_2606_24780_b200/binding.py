@@ -110,6 +110,7 @@ _SIGNATURES = {
     "bt_op_gemm_gelu_bwd_scratch_bytes": (_sz, [_i64, _i64]),
     "bt_op_gemm_gelu_bwd": (_i32, [_i64, _i64, _i64] + [_vp] * 3 + [_i32] + [_vp] * 3 + [_sz, _u32, _vp]),
     "bt_op_gemm_check": (_i32, [_vp, _vp]),
+    "bt_op_gemm_plan": (_i32, [_i64, _i64, _i64, _i32, _u32, _vp]),
     "bt_op_gemm": (_i32, [_i32, _i64, _i64, _i64] + [_vp] * 6 + [_sz, _u32, _vp]),
     "bt_op_attention_fwd": (_i32, [_vp, _vp, _i32, _i32, _i32, _i32, _vp, _vp, _vp, _u32, _vp]),
     "bt_op_attention_bwd": (_i32, [_vp] * 6 + [_i32] * 4 + [_vp] * 3 + [_sz, _u32, _vp]),
@@ -535,6 +536,13 @@ def bt_op_gemm_gelu_bwd(M, N, K, dy_split, w_split, h, form, dh_split, colsum, s
                         stream=None):
     _check(lib().bt_op_gemm_gelu_bwd(M, N, K, _ptr(dy_split), _ptr(w_split), _ptr(h), int(form), _ptr(dh_split),
                                      _ptr(colsum), _ptr(scratch), scratch_bytes, flags, _stream(stream)))
+
+
+def bt_op_gemm_plan(M, N, K, epilogue=False, flags=0):
+    """The planner's choice for a product: dict with tile width, pair tiles, K splits and the tail split."""
+    out = (ctypes.c_int32 * 6)()
+    _check(lib().bt_op_gemm_plan(M, N, K, int(bool(epilogue)), flags, ctypes.cast(out, ctypes.c_void_p)))
+    return dict(zip(("bn", "pair", "splits", "tail_tiles", "tail_splits", "tail_kbps"), list(out)))
 
 
 def bt_op_gemm_check(scratch, stream=None):

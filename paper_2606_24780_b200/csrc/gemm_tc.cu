@@ -785,6 +785,10 @@ Plan make_plan(int64_t M, int64_t N, int kb_total, int bk, int sms, bool can_spl
     const double kOverheadKb = 96.0 / bk;                     // pipeline fill + exposed epilogue, in k-blocks
     const double kb_seconds = 768.0 * (bk / 16.0) / 1.9e9;    // one 128x256 k-block of 3 MMAs at peak
     static const int kSplits[] = {1, 2, 3, 4, 5, 6, 8, 10, 12, 16, 20, 24, 32};
+    // The tensor core adds into its FP32 accumulator with truncation: a chain of n MMAs can drift by
+    // n 2^-25 of the running sum.  Where a K split is possible, no chain is longer than 8192 MMAs
+    // (K = 21,845: only the input gradient of the LM head, K = 50,304, is affected).
+    const int max_chain_kb = 8192 / (3 * (bk / 8));
     Plan best{256, 1, kb_total, 1e300, false, 0, 0, 0};
     for (int two = 0; two < 2; ++two) {
         if (two && (two_cta_mode == 0 || M < 256)) continue;
@@ -803,6 +807,7 @@ Plan make_plan(int64_t M, int64_t N, int kb_total, int bk, int sms, bool can_spl
                 const int kbps = (kb_total + sp - 1) / sp;
                 const int real_sp = (kb_total + kbps - 1) / kbps;
                 if (real_sp != sp) continue;
+                if (can_split && kbps > max_chain_kb && sp < 32) continue;
                 const long long units = tiles * sp;
                 const long long rounds = (units + slots - 1) / slots;
                 double cost = (double)rounds * (kbps + kOverheadKb) * (bn / 256.0) * pen;
@@ -813,7 +818,8 @@ Plan make_plan(int64_t M, int64_t N, int kb_total, int bk, int sms, bool can_spl
             // pairs: two rounds for 1.3 rounds of work).  Its tiles are cut into as many K ranges as fill
             // the idle slots, so the round costs a fraction of a tile's time plus a small reduction pass.
             const long long full_rounds = tiles / slots, tail = tiles % slots;
-            if (two && can_tail && g_tail_split && full_rounds >= 1 && tail > 0 && 2 * tail <= slots) {
+            if (two && can_tail && g_tail_split && full_rounds >= 1 && tail > 0 && 2 * tail <= slots &&
+                !(can_split && kb_total > max_chain_kb)) {
                 int sp = (int)(slots / tail);
                 if (sp > 8) sp = 8;
                 while (sp > 1 && kb_total / sp < 8) --sp;
@@ -851,6 +857,19 @@ bool gemm_tc_init(char* err, size_t errlen) {
 }
 
 size_t gemm_tc_partial_floats_bound() { return (size_t)kMaxUnitsForSplit * BM * 256; }
+
+// What the planner would choose for a product (host arithmetic only; 148 SMs are assumed where no
+// device has been initialised): out = {tile width, 1 if 256-row pair tiles, K splits, tail tiles,
+// K ranges per tail tile, k-blocks per range}.
+void gemm_tc_plan_info(int64_t M, int64_t N, int64_t K, bool can_split, bool can_tail, int two_cta_mode, int out[6]) {
+    const int sms = g_num_sms > 0 ? g_num_sms : 148;
+    const int kb_total = (int)((K + g_bk - 1) / g_bk);
+    const Plan p = make_plan(M, N, kb_total, g_bk, sms, can_split, gemm_tc_partial_floats_bound(),
+                             two_cta_mode >= 0 ? two_cta_mode : g_two_cta, can_tail);
+    out[0] = p.bn; out[1] = p.two_cta ? 1 : 0; out[2] = p.splits;
+    out[3] = p.tail_tiles; out[4] = p.tail_splits; out[5] = p.tail_kbps;
+}
+
 
 template <int BK>
 static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const SplitMat& A, const SplitMat& B,

@@ -306,6 +306,38 @@ def test_gemm(layout, M, N, K, flags):
         assert rel_max(host(D), ref) < 1e-4
 
 
+@pytest.mark.parametrize("layout,M,N,K", [(1, 4864, 1024, 1024), (0, 4860, 1000, 1028), (2, 4864, 1024, 1040),
+                                          (1, 8192, 768, 3072)])
+def test_gemm_tail_split(layout, M, N, K):
+    """Pair tiles whose last round is cut along K (76 tiles of 256 x 256 for 74 CTA pairs; 96 for the
+    MLP down-projection's shape): the reduction pass adds the K ranges and applies bias, residual and the
+    hi/lo planes; ragged rows, columns and k-blocks included."""
+    flags = b.BT_FLAG_GEMM_PAIR
+    plan = b.bt_op_gemm_plan(M, N, K, True, flags)
+    assert plan["pair"] == 1 and plan["tail_splits"] > 1 and plan["tail_tiles"] > 0, plan
+    a_shape = (K, M) if layout == 2 else (M, K)
+    b_shape = (N, K) if layout == 0 else (K, N)
+    A, Bm = si.normal_f32(170, a_shape), si.normal_f32(171, b_shape, 0.05)
+    bias, res = si.normal_f32(172, (N,)), si.normal_f32(173, (M, N))
+    A64 = A.astype(np.float64).T if layout == 2 else A.astype(np.float64)
+    B64 = Bm.astype(np.float64).T if layout == 0 else Bm.astype(np.float64)
+    As, Bs = empty(2, *a_shape), empty(2, *b_shape)
+    b.bt_op_split(dev(A), A.size, As)
+    b.bt_op_split(dev(Bm), Bm.size, Bs)
+    nb = b.bt_op_gemm_split_scratch_bytes()
+    sc = scratch(nb)
+    for use_epi in (False, True):
+        D, Ds = zeros(M, N), zeros(2, M, N)
+        b.bt_op_gemm_split_act(layout, M, N, K, As, Bs, D, Ds, 0, dev(bias) if use_epi else None,
+                               dev(res) if use_epi else None, sc, nb, flags)
+        b.bt_op_gemm_check(sc)
+        ref = A64 @ B64
+        if use_epi:
+            ref = ref + bias + res
+        assert rel_l2(host(D), ref) < 1e-4 and rel_max(host(D), ref) < 1e-4, (layout, M, N, K, use_epi)
+        check_split(Ds, host(D))
+
+
 def test_gemm_matches_oracle_linear_layer():
     """The three layouts are the forward, input-gradient and weight-gradient of a linear layer."""
     N, cin, cout = 640, 768, 1024

@@ -82,6 +82,24 @@ def test_null_and_misaligned_arguments_are_rejected(lib):
     assert b.bt_op_layernorm_bwd_scratch_bytes(1000, 768) > 0
 
 
+def test_gemm_planner_choices(lib):
+    """bt_op_gemm_plan is host arithmetic.  The projections with 768 output columns and a long K (96 pair
+    tiles for 74 CTA pairs) get a tail split; the same width with K = 768 keeps 192-wide single-CTA tiles;
+    products that fill their rounds are left alone; forcing single-CTA tiles rules the tail split out."""
+    p = b.bt_op_gemm_plan(8192, 768, 3072, True)
+    assert p["pair"] == 1 and p["bn"] == 256 and p["tail_tiles"] == 22 and p["tail_splits"] == 3 and p["tail_kbps"] * 3 >= 3072 // 16
+    p = b.bt_op_gemm_plan(8192, 768, 768, True)
+    assert p["pair"] == 0 and p["bn"] == 192 and p["tail_splits"] == 0
+    p = b.bt_op_gemm_plan(8192, 2304, 768, True)
+    assert p["pair"] == 1 and p["tail_splits"] == 0 and p["splits"] == 1
+    p = b.bt_op_gemm_plan(8192, 768, 3072, True, b.BT_FLAG_GEMM_SINGLE)
+    assert p["pair"] == 0 and p["tail_splits"] == 0
+    p = b.bt_op_gemm_plan(768, 768, 8192, False)          # a weight gradient: few tiles, K split over all of them
+    assert p["splits"] > 1 and p["tail_splits"] == 0
+    with pytest.raises(b.BtError):
+        b.bt_op_gemm_plan(0, 768, 768)
+
+
 def test_host_id_check(lib):
     """bt_first_invalid_id is what bt_train_step_host and the loader run on ids that are still on the
     host: the position of the first id outside [0, vocab), or -1."""
