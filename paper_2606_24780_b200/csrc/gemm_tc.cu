@@ -580,7 +580,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             rv[i] = (row < g.M) ? *reinterpret_cast<const float4*>(g.residual + (long long)row * g.ldd + col)
                                                 : make_float4(0.f, 0.f, 0.f, 0.f);
                         }
-                        if (g.act == 5 || g.act == 6) {   // h -> GELU'(h): 32 independent evaluations, none behind a store
+                        if ((g.act == 5 || g.act == 6) && !tail_partial) {   // h -> GELU'(h): 32 independent evaluations, none behind a store
                             const bool th = g.act == 6;
 #pragma unroll
                             for (int i = 0; i < 8; ++i)
@@ -595,14 +595,14 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                             float4 v = *reinterpret_cast<const float4*>(reinterpret_cast<const uint8_t*>(my_stage) +
                                                                         rr_ * kEpiPitch + cq * 16);
                             v = add4(v, bv);
-                            if (g.act >= 5) {   // GELU backward: the product times GELU'(h), and its column sums
+                            if (g.act >= 5 && !tail_partial) {   // GELU backward: the product times GELU'(h), and its column sums
                                 v = make_float4(v.x * rv[i].x, v.y * rv[i].y, v.z * rv[i].z, v.w * rv[i].w);
                                 csum = add4(csum, v);
                             } else if (g.residual && !tail_partial) {
                                 v = add4(v, rv[i]);
                             }
                             float4 pv = v;      // what the hi/lo planes receive
-                            if (g.act >= 1 && g.act <= 4) {   // GELU forward: the planes hold GELU(output) ...
+                            if (g.act >= 1 && g.act <= 4 && !tail_partial) {   // GELU forward: the planes hold GELU(output) ...
                                 const bool th = !(g.act & 1);
                                 float4 gp;
                                 gelu_both_f(v.x, th, pv.x, gp.x);
@@ -622,7 +622,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
                         }
                     }
                 }
-                if (g.act >= 5 && g.col_partial) {   // warp-uniform: the 32 rows of this warp, rows sub + 4 i in lane order
+                if (g.act >= 5 && g.col_partial && !tail_partial) {   // warp-uniform: the 32 rows of this warp, rows sub + 4 i in lane order
                     csum.x += __shfl_xor_sync(0xffffffffu, csum.x, 8);  csum.y += __shfl_xor_sync(0xffffffffu, csum.y, 8);
                     csum.z += __shfl_xor_sync(0xffffffffu, csum.z, 8);  csum.w += __shfl_xor_sync(0xffffffffu, csum.w, 8);
                     csum.x += __shfl_xor_sync(0xffffffffu, csum.x, 16); csum.y += __shfl_xor_sync(0xffffffffu, csum.y, 16);
@@ -736,11 +736,12 @@ constexpr int kMaxUnitsForSplit = 4 * 148;
 
 
 // The tail split's second pass: out = sum over the K ranges (in range order) of a tail tile's partial
-// tiles, then bias, residual and the hi/lo planes exactly as the GEMM's own epilogue writes them.
+// tiles, then the output path exactly as the GEMM's own epilogue runs it: bias, residual, the GELU
+// forward modes (act 1 - 4) and the hi/lo planes.
 __global__ void __launch_bounds__(256) tail_reduce_kernel(const float* __restrict__ partials, int splits, int tail_tiles,
                                                           int first_tile, int tiles_m, int bn, int M, int N, float* D,
                                                           long long ldd, const float* __restrict__ bias,
-                                                          const float* residual, float* d_hi, long long d_plane) {
+                                                          const float* residual, float* d_hi, long long d_plane, int act) {
     pdl_wait();
     pdl_trigger();
     const int bn4 = bn / 4;
@@ -757,10 +758,20 @@ __global__ void __launch_bounds__(256) tail_reduce_kernel(const float* __restric
         if (bias) t = add4(t, *reinterpret_cast<const float4*>(bias + col));
         const long long off = (long long)row * ldd + col;
         if (residual) t = add4(t, *reinterpret_cast<const float4*>(residual + off));
+        float4 pv = t;
+        if (act >= 1 && act <= 4) {
+            const bool th = !(act & 1);
+            float4 gp;
+            gelu_both_f(t.x, th, pv.x, gp.x);
+            gelu_both_f(t.y, th, pv.y, gp.y);
+            gelu_both_f(t.z, th, pv.z, gp.z);
+            gelu_both_f(t.w, th, pv.w, gp.w);
+            if (act >= 3) t = gp;
+        }
         if (D) *reinterpret_cast<float4*>(D + off) = t;
         if (d_hi) {
             float4 hh, ll;
-            split_tf32(t, hh, ll);
+            split_tf32(pv, hh, ll);
             *reinterpret_cast<float4*>(d_hi + off) = hh;
             *reinterpret_cast<float4*>(d_hi + d_plane + off) = ll;
         }
@@ -880,7 +891,9 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     const int sms = g_num_sms > 0 ? g_num_sms : 148;
     const int kb_total = (int)((K + BK - 1) / BK);
     const bool can_split = !bias && !residual && partials && ldd == N && D && !d_hi;
-    const bool can_tail = partials && act == 0 && (D || d_hi);
+    // (the GELU backward modes are left out: a reduction pass that also forms their column sums -- 32 rows
+    // per thread -- was measured slower than the second round it replaces)
+    const bool can_tail = partials && (D || d_hi) && act < 5;
     const Plan plan = make_plan(M, N, kb_total, BK, sms, can_split, max_partial_floats,
                                 two_cta_mode >= 0 ? two_cta_mode : g_two_cta, can_tail);
     const int bn = plan.bn;
@@ -930,9 +943,9 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
             const long long n4 = (long long)g.tail_tiles * 256 * (bn / 4);
             const long long want = (n4 + 255) / 256;
             const int rgrid = (int)(want < 148 * 16 ? want : 148 * 16);
-            BT_KERNEL_LAUNCH((tail_reduce_kernel), rgrid, 256, 0, s, (const float*)partials, g.tail_splits,
-                             g.tail_tiles, g.full_units, g.tiles_m, bn, g.M, g.N, D, (long long)ldd, bias, residual, d_hi,
-                             (long long)d_plane);
+            BT_KERNEL_LAUNCH((tail_reduce_kernel), rgrid, 256, 0, s, (const float*)partials, g.tail_splits, g.tail_tiles,
+                             g.full_units, g.tiles_m, bn, g.M, g.N, D, (long long)ldd, bias, residual, d_hi,
+                             (long long)d_plane, g.act);
             BT_COUNT_LAUNCH();
             return cudaGetLastError();
         }

@@ -338,6 +338,29 @@ def test_gemm_tail_split(layout, M, N, K):
         check_split(Ds, host(D))
 
 
+@pytest.mark.parametrize("act", [1, 4])
+def test_gemm_tail_split_with_gelu_epilogue(act):
+    """The forward GELU modes through the tail split: the reduction pass evaluates GELU (planes) and, in
+    modes 3 / 4, GELU' (D) for the tiles of the last round."""
+    M, N, K, flags = 4864, 1024, 1024, b.BT_FLAG_GEMM_PAIR
+    assert b.bt_op_gemm_plan(M, N, K, True, flags)["tail_splits"] > 1
+    x, w, bias = si.normal_f32(174, (M, K)), si.normal_f32(175, (K, N), 0.05), si.normal_f32(176, (N,), 0.5)
+    xs, ws = empty(2, M, K), empty(2, K, N)
+    b.bt_op_split(dev(x), M * K, xs)
+    b.bt_op_split(dev(w), K * N, ws)
+    D, Ds = empty(M, N), empty(2, M, N)
+    nb = b.bt_op_gemm_split_scratch_bytes()
+    sc = scratch(nb)
+    b.bt_op_gemm_split_act(1, M, N, K, xs, ws, D, Ds, act, dev(bias), None, sc, nb, flags)
+    b.bt_op_gemm_check(sc)
+    rh = x.astype(np.float64) @ w.astype(np.float64) + bias
+    tanh_form = act in (2, 4)
+    got = host(Ds)
+    assert rel_l2(got[0].astype(np.float64) + got[1], oracle.gelu_fwd(rh.ravel(), tanh_form).reshape(M, N)) < 1e-4
+    want_d = rh if act <= 2 else oracle.gelu_bwd(rh.ravel(), np.ones(rh.size), tanh_form).reshape(M, N)
+    assert rel_l2(host(D), want_d) < 1e-4
+
+
 def test_gemm_matches_oracle_linear_layer():
     """The three layouts are the forward, input-gradient and weight-gradient of a linear layer."""
     N, cin, cout = 640, 768, 1024
@@ -483,7 +506,8 @@ def test_gemm_epilogue_activation_planes(act, flags):
 
 
 _GELU_BWD_CASES = [(M, N, K, t, f) for (M, N, K) in [(520, 768, 256), (8, 32, 4), (1000, 352, 132)] for t in (0, 1)
-                   for f in (0, b.BT_FLAG_GEMM_SINGLE, b.BT_FLAG_GEMM_PAIR)] + [(4096, 3072, 768, 0, 0)]
+                   for f in (0, b.BT_FLAG_GEMM_SINGLE, b.BT_FLAG_GEMM_PAIR)] + [(4096, 3072, 768, 0, 0)] + \
+                  [(4864, 1024, 1024, t, b.BT_FLAG_GEMM_PAIR) for t in (0, 1)]   # 76 pair tiles: two rounds
 
 
 @pytest.mark.parametrize("M,N,K,tanh_form,flags", _GELU_BWD_CASES)
