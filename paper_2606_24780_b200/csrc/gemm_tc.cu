@@ -386,20 +386,26 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
 // ring gets deeper (32 KB stages instead of 48 KB).  The even CTA (leader) issues the MMAs and
 // owns the "stage full" and "accumulator drained" barriers; completion is broadcast to both CTAs'
 // "stage free" / "accumulator full" barriers by the commit.
+// The pair kernel has eight epilogue warps (two per tensor-memory lane quadrant, alternate 32-column
+// chunks): its main loop is math bound with stages to spare, so the staging tiles of four more warps
+// cost it nothing, while the epilogue of a CTA's last tile -- which nothing overlaps -- halves.
+constexpr int kEpiWarps2 = 8;
+constexpr int kThreads2 = 64 + 32 * kEpiWarps2;
+constexpr uint32_t kEpiStageBytes2 = kEpiWarps2 * 32u * kEpiPitch;
 template <int BN, int BK>
 struct Cfg2 {
     static constexpr uint32_t kATileBytes = 2u * BM * BK * 4u;          // this CTA's 128 rows, hi + lo
     static constexpr uint32_t kBTileBytes = 2u * (BN / 2) * BK * 4u;    // this CTA's half of the columns
     static constexpr uint32_t kStageBytes = kATileBytes + kBTileBytes;
-    static constexpr int kStagesFit = (int)((kSmemBudget - 2048u - kEpiStageBytes) / kStageBytes);
+    static constexpr int kStagesFit = (int)((kSmemBudget - 2048u - kEpiStageBytes2) / kStageBytes);
     static constexpr int kStages = kStagesFit > 8 ? 8 : kStagesFit;
     static constexpr uint32_t kAccStride = 256u;
     static constexpr uint32_t kTmemCols = 512u;
-    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + kEpiStageBytes + 256;
+    static constexpr size_t kSmemBytes = 1024 + (size_t)kStages * kStageBytes + kEpiStageBytes2 + 256;
 };
 
 template <bool A_MN, bool B_MN, int BN, int BK>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads2, 1)
 gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB, const GemmArgs g) {
     using C = Cfg2<BN, BK>;
     constexpr int BH = BN / 2;                         // B columns held by one CTA
@@ -407,7 +413,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const uint32_t epi_stage = smem_base + C::kStages * C::kStageBytes;
-    const uint32_t bars = epi_stage + kEpiStageBytes;
+    const uint32_t bars = epi_stage + kEpiStageBytes2;
     auto full_bar = [&](int s) { return bars + 8u * s; };
     auto empty_bar = [&](int s) { return bars + 8u * (C::kStages + s); };
     auto tfull_bar = [&](int a) { return bars + 8u * (2 * C::kStages + a); };
@@ -429,7 +435,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
         }
         for (int a = 0; a < 2; ++a) {
             mbar_init(tfull_bar(a), 1);
-            mbar_init(tempty_bar(a), 2 * kEpiWarps);   // used in the leader: both CTAs' epilogue warps
+            mbar_init(tempty_bar(a), 2 * kEpiWarps2);   // used in the leader: both CTAs' epilogue warps
         }
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -555,7 +561,7 @@ gemm_tc2_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__
             const int sub = lane >> 3, cq = lane & 7;
             const int row0 = tm * 2 * BM + (int)rank * BM + lane_group * 32;
 #pragma unroll 1
-            for (int c = 0; c < BN / 32; ++c) {
+            for (int c = (warp - 2) >> 2; c < BN / 32; c += 2) {   // the quadrant's two warps take alternate chunks
                 const int col0 = tn * BN + c * 32;
                 if (col0 >= g.N) break;  // warp-uniform
                 uint32_t rr[32];
@@ -924,7 +930,7 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     if (plan.two_cta) {
         const int pairs = (int)(units < sms / 2 ? units : sms / 2);
 #define BT_LAUNCH2(AM, BMN, BNV)                                                                             \
-    BT_KERNEL_LAUNCH((gemm_tc2_kernel<AM, BMN, BNV, BK>), 2 * pairs, kThreads, (Cfg2<BNV, BK>::kSmemBytes), s, tmA, tmB, g)
+    BT_KERNEL_LAUNCH((gemm_tc2_kernel<AM, BMN, BNV, BK>), 2 * pairs, kThreads2, (Cfg2<BNV, BK>::kSmemBytes), s, tmA, tmB, g)
 #define BT_LAUNCH2_BN(BNV)                                                                                   \
     do {                                                                                                     \
         if (layout == kNT) BT_LAUNCH2(false, false, BNV);                                                    \
