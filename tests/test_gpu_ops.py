@@ -361,6 +361,41 @@ def test_gemm_tail_split_with_gelu_epilogue(act):
     assert rel_l2(host(D), want_d) < 1e-4
 
 
+def _planner_sweep_shapes():
+    """Seeded shapes whose tile counts land on every side of the planner's choices: fewer tiles than
+    slots (K splits), one full round plus a small tail (tail split), several rounds, ragged edges."""
+    rng = np.random.RandomState(20240607)
+    shapes = []
+    for _ in range(14):
+        layout = int(rng.randint(0, 3))
+        M = int(rng.choice([256, 1280, 4864, 9472, 12800, 19200])) - 4 * int(rng.randint(0, 3)) * (layout != 2)
+        N = int(rng.choice([128, 768, 1024, 1536, 2304])) - 4 * int(rng.randint(0, 3)) * (layout == 0)
+        K = int(rng.choice([256, 768, 1024, 2304, 3072])) + 4 * int(rng.randint(0, 3))
+        shapes.append((layout, M, N, K))
+    return shapes
+
+
+@pytest.mark.parametrize("layout,M,N,K", _planner_sweep_shapes())
+def test_gemm_planner_sweep(layout, M, N, K):
+    """Whatever the planner picks for a shape (tile width, pair tiles, K split, tail split), the product
+    with bias and residual matches the FP64 product; the plan itself is reported on failure."""
+    plan = b.bt_op_gemm_plan(M, N, K, True)
+    a_shape = (K, M) if layout == 2 else (M, K)
+    b_shape = (N, K) if layout == 0 else (K, N)
+    A, Bm = si.normal_f32(180, a_shape), si.normal_f32(181, b_shape, 0.05)
+    bias, res = si.normal_f32(182, (N,)), si.normal_f32(183, (M, N))
+    A64 = A.astype(np.float64).T if layout == 2 else A.astype(np.float64)
+    B64 = Bm.astype(np.float64).T if layout == 0 else Bm.astype(np.float64)
+    nb = b.bt_op_gemm_scratch_bytes(layout, M, N, K)
+    sc = scratch(nb)
+    for use_epi in (True, False):
+        D = zeros(M, N)
+        b.bt_op_gemm(layout, M, N, K, dev(A), dev(Bm), D, dev(bias) if use_epi else None, dev(res) if use_epi else None,
+                     sc, nb, 0)
+        ref = A64 @ B64 + ((bias + res) if use_epi else 0.0)
+        assert rel_l2(host(D), ref) < 1e-4 and rel_max(host(D), ref) < 1e-4, (layout, M, N, K, use_epi, plan)
+
+
 def test_gemm_matches_oracle_linear_layer():
     """The three layouts are the forward, input-gradient and weight-gradient of a linear layer."""
     N, cin, cout = 640, 768, 1024
