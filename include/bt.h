@@ -537,7 +537,9 @@ BT_API bt_status bt_op_gelu_bwd_colsum(const float* x, const float* dy, int64_t 
  * target"): losses[n] = logsumexp(logits[n,:]) - logits[n, y_n]; dlogits = (softmax - onehot) *
  * inv_count; loss_mean (1 float) = inv_count * sum_n losses[n] in fixed order.  Vp % 4 == 0.
  * A target outside [0, Vp) counts as class 0 and its row + 1 is stored in *d_bad (device int32,
- * nullable, zeroed by the caller; first writer wins). */
+ * nullable, zeroed by the caller; first writer wins).  dlogits (raw) and dlogits_split (hi plane,
+ * then lo plane, N * Vp floats each) are both optional; for Vp <= 51,200 (rows held in registers)
+ * logits may be the hi plane of dlogits_split itself: the gradient then overwrites the logits. */
 BT_API bt_status bt_op_softmax_xent(const float* logits, const int32_t* targets, int64_t N, int32_t Vp,
                                     float inv_count, float* losses, float* loss_mean, float* dlogits,
                                     float* dlogits_split, int32_t* d_bad, void* stream);

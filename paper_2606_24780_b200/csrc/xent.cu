@@ -89,6 +89,92 @@ __global__ void __launch_bounds__(kXentThreads) xent_kernel(const float* logits,
     }
 }
 
+// The same row arithmetic for long rows and many more rows than SMs, as a row loop: one CTA per SM
+// keeps the NEXT row on its way into shared memory (16-byte asynchronous copies, each thread copying
+// exactly the elements it will read, so that completion needs no barrier) while the current row, held
+// in registers, is reduced and its gradient stored.  With the grid-per-row kernel an SM alternates
+// between a load phase, an arithmetic phase and a store phase (the row fills the register file, so a
+// second CTA cannot be resident); here the loads of row r + 1 run under the arithmetic and the
+// stores of row r.  Element-to-thread assignment and reduction order are those of xent_kernel, so the
+// results are bit-identical.
+__device__ __forceinline__ void cp_async16(float4* dst_smem, const float4* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(dst_smem)), "l"(src)
+                 : "memory");
+}
+
+template <int ITEMS>
+__global__ void __launch_bounds__(kXentThreads) xent_stream_kernel(const float* logits,   // may alias dl_hi (in place)
+                                                                   const int32_t* __restrict__ targets, int V4,
+                                                                   float inv_count, float* __restrict__ losses,
+                                                                   float* dl, float* dl_hi, float* dl_lo, int V, int* bad,
+                                                                   int64_t N) {
+    extern __shared__ float4 row_s[];
+    __shared__ float sm[kXentThreads / 32];
+    pdl_wait();
+    pdl_trigger();
+    auto fetch = [&](int64_t r) {
+        const float4* src = reinterpret_cast<const float4*>(logits) + r * V4;
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k) {
+            int idx = threadIdx.x + kXentThreads * k;
+            if (idx < V4) cp_async16(row_s + idx, src + idx);
+        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
+    };
+    if ((int64_t)blockIdx.x < N) fetch(blockIdx.x);
+    for (int64_t row = blockIdx.x; row < N; row += gridDim.x) {
+        const int64_t base = row * V4;
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        float4 v[ITEMS];
+        float mx = -INFINITY;
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k) {
+            int idx = threadIdx.x + kXentThreads * k;
+            if (idx < V4) {
+                v[k] = row_s[idx];
+                mx = fmaxf(mx, fmaxf(fmaxf(v[k].x, v[k].y), fmaxf(v[k].z, v[k].w)));
+            }
+        }
+        // this thread's part of the row is in registers (the maximum has consumed it): its shared-memory
+        // slots may take the next row
+        if (row + gridDim.x < N) fetch(row + gridDim.x);
+        mx = block_reduce(mx, true, sm);
+        float sum = 0.f;
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k) {
+            int idx = threadIdx.x + kXentThreads * k;
+            if (idx < V4) {
+                v[k].x = expf(v[k].x - mx);
+                v[k].y = expf(v[k].y - mx);
+                v[k].z = expf(v[k].z - mx);
+                v[k].w = expf(v[k].w - mx);
+                sum += (v[k].x + v[k].y) + (v[k].z + v[k].w);
+            }
+        }
+        sum = block_reduce(sum, false, sm);
+        const int t = checked_target(targets[row], V, row, bad);
+        if (threadIdx.x == 0) losses[row] = (mx + logf(sum)) - logits[row * V4 * 4 + t];
+        if (dl == nullptr && dl_hi == nullptr) continue;
+        __syncthreads();   // in place: the target's logit has been read before anyone stores
+        const float sc = inv_count / sum;
+#pragma unroll
+        for (int k = 0; k < ITEMS; ++k) {
+            int idx = threadIdx.x + kXentThreads * k;
+            if (idx < V4) {
+                float4 r = make_float4(v[k].x * sc, v[k].y * sc, v[k].z * sc, v[k].w * sc);
+                if ((t >> 2) == idx) {
+                    int j = t & 3;
+                    if (j == 0) r.x -= inv_count;
+                    else if (j == 1) r.y -= inv_count;
+                    else if (j == 2) r.z -= inv_count;
+                    else r.w -= inv_count;
+                }
+                store_raw_split(r, dl, dl_hi, dl_lo, base + idx);
+            }
+        }
+    }
+}
+
 // Rows longer than the register path covers: three passes over global memory (the second and
 // third are served by L2 for rows of a few hundred KB).
 __global__ void __launch_bounds__(kXentThreads) xent_generic_kernel(const float* __restrict__ logits,
@@ -148,6 +234,12 @@ __global__ void __launch_bounds__(1024) loss_mean_kernel(const float* __restrict
     if (threadIdx.x == 0) *loss_mean = (float)(sm[0] * (double)inv_count);
 }
 
+// BT_XENT_STREAM=0 keeps long rows on the grid-per-row kernel (for comparison runs).
+static const bool g_xent_stream = []() {
+    const char* v = getenv("BT_XENT_STREAM");
+    return !(v && v[0] == '0');
+}();
+
 // Rows up to this many columns take the one-pass kernel, which may write its output over its input.
 int softmax_xent_max_in_place_columns() { return 25 * kXentThreads * 4; }
 
@@ -163,7 +255,21 @@ cudaError_t launch_softmax_xent(const float* logits, const int32_t* targets, int
     else if (items <= 4) BT_XENT(4);
     else if (items <= 8) BT_XENT(8);
     else if (items <= 16) BT_XENT(16);
-    else if (items <= 25) BT_XENT(25);
+    else if (items <= 25) {
+        int dev = 0, sms = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const size_t row_bytes = (size_t)V4 * sizeof(float4);
+        if (g_xent_stream && N >= 4 * (int64_t)sms && row_bytes <= 220 * 1024) {
+            // set per call: the attribute is kept per device, and this runs once per step
+            cudaError_t e = cudaFuncSetAttribute(xent_stream_kernel<25>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+            if (e != cudaSuccess) return e;
+            BT_KERNEL_LAUNCH((xent_stream_kernel<25>), sms, kXentThreads, row_bytes, s, logits, targets, V4, inv_count, losses,
+                             dl, dl_hi, dl_lo, V, bad, N);
+        } else {
+            BT_XENT(25);
+        }
+    }
     else BT_KERNEL_LAUNCH((xent_generic_kernel), (int)N, kXentThreads, 0, s, logits, targets, V4, inv_count, losses, dl, dl_hi, dl_lo, V, bad);
 #undef BT_XENT
     BT_COUNT_LAUNCH();

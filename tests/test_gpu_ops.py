@@ -221,6 +221,38 @@ def test_softmax_xent(N, Vp):
     check_split(dls, host(dl))
 
 
+@pytest.mark.parametrize("N,Vp", [(640, 50304), (1201, 33000)])
+def test_softmax_xent_row_loop_kernel(N, Vp):
+    """Long rows with at least four rows per SM run as a row loop that fetches the next row while the
+    current one is reduced and stored.  Checked against the oracle, bit for bit against the
+    grid-per-row kernel (which the same rows take when handed over in pieces of fewer rows), and in
+    place (the gradient's hi plane written over the logits)."""
+    z = si.normal_f32(26, (N, Vp), 3.0)
+    z[1, 3] = 80.0
+    y = si.uniform_tokens(27, 1, N, Vp)[0].ravel()
+    inv = 1.0 / N
+    losses, lm, dl, dls = empty(N), empty(1), empty(N, Vp), empty(2, N, Vp)
+    b.bt_op_softmax_xent(dev(z), dev(y), N, Vp, inv, losses, lm, dl, dls)
+    rl, rdl = oracle.softmax_xent(z, y, inv)
+    assert rel_l2(host(losses), rl) < 1e-5 and np.abs(host(losses) - rl).max() < 1e-4
+    assert rel_l2(host(dl), rdl) < 1e-5
+    check_split(dls, host(dl))
+    # the same rows in pieces small enough for the grid-per-row kernel
+    zd, yd = dev(z), dev(y)
+    losses2, dl2 = empty(N), empty(N, Vp)
+    step = 300
+    for r0 in range(0, N, step):
+        n = min(step, N - r0)
+        b.bt_op_softmax_xent(zd[r0:r0 + n], yd[r0:r0 + n], n, Vp, inv, losses2[r0:r0 + n], None, dl2[r0:r0 + n], None)
+    assert np.array_equal(host(losses2), host(losses)) and np.array_equal(host(dl2), host(dl))
+    # in place: the hi plane of the gradient over the logits
+    buf = empty(2, N, Vp)
+    buf[0].copy_(zd)
+    losses3 = empty(N)
+    b.bt_op_softmax_xent(buf[0], yd, N, Vp, inv, losses3, None, None, buf)
+    assert np.array_equal(host(losses3), host(losses)) and np.array_equal(host(buf), host(dls))
+
+
 # ------------------------------------------------------------------ reductions
 
 @pytest.mark.parametrize("N,C", [(256, 64), (8192, 768), (1000, 3072), (33, 2304)])
