@@ -461,11 +461,14 @@ BT_API bt_status bt_op_gemm_split_act(int32_t layout, int64_t M, int64_t N, int6
 BT_API bt_status bt_op_gemm_check(const void* scratch, void* stream);
 /* What the wave-model planner chooses for a product of these sizes (host arithmetic, no launch; the
  * "Native GEMM Library" passage: tiles "tuned for highly irregular, low-parallelism gradient shapes").
- * epilogue != 0: a bias or residual is applied, which rules out a K split of all tiles.  out6 (host) =
+ * epilogue != 0: a bias or residual is applied, which rules out a K split of all tiles.  out7 (host) =
  * {tile width, 1 if 256-row tiles on CTA pairs, K splits over all tiles, tail tiles, K ranges per
- * tail tile, k-blocks per range}.  A tail split (entries 3-5 non-zero) cuts only the tiles of the last,
- * partly filled round along K and adds a small reduction pass. */
-BT_API bt_status bt_op_gemm_plan(int64_t M, int64_t N, int64_t K, int32_t epilogue, uint32_t flags, int32_t* out6);
+ * tail tile, k-blocks per range, group height of the tile raster}.  A tail split (entries 3-5 non-zero)
+ * cuts only the tiles of the last, partly filled round along K and adds a small reduction pass.  The
+ * raster walks groups of `group height` row tiles, inside a group row tiles fastest, then column tiles:
+ * the tiles in flight at one time share their A and B tiles through L2, and the height is chosen so that
+ * an operand larger than L2 is not fetched from HBM once per tile column (or row). */
+BT_API bt_status bt_op_gemm_plan(int64_t M, int64_t N, int64_t K, int32_t epilogue, uint32_t flags, int32_t* out7);
 /* The input-gradient product of the MLP down-projection with the GELU backward in its epilogue
  * (Kernel Design, fused element-wise epilogues; Appendix B "GELU Backward"): with dy_split
  * [2][M][K] (hi/lo planes of the gradient at the projection's output), w_split [2][K][N] (the

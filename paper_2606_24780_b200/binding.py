@@ -539,10 +539,11 @@ def bt_op_gemm_gelu_bwd(M, N, K, dy_split, w_split, h, form, dh_split, colsum, s
 
 
 def bt_op_gemm_plan(M, N, K, epilogue=False, flags=0):
-    """The planner's choice for a product: dict with tile width, pair tiles, K splits and the tail split."""
-    out = (ctypes.c_int32 * 6)()
+    """The planner's choice for a product: dict with tile width, pair tiles, K splits, the tail split and the
+    group height of the tile raster."""
+    out = (ctypes.c_int32 * 7)()
     _check(lib().bt_op_gemm_plan(M, N, K, int(bool(epilogue)), flags, ctypes.cast(out, ctypes.c_void_p)))
-    return dict(zip(("bn", "pair", "splits", "tail_tiles", "tail_splits", "tail_kbps"), list(out)))
+    return dict(zip(("bn", "pair", "splits", "tail_tiles", "tail_splits", "tail_kbps", "group_m"), list(out)))
 
 
 def bt_op_gemm_check(scratch, stream=None):

@@ -1337,13 +1337,13 @@ extern "C" bt_status bt_op_gemm_gelu_bwd(int64_t M, int64_t N, int64_t K, const 
     return BT_OK;
 }
 
-extern "C" bt_status bt_op_gemm_plan(int64_t M, int64_t N, int64_t K, int32_t epilogue, uint32_t flags, int32_t* out6) {
-    if (!out6) return fail(BT_ERR_INVALID_ARG, "gemm_plan: NULL argument");
+extern "C" bt_status bt_op_gemm_plan(int64_t M, int64_t N, int64_t K, int32_t epilogue, uint32_t flags, int32_t* out7) {
+    if (!out7) return fail(BT_ERR_INVALID_ARG, "gemm_plan: NULL argument");
     if (M < 1 || N < 1 || K < 1) return fail(BT_ERR_INVALID_ARG, "gemm_plan: bad sizes");
     const int two_cta_mode = (flags & BT_FLAG_GEMM_PAIR) ? 1 : (flags & BT_FLAG_GEMM_SINGLE) ? 0 : -1;
-    int out[6];
+    int out[7];
     gemm_tc_plan_info(M, N, K, /*can_split=*/!epilogue, /*can_tail=*/true, two_cta_mode, out);
-    for (int i = 0; i < 6; ++i) out6[i] = out[i];
+    for (int i = 0; i < 7; ++i) out7[i] = out[i];
     return BT_OK;
 }
 

@@ -70,6 +70,11 @@ struct GemmArgs {
     const float* bias;
     const float* residual;
     int tiles_m, tiles_n, splits, kb_per_split, kb_total;
+    // Raster of the tiles: groups of group_m row tiles; inside a group the row tiles run fastest, then the
+    // column tiles, then the next group.  The units that run at the same time then cover group_m row tiles
+    // by (slots / group_m) column tiles: each A and B tile among them is fetched from HBM once and served
+    // from L2 to the other CTAs.  group_m >= tiles_m is the plain row-fastest order, 1 column-fastest.
+    int group_m;
     float* partials;
     // Tail split (pair kernel, splits == 1): the tiles of the complete rounds run with the whole K; the
     // tail_tiles tiles of the last, partly filled round are cut into tail_splits K ranges, so that this
@@ -85,6 +90,21 @@ struct GemmArgs {
                         // 7: `residual` holds GELU'(h) itself and the output is (A B) o residual
     float* col_partial; // act 5 - 7: column sums of the output per 32-row group, [ceil(M / 32)][N] (nullable)
 };
+
+// Tile and K range of work unit u (K-split launches: all tiles' first range, then all second ranges, ...).
+__host__ __device__ __forceinline__ void raster_tile(int t, int tiles_m, int tiles_n, int group_m, int& tm, int& tn) {
+    const int per_group = group_m * tiles_n;
+    const int grp = t / per_group, rem = t - grp * per_group;
+    const int first = grp * group_m;
+    const int rows = min(group_m, tiles_m - first);   // the last group may be shorter
+    tn = rem / rows;
+    tm = first + (rem - tn * rows);
+}
+__device__ __forceinline__ void decode_unit(const GemmArgs& g, int u, int& tm, int& tn, int& sp) {
+    const int tiles = g.tiles_m * g.tiles_n;
+    sp = u / tiles;
+    raster_tile(u - sp * tiles, g.tiles_m, g.tiles_n, g.group_m, tm, tn);
+}
 
 // One work unit of the pair kernel: its tile, its k-block range and, for a partial result, the slot of
 // its partial tile (-1: the unit produces the output itself).
@@ -106,13 +126,12 @@ __device__ __forceinline__ PairUnit decode_pair_unit(const GemmArgs& g, int u) {
             w.kb1 = min(g.kb_total, w.kb0 + g.tail_kbps);
             w.partial = sp * g.tail_tiles + v % g.tail_tiles;
         }
-        w.tm = tile % g.tiles_m;
-        w.tn = tile / g.tiles_m;
+        int sp_unused;
+        decode_unit(g, tile, w.tm, w.tn, sp_unused);
         return w;
     }
-    const int r = u / g.tiles_m, sp = r / g.tiles_n;
-    w.tm = u % g.tiles_m;
-    w.tn = r % g.tiles_n;
+    int sp;
+    decode_unit(g, u, w.tm, w.tn, sp);
     w.kb0 = sp * g.kb_per_split;
     w.kb1 = min(g.kb_total, w.kb0 + g.kb_per_split);
     w.partial = g.splits > 1 ? sp : -1;
@@ -191,7 +210,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t it = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < units && ok; u += gridDim.x) {
-                const int tm = u % g.tiles_m, r = u / g.tiles_m, tn = r % g.tiles_n, sp = r / g.tiles_n;
+                int tm, tn, sp;
+                decode_unit(g, u, tm, tn, sp);
                 const int kb0 = sp * g.kb_per_split;
                 const int kb1 = min(g.kb_total, kb0 + g.kb_per_split);
                 for (int kb = kb0; kb < kb1; ++kb, ++it) {
@@ -229,7 +249,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
             uint32_t it = 0, ut = 0;
             bool ok = true;
             for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++ut) {
-                const int r = u / g.tiles_m, sp = r / g.tiles_n;
+                int tm, tn, sp;
+                decode_unit(g, u, tm, tn, sp);
                 const int kb0 = sp * g.kb_per_split;
                 const int kb1 = min(g.kb_total, kb0 + g.kb_per_split);
                 const int acc = ut & 1;
@@ -265,7 +286,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ 
         uint32_t ut = 0;
         bool ok = true;
         for (int u = blockIdx.x; u < units && ok; u += gridDim.x, ++ut) {
-            const int tm = u % g.tiles_m, r = u / g.tiles_m, tn = r % g.tiles_n, sp = r / g.tiles_n;
+            int tm, tn, sp;
+            decode_unit(g, u, tm, tn, sp);
             const int acc = ut & 1;
             const uint32_t aph = (ut >> 1) & 1u;
             if (!mbar_wait_warp(tfull_bar(acc), aph, g.err, 4)) { ok = false; break; }
@@ -662,6 +684,7 @@ int g_bk = 16;       // k-block depth in use (BT_GEMM_BK=32 selects the 128-byte
 int g_force_bn = 0;  // BT_GEMM_BN=128|192|256 pins the tile width (tuning aid)
 // Measured time of a CTA-pair tile relative to two single-CTA tiles of the same width: 256-wide pair
 // tiles run about 5 % faster (a third less operand data into shared memory), 192-wide ones slower.
+int g_group_m = 0;      // BT_GEMM_GROUPM=n pins the raster's group height (tuning aid); 0: chosen per GEMM
 int g_tail_split = 1;   // BT_GEMM_TAIL=0 turns the tail split off (tuning aid)
 double kTwoCtaFactor256 = 0.95, kTwoCtaFactor192 = 1.03;   // BT_GEMM_F256 / BT_GEMM_F192 override (tuning aid)
 int g_two_cta = -1;  // BT_GEMM_2CTA=0 never / 1 always (where the shape allows) / unset: the planner decides
@@ -710,6 +733,7 @@ void init_once() {
     if (const char* v = getenv("BT_GEMM_BK")) g_bk = (atoi(v) == 32) ? 32 : 16;
     if (const char* v = getenv("BT_GEMM_2CTA")) g_two_cta = atoi(v) ? 1 : 0;
     if (const char* v = getenv("BT_GEMM_TAIL")) g_tail_split = atoi(v) ? 1 : 0;
+    if (const char* v = getenv("BT_GEMM_GROUPM")) g_group_m = atoi(v) > 0 ? atoi(v) : 0;
     if (const char* v = getenv("BT_GEMM_F256")) kTwoCtaFactor256 = atof(v);
     if (const char* v = getenv("BT_GEMM_F192")) kTwoCtaFactor192 = atof(v);
     if (const char* v = getenv("BT_GEMM_BN")) {
@@ -745,7 +769,8 @@ constexpr int kMaxUnitsForSplit = 4 * 148;
 // tiles, then the output path exactly as the GEMM's own epilogue runs it: bias, residual, the GELU
 // forward modes (act 1 - 4) and the hi/lo planes.
 __global__ void __launch_bounds__(256) tail_reduce_kernel(const float* __restrict__ partials, int splits, int tail_tiles,
-                                                          int first_tile, int tiles_m, int bn, int M, int N, float* D,
+                                                          int first_tile, int tiles_m, int tiles_n, int group_m, int bn, int M, int N,
+                                                          float* D,
                                                           long long ldd, const float* __restrict__ bias,
                                                           const float* residual, float* d_hi, long long d_plane, int act) {
     pdl_wait();
@@ -756,7 +781,9 @@ __global__ void __launch_bounds__(256) tail_reduce_kernel(const float* __restric
         const int j = (int)(i / per_tile4);
         const long long r = i - (long long)j * per_tile4;
         const int lr = (int)(r / bn4), c4 = (int)(r - (long long)lr * bn4);
-        const int tile = first_tile + j, tm = tile % tiles_m, tn = tile / tiles_m;
+        const int tile = first_tile + j;
+        int tm, tn;
+        raster_tile(tile, tiles_m, tiles_n, group_m, tm, tn);
         const int row = tm * 256 + lr, col = tn * bn + 4 * c4;
         if (row >= M || col >= N) continue;
         float4 t = ld4(partials, (long long)j * per_tile4 + r);
@@ -878,13 +905,31 @@ size_t gemm_tc_partial_floats_bound() { return (size_t)kMaxUnitsForSplit * BM * 
 // What the planner would choose for a product (host arithmetic only; 148 SMs are assumed where no
 // device has been initialised): out = {tile width, 1 if 256-row pair tiles, K splits, tail tiles,
 // K ranges per tail tile, k-blocks per range}.
-void gemm_tc_plan_info(int64_t M, int64_t N, int64_t K, bool can_split, bool can_tail, int two_cta_mode, int out[6]) {
+// Group height of the tile raster.  The `slots` units that run at the same time cover g row tiles by
+// slots / g column tiles (several groups if a group has fewer units), walk K together, and share each A
+// and B tile among them through L2; what the next set of units needs again has by then been pushed out by
+// the operands and outputs streamed in between (an effective 40 MB of the L2 predicts the measured order
+// of the group heights).  With the plain row-fastest order and at least `slots` row tiles, A is fetched
+// from HBM once per tile column; with one row tile per group, B once per tile row.  Measured over the
+// GPT-2 shapes at 8,192 and 32,768 rows: with few tile columns (N = 768 ... 3,072) groups of 4 are
+// best or within 2 % of it (the units that share an A tile then sit on neighbouring CTAs); with many (the
+// LM head: 197) 8 to 32, and 4 re-reads B too often.  Group heights of 1 and 2 were up to 17 % slower
+// than 4 on the K-split LM-head input gradient and are not used.
+int choose_group_m(int tiles_m, int tiles_n, int slots) {
+    int g = g_group_m > 0 ? g_group_m : (4 * tiles_n <= slots ? 4 : 16);
+    return g < tiles_m ? g : tiles_m;
+}
+
+void gemm_tc_plan_info(int64_t M, int64_t N, int64_t K, bool can_split, bool can_tail, int two_cta_mode, int out[7]) {
     const int sms = g_num_sms > 0 ? g_num_sms : 148;
     const int kb_total = (int)((K + g_bk - 1) / g_bk);
     const Plan p = make_plan(M, N, kb_total, g_bk, sms, can_split, gemm_tc_partial_floats_bound(),
                              two_cta_mode >= 0 ? two_cta_mode : g_two_cta, can_tail);
     out[0] = p.bn; out[1] = p.two_cta ? 1 : 0; out[2] = p.splits;
     out[3] = p.tail_tiles; out[4] = p.tail_splits; out[5] = p.tail_kbps;
+    const int tiles_m = p.two_cta ? (int)((M + 2 * BM - 1) / (2 * BM)) : (int)((M + BM - 1) / BM);
+    const int tiles_n = (int)((N + p.bn - 1) / p.bn);
+    out[6] = choose_group_m(tiles_m, tiles_n, p.two_cta ? sms / 2 : sms);
 }
 
 
@@ -919,6 +964,7 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
     g.tiles_n = (int)((N + bn - 1) / bn);
     g.splits = plan.splits;
     g.kb_per_split = plan.kb_per_split; g.kb_total = kb_total;
+    g.group_m = choose_group_m(g.tiles_m, g.tiles_n, plan.two_cta ? sms / 2 : sms);
     g.partials = partials; g.err = err_word;
     g.tail_tiles = plan.tail_tiles; g.tail_splits = plan.tail_splits; g.tail_kbps = plan.tail_kbps;
     g.full_units = g.tiles_m * g.tiles_n - plan.tail_tiles;
@@ -950,7 +996,7 @@ static cudaError_t launch_bk(int layout, int64_t M, int64_t N, int64_t K, const 
             const long long want = (n4 + 255) / 256;
             const int rgrid = (int)(want < 148 * 16 ? want : 148 * 16);
             BT_KERNEL_LAUNCH((tail_reduce_kernel), rgrid, 256, 0, s, (const float*)partials, g.tail_splits, g.tail_tiles,
-                             g.full_units, g.tiles_m, bn, g.M, g.N, D, (long long)ldd, bias, residual, d_hi,
+                             g.full_units, g.tiles_m, g.tiles_n, g.group_m, bn, g.M, g.N, D, (long long)ldd, bias, residual, d_hi,
                              (long long)d_plane, g.act);
             BT_COUNT_LAUNCH();
             return cudaGetLastError();

@@ -428,6 +428,28 @@ def test_gemm_planner_sweep(layout, M, N, K):
         assert rel_l2(host(D), ref) < 1e-4 and rel_max(host(D), ref) < 1e-4, (layout, M, N, K, use_epi, plan)
 
 
+@pytest.mark.parametrize("layout,M,N,K", [(0, 4600, 5120, 264), (1, 4608, 4864, 512), (2, 4640, 5120, 1032),
+                                          (0, 2300, 772, 3080)])
+def test_gemm_tile_raster_groups(layout, M, N, K):
+    """The tiles are walked in groups of row tiles (4, or 16 with many tile columns) with a shorter last
+    group; every tile of the output must come out, whatever the order."""
+    plan = b.bt_op_gemm_plan(M, N, K, False)
+    tiles_m = -(-M // (256 if plan["pair"] else 128))
+    assert 1 < plan["group_m"] < tiles_m and tiles_m % plan["group_m"] != 0, plan
+    a_shape = (K, M) if layout == 2 else (M, K)
+    b_shape = (N, K) if layout == 0 else (K, N)
+    A, Bm = si.normal_f32(184, a_shape), si.normal_f32(185, b_shape, 0.05)
+    A64 = A.astype(np.float64).T if layout == 2 else A.astype(np.float64)
+    B64 = Bm.astype(np.float64).T if layout == 0 else Bm.astype(np.float64)
+    nb = b.bt_op_gemm_scratch_bytes(layout, M, N, K)
+    D = empty(M, N)
+    D.fill_(float("nan"))
+    b.bt_op_gemm(layout, M, N, K, dev(A), dev(Bm), D, None, None, scratch(nb), nb, 0)
+    ref = A64 @ B64
+    assert np.isfinite(host(D)).all()
+    assert rel_l2(host(D), ref) < 1e-4 and rel_max(host(D), ref) < 1e-4, plan
+
+
 def test_gemm_matches_oracle_linear_layer():
     """The three layouts are the forward, input-gradient and weight-gradient of a linear layer."""
     N, cin, cout = 640, 768, 1024

@@ -96,6 +96,13 @@ def test_gemm_planner_choices(lib):
     assert p["pair"] == 0 and p["tail_splits"] == 0
     p = b.bt_op_gemm_plan(768, 768, 8192, False)          # a weight gradient: few tiles, K split over all of them
     assert p["splits"] > 1 and p["tail_splits"] == 0
+    # raster of the tiles: groups of 4 row tiles where a group's units fit among those in flight (few tile
+    # columns), 16 with many tile columns (the LM head), never more than there are row tiles
+    assert b.bt_op_gemm_plan(8192, 768, 3072, True)["group_m"] == 4
+    assert b.bt_op_gemm_plan(8192, 2304, 768, True)["group_m"] == 4
+    assert b.bt_op_gemm_plan(8192, 50304, 768, False)["group_m"] == 16
+    assert b.bt_op_gemm_plan(50304, 768, 8192, False)["group_m"] == 4
+    assert b.bt_op_gemm_plan(512, 50304, 768, False)["group_m"] == 2
     with pytest.raises(b.BtError):
         b.bt_op_gemm_plan(0, 768, 768)
 
