@@ -15,6 +15,29 @@ cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, cons
                                     const float* o, const float* o_lo, const float* lse, float* dvec, int B, int T,
                                     int C, int H, float* dqkv_hi, int64_t dqkv_plane, float* rg_sums, int* err_word,
                                     cudaStream_t s);
+// Heads per group in the CTA order of the head_dim-64 tensor-core kernels: the smallest divisor of the
+// head count whose groups hold at least one and a half times as many CTAs as there are SMs (equal groups:
+// a short last group starts its long walks last and becomes the tail).  Measured: 16 - 32 heads at 8
+// blocks per head (forward -6 %, backward -1 to -2 %), 2 heads at 128 blocks (-6 % / -3 %), no gain at
+// 32 blocks, and groups smaller than the machine lose up to 13 % in the backward kernels.
+// BT_ATTN_HEAD_GROUP=n pins it (tuning aid).
+int attn_head_group(int heads, int blocks) {
+    static const int forced = []() {
+        const char* v = getenv("BT_ATTN_HEAD_GROUP");
+        return v ? atoi(v) : 0;
+    }();
+    if (forced > 0) return forced < heads ? forced : heads;
+    static const int sms = []() {
+        int dev = 0, n = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0) n = 148;
+        return n;
+    }();
+    if (blocks < 1) blocks = 1;
+    for (int g = 1; g < heads; ++g)
+        if (heads % g == 0 && 2 * g * blocks >= 3 * sms) return g;
+    return heads;
+}
+
 bool attention_mma_supports(int head_dim);
 cudaError_t launch_attention_fwd_mma(const float* qkv, int B, int T, int C, int H, float* o, float* o_hi,
                                      float* o_lo, float* lse, cudaStream_t s);

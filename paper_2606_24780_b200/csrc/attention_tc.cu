@@ -57,6 +57,7 @@ constexpr float kLn2 = 0.6931471805599453f;
 
 struct AttnArgs {
     int T, C, H;
+    int head_group;   // heads per group of the CTA order (grouped_block)
     float* o;
     float* o_hi;
     float* o_lo;
@@ -97,8 +98,10 @@ attn_fwd_tc_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constan
         reinterpret_cast<volatile uint32_t*>(smem_raw + (tmem_slot - smem_u32(smem_raw)));
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int qt = gridDim.y - 1 - blockIdx.y;           // heaviest query tiles first, over all heads
-    const int b = blockIdx.x / g.H, h = blockIdx.x % g.H;
+    int bh, yb;
+    grouped_block(g.head_group, bh, yb);
+    const int qt = gridDim.y - 1 - yb;                   // heaviest query tiles first, over the heads of a group
+    const int b = bh / g.H, h = bh % g.H;
     const int q0 = qt * BQ;
     const int last_row = min(q0 + BQ - 1, g.T - 1);
     const int n_kt = last_row / BKV + 1;
@@ -404,7 +407,7 @@ cudaError_t launch_attention_fwd_tc(const float* qkv_hi, int64_t qkv_plane, int 
               encode3(&tmK, qkv_hi, cols, rows, cols, qkv_plane, 32, BKV, CU_TENSOR_MAP_SWIZZLE_128B) &&
               encode3(&tmV, qkv_hi, cols, rows, cols, qkv_plane, 32, BKV, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B);
     if (!ok) return cudaErrorInvalidValue;
-    AttnArgs g{T, C, H, o, o_hi, o_lo, lse, err_word, g_trace_ptr};
+    AttnArgs g{T, C, H, attn_head_group(B * H, (T + BQ - 1) / BQ), o, o_hi, o_lo, lse, err_word, g_trace_ptr};
     dim3 grid(B * H, (T + BQ - 1) / BQ);
     BT_KERNEL_LAUNCH((attn_fwd_tc_kernel), grid, kThreads, kSmemBytes, s, tmQ, tmK, tmV, g);
     BT_COUNT_LAUNCH();

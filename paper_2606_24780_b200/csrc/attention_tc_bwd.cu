@@ -156,6 +156,7 @@ __device__ __forceinline__ float warp_rows_dot64(const float* a_hi, const float*
 
 struct BwdArgs {
     int T, C, H;
+    int head_group;           // heads per group of the CTA order (grouped_block)
     const float* qkv_hi;      // split qkv [2][B*T][3C]
     long long qkv_plane;
     const float* lse;
@@ -243,8 +244,10 @@ attn_bwd_dkv_tc_kernel(const __grid_constant__ CUtensorMap tmQk, const __grid_co
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     // grid = (sequence x head, key block): blocks are dispatched x-fastest, so all the key blocks
     // with the longest walks (low j0) start first and the short ones fill the tail
-    const int b = blockIdx.x / g.H, h = blockIdx.x % g.H;
-    const int j0 = blockIdx.y * BR;
+    int bh, yb;
+    grouped_block(g.head_group, bh, yb);
+    const int b = bh / g.H, h = bh % g.H;
+    const int j0 = yb * BR;
     const int row_base = b * g.T;
     const int n_qt = (g.T + BT64 - 1) / BT64, qt0 = j0 / BT64;
     const int n_t = n_qt - qt0;
@@ -572,8 +575,10 @@ attn_bwd_dq_tc_kernel(const __grid_constant__ CUtensorMap tmKk, const __grid_con
     const uint32_t tmem_slot = bars + 8u * 15;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int qt = gridDim.y - 1 - blockIdx.y;                  // heaviest query tiles first, over all heads
-    const int b = blockIdx.x / g.H, h = blockIdx.x % g.H;
+    int bh, yb;
+    grouped_block(g.head_group, bh, yb);
+    const int qt = gridDim.y - 1 - yb;                          // heaviest query tiles first, over the heads of a group
+    const int b = bh / g.H, h = bh % g.H;
     const int q0 = qt * BR;
     const int row_base = b * g.T;
     const int n_t = min(q0 + BR - 1, g.T - 1) / BKT + 1;         // key tiles up to the diagonal
@@ -842,7 +847,7 @@ cudaError_t launch_attention_bwd_tc(const float* qkv_hi, int64_t qkv_plane, cons
     ok = ok && enc3(&qk64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, false) &&  // 64-row K-major / MN-major tiles of qkv
          enc3(&qm64, qkv_hi, 3 * (int64_t)C, rows, qkv_plane, BKT, true);
     if (!ok) return cudaErrorInvalidValue;
-    BwdArgs g{T, C, H, qkv_hi, qkv_plane, lse, dvec, dvec, o, o_lo, do_hi, do_plane, dqkv_hi, dqkv_plane, err_word,
+    BwdArgs g{T, C, H, attn_head_group(B * H, (T + BR - 1) / BR), qkv_hi, qkv_plane, lse, dvec, dvec, o, o_lo, do_hi, do_plane, dqkv_hi, dqkv_plane, err_word,
               attention_tc_get_trace(), rg_sums, 4 * ((T + BR - 1) / BR)};
     dim3 gk(B * H, (T + BR - 1) / BR);
     // the dq kernel goes first: it also forms D = rowsum(dO o O), which the dkv kernel reads

@@ -328,6 +328,20 @@ __device__ __forceinline__ void rows_to_tmem(const float* src_hi, const float* s
 // A cluster of two CTAs on neighbouring SMs issues one MMA of M = 256: each CTA supplies its own
 // 128 rows of A and HALF of the B tile from its own shared memory and holds its own 128 rows of
 // the accumulator in its own tensor memory.  Only the even CTA (the leader) issues.
+// Work item of a CTA in a (sequence x head, block) grid whose CTAs start in the order of their linear
+// index (x fastest).  The heads are taken in groups of `head_group`: inside a group the heads run fastest,
+// then the blocks, then the next group, so that the CTAs in flight at one time belong to few heads and
+// share those heads' operand tiles through L2.  head_group <= 0 or >= gridDim.x: one group.
+__device__ __forceinline__ void grouped_block(int head_group, int& bh, int& y) {
+    const int nh = (int)gridDim.x, ny = (int)gridDim.y;
+    const int G = (head_group > 0 && head_group < nh) ? head_group : nh;
+    const int id = (int)blockIdx.y * nh + (int)blockIdx.x;
+    const int per = G * ny, grp = id / per, rem = id - grp * per;
+    const int first = grp * G, heads = min(G, nh - first);
+    y = rem / heads;
+    bh = first + (rem - y * heads);
+}
+
 __device__ __forceinline__ uint32_t cluster_ctarank() {
     uint32_t r;
     asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
