@@ -490,6 +490,7 @@ def test_attention_fwd_bwd(B, T, H, d, flags):
 
 TC_ATTN_SHAPES = [(2, 200, 3, 64), (1, 1024, 2, 64), (1, 1, 2, 64), (3, 129, 1, 64), (1, 130, 12, 64), (2, 64, 1, 64),
                   (1, 65, 1, 64), (1, 33, 1, 64),
+                  (28, 200, 8, 64),   # 224 heads x 2 blocks: the CTA order in two groups of 112 heads
                   (2, 200, 2, 128), (1, 1024, 1, 128), (1, 1, 2, 128), (2, 129, 1, 128), (1, 130, 3, 128),
                   (2, 64, 1, 128), (1, 33, 1, 128), (1, 300, 2, 128)]
 
