@@ -296,6 +296,10 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->attn_rg = b.take<float>(attention_bwd_rowgroups(m->maxB, m->T) * 3 * m->C);
     section(5);                      // backward temporaries (reused by every layer)
     m->partial_floats = gemm_tc_partial_floats_bound();
+    // the LM head's input gradient sums over the padded vocabulary: room for the K ranges that keep its
+    // accumulation chains within the planner's cap at any token count
+    if (!simt_gemm && gemm_tc_partial_floats_for_chain_cap(N, C, m->Vp) > m->partial_floats)
+        m->partial_floats = gemm_tc_partial_floats_for_chain_cap(N, C, m->Vp);
     m->partials = b.take<float>(m->partial_floats);
     m->ln_scratch = b.take<float>(layernorm_bwd_scratch_floats(N, (int)C));
     size_t cs = colsum_scratch_floats(N, (int)F);

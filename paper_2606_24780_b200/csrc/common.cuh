@@ -271,6 +271,7 @@ cudaError_t launch_gemm_tc(int layout, int64_t M, int64_t N, int64_t K, SplitMat
 // two_cta_mode: -1 the planner chooses between 128-row tiles on single CTAs and 256-row tiles on
 // CTA pairs (cta_group::2); 0 / 1 force the one or the other (1 applies where M >= 256).
 size_t gemm_tc_partial_floats_bound();
+size_t gemm_tc_partial_floats_for_chain_cap(int64_t M, int64_t N, int64_t K);
 // Heads per group in the CTA order of the head_dim-64 tensor-core attention kernels, for a grid of
 // `heads` (sequence x head) by `blocks` (query or key blocks) CTAs.
 int attn_head_group(int heads, int blocks);

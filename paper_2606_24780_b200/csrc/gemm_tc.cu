@@ -902,6 +902,15 @@ bool gemm_tc_init(char* err, size_t errlen) {
 
 size_t gemm_tc_partial_floats_bound() { return (size_t)kMaxUnitsForSplit * BM * 256; }
 
+// Partial-sum floats a product needs so that the planner can keep every accumulation chain within its
+// cap (8192 MMAs) by cutting K: 0 where the whole K fits in one chain.
+size_t gemm_tc_partial_floats_for_chain_cap(int64_t M, int64_t N, int64_t K) {
+    const int bk = g_bk > 0 ? g_bk : 16;
+    const int64_t kb_total = (K + bk - 1) / bk, max_chain_kb = 8192 / (3 * (bk / 8));
+    const int64_t splits = (kb_total + max_chain_kb - 1) / max_chain_kb;
+    return splits > 1 ? (size_t)splits * (size_t)M * (size_t)N : 0;
+}
+
 // What the planner would choose for a product (host arithmetic only; 148 SMs are assumed where no
 // device has been initialised): out = {tile width, 1 if 256-row pair tiles, K splits, tail tiles,
 // K ranges per tail tile, k-blocks per range}.
