@@ -298,8 +298,13 @@ size_t layout(bt_model* m, uint8_t* base) {
     m->partial_floats = gemm_tc_partial_floats_bound();
     // the LM head's input gradient sums over the padded vocabulary: room for the K ranges that keep its
     // accumulation chains within the planner's cap at any token count
-    if (!simt_gemm && gemm_tc_partial_floats_for_chain_cap(N, C, m->Vp) > m->partial_floats)
-        m->partial_floats = gemm_tc_partial_floats_for_chain_cap(N, C, m->Vp);
+    // (and for its weight gradient, which sums over the tokens)
+    if (!simt_gemm) {
+        const size_t need_dx = gemm_tc_partial_floats_for_chain_cap(N, C, m->Vp);
+        const size_t need_dw = gemm_tc_partial_floats_for_chain_cap(m->Vp, C, N);
+        if (need_dx > m->partial_floats) m->partial_floats = need_dx;
+        if (need_dw > m->partial_floats) m->partial_floats = need_dw;
+    }
     m->partials = b.take<float>(m->partial_floats);
     m->ln_scratch = b.take<float>(layernorm_bwd_scratch_floats(N, (int)C));
     size_t cs = colsum_scratch_floats(N, (int)F);
