@@ -467,7 +467,10 @@ BT_API bt_status bt_op_gemm_check(const void* scratch, void* stream);
  * cuts only the tiles of the last, partly filled round along K and adds a small reduction pass.  The
  * raster walks groups of `group height` row tiles, inside a group row tiles fastest, then column tiles:
  * the tiles in flight at one time share their A and B tiles through L2, and the height is chosen so that
- * an operand larger than L2 is not fetched from HBM once per tile column (or row). */
+ * an operand larger than L2 is not fetched from HBM once per tile column (or row).  The answer is the
+ * one for the per-op calls, whose partial-sum buffer has a fixed size; a model sizes its own buffer so
+ * that the LM head's two backward products can always be cut along K, and may therefore split where
+ * this call reports none. */
 BT_API bt_status bt_op_gemm_plan(int64_t M, int64_t N, int64_t K, int32_t epilogue, uint32_t flags, int32_t* out7);
 /* The input-gradient product of the MLP down-projection with the GELU backward in its epilogue
  * (Kernel Design, fused element-wise epilogues; Appendix B "GELU Backward"): with dy_split
